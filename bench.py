@@ -1,0 +1,378 @@
+#!/usr/bin/env python
+"""Benchmark of the R-TOSS hot path on B200.
+
+A step is one pass of the whole hot path over one batch of synthetic input:
+pattern selection (Algorithm 2 / 3 of arXiv 2303.02191), packing, and the
+pattern-sparse convolution, for each layer of the workload.  Default workload
+"layer128": batch 8, bf16 --
+  3x3 128->128 @80x80 with 3-entry patterns, the same layer with 2-entry
+  patterns, and a 1x1 256->128 @80x80 whose weights are regrouped into 3x3
+  blocks and pruned with the 3-entry patterns.
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2303_02191_b200 import synth  # noqa: E402
+
+# nominal FP32 FMA peak: 148 SMs x 128 lanes x 2 FLOP x 1.965 GHz (maximum SM clock)
+ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+def workload_layers(name):
+    """-> (batch N, dtype, list of (layer dict, k, preset name))."""
+    if name == "layer128":
+        l3 = dict(name="conv3x3_128", ksize=3, stride=1, cin=128, cout=128, H=80, W=80, act="silu", wid=0)
+        l1 = dict(name="conv1x1_256_128", ksize=1, stride=1, cin=256, cout=128, H=80, W=80, act="silu", wid=2)
+        return 8, "bf16", [(l3, 3, "conn4"), (dict(l3, wid=1), 2, "conn4"), (l1, 3, "conn4")]
+    if name == "layer32":
+        l3 = dict(name="conv3x3_32", ksize=3, stride=1, cin=32, cout=32, H=32, W=32, act="none", wid=0)
+        return 1, "f32", [(l3, 4, "centre8")]
+    if name in ("yolov5s_b1", "yolov5s_b16"):
+        return (1 if name.endswith("b1") else 16), "bf16", [(L, 4, "centre8") for L in synth.yolov5s_stack()]
+    if name == "retinanet_b4":
+        return 4, "bf16", [(L, 4, "centre8") for L in synth.retinanet_r50fpn_stack()]
+    raise SystemExit("unknown workload " + name)
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index = index
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40,
+                 "hw_power_brake": 0x80}
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# --------------------------------------------------------------------------- CPU oracle legs
+
+def oracle_step(layers_k, dtype, n_sample, frac=1.0, seed=0):
+    """One pass of the hot path in the CPU oracle on n_sample images.  With frac < 1 each convolution
+    computes only the first ceil(frac*Cout) output channels (selection and packing always see the whole
+    layer).  Returns (seconds, fraction of the full per-image multiply-adds that was computed)."""
+    from oracle import rtoss_oracle as orc
+    odt = {"f32": orc.DT_F32, "bf16": orc.DT_BF16, "f16": orc.DT_F16}[dtype]
+    act = {"none": orc.ACT_NONE, "relu": orc.ACT_RELU, "silu": orc.ACT_SILU}
+    prepared, done, full = [], 0.0, 0.0
+    for (L, k, preset) in layers_k:
+        masks = orc.pattern_preset(k, orc.PRESET_CENTRE8 if preset == "centre8" else orc.PRESET_CONN4)
+        x = synth.round_like(synth.activations(seed, L["wid"], n_sample, L["cin"], L["H"], L["W"]), dtype)
+        w = synth.kaiming_weights(seed, L["wid"], L["cout"], L["cin"], L["ksize"])
+        b = synth.bias(seed, L["wid"], L["cout"])
+        cs = max(1, min(L["cout"], int(np.ceil(frac * L["cout"]))))
+        fl = synth.layer_nnz_flops(L, 1, k)
+        full += fl
+        done += fl * cs / L["cout"]
+        prepared.append((L, k, masks, x, w, b, cs))
+    t0 = time.perf_counter()
+    for (L, k, masks, x, w, b, cs) in prepared:
+        if L["ksize"] == 3:
+            pid = orc.select_3x3(w, masks)
+            val, _, _ = orc.pack_3x3(w, masks, k, pid, odt)
+            wd = orc.unpack_3x3(val, L["cout"], L["cin"], masks, k, pid)
+            orc.conv3x3(x, wd[:cs], b[:cs], L["stride"], act[L["act"]], odt)
+        else:
+            w2 = w.reshape(L["cout"], L["cin"])
+            pid = orc.select_1x1(w2, masks)
+            val = orc.pack_1x1(w2, masks, k, pid, odt)
+            wd = orc.unpack_1x1(val, L["cout"], L["cin"], masks, k, pid)
+            orc.conv1x1(x, wd[:cs], b[:cs], L["stride"], act[L["act"]], odt)
+    return time.perf_counter() - t0, done / full
+
+
+def cpu_baseline_sample(layers_k, dtype, N, budget_s):
+    """Time the oracle on a bounded sample: one image, a fraction of the output channels sized from a
+    small calibration pass so that the timed pass takes about budget_s."""
+    t_cal, f_cal = oracle_step(layers_k, dtype, 1, 1.0 / 16)
+    t_image = t_cal / f_cal
+    frac = min(1.0, max(1.0 / 64, budget_s / max(t_image, 1e-6)))
+    n = min(N, max(1, int(budget_s / t_image))) if frac >= 1.0 else 1
+    t, f = oracle_step(layers_k, dtype, n, frac)
+    return n * f / t, t, f, n
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    N, dtype, layers_k = workload_layers(args.workload)
+    # size the per-step sample so that warmup + steps stay within about two minutes
+    t_cal, f_cal = oracle_step(layers_k, dtype, 1, 1.0 / 16)
+    per_step = 120.0 / max(1, args.steps + args.warmup)
+    frac = min(1.0, max(1.0 / 64, f_cal * per_step / max(t_cal, 1e-6)))
+    for _ in range(max(args.warmup, 0)):
+        oracle_step(layers_k, dtype, 1, frac)
+    res = [oracle_step(layers_k, dtype, 1, frac) for _ in range(args.steps)]
+    t = float(np.mean([r[0] for r in res]))
+    f = res[0][1]
+    value = f / t
+    cores = os.cpu_count()
+    sample = ("per step: 1 image of the batch of %d, the first %.3f of every layer's output channels, "
+              "whole-layer select and pack; images/s = fraction / seconds") % (N, f)
+    print(json.dumps({
+        "impl": "reference", "metric": "pattern-sparse conv images/sec", "value": value, "unit": "images/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
+        "config": {"workload": args.workload, "batch": N},
+        "cpu_baseline": {"value": value, "unit": "images/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# --------------------------------------------------------------------------- GPU arm
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2303_02191_b200 import binding as rt
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+    ctx = rt.Context(local_rank)
+    tdt = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}
+
+    N, dtype, layers_k = workload_layers(args.workload)
+    elem = 4 if dtype == "f32" else 2
+    cdt = rt.DTYPE_NAMES[dtype]
+    preset_of = {"centre8": rt.PRESET_CENTRE8, "conn4": rt.PRESET_CONN4}
+
+    # ---- resident inputs (replicas: every rank holds its own batch and weights; no data-path collective)
+    weights, L_state = {}, []
+    for (L, k, preset) in layers_k:
+        masks = rt.rtoss_pattern_preset(k, preset_of[preset])
+        if L["wid"] not in weights:
+            w = torch.from_numpy(synth.kaiming_weights(rank, L["wid"], L["cout"], L["cin"], L["ksize"])).to(dev)
+            b = torch.from_numpy(synth.bias(rank, L["wid"], L["cout"])).to(dev)
+            n_k = L["cout"] * L["cin"] if L["ksize"] == 3 else (L["cout"] * L["cin"]) // 9
+            pid = torch.empty(max(n_k, 1), dtype=torch.uint8, device=dev)
+            weights[L["wid"]] = dict(w=w, b=b, pid=pid, packed=None, masks=masks, k=k, ksize=L["ksize"])
+        Ho, Wo = synth.out_hw(L["H"], L["W"], L["stride"])
+        xh = torch.from_numpy(synth.activations(rank, len(L_state), N, L["cin"], L["H"], L["W"])).to(tdt[dtype])
+        st = dict(L=L, k=k, x=xh.to(dev), y=torch.empty(N, L["cout"], Ho, Wo, dtype=tdt[dtype], device=dev),
+                  xh=xh.pin_memory(), yh=torch.empty(N, L["cout"], Ho, Wo, dtype=tdt[dtype]).pin_memory(),
+                  Ho=Ho, Wo=Wo, wt=weights[L["wid"]])
+        L_state.append(st)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)   # larger than the 126 MB L2
+
+    def prune_weights():
+        launches = 0
+        for wt in weights.values():
+            ctx.rtoss_select_patterns(wt["w"], wt["ksize"], wt["masks"], wt["k"], pid=wt["pid"])
+            wt["packed"] = ctx.rtoss_pack(wt["w"], wt["ksize"], wt["masks"], wt["k"], wt["pid"], cdt, into=wt["packed"])
+            launches += 3 if wt["ksize"] == 3 else 2
+        return launches
+
+    def conv(st, ev=None):
+        L = st["L"]
+        fn = ctx.rtoss_conv3x3_pattern if L["ksize"] == 3 else ctx.rtoss_conv1x1_pattern
+        if ev:
+            ev[0].record()
+        fn(st["wt"]["packed"], st["x"], st["y"], N, L["H"], L["W"], L["stride"], rt.NCHW, rt.ACT_NAMES[L["act"]], st["wt"]["b"])
+        if ev:
+            ev[1].record()
+
+    def step(evs=None):
+        n = prune_weights()
+        for i, st in enumerate(L_state):
+            conv(st, evs[i] if evs else None)
+        return n + len(L_state)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+        flush.zero_()
+    barrier()
+
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler.start()
+    step_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    conv_ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in L_state]
+               for _ in range(args.steps)]
+    launches = 0
+    barrier()
+    for s in range(args.steps):
+        flush.zero_()                       # L2 flush between timed iterations, outside the step's events
+        step_ev[s][0].record()
+        launches += step(conv_ev[s])
+        step_ev[s][1].record()
+    barrier()
+    clocks = sampler.stop()
+    step_ms = np.array([a.elapsed_time(b) for a, b in step_ev])
+    total_ms = float(step_ms.sum())
+    conv_ms = np.array([[a.elapsed_time(b) for a, b in row] for row in conv_ev]).mean(axis=0)
+
+    # ---- end to end through the host-buffer entry point (pinned host tensors, copies inside the timed region)
+    torch.cuda.synchronize()
+    e2e_steps = max(3, min(args.steps, 20))
+    for st in L_state[:1]:
+        ctx.rtoss_conv_pattern_host(st["wt"]["packed"], st["xh"], st["yh"], N, st["L"]["H"], st["L"]["W"], st["L"]["stride"],
+                                    rt.NCHW, rt.ACT_NAMES[st["L"]["act"]], st["wt"]["b"])
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        prune_weights()
+        torch.cuda.synchronize()
+        for st in L_state:
+            L = st["L"]
+            ctx.rtoss_conv_pattern_host(st["wt"]["packed"], st["xh"], st["yh"], N, L["H"], L["W"], L["stride"], rt.NCHW,
+                                        rt.ACT_NAMES[L["act"]], st["wt"]["b"])
+    torch.cuda.synchronize()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    h2d = sum(st["xh"].numel() * elem for st in L_state)
+    d2h = sum(st["yh"].numel() * elem for st in L_state)
+
+    if world > 1:
+        t = torch.tensor([total_ms, e2e_s], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_s = float(t[0]), float(t[1])
+
+    if rank == 0:
+        ms_per_step = total_ms / args.steps
+        value = world * N / (ms_per_step * 1e-3)
+        flops = [synth.layer_nnz_flops(st["L"], N, st["k"]) for st in L_state]
+        bytes_ = [synth.layer_bytes(st["L"], N, st["k"], elem) for st in L_state]
+        top = int(np.argmax(conv_ms))
+        hbm_peak, peak_kind = read_peaks()
+        t_top = conv_ms[top] * 1e-3
+        alu_t, hbm_t = flops[top] / (ALU_PEAK_TFLOPS * 1e12), bytes_[top] / (hbm_peak * 1e9)
+        if alu_t >= hbm_t:
+            roof = {"bound": "alu", "achieved": flops[top] / t_top / 1e12, "peak": ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
+                    "peak_kind": "derived: 148 SM x 128 FMA lanes x 2 x 1.965 GHz"}
+        else:
+            roof = {"bound": "hbm", "achieved": bytes_[top] / t_top / 1e9, "peak": hbm_peak, "unit": "GB/s",
+                    "peak_kind": "of " + peak_kind}
+        roof["frac"] = roof["achieved"] / roof["peak"]
+        roof["traffic"] = None
+        roof["kernel"] = L_state[top]["L"]["name"] + " k=%d" % L_state[top]["k"]
+        roof["kernel_ms"] = float(conv_ms[top])
+        roof["nnz_flop_per_launch"] = flops[top]
+        roof["algorithmic_bytes_per_launch"] = bytes_[top]
+        out = {
+            "metric": "pattern-sparse conv images/sec", "value": value, "unit": "images/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
+            "config": {"workload": args.workload, "batch": N, "layout": "NCHW", "l2": "flushed between steps (256 MB write)",
+                       "layers": len(L_state), "multi_gpu": "replicas only"},
+            "nnz_gflops_per_s": sum(flops) / (ms_per_step * 1e-3) / 1e9 * world,
+            "conv_ms": [float(v) for v in conv_ms] if len(conv_ms) <= 8 else None,
+            "conv_ms_sum": float(conv_ms.sum()),
+            "roofline": roof, "clocks": clocks,
+            "e2e": {"value": world * N / e2e_s, "unit": "images/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": launches,
+        }
+        if args.cpu_baseline:
+            v_cpu, t_cpu, f_cpu, n_cpu = cpu_baseline_sample(layers_k, dtype, N, 15.0)
+            out["cpu_baseline"] = {"value": v_cpu, "unit": "images/s", "cores": os.cpu_count(), "kind": "oracle",
+                                   "sample": "%d image(s) of the batch of %d, the first %.3f of every layer's output channels, "
+                                             "one pass of %.1f s; images/s = images x fraction / seconds" % (n_cpu, N, f_cpu, t_cpu)}
+        print(json.dumps(out))
+    for wt in weights.values():
+        if wt["packed"] is not None:
+            wt["packed"].close()
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="layer128")
+    ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1 or args.gpus == 1:
+        if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+            args.cpu_baseline = False
+        run_gpu(args)
+    else:
+        raise SystemExit("for --gpus N > 1 launch with: python -m torch.distributed.run --nproc-per-node N bench.py --gpus N")
+
+
+if __name__ == "__main__":
+    main()

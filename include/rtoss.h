@@ -1,0 +1,206 @@
+/*
+ * librtoss -- R-TOSS hot path on NVIDIA B200 (sm_100a), C ABI.
+ *
+ * R-TOSS (arXiv 2303.02191) prunes every 3x3 convolution kernel to the k taps
+ * of one pattern out of a small pattern table, choosing per kernel the pattern
+ * that retains the largest L2 norm (Section IV.C, Algorithm 2); 1x1 weights
+ * are first regrouped, nine at a time, into temporary 3x3 matrices and pruned
+ * with the same patterns (Section IV.D, Algorithm 3).  This library performs
+ * that selection on the GPU, packs the surviving weights, and runs inference
+ * convolution directly on the packed form.
+ *
+ * Conventions
+ *   - Tap numbering inside a 3x3 kernel: t = 3*row + col.  A pattern is a
+ *     9-bit mask, bit t set = tap t kept; every mask of a table has exactly k
+ *     bits.  A pattern id ("pid") is an index into the table.
+ *   - Pointers named *_dev are device pointers on the context's device,
+ *     *_host are host pointers.  The caller owns every buffer it passes.
+ *     Device pointers of tensors must be 16-byte aligned.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls only enqueue work on it and never synchronise, unless stated.
+ *   - Every call returns an rtoss_status; argument errors are detected on the
+ *     host before anything is launched.  Nothing throws or aborts.
+ *   - There is no CPU fallback: without a CUDA device rtoss_create fails.
+ */
+#ifndef RTOSS_H
+#define RTOSS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    RTOSS_OK = 0,
+    RTOSS_ERR_INVALID_ARG = 1,       /* null pointer, non-positive size, bad enum */
+    RTOSS_ERR_BAD_PATTERN_TABLE = 2, /* mask outside 1..511, popcount != k, duplicate, P outside 1..255 */
+    RTOSS_ERR_UNSUPPORTED = 3,       /* valid request the library has no kernel for */
+    RTOSS_ERR_ALIGNMENT = 4,         /* a tensor pointer is not 16-byte aligned */
+    RTOSS_ERR_ALLOC = 5,             /* device or host allocation failed */
+    RTOSS_ERR_CUDA = 6,              /* a CUDA runtime call failed; see rtoss_last_error */
+    RTOSS_ERR_TIMEOUT = 7            /* a bounded device-side wait gave up */
+} rtoss_status;
+
+typedef enum { RTOSS_F32 = 0, RTOSS_BF16 = 1, RTOSS_F16 = 2 } rtoss_dtype;
+typedef enum { RTOSS_NCHW = 0, RTOSS_NHWC = 1 } rtoss_layout;
+typedef enum { RTOSS_ACT_NONE = 0, RTOSS_ACT_RELU = 1, RTOSS_ACT_SILU = 2 } rtoss_act;
+typedef enum {
+    RTOSS_PRESET_ALL = 0,     /* every k-subset of the 9 taps (Eq. 1) */
+    RTOSS_PRESET_CONN4 = 1,   /* k-subsets forming one edge-connected set (Section IV.B, criterion 1) */
+    RTOSS_PRESET_CENTRE8 = 2, /* k = 4: the four 2x2 blocks through the centre + the four T shapes */
+    RTOSS_PRESET_DENSE = 3    /* k = 9: the single all-taps mask (no pruning) */
+} rtoss_preset;
+
+typedef struct rtoss_ctx rtoss_ctx;       /* per-device state: error text, host-path workspace */
+typedef struct rtoss_packed rtoss_packed; /* one layer's pruned weights in packed form, on the device */
+
+/* Create / destroy a context on CUDA device `device`.  rtoss_create fails with
+ * RTOSS_ERR_CUDA when the device cannot be used.  rtoss_destroy frees the
+ * context's workspace; packed handles are freed separately. */
+rtoss_status rtoss_create(int device, rtoss_ctx** ctx);
+void rtoss_destroy(rtoss_ctx* ctx);
+const char* rtoss_status_string(rtoss_status s);
+/* Text of the last error recorded on this context ("" if none).  Valid until
+ * the next failing call on the same context. */
+const char* rtoss_last_error(const rtoss_ctx* ctx);
+
+/* ---- host-only steps (no GPU needed) ------------------------------------- */
+
+/* Pattern table presets (Section IV.B: Eq. 1 enumerates all C(9,k) masks;
+ * criterion 1 drops those whose kept taps are not adjacent).  Writes the masks
+ * in ascending numeric order into masks_host.  *P is the capacity on entry and
+ * the count on return.  RTOSS_ERR_INVALID_ARG for a bad k/preset pairing or
+ * too small a capacity. */
+rtoss_status rtoss_pattern_preset(int k, rtoss_preset preset, uint16_t* masks_host, int* P);
+
+/* Check a caller-supplied table: 1 <= P <= 255, 1 <= k <= 9, every mask in
+ * 1..511 with exactly k bits, no duplicates.  RTOSS_OK or
+ * RTOSS_ERR_BAD_PATTERN_TABLE. */
+rtoss_status rtoss_pattern_table_validate(const uint16_t* masks_host, int P, int k);
+
+/* One node of the model graph for the layer grouping.  Nodes are listed in
+ * topological order; `inputs` holds the ids of the producing nodes. */
+typedef struct {
+    int is_conv;       /* 1 = convolution layer, 0 = any other operation */
+    int cout, cin;     /* convolution shape (ignored for other nodes) */
+    int ksize;         /* 1 or 3 (ignored for other nodes) */
+    int n_inputs;
+    const int* inputs; /* n_inputs node ids, each < this node's id */
+} rtoss_layer_node;
+
+/* Layer grouping by depth-first search (Section IV.A, Algorithm 1).  For each
+ * convolution the search walks backwards from its inputs, in listed order and
+ * through non-convolution nodes, and the first convolution reached is its
+ * parent (one parent per child).  A convolution with none upstream is its own
+ * parent and founds a group.  A child joins its parent's group when it has the
+ * parent's kernel size and (cout, cin) -- then it may reuse the parent's
+ * pattern ids kernel by kernel -- otherwise it founds a new group.
+ * parent[i] = group[i] = -1 for non-convolution nodes.  *n_groups (nullable)
+ * receives the group count.  RTOSS_ERR_INVALID_ARG on a malformed graph. */
+rtoss_status rtoss_group_layers(const rtoss_layer_node* nodes, int L, int* parent, int* group, int* n_groups);
+
+/* ---- selection (Algorithm 2; Algorithm 3 for ksize = 1) -------------------- */
+
+/* For every kernel, the id of the pattern that retains the largest sum of
+ * squared weights (equivalently the largest L2 norm).  The arithmetic is
+ * fixed so that ids are reproducible bit for bit: squares rounded to fp32,
+ * summed in fp32 over the pattern's taps in ascending order, first strictly
+ * larger sum wins (ties -> lowest id; a NaN sum never wins).
+ *   ksize = 3: w_dev is [Cout][Cin][3][3] contiguous; pid_dev gets Cout*Cin
+ *              bytes, pid_dev[co*Cin+ci].
+ *   ksize = 1: w_dev is [Cout][Cin]; the flat list is cut into G =
+ *              floor(Cout*Cin/9) runs of nine, run g viewed as a row-major
+ *              3x3; pid_dev gets G bytes.  The Cout*Cin - 9G trailing weights
+ *              are pruned by the later steps.
+ * w_dtype may be fp32, bf16 or fp16 (widened exactly).  masks_host is
+ * validated (RTOSS_ERR_BAD_PATTERN_TABLE). */
+rtoss_status rtoss_select_patterns(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, int Cout, int Cin,
+                                   int ksize, const uint16_t* masks_host, int P, int k, uint8_t* pid_dev,
+                                   void* cuda_stream);
+
+/* ---- packing (Section IV.C: "kernels with similar patterns are grouped") --- */
+
+/* Build the packed form of one layer from its weights and pattern ids:
+ *   val  [n_kernels*k]  kept weights, ascending tap order inside a kernel,
+ *                       rounded (nearest even) to compute_dtype;
+ *   pid  [n_kernels]    copy of the ids;
+ *   ksize 3 only: for each input channel ci a stable counting sort of the
+ *   filters by pattern id: perm[ci*Cout+i] = filter at position i,
+ *   bucket_off[ci*(P+1)+p] = first position of pattern p (entry P = Cout).
+ * n_kernels = Cout*Cin (ksize 3) or floor(Cout*Cin/9) (ksize 1).
+ * *out must be NULL or an existing handle.  NULL: a new handle is created and
+ * its device memory allocated (RTOSS_ERR_ALLOC on failure).  Existing handle
+ * of the same layer shape, P, k and dtype: it is re-packed in place without
+ * any allocation (the paper re-selects patterns in every pruning iteration);
+ * a handle of another shape is RTOSS_ERR_INVALID_ARG.  The work is enqueued
+ * on the stream; the handle is usable by later calls on the same stream.
+ * Free with rtoss_packed_destroy (which synchronises the device). */
+rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, int Cout, int Cin, int ksize,
+                        const uint16_t* masks_host, int P, int k, const uint8_t* pid_dev,
+                        rtoss_dtype compute_dtype, rtoss_packed** out, void* cuda_stream);
+
+typedef struct {
+    int Cout, Cin, ksize, P, k;
+    rtoss_dtype dtype;   /* type of val */
+    int64_t n_kernels;   /* entries of pid */
+    int64_t n_values;    /* entries of val = n_kernels*k */
+} rtoss_packed_info;
+rtoss_status rtoss_packed_info_get(const rtoss_packed* p, rtoss_packed_info* info);
+
+/* Copy the canonical arrays to caller-owned host buffers (any may be NULL to
+ * skip it).  Sizes: pid n_kernels bytes; val n_values elements of the packed
+ * dtype; perm Cin*Cout and bucket_off Cin*(P+1) uint32 (ksize 3 only; ignored
+ * for ksize 1).  Synchronises the stream. */
+rtoss_status rtoss_packed_export(rtoss_ctx* ctx, const rtoss_packed* p, uint8_t* pid_host, void* val_host,
+                                 uint32_t* perm_host, uint32_t* bucket_off_host, void* cuda_stream);
+
+/* Expand to dense masked weights W (.) M ([Cout][Cin][3][3] or [Cout][Cin]) in
+ * the packed dtype; pruned positions are +0. */
+rtoss_status rtoss_packed_to_dense(rtoss_ctx* ctx, const rtoss_packed* p, void* w_masked_dev, void* cuda_stream);
+void rtoss_packed_destroy(rtoss_packed* p);
+
+/* ---- inference convolution over the packed weights ------------------------ */
+
+typedef struct {
+    int N, H, W;            /* batch and INPUT height / width */
+    int stride;             /* 1 or 2 */
+    rtoss_layout layout;    /* of x and y */
+    rtoss_dtype io_dtype;   /* of x and y; accumulation is always fp32 */
+    rtoss_act act;
+    const float* bias_dev;  /* [Cout] fp32, or NULL */
+    int y_channel_offset;   /* y may be a channel slice of a wider tensor: */
+    int y_channel_stride;   /*   channels of that tensor, 0 = Cout */
+} rtoss_conv_desc;
+
+/* y[n,co,oy,ox] = act( bias[co] + sum_ci sum_{t in mask(pid[co,ci])}
+ *                      w[co,ci,t] * x[n,ci,oy*s+r-1,ox*s+c-1] ),  t = 3r+c,
+ * zero outside the image (padding 1); Ho = (H-1)/s+1, Wo = (W-1)/s+1.  Only
+ * the k kept taps of each kernel are multiplied (the cost model of Section
+ * II.B: work proportional to the non-zero weights).  x: N x Cin x H x W in the
+ * given layout, y: N x Cs x Ho x Wo with Cs = y_channel_stride (or Cout),
+ * written at channels [offset, offset+Cout).  x and y must not overlap.  The
+ * packed handle must come from rtoss_pack with ksize 3. */
+rtoss_status rtoss_conv3x3_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const void* x_dev, void* y_dev,
+                                   const rtoss_conv_desc* desc, void* cuda_stream);
+
+/* y[n,co,oy,ox] = act( bias[co] + sum over kept flat positions e = co*Cin+ci
+ *                      of w[e] * x[n,ci,oy*s,ox*s] ); position e is kept when
+ * it lies in a full run g = e/9 and tap e%9 is in mask(pid[g]) (Section IV.D).
+ * No padding; Ho = (H-1)/s+1.  Handle from rtoss_pack with ksize 1. */
+rtoss_status rtoss_conv1x1_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const void* x_dev, void* y_dev,
+                                   const rtoss_conv_desc* desc, void* cuda_stream);
+
+/* Same convolutions with HOST buffers: copies x to the device, runs the
+ * kernel for the handle's ksize, copies y back and waits for it.  x_host and
+ * y_host are dense tensors in desc's layout and dtype (y_channel_* apply).
+ * Uses (and grows on demand) the context's device workspace, so concurrent
+ * calls on one context are not allowed.  bias_dev stays a device pointer. */
+rtoss_status rtoss_conv_pattern_host(rtoss_ctx* ctx, const rtoss_packed* p, const void* x_host, void* y_host,
+                                     const rtoss_conv_desc* desc);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RTOSS_H */

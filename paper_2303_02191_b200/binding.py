@@ -1,0 +1,261 @@
+"""ctypes binding of ``librtoss.so`` (declared in ``include/rtoss.h``).
+
+Argument marshalling only: every step runs in the library's CUDA kernels.
+Importing this module loads the library and raises ``RuntimeError`` when it is
+missing; there is no CPU fallback.  Tensors are torch CUDA tensors (torch is
+used for device memory and streams only).
+"""
+import ctypes
+import os
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "librtoss.so")
+
+OK = 0
+F32, BF16, F16 = 0, 1, 2
+NCHW, NHWC = 0, 1
+ACT_NONE, ACT_RELU, ACT_SILU = 0, 1, 2
+PRESET_ALL, PRESET_CONN4, PRESET_CENTRE8, PRESET_DENSE = 0, 1, 2, 3
+DTYPE_NAMES = {"f32": F32, "bf16": BF16, "f16": F16}
+ACT_NAMES = {"none": ACT_NONE, "relu": ACT_RELU, "silu": ACT_SILU}
+
+SYMBOLS = [
+    "rtoss_create", "rtoss_destroy", "rtoss_status_string", "rtoss_last_error", "rtoss_pattern_preset",
+    "rtoss_pattern_table_validate", "rtoss_group_layers", "rtoss_select_patterns", "rtoss_pack",
+    "rtoss_packed_info_get", "rtoss_packed_export", "rtoss_packed_to_dense", "rtoss_packed_destroy",
+    "rtoss_conv3x3_pattern", "rtoss_conv1x1_pattern", "rtoss_conv_pattern_host",
+]
+
+
+class RtossError(RuntimeError):
+    def __init__(self, status, text):
+        super().__init__("rtoss status %d: %s" % (status, text))
+        self.status = status
+
+
+class LayerNode(ctypes.Structure):
+    _fields_ = [("is_conv", ctypes.c_int), ("cout", ctypes.c_int), ("cin", ctypes.c_int), ("ksize", ctypes.c_int),
+                ("n_inputs", ctypes.c_int), ("inputs", ctypes.POINTER(ctypes.c_int))]
+
+
+class PackedInfo(ctypes.Structure):
+    _fields_ = [("Cout", ctypes.c_int), ("Cin", ctypes.c_int), ("ksize", ctypes.c_int), ("P", ctypes.c_int),
+                ("k", ctypes.c_int), ("dtype", ctypes.c_int), ("n_kernels", ctypes.c_int64),
+                ("n_values", ctypes.c_int64)]
+
+
+class ConvDesc(ctypes.Structure):
+    _fields_ = [("N", ctypes.c_int), ("H", ctypes.c_int), ("W", ctypes.c_int), ("stride", ctypes.c_int),
+                ("layout", ctypes.c_int), ("io_dtype", ctypes.c_int), ("act", ctypes.c_int),
+                ("bias_dev", ctypes.c_void_p), ("y_channel_offset", ctypes.c_int), ("y_channel_stride", ctypes.c_int)]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError("librtoss.so not built (%s): run `python -m paper_2303_02191_b200._build`; "
+                           "there is no CPU fallback" % LIB_PATH)
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ci = ctypes.c_void_p, ctypes.c_int
+    lib.rtoss_create.argtypes = [ci, ctypes.POINTER(vp)]
+    lib.rtoss_destroy.argtypes = [vp]
+    lib.rtoss_destroy.restype = None
+    lib.rtoss_status_string.argtypes = [ci]
+    lib.rtoss_status_string.restype = ctypes.c_char_p
+    lib.rtoss_last_error.argtypes = [vp]
+    lib.rtoss_last_error.restype = ctypes.c_char_p
+    lib.rtoss_pattern_preset.argtypes = [ci, ci, vp, ctypes.POINTER(ci)]
+    lib.rtoss_pattern_table_validate.argtypes = [vp, ci, ci]
+    lib.rtoss_group_layers.argtypes = [ctypes.POINTER(LayerNode), ci, vp, vp, ctypes.POINTER(ci)]
+    lib.rtoss_select_patterns.argtypes = [vp, vp, ci, ci, ci, ci, vp, ci, ci, vp, vp]
+    lib.rtoss_pack.argtypes = [vp, vp, ci, ci, ci, ci, vp, ci, ci, vp, ci, ctypes.POINTER(vp), vp]
+    lib.rtoss_packed_info_get.argtypes = [vp, ctypes.POINTER(PackedInfo)]
+    lib.rtoss_packed_export.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.rtoss_packed_to_dense.argtypes = [vp, vp, vp, vp]
+    lib.rtoss_packed_destroy.argtypes = [vp]
+    lib.rtoss_packed_destroy.restype = None
+    lib.rtoss_conv3x3_pattern.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ConvDesc), vp]
+    lib.rtoss_conv1x1_pattern.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ConvDesc), vp]
+    lib.rtoss_conv_pattern_host.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ConvDesc)]
+    return lib
+
+
+lib = _load()
+
+
+def status_string(s):
+    return lib.rtoss_status_string(int(s)).decode()
+
+
+def _masks_arr(masks):
+    return np.ascontiguousarray(masks, dtype=np.uint16)
+
+
+def _np_ptr(a):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def rtoss_pattern_preset(k, preset):
+    """-> numpy uint16 masks (host only)."""
+    out = np.zeros(512, dtype=np.uint16)
+    n = ctypes.c_int(512)
+    st = lib.rtoss_pattern_preset(int(k), int(preset), _np_ptr(out), ctypes.byref(n))
+    if st != OK:
+        raise RtossError(st, status_string(st))
+    return out[:n.value].copy()
+
+
+def rtoss_pattern_table_validate(masks, k):
+    m = _masks_arr(masks)
+    return lib.rtoss_pattern_table_validate(_np_ptr(m), len(m), int(k))
+
+
+def rtoss_group_layers(nodes):
+    """nodes: list of dict(kind, cout, cin, ksize, inputs) -> (parent, group, n_groups) (host only)."""
+    L = len(nodes)
+    arr = (LayerNode * max(L, 1))()
+    keep = []
+    for i, nd in enumerate(nodes):
+        ins = list(nd.get("inputs", []))
+        buf = (ctypes.c_int * max(len(ins), 1))(*ins)
+        keep.append(buf)
+        arr[i] = LayerNode(1 if nd["kind"] == "conv" else 0, nd.get("cout", 0), nd.get("cin", 0), nd.get("ksize", 0),
+                           len(ins), ctypes.cast(buf, ctypes.POINTER(ctypes.c_int)))
+    parent = np.zeros(max(L, 1), dtype=np.int32)
+    group = np.zeros(max(L, 1), dtype=np.int32)
+    ng = ctypes.c_int(0)
+    st = lib.rtoss_group_layers(arr, L, _np_ptr(parent), _np_ptr(group), ctypes.byref(ng))
+    if st != OK:
+        raise RtossError(st, status_string(st))
+    return parent[:L], group[:L], ng.value
+
+
+def _torch_dtype_code(t):
+    import torch
+    return {torch.float32: F32, torch.bfloat16: BF16, torch.float16: F16}[t.dtype]
+
+
+def _stream():
+    import torch
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class Context:
+    """Owns an rtoss_ctx on one CUDA device."""
+
+    def __init__(self, device=0):
+        h = ctypes.c_void_p()
+        st = lib.rtoss_create(int(device), ctypes.byref(h))
+        if st != OK:
+            raise RtossError(st, "rtoss_create: " + status_string(st) + " (a CUDA device is required)")
+        self.h = h
+        self.device = device
+
+    def close(self):
+        if self.h:
+            lib.rtoss_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st):
+        if st != OK:
+            raise RtossError(st, status_string(st) + " -- " + lib.rtoss_last_error(self.h).decode())
+
+    # -- the four calls of the hot path ------------------------------------------------
+    def rtoss_select_patterns(self, w, ksize, masks, k, pid=None):
+        """w: CUDA tensor [Cout,Cin,3,3] or [Cout,Cin(,1,1)] -> uint8 CUDA tensor of pattern ids."""
+        import torch
+        Cout, Cin = int(w.shape[0]), int(w.shape[1])
+        m = _masks_arr(masks)
+        n = Cout * Cin if ksize == 3 else (Cout * Cin) // 9
+        if pid is None:
+            pid = torch.empty(max(n, 1), dtype=torch.uint8, device=w.device)
+        self._check(lib.rtoss_select_patterns(self.h, w.data_ptr(), _torch_dtype_code(w), Cout, Cin, int(ksize),
+                                              _np_ptr(m), len(m), int(k), pid.data_ptr(), _stream()))
+        return pid[:n]
+
+    def rtoss_pack(self, w, ksize, masks, k, pid, compute_dtype, into=None):
+        """New packed handle, or re-pack `into` (an existing handle of the same layer) without allocating."""
+        Cout, Cin = int(w.shape[0]), int(w.shape[1])
+        m = _masks_arr(masks)
+        h = ctypes.c_void_p(into.h.value) if into is not None else ctypes.c_void_p()
+        self._check(lib.rtoss_pack(self.h, w.data_ptr(), _torch_dtype_code(w), Cout, Cin, int(ksize), _np_ptr(m),
+                                   len(m), int(k), pid.data_ptr(), int(compute_dtype), ctypes.byref(h), _stream()))
+        return into if into is not None else Packed(self, h)
+
+    def _desc(self, x_shape_nchw, stride, layout, io_dtype, act, bias, y_off, y_stride):
+        N, _, H, W = x_shape_nchw
+        return ConvDesc(int(N), int(H), int(W), int(stride), int(layout), int(io_dtype), int(act),
+                        bias.data_ptr() if bias is not None else None, int(y_off), int(y_stride))
+
+    def rtoss_conv3x3_pattern(self, packed, x, y, N, H, W, stride=1, layout=NCHW, act=ACT_NONE, bias=None,
+                              y_channel_offset=0, y_channel_stride=0):
+        d = self._desc((N, 0, H, W), stride, layout, _torch_dtype_code(x), act, bias, y_channel_offset, y_channel_stride)
+        self._check(lib.rtoss_conv3x3_pattern(self.h, packed.h, x.data_ptr(), y.data_ptr(), ctypes.byref(d), _stream()))
+        return y
+
+    def rtoss_conv1x1_pattern(self, packed, x, y, N, H, W, stride=1, layout=NCHW, act=ACT_NONE, bias=None,
+                              y_channel_offset=0, y_channel_stride=0):
+        d = self._desc((N, 0, H, W), stride, layout, _torch_dtype_code(x), act, bias, y_channel_offset, y_channel_stride)
+        self._check(lib.rtoss_conv1x1_pattern(self.h, packed.h, x.data_ptr(), y.data_ptr(), ctypes.byref(d), _stream()))
+        return y
+
+    def rtoss_conv_pattern_host(self, packed, x_host, y_host, N, H, W, stride=1, layout=NCHW, act=ACT_NONE, bias=None,
+                                y_channel_offset=0, y_channel_stride=0):
+        """x_host / y_host: CPU torch tensors (pinned or not); blocks until y_host is written."""
+        d = self._desc((N, 0, H, W), stride, layout, _torch_dtype_code(x_host), act, bias, y_channel_offset,
+                       y_channel_stride)
+        self._check(lib.rtoss_conv_pattern_host(self.h, packed.h, x_host.data_ptr(), y_host.data_ptr(), ctypes.byref(d)))
+        return y_host
+
+
+class Packed:
+    """Owns an rtoss_packed handle."""
+
+    def __init__(self, ctx, h):
+        self.ctx = ctx
+        self.h = h
+        info = PackedInfo()
+        lib.rtoss_packed_info_get(h, ctypes.byref(info))
+        self.info = info
+
+    def export(self):
+        """-> dict of numpy arrays: pid, val (uint16 bits for 16-bit types, float32 else), perm, bucket_off."""
+        i = self.info
+        pid = np.zeros(max(i.n_kernels, 1), dtype=np.uint8)
+        val = np.zeros(max(i.n_values, 1), dtype=np.float32 if i.dtype == F32 else np.uint16)
+        perm = np.zeros(max(i.Cin * i.Cout, 1), dtype=np.uint32)
+        off = np.zeros(max(i.Cin * (i.P + 1), 1), dtype=np.uint32)
+        self.ctx._check(lib.rtoss_packed_export(self.ctx.h, self.h, _np_ptr(pid), _np_ptr(val), _np_ptr(perm),
+                                                _np_ptr(off), _stream()))
+        out = dict(pid=pid[:i.n_kernels], val=val[:i.n_values])
+        if i.ksize == 3:
+            out["perm"] = perm[:i.Cin * i.Cout]
+            out["bucket_off"] = off[:i.Cin * (i.P + 1)]
+        return out
+
+    def to_dense(self):
+        import torch
+        i = self.info
+        td = {F32: torch.float32, BF16: torch.bfloat16, F16: torch.float16}[i.dtype]
+        shape = (i.Cout, i.Cin, 3, 3) if i.ksize == 3 else (i.Cout, i.Cin)
+        out = torch.empty(shape, dtype=td, device="cuda:%d" % self.ctx.device)
+        self.ctx._check(lib.rtoss_packed_to_dense(self.ctx.h, self.h, out.data_ptr(), _stream()))
+        return out
+
+    def close(self):
+        if self.h:
+            lib.rtoss_packed_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

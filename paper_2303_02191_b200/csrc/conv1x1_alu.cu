@@ -1,0 +1,231 @@
+// Pattern-sparse 1x1 convolution on the FP32 FMA pipes.
+//
+// The 1x1 weights of a layer, flattened filter-major, were cut into runs of
+// nine and each run pruned to the k taps of its pattern (Section IV.D,
+// Algorithm 3 of arXiv 2303.02191).  Row co of the [Cout][Cin] matrix therefore
+// keeps about Cin*k/9 entries at irregular positions: a sparse-matrix x
+// dense-matrix product.  A thread keeps CO_T x 32 accumulators (CO_T filters,
+// 32 pixels); per input channel it loads its 32 activations once and, for each
+// of its filters, issues the 32 FMAs only when the (co,ci) weight survived
+// (warp-uniform keep bit, uniform branch).
+#include "conv_common.cuh"
+
+namespace {
+
+using namespace rtoss_dev;
+
+constexpr int kWarps = 8;
+constexpr int kThreads = kWarps * 32;
+constexpr int kCiChunk = 8;
+constexpr int kCoT = 4;
+constexpr int kCoBlock = kWarps * kCoT;  // 32
+constexpr int kPxThread = 32;
+constexpr int kPxTile = 32 * kPxThread;  // 1024 output pixels per CTA
+
+struct Conv1Args {
+    const void* x;
+    void* y;
+    const void* val;
+    const uint8_t* pid;
+    const uint16_t* masks;
+    const float* bias;
+    int val_dtype;
+    int N, Cin, Cout, H, W, Ho, Wo, k, P, stride;
+    long long G;  // full runs of nine
+    int tiles;    // pixel tiles per image
+    int layout, act;
+    int y_c_off, y_c_stride;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads, 1) conv1x1_alu_kernel(const Conv1Args a) {
+    __shared__ __align__(16) float sX[kCiChunk][kPxTile];
+    __shared__ float sW[kCiChunk][kCoBlock];
+    __shared__ unsigned sBits[kCoBlock];
+    __shared__ int tabG[kPxTile];
+    __shared__ uint16_t smask[256];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n = blockIdx.x / a.tiles;
+    const int tile = blockIdx.x - n * a.tiles;
+    const int co0 = blockIdx.y * kCoBlock;
+    const int HoWo = a.Ho * a.Wo;
+    const int pix0 = tile * kPxTile;
+    const size_t HW = (size_t)a.H * a.W;
+
+    for (int e = tid; e < kPxTile; e += kThreads) {
+        const int op = pix0 + e;
+        int g = -1;
+        if (op < HoWo) {
+            const int oy = op / a.Wo, ox = op - oy * a.Wo;
+            g = oy * a.stride * a.W + ox * a.stride;
+        }
+        tabG[e] = g;
+    }
+    for (int p = tid; p < 256; p += kThreads) smask[p] = p < a.P ? a.masks[p] : 0;
+
+    float acc[kCoT][kPxThread];
+#pragma unroll
+    for (int c = 0; c < kCoT; ++c)
+#pragma unroll
+        for (int i = 0; i < kPxThread; ++i) acc[c][i] = 0.f;
+
+    const T* __restrict__ xg = reinterpret_cast<const T*>(a.x);
+    // contiguous fast path: NCHW, stride 1, whole tile inside the image, 16-byte aligned rows of the tile
+    constexpr int kVec = 16 / sizeof(T);
+    const bool fast = a.layout == RTOSS_NCHW && a.stride == 1 && pix0 + kPxTile <= HoWo && (HW % kVec) == 0;
+
+    for (int ci0 = 0; ci0 < a.Cin; ci0 += kCiChunk) {
+        __syncthreads();
+        if (fast) {
+            for (int i = tid; i < kCiChunk * (kPxTile / kVec); i += kThreads) {
+                const int cl = i / (kPxTile / kVec), v = i - cl * (kPxTile / kVec);
+                const int ci = ci0 + cl;
+                float* dst = &sX[cl][v * kVec];
+                if (ci < a.Cin) {
+                    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(xg + ((size_t)n * a.Cin + ci) * HW + pix0) + v);
+                    const T* rv = reinterpret_cast<const T*>(&raw);
+#pragma unroll
+                    for (int q = 0; q < kVec; ++q) dst[q] = to_f32<T>(rv[q]);
+                } else {
+#pragma unroll
+                    for (int q = 0; q < kVec; ++q) dst[q] = 0.f;
+                }
+            }
+        } else if (a.layout == RTOSS_NCHW) {
+            for (int cl = 0; cl < kCiChunk; ++cl) {
+                const int ci = ci0 + cl;
+                const T* plane_ptr = xg + ((size_t)n * a.Cin + (ci < a.Cin ? ci : 0)) * HW;
+                for (int e = tid; e < kPxTile; e += kThreads) {
+                    const int g = tabG[e];
+                    sX[cl][e] = (g >= 0 && ci < a.Cin) ? to_f32<T>(plane_ptr[g]) : 0.f;
+                }
+            }
+        } else {
+            const T* img = xg + (size_t)n * HW * a.Cin;
+            for (int i = tid; i < kPxTile * kCiChunk; i += kThreads) {
+                const int cl = i & (kCiChunk - 1), e = i >> 3;
+                const int ci = ci0 + cl;
+                const int g = tabG[e];
+                sX[cl][e] = (g >= 0 && ci < a.Cin) ? to_f32<T>(img[(size_t)g * a.Cin + ci]) : 0.f;
+            }
+        }
+        // weights of this chunk: thread i -> (filter i/8, channel i%8); keep bits gathered by ballot
+        {
+            const int cl = tid & (kCiChunk - 1), col = tid >> 3;
+            const int co = co0 + col, ci = ci0 + cl;
+            float w = 0.f;
+            bool keep = false;
+            if (co < a.Cout && ci < a.Cin) {
+                const long long e = (long long)co * a.Cin + ci;
+                const long long g = e / 9;
+                const int t = (int)(e - 9 * g);
+                if (g < a.G) {
+                    const unsigned m = smask[a.pid[g]];
+                    if (m & (1u << t)) {
+                        keep = true;
+                        w = load_val(a.val, (size_t)(g * a.k + __popc(m & ((1u << t) - 1u))), a.val_dtype);
+                    }
+                }
+            }
+            sW[cl][col] = w;
+            const unsigned ballot = __ballot_sync(0xFFFFFFFFu, keep);
+            if (cl == 0) sBits[col] = (ballot >> ((lane >> 3) * 8)) & 0xFFu;
+        }
+        __syncthreads();
+
+        unsigned bits[kCoT];
+#pragma unroll
+        for (int c = 0; c < kCoT; ++c) bits[c] = sBits[warp * kCoT + c];
+#pragma unroll 1
+        for (int cl = 0; cl < kCiChunk; ++cl) {
+            float xv[kPxThread];
+#pragma unroll
+            for (int j = 0; j < kPxThread / 4; ++j) {
+                const float4 v = *reinterpret_cast<const float4*>(&sX[cl][j * 128 + lane * 4]);
+                xv[4 * j] = v.x; xv[4 * j + 1] = v.y; xv[4 * j + 2] = v.z; xv[4 * j + 3] = v.w;
+            }
+#pragma unroll
+            for (int c = 0; c < kCoT; ++c) {
+                if ((bits[c] >> cl) & 1u) {
+                    const float w = sW[cl][warp * kCoT + c];
+#pragma unroll
+                    for (int i = 0; i < kPxThread; ++i) acc[c][i] = fmaf(w, xv[i], acc[c][i]);
+                }
+            }
+        }
+    }
+
+    T* __restrict__ yg = reinterpret_cast<T*>(a.y);
+    const int Cs = a.y_c_stride;
+#pragma unroll
+    for (int c = 0; c < kCoT; ++c) {
+        const int co = co0 + warp * kCoT + c;
+        if (co >= a.Cout) continue;
+        const float b = a.bias ? a.bias[co] : 0.f;
+#pragma unroll
+        for (int j = 0; j < kPxThread / 4; ++j) {
+            const int op = pix0 + j * 128 + lane * 4;
+            if (op >= HoWo) continue;
+            if (a.layout == RTOSS_NCHW) {
+                T* dst = yg + ((size_t)n * Cs + a.y_c_off + co) * HoWo + op;
+                if ((HoWo & 3) == 0) {  // op is a multiple of 4 and so is every plane start: aligned 4-element store
+                    __align__(16) T tmp[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) tmp[q] = from_f32<T>(activate(acc[c][4 * j + q] + b, a.act));
+                    if (sizeof(T) == 4) *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(tmp);
+                    else *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(tmp);
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        if (op + q < HoWo) dst[q] = from_f32<T>(activate(acc[c][4 * j + q] + b, a.act));
+                }
+            } else {
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (op + q < HoWo)
+                        yg[((size_t)n * HoWo + op + q) * Cs + a.y_c_off + co] =
+                            from_f32<T>(activate(acc[c][4 * j + q] + b, a.act));
+            }
+        }
+    }
+}
+
+}  // namespace
+
+int rtoss_launch_conv1x1(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y, const rtoss_conv_desc* d,
+                         void* stream) {
+    (void)ctx;
+    Conv1Args a;
+    a.x = x;
+    a.y = y;
+    a.val = p->val;
+    a.pid = p->pid;
+    a.masks = p->masks_dev;
+    a.bias = d->bias_dev;
+    a.val_dtype = (int)p->dtype;
+    a.N = d->N;
+    a.Cin = p->Cin;
+    a.Cout = p->Cout;
+    a.H = d->H;
+    a.W = d->W;
+    a.stride = d->stride;
+    a.Ho = (d->H - 1) / d->stride + 1;
+    a.Wo = (d->W - 1) / d->stride + 1;
+    a.k = p->k;
+    a.P = p->P;
+    a.G = p->n_kernels;
+    a.tiles = (a.Ho * a.Wo + kPxTile - 1) / kPxTile;
+    a.layout = (int)d->layout;
+    a.act = (int)d->act;
+    a.y_c_off = d->y_channel_offset;
+    a.y_c_stride = d->y_channel_stride ? d->y_channel_stride : p->Cout;
+    dim3 grid((unsigned)((size_t)a.tiles * a.N), (unsigned)((a.Cout + kCoBlock - 1) / kCoBlock));
+    cudaStream_t s = (cudaStream_t)stream;
+    switch (d->io_dtype) {
+        case RTOSS_F32: conv1x1_alu_kernel<float><<<grid, kThreads, 0, s>>>(a); break;
+        case RTOSS_BF16: conv1x1_alu_kernel<__nv_bfloat16><<<grid, kThreads, 0, s>>>(a); break;
+        case RTOSS_F16: conv1x1_alu_kernel<__half><<<grid, kThreads, 0, s>>>(a); break;
+    }
+    return (int)cudaGetLastError();
+}

@@ -1,0 +1,349 @@
+// C-ABI entry points of librtoss that touch the device: argument validation,
+// handle lifetimes, kernel launches.  See include/rtoss.h for the contract.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "rtoss.h"
+#include "rtoss_internal.h"
+
+namespace {
+
+void set_err(rtoss_ctx* ctx, const char* what, const char* detail) {
+    if (ctx) snprintf(ctx->err, sizeof(ctx->err), "%s%s%s", what, detail ? ": " : "", detail ? detail : "");
+}
+
+rtoss_status cuda_fail(rtoss_ctx* ctx, const char* where, int e) {
+    set_err(ctx, where, cudaGetErrorString((cudaError_t)e));
+    return RTOSS_ERR_CUDA;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool dtype_ok(int d) { return d == RTOSS_F32 || d == RTOSS_BF16 || d == RTOSS_F16; }
+
+MaskTable make_table(const uint16_t* masks, int P) {
+    MaskTable t;
+    memset(&t, 0, sizeof(t));
+    memcpy(t.m, masks, sizeof(uint16_t) * (size_t)P);
+    return t;
+}
+
+rtoss_status check_layer(rtoss_ctx* ctx, int Cout, int Cin, int ksize) {
+    if (Cout < 1 || Cin < 1 || (ksize != 1 && ksize != 3)) {
+        set_err(ctx, "layer shape", "need Cout, Cin >= 1 and ksize 1 or 3");
+        return RTOSS_ERR_INVALID_ARG;
+    }
+    if ((int64_t)Cout * Cin > (int64_t)1 << 28) {
+        set_err(ctx, "layer shape", "Cout*Cin above 2^28");
+        return RTOSS_ERR_UNSUPPORTED;
+    }
+    return RTOSS_OK;
+}
+
+rtoss_status check_conv(rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y, const rtoss_conv_desc* d,
+                        int ksize, bool device_ptrs) {
+    if (!ctx) return RTOSS_ERR_INVALID_ARG;
+    if (!p || !x || !y || !d) {
+        set_err(ctx, "conv", "null argument");
+        return RTOSS_ERR_INVALID_ARG;
+    }
+    if (p->ksize != ksize) {
+        set_err(ctx, "conv", "packed handle has the other kernel size");
+        return RTOSS_ERR_INVALID_ARG;
+    }
+    if (p->device != ctx->device) {
+        set_err(ctx, "conv", "packed handle lives on another device");
+        return RTOSS_ERR_INVALID_ARG;
+    }
+    if (d->N < 1 || d->H < 1 || d->W < 1 || (d->stride != 1 && d->stride != 2) || !dtype_ok(d->io_dtype) ||
+        (d->layout != RTOSS_NCHW && d->layout != RTOSS_NHWC) ||
+        (d->act != RTOSS_ACT_NONE && d->act != RTOSS_ACT_RELU && d->act != RTOSS_ACT_SILU)) {
+        set_err(ctx, "conv", "bad descriptor (N,H,W >= 1; stride 1|2; dtype; layout; act)");
+        return RTOSS_ERR_INVALID_ARG;
+    }
+    const int cs = d->y_channel_stride ? d->y_channel_stride : p->Cout;
+    if (d->y_channel_offset < 0 || cs < d->y_channel_offset + p->Cout) {
+        set_err(ctx, "conv", "output channel slice does not fit y_channel_stride");
+        return RTOSS_ERR_INVALID_ARG;
+    }
+    if ((int64_t)d->H * d->W > (int64_t)1 << 30) {
+        set_err(ctx, "conv", "H*W above 2^30");
+        return RTOSS_ERR_UNSUPPORTED;
+    }
+    if (device_ptrs && (!aligned16(x) || !aligned16(y))) {
+        set_err(ctx, "conv", "x and y must be 16-byte aligned");
+        return RTOSS_ERR_ALIGNMENT;
+    }
+    return RTOSS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+rtoss_status rtoss_create(int device, rtoss_ctx** out) {
+    if (!out) return RTOSS_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    cudaError_t e = cudaGetDeviceCount(&count);
+    if (e != cudaSuccess || device < 0 || device >= count) return RTOSS_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return RTOSS_ERR_CUDA;
+    if (prop.major < 10) return RTOSS_ERR_UNSUPPORTED;  // kernels are built for sm_100a only
+    rtoss_ctx* c = new (std::nothrow) rtoss_ctx();
+    if (!c) return RTOSS_ERR_ALLOC;
+    memset(c, 0, sizeof(*c));
+    c->device = device;
+    c->sm_count = prop.multiProcessorCount;
+    *out = c;
+    return RTOSS_OK;
+}
+
+void rtoss_destroy(rtoss_ctx* ctx) {
+    if (!ctx) return;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaSetDevice(ctx->device);
+    if (ctx->h_stream) {
+        cudaStreamSynchronize((cudaStream_t)ctx->h_stream);
+        cudaStreamDestroy((cudaStream_t)ctx->h_stream);
+    }
+    if (ctx->ws_x) cudaFree(ctx->ws_x);
+    if (ctx->ws_y) cudaFree(ctx->ws_y);
+    cudaSetDevice(prev);
+    delete ctx;
+}
+
+const char* rtoss_last_error(const rtoss_ctx* ctx) { return ctx ? ctx->err : ""; }
+
+rtoss_status rtoss_select_patterns(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, int Cout, int Cin, int ksize,
+                                   const uint16_t* masks_host, int P, int k, uint8_t* pid_dev, void* cuda_stream) {
+    if (!ctx) return RTOSS_ERR_INVALID_ARG;
+    if (!w_dev || !pid_dev || !masks_host || !dtype_ok(w_dtype)) {
+        set_err(ctx, "select", "null argument or bad dtype");
+        return RTOSS_ERR_INVALID_ARG;
+    }
+    rtoss_status st = check_layer(ctx, Cout, Cin, ksize);
+    if (st != RTOSS_OK) return st;
+    if (!rtoss_table_ok(masks_host, P, k)) {
+        set_err(ctx, "select", "pattern table invalid");
+        return RTOSS_ERR_BAD_PATTERN_TABLE;
+    }
+    if (!aligned16(w_dev)) {
+        set_err(ctx, "select", "weights must be 16-byte aligned");
+        return RTOSS_ERR_ALIGNMENT;
+    }
+    const int64_t n = ksize == 3 ? (int64_t)Cout * Cin : ((int64_t)Cout * Cin) / 9;
+    cudaSetDevice(ctx->device);
+    int e = rtoss_launch_select(w_dev, w_dtype, n, make_table(masks_host, P), P, pid_dev, cuda_stream);
+    return e ? cuda_fail(ctx, "select launch", e) : RTOSS_OK;
+}
+
+rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, int Cout, int Cin, int ksize,
+                        const uint16_t* masks_host, int P, int k, const uint8_t* pid_dev, rtoss_dtype compute_dtype,
+                        rtoss_packed** out, void* cuda_stream) {
+    if (!ctx) return RTOSS_ERR_INVALID_ARG;
+    if (!w_dev || !pid_dev || !masks_host || !out || !dtype_ok(w_dtype) || !dtype_ok(compute_dtype)) {
+        set_err(ctx, "pack", "null argument or bad dtype");
+        return RTOSS_ERR_INVALID_ARG;
+    }
+    rtoss_status st = check_layer(ctx, Cout, Cin, ksize);
+    if (st != RTOSS_OK) return st;
+    if (!rtoss_table_ok(masks_host, P, k)) {
+        set_err(ctx, "pack", "pattern table invalid");
+        return RTOSS_ERR_BAD_PATTERN_TABLE;
+    }
+    if (!aligned16(w_dev)) {
+        set_err(ctx, "pack", "weights must be 16-byte aligned");
+        return RTOSS_ERR_ALIGNMENT;
+    }
+    cudaSetDevice(ctx->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaSuccess;
+    rtoss_packed* p = *out;
+    const bool reuse = p != nullptr;
+    if (reuse) {
+        // re-pack into an existing handle (e.g. after another pruning iteration): same layer, no allocation
+        if (p->device != ctx->device || p->Cout != Cout || p->Cin != Cin || p->ksize != ksize || p->P != P || p->k != k ||
+            p->dtype != compute_dtype) {
+            set_err(ctx, "pack", "existing handle describes another layer, table size or dtype");
+            return RTOSS_ERR_INVALID_ARG;
+        }
+        memset(p->masks, 0, sizeof(p->masks));
+        memcpy(p->masks, masks_host, sizeof(uint16_t) * (size_t)P);
+    } else {
+        p = new (std::nothrow) rtoss_packed();
+        if (!p) return RTOSS_ERR_ALLOC;
+        memset(p, 0, sizeof(*p));
+        p->device = ctx->device;
+        p->Cout = Cout;
+        p->Cin = Cin;
+        p->ksize = ksize;
+        p->P = P;
+        p->k = k;
+        p->dtype = compute_dtype;
+        p->n_kernels = ksize == 3 ? (int64_t)Cout * Cin : ((int64_t)Cout * Cin) / 9;
+        memcpy(p->masks, masks_host, sizeof(uint16_t) * (size_t)P);
+        const size_t nk = (size_t)(p->n_kernels > 0 ? p->n_kernels : 1);
+        e = cudaMalloc((void**)&p->pid, nk);
+        if (e == cudaSuccess) e = cudaMalloc(&p->val, nk * (size_t)k * rtoss_dtype_size(compute_dtype));
+        if (e == cudaSuccess) e = cudaMalloc((void**)&p->masks_dev, sizeof(uint16_t) * 256);
+        if (e == cudaSuccess && ksize == 3) {
+            e = cudaMalloc((void**)&p->perm, sizeof(uint32_t) * (size_t)Cin * Cout);
+            if (e == cudaSuccess) e = cudaMalloc((void**)&p->bucket_off, sizeof(uint32_t) * (size_t)Cin * (P + 1));
+        }
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            rtoss_packed_destroy(p);
+            set_err(ctx, "pack", "device allocation failed");
+            return RTOSS_ERR_ALLOC;
+        }
+    }
+    int le = 0;
+    // the mask table is copied from the handle's own (pageable) storage: the copy is staged before return
+    e = cudaMemcpyAsync(p->masks_dev, p->masks, sizeof(uint16_t) * 256, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess && p->n_kernels > 0)
+        e = cudaMemcpyAsync(p->pid, pid_dev, (size_t)p->n_kernels, cudaMemcpyDeviceToDevice, s);
+    if (e == cudaSuccess)
+        le = rtoss_launch_pack_values(w_dev, w_dtype, p->n_kernels, make_table(masks_host, P), pid_dev, k, p->val,
+                                      compute_dtype, cuda_stream);
+    if (e == cudaSuccess && !le && ksize == 3)
+        le = rtoss_launch_pack_order(pid_dev, Cout, Cin, P, p->perm, p->bucket_off, cuda_stream);
+    if (e != cudaSuccess || le) {
+        rtoss_status r = cuda_fail(ctx, "pack launch", e != cudaSuccess ? (int)e : le);
+        if (!reuse) rtoss_packed_destroy(p);
+        return r;
+    }
+    *out = p;
+    return RTOSS_OK;
+}
+
+rtoss_status rtoss_packed_info_get(const rtoss_packed* p, rtoss_packed_info* info) {
+    if (!p || !info) return RTOSS_ERR_INVALID_ARG;
+    info->Cout = p->Cout;
+    info->Cin = p->Cin;
+    info->ksize = p->ksize;
+    info->P = p->P;
+    info->k = p->k;
+    info->dtype = p->dtype;
+    info->n_kernels = p->n_kernels;
+    info->n_values = p->n_kernels * p->k;
+    return RTOSS_OK;
+}
+
+rtoss_status rtoss_packed_export(rtoss_ctx* ctx, const rtoss_packed* p, uint8_t* pid_host, void* val_host,
+                                 uint32_t* perm_host, uint32_t* bucket_off_host, void* cuda_stream) {
+    if (!ctx || !p) return RTOSS_ERR_INVALID_ARG;
+    cudaSetDevice(p->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaSuccess;
+    if (pid_host && p->n_kernels > 0) e = cudaMemcpyAsync(pid_host, p->pid, (size_t)p->n_kernels, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && val_host && p->n_kernels > 0)
+        e = cudaMemcpyAsync(val_host, p->val, (size_t)p->n_kernels * p->k * rtoss_dtype_size(p->dtype),
+                            cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && p->ksize == 3 && perm_host)
+        e = cudaMemcpyAsync(perm_host, p->perm, sizeof(uint32_t) * (size_t)p->Cin * p->Cout, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && p->ksize == 3 && bucket_off_host)
+        e = cudaMemcpyAsync(bucket_off_host, p->bucket_off, sizeof(uint32_t) * (size_t)p->Cin * (p->P + 1),
+                            cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    return e == cudaSuccess ? RTOSS_OK : cuda_fail(ctx, "packed export", (int)e);
+}
+
+rtoss_status rtoss_packed_to_dense(rtoss_ctx* ctx, const rtoss_packed* p, void* w_masked_dev, void* cuda_stream) {
+    if (!ctx || !p || !w_masked_dev) return RTOSS_ERR_INVALID_ARG;
+    cudaSetDevice(p->device);
+    int e = rtoss_launch_to_dense(p, w_masked_dev, cuda_stream);
+    return e ? cuda_fail(ctx, "to_dense launch", e) : RTOSS_OK;
+}
+
+void rtoss_packed_destroy(rtoss_packed* p) {
+    if (!p) return;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaSetDevice(p->device);
+    cudaDeviceSynchronize();
+    if (p->pid) cudaFree(p->pid);
+    if (p->val) cudaFree(p->val);
+    if (p->perm) cudaFree(p->perm);
+    if (p->bucket_off) cudaFree(p->bucket_off);
+    if (p->masks_dev) cudaFree(p->masks_dev);
+    cudaSetDevice(prev);
+    delete p;
+}
+
+rtoss_status rtoss_conv3x3_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const void* x_dev, void* y_dev,
+                                   const rtoss_conv_desc* desc, void* cuda_stream) {
+    rtoss_status st = check_conv(ctx, p, x_dev, y_dev, desc, 3, true);
+    if (st != RTOSS_OK) return st;
+    cudaSetDevice(ctx->device);
+    int e = rtoss_launch_conv3x3(ctx, p, x_dev, y_dev, desc, cuda_stream);
+    return e ? cuda_fail(ctx, "conv3x3 launch", e) : RTOSS_OK;
+}
+
+rtoss_status rtoss_conv1x1_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const void* x_dev, void* y_dev,
+                                   const rtoss_conv_desc* desc, void* cuda_stream) {
+    rtoss_status st = check_conv(ctx, p, x_dev, y_dev, desc, 1, true);
+    if (st != RTOSS_OK) return st;
+    cudaSetDevice(ctx->device);
+    int e = rtoss_launch_conv1x1(ctx, p, x_dev, y_dev, desc, cuda_stream);
+    return e ? cuda_fail(ctx, "conv1x1 launch", e) : RTOSS_OK;
+}
+
+rtoss_status rtoss_conv_pattern_host(rtoss_ctx* ctx, const rtoss_packed* p, const void* x_host, void* y_host,
+                                     const rtoss_conv_desc* desc) {
+    if (!ctx || !p) return RTOSS_ERR_INVALID_ARG;
+    rtoss_status st = check_conv(ctx, p, x_host, y_host, desc, p->ksize, false);
+    if (st != RTOSS_OK) return st;
+    cudaSetDevice(ctx->device);
+    const size_t es = rtoss_dtype_size(desc->io_dtype);
+    const int Ho = (desc->H - 1) / desc->stride + 1, Wo = (desc->W - 1) / desc->stride + 1;
+    const int cs = desc->y_channel_stride ? desc->y_channel_stride : p->Cout;
+    const size_t xb = (size_t)desc->N * p->Cin * desc->H * desc->W * es;
+    const size_t yb = (size_t)desc->N * cs * Ho * Wo * es;
+    cudaError_t e = cudaSuccess;
+    if (!ctx->h_stream) {
+        cudaStream_t s;
+        e = cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking);
+        if (e != cudaSuccess) return cuda_fail(ctx, "host path stream", (int)e);
+        ctx->h_stream = s;
+    }
+    if (ctx->ws_x_bytes < xb) {
+        if (ctx->ws_x) cudaFree(ctx->ws_x);
+        ctx->ws_x = nullptr;
+        ctx->ws_x_bytes = 0;
+        if (cudaMalloc(&ctx->ws_x, xb) != cudaSuccess) {
+            cudaGetLastError();
+            set_err(ctx, "host path", "workspace allocation failed");
+            return RTOSS_ERR_ALLOC;
+        }
+        ctx->ws_x_bytes = xb;
+    }
+    if (ctx->ws_y_bytes < yb) {
+        if (ctx->ws_y) cudaFree(ctx->ws_y);
+        ctx->ws_y = nullptr;
+        ctx->ws_y_bytes = 0;
+        if (cudaMalloc(&ctx->ws_y, yb) != cudaSuccess) {
+            cudaGetLastError();
+            set_err(ctx, "host path", "workspace allocation failed");
+            return RTOSS_ERR_ALLOC;
+        }
+        ctx->ws_y_bytes = yb;
+    }
+    cudaStream_t s = (cudaStream_t)ctx->h_stream;
+    const bool slice = cs != p->Cout;
+    e = cudaMemcpyAsync(ctx->ws_x, x_host, xb, cudaMemcpyHostToDevice, s);
+    // a channel slice leaves the other channels of y untouched: bring the caller's y over first
+    if (e == cudaSuccess && slice) e = cudaMemcpyAsync(ctx->ws_y, y_host, yb, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, "host path copy in", (int)e);
+    int le = p->ksize == 3 ? rtoss_launch_conv3x3(ctx, p, ctx->ws_x, ctx->ws_y, desc, s)
+                           : rtoss_launch_conv1x1(ctx, p, ctx->ws_x, ctx->ws_y, desc, s);
+    if (le) return cuda_fail(ctx, "host path launch", le);
+    e = cudaMemcpyAsync(y_host, ctx->ws_y, yb, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    return e == cudaSuccess ? RTOSS_OK : cuda_fail(ctx, "host path copy out", (int)e);
+}
+
+}  // extern "C"

@@ -1,0 +1,57 @@
+// Internal definitions shared by the translation units of librtoss.
+#ifndef RTOSS_INTERNAL_H
+#define RTOSS_INTERNAL_H
+
+#include <cstddef>
+#include <cstdint>
+
+#include "rtoss.h"
+
+struct rtoss_ctx {
+    int device;
+    int sm_count;
+    char err[256];
+    // device workspace of the host-buffer path (grown on demand)
+    void* ws_x;
+    size_t ws_x_bytes;
+    void* ws_y;
+    size_t ws_y_bytes;
+    void* h_stream;  // cudaStream_t owned by the context, used by the host-buffer path
+};
+
+struct rtoss_packed {
+    int device;
+    int Cout, Cin, ksize, P, k;
+    rtoss_dtype dtype;
+    int64_t n_kernels;
+    uint8_t* pid;          // [n_kernels]
+    void* val;             // [n_kernels*k] in dtype
+    uint32_t* perm;        // [Cin*Cout]      (ksize 3)
+    uint32_t* bucket_off;  // [Cin*(P+1)]     (ksize 3)
+    uint16_t* masks_dev;   // [256]
+    uint16_t masks[256];
+};
+
+// Pattern table passed by value to kernels (constant bank, uniform reads).
+struct MaskTable {
+    uint16_t m[256];
+};
+
+bool rtoss_table_ok(const uint16_t* masks, int P, int k);
+
+static inline size_t rtoss_dtype_size(rtoss_dtype d) { return d == RTOSS_F32 ? 4 : 2; }
+
+// kernel launchers (select_pack.cu, conv3x3_alu.cu, conv1x1_alu.cu); each returns a cudaError_t as int
+int rtoss_launch_select(const void* w, rtoss_dtype wdt, int64_t n_kernels, const MaskTable& t, int P, uint8_t* pid,
+                        void* stream);
+int rtoss_launch_pack_values(const void* w, rtoss_dtype wdt, int64_t n_kernels, const MaskTable& t, const uint8_t* pid,
+                             int k, void* val, rtoss_dtype vdt, void* stream);
+int rtoss_launch_pack_order(const uint8_t* pid, int Cout, int Cin, int P, uint32_t* perm, uint32_t* bucket_off,
+                            void* stream);
+int rtoss_launch_to_dense(const rtoss_packed* p, void* w_out, void* stream);
+int rtoss_launch_conv3x3(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y,
+                         const rtoss_conv_desc* d, void* stream);
+int rtoss_launch_conv1x1(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y,
+                         const rtoss_conv_desc* d, void* stream);
+
+#endif

@@ -1,0 +1,266 @@
+// Pattern selection (Algorithm 2 / Algorithm 3 of arXiv 2303.02191) and the
+// packing kernels.  All three are bandwidth-bound streaming passes over the
+// weights: 9 values read per kernel, one byte (pid) or k values written.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include "rtoss_internal.h"
+
+namespace {
+
+constexpr int kSelThreads = 256;  // kernels per block iteration
+
+template <typename T> __device__ __forceinline__ float widen(T v);
+template <> __device__ __forceinline__ float widen<float>(float v) { return v; }
+template <> __device__ __forceinline__ float widen<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <> __device__ __forceinline__ float widen<__half>(__half v) { return __half2float(v); }
+
+template <typename T> __device__ __forceinline__ T narrow(float v);
+template <> __device__ __forceinline__ float narrow<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 narrow<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+template <> __device__ __forceinline__ __half narrow<__half>(float v) { return __float2half_rn(v); }
+
+// Copy the 9*count weights of `count` consecutive kernels starting at kernel
+// `first` into shared memory, coalesced, 16 bytes per thread where the chunk is
+// whole.  The base pointer is 16-byte aligned and a full chunk is a multiple
+// of 16 bytes, so every full chunk starts on a 16-byte boundary.
+template <typename T>
+__device__ __forceinline__ void stage_kernels(const T* __restrict__ w, int64_t first, int count, T* smem) {
+    const T* src = w + first * 9;
+    constexpr int kVecElems = 16 / sizeof(T);
+    if (count == kSelThreads) {
+        const int nvec = kSelThreads * 9 / kVecElems;
+        const uint4* s4 = reinterpret_cast<const uint4*>(src);
+        uint4* d4 = reinterpret_cast<uint4*>(smem);
+        for (int i = threadIdx.x; i < nvec; i += kSelThreads) d4[i] = __ldg(s4 + i);
+    } else {
+        for (int i = threadIdx.x; i < count * 9; i += kSelThreads) smem[i] = src[i];
+    }
+}
+
+// One thread per kernel: squares in fp32, pattern sums in fp32 over ascending
+// taps, first strictly larger sum wins.  __fmul_rn / __fadd_rn keep the
+// compiler from contracting or reordering the arithmetic.
+template <typename T>
+__global__ void __launch_bounds__(kSelThreads) select_kernel(const T* __restrict__ w, int64_t n_kernels, MaskTable table,
+                                                             int P, uint8_t* __restrict__ pid) {
+    __shared__ __align__(16) T sw[kSelThreads * 9];
+    const int64_t n_chunks = (n_kernels + kSelThreads - 1) / kSelThreads;
+    for (int64_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
+        const int64_t first = chunk * kSelThreads;
+        const int count = (int)min((int64_t)kSelThreads, n_kernels - first);
+        __syncthreads();
+        stage_kernels<T>(w, first, count, sw);
+        __syncthreads();
+        if ((int)threadIdx.x < count) {
+            float q[9];
+#pragma unroll
+            for (int t = 0; t < 9; ++t) {
+                float v = widen<T>(sw[threadIdx.x * 9 + t]);
+                q[t] = __fmul_rn(v, v);
+            }
+            int best = 0;
+            float best_s = 0.f;
+            for (int p = 0; p < P; ++p) {
+                const unsigned m = table.m[p];
+                float s = 0.f;
+#pragma unroll
+                for (int t = 0; t < 9; ++t)
+                    if (m & (1u << t)) s = __fadd_rn(s, q[t]);
+                if (p == 0) {
+                    best_s = s;
+                } else if (s > best_s || (best_s != best_s && s == s)) {
+                    best = p;
+                    best_s = s;
+                }
+            }
+            pid[first + threadIdx.x] = (uint8_t)best;
+        }
+    }
+}
+
+// Gather the k kept values of each kernel (ascending tap order) and round them
+// to the packed type.
+template <typename T, typename V>
+__global__ void __launch_bounds__(kSelThreads) pack_values_kernel(const T* __restrict__ w, int64_t n_kernels,
+                                                                  MaskTable table, const uint8_t* __restrict__ pid, int k,
+                                                                  V* __restrict__ val) {
+    __shared__ __align__(16) T sw[kSelThreads * 9];
+    const int64_t n_chunks = (n_kernels + kSelThreads - 1) / kSelThreads;
+    for (int64_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
+        const int64_t first = chunk * kSelThreads;
+        const int count = (int)min((int64_t)kSelThreads, n_kernels - first);
+        __syncthreads();
+        stage_kernels<T>(w, first, count, sw);
+        __syncthreads();
+        if ((int)threadIdx.x < count) {
+            const int64_t i = first + threadIdx.x;
+            const unsigned m = table.m[pid[i]];
+            V* out = val + i * k;
+            int j = 0;
+#pragma unroll
+            for (int t = 0; t < 9; ++t)
+                if (m & (1u << t)) out[j++] = narrow<V>(widen<T>(sw[threadIdx.x * 9 + t]));
+        }
+    }
+}
+
+// Per input channel: stable counting sort of the filters by pattern id.  One
+// warp per channel; ranks inside a group of 32 filters come from
+// __match_any_sync, running bucket fill levels live in shared memory.
+constexpr int kOrderWarps = 4;
+__global__ void __launch_bounds__(kOrderWarps * 32) pack_order_kernel(const uint8_t* __restrict__ pid, int Cout, int Cin,
+                                                                      int P, uint32_t* __restrict__ perm,
+                                                                      uint32_t* __restrict__ bucket_off) {
+    __shared__ uint32_t fill_all[kOrderWarps][256];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint32_t* fill = fill_all[warp];
+    const int ci = blockIdx.x * kOrderWarps + warp;
+    if (ci >= Cin) return;  // whole warp leaves together; no block-wide barrier below
+    for (int p = lane; p < 256; p += 32) fill[p] = 0;
+    __syncwarp();
+    // pass 1: histogram
+    for (int base = 0; base < Cout; base += 32) {
+        const int co = base + lane;
+        const unsigned key = co < Cout ? pid[(size_t)co * Cin + ci] : 0xFFFFu;
+        const unsigned peers = __match_any_sync(0xFFFFFFFFu, key);
+        if (co < Cout && lane == __ffs(peers) - 1) fill[key] += __popc(peers);
+        __syncwarp();
+    }
+    // exclusive scan over the P buckets (P <= 255: eight per lane, then a warp scan of lane totals)
+    uint32_t local[8];
+    uint32_t sum = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int p = lane * 8 + j;
+        local[j] = sum;
+        sum += (p < P) ? fill[p] : 0;
+    }
+    uint32_t incl = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= d) incl += o;
+    }
+    const uint32_t excl = incl - sum;
+    __syncwarp();
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int p = lane * 8 + j;
+        if (p < P) {
+            fill[p] = excl + local[j];
+            bucket_off[(size_t)ci * (P + 1) + p] = excl + local[j];
+        }
+    }
+    if (lane == 0) bucket_off[(size_t)ci * (P + 1) + P] = (uint32_t)Cout;
+    __syncwarp();
+    // pass 2: placement, filters in ascending order inside each bucket
+    for (int base = 0; base < Cout; base += 32) {
+        const int co = base + lane;
+        const unsigned key = co < Cout ? pid[(size_t)co * Cin + ci] : 0xFFFFu;
+        const unsigned peers = __match_any_sync(0xFFFFFFFFu, key);
+        const unsigned before = peers & ((1u << lane) - 1u);
+        if (co < Cout) perm[(size_t)ci * Cout + fill[key] + __popc(before)] = (uint32_t)co;
+        __syncwarp();
+        if (co < Cout && before == 0) fill[key] += __popc(peers);
+        __syncwarp();
+    }
+}
+
+// Dense masked weights from the packed form, one thread per dense element.
+template <typename V>
+__global__ void to_dense_kernel(const V* __restrict__ val, const uint8_t* __restrict__ pid,
+                                const uint16_t* __restrict__ masks, int k, int64_t n_kernels, int64_t n_dense,
+                                V* __restrict__ out) {
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n_dense; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t g = e / 9;
+        const int t = (int)(e - 9 * g);
+        V v = narrow<V>(0.f);
+        if (g < n_kernels) {
+            const unsigned m = masks[pid[g]];
+            if (m & (1u << t)) v = val[g * k + __popc(m & ((1u << t) - 1u))];
+        }
+        out[e] = v;
+    }
+}
+
+int grid_for(int64_t n_chunks) {
+    int64_t g = n_chunks < 1 ? 1 : n_chunks;
+    const int64_t cap = 148 * 8;
+    return (int)(g > cap ? cap : g);
+}
+
+}  // namespace
+
+int rtoss_launch_select(const void* w, rtoss_dtype wdt, int64_t n_kernels, const MaskTable& t, int P, uint8_t* pid,
+                        void* stream) {
+    if (n_kernels <= 0) return 0;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int grid = grid_for((n_kernels + kSelThreads - 1) / kSelThreads);
+    switch (wdt) {
+        case RTOSS_F32: select_kernel<float><<<grid, kSelThreads, 0, s>>>((const float*)w, n_kernels, t, P, pid); break;
+        case RTOSS_BF16:
+            select_kernel<__nv_bfloat16><<<grid, kSelThreads, 0, s>>>((const __nv_bfloat16*)w, n_kernels, t, P, pid);
+            break;
+        case RTOSS_F16: select_kernel<__half><<<grid, kSelThreads, 0, s>>>((const __half*)w, n_kernels, t, P, pid); break;
+    }
+    return (int)cudaGetLastError();
+}
+
+template <typename T>
+static int launch_pack_values_t(const T* w, int64_t n, const MaskTable& t, const uint8_t* pid, int k, void* val,
+                                rtoss_dtype vdt, cudaStream_t s) {
+    const int grid = grid_for((n + kSelThreads - 1) / kSelThreads);
+    switch (vdt) {
+        case RTOSS_F32: pack_values_kernel<T, float><<<grid, kSelThreads, 0, s>>>(w, n, t, pid, k, (float*)val); break;
+        case RTOSS_BF16:
+            pack_values_kernel<T, __nv_bfloat16><<<grid, kSelThreads, 0, s>>>(w, n, t, pid, k, (__nv_bfloat16*)val);
+            break;
+        case RTOSS_F16: pack_values_kernel<T, __half><<<grid, kSelThreads, 0, s>>>(w, n, t, pid, k, (__half*)val); break;
+    }
+    return (int)cudaGetLastError();
+}
+
+int rtoss_launch_pack_values(const void* w, rtoss_dtype wdt, int64_t n_kernels, const MaskTable& t, const uint8_t* pid,
+                             int k, void* val, rtoss_dtype vdt, void* stream) {
+    if (n_kernels <= 0) return 0;
+    cudaStream_t s = (cudaStream_t)stream;
+    switch (wdt) {
+        case RTOSS_F32: return launch_pack_values_t<float>((const float*)w, n_kernels, t, pid, k, val, vdt, s);
+        case RTOSS_BF16:
+            return launch_pack_values_t<__nv_bfloat16>((const __nv_bfloat16*)w, n_kernels, t, pid, k, val, vdt, s);
+        case RTOSS_F16: return launch_pack_values_t<__half>((const __half*)w, n_kernels, t, pid, k, val, vdt, s);
+    }
+    return (int)cudaErrorInvalidValue;
+}
+
+int rtoss_launch_pack_order(const uint8_t* pid, int Cout, int Cin, int P, uint32_t* perm, uint32_t* bucket_off,
+                            void* stream) {
+    const int grid = (Cin + kOrderWarps - 1) / kOrderWarps;
+    pack_order_kernel<<<grid, kOrderWarps * 32, 0, (cudaStream_t)stream>>>(pid, Cout, Cin, P, perm, bucket_off);
+    return (int)cudaGetLastError();
+}
+
+int rtoss_launch_to_dense(const rtoss_packed* p, void* w_out, void* stream) {
+    const int64_t n_dense = p->ksize == 3 ? p->n_kernels * 9 : (int64_t)p->Cout * p->Cin;
+    if (n_dense <= 0) return 0;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int threads = 256;
+    const int grid = grid_for((n_dense + threads - 1) / threads);
+    switch (p->dtype) {
+        case RTOSS_F32:
+            to_dense_kernel<float><<<grid, threads, 0, s>>>((const float*)p->val, p->pid, p->masks_dev, p->k, p->n_kernels,
+                                                            n_dense, (float*)w_out);
+            break;
+        case RTOSS_BF16:
+            to_dense_kernel<__nv_bfloat16><<<grid, threads, 0, s>>>((const __nv_bfloat16*)p->val, p->pid, p->masks_dev,
+                                                                    p->k, p->n_kernels, n_dense, (__nv_bfloat16*)w_out);
+            break;
+        case RTOSS_F16:
+            to_dense_kernel<__half><<<grid, threads, 0, s>>>((const __half*)p->val, p->pid, p->masks_dev, p->k,
+                                                             p->n_kernels, n_dense, (__half*)w_out);
+            break;
+    }
+    return (int)cudaGetLastError();
+}
