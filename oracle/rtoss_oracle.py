@@ -24,10 +24,14 @@ _lib = None
 
 def build(force=False):
     """Compile the oracle (gcc, OpenMP, no FP contraction)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    import hashlib
+    stamp = _LIB + ".stamp"
+    fp = hashlib.sha256(open(_SRC, "rb").read()).hexdigest()
+    if force or not os.path.exists(_LIB) or not os.path.exists(stamp) or open(stamp).read().strip() != fp:
         cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fPIC", "-shared",
                _SRC, "-o", _LIB, "-lm"]
         subprocess.check_call(cmd)
+        open(stamp, "w").write(fp)
     return _LIB
 
 

@@ -51,7 +51,23 @@ def _compile(nvcc, src, verbose):
     return obj
 
 
+def _fingerprint():
+    """Hash of every source and header plus the flags: the library is rebuilt only when it changes
+    (file times do not survive a copy of the tree)."""
+    import hashlib
+    h = hashlib.sha256(" ".join(NVCC_FLAGS[:3] + ARCH).encode())
+    files = [os.path.join(CSRC, f) for f in sorted(os.listdir(CSRC))] + [os.path.join(INC, f) for f in sorted(os.listdir(INC))]
+    for f in files:
+        h.update(os.path.basename(f).encode())
+        h.update(open(f, "rb").read())
+    return h.hexdigest()
+
+
 def build(verbose=False, force=False):
+    stamp = LIB + ".stamp"
+    fp = _fingerprint()
+    if not force and not verbose and os.path.exists(LIB) and os.path.exists(stamp) and open(stamp).read().strip() == fp:
+        return LIB
     nvcc = _nvcc()
     os.makedirs(OBJ, exist_ok=True)
     if force:
@@ -63,6 +79,7 @@ def build(verbose=False, force=False):
     if (not os.path.exists(LIB)) or any(os.path.getmtime(o) > os.path.getmtime(LIB) for o in objs):
         cmd = [nvcc, "-shared", "-o", LIB] + objs + ARCH + ["-Xcompiler", "-fPIC", "-cudart", "static"]
         subprocess.check_call(cmd)
+    open(stamp, "w").write(fp)
     return LIB
 
 
