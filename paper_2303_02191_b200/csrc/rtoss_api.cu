@@ -121,7 +121,8 @@ const char* rtoss_last_error(const rtoss_ctx* ctx) { return ctx ? ctx->err : "";
 rtoss_status rtoss_select_patterns(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, int Cout, int Cin, int ksize,
                                    const uint16_t* masks_host, int P, int k, uint8_t* pid_dev, void* cuda_stream) {
     if (!ctx) return RTOSS_ERR_INVALID_ARG;
-    if (!w_dev || !pid_dev || !masks_host || !dtype_ok(w_dtype)) {
+    const bool none_sel = ksize == 1 && (int64_t)Cout * Cin < 9;  // no full run of nine: nothing to write
+    if (!w_dev || (!pid_dev && !none_sel) || !masks_host || !dtype_ok(w_dtype)) {
         set_err(ctx, "select", "null argument or bad dtype");
         return RTOSS_ERR_INVALID_ARG;
     }
@@ -145,7 +146,8 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
                         const uint16_t* masks_host, int P, int k, const uint8_t* pid_dev, rtoss_dtype compute_dtype,
                         rtoss_packed** out, void* cuda_stream) {
     if (!ctx) return RTOSS_ERR_INVALID_ARG;
-    if (!w_dev || !pid_dev || !masks_host || !out || !dtype_ok(w_dtype) || !dtype_ok(compute_dtype)) {
+    const bool none_sel = ksize == 1 && (int64_t)Cout * Cin < 9;  // no full run of nine: pid may be NULL
+    if (!w_dev || (!pid_dev && !none_sel) || !masks_host || !out || !dtype_ok(w_dtype) || !dtype_ok(compute_dtype)) {
         set_err(ctx, "pack", "null argument or bad dtype");
         return RTOSS_ERR_INVALID_ARG;
     }
