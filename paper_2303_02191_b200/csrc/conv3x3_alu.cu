@@ -21,9 +21,16 @@
 //     are read once; each tap whose mask bit is set runs PH*PW FMAs with static
 //     register indices; cleared taps are skipped by a uniform branch.  Only
 //     k*PH*PW FMAs are issued per kernel.
-//   * Input channels are staged CI_CHUNK at a time: activations converted to
-//     fp32 once per tile (zero outside the image = the padding), weights
-//     expanded from the packed (pid, k values) form into 9 slots + mask.
+//   * Input channels are processed kCiChunk at a time through a two-stage
+//     pipeline: while chunk i is being computed, the raw bytes of chunk i+1
+//     (activations in their storage type, packed values and pattern ids) arrive
+//     in shared memory through cp.async.  Before computing a chunk its raw bytes
+//     are converted once: activations to fp32 (zero outside the image = the
+//     padding), weights from (pid, k values) to 9 slots + mask.
+//   * cp.async needs aligned rows.  NCHW: image rows must start on a multiple of
+//     4, 8 or 16 bytes (the widest that divides W*elem is used); NHWC: Cin a
+//     multiple of 8.  Weights: Cin a multiple of 8.  Anything else takes a plain
+//     load-convert-store path inside the same kernel.
 #include "conv_common.cuh"
 
 namespace {
@@ -35,6 +42,8 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kCiChunk = 8;
 constexpr int kWSlots = 12;  // 9 weights, mask, 2 pad: three float4 per kernel
 
+enum XMode { X_SYNC = 0, X_NCHW_VEC = 1, X_NHWC_VEC = 2 };
+
 struct Conv3Args {
     const void* x;
     void* y;
@@ -42,13 +51,27 @@ struct Conv3Args {
     const uint8_t* pid;
     const uint16_t* masks;
     const float* bias;
-    int val_dtype;
+    int val_dtype, val_esize;
     int N, Cin, Cout, H, W, Ho, Wo, k, P;
     int LX, LY, tiles_x, tiles_y;
-    int TH_in, TW_in, TWP, plane;  // staged tile: rows, cols, row pitch, channel pitch (floats)
+    int TH_in, TW_in, TWP, plane;  // staged fp32 tile: rows, cols, row pitch, channel pitch (floats)
+    int xmode;                     // XMode
+    int vb;                        // bytes per cp.async of activations (4, 8, 16)
+    int EV;                        // raw vectors per channel plane (NCHW) or pixels per tile (NHWC)
+    int w_async;                   // packed weights arrive through cp.async
     int layout, act;
     int y_c_off, y_c_stride;
+    // byte offsets of the shared-memory regions
+    int off_sW, off_rawX, rawX_bytes, off_rawV, rawV_bytes, off_rawP, off_tab;
 };
+
+__device__ __forceinline__ void cp_async(void* smem_dst, const void* gsrc, int bytes) {
+    const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
+    if (bytes == 16) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gsrc) : "memory");
+    else if (bytes == 8) asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(s), "l"(gsrc) : "memory");
+    else asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(s), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 template <int S, int PH, int PW, int R, int C>
 __device__ __forceinline__ void fma_tap(float (&acc)[PH][PW], const float (&win)[(PH - 1) * S + 3][(PW - 1) * S + 3],
@@ -65,10 +88,16 @@ __global__ void __launch_bounds__(kThreads, 1) conv3x3_alu_kernel(const Conv3Arg
     constexpr int WIN_W = (PW - 1) * S + 3;
     constexpr int CO_BLOCK = kWarps * CO_T;
 
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    float* sX = reinterpret_cast<float*>(smem_raw);                        // [kCiChunk][plane]
-    float* sW = sX + kCiChunk * a.plane;                                   // [kCiChunk][CO_BLOCK][kWSlots]
-    int* tabG = reinterpret_cast<int*>(sW + kCiChunk * CO_BLOCK * kWSlots);  // [TH_in*TWP]
+    constexpr int VE16 = 16 / (int)sizeof(T);
+    static_assert(kCiChunk == 8, "index arithmetic below assumes chunks of 8 channels");
+
+    extern __shared__ __align__(16) unsigned char smem[];
+    float* sX = reinterpret_cast<float*>(smem);             // [kCiChunk][plane]
+    float* sW = reinterpret_cast<float*>(smem + a.off_sW);   // [kCiChunk][CO_BLOCK][kWSlots]
+    unsigned char* rawX = smem + a.off_rawX;                 // [2][rawX_bytes]
+    unsigned char* rawV = smem + a.off_rawV;                 // [2][CO_BLOCK][8*k*val_esize]
+    unsigned char* rawP = smem + a.off_rawP;                 // [2][CO_BLOCK][8]
+    int* tab_g = reinterpret_cast<int*>(smem + a.off_tab);   // global element offset per table entry, -1 = outside
     __shared__ uint16_t smask[256];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -85,12 +114,32 @@ __global__ void __launch_bounds__(kThreads, 1) conv3x3_alu_kernel(const Conv3Arg
     const int ox0 = tx * a.LX * PW, oy0 = ty * a.LY * PH;  // first output pixel of the tile
     const int ix0 = ox0 * S - 1, iy0 = oy0 * S - 1;        // input coordinate of staged element (0,0)
 
-    const int tile_elems = a.TH_in * a.TWP;
-    for (int e = tid; e < tile_elems; e += kThreads) {
-        const int r = e / a.TWP, c = e - r * a.TWP;
-        const int iy = iy0 + r, ix = ix0 + c;
-        const bool ok = c < a.TW_in && iy >= 0 && iy < a.H && ix >= 0 && ix < a.W;
-        tabG[e] = ok ? iy * a.W + ix : -1;
+    // ---- tables, built once per CTA
+    // X_SYNC / X_NHWC_VEC: one entry per staged element (r, c) of a channel plane, pitch TWP / TW_in;
+    //             tab_s = its offset in the fp32 plane.
+    // X_NCHW_VEC: one entry per raw vector (r, j); tab_g = offset of its first element in the channel
+    //             plane, tab_s = its row packed with the (biased) destination column of its first element,
+    //             which may lie left of the tile.
+    const int veq = a.vb / (int)sizeof(T);  // elements per activation vector (NCHW vector mode)
+    const int n_tab = a.xmode == X_SYNC ? a.TH_in * a.TWP : a.EV;
+    int* tab_s = tab_g + n_tab;
+    if (a.xmode == X_NCHW_VEC) {
+        const int nv = a.EV / a.TH_in;
+        for (int e = tid; e < n_tab; e += kThreads) {
+            const int r = e / nv, j = e - r * nv;
+            const int iy = iy0 + r, ix = ox0 * S - veq + j * veq;
+            tab_g[e] = (iy >= 0 && iy < a.H && ix >= 0 && ix < a.W) ? iy * a.W + ix : -1;
+            tab_s[e] = (r << 16) | (j * veq - (veq - 1) + 16);
+        }
+    } else {
+        const int pitch = a.xmode == X_SYNC ? a.TWP : a.TW_in;
+        for (int e = tid; e < n_tab; e += kThreads) {
+            const int r = e / pitch, c = e - r * pitch;
+            const int iy = iy0 + r, ix = ix0 + c;
+            const bool ok = c < a.TW_in && iy >= 0 && iy < a.H && ix >= 0 && ix < a.W;
+            tab_g[e] = ok ? iy * a.W + ix : -1;
+            tab_s[e] = r * a.TWP + c;
+        }
     }
     for (int p = tid; p < 256; p += kThreads) smask[p] = p < a.P ? a.masks[p] : 0;
 
@@ -104,30 +153,98 @@ __global__ void __launch_bounds__(kThreads, 1) conv3x3_alu_kernel(const Conv3Arg
 
     const T* __restrict__ xg = reinterpret_cast<const T*>(a.x);
     const size_t HW = (size_t)a.H * a.W;
+    const int vrow_bytes = 8 * a.k * a.val_esize;  // packed values of 8 consecutive channels of one filter
+    __syncthreads();                                // tables visible before the first issue
 
-    for (int ci0 = 0; ci0 < a.Cin; ci0 += kCiChunk) {
-        __syncthreads();  // previous chunk fully consumed (also orders tabG / smask on the first pass)
-        // ---- stage activations: fp32, zero where the tap falls outside the image
-        if (a.layout == RTOSS_NCHW) {
+    // ---- asynchronous part of staging chunk ci0 into raw buffer `buf`
+    auto issue = [&](int ci0, int buf) {
+        if (a.xmode == X_NCHW_VEC) {
+            const int ci = ci0 + warp;  // one warp per channel of the chunk
+            if (ci < a.Cin) {
+                const T* plane_ptr = xg + ((size_t)n * a.Cin + ci) * HW;
+                unsigned char* dst = rawX + (size_t)buf * a.rawX_bytes + (size_t)warp * a.EV * a.vb;
+                for (int e = lane; e < a.EV; e += 32) {
+                    const int g = tab_g[e];
+                    if (g >= 0) cp_async(dst + (size_t)e * a.vb, plane_ptr + g, a.vb);
+                }
+            }
+        } else if (a.xmode == X_NHWC_VEC) {
+            constexpr int VPP = 8 / VE16;  // 16-byte vectors per pixel for 8 channels
+            const T* img = xg + (size_t)n * HW * a.Cin + ci0;
+            unsigned char* dst = rawX + (size_t)buf * a.rawX_bytes;
+            for (int i = tid; i < a.EV * VPP; i += kThreads) {
+                const int e = i / VPP, h = i - e * VPP;
+                const int g = tab_g[e];
+                if (g >= 0) cp_async(dst + (size_t)i * 16, img + (size_t)g * a.Cin + h * VE16, 16);
+            }
+        }
+        if (a.w_async) {
+            const int nvw = vrow_bytes / 16;
+            unsigned char* dv = rawV + (size_t)buf * a.rawV_bytes;
+            for (int i = tid; i < CO_BLOCK * nvw; i += kThreads) {
+                const int col = i / nvw, j = i - col * nvw;
+                const int co = co0 + col;
+                if (co < a.Cout)
+                    cp_async(dv + (size_t)col * vrow_bytes + j * 16,
+                             reinterpret_cast<const unsigned char*>(a.val) +
+                                 ((size_t)co * a.Cin + ci0) * a.k * a.val_esize + j * 16, 16);
+            }
+            if (tid < CO_BLOCK && co0 + tid < a.Cout)
+                cp_async(rawP + (size_t)buf * CO_BLOCK * 8 + tid * 8, a.pid + (size_t)(co0 + tid) * a.Cin + ci0, 8);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+
+    // ---- conversion of chunk ci0 (raw buffer `buf`, or straight from global memory) into sX / sW
+    auto convert = [&](int ci0, int buf) {
+        if (a.xmode == X_NCHW_VEC) {
+            const int ci = ci0 + warp;
+            const unsigned char* src = rawX + (size_t)buf * a.rawX_bytes + (size_t)warp * a.EV * a.vb;
+            float* dst = sX + warp * a.plane;
+            for (int e = lane; e < a.EV; e += 32) {
+                const bool ok = tab_g[e] >= 0 && ci < a.Cin;
+                const int s = tab_s[e];
+                const int r = s >> 16, c0 = (s & 0xFFFF) - 16;  // destination row, column of element 0 (>= -(veq-1))
+                const T* rv = reinterpret_cast<const T*>(src + (size_t)e * a.vb);
+#pragma unroll
+                for (int q = 0; q < VE16; ++q) {
+                    if (q < veq) {
+                        const int c = c0 + q;
+                        if (c >= 0 && c < a.TWP) dst[r * a.TWP + c] = ok ? to_f32<T>(rv[q]) : 0.f;
+                    }
+                }
+            }
+        } else if (a.xmode == X_NHWC_VEC) {
+            const unsigned char* src = rawX + (size_t)buf * a.rawX_bytes;
+            for (int e = tid; e < a.EV; e += kThreads) {
+                const bool ok = tab_g[e] >= 0;
+                const int s = tab_s[e];
+                const T* rv = reinterpret_cast<const T*>(src + (size_t)e * (8 * sizeof(T)));
+#pragma unroll
+                for (int cl = 0; cl < 8; ++cl) sX[cl * a.plane + s] = ok ? to_f32<T>(rv[cl]) : 0.f;
+            }
+        } else if (a.layout == RTOSS_NCHW) {
+            const int tile_elems = a.TH_in * a.TWP;
             for (int cl = 0; cl < kCiChunk; ++cl) {
                 const int ci = ci0 + cl;
                 const T* plane_ptr = xg + ((size_t)n * a.Cin + (ci < a.Cin ? ci : 0)) * HW;
                 float* dst = sX + cl * a.plane;
                 for (int e = tid; e < tile_elems; e += kThreads) {
-                    const int g = tabG[e];
+                    const int g = tab_g[e];
                     dst[e] = (g >= 0 && ci < a.Cin) ? to_f32<T>(plane_ptr[g]) : 0.f;
                 }
             }
         } else {
+            const int tile_elems = a.TH_in * a.TWP;
             const T* img = xg + (size_t)n * HW * a.Cin;
             for (int i = tid; i < tile_elems * kCiChunk; i += kThreads) {
                 const int cl = i & (kCiChunk - 1), e = i >> 3;
                 const int ci = ci0 + cl;
-                const int g = tabG[e];
+                const int g = tab_g[e];
                 sX[cl * a.plane + e] = (g >= 0 && ci < a.Cin) ? to_f32<T>(img[(size_t)g * a.Cin + ci]) : 0.f;
             }
         }
-        // ---- stage weights: expand (pid, k values) to 9 slots + mask
+        // weights: expand (pid, k values) of each (filter, channel) of the chunk to 9 slots + mask
         for (int i = tid; i < CO_BLOCK * kCiChunk; i += kThreads) {
             const int cl = i % kCiChunk, col = i / kCiChunk;
             const int co = co0 + col, ci = ci0 + cl;
@@ -136,18 +253,36 @@ __global__ void __launch_bounds__(kThreads, 1) conv3x3_alu_kernel(const Conv3Arg
             for (int t = 0; t < 9; ++t) wv[t] = 0.f;
             unsigned m = 0;
             if (co < a.Cout && ci < a.Cin) {
-                const size_t kid = (size_t)co * a.Cin + ci;
-                m = smask[a.pid[kid]];
-                size_t j = kid * a.k;
+                if (a.w_async) {
+                    m = smask[rawP[(size_t)buf * CO_BLOCK * 8 + col * 8 + cl]];
+                    const void* vals = rawV + (size_t)buf * a.rawV_bytes + (size_t)col * vrow_bytes;
+                    int j = cl * a.k;
 #pragma unroll
-                for (int t = 0; t < 9; ++t)
-                    if (m & (1u << t)) wv[t] = load_val(a.val, j++, a.val_dtype);
+                    for (int t = 0; t < 9; ++t)
+                        if (m & (1u << t)) wv[t] = load_val(vals, j++, a.val_dtype);
+                } else {
+                    const size_t kid = (size_t)co * a.Cin + ci;
+                    m = smask[a.pid[kid]];
+                    size_t j = kid * a.k;
+#pragma unroll
+                    for (int t = 0; t < 9; ++t)
+                        if (m & (1u << t)) wv[t] = load_val(a.val, j++, a.val_dtype);
+                }
             }
             float4* dst = reinterpret_cast<float4*>(sW + ((size_t)cl * CO_BLOCK + col) * kWSlots);
             dst[0] = make_float4(wv[0], wv[1], wv[2], wv[3]);
             dst[1] = make_float4(wv[4], wv[5], wv[6], wv[7]);
             dst[2] = make_float4(wv[8], __uint_as_float(m), 0.f, 0.f);
         }
+    };
+
+    const int n_chunks = (a.Cin + kCiChunk - 1) / kCiChunk;
+    issue(0, 0);
+    for (int ch = 0; ch < n_chunks; ++ch) {
+        cp_async_wait_all();
+        __syncthreads();  // raw bytes of this chunk visible to all; everyone is done computing the previous chunk
+        if (ch + 1 < n_chunks) issue((ch + 1) * kCiChunk, (ch + 1) & 1);
+        convert(ch * kCiChunk, ch & 1);
         __syncthreads();
 
         // ---- compute
@@ -202,7 +337,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv3x3_alu_kernel(const Conv3Arg
                 T* row = yg + (((size_t)n * Cs + a.y_c_off + co) * a.Ho + oy) * a.Wo;
                 const bool vec = ((size_t)a.Wo * sizeof(T)) % 16 == 0 && ox_first + PW <= a.Wo && (PW * sizeof(T)) % 16 == 0;
                 if (vec) {
-                    T tmp[PW];
+                    __align__(16) T tmp[PW];
 #pragma unroll
                     for (int px = 0; px < PW; ++px) tmp[px] = from_f32<T>(activate(acc[c][py][px] + b, a.act));
                     const uint4* src = reinterpret_cast<const uint4*>(tmp);
@@ -246,22 +381,76 @@ void choose_lanes(int Ho, int Wo, int PH, int PW, int* LX, int* LY) {
         }
 }
 
+inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
 template <typename T, int S, int PH, int PW, int CO_T>
 int launch_variant(Conv3Args& a, cudaStream_t stream) {
+    constexpr int CO_BLOCK = kWarps * CO_T;
+    const int es = (int)sizeof(T);
     choose_lanes(a.Ho, a.Wo, PH, PW, &a.LX, &a.LY);
     a.tiles_x = (a.Wo + a.LX * PW - 1) / (a.LX * PW);
     a.tiles_y = (a.Ho + a.LY * PH - 1) / (a.LY * PH);
     a.TW_in = (a.LX * PW - 1) * S + 3;
     a.TH_in = (a.LY * PH - 1) * S + 3;
-    a.TWP = (a.TW_in + 3) / 4 * 4;
-    const int elems = a.TH_in * a.TWP;
-    a.plane = (elems + 31) / 32 * 32 + 4;
-    const size_t smem = sizeof(float) * ((size_t)kCiChunk * a.plane + (size_t)kCiChunk * kWarps * CO_T * kWSlots) +
-                        sizeof(int) * (size_t)elems;
+    a.TWP = round_up(a.TW_in, 4);
+    a.plane = round_up(a.TH_in * a.TWP, 32) + 4;
+
+    a.w_async = (a.Cin % 8 == 0) ? 1 : 0;
+    a.rawV_bytes = a.w_async ? CO_BLOCK * 8 * a.k * a.val_esize : 0;
+    const int fixed_bytes = (int)sizeof(float) * kCiChunk * (a.plane + CO_BLOCK * kWSlots) + 2 * a.rawV_bytes +
+                            (a.w_async ? 2 * CO_BLOCK * 8 : 0);
+    const int smem_cap = 200 * 1024;
+
+    // how the activations travel: cp.async where rows are aligned and the raw buffers fit, else plain loads
+    a.xmode = X_SYNC;
+    a.vb = 0;
+    a.EV = 0;
+    int n_tab = a.TH_in * a.TWP;
+    a.rawX_bytes = 0;
+    const bool x16 = (reinterpret_cast<uintptr_t>(a.x) & 15) == 0;
+    if (a.layout == RTOSS_NCHW && x16) {
+        const int row_bytes = a.W * es;
+        const int vb = row_bytes % 16 == 0 ? 16 : row_bytes % 8 == 0 ? 8 : row_bytes % 4 == 0 ? 4 : 0;
+        if (vb >= es && vb > 0) {
+            const int veq = vb / es;
+            const int nv = round_up(veq - 1 + a.TW_in, veq) / veq;
+            const int raw = round_up(kCiChunk * a.TH_in * nv * vb, 16);
+            if (fixed_bytes + 2 * raw + 8 * a.TH_in * nv <= smem_cap) {
+                a.xmode = X_NCHW_VEC;
+                a.vb = vb;
+                a.EV = a.TH_in * nv;
+                n_tab = a.EV;
+                a.rawX_bytes = raw;
+            }
+        }
+    } else if (a.layout == RTOSS_NHWC && x16 && a.Cin % 8 == 0) {
+        const int raw = round_up(a.TH_in * a.TW_in * 8 * es, 16);
+        if (fixed_bytes + 2 * raw + 8 * a.TH_in * a.TW_in <= smem_cap) {
+            a.xmode = X_NHWC_VEC;
+            a.vb = 16;
+            a.EV = a.TH_in * a.TW_in;
+            n_tab = a.EV;
+            a.rawX_bytes = raw;
+        }
+    }
+
+    int off = (int)sizeof(float) * kCiChunk * a.plane;
+    a.off_sW = off;
+    off += (int)sizeof(float) * kCiChunk * CO_BLOCK * kWSlots;
+    a.off_rawX = off;
+    off += 2 * a.rawX_bytes;
+    a.off_rawV = off;
+    off += 2 * a.rawV_bytes;
+    a.off_rawP = off;
+    off += a.w_async ? 2 * CO_BLOCK * 8 : 0;
+    a.off_tab = off;
+    off += 2 * (int)sizeof(int) * n_tab;
+    const size_t smem = (size_t)off;
+    if (smem > 220 * 1024) return (int)cudaErrorInvalidConfiguration;
     auto kern = conv3x3_alu_kernel<T, S, PH, PW, CO_T>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return (int)e;
-    dim3 grid((unsigned)((size_t)a.tiles_x * a.tiles_y * a.N), (unsigned)((a.Cout + kWarps * CO_T - 1) / (kWarps * CO_T)));
+    dim3 grid((unsigned)((size_t)a.tiles_x * a.tiles_y * a.N), (unsigned)((a.Cout + CO_BLOCK - 1) / CO_BLOCK));
     kern<<<grid, kThreads, smem, stream>>>(a);
     return (int)cudaGetLastError();
 }
@@ -285,6 +474,7 @@ int rtoss_launch_conv3x3(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     a.masks = p->masks_dev;
     a.bias = d->bias_dev;
     a.val_dtype = (int)p->dtype;
+    a.val_esize = (int)rtoss_dtype_size(p->dtype);
     a.N = d->N;
     a.Cin = p->Cin;
     a.Cout = p->Cout;

@@ -88,6 +88,11 @@ SHAPES_3x3 = [
     (3, 16, 16, 20, 20, 1, 9, "bf16", "silu", "nchw", True),    # k = 9: no pruning
     (1, 9, 5, 12, 100, 1, 5, "f32", "silu", "nchw", True),      # 5-entry patterns, wide image
     (1, 64, 64, 16, 16, 2, 1, "f16", "relu", "nchw", True),     # 1-entry patterns
+    (2, 16, 32, 25, 34, 1, 4, "bf16", "relu", "nchw", True),    # rows 68 bytes: 4-byte async copies
+    (1, 24, 32, 50, 68, 2, 4, "bf16", "relu", "nchw", True),    # rows 136 bytes: 8-byte async copies
+    (1, 8, 16, 11, 6, 1, 3, "f32", "none", "nchw", True),       # fp32 rows of 24 bytes
+    (1, 16, 24, 30, 22, 1, 4, "f32", "silu", "nhwc", True),     # fp32 NHWC, two 16-byte vectors per pixel
+    (1, 40, 36, 200, 272, 2, 4, "bf16", "relu", "nchw", False), # large image, stride 2, many tiles
 ]
 
 
