@@ -302,9 +302,17 @@ __global__ void __launch_bounds__(kThreads, 1) conv3x3_alu_kernel(const Conv3Arg
                 for (int c = (WIN_W / 4) * 4; c < WIN_W; ++c) win[r][c] = row[c];
             }
             const float4* wp = reinterpret_cast<const float4*>(sW + ((size_t)cl * CO_BLOCK + warp * CO_T) * kWSlots);
+            // the weights of filter c+1 are fetched before the FMAs of filter c, so the shared-memory
+            // latency is covered by arithmetic instead of being exposed at every filter
+            float4 n0 = wp[0], n1 = wp[1], n2 = wp[2];
 #pragma unroll
             for (int c = 0; c < CO_T; ++c) {
-                const float4 w0 = wp[c * 3], w1 = wp[c * 3 + 1], w2 = wp[c * 3 + 2];
+                const float4 w0 = n0, w1 = n1, w2 = n2;
+                if (c + 1 < CO_T) {
+                    n0 = wp[(c + 1) * 3];
+                    n1 = wp[(c + 1) * 3 + 1];
+                    n2 = wp[(c + 1) * 3 + 2];
+                }
                 const unsigned m = __float_as_uint(w2.y);
                 if (m & 0x001) fma_tap<S, PH, PW, 0, 0>(acc[c], win, w0.x);
                 if (m & 0x002) fma_tap<S, PH, PW, 0, 1>(acc[c], win, w0.y);
