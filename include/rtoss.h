@@ -53,6 +53,12 @@ typedef enum {
     RTOSS_PRESET_DENSE = 3    /* k = 9: the single all-taps mask (no pruning) */
 } rtoss_preset;
 
+typedef enum {
+    RTOSS_PATH_AUTO = 0,   /* tensor path where the call qualifies, FMA path otherwise */
+    RTOSS_PATH_FMA = 1,    /* gather of the k kept taps on the FP32 FMA pipes (any dtype, layout, stride) */
+    RTOSS_PATH_TENSOR = 2  /* masked dense implicit GEMM on tcgen05; RTOSS_ERR_UNSUPPORTED if the call does not qualify */
+} rtoss_path;
+
 typedef struct rtoss_ctx rtoss_ctx;       /* per-device state: error text, host-path workspace */
 typedef struct rtoss_packed rtoss_packed; /* one layer's pruned weights in packed form, on the device */
 
@@ -172,6 +178,7 @@ typedef struct {
     const float* bias_dev;  /* [Cout] fp32, or NULL */
     int y_channel_offset;   /* y may be a channel slice of a wider tensor: */
     int y_channel_stride;   /*   channels of that tensor, 0 = Cout */
+    rtoss_path path;        /* which kernel family runs the call */
 } rtoss_conv_desc;
 
 /* y[n,co,oy,ox] = act( bias[co] + sum_ci sum_{t in mask(pid[co,ci])}
@@ -191,6 +198,16 @@ rtoss_status rtoss_conv3x3_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const 
  * No padding; Ho = (H-1)/s+1.  Handle from rtoss_pack with ksize 1. */
 rtoss_status rtoss_conv1x1_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const void* x_dev, void* y_dev,
                                    const rtoss_conv_desc* desc, void* cuda_stream);
+
+/* The tensor path (RTOSS_PATH_TENSOR, or RTOSS_PATH_AUTO when it applies) takes: bf16 / fp16 NHWC,
+ * stride 1, io_dtype equal to the packed dtype, Cin a multiple of 8, Cout a multiple of 16 (of 128
+ * above 256), W + 2 <= 256, output channel offset and stride multiples of 8.  It multiplies the pruned
+ * taps as zeros on the tensor cores; results agree with the FMA path to fp32 summation order.
+ *
+ * Device-side waits of that path are bounded.  If one runs out, the kernel records a non-zero code in
+ * the context and returns; rtoss_device_status synchronises the device, reports the code
+ * (RTOSS_ERR_TIMEOUT when non-zero) and clears it. */
+rtoss_status rtoss_device_status(rtoss_ctx* ctx, int* code);
 
 /* Same convolutions with HOST buffers: copies x to the device, runs the
  * kernel for the handle's ksize, copies y back and waits for it.  x_host and

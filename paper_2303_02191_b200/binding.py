@@ -18,6 +18,7 @@ F32, BF16, F16 = 0, 1, 2
 NCHW, NHWC = 0, 1
 ACT_NONE, ACT_RELU, ACT_SILU = 0, 1, 2
 PRESET_ALL, PRESET_CONN4, PRESET_CENTRE8, PRESET_DENSE = 0, 1, 2, 3
+PATH_AUTO, PATH_FMA, PATH_TENSOR = 0, 1, 2
 DTYPE_NAMES = {"f32": F32, "bf16": BF16, "f16": F16}
 ACT_NAMES = {"none": ACT_NONE, "relu": ACT_RELU, "silu": ACT_SILU}
 
@@ -25,7 +26,7 @@ SYMBOLS = [
     "rtoss_create", "rtoss_destroy", "rtoss_status_string", "rtoss_last_error", "rtoss_pattern_preset",
     "rtoss_pattern_table_validate", "rtoss_group_layers", "rtoss_select_patterns", "rtoss_pack",
     "rtoss_packed_info_get", "rtoss_packed_export", "rtoss_packed_to_dense", "rtoss_packed_destroy",
-    "rtoss_conv3x3_pattern", "rtoss_conv1x1_pattern", "rtoss_conv_pattern_host",
+    "rtoss_conv3x3_pattern", "rtoss_conv1x1_pattern", "rtoss_conv_pattern_host", "rtoss_device_status",
 ]
 
 
@@ -49,7 +50,8 @@ class PackedInfo(ctypes.Structure):
 class ConvDesc(ctypes.Structure):
     _fields_ = [("N", ctypes.c_int), ("H", ctypes.c_int), ("W", ctypes.c_int), ("stride", ctypes.c_int),
                 ("layout", ctypes.c_int), ("io_dtype", ctypes.c_int), ("act", ctypes.c_int),
-                ("bias_dev", ctypes.c_void_p), ("y_channel_offset", ctypes.c_int), ("y_channel_stride", ctypes.c_int)]
+                ("bias_dev", ctypes.c_void_p), ("y_channel_offset", ctypes.c_int), ("y_channel_stride", ctypes.c_int),
+                ("path", ctypes.c_int)]
 
 
 def _load():
@@ -78,6 +80,7 @@ def _load():
     lib.rtoss_conv3x3_pattern.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ConvDesc), vp]
     lib.rtoss_conv1x1_pattern.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ConvDesc), vp]
     lib.rtoss_conv_pattern_host.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ConvDesc)]
+    lib.rtoss_device_status.argtypes = [vp, ctypes.POINTER(ci)]
     return lib
 
 
@@ -189,28 +192,38 @@ class Context:
                                    len(m), int(k), pid.data_ptr(), int(compute_dtype), ctypes.byref(h), _stream()))
         return into if into is not None else Packed(self, h)
 
-    def _desc(self, x_shape_nchw, stride, layout, io_dtype, act, bias, y_off, y_stride):
+    def _desc(self, x_shape_nchw, stride, layout, io_dtype, act, bias, y_off, y_stride, path=PATH_AUTO):
         N, _, H, W = x_shape_nchw
         return ConvDesc(int(N), int(H), int(W), int(stride), int(layout), int(io_dtype), int(act),
-                        bias.data_ptr() if bias is not None else None, int(y_off), int(y_stride))
+                        bias.data_ptr() if bias is not None else None, int(y_off), int(y_stride), int(path))
+
+    def rtoss_device_status(self):
+        """Synchronise the device and return the code a timed-out device wait left (0 = none)."""
+        code = ctypes.c_int(0)
+        st = lib.rtoss_device_status(self.h, ctypes.byref(code))
+        if st not in (OK, 7):
+            self._check(st)
+        return code.value
 
     def rtoss_conv3x3_pattern(self, packed, x, y, N, H, W, stride=1, layout=NCHW, act=ACT_NONE, bias=None,
-                              y_channel_offset=0, y_channel_stride=0):
-        d = self._desc((N, 0, H, W), stride, layout, _torch_dtype_code(x), act, bias, y_channel_offset, y_channel_stride)
+                              y_channel_offset=0, y_channel_stride=0, path=PATH_AUTO):
+        d = self._desc((N, 0, H, W), stride, layout, _torch_dtype_code(x), act, bias, y_channel_offset, y_channel_stride,
+                       path)
         self._check(lib.rtoss_conv3x3_pattern(self.h, packed.h, x.data_ptr(), y.data_ptr(), ctypes.byref(d), _stream()))
         return y
 
     def rtoss_conv1x1_pattern(self, packed, x, y, N, H, W, stride=1, layout=NCHW, act=ACT_NONE, bias=None,
-                              y_channel_offset=0, y_channel_stride=0):
-        d = self._desc((N, 0, H, W), stride, layout, _torch_dtype_code(x), act, bias, y_channel_offset, y_channel_stride)
+                              y_channel_offset=0, y_channel_stride=0, path=PATH_AUTO):
+        d = self._desc((N, 0, H, W), stride, layout, _torch_dtype_code(x), act, bias, y_channel_offset, y_channel_stride,
+                       path)
         self._check(lib.rtoss_conv1x1_pattern(self.h, packed.h, x.data_ptr(), y.data_ptr(), ctypes.byref(d), _stream()))
         return y
 
     def rtoss_conv_pattern_host(self, packed, x_host, y_host, N, H, W, stride=1, layout=NCHW, act=ACT_NONE, bias=None,
-                                y_channel_offset=0, y_channel_stride=0):
+                                y_channel_offset=0, y_channel_stride=0, path=PATH_AUTO):
         """x_host / y_host: CPU torch tensors (pinned or not); blocks until y_host is written."""
         d = self._desc((N, 0, H, W), stride, layout, _torch_dtype_code(x_host), act, bias, y_channel_offset,
-                       y_channel_stride)
+                       y_channel_stride, path)
         self._check(lib.rtoss_conv_pattern_host(self.h, packed.h, x_host.data_ptr(), y_host.data_ptr(), ctypes.byref(d)))
         return y_host
 

@@ -1,0 +1,497 @@
+// Tensor-core path of the pattern convolutions (bf16 / fp16, NHWC, stride 1).
+//
+// Per-kernel patterns cannot be compacted into a dense contraction (every
+// filter keeps different (channel, tap) positions), so this path evaluates the
+// convolution of Section II.B of arXiv 2303.02191 as a masked dense implicit
+// GEMM on the 5th-generation tensor cores: the pruned taps are multiplied as
+// zeros.  It performs 9/k times the non-zero FLOPs and is still several times
+// faster than the FMA-pipe gather for 16-bit data; the FMA path stays the one
+// for fp32 and for shapes this kernel does not take.
+//
+// GEMM view:  D[pixel, co] = sum over taps t and channels ci of
+//                            X[pixel shifted by t, ci] * Wt[t][co][ci]
+//   * A CTA owns TH output rows of one image (all columns) and N_T output
+//     channels.  The input rows it needs (with the one-pixel halo, zero-filled
+//     by TMA outside the image) are staged once per block of 64 channels as a
+//     flat list of "padded pixels", 128 bytes (64 channels) each, row pitch
+//     Wp = W + 2 pixels.  In that list the input pixel of tap (r, c) for output
+//     position p is at p + r*Wp + c: the A operand of every tap is the SAME
+//     shared-memory tile read from a different start row, so the halo tile is
+//     loaded once and used by all nine taps.  Output positions run over the
+//     padded pitch too; the two junk positions per row are computed and dropped.
+//   * M = 128 positions per MMA (nMB blocks per CTA), N = N_T filters, K = 16
+//     channels per instruction, accumulators in TMEM (nMB * N_T columns).
+//   * Weights are the dense-expanded form Wt[t][co][ci] that rtoss_pack builds
+//     next to the packed arrays; one TMA box per (tap, channel block).
+//   * Warp roles: warp 0 issues TMA, warp 1 issues tcgen05.mma and owns the
+//     TMEM allocation, warps 2..5 run the epilogue (tcgen05.ld, bias,
+//     activation, rounding, 16-byte NHWC stores).
+//   * Every mbarrier wait is bounded; a wait that runs out records a code in
+//     the context's status word and the CTA leaves through the normal exit
+//     (TMEM is always released).
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include "conv_common.cuh"
+
+namespace {
+
+using namespace rtoss_dev;
+
+constexpr int kTcThreads = 192;
+constexpr int kKBlock = 64;       // channels per staged block: 128 bytes of bf16 / fp16
+constexpr int kRowBytes = 128;    // one padded pixel, one channel block
+constexpr long long kWaitCycles = 2000000000LL;  // about one second
+
+struct TcArgs {
+    void* y;
+    const float* bias;
+    int* status;
+    int N, H, W, Cin, Cout;
+    int Wp, TH, taps, pad;       // padded pitch, output rows per CTA, 9 or 1, 1 or 0
+    int nMB, N_T, ncb;           // M blocks per CTA, filters per CTA, channel blocks
+    int tiles_y, co_tiles;
+    int a_stage_bytes, b_stage_bytes, NB;
+    unsigned a_tx_bytes, b_tx_bytes;
+    int act, y_c_off, y_c_stride, is_bf16;
+    unsigned idesc;
+    int tmem_cols;
+};
+
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait on a phase parity; false when the limit ran out.
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
+    const long long t0 = clock64();
+    for (;;) {
+        unsigned done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if (clock64() - t0 > kWaitCycles) return false;
+    }
+}
+
+__device__ __forceinline__ void tma_load_4d(unsigned dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            unsigned bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(unsigned dst, const CUtensorMap* map, int c0, int c1, int c2, unsigned bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor, K-major operand with 128-byte swizzle: rows of 128 bytes, groups
+// of 8 rows 1024 bytes apart.  The start may be any 16-byte aligned address inside a tile whose base
+// is 1024-byte aligned; the row phase of the start (address bits 7..9) goes into the base-offset field.
+__device__ __forceinline__ unsigned long long make_sw128_desc(unsigned addr) {
+    unsigned long long d = 0;
+    d |= (unsigned long long)((addr & 0x3FFFFu) >> 4);        // start address
+    d |= (unsigned long long)1 << 16;                          // leading byte offset (unused for swizzled K-major)
+    d |= (unsigned long long)(1024 >> 4) << 32;                // stride byte offset: 8 rows * 128 bytes
+    d |= (unsigned long long)1 << 46;                          // descriptor version of this architecture
+    d |= (unsigned long long)((addr >> 7) & 7u) << 49;         // base offset
+    d |= (unsigned long long)2 << 61;                          // 128-byte swizzle
+    return d;
+}
+
+__device__ __forceinline__ void umma_f16(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc,
+                                         unsigned idesc, unsigned accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrive on an mbarrier once all tcgen05.mma issued so far by this thread have completed.
+__device__ __forceinline__ void umma_commit(unsigned bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(unsigned taddr, unsigned (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+
+template <typename T>
+__device__ __forceinline__ unsigned pack2(float a, float b);
+template <>
+__device__ __forceinline__ unsigned pack2<__nv_bfloat16>(float a, float b) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<unsigned*>(&v);
+}
+template <>
+__device__ __forceinline__ unsigned pack2<__half>(float a, float b) {
+    __half2 v = __floats2half2_rn(a, b);
+    return *reinterpret_cast<unsigned*>(&v);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kTcThreads, 1)
+conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcArgs a) {
+    extern __shared__ unsigned char smem_dyn[];
+    // tiles need 1024-byte alignment for the 128-byte swizzle pattern
+    const unsigned base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    const unsigned sA = base;                                        // [2][a_stage_bytes]
+    const unsigned sB = sA + 2u * a.a_stage_bytes;                   // [NB][b_stage_bytes]
+    const unsigned sBar = sB + (unsigned)a.NB * a.b_stage_bytes;     // barriers, 8 bytes each
+    const unsigned bar_fullA = sBar, bar_emptyA = sBar + 16, bar_fullB = sBar + 32;
+    const unsigned bar_emptyB = bar_fullB + 8u * a.NB, bar_dfull = bar_emptyB + 8u * a.NB;
+    const unsigned s_tmem_ptr = bar_dfull + 8;
+    unsigned char* gen_base = smem_dyn + (base - smem_u32(smem_dyn));
+    volatile unsigned* tmem_ptr_gen = reinterpret_cast<volatile unsigned*>(gen_base + (s_tmem_ptr - base));
+    float* s_bias = reinterpret_cast<float*>(gen_base + (s_tmem_ptr + 8 - base));  // [N_T]
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int bid = blockIdx.x;
+    const int cot = bid % a.co_tiles;
+    bid /= a.co_tiles;
+    const int ty = bid % a.tiles_y;
+    const int n = bid / a.tiles_y;
+    const int y0 = ty * a.TH, co0 = cot * a.N_T;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_fullA + 8 * i, 1);
+            mbar_init(bar_emptyA + 8 * i, 1);
+        }
+        for (int i = 0; i < a.NB; ++i) {
+            mbar_init(bar_fullB + 8 * i, 1);
+            mbar_init(bar_emptyB + 8 * i, 1);
+        }
+        mbar_init(bar_dfull, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+    }
+    for (int i = threadIdx.x; i < a.N_T; i += kTcThreads) s_bias[i] = (a.bias && co0 + i < a.Cout) ? a.bias[co0 + i] : 0.f;
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s_tmem_ptr), "r"(a.tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const unsigned tmem_base = *tmem_ptr_gen;
+
+    if (warp == 0) {
+        // ---------------- TMA producer
+        if (lane == 0) {
+            bool ok = true;
+            for (int cb = 0; cb < a.ncb && ok; ++cb) {
+                const int sa = cb & 1;
+                ok = mbar_wait(bar_emptyA + 8 * sa, ((cb >> 1) & 1) ^ 1);
+                if (!ok) break;
+                mbar_expect_tx(bar_fullA + 8 * sa, a.a_tx_bytes);
+                tma_load_4d(sA + sa * a.a_stage_bytes, &tmA, cb * kKBlock, -a.pad, y0 - a.pad, n, bar_fullA + 8 * sa);
+                for (int t = 0; t < a.taps; ++t) {
+                    const int it = cb * a.taps + t, sb = it % a.NB;
+                    ok = mbar_wait(bar_emptyB + 8 * sb, ((it / a.NB) & 1) ^ 1);
+                    if (!ok) break;
+                    mbar_expect_tx(bar_fullB + 8 * sb, a.b_tx_bytes);
+                    tma_load_3d(sB + sb * a.b_stage_bytes, &tmB, cb * kKBlock, co0, t, bar_fullB + 8 * sb);
+                }
+            }
+            if (!ok) atomicExch(a.status, 1);
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer
+        if (lane == 0) {
+            bool ok = true;
+            for (int cb = 0; cb < a.ncb && ok; ++cb) {
+                const int sa = cb & 1;
+                ok = mbar_wait(bar_fullA + 8 * sa, (cb >> 1) & 1);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const unsigned a_tile = sA + sa * a.a_stage_bytes;
+                for (int t = 0; t < a.taps; ++t) {
+                    const int it = cb * a.taps + t, sb = it % a.NB;
+                    ok = mbar_wait(bar_fullB + 8 * sb, (it / a.NB) & 1);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const int shift = a.taps == 9 ? (t / 3) * a.Wp + (t % 3) : 0;
+                    const unsigned b_tile = sB + sb * a.b_stage_bytes;
+                    for (int mb = 0; mb < a.nMB; ++mb) {
+                        const unsigned a_rows = a_tile + (unsigned)(mb * 128 + shift) * kRowBytes;
+#pragma unroll
+                        for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
+                            umma_f16(tmem_base + (unsigned)(mb * a.N_T), make_sw128_desc(a_rows + k4 * 32),
+                                     make_sw128_desc(b_tile + k4 * 32), a.idesc, (cb | t | k4) != 0);
+                        }
+                    }
+                    umma_commit(bar_emptyB + 8 * sb);  // this weight slot may be refilled once the MMAs have read it
+                }
+                if (ok) umma_commit(bar_emptyA + 8 * sa);
+            }
+            if (ok) umma_commit(bar_dfull);
+            else atomicExch(a.status, 2);
+        }
+    } else {
+        // ---------------- epilogue: TMEM -> registers -> bias / activation -> NHWC global
+        const int quarter = warp & 3;  // TMEM lanes a warp may read: 32 * (warp id mod 4)
+        const bool ok = mbar_wait(bar_dfull, 0);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok) {
+            T* __restrict__ yg = reinterpret_cast<T*>(a.y);
+            for (int mb = 0; mb < a.nMB; ++mb) {
+                const int p = mb * 128 + quarter * 32 + lane;
+                const int oyl = p / a.Wp, ox = p - oyl * a.Wp;
+                const int oy = y0 + oyl;
+                const bool valid = oyl < a.TH && ox < a.W && oy < a.H;
+                T* dst = yg + (((size_t)n * a.H + oy) * a.W + ox) * a.y_c_stride + a.y_c_off + co0;
+                for (int c0 = 0; c0 < a.N_T; c0 += 32) {
+                    unsigned r[32];
+                    tmem_ld32(tmem_base + ((unsigned)(quarter * 32) << 16) + (unsigned)(mb * a.N_T + c0), r);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (valid) {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {  // 8 filters = 16 bytes per store
+                            if (co0 + c0 + v * 8 < a.Cout) {
+                                uint4 o;
+                                unsigned* ow = reinterpret_cast<unsigned*>(&o);
+#pragma unroll
+                                for (int h = 0; h < 4; ++h) {
+                                    const int c = c0 + v * 8 + h * 2;
+                                    const float f0 = activate(__uint_as_float(r[v * 8 + h * 2]) + s_bias[c], a.act);
+                                    const float f1 = activate(__uint_as_float(r[v * 8 + h * 2 + 1]) + s_bias[c + 1], a.act);
+                                    ow[h] = pack2<T>(f0, f1);
+                                }
+                                *reinterpret_cast<uint4*>(dst + c0 + v * 8) = o;
+                            }
+                        }
+                    }
+                }
+            }
+        } else if (lane == 0) {
+            atomicExch(a.status, 3);
+        }
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(a.tmem_cols) : "memory");
+    }
+}
+
+// Dense-expanded weights for the tensor path: out[t][co][ci] = kept value or +0.
+template <typename V>
+__global__ void expand_taps_kernel(const V* __restrict__ val, const uint8_t* __restrict__ pid,
+                                   const uint16_t* __restrict__ masks, int k, int Cout, int Cin, V* __restrict__ out) {
+    const size_t n = (size_t)Cout * Cin;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const unsigned m = masks[pid[i]];
+        size_t j = i * k;
+#pragma unroll
+        for (int t = 0; t < 9; ++t) {
+            V v = from_f32<V>(0.f);
+            if (m & (1u << t)) v = val[j++];
+            out[(size_t)t * n + i] = v;
+        }
+    }
+}
+
+PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
+    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(p);
+    }
+    return fn;
+}
+
+inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
+struct TcPlan {
+    int TH, nMB, N_T, NB, a_rows, smem;
+};
+
+// Choose rows per CTA: fill the 128-row MMA blocks well, few wasted rows at the image bottom, fit
+// TMEM (nMB*N_T <= 512 columns) and shared memory.
+bool plan_tc(int H, int W, int Wp, int pad, int N_T, TcPlan* out) {
+    const int smem_cap = 224 * 1024;
+    double best = -1;
+    for (int th = 1; th <= H && th + 2 * pad <= 256; ++th) {
+        const int m_total = th * Wp;
+        const int nmb = (m_total + 127) / 128;
+        if ((nmb - 1) * N_T + round_up(N_T, 32) > 512 || nmb > 4) break;
+        const int a_rows = round_up(nmb * 128 + 2 * pad * Wp + 2 * pad, 8);
+        const int a_bytes = a_rows * kRowBytes;
+        const int b_bytes = N_T * kRowBytes;
+        int nb = (smem_cap - 2048 - 2 * a_bytes - 4 * (N_T + 32)) / b_bytes;
+        if (nb < 2) continue;
+        if (nb > 6) nb = 6;
+        const double eff = (double)(th * W) / (nmb * 128) * H / (double)((H + th - 1) / th * th);
+        const double score = eff + 1e-4 * th;
+        if (score > best) {
+            best = score;
+            out->TH = th;
+            out->nMB = nmb;
+            out->N_T = N_T;
+            out->NB = nb;
+            out->a_rows = a_rows;
+            out->smem = 2 * a_bytes + nb * b_bytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + 4 * (N_T + 32);
+        }
+    }
+    return best > 0;
+}
+
+}  // namespace
+
+bool rtoss_tc_weights_eligible(const rtoss_packed* p) {
+    return (p->dtype == RTOSS_BF16 || p->dtype == RTOSS_F16) && p->Cin % 8 == 0 && p->Cout % 16 == 0;
+}
+
+int rtoss_launch_expand_taps(const rtoss_packed* p, void* out, void* stream) {
+    const size_t n = (size_t)p->Cout * p->Cin;
+    const int threads = 256;
+    size_t g = (n + threads - 1) / threads;
+    if (g > 148 * 8) g = 148 * 8;
+    if (p->dtype == RTOSS_BF16)
+        expand_taps_kernel<__nv_bfloat16><<<(int)g, threads, 0, (cudaStream_t)stream>>>(
+            (const __nv_bfloat16*)p->val, p->pid, p->masks_dev, p->k, p->Cout, p->Cin, (__nv_bfloat16*)out);
+    else
+        expand_taps_kernel<__half><<<(int)g, threads, 0, (cudaStream_t)stream>>>((const __half*)p->val, p->pid, p->masks_dev,
+                                                                                 p->k, p->Cout, p->Cin, (__half*)out);
+    return (int)cudaGetLastError();
+}
+
+// Filters per CTA: the whole layer up to 128, else tiles of 128 (or the whole layer up to 256 when
+// it is not a multiple of 128); 0 = no tiling this kernel takes.
+static int tc_pick_nt(int Cout) {
+    if (Cout <= 128) return Cout;
+    if (Cout % 128 == 0) return 128;
+    return Cout <= 256 ? Cout : 0;
+}
+
+// Can this call run on the tensor path?
+bool rtoss_tc_eligible(const rtoss_packed* p, const rtoss_conv_desc* d, const void* x, const void* y) {
+    if (!p->wtc || !rtoss_tc_weights_eligible(p)) return false;
+    if (d->layout != RTOSS_NHWC || d->stride != 1 || (int)d->io_dtype != (int)p->dtype) return false;
+    const int pad = p->ksize == 3 ? 1 : 0;
+    if (d->W + 2 * pad > 256) return false;
+    const int cs = d->y_channel_stride ? d->y_channel_stride : p->Cout;
+    if (cs % 8 != 0 || d->y_channel_offset % 8 != 0) return false;  // 16-byte output stores
+    if ((reinterpret_cast<uintptr_t>(x) & 15) || (reinterpret_cast<uintptr_t>(y) & 15)) return false;
+    if (!encode_fn()) return false;
+    const int N_T = tc_pick_nt(p->Cout);
+    if (N_T == 0) return false;
+    TcPlan plan;
+    return plan_tc(d->H, d->W, d->W + 2 * pad, pad, N_T, &plan);
+}
+
+int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y, const rtoss_conv_desc* d,
+                         void* stream) {
+    const int pad = p->ksize == 3 ? 1 : 0;
+    const int taps = p->ksize == 3 ? 9 : 1;
+    const int Wp = d->W + 2 * pad;
+    const int N_T = tc_pick_nt(p->Cout);
+    if (N_T == 0) return (int)cudaErrorInvalidConfiguration;
+    TcPlan plan;
+    if (!plan_tc(d->H, d->W, Wp, pad, N_T, &plan)) return (int)cudaErrorInvalidConfiguration;
+
+    TcArgs a;
+    a.y = y;
+    a.bias = d->bias_dev;
+    a.status = ctx->dev_status;
+    a.N = d->N;
+    a.H = d->H;
+    a.W = d->W;
+    a.Cin = p->Cin;
+    a.Cout = p->Cout;
+    a.Wp = Wp;
+    a.TH = plan.TH;
+    a.taps = taps;
+    a.pad = pad;
+    a.nMB = plan.nMB;
+    a.N_T = N_T;
+    a.ncb = (p->Cin + kKBlock - 1) / kKBlock;
+    a.tiles_y = (d->H + plan.TH - 1) / plan.TH;
+    a.co_tiles = (p->Cout + N_T - 1) / N_T;
+    a.a_stage_bytes = plan.a_rows * kRowBytes;
+    a.b_stage_bytes = N_T * kRowBytes;
+    a.NB = plan.NB;
+    a.a_tx_bytes = (unsigned)(kKBlock * 2 * Wp * (plan.TH + 2 * pad));
+    a.b_tx_bytes = (unsigned)(kKBlock * 2 * N_T);
+    a.act = (int)d->act;
+    a.y_c_off = d->y_channel_offset;
+    a.y_c_stride = d->y_channel_stride ? d->y_channel_stride : p->Cout;
+    a.is_bf16 = p->dtype == RTOSS_BF16;
+    // instruction descriptor: fp32 accumulate, A and B of the io type, both K-major, N/8 and M/16
+    const unsigned fmt = a.is_bf16 ? 1u : 0u;
+    a.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((unsigned)(N_T >> 3) << 17) | ((unsigned)(128 >> 4) << 24);
+    const int cols = (plan.nMB - 1) * N_T + round_up(N_T, 32);  // the epilogue reads 32 columns at a time
+    int alloc = 32;
+    while (alloc < cols) alloc <<= 1;
+    a.tmem_cols = alloc;
+
+    PFN_cuTensorMapEncodeTiled_v12000 enc = encode_fn();
+    if (!enc) return (int)cudaErrorNotSupported;
+    const CUtensorMapDataType dt = a.is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+    CUtensorMap tmA, tmB;
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)p->Cin, (cuuint64_t)d->W, (cuuint64_t)d->H, (cuuint64_t)d->N};
+        cuuint64_t strides[3] = {(cuuint64_t)p->Cin * 2, (cuuint64_t)d->W * p->Cin * 2, (cuuint64_t)d->H * d->W * p->Cin * 2};
+        cuuint32_t box[4] = {(cuuint32_t)kKBlock, (cuuint32_t)Wp, (cuuint32_t)(plan.TH + 2 * pad), 1};
+        cuuint32_t es[4] = {1, 1, 1, 1};
+        CUresult r = enc(&tmA, dt, 4, const_cast<void*>(x), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return (int)cudaErrorInvalidValue;
+    }
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)p->Cin, (cuuint64_t)p->Cout, (cuuint64_t)taps};
+        cuuint64_t strides[2] = {(cuuint64_t)p->Cin * 2, (cuuint64_t)p->Cout * p->Cin * 2};
+        cuuint32_t box[3] = {(cuuint32_t)kKBlock, (cuuint32_t)N_T, 1};
+        cuuint32_t es[3] = {1, 1, 1};
+        CUresult r = enc(&tmB, dt, 3, p->wtc, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return (int)cudaErrorInvalidValue;
+    }
+    const size_t smem = (size_t)plan.smem;
+    dim3 grid((unsigned)((size_t)d->N * a.tiles_y * a.co_tiles));
+    cudaError_t e;
+    if (a.is_bf16) {
+        auto kern = conv_tc_kernel<__nv_bfloat16>;
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return (int)e;
+        kern<<<grid, kTcThreads, smem, (cudaStream_t)stream>>>(tmA, tmB, a);
+    } else {
+        auto kern = conv_tc_kernel<__half>;
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return (int)e;
+        kern<<<grid, kTcThreads, smem, (cudaStream_t)stream>>>(tmA, tmB, a);
+    }
+    return (int)cudaGetLastError();
+}

@@ -59,8 +59,9 @@ rtoss_status check_conv(rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
     }
     if (d->N < 1 || d->H < 1 || d->W < 1 || (d->stride != 1 && d->stride != 2) || !dtype_ok(d->io_dtype) ||
         (d->layout != RTOSS_NCHW && d->layout != RTOSS_NHWC) ||
-        (d->act != RTOSS_ACT_NONE && d->act != RTOSS_ACT_RELU && d->act != RTOSS_ACT_SILU)) {
-        set_err(ctx, "conv", "bad descriptor (N,H,W >= 1; stride 1|2; dtype; layout; act)");
+        (d->act != RTOSS_ACT_NONE && d->act != RTOSS_ACT_RELU && d->act != RTOSS_ACT_SILU) ||
+        (d->path != RTOSS_PATH_AUTO && d->path != RTOSS_PATH_FMA && d->path != RTOSS_PATH_TENSOR)) {
+        set_err(ctx, "conv", "bad descriptor (N,H,W >= 1; stride 1|2; dtype; layout; act; path)");
         return RTOSS_ERR_INVALID_ARG;
     }
     const int cs = d->y_channel_stride ? d->y_channel_stride : p->Cout;
@@ -77,6 +78,21 @@ rtoss_status check_conv(rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
         return RTOSS_ERR_ALIGNMENT;
     }
     return RTOSS_OK;
+}
+
+// Pick the kernel family for one convolution call and launch it.  Returns the CUDA error code of
+// the launch; *st is set when the requested path cannot take the call.
+int dispatch_conv(rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y, const rtoss_conv_desc* d, void* stream,
+                  rtoss_status* st) {
+    *st = RTOSS_OK;
+    const bool tc_ok = d->path != RTOSS_PATH_FMA && rtoss_tc_eligible(p, d, x, y);
+    if (d->path == RTOSS_PATH_TENSOR && !tc_ok) {
+        set_err(ctx, "conv", "the tensor path does not take this call (see rtoss.h for its conditions)");
+        *st = RTOSS_ERR_UNSUPPORTED;
+        return 0;
+    }
+    if (tc_ok) return rtoss_launch_conv_tc(ctx, p, x, y, d, stream);
+    return p->ksize == 3 ? rtoss_launch_conv3x3(ctx, p, x, y, d, stream) : rtoss_launch_conv1x1(ctx, p, x, y, d, stream);
 }
 
 }  // namespace
@@ -97,6 +113,17 @@ rtoss_status rtoss_create(int device, rtoss_ctx** out) {
     memset(c, 0, sizeof(*c));
     c->device = device;
     c->sm_count = prop.multiProcessorCount;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaSetDevice(device);
+    cudaError_t se = cudaMalloc((void**)&c->dev_status, sizeof(int));
+    if (se == cudaSuccess) se = cudaMemset(c->dev_status, 0, sizeof(int));
+    cudaSetDevice(prev);
+    if (se != cudaSuccess) {
+        cudaGetLastError();
+        delete c;
+        return RTOSS_ERR_ALLOC;
+    }
     *out = c;
     return RTOSS_OK;
 }
@@ -112,6 +139,7 @@ void rtoss_destroy(rtoss_ctx* ctx) {
     }
     if (ctx->ws_x) cudaFree(ctx->ws_x);
     if (ctx->ws_y) cudaFree(ctx->ws_y);
+    if (ctx->dev_status) cudaFree(ctx->dev_status);
     cudaSetDevice(prev);
     delete ctx;
 }
@@ -196,6 +224,8 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
             e = cudaMalloc((void**)&p->perm, sizeof(uint32_t) * (size_t)Cin * Cout);
             if (e == cudaSuccess) e = cudaMalloc((void**)&p->bucket_off, sizeof(uint32_t) * (size_t)Cin * (P + 1));
         }
+        if (e == cudaSuccess && rtoss_tc_weights_eligible(p))
+            e = cudaMalloc(&p->wtc, (size_t)(ksize == 3 ? 9 : 1) * Cout * Cin * rtoss_dtype_size(compute_dtype));
         if (e != cudaSuccess) {
             cudaGetLastError();
             rtoss_packed_destroy(p);
@@ -213,6 +243,9 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
                                       compute_dtype, cuda_stream);
     if (e == cudaSuccess && !le && ksize == 3)
         le = rtoss_launch_pack_order(pid_dev, Cout, Cin, P, p->perm, p->bucket_off, cuda_stream);
+    // the tensor path reads dense-expanded weights: built here from the packed arrays just written
+    if (e == cudaSuccess && !le && p->wtc)
+        le = ksize == 3 ? rtoss_launch_expand_taps(p, p->wtc, cuda_stream) : rtoss_launch_to_dense(p, p->wtc, cuda_stream);
     if (e != cudaSuccess || le) {
         rtoss_status r = cuda_fail(ctx, "pack launch", e != cudaSuccess ? (int)e : le);
         if (!reuse) rtoss_packed_destroy(p);
@@ -272,6 +305,7 @@ void rtoss_packed_destroy(rtoss_packed* p) {
     if (p->perm) cudaFree(p->perm);
     if (p->bucket_off) cudaFree(p->bucket_off);
     if (p->masks_dev) cudaFree(p->masks_dev);
+    if (p->wtc) cudaFree(p->wtc);
     cudaSetDevice(prev);
     delete p;
 }
@@ -281,7 +315,8 @@ rtoss_status rtoss_conv3x3_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const 
     rtoss_status st = check_conv(ctx, p, x_dev, y_dev, desc, 3, true);
     if (st != RTOSS_OK) return st;
     cudaSetDevice(ctx->device);
-    int e = rtoss_launch_conv3x3(ctx, p, x_dev, y_dev, desc, cuda_stream);
+    int e = dispatch_conv(ctx, p, x_dev, y_dev, desc, cuda_stream, &st);
+    if (st != RTOSS_OK) return st;
     return e ? cuda_fail(ctx, "conv3x3 launch", e) : RTOSS_OK;
 }
 
@@ -290,8 +325,23 @@ rtoss_status rtoss_conv1x1_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const 
     rtoss_status st = check_conv(ctx, p, x_dev, y_dev, desc, 1, true);
     if (st != RTOSS_OK) return st;
     cudaSetDevice(ctx->device);
-    int e = rtoss_launch_conv1x1(ctx, p, x_dev, y_dev, desc, cuda_stream);
+    int e = dispatch_conv(ctx, p, x_dev, y_dev, desc, cuda_stream, &st);
+    if (st != RTOSS_OK) return st;
     return e ? cuda_fail(ctx, "conv1x1 launch", e) : RTOSS_OK;
+}
+
+rtoss_status rtoss_device_status(rtoss_ctx* ctx, int* code) {
+    if (!ctx || !code) return RTOSS_ERR_INVALID_ARG;
+    cudaSetDevice(ctx->device);
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(code, ctx->dev_status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(ctx, "device status", (int)e);
+    if (*code != 0) {
+        cudaMemset(ctx->dev_status, 0, sizeof(int));
+        set_err(ctx, "device status", "a bounded wait in a tensor-path kernel ran out");
+        return RTOSS_ERR_TIMEOUT;
+    }
+    return RTOSS_OK;
 }
 
 rtoss_status rtoss_conv_pattern_host(rtoss_ctx* ctx, const rtoss_packed* p, const void* x_host, void* y_host,
@@ -340,8 +390,8 @@ rtoss_status rtoss_conv_pattern_host(rtoss_ctx* ctx, const rtoss_packed* p, cons
     // a channel slice leaves the other channels of y untouched: bring the caller's y over first
     if (e == cudaSuccess && slice) e = cudaMemcpyAsync(ctx->ws_y, y_host, yb, cudaMemcpyHostToDevice, s);
     if (e != cudaSuccess) return cuda_fail(ctx, "host path copy in", (int)e);
-    int le = p->ksize == 3 ? rtoss_launch_conv3x3(ctx, p, ctx->ws_x, ctx->ws_y, desc, s)
-                           : rtoss_launch_conv1x1(ctx, p, ctx->ws_x, ctx->ws_y, desc, s);
+    int le = dispatch_conv(ctx, p, ctx->ws_x, ctx->ws_y, desc, s, &st);
+    if (st != RTOSS_OK) return st;
     if (le) return cuda_fail(ctx, "host path launch", le);
     e = cudaMemcpyAsync(y_host, ctx->ws_y, yb, cudaMemcpyDeviceToHost, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);

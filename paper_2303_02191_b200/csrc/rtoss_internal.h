@@ -17,6 +17,7 @@ struct rtoss_ctx {
     void* ws_y;
     size_t ws_y_bytes;
     void* h_stream;  // cudaStream_t owned by the context, used by the host-buffer path
+    int* dev_status;  // device word: 0, or the code of a bounded device-side wait that ran out
 };
 
 struct rtoss_packed {
@@ -29,6 +30,7 @@ struct rtoss_packed {
     uint32_t* perm;        // [Cin*Cout]      (ksize 3)
     uint32_t* bucket_off;  // [Cin*(P+1)]     (ksize 3)
     uint16_t* masks_dev;   // [256]
+    void* wtc;             // tensor path: dense-expanded weights [taps][Cout][Cin] in dtype, or NULL
     uint16_t masks[256];
 };
 
@@ -52,6 +54,12 @@ int rtoss_launch_to_dense(const rtoss_packed* p, void* w_out, void* stream);
 int rtoss_launch_conv3x3(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y,
                          const rtoss_conv_desc* d, void* stream);
 int rtoss_launch_conv1x1(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y,
+                         const rtoss_conv_desc* d, void* stream);
+// tensor path (conv_tc.cu)
+bool rtoss_tc_weights_eligible(const rtoss_packed* p);
+int rtoss_launch_expand_taps(const rtoss_packed* p, void* out, void* stream);
+bool rtoss_tc_eligible(const rtoss_packed* p, const rtoss_conv_desc* d, const void* x, const void* y);
+int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y,
                          const rtoss_conv_desc* d, void* stream);
 
 #endif

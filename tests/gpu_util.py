@@ -67,7 +67,7 @@ def val_as_f32(exported_val, dt):
     return t.float().numpy()
 
 
-def run_conv(packed, ksize, x, dt, stride, act, bias, layout="nchw", y_off=0, y_stride=0, host=False):
+def run_conv(packed, ksize, x, dt, stride, act, bias, layout="nchw", y_off=0, y_stride=0, host=False, path=0):
     """x numpy fp32 NCHW (already rounded to dt) -> y numpy fp32 NCHW."""
     c = ctx()
     N, Cin, H, W = x.shape
@@ -81,12 +81,12 @@ def run_conv(packed, ksize, x, dt, stride, act, bias, layout="nchw", y_off=0, y_
         xh = to_dev(x, dt, layout).cpu().pin_memory()
         yh = torch.full(yshape, 7.0, dtype=TORCH_DT[dt]).pin_memory()
         torch.cuda.synchronize()
-        c.rtoss_conv_pattern_host(packed, xh, yh, N, H, W, stride, lay, rt.ACT_NAMES[act], bd, y_off, y_stride)
+        c.rtoss_conv_pattern_host(packed, xh, yh, N, H, W, stride, lay, rt.ACT_NAMES[act], bd, y_off, y_stride, path)
         return from_dev(yh, layout)
     xd = to_dev(x, dt, layout)
     yd = torch.full(yshape, 7.0, dtype=TORCH_DT[dt], device="cuda")
     fn = c.rtoss_conv3x3_pattern if ksize == 3 else c.rtoss_conv1x1_pattern
-    fn(packed, xd, yd, N, H, W, stride, lay, rt.ACT_NAMES[act], bd, y_off, y_stride)
+    fn(packed, xd, yd, N, H, W, stride, lay, rt.ACT_NAMES[act], bd, y_off, y_stride, path)
     torch.cuda.synchronize()
     return from_dev(yd, layout)
 
@@ -98,7 +98,7 @@ def oracle_conv(ksize, x, wd, bias, stride, act, dt):
 
 
 def check_layer(seed, tid, ksize, N, Cin, Cout, H, W, stride, k, masks, dt, act="none", layout="nchw",
-                use_bias=True, host=False):
+                use_bias=True, host=False, path=0):
     """Full parity of one layer: pattern ids and packed arrays bit-exact, outputs within TOL[dt]."""
     x = synth.round_like(synth.activations(seed, tid, N, Cin, H, W), dt)
     w = synth.kaiming_weights(seed, tid, Cout, Cin, ksize)
@@ -111,7 +111,7 @@ def check_layer(seed, tid, ksize, N, Cin, Cout, H, W, stride, k, masks, dt, act=
     assert np.array_equal(val_as_f32(ex["val"], dt).view(np.uint32), arrays["val"].view(np.uint32)), "packed values differ"
     if ksize == 3:
         assert np.array_equal(ex["perm"], arrays["perm"]) and np.array_equal(ex["bucket_off"], arrays["bucket_off"])
-    y = run_conv(packed, ksize, x, dt, stride, act, b, layout, host=host)
+    y = run_conv(packed, ksize, x, dt, stride, act, b, layout, host=host, path=path)
     ref = oracle_conv(ksize, x, wd, b, stride, act, dt)
     err = orc.rel_err(y, ref)
     assert y.shape == ref.shape

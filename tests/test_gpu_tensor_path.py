@@ -1,0 +1,114 @@
+"""GPU parity of the tensor-core path (tcgen05 masked dense implicit GEMM, bf16 / fp16 NHWC) against
+the CPU oracle, and agreement with the FMA path on the same inputs."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    from oracle import rtoss_oracle as orc
+    from paper_2303_02191_b200 import binding as rt
+    from paper_2303_02191_b200 import synth
+    import gpu_util as gu
+
+
+def _table(k):
+    if k == 4:
+        return orc.pattern_preset(4, orc.PRESET_CENTRE8)
+    if k == 9:
+        return orc.pattern_preset(9, orc.PRESET_DENSE)
+    return orc.pattern_preset(k, orc.PRESET_CONN4)
+
+
+def _no_timeout():
+    assert gu.ctx().rtoss_device_status() == 0, "a device-side wait of the tensor path ran out"
+
+
+def test_tensor_path_smallest_case():
+    """One CTA, one channel block: the first thing to run after any change to the kernel."""
+    gu.check_layer(20, 1, 3, 1, 64, 64, 8, 8, 1, 4, _table(4), "bf16", "none", "nhwc", use_bias=False, path=rt.PATH_TENSOR)
+    _no_timeout()
+
+
+CASES = [
+    # ksize, N, Cin, Cout, H, W, k, dt, act
+    (3, 1, 128, 128, 80, 80, 3, "bf16", "silu"),      # the 128-channel layer, one image
+    (3, 2, 64, 64, 40, 40, 4, "bf16", "silu"),
+    (3, 1, 32, 64, 20, 20, 4, "bf16", "relu"),        # half-filled channel block
+    (3, 1, 72, 48, 13, 17, 2, "f16", "none"),         # ragged channel block, N_T not a multiple of 32, odd size
+    (3, 1, 256, 256, 20, 20, 4, "bf16", "silu"),      # two filter tiles
+    (3, 1, 64, 512, 7, 9, 4, "bf16", "relu"),         # four filter tiles, tiny image
+    (3, 2, 128, 16, 25, 34, 9, "bf16", "none"),       # dense table, narrow N
+    (3, 1, 64, 64, 1, 1, 4, "bf16", "none"),          # single pixel
+    (3, 1, 64, 32, 3, 200, 3, "f16", "silu"),         # wide image
+    (1, 1, 256, 128, 80, 80, 3, "bf16", "silu"),      # the 256->128 1x1 layer, one image
+    (1, 2, 64, 32, 20, 20, 4, "bf16", "silu"),
+    (1, 1, 1024, 512, 20, 20, 4, "bf16", "silu"),
+    (1, 1, 40, 80, 13, 17, 2, "f16", "relu"),
+    (1, 1, 512, 2048, 25, 34, 4, "bf16", "relu"),
+]
+
+
+@pytest.mark.parametrize("case", CASES, ids=lambda c: "-".join(str(v) for v in c))
+def test_tensor_path_against_oracle(case):
+    ks, N, Cin, Cout, H, W, k, dt, act = case
+    gu.check_layer(21, 400 + Cin + Cout, ks, N, Cin, Cout, H, W, 1, k, _table(k), dt, act, "nhwc", path=rt.PATH_TENSOR)
+    _no_timeout()
+
+
+@pytest.mark.parametrize("ksize", [3, 1])
+def test_tensor_and_fma_paths_agree(ksize):
+    masks = _table(4)
+    N, Cin, Cout, H, W = 2, 128, 128, 30, 30
+    x = synth.round_like(synth.activations(22, ksize, N, Cin, H, W), "bf16")
+    w = synth.kaiming_weights(22, ksize, Cout, Cin, ksize)
+    b = synth.bias(22, ksize, Cout)
+    _, packed = gu.select_pack(w, ksize, masks, 4, "bf16")
+    y_t = gu.run_conv(packed, ksize, x, "bf16", 1, "silu", b, "nhwc", path=rt.PATH_TENSOR)
+    y_f = gu.run_conv(packed, ksize, x, "bf16", 1, "silu", b, "nhwc", path=rt.PATH_FMA)
+    y_a = gu.run_conv(packed, ksize, x, "bf16", 1, "silu", b, "nhwc", path=rt.PATH_AUTO)
+    assert np.array_equal(y_a, y_t)                      # auto picks the tensor path here
+    assert orc.rel_err(y_t, y_f) <= 1e-2                 # same fp32 accumulation, different order: one bf16 ulp at most
+    assert (y_t != y_f).mean() < 0.05
+    _no_timeout()
+    packed.close()
+
+
+def test_tensor_path_channel_slice_and_batch_sampled():
+    masks = _table(3)
+    N, Cin, Cout, H, W = 8, 128, 128, 80, 80
+    x = synth.round_like(synth.activations(23, 1, N, Cin, H, W), "bf16")
+    w = synth.kaiming_weights(23, 1, Cout, Cin, 3)
+    b = synth.bias(23, 1, Cout)
+    _, packed = gu.select_pack(w, 3, masks, 3, "bf16")
+    _, wd, _ = gu.oracle_weights(w, 3, masks, 3, "bf16")
+    y = gu.run_conv(packed, 3, x, "bf16", 1, "silu", b, "nhwc", y_off=64, y_stride=256, path=rt.PATH_TENSOR)
+    assert (y[:, :64] == 7.0).all() and (y[:, 192:] == 7.0).all()
+    rng = np.random.default_rng(7)
+    npts = 4000
+    idx = np.stack([rng.integers(0, N, npts), rng.integers(0, Cout, npts), rng.integers(0, H, npts),
+                    rng.integers(0, W, npts)], axis=1).astype(np.int32)
+    idx[:4] = [[0, 0, 0, 0], [0, 0, 0, W - 1], [N - 1, Cout - 1, H - 1, W - 1], [N - 1, 0, H - 1, 0]]
+    ref = orc.conv_points(3, x, wd, b, 1, orc.ACT_SILU, orc.DT_BF16, idx)
+    got = y[idx[:, 0], 64 + idx[:, 1], idx[:, 2], idx[:, 3]]
+    rms = float(np.sqrt(np.mean(ref.astype(np.float64) ** 2)))
+    assert np.max(np.abs(got - ref) / np.maximum(np.abs(ref), rms)) <= 2e-2
+    _no_timeout()
+    packed.close()
+
+
+def test_tensor_path_refuses_what_it_cannot_take():
+    masks = _table(4)
+    w = synth.kaiming_weights(24, 1, 64, 64, 3)
+    _, packed = gu.select_pack(w, 3, masks, 4, "bf16")
+    x = synth.round_like(synth.activations(24, 1, 1, 64, 8, 8), "bf16")
+    with pytest.raises(rt.RtossError) as e:                                  # NCHW is not taken by the tensor path
+        gu.run_conv(packed, 3, x, "bf16", 1, "none", None, "nchw", path=rt.PATH_TENSOR)
+    assert e.value.status == 3
+    with pytest.raises(rt.RtossError) as e:                                  # nor stride 2
+        gu.run_conv(packed, 3, x, "bf16", 2, "none", None, "nhwc", path=rt.PATH_TENSOR)
+    assert e.value.status == 3
+    y = gu.run_conv(packed, 3, x, "bf16", 2, "none", None, "nhwc", path=rt.PATH_AUTO)   # auto falls back to FMA
+    assert np.isfinite(y).all()
+    packed.close()
