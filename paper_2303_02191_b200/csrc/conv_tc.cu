@@ -99,14 +99,15 @@ __device__ __forceinline__ void tma_load_3d(unsigned dst, const CUtensorMap* map
 
 // Shared-memory matrix descriptor, K-major operand with 128-byte swizzle: rows of 128 bytes, groups
 // of 8 rows 1024 bytes apart.  The start may be any 16-byte aligned address inside a tile whose base
-// is 1024-byte aligned; the row phase of the start (address bits 7..9) goes into the base-offset field.
+// is 1024-byte aligned: the swizzle is a function of the absolute shared-memory address, the same
+// function TMA applied when it wrote the tile, so a start in the middle of an 8-row group (a tap
+// shift) or 32 bytes into a row (a K step) needs no correction (base-offset field 0).
 __device__ __forceinline__ unsigned long long make_sw128_desc(unsigned addr) {
     unsigned long long d = 0;
     d |= (unsigned long long)((addr & 0x3FFFFu) >> 4);        // start address
     d |= (unsigned long long)1 << 16;                          // leading byte offset (unused for swizzled K-major)
     d |= (unsigned long long)(1024 >> 4) << 32;                // stride byte offset: 8 rows * 128 bytes
     d |= (unsigned long long)1 << 46;                          // descriptor version of this architecture
-    d |= (unsigned long long)((addr >> 7) & 7u) << 49;         // base offset
     d |= (unsigned long long)2 << 61;                          // 128-byte swizzle
     return d;
 }
