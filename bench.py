@@ -50,10 +50,10 @@ def read_peaks():
     if os.path.exists(path):
         try:
             d = json.load(open(path))
-            return float(d["hbm_gbs"]), "measured"
+            return float(d["hbm_gbs"]), float(d["bf16_tflops_sustained"]), "measured"
         except Exception:
             pass
-    return 6650.0, "fallback"
+    return 6650.0, 1400.0, "fallback"
 
 
 class ClockSampler(threading.Thread):
@@ -211,6 +211,8 @@ def run_gpu(args):
     elem = 4 if dtype == "f32" else 2
     cdt = rt.DTYPE_NAMES[dtype]
     preset_of = {"centre8": rt.PRESET_CENTRE8, "conn4": rt.PRESET_CONN4}
+    # 16-bit activations travel NHWC (what the tensor path takes), fp32 NCHW
+    layout = rt.NCHW if (dtype == "f32" or args.layout == "nchw") else rt.NHWC
 
     # ---- resident inputs (replicas: every rank holds its own batch and weights; no data-path collective)
     weights, L_state = {}, []
@@ -224,9 +226,13 @@ def run_gpu(args):
             weights[L["wid"]] = dict(w=w, b=b, pid=pid, packed=None, masks=masks, k=k, ksize=L["ksize"])
         Ho, Wo = synth.out_hw(L["H"], L["W"], L["stride"])
         xh = torch.from_numpy(synth.activations(rank, len(L_state), N, L["cin"], L["H"], L["W"])).to(tdt[dtype])
-        st = dict(L=L, k=k, x=xh.to(dev), y=torch.empty(N, L["cout"], Ho, Wo, dtype=tdt[dtype], device=dev),
-                  xh=xh.pin_memory(), yh=torch.empty(N, L["cout"], Ho, Wo, dtype=tdt[dtype]).pin_memory(),
-                  Ho=Ho, Wo=Wo, wt=weights[L["wid"]])
+        yshape = (N, L["cout"], Ho, Wo)
+        if layout == rt.NHWC:
+            xh = xh.permute(0, 2, 3, 1).contiguous()
+            yshape = (N, Ho, Wo, L["cout"])
+        st = dict(L=L, k=k, x=xh.to(dev), y=torch.empty(yshape, dtype=tdt[dtype], device=dev),
+                  xh=xh.pin_memory(), yh=torch.empty(yshape, dtype=tdt[dtype]).pin_memory(),
+                  Ho=Ho, Wo=Wo, wt=weights[L["wid"]], path=rt.PATH_FMA)
         L_state.append(st)
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)   # larger than the 126 MB L2
 
@@ -243,7 +249,8 @@ def run_gpu(args):
         fn = ctx.rtoss_conv3x3_pattern if L["ksize"] == 3 else ctx.rtoss_conv1x1_pattern
         if ev:
             ev[0].record()
-        fn(st["wt"]["packed"], st["x"], st["y"], N, L["H"], L["W"], L["stride"], rt.NCHW, rt.ACT_NAMES[L["act"]], st["wt"]["b"])
+        fn(st["wt"]["packed"], st["x"], st["y"], N, L["H"], L["W"], L["stride"], layout, rt.ACT_NAMES[L["act"]], st["wt"]["b"],
+           path=st["path"])
         if ev:
             ev[1].record()
 
@@ -258,6 +265,20 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    # which kernel family takes each layer: the tensor path where the call qualifies, else the FMA path
+    prune_weights()
+    for st in L_state:
+        if args.path != "fma":
+            try:
+                st["path"] = rt.PATH_TENSOR
+                conv(st)
+            except rt.RtossError as err:
+                if err.status != 3:
+                    raise
+                st["path"] = rt.PATH_FMA
+    torch.cuda.synchronize()
+    if ctx.rtoss_device_status() != 0:
+        raise SystemExit("a device-side wait of the tensor path ran out")
     for _ in range(max(args.warmup, 3)):
         step()
         flush.zero_()
@@ -286,7 +307,7 @@ def run_gpu(args):
     e2e_steps = max(3, min(args.steps, 20))
     for st in L_state[:1]:
         ctx.rtoss_conv_pattern_host(st["wt"]["packed"], st["xh"], st["yh"], N, st["L"]["H"], st["L"]["W"], st["L"]["stride"],
-                                    rt.NCHW, rt.ACT_NAMES[st["L"]["act"]], st["wt"]["b"])
+                                    layout, rt.ACT_NAMES[st["L"]["act"]], st["wt"]["b"], path=st["path"])
     barrier()
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
@@ -294,8 +315,8 @@ def run_gpu(args):
         torch.cuda.synchronize()
         for st in L_state:
             L = st["L"]
-            ctx.rtoss_conv_pattern_host(st["wt"]["packed"], st["xh"], st["yh"], N, L["H"], L["W"], L["stride"], rt.NCHW,
-                                        rt.ACT_NAMES[L["act"]], st["wt"]["b"])
+            ctx.rtoss_conv_pattern_host(st["wt"]["packed"], st["xh"], st["yh"], N, L["H"], L["W"], L["stride"], layout,
+                                        rt.ACT_NAMES[L["act"]], st["wt"]["b"], path=st["path"])
     torch.cuda.synchronize()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
     h2d = sum(st["xh"].numel() * elem for st in L_state)
@@ -312,18 +333,22 @@ def run_gpu(args):
         flops = [synth.layer_nnz_flops(st["L"], N, st["k"]) for st in L_state]
         bytes_ = [synth.layer_bytes(st["L"], N, st["k"], elem) for st in L_state]
         top = int(np.argmax(conv_ms))
-        hbm_peak, peak_kind = read_peaks()
+        hbm_peak, tc_peak, peak_kind = read_peaks()
         t_top = conv_ms[top] * 1e-3
-        alu_t, hbm_t = flops[top] / (ALU_PEAK_TFLOPS * 1e12), bytes_[top] / (hbm_peak * 1e9)
-        if alu_t >= hbm_t:
-            roof = {"bound": "alu", "achieved": flops[top] / t_top / 1e12, "peak": ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
-                    "peak_kind": "derived: 148 SM x 128 FMA lanes x 2 x 1.965 GHz"}
+        on_tc = L_state[top]["path"] == rt.PATH_TENSOR
+        pipe_peak = tc_peak if on_tc else ALU_PEAK_TFLOPS          # TFLOP/s of the pipe the kernel uses
+        pipe_t, hbm_t = flops[top] / (pipe_peak * 1e12), bytes_[top] / (hbm_peak * 1e9)
+        if pipe_t >= hbm_t:
+            roof = {"bound": "tensor" if on_tc else "alu", "achieved": flops[top] / t_top / 1e12, "peak": pipe_peak,
+                    "unit": "TFLOP/s",
+                    "peak_kind": ("of %s (bf16 cuBLAS, sustained)" % peak_kind) if on_tc
+                    else "derived: 148 SM x 128 FMA lanes x 2 x 1.965 GHz"}
         else:
             roof = {"bound": "hbm", "achieved": bytes_[top] / t_top / 1e9, "peak": hbm_peak, "unit": "GB/s",
                     "peak_kind": "of " + peak_kind}
         roof["frac"] = roof["achieved"] / roof["peak"]
         roof["traffic"] = None
-        roof["kernel"] = L_state[top]["L"]["name"] + " k=%d" % L_state[top]["k"]
+        roof["kernel"] = ("conv_tc_kernel " if on_tc else "conv_alu_kernel ") + L_state[top]["L"]["name"] + " k=%d" % L_state[top]["k"]
         roof["kernel_ms"] = float(conv_ms[top])
         roof["nnz_flop_per_launch"] = flops[top]
         roof["algorithmic_bytes_per_launch"] = bytes_[top]
@@ -331,8 +356,10 @@ def run_gpu(args):
             "metric": "pattern-sparse conv images/sec", "value": value, "unit": "images/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
-            "config": {"workload": args.workload, "batch": N, "layout": "NCHW", "l2": "flushed between steps (256 MB write)",
-                       "layers": len(L_state), "multi_gpu": "replicas only"},
+            "config": {"workload": args.workload, "batch": N, "layout": "NHWC" if layout == rt.NHWC else "NCHW",
+                       "l2": "flushed between steps (256 MB write)", "layers": len(L_state), "multi_gpu": "replicas only",
+                       "tensor_path_layers": sum(1 for st in L_state if st["path"] == rt.PATH_TENSOR),
+                       "fma_path_layers": sum(1 for st in L_state if st["path"] == rt.PATH_FMA)},
             "nnz_gflops_per_s": sum(flops) / (ms_per_step * 1e-3) / 1e9 * world,
             "conv_ms": [float(v) for v in conv_ms] if len(conv_ms) <= 8 else None,
             "conv_ms_sum": float(conv_ms.sum()),
@@ -362,6 +389,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="layer128")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--path", default="auto", choices=["auto", "fma"], help="fma: keep every layer on the FMA path")
+    ap.add_argument("--layout", default="auto", choices=["auto", "nchw"], help="nchw: NCHW activations also for 16-bit types")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
