@@ -24,8 +24,10 @@
 //   * Weights are the dense-expanded form Wt[t][co][ci] that rtoss_pack builds
 //     next to the packed arrays; one TMA box per (tap, channel block).
 //   * Warp roles: warp 0 issues TMA, warp 1 issues tcgen05.mma and owns the
-//     TMEM allocation, warps 2..5 run the epilogue (tcgen05.ld, bias,
-//     activation, rounding, 16-byte NHWC stores).
+//     TMEM allocation, warps 2..9 run the epilogue (tcgen05.ld, bias,
+//     activation, rounding, 16-byte NHWC stores).  Where shared memory and
+//     TMEM allow, two CTAs share an SM so that one CTA's epilogue runs under
+//     the other's MMAs.
 //   * Every mbarrier wait is bounded; a wait that runs out records a code in
 //     the context's status word and the CTA leaves through the normal exit
 //     (TMEM is always released).
@@ -38,7 +40,7 @@ namespace {
 
 using namespace rtoss_dev;
 
-constexpr int kTcThreads = 192;
+constexpr int kTcThreads = 320;    // TMA warp, MMA warp, eight epilogue warps
 constexpr int kKBlock = 64;       // channels per staged block: 128 bytes of bf16 / fp16
 constexpr int kRowBytes = 128;    // one padded pixel, one channel block
 constexpr long long kWaitCycles = 2000000000LL;  // about one second
@@ -51,7 +53,7 @@ struct TcArgs {
     int Wp, TH, taps, pad;       // padded pitch, output rows per CTA, 9 or 1, 1 or 0
     int nMB, N_T, ncb;           // M blocks per CTA, filters per CTA, channel blocks
     int tiles_y, co_tiles;
-    int a_stage_bytes, b_stage_bytes, NB;
+    int a_stage_bytes, b_stage_bytes, NA, NB;  // stage sizes, activation stages (1 or 2), weight slots
     unsigned a_tx_bytes, b_tx_bytes;
     int act, y_c_off, y_c_stride, is_bf16;
     unsigned idesc;
@@ -139,6 +141,14 @@ __device__ __forceinline__ void tmem_ld32(unsigned taddr, unsigned (&r)[32]) {
         : "memory");
 }
 
+// Epilogue activation for 16-bit outputs: SiLU through the fast exponential and reciprocal (error far
+// below half an ulp of bf16 / fp16).
+__device__ __forceinline__ float activate16(float v, int act) {
+    if (act == RTOSS_ACT_RELU) return fmaxf(v, 0.f);
+    if (act == RTOSS_ACT_SILU) return __fdividef(v, 1.f + __expf(-v));
+    return v;
+}
+
 template <typename T>
 __device__ __forceinline__ unsigned pack2(float a, float b);
 template <>
@@ -153,13 +163,13 @@ __device__ __forceinline__ unsigned pack2<__half>(float a, float b) {
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcThreads, 2)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcArgs a) {
     extern __shared__ unsigned char smem_dyn[];
     // tiles need 1024-byte alignment for the 128-byte swizzle pattern
     const unsigned base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
-    const unsigned sA = base;                                        // [2][a_stage_bytes]
-    const unsigned sB = sA + 2u * a.a_stage_bytes;                   // [NB][b_stage_bytes]
+    const unsigned sA = base;                                        // [NA][a_stage_bytes]
+    const unsigned sB = sA + (unsigned)a.NA * a.a_stage_bytes;       // [NB][b_stage_bytes]
     const unsigned sBar = sB + (unsigned)a.NB * a.b_stage_bytes;     // barriers, 8 bytes each
     const unsigned bar_fullA = sBar, bar_emptyA = sBar + 16, bar_fullB = sBar + 32;
     const unsigned bar_emptyB = bar_fullB + 8u * a.NB, bar_dfull = bar_emptyB + 8u * a.NB;
@@ -206,8 +216,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (lane == 0) {
             bool ok = true;
             for (int cb = 0; cb < a.ncb && ok; ++cb) {
-                const int sa = cb & 1;
-                ok = mbar_wait(bar_emptyA + 8 * sa, ((cb >> 1) & 1) ^ 1);
+                const int sa = cb % a.NA;
+                ok = mbar_wait(bar_emptyA + 8 * sa, ((cb / a.NA) & 1) ^ 1);
                 if (!ok) break;
                 mbar_expect_tx(bar_fullA + 8 * sa, a.a_tx_bytes);
                 tma_load_4d(sA + sa * a.a_stage_bytes, &tmA, cb * kKBlock, -a.pad, y0 - a.pad, n, bar_fullA + 8 * sa);
@@ -226,8 +236,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (lane == 0) {
             bool ok = true;
             for (int cb = 0; cb < a.ncb && ok; ++cb) {
-                const int sa = cb & 1;
-                ok = mbar_wait(bar_fullA + 8 * sa, (cb >> 1) & 1);
+                const int sa = cb % a.NA;
+                ok = mbar_wait(bar_fullA + 8 * sa, (cb / a.NA) & 1);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const unsigned a_tile = sA + sa * a.a_stage_bytes;
@@ -255,7 +265,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
     } else {
         // ---------------- epilogue: TMEM -> registers -> bias / activation -> NHWC global
-        const int quarter = warp & 3;  // TMEM lanes a warp may read: 32 * (warp id mod 4)
+        const int quarter = warp & 3;      // TMEM lanes a warp may read: 32 * (warp id mod 4)
+        const int half = (warp - 2) >> 2;  // two warps share a lane quarter and alternate 32-column chunks
         const bool ok = mbar_wait(bar_dfull, 0);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (ok) {
@@ -266,7 +277,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int oy = y0 + oyl;
                 const bool valid = oyl < a.TH && ox < a.W && oy < a.H;
                 T* dst = yg + (((size_t)n * a.H + oy) * a.W + ox) * a.y_c_stride + a.y_c_off + co0;
-                for (int c0 = 0; c0 < a.N_T; c0 += 32) {
+                for (int c0 = half * 32; c0 < a.N_T; c0 += 64) {
                     unsigned r[32];
                     tmem_ld32(tmem_base + ((unsigned)(quarter * 32) << 16) + (unsigned)(mb * a.N_T + c0), r);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -279,8 +290,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                                 for (int h = 0; h < 4; ++h) {
                                     const int c = c0 + v * 8 + h * 2;
-                                    const float f0 = activate(__uint_as_float(r[v * 8 + h * 2]) + s_bias[c], a.act);
-                                    const float f1 = activate(__uint_as_float(r[v * 8 + h * 2 + 1]) + s_bias[c + 1], a.act);
+                                    const float f0 = activate16(__uint_as_float(r[v * 8 + h * 2]) + s_bias[c], a.act);
+                                    const float f1 = activate16(__uint_as_float(r[v * 8 + h * 2 + 1]) + s_bias[c + 1], a.act);
                                     ow[h] = pack2<T>(f0, f1);
                                 }
                                 *reinterpret_cast<uint4*>(dst + c0 + v * 8) = o;
@@ -336,34 +347,43 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 struct TcPlan {
-    int TH, nMB, N_T, NB, a_rows, smem;
+    int TH, nMB, N_T, NA, NB, a_rows, smem;
 };
 
-// Choose rows per CTA: fill the 128-row MMA blocks well, few wasted rows at the image bottom, fit
-// TMEM (nMB*N_T <= 512 columns) and shared memory.
+// Choose rows per CTA.  Two shapes are tried for every TH: "shared" (one activation stage, at most
+// 256 TMEM columns, at most half an SM's shared memory, so that two CTAs are co-resident and one's
+// epilogue runs under the other's MMAs) and "alone" (two activation stages, the whole SM).  Score:
+// how full the 128-row MMA blocks are, how few rows are wasted at the image bottom, with a bonus
+// for the shared shape.
 bool plan_tc(int H, int W, int Wp, int pad, int N_T, TcPlan* out) {
-    const int smem_cap = 224 * 1024;
+    const int b_bytes = N_T * kRowBytes;
+    const int fixed = 1024 /*alignment slack*/ + 256 /*barriers*/ + 4 * (N_T + 32);
     double best = -1;
     for (int th = 1; th <= H && th + 2 * pad <= 256; ++th) {
-        const int m_total = th * Wp;
-        const int nmb = (m_total + 127) / 128;
-        if ((nmb - 1) * N_T + round_up(N_T, 32) > 512 || nmb > 4) break;
+        const int nmb = (th * Wp + 127) / 128;
+        const int cols = (nmb - 1) * N_T + round_up(N_T, 32);
+        if (cols > 512 || nmb > 4) break;
         const int a_rows = round_up(nmb * 128 + 2 * pad * Wp + 2 * pad, 8);
         const int a_bytes = a_rows * kRowBytes;
-        const int b_bytes = N_T * kRowBytes;
-        int nb = (smem_cap - 2048 - 2 * a_bytes - 4 * (N_T + 32)) / b_bytes;
-        if (nb < 2) continue;
-        if (nb > 6) nb = 6;
         const double eff = (double)(th * W) / (nmb * 128) * H / (double)((H + th - 1) / th * th);
-        const double score = eff + 1e-4 * th;
-        if (score > best) {
-            best = score;
-            out->TH = th;
-            out->nMB = nmb;
-            out->N_T = N_T;
-            out->NB = nb;
-            out->a_rows = a_rows;
-            out->smem = 2 * a_bytes + nb * b_bytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + 4 * (N_T + 32);
+        for (int shared = 1; shared >= 0; --shared) {
+            const int cap = shared ? 113 * 1024 : 226 * 1024;
+            const int na = shared ? 1 : 2;
+            if (shared && cols > 256) continue;
+            int nb = (cap - fixed - na * a_bytes) / b_bytes;
+            if (nb < (shared ? 3 : 2)) continue;
+            if (nb > 6) nb = 6;
+            const double score = eff * (shared ? 1.0 : 0.75) + 1e-4 * th;
+            if (score > best) {
+                best = score;
+                out->TH = th;
+                out->nMB = nmb;
+                out->N_T = N_T;
+                out->NA = na;
+                out->NB = nb;
+                out->a_rows = a_rows;
+                out->smem = na * a_bytes + nb * b_bytes + fixed;
+            }
         }
     }
     return best > 0;
@@ -443,6 +463,7 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     a.co_tiles = (p->Cout + N_T - 1) / N_T;
     a.a_stage_bytes = plan.a_rows * kRowBytes;
     a.b_stage_bytes = N_T * kRowBytes;
+    a.NA = plan.NA;
     a.NB = plan.NB;
     a.a_tx_bytes = (unsigned)(kKBlock * 2 * Wp * (plan.TH + 2 * pad));
     a.b_tx_bytes = (unsigned)(kKBlock * 2 * N_T);
