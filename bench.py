@@ -284,22 +284,56 @@ def run_gpu(args):
         flush.zero_()
     barrier()
 
+    # The step is launch-bound when driven call by call from Python (about twenty small launches for
+    # ~100 us of GPU work), so the timed region replays it as ONE CUDA graph, as a deployment would.
+    graph = None
+    if args.graph:
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                step()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                launches_per_step = step()
+            graph.replay()
+            torch.cuda.synchronize()
+        except Exception as err:  # keep measuring, say so in the line
+            sys.stderr.write("graph capture failed, timing eager launches: %r\n" % (err,))
+            graph = None
+            torch.cuda.synchronize()
     sampler = ClockSampler(physical_gpu_index(local_rank))
     sampler.start()
     step_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    conv_ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in L_state]
-               for _ in range(args.steps)]
     launches = 0
     barrier()
     for s in range(args.steps):
         flush.zero_()                       # L2 flush between timed iterations, outside the step's events
         step_ev[s][0].record()
-        launches += step(conv_ev[s])
+        if graph is not None:
+            graph.replay()
+            launches += launches_per_step
+        else:
+            launches += step()
         step_ev[s][1].record()
     barrier()
-    clocks = sampler.stop()
     step_ms = np.array([a.elapsed_time(b) for a, b in step_ev])
     total_ms = float(step_ms.sum())
+
+    # Per-kernel durations for the roofline: the same K steps again, launched one by one, every convolution
+    # between its own pair of events.  The 256 MB flush write queued right before each launch both empties
+    # L2 and keeps the GPU busy while the host enqueues the launch, so the interval is the kernel alone.
+    conv_ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in L_state]
+               for _ in range(args.steps)]
+    for s in range(args.steps):
+        prune_weights()
+        for i, st in enumerate(L_state):
+            flush.zero_()
+            conv(st, conv_ev[s][i])
+    barrier()
+    clocks = sampler.stop()
     conv_ms = np.array([[a.elapsed_time(b) for a, b in row] for row in conv_ev]).mean(axis=0)
 
     # ---- end to end through the host-buffer entry point (pinned host tensors, copies inside the timed region)
@@ -358,6 +392,7 @@ def run_gpu(args):
             "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
             "config": {"workload": args.workload, "batch": N, "layout": "NHWC" if layout == rt.NHWC else "NCHW",
                        "l2": "flushed between steps (256 MB write)", "layers": len(L_state), "multi_gpu": "replicas only",
+                       "launch": "one CUDA graph per step" if graph is not None else "eager",
                        "tensor_path_layers": sum(1 for st in L_state if st["path"] == rt.PATH_TENSOR),
                        "fma_path_layers": sum(1 for st in L_state if st["path"] == rt.PATH_FMA)},
             "nnz_gflops_per_s": sum(flops) / (ms_per_step * 1e-3) / 1e9 * world,
@@ -389,6 +424,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="layer128")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--no-graph", dest="graph", action="store_false", help="time eager launches instead of a CUDA graph")
     ap.add_argument("--path", default="auto", choices=["auto", "fma"], help="fma: keep every layer on the FMA path")
     ap.add_argument("--layout", default="auto", choices=["auto", "nchw"], help="nchw: NCHW activations also for 16-bit types")
     args = ap.parse_args()

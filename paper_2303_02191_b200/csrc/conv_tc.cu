@@ -34,6 +34,8 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
+#include <cstring>
+
 #include "conv_common.cuh"
 
 namespace {
@@ -482,38 +484,56 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     PFN_cuTensorMapEncodeTiled_v12000 enc = encode_fn();
     if (!enc) return (int)cudaErrorNotSupported;
     const CUtensorMapDataType dt = a.is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
-    CUtensorMap tmA, tmB;
-    {
+    // activations: descriptor cached per (pointer, shape, box)
+    const int key[6] = {d->N, d->H, d->W, p->Cin, plan.TH + 2 * pad, Wp * 4 + (int)p->dtype};
+    rtoss_tmap_entry* ea = nullptr;
+    for (rtoss_tmap_entry& e : ctx->tmap_cache)
+        if (e.valid && e.base == x && memcmp(e.dims, key, sizeof(key)) == 0) ea = &e;
+    if (!ea) {
+        ea = &ctx->tmap_cache[ctx->tmap_next];
+        ctx->tmap_next = (ctx->tmap_next + 1) % 32;
         cuuint64_t dims[4] = {(cuuint64_t)p->Cin, (cuuint64_t)d->W, (cuuint64_t)d->H, (cuuint64_t)d->N};
         cuuint64_t strides[3] = {(cuuint64_t)p->Cin * 2, (cuuint64_t)d->W * p->Cin * 2, (cuuint64_t)d->H * d->W * p->Cin * 2};
         cuuint32_t box[4] = {(cuuint32_t)kKBlock, (cuuint32_t)Wp, (cuuint32_t)(plan.TH + 2 * pad), 1};
         cuuint32_t es[4] = {1, 1, 1, 1};
-        CUresult r = enc(&tmA, dt, 4, const_cast<void*>(x), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        ea->valid = 0;
+        CUresult r = enc(reinterpret_cast<CUtensorMap*>(ea->map), dt, 4, const_cast<void*>(x), dims, strides, box, es,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return (int)cudaErrorInvalidValue;
+        ea->base = x;
+        memcpy(ea->dims, key, sizeof(key));
+        ea->valid = 1;
     }
-    {
+    // weights: one descriptor per handle
+    rtoss_tmap_entry* eb = &p->wtc_map;
+    if (!eb->valid || eb->base != p->wtc || eb->dims[0] != N_T) {
         cuuint64_t dims[3] = {(cuuint64_t)p->Cin, (cuuint64_t)p->Cout, (cuuint64_t)taps};
         cuuint64_t strides[2] = {(cuuint64_t)p->Cin * 2, (cuuint64_t)p->Cout * p->Cin * 2};
         cuuint32_t box[3] = {(cuuint32_t)kKBlock, (cuuint32_t)N_T, 1};
         cuuint32_t es[3] = {1, 1, 1};
-        CUresult r = enc(&tmB, dt, 3, p->wtc, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        eb->valid = 0;
+        CUresult r = enc(reinterpret_cast<CUtensorMap*>(eb->map), dt, 3, p->wtc, dims, strides, box, es,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return (int)cudaErrorInvalidValue;
+        eb->base = p->wtc;
+        eb->dims[0] = N_T;
+        eb->valid = 1;
     }
+    const CUtensorMap& tmA = *reinterpret_cast<const CUtensorMap*>(ea->map);
+    const CUtensorMap& tmB = *reinterpret_cast<const CUtensorMap*>(eb->map);
     const size_t smem = (size_t)plan.smem;
     dim3 grid((unsigned)((size_t)d->N * a.tiles_y * a.co_tiles));
-    cudaError_t e;
-    if (a.is_bf16) {
-        auto kern = conv_tc_kernel<__nv_bfloat16>;
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static bool attr_set = false;  // both instantiations may use up to the whole shared memory of an SM
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(conv_tc_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return (int)e;
-        kern<<<grid, kTcThreads, smem, (cudaStream_t)stream>>>(tmA, tmB, a);
-    } else {
-        auto kern = conv_tc_kernel<__half>;
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return (int)e;
-        kern<<<grid, kTcThreads, smem, (cudaStream_t)stream>>>(tmA, tmB, a);
+        attr_set = true;
     }
+    if (a.is_bf16) conv_tc_kernel<__nv_bfloat16><<<grid, kTcThreads, smem, (cudaStream_t)stream>>>(tmA, tmB, a);
+    else conv_tc_kernel<__half><<<grid, kTcThreads, smem, (cudaStream_t)stream>>>(tmA, tmB, a);
     return (int)cudaGetLastError();
 }

@@ -194,6 +194,7 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
     cudaError_t e = cudaSuccess;
     rtoss_packed* p = *out;
     const bool reuse = p != nullptr;
+    bool masks_changed = true;
     if (reuse) {
         // re-pack into an existing handle (e.g. after another pruning iteration): same layer, no allocation
         if (p->device != ctx->device || p->Cout != Cout || p->Cin != Cin || p->ksize != ksize || p->P != P || p->k != k ||
@@ -201,8 +202,11 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
             set_err(ctx, "pack", "existing handle describes another layer, table size or dtype");
             return RTOSS_ERR_INVALID_ARG;
         }
-        memset(p->masks, 0, sizeof(p->masks));
-        memcpy(p->masks, masks_host, sizeof(uint16_t) * (size_t)P);
+        masks_changed = memcmp(p->masks, masks_host, sizeof(uint16_t) * (size_t)P) != 0;
+        if (masks_changed) {
+            memset(p->masks, 0, sizeof(p->masks));
+            memcpy(p->masks, masks_host, sizeof(uint16_t) * (size_t)P);
+        }
     } else {
         p = new (std::nothrow) rtoss_packed();
         if (!p) return RTOSS_ERR_ALLOC;
@@ -235,7 +239,7 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
     }
     int le = 0;
     // the mask table is copied from the handle's own (pageable) storage: the copy is staged before return
-    e = cudaMemcpyAsync(p->masks_dev, p->masks, sizeof(uint16_t) * 256, cudaMemcpyHostToDevice, s);
+    if (masks_changed) e = cudaMemcpyAsync(p->masks_dev, p->masks, sizeof(uint16_t) * 256, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess && p->n_kernels > 0)
         e = cudaMemcpyAsync(p->pid, pid_dev, (size_t)p->n_kernels, cudaMemcpyDeviceToDevice, s);
     if (e == cudaSuccess)

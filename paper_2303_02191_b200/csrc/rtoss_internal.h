@@ -7,6 +7,14 @@
 
 #include "rtoss.h"
 
+// Host-side cache of encoded TMA descriptors (encoding costs microseconds per call).
+struct rtoss_tmap_entry {
+    const void* base;
+    int dims[6];  // what the descriptor was encoded for
+    int valid;
+    alignas(64) unsigned char map[128];
+};
+
 struct rtoss_ctx {
     int device;
     int sm_count;
@@ -18,6 +26,8 @@ struct rtoss_ctx {
     size_t ws_y_bytes;
     void* h_stream;  // cudaStream_t owned by the context, used by the host-buffer path
     int* dev_status;  // device word: 0, or the code of a bounded device-side wait that ran out
+    mutable rtoss_tmap_entry tmap_cache[32];  // activation descriptors of the tensor path, round robin
+    mutable int tmap_next;
 };
 
 struct rtoss_packed {
@@ -31,6 +41,7 @@ struct rtoss_packed {
     uint32_t* bucket_off;  // [Cin*(P+1)]     (ksize 3)
     uint16_t* masks_dev;   // [256]
     void* wtc;             // tensor path: dense-expanded weights [taps][Cout][Cin] in dtype, or NULL
+    mutable rtoss_tmap_entry wtc_map;  // its TMA descriptor, encoded at first use
     uint16_t masks[256];
 };
 
