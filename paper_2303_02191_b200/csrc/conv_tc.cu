@@ -23,11 +23,12 @@
 //     channels per instruction, accumulators in TMEM (nMB * N_T columns).
 //   * Weights are the dense-expanded form Wt[t][co][ci] that rtoss_pack builds
 //     next to the packed arrays; one TMA box per (tap, channel block).
-//   * Warp roles: warp 0 issues TMA, warp 1 issues tcgen05.mma and owns the
-//     TMEM allocation, warps 2..9 run the epilogue (tcgen05.ld, bias,
-//     activation, rounding, 16-byte NHWC stores).  Where shared memory and
-//     TMEM allow, two CTAs share an SM so that one CTA's epilogue runs under
-//     the other's MMAs.
+//   * Persistent CTAs, one per SM, each walking a strided list of tiles.  Warp
+//     roles: warp 0 issues TMA, warp 1 issues tcgen05.mma and owns the TMEM
+//     allocation, warps 2..9 run the epilogue (tcgen05.ld, bias, activation,
+//     rounding, 16-byte NHWC stores).  Activation and weight stages form rings
+//     that run on across tiles; with two accumulator stages in TMEM the
+//     epilogue of a tile runs under the MMAs of the next one.
 //   * Every mbarrier wait is bounded; a wait that runs out records a code in
 //     the context's status word and the CTA leaves through the normal exit
 //     (TMEM is always released).
@@ -43,6 +44,8 @@ namespace {
 using namespace rtoss_dev;
 
 constexpr int kTcThreads = 320;    // TMA warp, MMA warp, eight epilogue warps
+constexpr int kEpiWarps = 8;
+constexpr int kMaxA = 4, kMaxB = 8;  // most activation stages / weight slots
 constexpr int kKBlock = 64;       // channels per staged block: 128 bytes of bf16 / fp16
 constexpr int kRowBytes = 128;    // one padded pixel, one channel block
 constexpr long long kWaitCycles = 2000000000LL;  // about one second
@@ -55,7 +58,8 @@ struct TcArgs {
     int Wp, TH, taps, pad;       // padded pitch, output rows per CTA, 9 or 1, 1 or 0
     int nMB, N_T, ncb;           // M blocks per CTA, filters per CTA, channel blocks
     int tiles_y, co_tiles;
-    int a_stage_bytes, b_stage_bytes, NA, NB;  // stage sizes, activation stages (1 or 2), weight slots
+    int a_stage_bytes, b_stage_bytes, NA, NB;  // stage sizes, activation stages, weight slots
+    int AS, acc_cols;                          // accumulator stages in TMEM and columns per stage
     unsigned a_tx_bytes, b_tx_bytes;
     int act, y_c_off, y_c_stride, is_bf16;
     unsigned idesc;
@@ -165,7 +169,7 @@ __device__ __forceinline__ unsigned pack2<__half>(float a, float b) {
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kTcThreads, 2)
+__global__ void __launch_bounds__(kTcThreads, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcArgs a) {
     extern __shared__ unsigned char smem_dyn[];
     // tiles need 1024-byte alignment for the 128-byte swizzle pattern
@@ -173,23 +177,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const unsigned sA = base;                                        // [NA][a_stage_bytes]
     const unsigned sB = sA + (unsigned)a.NA * a.a_stage_bytes;       // [NB][b_stage_bytes]
     const unsigned sBar = sB + (unsigned)a.NB * a.b_stage_bytes;     // barriers, 8 bytes each
-    const unsigned bar_fullA = sBar, bar_emptyA = sBar + 16, bar_fullB = sBar + 32;
-    const unsigned bar_emptyB = bar_fullB + 8u * a.NB, bar_dfull = bar_emptyB + 8u * a.NB;
-    const unsigned s_tmem_ptr = bar_dfull + 8;
-    unsigned char* gen_base = smem_dyn + (base - smem_u32(smem_dyn));
-    volatile unsigned* tmem_ptr_gen = reinterpret_cast<volatile unsigned*>(gen_base + (s_tmem_ptr - base));
-    float* s_bias = reinterpret_cast<float*>(gen_base + (s_tmem_ptr + 8 - base));  // [N_T]
+    const unsigned bar_fullA = sBar, bar_emptyA = sBar + 8 * kMaxA;
+    const unsigned bar_fullB = bar_emptyA + 8 * kMaxA, bar_emptyB = bar_fullB + 8 * kMaxB;
+    const unsigned bar_accFull = bar_emptyB + 8 * kMaxB, bar_accEmpty = bar_accFull + 16;
+    const unsigned s_tmem_ptr = bar_accEmpty + 16;
+    volatile unsigned* tmem_ptr_gen = reinterpret_cast<volatile unsigned*>(smem_dyn + (s_tmem_ptr - smem_u32(smem_dyn)));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int bid = blockIdx.x;
-    const int cot = bid % a.co_tiles;
-    bid /= a.co_tiles;
-    const int ty = bid % a.tiles_y;
-    const int n = bid / a.tiles_y;
-    const int y0 = ty * a.TH, co0 = cot * a.N_T;
+    const int n_tiles = a.N * a.tiles_y * a.co_tiles;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < a.NA; ++i) {
             mbar_init(bar_fullA + 8 * i, 1);
             mbar_init(bar_emptyA + 8 * i, 1);
         }
@@ -197,12 +195,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             mbar_init(bar_fullB + 8 * i, 1);
             mbar_init(bar_emptyB + 8 * i, 1);
         }
-        mbar_init(bar_dfull, 1);
+        for (int i = 0; i < a.AS; ++i) {
+            mbar_init(bar_accFull + 8 * i, 1);
+            mbar_init(bar_accEmpty + 8 * i, kEpiWarps);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
     }
-    for (int i = threadIdx.x; i < a.N_T; i += kTcThreads) s_bias[i] = (a.bias && co0 + i < a.Cout) ? a.bias[co0 + i] : 0.f;
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s_tmem_ptr), "r"(a.tmem_cols)
                      : "memory");
@@ -213,22 +213,33 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const unsigned tmem_base = *tmem_ptr_gen;
 
+    // Every role walks the same list of tiles: tile = blockIdx.x, + gridDim.x, ...  A tile is (image,
+    // row band, filter tile) with the filter tile fastest, so CTAs working side by side read the same
+    // activations from L2.  Stage counters run on across tiles, which lets the producer fetch the next
+    // tile's operands while the current one is still being multiplied, and the two accumulator stages
+    // let the epilogue of one tile run under the MMAs of the next.
     if (warp == 0) {
         // ---------------- TMA producer
         if (lane == 0) {
             bool ok = true;
-            for (int cb = 0; cb < a.ncb && ok; ++cb) {
-                const int sa = cb % a.NA;
-                ok = mbar_wait(bar_emptyA + 8 * sa, ((cb / a.NA) & 1) ^ 1);
-                if (!ok) break;
-                mbar_expect_tx(bar_fullA + 8 * sa, a.a_tx_bytes);
-                tma_load_4d(sA + sa * a.a_stage_bytes, &tmA, cb * kKBlock, -a.pad, y0 - a.pad, n, bar_fullA + 8 * sa);
-                for (int t = 0; t < a.taps; ++t) {
-                    const int it = cb * a.taps + t, sb = it % a.NB;
-                    ok = mbar_wait(bar_emptyB + 8 * sb, ((it / a.NB) & 1) ^ 1);
+            int ga = 0, gb = 0;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                const int cot = tile % a.co_tiles, rest = tile / a.co_tiles;
+                const int ty = rest % a.tiles_y, n = rest / a.tiles_y;
+                const int y0 = ty * a.TH, co0 = cot * a.N_T;
+                for (int cb = 0; cb < a.ncb && ok; ++cb, ++ga) {
+                    const int sa = ga % a.NA;
+                    ok = mbar_wait(bar_emptyA + 8 * sa, ((ga / a.NA) & 1) ^ 1);
                     if (!ok) break;
-                    mbar_expect_tx(bar_fullB + 8 * sb, a.b_tx_bytes);
-                    tma_load_3d(sB + sb * a.b_stage_bytes, &tmB, cb * kKBlock, co0, t, bar_fullB + 8 * sb);
+                    mbar_expect_tx(bar_fullA + 8 * sa, a.a_tx_bytes);
+                    tma_load_4d(sA + sa * a.a_stage_bytes, &tmA, cb * kKBlock, -a.pad, y0 - a.pad, n, bar_fullA + 8 * sa);
+                    for (int t = 0; t < a.taps; ++t, ++gb) {
+                        const int sb = gb % a.NB;
+                        ok = mbar_wait(bar_emptyB + 8 * sb, ((gb / a.NB) & 1) ^ 1);
+                        if (!ok) break;
+                        mbar_expect_tx(bar_fullB + 8 * sb, a.b_tx_bytes);
+                        tma_load_3d(sB + sb * a.b_stage_bytes, &tmB, cb * kKBlock, co0, t, bar_fullB + 8 * sb);
+                    }
                 }
             }
             if (!ok) atomicExch(a.status, 1);
@@ -237,42 +248,58 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // ---------------- MMA issuer
         if (lane == 0) {
             bool ok = true;
-            for (int cb = 0; cb < a.ncb && ok; ++cb) {
-                const int sa = cb % a.NA;
-                ok = mbar_wait(bar_fullA + 8 * sa, (cb / a.NA) & 1);
+            int ga = 0, gb = 0, gt = 0;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++gt) {
+                const int as = gt % a.AS;
+                ok = mbar_wait(bar_accEmpty + 8 * as, ((gt / a.AS) & 1) ^ 1);  // epilogue has drained this stage
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const unsigned a_tile = sA + sa * a.a_stage_bytes;
-                for (int t = 0; t < a.taps; ++t) {
-                    const int it = cb * a.taps + t, sb = it % a.NB;
-                    ok = mbar_wait(bar_fullB + 8 * sb, (it / a.NB) & 1);
+                const unsigned d_base = tmem_base + (unsigned)(as * a.acc_cols);
+                for (int cb = 0; cb < a.ncb && ok; ++cb, ++ga) {
+                    const int sa = ga % a.NA;
+                    ok = mbar_wait(bar_fullA + 8 * sa, (ga / a.NA) & 1);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const int shift = a.taps == 9 ? (t / 3) * a.Wp + (t % 3) : 0;
-                    const unsigned b_tile = sB + sb * a.b_stage_bytes;
-                    for (int mb = 0; mb < a.nMB; ++mb) {
-                        const unsigned a_rows = a_tile + (unsigned)(mb * 128 + shift) * kRowBytes;
+                    const unsigned a_tile = sA + sa * a.a_stage_bytes;
+                    for (int t = 0; t < a.taps; ++t, ++gb) {
+                        const int sb = gb % a.NB;
+                        ok = mbar_wait(bar_fullB + 8 * sb, (gb / a.NB) & 1);
+                        if (!ok) break;
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        const int shift = a.taps == 9 ? (t / 3) * a.Wp + (t % 3) : 0;
+                        const unsigned b_tile = sB + sb * a.b_stage_bytes;
+                        for (int mb = 0; mb < a.nMB; ++mb) {
+                            const unsigned a_rows = a_tile + (unsigned)(mb * 128 + shift) * kRowBytes;
 #pragma unroll
-                        for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
-                            umma_f16(tmem_base + (unsigned)(mb * a.N_T), make_sw128_desc(a_rows + k4 * 32),
-                                     make_sw128_desc(b_tile + k4 * 32), a.idesc, (cb | t | k4) != 0);
+                            for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
+                                umma_f16(d_base + (unsigned)(mb * a.N_T), make_sw128_desc(a_rows + k4 * 32),
+                                         make_sw128_desc(b_tile + k4 * 32), a.idesc, (cb | t | k4) != 0);
+                            }
                         }
+                        umma_commit(bar_emptyB + 8 * sb);  // this weight slot may be refilled once the MMAs have read it
                     }
-                    umma_commit(bar_emptyB + 8 * sb);  // this weight slot may be refilled once the MMAs have read it
+                    if (ok) umma_commit(bar_emptyA + 8 * sa);
                 }
-                if (ok) umma_commit(bar_emptyA + 8 * sa);
+                if (ok) umma_commit(bar_accFull + 8 * as);
             }
-            if (ok) umma_commit(bar_dfull);
-            else atomicExch(a.status, 2);
+            if (!ok) atomicExch(a.status, 2);
         }
     } else {
         // ---------------- epilogue: TMEM -> registers -> bias / activation -> NHWC global
         const int quarter = warp & 3;      // TMEM lanes a warp may read: 32 * (warp id mod 4)
         const int half = (warp - 2) >> 2;  // two warps share a lane quarter and alternate 32-column chunks
-        const bool ok = mbar_wait(bar_dfull, 0);
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (ok) {
-            T* __restrict__ yg = reinterpret_cast<T*>(a.y);
+        T* __restrict__ yg = reinterpret_cast<T*>(a.y);
+        bool ok = true;
+        int gt = 0;
+        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++gt) {
+            const int cot = tile % a.co_tiles, rest = tile / a.co_tiles;
+            const int ty = rest % a.tiles_y, n = rest / a.tiles_y;
+            const int y0 = ty * a.TH, co0 = cot * a.N_T;
+            const int as = gt % a.AS;
+            ok = mbar_wait(bar_accFull + 8 * as, (gt / a.AS) & 1);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const unsigned d_base = tmem_base + (unsigned)(as * a.acc_cols) + ((unsigned)(quarter * 32) << 16);
             for (int mb = 0; mb < a.nMB; ++mb) {
                 const int p = mb * 128 + quarter * 32 + lane;
                 const int oyl = p / a.Wp, ox = p - oyl * a.Wp;
@@ -281,19 +308,29 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 T* dst = yg + (((size_t)n * a.H + oy) * a.W + ox) * a.y_c_stride + a.y_c_off + co0;
                 for (int c0 = half * 32; c0 < a.N_T; c0 += 64) {
                     unsigned r[32];
-                    tmem_ld32(tmem_base + ((unsigned)(quarter * 32) << 16) + (unsigned)(mb * a.N_T + c0), r);
+                    tmem_ld32(d_base + (unsigned)(mb * a.N_T + c0), r);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                     if (valid) {
 #pragma unroll
                         for (int v = 0; v < 4; ++v) {  // 8 filters = 16 bytes per store
-                            if (co0 + c0 + v * 8 < a.Cout) {
+                            const int co = co0 + c0 + v * 8;
+                            if (co < a.Cout) {
+                                float bv[8];
+                                if (a.bias) {
+                                    const float4 b0 = __ldg(reinterpret_cast<const float4*>(a.bias + co));
+                                    const float4 b1 = __ldg(reinterpret_cast<const float4*>(a.bias + co) + 1);
+                                    bv[0] = b0.x; bv[1] = b0.y; bv[2] = b0.z; bv[3] = b0.w;
+                                    bv[4] = b1.x; bv[5] = b1.y; bv[6] = b1.z; bv[7] = b1.w;
+                                } else {
+#pragma unroll
+                                    for (int h = 0; h < 8; ++h) bv[h] = 0.f;
+                                }
                                 uint4 o;
                                 unsigned* ow = reinterpret_cast<unsigned*>(&o);
 #pragma unroll
                                 for (int h = 0; h < 4; ++h) {
-                                    const int c = c0 + v * 8 + h * 2;
-                                    const float f0 = activate16(__uint_as_float(r[v * 8 + h * 2]) + s_bias[c], a.act);
-                                    const float f1 = activate16(__uint_as_float(r[v * 8 + h * 2 + 1]) + s_bias[c + 1], a.act);
+                                    const float f0 = activate16(__uint_as_float(r[v * 8 + h * 2]) + bv[h * 2], a.act);
+                                    const float f1 = activate16(__uint_as_float(r[v * 8 + h * 2 + 1]) + bv[h * 2 + 1], a.act);
                                     ow[h] = pack2<T>(f0, f1);
                                 }
                                 *reinterpret_cast<uint4*>(dst + c0 + v * 8) = o;
@@ -302,9 +339,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                 }
             }
-        } else if (lane == 0) {
-            atomicExch(a.status, 3);
+            // this warp has read everything it needs from the accumulator stage
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_accEmpty + 8 * as) : "memory");
         }
+        if (!ok && lane == 0) atomicExch(a.status, 3);
     }
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -349,17 +389,16 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 struct TcPlan {
-    int TH, nMB, N_T, NA, NB, a_rows, smem;
+    int TH, nMB, N_T, NA, NB, AS, acc_cols, a_rows, smem;
 };
 
-// Choose rows per CTA.  Two shapes are tried for every TH: "shared" (one activation stage, at most
-// 256 TMEM columns, at most half an SM's shared memory, so that two CTAs are co-resident and one's
-// epilogue runs under the other's MMAs) and "alone" (two activation stages, the whole SM).  Score:
-// how full the 128-row MMA blocks are, how few rows are wasted at the image bottom, with a bonus
-// for the shared shape.
-bool plan_tc(int H, int W, int Wp, int pad, int N_T, TcPlan* out) {
+// Choose rows per CTA tile: fill the 128-row MMA blocks well, waste few rows at the image bottom,
+// prefer shapes that leave room for two accumulator stages (at most 256 TMEM columns per tile) and
+// whose tile count spreads over the SMs.
+bool plan_tc(int N, int H, int W, int Wp, int pad, int N_T, int co_tiles, int sm_count, TcPlan* out) {
     const int b_bytes = N_T * kRowBytes;
-    const int fixed = 1024 /*alignment slack*/ + 256 /*barriers*/ + 4 * (N_T + 32);
+    const int fixed = 1024 /*alignment slack*/ + 512 /*barriers*/;
+    const int cap = 226 * 1024;
     double best = -1;
     for (int th = 1; th <= H && th + 2 * pad <= 256; ++th) {
         const int nmb = (th * Wp + 127) / 128;
@@ -367,25 +406,30 @@ bool plan_tc(int H, int W, int Wp, int pad, int N_T, TcPlan* out) {
         if (cols > 512 || nmb > 4) break;
         const int a_rows = round_up(nmb * 128 + 2 * pad * Wp + 2 * pad, 8);
         const int a_bytes = a_rows * kRowBytes;
+        const int as = cols <= 256 ? 2 : 1;
+        int na = (cap - fixed - 3 * b_bytes) / a_bytes;
+        if (na < 1) continue;
+        if (na > kMaxA) na = kMaxA;
+        if (na > 2 && pad) na = 2;  // 3x3: a channel block feeds nine taps, two stages cover the load
+        int nb = (cap - fixed - na * a_bytes) / b_bytes;
+        if (nb > kMaxB) nb = kMaxB;
+        if (nb < 2) continue;
+        const long tiles = (long)N * ((H + th - 1) / th) * co_tiles;
+        const double waves = (double)tiles / sm_count;
+        const double balance = waves / (double)((tiles + sm_count - 1) / sm_count);  // 1 = every SM equally loaded
         const double eff = (double)(th * W) / (nmb * 128) * H / (double)((H + th - 1) / th * th);
-        for (int shared = 1; shared >= 0; --shared) {
-            const int cap = shared ? 113 * 1024 : 226 * 1024;
-            const int na = shared ? 1 : 2;
-            if (shared && cols > 256) continue;
-            int nb = (cap - fixed - na * a_bytes) / b_bytes;
-            if (nb < (shared ? 3 : 2)) continue;
-            if (nb > 6) nb = 6;
-            const double score = eff * (shared ? 1.0 : 0.75) + 1e-4 * th;
-            if (score > best) {
-                best = score;
-                out->TH = th;
-                out->nMB = nmb;
-                out->N_T = N_T;
-                out->NA = na;
-                out->NB = nb;
-                out->a_rows = a_rows;
-                out->smem = na * a_bytes + nb * b_bytes + fixed;
-            }
+        const double score = eff * (as == 2 ? 1.0 : 0.8) * (0.5 + 0.5 * balance) + 1e-4 * th;
+        if (score > best) {
+            best = score;
+            out->TH = th;
+            out->nMB = nmb;
+            out->N_T = N_T;
+            out->NA = na;
+            out->NB = nb;
+            out->AS = as;
+            out->acc_cols = cols;
+            out->a_rows = a_rows;
+            out->smem = na * a_bytes + nb * b_bytes + fixed;
         }
     }
     return best > 0;
@@ -428,11 +472,12 @@ bool rtoss_tc_eligible(const rtoss_packed* p, const rtoss_conv_desc* d, const vo
     const int cs = d->y_channel_stride ? d->y_channel_stride : p->Cout;
     if (cs % 8 != 0 || d->y_channel_offset % 8 != 0) return false;  // 16-byte output stores
     if ((reinterpret_cast<uintptr_t>(x) & 15) || (reinterpret_cast<uintptr_t>(y) & 15)) return false;
+    if (reinterpret_cast<uintptr_t>(d->bias_dev) & 15) return false;  // the epilogue reads the bias as float4
     if (!encode_fn()) return false;
     const int N_T = tc_pick_nt(p->Cout);
     if (N_T == 0) return false;
     TcPlan plan;
-    return plan_tc(d->H, d->W, d->W + 2 * pad, pad, N_T, &plan);
+    return plan_tc(d->N, d->H, d->W, d->W + 2 * pad, pad, N_T, (p->Cout + N_T - 1) / N_T, 148, &plan);
 }
 
 int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y, const rtoss_conv_desc* d,
@@ -443,7 +488,8 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     const int N_T = tc_pick_nt(p->Cout);
     if (N_T == 0) return (int)cudaErrorInvalidConfiguration;
     TcPlan plan;
-    if (!plan_tc(d->H, d->W, Wp, pad, N_T, &plan)) return (int)cudaErrorInvalidConfiguration;
+    const int sms = ctx->sm_count > 0 ? ctx->sm_count : 148;
+    if (!plan_tc(d->N, d->H, d->W, Wp, pad, N_T, (p->Cout + N_T - 1) / N_T, sms, &plan)) return (int)cudaErrorInvalidConfiguration;
 
     TcArgs a;
     a.y = y;
@@ -467,6 +513,8 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     a.b_stage_bytes = N_T * kRowBytes;
     a.NA = plan.NA;
     a.NB = plan.NB;
+    a.AS = plan.AS;
+    a.acc_cols = plan.acc_cols;
     a.a_tx_bytes = (unsigned)(kKBlock * 2 * Wp * (plan.TH + 2 * pad));
     a.b_tx_bytes = (unsigned)(kKBlock * 2 * N_T);
     a.act = (int)d->act;
@@ -476,7 +524,7 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     // instruction descriptor: fp32 accumulate, A and B of the io type, both K-major, N/8 and M/16
     const unsigned fmt = a.is_bf16 ? 1u : 0u;
     a.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((unsigned)(N_T >> 3) << 17) | ((unsigned)(128 >> 4) << 24);
-    const int cols = (plan.nMB - 1) * N_T + round_up(N_T, 32);  // the epilogue reads 32 columns at a time
+    const int cols = plan.AS * plan.acc_cols;  // acc_cols already allows the epilogue's 32-column reads
     int alloc = 32;
     while (alloc < cols) alloc <<= 1;
     a.tmem_cols = alloc;
@@ -523,8 +571,10 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     }
     const CUtensorMap& tmA = *reinterpret_cast<const CUtensorMap*>(ea->map);
     const CUtensorMap& tmB = *reinterpret_cast<const CUtensorMap*>(eb->map);
-    const size_t smem = (size_t)plan.smem;
-    dim3 grid((unsigned)((size_t)d->N * a.tiles_y * a.co_tiles));
+    // at least half an SM's shared memory, so that a second CTA (which would wait for TMEM) never shares the SM
+    const size_t smem = (size_t)(plan.smem > 116 * 1024 ? plan.smem : 116 * 1024);
+    const size_t n_tiles = (size_t)d->N * a.tiles_y * a.co_tiles;
+    dim3 grid((unsigned)(n_tiles < (size_t)sms ? n_tiles : (size_t)sms));
     static bool attr_set = false;  // both instantiations may use up to the whole shared memory of an SM
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
