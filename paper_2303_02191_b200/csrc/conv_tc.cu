@@ -8,27 +8,34 @@
 // faster than the FMA-pipe gather for 16-bit data; the FMA path stays the one
 // for fp32 and for shapes this kernel does not take.
 //
-// GEMM view:  D[pixel, co] = sum over taps t and channels ci of
-//                            X[pixel shifted by t, ci] * Wt[t][co][ci]
-//   * A CTA owns TH output rows of one image (all columns) and N_T output
+// GEMM view:  D[co, position] = sum over taps t and channels ci of
+//                               Wt[t][co][ci] * X[position shifted by t, ci]
+//   * A CTA tile is TH output rows of one image (all columns) times 128 output
 //     channels.  The input rows it needs (with the one-pixel halo, zero-filled
 //     by TMA outside the image) are staged once per block of 64 channels as a
 //     flat list of "padded pixels", 128 bytes (64 channels) each, row pitch
 //     Wp = W + 2 pixels.  In that list the input pixel of tap (r, c) for output
-//     position p is at p + r*Wp + c: the A operand of every tap is the SAME
-//     shared-memory tile read from a different start row, so the halo tile is
-//     loaded once and used by all nine taps.  Output positions run over the
-//     padded pitch too; the two junk positions per row are computed and dropped.
-//   * M = 128 positions per MMA (nMB blocks per CTA), N = N_T filters, K = 16
-//     channels per instruction, accumulators in TMEM (nMB * N_T columns).
+//     position p is at p + r*Wp + c: the activation operand of every tap is
+//     the SAME shared-memory tile read from a different start row, so the halo
+//     tile is loaded once and used by all nine taps.  Output positions run over
+//     the padded pitch too; the two junk positions per row are computed and
+//     dropped.
+//   * Operand roles: the weights are the M operand (128 filters = the 128 TMEM
+//     lanes), the positions are the N operand (up to 256 per instruction), K =
+//     16 channels per instruction.  One instruction costs about 140 cycles
+//     whatever N is (the 128-row M operand is fetched at a row per cycle), so N
+//     must be wide: 128 x 256 x 16 per instruction runs near the tensor peak,
+//     128 x 128 x 16 at half of it (measured on this kernel with both roles).
 //   * Weights are the dense-expanded form Wt[t][co][ci] that rtoss_pack builds
-//     next to the packed arrays; one TMA box per (tap, channel block).
+//     next to the packed arrays; one TMA box per (tap, channel block); filters
+//     beyond Cout are zero-filled by TMA.
 //   * Persistent CTAs, one per SM, each walking a strided list of tiles.  Warp
 //     roles: warp 0 issues TMA, warp 1 issues tcgen05.mma and owns the TMEM
 //     allocation, warps 2..9 run the epilogue (tcgen05.ld, bias, activation,
-//     rounding, 16-byte NHWC stores).  Activation and weight stages form rings
-//     that run on across tiles; with two accumulator stages in TMEM the
-//     epilogue of a tile runs under the MMAs of the next one.
+//     rounding, NHWC stores: a warp holds 32 consecutive filters of one
+//     position, i.e. 64 contiguous bytes per store instruction).  Activation
+//     and weight stages form rings that run on across tiles; two accumulator
+//     stages in TMEM let the epilogue of a tile run under the MMAs of the next.
 //   * Every mbarrier wait is bounded; a wait that runs out records a code in
 //     the context's status word and the CTA leaves through the normal exit
 //     (TMEM is always released).
@@ -46,6 +53,7 @@ using namespace rtoss_dev;
 constexpr int kTcThreads = 320;    // TMA warp, MMA warp, eight epilogue warps
 constexpr int kEpiWarps = 8;
 constexpr int kMaxA = 4, kMaxB = 8;  // most activation stages / weight slots
+constexpr int kMTile = 128;          // filters per tile = TMEM lanes
 constexpr int kKBlock = 64;       // channels per staged block: 128 bytes of bf16 / fp16
 constexpr int kRowBytes = 128;    // one padded pixel, one channel block
 constexpr long long kWaitCycles = 2000000000LL;  // about one second
@@ -55,8 +63,8 @@ struct TcArgs {
     const float* bias;
     int* status;
     int N, H, W, Cin, Cout;
-    int Wp, TH, taps, pad;       // padded pitch, output rows per CTA, 9 or 1, 1 or 0
-    int nMB, N_T, ncb;           // M blocks per CTA, filters per CTA, channel blocks
+    int Wp, TH, taps, pad;       // padded pitch, output rows per CTA tile, 9 or 1, 1 or 0
+    int N_px, ncb;               // positions per tile (the MMA's N, multiple of 16), channel blocks
     int tiles_y, co_tiles;
     int a_stage_bytes, b_stage_bytes, NA, NB;  // stage sizes, activation stages, weight slots
     int AS, acc_cols;                          // accumulator stages in TMEM and columns per stage
@@ -226,7 +234,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
                 const int cot = tile % a.co_tiles, rest = tile / a.co_tiles;
                 const int ty = rest % a.tiles_y, n = rest / a.tiles_y;
-                const int y0 = ty * a.TH, co0 = cot * a.N_T;
+                const int y0 = ty * a.TH, co0 = cot * kMTile;
                 for (int cb = 0; cb < a.ncb && ok; ++cb, ++ga) {
                     const int sa = ga % a.NA;
                     ok = mbar_wait(bar_emptyA + 8 * sa, ((ga / a.NA) & 1) ^ 1);
@@ -267,14 +275,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         if (!ok) break;
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                         const int shift = a.taps == 9 ? (t / 3) * a.Wp + (t % 3) : 0;
-                        const unsigned b_tile = sB + sb * a.b_stage_bytes;
-                        for (int mb = 0; mb < a.nMB; ++mb) {
-                            const unsigned a_rows = a_tile + (unsigned)(mb * 128 + shift) * kRowBytes;
+                        const unsigned w_tile = sB + sb * a.b_stage_bytes;                 // M operand: 128 filters
+                        const unsigned x_rows = a_tile + (unsigned)shift * kRowBytes;    // N operand: N_px positions
 #pragma unroll
-                            for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
-                                umma_f16(d_base + (unsigned)(mb * a.N_T), make_sw128_desc(a_rows + k4 * 32),
-                                         make_sw128_desc(b_tile + k4 * 32), a.idesc, (cb | t | k4) != 0);
-                            }
+                        for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
+                            umma_f16(d_base, make_sw128_desc(w_tile + k4 * 32), make_sw128_desc(x_rows + k4 * 32), a.idesc,
+                                     (cb | t | k4) != 0);
                         }
                         umma_commit(bar_emptyB + 8 * sb);  // this weight slot may be refilled once the MMAs have read it
                     }
@@ -294,48 +300,29 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++gt) {
             const int cot = tile % a.co_tiles, rest = tile / a.co_tiles;
             const int ty = rest % a.tiles_y, n = rest / a.tiles_y;
-            const int y0 = ty * a.TH, co0 = cot * a.N_T;
+            const int y0 = ty * a.TH, co0 = cot * kMTile;
             const int as = gt % a.AS;
             ok = mbar_wait(bar_accFull + 8 * as, (gt / a.AS) & 1);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const unsigned d_base = tmem_base + (unsigned)(as * a.acc_cols) + ((unsigned)(quarter * 32) << 16);
-            for (int mb = 0; mb < a.nMB; ++mb) {
-                const int p = mb * 128 + quarter * 32 + lane;
-                const int oyl = p / a.Wp, ox = p - oyl * a.Wp;
-                const int oy = y0 + oyl;
-                const bool valid = oyl < a.TH && ox < a.W && oy < a.H;
-                T* dst = yg + (((size_t)n * a.H + oy) * a.W + ox) * a.y_c_stride + a.y_c_off + co0;
-                for (int c0 = half * 32; c0 < a.N_T; c0 += 64) {
-                    unsigned r[32];
-                    tmem_ld32(d_base + (unsigned)(mb * a.N_T + c0), r);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    if (valid) {
+            const int co = co0 + quarter * 32 + lane;  // this thread's filter: TMEM lane = filter
+            const bool co_ok = co < a.Cout;
+            const float bv = (a.bias && co_ok) ? __ldg(a.bias + co) : 0.f;
+            T* ybase = yg + ((size_t)n * a.H * a.W) * a.y_c_stride + a.y_c_off + co;
+            for (int c0 = half * 32; c0 < a.N_px; c0 += 64) {
+                unsigned r[32];
+                tmem_ld32(d_base + (unsigned)c0, r);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                int oyl = c0 / a.Wp, ox = c0 - oyl * a.Wp;  // position c0 + j, warp-uniform
 #pragma unroll
-                        for (int v = 0; v < 4; ++v) {  // 8 filters = 16 bytes per store
-                            const int co = co0 + c0 + v * 8;
-                            if (co < a.Cout) {
-                                float bv[8];
-                                if (a.bias) {
-                                    const float4 b0 = __ldg(reinterpret_cast<const float4*>(a.bias + co));
-                                    const float4 b1 = __ldg(reinterpret_cast<const float4*>(a.bias + co) + 1);
-                                    bv[0] = b0.x; bv[1] = b0.y; bv[2] = b0.z; bv[3] = b0.w;
-                                    bv[4] = b1.x; bv[5] = b1.y; bv[6] = b1.z; bv[7] = b1.w;
-                                } else {
-#pragma unroll
-                                    for (int h = 0; h < 8; ++h) bv[h] = 0.f;
-                                }
-                                uint4 o;
-                                unsigned* ow = reinterpret_cast<unsigned*>(&o);
-#pragma unroll
-                                for (int h = 0; h < 4; ++h) {
-                                    const float f0 = activate16(__uint_as_float(r[v * 8 + h * 2]) + bv[h * 2], a.act);
-                                    const float f1 = activate16(__uint_as_float(r[v * 8 + h * 2 + 1]) + bv[h * 2 + 1], a.act);
-                                    ow[h] = pack2<T>(f0, f1);
-                                }
-                                *reinterpret_cast<uint4*>(dst + c0 + v * 8) = o;
-                            }
-                        }
+                for (int j = 0; j < 32; ++j) {
+                    const int oy = y0 + oyl;
+                    if (co_ok && oyl < a.TH && ox < a.W && oy < a.H)
+                        ybase[((size_t)oy * a.W + ox) * a.y_c_stride] = from_f32<T>(activate16(__uint_as_float(r[j]) + bv, a.act));
+                    if (++ox == a.Wp) {
+                        ox = 0;
+                        ++oyl;
                     }
                 }
             }
@@ -389,24 +376,21 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 struct TcPlan {
-    int TH, nMB, N_T, NA, NB, AS, acc_cols, a_rows, smem;
+    int TH, N_px, NA, NB, a_rows, smem;
 };
 
-// Choose rows per CTA tile: fill the 128-row MMA blocks well, waste few rows at the image bottom,
-// prefer shapes that leave room for two accumulator stages (at most 256 TMEM columns per tile) and
-// whose tile count spreads over the SMs.
-bool plan_tc(int N, int H, int W, int Wp, int pad, int N_T, int co_tiles, int sm_count, TcPlan* out) {
-    const int b_bytes = N_T * kRowBytes;
+// Choose rows per tile: as many positions (rows * padded pitch) as fit one 256-wide MMA, few rows
+// wasted at the image bottom, and a tile count that spreads over the SMs.
+bool plan_tc(int N, int H, int W, int Wp, int pad, int co_tiles, int sm_count, TcPlan* out) {
+    const int b_bytes = kMTile * kRowBytes;
     const int fixed = 1024 /*alignment slack*/ + 512 /*barriers*/;
     const int cap = 226 * 1024;
     double best = -1;
     for (int th = 1; th <= H && th + 2 * pad <= 256; ++th) {
-        const int nmb = (th * Wp + 127) / 128;
-        const int cols = (nmb - 1) * N_T + round_up(N_T, 32);
-        if (cols > 512 || nmb > 4) break;
-        const int a_rows = round_up(nmb * 128 + 2 * pad * Wp + 2 * pad, 8);
+        if (th * Wp > 256) break;
+        const int n_px = round_up(th * Wp, 16);
+        const int a_rows = round_up(n_px + 2 * pad * Wp + 2 * pad, 8);
         const int a_bytes = a_rows * kRowBytes;
-        const int as = cols <= 256 ? 2 : 1;
         int na = (cap - fixed - 3 * b_bytes) / a_bytes;
         if (na < 1) continue;
         if (na > kMaxA) na = kMaxA;
@@ -417,17 +401,15 @@ bool plan_tc(int N, int H, int W, int Wp, int pad, int N_T, int co_tiles, int sm
         const long tiles = (long)N * ((H + th - 1) / th) * co_tiles;
         const double waves = (double)tiles / sm_count;
         const double balance = waves / (double)((tiles + sm_count - 1) / sm_count);  // 1 = every SM equally loaded
-        const double eff = (double)(th * W) / (nmb * 128) * H / (double)((H + th - 1) / th * th);
-        const double score = eff * (as == 2 ? 1.0 : 0.8) * (0.5 + 0.5 * balance) + 1e-4 * th;
+        // an instruction costs about the same for any N: what counts is useful positions per instruction
+        const double eff = (double)(th * W) / 256.0 * H / (double)((H + th - 1) / th * th);
+        const double score = eff * (0.5 + 0.5 * balance) + 1e-4 * th;
         if (score > best) {
             best = score;
             out->TH = th;
-            out->nMB = nmb;
-            out->N_T = N_T;
+            out->N_px = n_px;
             out->NA = na;
             out->NB = nb;
-            out->AS = as;
-            out->acc_cols = cols;
             out->a_rows = a_rows;
             out->smem = na * a_bytes + nb * b_bytes + fixed;
         }
@@ -438,7 +420,7 @@ bool plan_tc(int N, int H, int W, int Wp, int pad, int N_T, int co_tiles, int sm
 }  // namespace
 
 bool rtoss_tc_weights_eligible(const rtoss_packed* p) {
-    return (p->dtype == RTOSS_BF16 || p->dtype == RTOSS_F16) && p->Cin % 8 == 0 && p->Cout % 16 == 0;
+    return (p->dtype == RTOSS_BF16 || p->dtype == RTOSS_F16) && p->Cin % 8 == 0;  // 16-byte rows for TMA
 }
 
 int rtoss_launch_expand_taps(const rtoss_packed* p, void* out, void* stream) {
@@ -455,29 +437,16 @@ int rtoss_launch_expand_taps(const rtoss_packed* p, void* out, void* stream) {
     return (int)cudaGetLastError();
 }
 
-// Filters per CTA: the whole layer up to 128, else tiles of 128 (or the whole layer up to 256 when
-// it is not a multiple of 128); 0 = no tiling this kernel takes.
-static int tc_pick_nt(int Cout) {
-    if (Cout <= 128) return Cout;
-    if (Cout % 128 == 0) return 128;
-    return Cout <= 256 ? Cout : 0;
-}
-
 // Can this call run on the tensor path?
 bool rtoss_tc_eligible(const rtoss_packed* p, const rtoss_conv_desc* d, const void* x, const void* y) {
     if (!p->wtc || !rtoss_tc_weights_eligible(p)) return false;
     if (d->layout != RTOSS_NHWC || d->stride != 1 || (int)d->io_dtype != (int)p->dtype) return false;
     const int pad = p->ksize == 3 ? 1 : 0;
     if (d->W + 2 * pad > 256) return false;
-    const int cs = d->y_channel_stride ? d->y_channel_stride : p->Cout;
-    if (cs % 8 != 0 || d->y_channel_offset % 8 != 0) return false;  // 16-byte output stores
     if ((reinterpret_cast<uintptr_t>(x) & 15) || (reinterpret_cast<uintptr_t>(y) & 15)) return false;
-    if (reinterpret_cast<uintptr_t>(d->bias_dev) & 15) return false;  // the epilogue reads the bias as float4
     if (!encode_fn()) return false;
-    const int N_T = tc_pick_nt(p->Cout);
-    if (N_T == 0) return false;
     TcPlan plan;
-    return plan_tc(d->N, d->H, d->W, d->W + 2 * pad, pad, N_T, (p->Cout + N_T - 1) / N_T, 148, &plan);
+    return plan_tc(d->N, d->H, d->W, d->W + 2 * pad, pad, (p->Cout + kMTile - 1) / kMTile, 148, &plan);
 }
 
 int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y, const rtoss_conv_desc* d,
@@ -485,11 +454,11 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     const int pad = p->ksize == 3 ? 1 : 0;
     const int taps = p->ksize == 3 ? 9 : 1;
     const int Wp = d->W + 2 * pad;
-    const int N_T = tc_pick_nt(p->Cout);
-    if (N_T == 0) return (int)cudaErrorInvalidConfiguration;
-    TcPlan plan;
+    const int N_T = kMTile;
     const int sms = ctx->sm_count > 0 ? ctx->sm_count : 148;
-    if (!plan_tc(d->N, d->H, d->W, Wp, pad, N_T, (p->Cout + N_T - 1) / N_T, sms, &plan)) return (int)cudaErrorInvalidConfiguration;
+    TcPlan plan;
+    if (!plan_tc(d->N, d->H, d->W, Wp, pad, (p->Cout + kMTile - 1) / kMTile, sms, &plan))
+        return (int)cudaErrorInvalidConfiguration;
 
     TcArgs a;
     a.y = y;
@@ -504,8 +473,7 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     a.TH = plan.TH;
     a.taps = taps;
     a.pad = pad;
-    a.nMB = plan.nMB;
-    a.N_T = N_T;
+    a.N_px = plan.N_px;
     a.ncb = (p->Cin + kKBlock - 1) / kKBlock;
     a.tiles_y = (d->H + plan.TH - 1) / plan.TH;
     a.co_tiles = (p->Cout + N_T - 1) / N_T;
@@ -513,8 +481,8 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     a.b_stage_bytes = N_T * kRowBytes;
     a.NA = plan.NA;
     a.NB = plan.NB;
-    a.AS = plan.AS;
-    a.acc_cols = plan.acc_cols;
+    a.AS = 2;
+    a.acc_cols = round_up(plan.N_px, 32);  // the epilogue reads 32 columns at a time
     a.a_tx_bytes = (unsigned)(kKBlock * 2 * Wp * (plan.TH + 2 * pad));
     a.b_tx_bytes = (unsigned)(kKBlock * 2 * N_T);
     a.act = (int)d->act;
@@ -523,8 +491,8 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     a.is_bf16 = p->dtype == RTOSS_BF16;
     // instruction descriptor: fp32 accumulate, A and B of the io type, both K-major, N/8 and M/16
     const unsigned fmt = a.is_bf16 ? 1u : 0u;
-    a.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((unsigned)(N_T >> 3) << 17) | ((unsigned)(128 >> 4) << 24);
-    const int cols = plan.AS * plan.acc_cols;  // acc_cols already allows the epilogue's 32-column reads
+    a.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((unsigned)(plan.N_px >> 3) << 17) | ((unsigned)(kMTile >> 4) << 24);
+    const int cols = a.AS * a.acc_cols;
     int alloc = 32;
     while (alloc < cols) alloc <<= 1;
     a.tmem_cols = alloc;

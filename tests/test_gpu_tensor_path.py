@@ -47,6 +47,8 @@ CASES = [
     (1, 1, 1024, 512, 20, 20, 4, "bf16", "silu"),
     (1, 1, 40, 80, 13, 17, 2, "f16", "relu"),
     (1, 1, 512, 2048, 25, 34, 4, "bf16", "relu"),
+    (3, 1, 24, 20, 9, 11, 3, "bf16", "silu"),         # filter count not a multiple of 16, 24 channels
+    (1, 3, 8, 200, 5, 254, 2, "f16", "none"),         # widest image the path takes, filter tiles 128 + 72
 ]
 
 
@@ -83,15 +85,15 @@ def test_tensor_path_channel_slice_and_batch_sampled():
     b = synth.bias(23, 1, Cout)
     _, packed = gu.select_pack(w, 3, masks, 3, "bf16")
     _, wd, _ = gu.oracle_weights(w, 3, masks, 3, "bf16")
-    y = gu.run_conv(packed, 3, x, "bf16", 1, "silu", b, "nhwc", y_off=64, y_stride=256, path=rt.PATH_TENSOR)
-    assert (y[:, :64] == 7.0).all() and (y[:, 192:] == 7.0).all()
+    y = gu.run_conv(packed, 3, x, "bf16", 1, "silu", b, "nhwc", y_off=61, y_stride=251, path=rt.PATH_TENSOR)
+    assert (y[:, :61] == 7.0).all() and (y[:, 189:] == 7.0).all()
     rng = np.random.default_rng(7)
     npts = 4000
     idx = np.stack([rng.integers(0, N, npts), rng.integers(0, Cout, npts), rng.integers(0, H, npts),
                     rng.integers(0, W, npts)], axis=1).astype(np.int32)
     idx[:4] = [[0, 0, 0, 0], [0, 0, 0, W - 1], [N - 1, Cout - 1, H - 1, W - 1], [N - 1, 0, H - 1, 0]]
     ref = orc.conv_points(3, x, wd, b, 1, orc.ACT_SILU, orc.DT_BF16, idx)
-    got = y[idx[:, 0], 64 + idx[:, 1], idx[:, 2], idx[:, 3]]
+    got = y[idx[:, 0], 61 + idx[:, 1], idx[:, 2], idx[:, 3]]
     rms = float(np.sqrt(np.mean(ref.astype(np.float64) ** 2)))
     assert np.max(np.abs(got - ref) / np.maximum(np.abs(ref), rms)) <= 2e-2
     _no_timeout()
