@@ -54,6 +54,7 @@ constexpr int kTcThreads = 320;    // TMA warp, MMA warp, eight epilogue warps
 constexpr int kEpiWarps = 8;
 constexpr int kMaxA = 4, kMaxB = 8;  // most activation stages / weight slots
 constexpr int kMTile = 128;          // filters per tile = TMEM lanes
+constexpr int kPatchPitch = 80;      // bytes per position row of an epilogue transpose patch (64 + pad)
 constexpr int kKBlock = 64;       // channels per staged block: 128 bytes of bf16 / fp16
 constexpr int kRowBytes = 128;    // one padded pixel, one channel block
 constexpr long long kWaitCycles = 2000000000LL;  // about one second
@@ -190,6 +191,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const unsigned bar_accFull = bar_emptyB + 8 * kMaxB, bar_accEmpty = bar_accFull + 16;
     const unsigned s_tmem_ptr = bar_accEmpty + 16;
     volatile unsigned* tmem_ptr_gen = reinterpret_cast<volatile unsigned*>(smem_dyn + (s_tmem_ptr - smem_u32(smem_dyn)));
+    unsigned char* epi_patch = smem_dyn + (s_tmem_ptr + 16 - smem_u32(smem_dyn));  // [kEpiWarps][32][kPatchPitch], 16-byte aligned
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = a.N * a.tiles_y * a.co_tiles;
@@ -309,22 +311,48 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int co = co0 + quarter * 32 + lane;  // this thread's filter: TMEM lane = filter
             const bool co_ok = co < a.Cout;
             const float bv = (a.bias && co_ok) ? __ldg(a.bias + co) : 0.f;
-            T* ybase = yg + ((size_t)n * a.H * a.W) * a.y_c_stride + a.y_c_off + co;
+            // A warp holds 32 filters (lanes) x 32 positions (registers); NHWC wants the filters of one
+            // position side by side.  The chunk is turned through a private shared-memory patch
+            // (position-major rows of 64 + 16 pad bytes) so that global stores are 16 bytes per lane,
+            // four lanes covering the 64 contiguous bytes of one position.
+            unsigned char* patch = epi_patch + (warp - 2) * (32 * kPatchPitch);
+            const bool vec_ok = (a.y_c_stride % 8 == 0) && ((a.y_c_off + co0) % 8 == 0) && (co0 + quarter * 32 + 32 <= a.Cout);
             for (int c0 = half * 32; c0 < a.N_px; c0 += 64) {
                 unsigned r[32];
                 tmem_ld32(d_base + (unsigned)c0, r);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                int oyl = c0 / a.Wp, ox = c0 - oyl * a.Wp;  // position c0 + j, warp-uniform
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int oy = y0 + oyl;
-                    if (co_ok && oyl < a.TH && ox < a.W && oy < a.H)
-                        ybase[((size_t)oy * a.W + ox) * a.y_c_stride] = from_f32<T>(activate16(__uint_as_float(r[j]) + bv, a.act));
-                    if (++ox == a.Wp) {
-                        ox = 0;
-                        ++oyl;
+                for (int j = 0; j < 32; ++j)
+                    *reinterpret_cast<T*>(patch + j * kPatchPitch + lane * 2) =
+                        from_f32<T>(activate16(__uint_as_float(r[j]) + bv, a.act));
+                __syncwarp();
+                if (vec_ok) {
+#pragma unroll
+                    for (int it = 0; it < 4; ++it) {
+                        const int i = it * 32 + lane, j = i >> 2, v = i & 3;  // position j of the chunk, 8-filter group v
+                        const int pos = c0 + j;
+                        const int oyl = pos / a.Wp, ox = pos - oyl * a.Wp, oy = y0 + oyl;
+                        if (oyl < a.TH && ox < a.W && oy < a.H) {
+                            const uint4 o = *reinterpret_cast<const uint4*>(patch + j * kPatchPitch + v * 16);
+                            *reinterpret_cast<uint4*>(yg + (((size_t)n * a.H + oy) * a.W + ox) * a.y_c_stride + a.y_c_off + co0 +
+                                                      quarter * 32 + v * 8) = o;
+                        }
+                    }
+                } else {
+                    // ragged filter counts or unaligned channel slices: element stores, lane = filter
+                    int oyl = c0 / a.Wp, ox = c0 - oyl * a.Wp;
+                    for (int j = 0; j < 32; ++j) {
+                        const int oy = y0 + oyl;
+                        if (co_ok && oyl < a.TH && ox < a.W && oy < a.H)
+                            yg[(((size_t)n * a.H + oy) * a.W + ox) * a.y_c_stride + a.y_c_off + co] =
+                                *reinterpret_cast<const T*>(patch + j * kPatchPitch + lane * 2);
+                        if (++ox == a.Wp) {
+                            ox = 0;
+                            ++oyl;
+                        }
                     }
                 }
+                __syncwarp();
             }
             // this warp has read everything it needs from the accumulator stage
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -383,7 +411,7 @@ struct TcPlan {
 // wasted at the image bottom, and a tile count that spreads over the SMs.
 bool plan_tc(int N, int H, int W, int Wp, int pad, int co_tiles, int sm_count, TcPlan* out) {
     const int b_bytes = kMTile * kRowBytes;
-    const int fixed = 1024 /*alignment slack*/ + 512 /*barriers*/;
+    const int fixed = 1024 /*alignment slack*/ + 512 /*barriers*/ + kEpiWarps * 32 * kPatchPitch /*epilogue patches*/;
     const int cap = 226 * 1024;
     double best = -1;
     for (int th = 1; th <= H && th + 2 * pad <= 256; ++th) {
