@@ -67,7 +67,8 @@ struct TcArgs {
     int Wp, TH, taps, pad;       // padded pitch, output rows per CTA tile, 9 or 1, 1 or 0
     int N_px, ncb;               // positions per tile (the MMA's N, multiple of 16), channel blocks
     int tiles_y, co_tiles;
-    int a_stage_bytes, b_stage_bytes, NA, NB;  // stage sizes, activation stages, weight slots
+    int a_stage_bytes, b_stage_bytes, NA, NB;  // stage sizes, activation stages, weight stages
+    int G;                                     // taps per weight stage (one barrier round trip per G taps)
     int AS, acc_cols;                          // accumulator stages in TMEM and columns per stage
     unsigned a_tx_bytes, b_tx_bytes;
     int act, y_c_off, y_c_stride, is_bf16;
@@ -84,18 +85,22 @@ __device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 // Bounded wait on a phase parity; false when the limit ran out.
+__device__ __forceinline__ unsigned mbar_try(unsigned bar, unsigned parity) {
+    unsigned done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return done;
+}
 __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
+    if (mbar_try(bar, parity)) return true;  // the common case costs one instruction, no clock read
     const long long t0 = clock64();
     for (;;) {
-        unsigned done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done)
-            : "r"(bar), "r"(parity)
-            : "memory");
-        if (done) return true;
+        if (mbar_try(bar, parity)) return true;
         if (clock64() - t0 > kWaitCycles) return false;
     }
 }
@@ -162,6 +167,18 @@ __device__ __forceinline__ float activate16(float v, int act) {
     if (act == RTOSS_ACT_RELU) return fmaxf(v, 0.f);
     if (act == RTOSS_ACT_SILU) return __fdividef(v, 1.f + __expf(-v));
     return v;
+}
+
+// One 32-position chunk of one filter: bias, activation, rounding, into the transpose patch.
+template <typename T, int ACT>
+__device__ __forceinline__ void act_to_patch(const unsigned (&r)[32], float bv, unsigned char* col) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        float v = __uint_as_float(r[j]) + bv;
+        if (ACT == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
+        if (ACT == RTOSS_ACT_SILU) v = __fdividef(v, 1.f + __expf(-v));
+        *reinterpret_cast<T*>(col + j * kPatchPitch) = from_f32<T>(v);
+    }
 }
 
 template <typename T>
@@ -243,17 +260,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (!ok) break;
                     mbar_expect_tx(bar_fullA + 8 * sa, a.a_tx_bytes);
                     tma_load_4d(sA + sa * a.a_stage_bytes, &tmA, cb * kKBlock, -a.pad, y0 - a.pad, n, bar_fullA + 8 * sa);
-                    for (int t = 0; t < a.taps; ++t, ++gb) {
+                    for (int t0 = 0; t0 < a.taps; t0 += a.G, ++gb) {
                         const int sb = gb % a.NB;
                         ok = mbar_wait(bar_emptyB + 8 * sb, ((gb / a.NB) & 1) ^ 1);
                         if (!ok) break;
-                        mbar_expect_tx(bar_fullB + 8 * sb, a.b_tx_bytes);
-                        tma_load_3d(sB + sb * a.b_stage_bytes, &tmB, cb * kKBlock, co0, t, bar_fullB + 8 * sb);
+                        mbar_expect_tx(bar_fullB + 8 * sb, a.b_tx_bytes * a.G);
+                        for (int i = 0; i < a.G; ++i)
+                            tma_load_3d(sB + sb * a.b_stage_bytes + i * (kMTile * kRowBytes), &tmB, cb * kKBlock, co0, t0 + i,
+                                        bar_fullB + 8 * sb);
                     }
                 }
             }
             if (!ok) atomicExch(a.status, 1);
         }
+        __syncwarp();  // lanes 1..31 wait here for lane 0: the warp reaches the final barrier as one
     } else if (warp == 1) {
         // ---------------- MMA issuer
         if (lane == 0) {
@@ -271,27 +291,36 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const unsigned a_tile = sA + sa * a.a_stage_bytes;
-                    for (int t = 0; t < a.taps; ++t, ++gb) {
+                    for (int t0 = 0; t0 < a.taps; t0 += a.G, ++gb) {
                         const int sb = gb % a.NB;
                         ok = mbar_wait(bar_fullB + 8 * sb, (gb / a.NB) & 1);
                         if (!ok) break;
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                        const int shift = a.taps == 9 ? (t / 3) * a.Wp + (t % 3) : 0;
-                        const unsigned w_tile = sB + sb * a.b_stage_bytes;                 // M operand: 128 filters
-                        const unsigned x_rows = a_tile + (unsigned)shift * kRowBytes;    // N operand: N_px positions
+                        for (int i = 0; i < a.G; ++i) {
+                            const int t = t0 + i;
+                            const int shift = a.taps == 9 ? (t / 3) * a.Wp + (t % 3) : 0;
+                            const unsigned w_tile = sB + sb * a.b_stage_bytes + i * (kMTile * kRowBytes);  // M operand: 128 filters
+                            const unsigned x_rows = a_tile + (unsigned)shift * kRowBytes;                   // N operand: N_px positions
 #pragma unroll
-                        for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
-                            umma_f16(d_base, make_sw128_desc(w_tile + k4 * 32), make_sw128_desc(x_rows + k4 * 32), a.idesc,
-                                     (cb | t | k4) != 0);
+                            for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
+                                umma_f16(d_base, make_sw128_desc(w_tile + k4 * 32), make_sw128_desc(x_rows + k4 * 32), a.idesc,
+                                         (cb | t | k4) != 0);
+                            }
                         }
-                        umma_commit(bar_emptyB + 8 * sb);  // this weight slot may be refilled once the MMAs have read it
+                        umma_commit(bar_emptyB + 8 * sb);  // this weight stage may be refilled once the MMAs have read it
                     }
                     if (ok) umma_commit(bar_emptyA + 8 * sa);
                 }
                 if (ok) umma_commit(bar_accFull + 8 * as);
             }
+            // TMEM may only be released after the epilogue has drained the last tiles
+            for (int i = 0; i < a.AS && i < gt && ok; ++i) {
+                const int g = gt - 1 - i;
+                ok = mbar_wait(bar_accEmpty + 8 * (g % a.AS), (g / a.AS) & 1);
+            }
             if (!ok) atomicExch(a.status, 2);
         }
+        __syncwarp();
     } else {
         // ---------------- epilogue: TMEM -> registers -> bias / activation -> NHWC global
         const int quarter = warp & 3;      // TMEM lanes a warp may read: 32 * (warp id mod 4)
@@ -321,10 +350,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 unsigned r[32];
                 tmem_ld32(d_base + (unsigned)c0, r);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    *reinterpret_cast<T*>(patch + j * kPatchPitch + lane * 2) =
-                        from_f32<T>(activate16(__uint_as_float(r[j]) + bv, a.act));
+                // the activation is picked outside the loop: 32 independent, branch-free chains
+                if (a.act == RTOSS_ACT_SILU) act_to_patch<T, RTOSS_ACT_SILU>(r, bv, patch + lane * 2);
+                else if (a.act == RTOSS_ACT_RELU) act_to_patch<T, RTOSS_ACT_RELU>(r, bv, patch + lane * 2);
+                else act_to_patch<T, RTOSS_ACT_NONE>(r, bv, patch + lane * 2);
                 __syncwarp();
                 if (vec_ok) {
 #pragma unroll
@@ -404,22 +433,23 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 struct TcPlan {
-    int TH, N_px, NA, NB, a_rows, smem;
+    int TH, N_px, NA, NB, G, a_rows, smem;
 };
 
 // Choose rows per tile: as many positions (rows * padded pitch) as fit one 256-wide MMA, few rows
 // wasted at the image bottom, and a tile count that spreads over the SMs.
 bool plan_tc(int N, int H, int W, int Wp, int pad, int co_tiles, int sm_count, TcPlan* out) {
-    const int b_bytes = kMTile * kRowBytes;
+    const int G = pad ? 3 : 1;  // 3x3: one weight stage holds a kernel row of three taps
+    const int b_bytes = G * kMTile * kRowBytes;
     const int fixed = 1024 /*alignment slack*/ + 512 /*barriers*/ + kEpiWarps * 32 * kPatchPitch /*epilogue patches*/;
-    const int cap = 226 * 1024;
+    const int cap = 227 * 1024 - 64;
     double best = -1;
     for (int th = 1; th <= H && th + 2 * pad <= 256; ++th) {
         if (th * Wp > 256) break;
         const int n_px = round_up(th * Wp, 16);
         const int a_rows = round_up(n_px + 2 * pad * Wp + 2 * pad, 8);
         const int a_bytes = a_rows * kRowBytes;
-        int na = (cap - fixed - 3 * b_bytes) / a_bytes;
+        int na = (cap - fixed - 2 * b_bytes) / a_bytes;
         if (na < 1) continue;
         if (na > kMaxA) na = kMaxA;
         if (na > 2 && pad) na = 2;  // 3x3: a channel block feeds nine taps, two stages cover the load
@@ -438,6 +468,7 @@ bool plan_tc(int N, int H, int W, int Wp, int pad, int co_tiles, int sm_count, T
             out->N_px = n_px;
             out->NA = na;
             out->NB = nb;
+            out->G = G;
             out->a_rows = a_rows;
             out->smem = na * a_bytes + nb * b_bytes + fixed;
         }
@@ -506,7 +537,8 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     a.tiles_y = (d->H + plan.TH - 1) / plan.TH;
     a.co_tiles = (p->Cout + N_T - 1) / N_T;
     a.a_stage_bytes = plan.a_rows * kRowBytes;
-    a.b_stage_bytes = N_T * kRowBytes;
+    a.b_stage_bytes = plan.G * N_T * kRowBytes;
+    a.G = plan.G;
     a.NA = plan.NA;
     a.NB = plan.NB;
     a.AS = 2;
