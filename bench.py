@@ -188,6 +188,25 @@ def run_reference(args):
     }))
 
 
+# --------------------------------------------------------------------------- multi-rank bookkeeping
+
+def max_over_ranks(values, device, world):
+    """Replicas only: ranks exchange nothing on the data path; the timed intervals are reduced with MAX
+    so that the reported time is the slowest rank's."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_value(images_per_rank, world, ms_per_step):
+    """Weak scaling: every rank processes its own batch; the job's images/s is the sum."""
+    return world * images_per_rank / (ms_per_step * 1e-3)
+
+
 # --------------------------------------------------------------------------- GPU arm
 
 def run_gpu(args):
@@ -356,14 +375,11 @@ def run_gpu(args):
     h2d = sum(st["xh"].numel() * elem for st in L_state)
     d2h = sum(st["yh"].numel() * elem for st in L_state)
 
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_s], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_s = float(t[0]), float(t[1])
+    total_ms, e2e_s = max_over_ranks([total_ms, e2e_s], dev, world)
 
     if rank == 0:
         ms_per_step = total_ms / args.steps
-        value = world * N / (ms_per_step * 1e-3)
+        value = whole_job_value(N, world, ms_per_step)
         flops = [synth.layer_nnz_flops(st["L"], N, st["k"]) for st in L_state]
         bytes_ = [synth.layer_bytes(st["L"], N, st["k"], elem) for st in L_state]
         top = int(np.argmax(conv_ms))
