@@ -167,6 +167,27 @@ rtoss_status rtoss_packed_export(rtoss_ctx* ctx, const rtoss_packed* p, uint8_t*
 rtoss_status rtoss_packed_to_dense(rtoss_ctx* ctx, const rtoss_packed* p, void* w_masked_dev, void* cuda_stream);
 void rtoss_packed_destroy(rtoss_packed* p);
 
+/* Pruned dense weights with no allocation anywhere (the paper has no counterpart: this entry point
+ * exists for deployment, not for the method).  Same result as rtoss_select_patterns followed by
+ * rtoss_pack (compute type = w_dtype) and rtoss_packed_to_dense: w_pruned_dev receives W (.) mask,
+ * [Cout][Cin][3][3] or [Cout][Cin] in w_dtype, pruned positions +0.  It is meant for callers that
+ * cannot call cudaMalloc: a process whose device memory was all handed to its own arena at start-up,
+ * or a loop that cannot afford the device-wide synchronisation cudaMalloc / cudaFree imply.  It needs
+ * no context and no packed handle and works on the current device.
+ *   - The pattern ids, the one intermediate, live in a fixed 1 MiB device array inside the library
+ *     (held by every GPU that loads the library until the process exits).  A layer with more than
+ *     2^20 kernels (Cout*Cin for ksize 3, floor(Cout*Cin/9) for ksize 1) is refused with
+ *     RTOSS_ERR_UNSUPPORTED.
+ *   - The first call on a device looks the array's address up (cudaGetSymbolAddress); make that first
+ *     call outside any stream capture.
+ *   - All calls on a device share the array and it keeps the last call's ids.  Each call overwrites
+ *     what it reads, so nothing needs clearing, but two calls whose kernels overlap on the GPU (two
+ *     streams, two host threads) race on it: keep calls on one device in stream order.
+ * Errors: RTOSS_ERR_INVALID_ARG, RTOSS_ERR_BAD_PATTERN_TABLE, RTOSS_ERR_ALIGNMENT (16 bytes),
+ * RTOSS_ERR_UNSUPPORTED (too many kernels), RTOSS_ERR_CUDA. */
+rtoss_status rtoss_prune_dense_static(const void* w_dev, rtoss_dtype w_dtype, int Cout, int Cin, int ksize,
+                                      const uint16_t* masks_host, int P, int k, void* w_pruned_dev, void* cuda_stream);
+
 /* ---- inference convolution over the packed weights ------------------------ */
 
 typedef struct {

@@ -26,7 +26,7 @@ SYMBOLS = [
     "rtoss_create", "rtoss_destroy", "rtoss_status_string", "rtoss_last_error", "rtoss_pattern_preset",
     "rtoss_pattern_table_validate", "rtoss_group_layers", "rtoss_select_patterns", "rtoss_pack",
     "rtoss_packed_info_get", "rtoss_packed_export", "rtoss_packed_to_dense", "rtoss_packed_destroy",
-    "rtoss_conv3x3_pattern", "rtoss_conv1x1_pattern", "rtoss_conv_pattern_host", "rtoss_device_status",
+    "rtoss_conv3x3_pattern", "rtoss_conv1x1_pattern", "rtoss_conv_pattern_host", "rtoss_device_status", "rtoss_prune_dense_static",
 ]
 
 
@@ -81,6 +81,7 @@ def _load():
     lib.rtoss_conv1x1_pattern.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ConvDesc), vp]
     lib.rtoss_conv_pattern_host.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ConvDesc)]
     lib.rtoss_device_status.argtypes = [vp, ctypes.POINTER(ci)]
+    lib.rtoss_prune_dense_static.argtypes = [vp, ci, ci, ci, ci, vp, ci, ci, vp, vp]
     return lib
 
 
@@ -132,6 +133,20 @@ def rtoss_group_layers(nodes):
     if st != OK:
         raise RtossError(st, status_string(st))
     return parent[:L], group[:L], ng.value
+
+
+def rtoss_prune_dense_static(w, ksize, masks, k, out=None):
+    """Pruned dense weights W (.) mask without any allocation inside the library (the ids live in a fixed
+    device array of the library; at most 2^20 kernels).  `out` is a caller-owned tensor like `w`; the one
+    created here when it is omitted is the caller's convenience, not the library's doing.  Returns the
+    status code together with the tensor so that callers can test for RTOSS_ERR_UNSUPPORTED."""
+    import torch
+    m = _masks_arr(masks)
+    if out is None:
+        out = torch.empty_like(w)
+    st = lib.rtoss_prune_dense_static(w.data_ptr(), _torch_dtype_code(w), int(w.shape[0]), int(w.shape[1]), int(ksize),
+                                      _np_ptr(m), len(m), int(k), out.data_ptr(), _stream())
+    return st, out
 
 
 def _torch_dtype_code(t):

@@ -5,6 +5,8 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
+#include <cstring>
+
 #include "rtoss_internal.h"
 
 namespace {
@@ -263,4 +265,100 @@ int rtoss_launch_to_dense(const rtoss_packed* p, void* w_out, void* stream) {
             break;
     }
     return (int)cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Pruning without any allocation.
+//
+// rtoss_select_patterns + rtoss_pack + rtoss_packed_to_dense produce the pruned dense weights
+// W (.) mask, but rtoss_pack allocates the packed handle with cudaMalloc.  Some callers cannot do
+// that: a serving process that handed all device memory to its own arena at start-up (a later
+// cudaMalloc simply fails), or a control loop that may not take cudaMalloc / cudaFree's implicit
+// device-wide synchronisation in the middle of its frames.  For them the pattern ids, the only
+// intermediate of that chain, live in the fixed array below instead of a per-call buffer.
+//
+// The array is part of the library image: every GPU whose context loads the library holds
+// kStaticPidBytes of device memory for it until the process exits.  All calls on a device share it.
+
+constexpr size_t kStaticPidBytes = (size_t)1 << 20;  // one pattern id per kernel: at most 2^20 kernels per call
+static __device__ __align__(256) unsigned char g_static_pid[kStaticPidBytes];
+
+namespace {
+
+// Dense masked weights straight from the weights and the pattern ids: out[e] = w[e] if position e is
+// kept by the pattern of its kernel (or run of nine), else +0.
+template <typename T>
+__global__ void mask_dense_kernel(const T* __restrict__ w, const uint8_t* __restrict__ pid, MaskTable table,
+                                  int64_t n_kernels, int64_t n_dense, T* __restrict__ out) {
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n_dense; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t g = e / 9;
+        const int t = (int)(e - 9 * g);
+        T v = narrow<T>(0.f);
+        if (g < n_kernels && (table.m[pid[g]] & (1u << t))) v = w[e];
+        out[e] = v;
+    }
+}
+
+// Device address of g_static_pid on the current device.  In host code the symbol's name is only a
+// handle for the runtime, never a pointer a kernel could use: the address has to be asked for, once
+// per device, with that device current.
+unsigned char* static_pid_address(cudaError_t* err) {
+    static unsigned char* cached[64] = {nullptr};
+    int dev = -1;
+    *err = cudaGetDevice(&dev);
+    if (*err != cudaSuccess) return nullptr;
+    if (dev < 0 || dev >= 64) {
+        *err = cudaErrorInvalidDevice;
+        return nullptr;
+    }
+    if (!cached[dev]) {
+        void* p = nullptr;
+        *err = cudaGetSymbolAddress(&p, g_static_pid);
+        if (*err != cudaSuccess) return nullptr;
+        cached[dev] = static_cast<unsigned char*>(p);
+    }
+    return cached[dev];
+}
+
+}  // namespace
+
+extern "C" rtoss_status rtoss_prune_dense_static(const void* w_dev, rtoss_dtype w_dtype, int Cout, int Cin, int ksize,
+                                                 const uint16_t* masks_host, int P, int k, void* w_pruned_dev,
+                                                 void* cuda_stream) {
+    if (!w_dev || !w_pruned_dev || !masks_host) return RTOSS_ERR_INVALID_ARG;
+    if (w_dtype != RTOSS_F32 && w_dtype != RTOSS_BF16 && w_dtype != RTOSS_F16) return RTOSS_ERR_INVALID_ARG;
+    if (Cout < 1 || Cin < 1 || (ksize != 1 && ksize != 3)) return RTOSS_ERR_INVALID_ARG;
+    if (!rtoss_table_ok(masks_host, P, k)) return RTOSS_ERR_BAD_PATTERN_TABLE;
+    if ((reinterpret_cast<uintptr_t>(w_dev) & 15) || (reinterpret_cast<uintptr_t>(w_pruned_dev) & 15))
+        return RTOSS_ERR_ALIGNMENT;
+    const int64_t total = (int64_t)Cout * Cin;
+    const int64_t n_kernels = ksize == 3 ? total : total / 9;
+    if (n_kernels > (int64_t)kStaticPidBytes) return RTOSS_ERR_UNSUPPORTED;  // more kernels than the fixed array holds
+    cudaError_t ce;
+    unsigned char* pid = static_pid_address(&ce);
+    if (!pid) return RTOSS_ERR_CUDA;
+    MaskTable table;
+    memset(&table, 0, sizeof(table));
+    memcpy(table.m, masks_host, sizeof(uint16_t) * (size_t)P);
+    // every pattern id this call reads is written by this call first: nothing in the array has to start at zero
+    int e = rtoss_launch_select(w_dev, w_dtype, n_kernels, table, P, pid, cuda_stream);
+    if (e) return RTOSS_ERR_CUDA;
+    const int64_t n_dense = ksize == 3 ? total * 9 : total;
+    const int threads = 256;
+    const int grid = grid_for((n_dense + threads - 1) / threads);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    switch (w_dtype) {
+        case RTOSS_F32:
+            mask_dense_kernel<float><<<grid, threads, 0, s>>>((const float*)w_dev, pid, table, n_kernels, n_dense, (float*)w_pruned_dev);
+            break;
+        case RTOSS_BF16:
+            mask_dense_kernel<__nv_bfloat16><<<grid, threads, 0, s>>>((const __nv_bfloat16*)w_dev, pid, table, n_kernels, n_dense,
+                                                                      (__nv_bfloat16*)w_pruned_dev);
+            break;
+        case RTOSS_F16:
+            mask_dense_kernel<__half><<<grid, threads, 0, s>>>((const __half*)w_dev, pid, table, n_kernels, n_dense,
+                                                               (__half*)w_pruned_dev);
+            break;
+    }
+    return cudaGetLastError() == cudaSuccess ? RTOSS_OK : RTOSS_ERR_CUDA;
 }
