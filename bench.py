@@ -357,7 +357,9 @@ def run_gpu(args):
 
     # ---- end to end through the host-buffer entry point (pinned host tensors, copies inside the timed region)
     torch.cuda.synchronize()
-    e2e_steps = max(3, min(args.steps, 20))
+    h2d = sum(st["xh"].numel() * elem for st in L_state)
+    d2h = sum(st["yh"].numel() * elem for st in L_state)
+    e2e_steps = max(2, min(args.steps, 20, int(2e10 / (h2d + d2h))))   # bounded: about 20 GB over PCIe at most
     for st in L_state[:1]:
         ctx.rtoss_conv_pattern_host(st["wt"]["packed"], st["xh"], st["yh"], N, st["L"]["H"], st["L"]["W"], st["L"]["stride"],
                                     layout, rt.ACT_NAMES[st["L"]["act"]], st["wt"]["b"], path=st["path"])
@@ -372,8 +374,6 @@ def run_gpu(args):
                                         rt.ACT_NAMES[L["act"]], st["wt"]["b"], path=st["path"])
     torch.cuda.synchronize()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
-    h2d = sum(st["xh"].numel() * elem for st in L_state)
-    d2h = sum(st["yh"].numel() * elem for st in L_state)
 
     total_ms, e2e_s = max_over_ranks([total_ms, e2e_s], dev, world)
 
