@@ -221,8 +221,8 @@ rtoss_status rtoss_conv1x1_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const 
                                    const rtoss_conv_desc* desc, void* cuda_stream);
 
 /* The tensor path (RTOSS_PATH_TENSOR, or RTOSS_PATH_AUTO when it applies) takes: bf16 / fp16 NHWC,
- * stride 1, io_dtype equal to the packed dtype, Cin a multiple of 8, W + 2 <= 256.  It multiplies the
- * pruned taps as zeros on the tensor cores; results agree with the FMA path to fp32 summation order.
+ * stride 1 or 2, io_dtype equal to the packed dtype, Cin a multiple of 8.  It multiplies the pruned
+ * taps as zeros on the tensor cores; results agree with the FMA path to fp32 summation order.
  *
  * Device-side waits of that path are bounded.  If one runs out, the kernel records a non-zero code in
  * the context and returns; rtoss_device_status synchronises the device, reports the code

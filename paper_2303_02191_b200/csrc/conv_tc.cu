@@ -63,10 +63,14 @@ struct TcArgs {
     void* y;
     const float* bias;
     int* status;
-    int N, H, W, Cin, Cout;
-    int Wp, TH, taps, pad;       // padded pitch, output rows per CTA tile, 9 or 1, 1 or 0
+    int N, Ho, Wo, Cin, Cout;    // output image size
+    int S;                       // stride
+    int Wq, TH, TW, taps;        // position pitch, output rows and columns per tile, 9 or 1
     int N_px, ncb;               // positions per tile (the MMA's N, multiple of 16), channel blocks
-    int tiles_y, co_tiles;
+    int tiles_y, tiles_x, co_tiles;
+    int n_sub, sub_bytes;        // staged sub-tiles per channel block (4 input phases for 3x3 stride 2) and their size
+    int x_add[4], y_add[4];      // TMA start coordinate of sub-tile s: x = x0*S + x_add[s], y = y0*S + y_add[s]
+    int tap_sub[9], tap_shift[9];  // which sub-tile tap t reads, and from which start row
     int a_stage_bytes, b_stage_bytes, NA, NB;  // stage sizes, activation stages, weight stages
     int G;                                     // taps per weight stage (one barrier round trip per G taps)
     int AS, acc_cols;                          // accumulator stages in TMEM and columns per stage
@@ -209,7 +213,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     unsigned char* epi_patch = smem_dyn + (s_tmem_ptr + 16 - smem_u32(smem_dyn));  // [kEpiWarps][32][kPatchPitch], 16-byte aligned
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_tiles = a.N * a.tiles_y * a.co_tiles;
+    const int n_tiles = a.N * a.tiles_y * a.tiles_x * a.co_tiles;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < a.NA; ++i) {
@@ -249,15 +253,21 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             bool ok = true;
             int ga = 0, gb = 0;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-                const int cot = tile % a.co_tiles, rest = tile / a.co_tiles;
+                int rest = tile;
+                const int cot = rest % a.co_tiles;
+                rest /= a.co_tiles;
+                const int tx = rest % a.tiles_x;
+                rest /= a.tiles_x;
                 const int ty = rest % a.tiles_y, n = rest / a.tiles_y;
-                const int y0 = ty * a.TH, co0 = cot * kMTile;
+                const int y0 = ty * a.TH, x0 = tx * a.TW, co0 = cot * kMTile;
                 for (int cb = 0; cb < a.ncb && ok; ++cb, ++ga) {
                     const int sa = ga % a.NA;
                     ok = mbar_wait(bar_emptyA + 8 * sa, ((ga / a.NA) & 1) ^ 1);
                     if (!ok) break;
-                    mbar_expect_tx(bar_fullA + 8 * sa, a.a_tx_bytes);
-                    tma_load_4d(sA + sa * a.a_stage_bytes, &tmA, cb * kKBlock, -a.pad, y0 - a.pad, n, bar_fullA + 8 * sa);
+                    mbar_expect_tx(bar_fullA + 8 * sa, a.a_tx_bytes * a.n_sub);
+                    for (int sub = 0; sub < a.n_sub; ++sub)
+                        tma_load_4d(sA + sa * a.a_stage_bytes + sub * a.sub_bytes, &tmA, cb * kKBlock, x0 * a.S + a.x_add[sub],
+                                    y0 * a.S + a.y_add[sub], n, bar_fullA + 8 * sa);
                     for (int t0 = 0; t0 < a.taps; t0 += a.G, ++gb) {
                         const int sb = gb % a.NB;
                         ok = mbar_wait(bar_emptyB + 8 * sb, ((gb / a.NB) & 1) ^ 1);
@@ -296,9 +306,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                         for (int i = 0; i < a.G; ++i) {
                             const int t = t0 + i;
-                            const int shift = a.taps == 9 ? (t / 3) * a.Wp + (t % 3) : 0;
                             const unsigned w_tile = sB + sb * a.b_stage_bytes + i * (kMTile * kRowBytes);  // M operand: 128 filters
-                            const unsigned x_rows = a_tile + (unsigned)shift * kRowBytes;                   // N operand: N_px positions
+                            const unsigned x_rows = a_tile + (unsigned)(a.tap_sub[t] * a.sub_bytes + a.tap_shift[t] * kRowBytes);  // N operand
 #pragma unroll
                             for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
                                 umma_f16(d_base, make_sw128_desc(w_tile + k4 * 32), make_sw128_desc(x_rows + k4 * 32), a.idesc,
@@ -327,9 +336,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         bool ok = true;
         int gt = 0;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++gt) {
-            const int cot = tile % a.co_tiles, rest = tile / a.co_tiles;
+            int rest = tile;
+            const int cot = rest % a.co_tiles;
+            rest /= a.co_tiles;
+            const int tx = rest % a.tiles_x;
+            rest /= a.tiles_x;
             const int ty = rest % a.tiles_y, n = rest / a.tiles_y;
-            const int y0 = ty * a.TH, co0 = cot * kMTile;
+            const int y0 = ty * a.TH, x0 = tx * a.TW, co0 = cot * kMTile;
             const int as = gt % a.AS;
             ok = mbar_wait(bar_accFull + 8 * as, (gt / a.AS) & 1);
             if (!ok) break;
@@ -358,23 +371,23 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     for (int it = 0; it < 4; ++it) {
                         const int i = it * 32 + lane, j = i >> 2, v = i & 3;  // position j of the chunk, 8-filter group v
                         const int pos = c0 + j;
-                        const int oyl = pos / a.Wp, ox = pos - oyl * a.Wp, oy = y0 + oyl;
-                        if (oyl < a.TH && ox < a.W && oy < a.H) {
+                        const int oyl = pos / a.Wq, oxl = pos - oyl * a.Wq, oy = y0 + oyl, ox = x0 + oxl;
+                        if (oyl < a.TH && oxl < a.TW && ox < a.Wo && oy < a.Ho) {
                             const uint4 o = *reinterpret_cast<const uint4*>(patch + j * kPatchPitch + v * 16);
-                            *reinterpret_cast<uint4*>(yg + (((size_t)n * a.H + oy) * a.W + ox) * a.y_c_stride + a.y_c_off + co0 +
+                            *reinterpret_cast<uint4*>(yg + (((size_t)n * a.Ho + oy) * a.Wo + ox) * a.y_c_stride + a.y_c_off + co0 +
                                                       quarter * 32 + v * 8) = o;
                         }
                     }
                 } else {
                     // ragged filter counts or unaligned channel slices: element stores, lane = filter
-                    int oyl = c0 / a.Wp, ox = c0 - oyl * a.Wp;
+                    int oyl = c0 / a.Wq, oxl = c0 - oyl * a.Wq;
                     for (int j = 0; j < 32; ++j) {
-                        const int oy = y0 + oyl;
-                        if (co_ok && oyl < a.TH && ox < a.W && oy < a.H)
-                            yg[(((size_t)n * a.H + oy) * a.W + ox) * a.y_c_stride + a.y_c_off + co] =
+                        const int oy = y0 + oyl, ox = x0 + oxl;
+                        if (co_ok && oyl < a.TH && oxl < a.TW && ox < a.Wo && oy < a.Ho)
+                            yg[(((size_t)n * a.Ho + oy) * a.Wo + ox) * a.y_c_stride + a.y_c_off + co] =
                                 *reinterpret_cast<const T*>(patch + j * kPatchPitch + lane * 2);
-                        if (++ox == a.Wp) {
-                            ox = 0;
+                        if (++oxl == a.Wq) {
+                            oxl = 0;
                             ++oyl;
                         }
                     }
@@ -431,44 +444,73 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 struct TcPlan {
-    int TH, N_px, NA, NB, G, a_rows, smem;
+    int TH, TW, Wq, N_px, NA, NB, G, n_sub, sub_rows, rows_staged, tiles_x, smem;
 };
 
-// Choose rows per tile: as many positions (rows * padded pitch) as fit one 256-wide MMA, few rows
-// wasted at the image bottom, and a tile count that spreads over the SMs.
-bool plan_tc(int N, int H, int W, int Wp, int pad, int co_tiles, int sm_count, TcPlan* out) {
-    const int G = pad ? 3 : 1;  // 3x3: one weight stage holds a kernel row of three taps
-    const int b_bytes = G * kMTile * kRowBytes;
+// Geometry of a tile.  Positions of a tile run over TH rows of pitch Wq = TW + (columns of halo the
+// staged rows carry); every tap reads the staged list from a shifted start row.
+//   3x3 stride 1: one staged tile, TH+2 rows of TW+2 pixels, tap (r,c) at shift r*Wq + c.
+//   1x1:          one staged tile, TH rows of TW pixels (stride 2: every second pixel and row, picked by
+//                 the TMA element strides), shift 0.
+//   3x3 stride 2: four staged tiles, one per (row parity, column parity) of the input, each TH+1 rows of
+//                 TW+1 pixels fetched with element strides 2; tap r reads the odd rows for r = 0, 2 and
+//                 the even rows for r = 1, one staged row further down for r = 1, 2; columns alike.
+// The plan picks TH, the column segment TW (images wider than a TMA box are cut into segments), the
+// ring depths, and how many taps share a weight stage.
+bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count, TcPlan* out) {
+    const int halo = ksize == 3 ? (S == 1 ? 2 : 1) : 0;
+    const int n_sub = (ksize == 3 && S == 2) ? 4 : 1;
+    const int max_pitch = S == 1 ? 256 : 128;  // TMA box: at most 256 elements traversed per dimension
     const int fixed = 1024 /*alignment slack*/ + 512 /*barriers*/ + kEpiWarps * 32 * kPatchPitch /*epilogue patches*/;
     const int cap = 227 * 1024 - 64;
     double best = -1;
-    for (int th = 1; th <= H && th + 2 * pad <= 256; ++th) {
-        if (th * Wp > 256) break;
-        const int n_px = round_up(th * Wp, 16);
-        const int a_rows = round_up(n_px + 2 * pad * Wp + 2 * pad, 8);
-        const int a_bytes = a_rows * kRowBytes;
-        int na = (cap - fixed - 2 * b_bytes) / a_bytes;
-        if (na < 1) continue;
-        if (na > kMaxA) na = kMaxA;
-        if (na > 2 && pad) na = 2;  // 3x3: a channel block feeds nine taps, two stages cover the load
-        int nb = (cap - fixed - na * a_bytes) / b_bytes;
-        if (nb > kMaxB) nb = kMaxB;
-        if (nb < 2) continue;
-        const long tiles = (long)N * ((H + th - 1) / th) * co_tiles;
-        const double waves = (double)tiles / sm_count;
-        const double balance = waves / (double)((tiles + sm_count - 1) / sm_count);  // 1 = every SM equally loaded
-        // an instruction costs about the same for any N: what counts is useful positions per instruction
-        const double eff = (double)(th * W) / 256.0 * H / (double)((H + th - 1) / th * th);
-        const double score = eff * (0.5 + 0.5 * balance) + 1e-4 * th;
-        if (score > best) {
-            best = score;
-            out->TH = th;
-            out->N_px = n_px;
-            out->NA = na;
-            out->NB = nb;
-            out->G = G;
-            out->a_rows = a_rows;
-            out->smem = na * a_bytes + nb * b_bytes + fixed;
+    for (int nseg = 1; nseg <= 16; ++nseg) {
+        const int tw = (Wo + nseg - 1) / nseg;
+        const int wq = tw + halo;
+        if (wq > max_pitch || wq > 256) continue;
+        for (int th = 1; th <= Ho; ++th) {
+            const int rows_staged = th + halo;
+            if (th * wq > 256 || rows_staged * S > 256) break;
+            const int n_px = round_up(th * wq, 16);
+            const int max_shift = ksize == 3 ? (S == 1 ? 2 * wq + 2 : wq + 1) : 0;
+            const int need_rows = n_px + max_shift > rows_staged * wq ? n_px + max_shift : rows_staged * wq;
+            const int sub_rows = round_up(need_rows, 8);
+            const int a_bytes = n_sub * sub_rows * kRowBytes;
+            for (int G = (ksize == 3 ? 3 : 1); G >= 1; G -= 2) {
+                const int b_bytes = G * kMTile * kRowBytes;
+                int na = (cap - fixed - 2 * b_bytes) / a_bytes;
+                if (na < 1) continue;
+                if (na > kMaxA) na = kMaxA;
+                if (na > 2 && ksize == 3) na = 2;  // a channel block feeds nine taps: two stages cover the load
+                int nb = (cap - fixed - na * a_bytes) / b_bytes;
+                if (nb > kMaxB) nb = kMaxB;
+                if (nb < 2) continue;
+                const long tiles = (long)N * ((Ho + th - 1) / th) * nseg * co_tiles;
+                const double waves = (double)tiles / sm_count;
+                const double balance = waves / (double)((tiles + sm_count - 1) / sm_count);  // 1 = SMs equally loaded
+                // an instruction costs about the same for any N: what counts is useful positions per instruction
+                const double eff = (double)(th * tw) / 256.0 * Ho / (double)((Ho + th - 1) / th * th) * Wo / (double)(tw * nseg);
+                const double halo_cost = (double)(th * tw) / (double)(rows_staged * wq);  // staged pixels that are outputs
+                const double score = eff * (0.5 + 0.5 * balance) * (G == 3 || ksize == 1 ? 1.0 : 0.8) * (na >= 2 ? 1.0 : 0.8) *
+                                         (0.8 + 0.2 * halo_cost) +
+                                     1e-4 * th;
+                if (score > best) {
+                    best = score;
+                    out->TH = th;
+                    out->TW = tw;
+                    out->Wq = wq;
+                    out->N_px = n_px;
+                    out->NA = na;
+                    out->NB = nb;
+                    out->G = G;
+                    out->n_sub = n_sub;
+                    out->sub_rows = sub_rows;
+                    out->rows_staged = rows_staged;
+                    out->tiles_x = nseg;
+                    out->smem = na * a_bytes + nb * b_bytes + fixed;
+                }
+                break;  // the largest G that fits is taken for this (th, tw)
+            }
         }
     }
     return best > 0;
@@ -497,24 +539,23 @@ int rtoss_launch_expand_taps(const rtoss_packed* p, void* out, void* stream) {
 // Can this call run on the tensor path?
 bool rtoss_tc_eligible(const rtoss_packed* p, const rtoss_conv_desc* d, const void* x, const void* y) {
     if (!p->wtc || !rtoss_tc_weights_eligible(p)) return false;
-    if (d->layout != RTOSS_NHWC || d->stride != 1 || (int)d->io_dtype != (int)p->dtype) return false;
-    const int pad = p->ksize == 3 ? 1 : 0;
-    if (d->W + 2 * pad > 256) return false;
+    if (d->layout != RTOSS_NHWC || (int)d->io_dtype != (int)p->dtype) return false;
     if ((reinterpret_cast<uintptr_t>(x) & 15) || (reinterpret_cast<uintptr_t>(y) & 15)) return false;
     if (!encode_fn()) return false;
+    const int Ho = (d->H - 1) / d->stride + 1, Wo = (d->W - 1) / d->stride + 1;
     TcPlan plan;
-    return plan_tc(d->N, d->H, d->W, d->W + 2 * pad, pad, (p->Cout + kMTile - 1) / kMTile, 148, &plan);
+    return plan_tc(d->N, Ho, Wo, p->ksize, d->stride, (p->Cout + kMTile - 1) / kMTile, 148, &plan);
 }
 
 int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y, const rtoss_conv_desc* d,
                          void* stream) {
-    const int pad = p->ksize == 3 ? 1 : 0;
     const int taps = p->ksize == 3 ? 9 : 1;
-    const int Wp = d->W + 2 * pad;
+    const int S = d->stride;
+    const int Ho = (d->H - 1) / S + 1, Wo = (d->W - 1) / S + 1;
     const int N_T = kMTile;
     const int sms = ctx->sm_count > 0 ? ctx->sm_count : 148;
     TcPlan plan;
-    if (!plan_tc(d->N, d->H, d->W, Wp, pad, (p->Cout + kMTile - 1) / kMTile, sms, &plan))
+    if (!plan_tc(d->N, Ho, Wo, p->ksize, S, (p->Cout + kMTile - 1) / kMTile, sms, &plan))
         return (int)cudaErrorInvalidConfiguration;
 
     TcArgs a;
@@ -522,26 +563,47 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     a.bias = d->bias_dev;
     a.status = ctx->dev_status;
     a.N = d->N;
-    a.H = d->H;
-    a.W = d->W;
+    a.Ho = Ho;
+    a.Wo = Wo;
+    a.S = S;
     a.Cin = p->Cin;
     a.Cout = p->Cout;
-    a.Wp = Wp;
+    a.Wq = plan.Wq;
     a.TH = plan.TH;
+    a.TW = plan.TW;
     a.taps = taps;
-    a.pad = pad;
+    a.tiles_x = plan.tiles_x;
+    a.n_sub = plan.n_sub;
+    a.sub_bytes = plan.sub_rows * kRowBytes;
+    for (int i = 0; i < 4; ++i) a.x_add[i] = a.y_add[i] = 0;
+    for (int t = 0; t < 9; ++t) a.tap_sub[t] = a.tap_shift[t] = 0;
+    if (p->ksize == 3 && S == 1) {
+        a.x_add[0] = a.y_add[0] = -1;
+        for (int t = 0; t < 9; ++t) a.tap_shift[t] = (t / 3) * plan.Wq + (t % 3);
+    } else if (p->ksize == 3) {
+        // sub-tile index = 2*(row parity) + (column parity); parity 0 = even input rows / columns
+        for (int sub = 0; sub < 4; ++sub) {
+            a.y_add[sub] = (sub >> 1) ? -1 : -2;
+            a.x_add[sub] = (sub & 1) ? -1 : -2;
+        }
+        for (int t = 0; t < 9; ++t) {
+            const int r = t / 3, c = t % 3;
+            a.tap_sub[t] = 2 * (r == 1 ? 0 : 1) + (c == 1 ? 0 : 1);
+            a.tap_shift[t] = (r == 0 ? 0 : 1) * plan.Wq + (c == 0 ? 0 : 1);
+        }
+    }
     a.N_px = plan.N_px;
     a.ncb = (p->Cin + kKBlock - 1) / kKBlock;
-    a.tiles_y = (d->H + plan.TH - 1) / plan.TH;
+    a.tiles_y = (Ho + plan.TH - 1) / plan.TH;
     a.co_tiles = (p->Cout + N_T - 1) / N_T;
-    a.a_stage_bytes = plan.a_rows * kRowBytes;
+    a.a_stage_bytes = plan.n_sub * plan.sub_rows * kRowBytes;
     a.b_stage_bytes = plan.G * N_T * kRowBytes;
     a.G = plan.G;
     a.NA = plan.NA;
     a.NB = plan.NB;
     a.AS = 2;
     a.acc_cols = round_up(plan.N_px, 32);  // the epilogue reads 32 columns at a time
-    a.a_tx_bytes = (unsigned)(kKBlock * 2 * Wp * (plan.TH + 2 * pad));
+    a.a_tx_bytes = (unsigned)(kKBlock * 2 * plan.Wq * plan.rows_staged);  // per sub-tile
     a.b_tx_bytes = (unsigned)(kKBlock * 2 * N_T);
     a.act = (int)d->act;
     a.y_c_off = d->y_channel_offset;
@@ -559,7 +621,7 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     if (!enc) return (int)cudaErrorNotSupported;
     const CUtensorMapDataType dt = a.is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
     // activations: descriptor cached per (pointer, shape, box)
-    const int key[6] = {d->N, d->H, d->W, p->Cin, plan.TH + 2 * pad, Wp * 4 + (int)p->dtype};
+    const int key[6] = {d->N, d->H, d->W, p->Cin, plan.rows_staged * 8 + S, plan.Wq * 4 + (int)p->dtype};
     rtoss_tmap_entry* ea = nullptr;
     for (rtoss_tmap_entry& e : ctx->tmap_cache)
         if (e.valid && e.base == x && memcmp(e.dims, key, sizeof(key)) == 0) ea = &e;
@@ -568,8 +630,9 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
         ctx->tmap_next = (ctx->tmap_next + 1) % 32;
         cuuint64_t dims[4] = {(cuuint64_t)p->Cin, (cuuint64_t)d->W, (cuuint64_t)d->H, (cuuint64_t)d->N};
         cuuint64_t strides[3] = {(cuuint64_t)p->Cin * 2, (cuuint64_t)d->W * p->Cin * 2, (cuuint64_t)d->H * d->W * p->Cin * 2};
-        cuuint32_t box[4] = {(cuuint32_t)kKBlock, (cuuint32_t)Wp, (cuuint32_t)(plan.TH + 2 * pad), 1};
-        cuuint32_t es[4] = {1, 1, 1, 1};
+        // with element strides the box is counted in traversed elements: S*n covers n fetched pixels
+        cuuint32_t box[4] = {(cuuint32_t)kKBlock, (cuuint32_t)(plan.Wq * S), (cuuint32_t)(plan.rows_staged * S), 1};
+        cuuint32_t es[4] = {1, (cuuint32_t)S, (cuuint32_t)S, 1};
         ea->valid = 0;
         CUresult r = enc(reinterpret_cast<CUtensorMap*>(ea->map), dt, 4, const_cast<void*>(x), dims, strides, box, es,
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -599,7 +662,7 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     const CUtensorMap& tmB = *reinterpret_cast<const CUtensorMap*>(eb->map);
     // at least half an SM's shared memory, so that a second CTA (which would wait for TMEM) never shares the SM
     const size_t smem = (size_t)(plan.smem > 116 * 1024 ? plan.smem : 116 * 1024);
-    const size_t n_tiles = (size_t)d->N * a.tiles_y * a.co_tiles;
+    const size_t n_tiles = (size_t)d->N * a.tiles_y * a.tiles_x * a.co_tiles;
     dim3 grid((unsigned)(n_tiles < (size_t)sms ? n_tiles : (size_t)sms));
     static bool attr_set = false;  // both instantiations may use up to the whole shared memory of an SM
     if (!attr_set) {

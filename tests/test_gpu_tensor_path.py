@@ -32,7 +32,7 @@ def test_tensor_path_smallest_case():
 
 
 CASES = [
-    # ksize, N, Cin, Cout, H, W, k, dt, act
+    # ksize, N, Cin, Cout, H, W, k, dt, act   (stride 1)
     (3, 1, 128, 128, 80, 80, 3, "bf16", "silu"),      # the 128-channel layer, one image
     (3, 2, 64, 64, 40, 40, 4, "bf16", "silu"),
     (3, 1, 32, 64, 20, 20, 4, "bf16", "relu"),        # half-filled channel block
@@ -50,6 +50,28 @@ CASES = [
     (3, 1, 24, 20, 9, 11, 3, "bf16", "silu"),         # filter count not a multiple of 16, 24 channels
     (1, 3, 8, 200, 5, 254, 2, "f16", "none"),         # widest image the path takes, filter tiles 128 + 72
 ]
+
+
+STRIDED_AND_WIDE = [
+    # ksize, stride, N, Cin, Cout, H, W, k, dt, act
+    (3, 2, 1, 64, 128, 40, 40, 4, "bf16", "silu"),     # downsampling conv, even size
+    (3, 2, 2, 128, 128, 25, 34, 4, "bf16", "relu"),    # odd height
+    (3, 2, 1, 32, 64, 13, 17, 3, "f16", "none"),       # both odd
+    (3, 2, 1, 72, 40, 9, 250, 2, "bf16", "silu"),      # wide, stride 2: column segments
+    (3, 2, 1, 256, 256, 2, 2, 4, "bf16", "none"),      # one output pixel
+    (1, 2, 1, 256, 512, 50, 68, 4, "bf16", "none"),    # strided 1x1 (downsample branch)
+    (1, 2, 2, 64, 32, 7, 9, 3, "f16", "relu"),
+    (3, 1, 1, 64, 64, 10, 272, 4, "bf16", "relu"),     # wider than one TMA box: column segments
+    (1, 1, 1, 64, 256, 6, 300, 4, "bf16", "relu"),
+    (3, 1, 1, 16, 24, 5, 700, 3, "f16", "silu"),
+]
+
+
+@pytest.mark.parametrize("case", STRIDED_AND_WIDE, ids=lambda c: "-".join(str(v) for v in c))
+def test_tensor_path_strided_and_wide(case):
+    ks, s, N, Cin, Cout, H, W, k, dt, act = case
+    gu.check_layer(25, 700 + Cin + W, ks, N, Cin, Cout, H, W, s, k, _table(k), dt, act, "nhwc", path=rt.PATH_TENSOR)
+    _no_timeout()
 
 
 @pytest.mark.parametrize("case", CASES, ids=lambda c: "-".join(str(v) for v in c))
@@ -108,9 +130,13 @@ def test_tensor_path_refuses_what_it_cannot_take():
     with pytest.raises(rt.RtossError) as e:                                  # NCHW is not taken by the tensor path
         gu.run_conv(packed, 3, x, "bf16", 1, "none", None, "nchw", path=rt.PATH_TENSOR)
     assert e.value.status == 3
-    with pytest.raises(rt.RtossError) as e:                                  # nor stride 2
-        gu.run_conv(packed, 3, x, "bf16", 2, "none", None, "nhwc", path=rt.PATH_TENSOR)
-    assert e.value.status == 3
-    y = gu.run_conv(packed, 3, x, "bf16", 2, "none", None, "nhwc", path=rt.PATH_AUTO)   # auto falls back to FMA
+    y = gu.run_conv(packed, 3, x, "bf16", 1, "none", None, "nchw", path=rt.PATH_AUTO)   # auto falls back to FMA
     assert np.isfinite(y).all()
+    packed.close()
+    w8 = synth.kaiming_weights(24, 2, 16, 12, 3)                             # Cin not a multiple of 8
+    _, packed = gu.select_pack(w8, 3, masks, 4, "bf16")
+    x8 = synth.round_like(synth.activations(24, 2, 1, 12, 8, 8), "bf16")
+    with pytest.raises(rt.RtossError) as e:
+        gu.run_conv(packed, 3, x8, "bf16", 1, "none", None, "nhwc", path=rt.PATH_TENSOR)
+    assert e.value.status == 3
     packed.close()
