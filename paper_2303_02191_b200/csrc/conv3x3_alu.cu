@@ -372,6 +372,106 @@ struct Variant {
     int S, PH, PW, CO_T;
 };
 
+// ---------------------------------------------------------------------------------------------
+// Layers with very few input channels (the 3-channel stem of a detector): one thread per output
+// pixel, its 3x3xCIN input neighbourhood in registers, 32 filters per thread in sequence with the
+// dense-expanded weights (pruned taps are zeros) broadcast from shared memory.  The layer is bound
+// by its output traffic; with 9*CIN <= 36 multiply-adds per output the zeros cost less than
+// skipping them would.
+constexpr int kStemCo = 32;
+
+template <typename T, int CIN>
+__global__ void __launch_bounds__(256) conv3x3_small_cin_kernel(const Conv3Args a, int stride) {
+    __shared__ float sWd[kStemCo][CIN * 9 + 1];  // [filter][ci*9 + tap], last = bias
+    __shared__ uint16_t smask[256];
+    const int co0 = blockIdx.y * kStemCo;
+    for (int p = threadIdx.x; p < 256; p += blockDim.x) smask[p] = p < a.P ? a.masks[p] : 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < kStemCo * CIN; i += blockDim.x) {
+        const int col = i / CIN, ci = i - col * CIN, co = co0 + col;
+        float wv[9];
+#pragma unroll
+        for (int t = 0; t < 9; ++t) wv[t] = 0.f;
+        if (co < a.Cout) {
+            const size_t kid = (size_t)co * CIN + ci;
+            const unsigned m = smask[a.pid[kid]];
+            size_t j = kid * a.k;
+#pragma unroll
+            for (int t = 0; t < 9; ++t)
+                if (m & (1u << t)) wv[t] = load_val(a.val, j++, a.val_dtype);
+        }
+#pragma unroll
+        for (int t = 0; t < 9; ++t) sWd[col][ci * 9 + t] = wv[t];
+        if (ci == 0) sWd[col][CIN * 9] = (a.bias && co < a.Cout) ? a.bias[co] : 0.f;
+    }
+    __syncthreads();
+
+    const long long total = (long long)a.N * a.Ho * a.Wo;
+    const long long pix = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (pix >= total) return;
+    const int ox = (int)(pix % a.Wo);
+    const long long r1 = pix / a.Wo;
+    const int oy = (int)(r1 % a.Ho), n = (int)(r1 / a.Ho);
+    const T* __restrict__ xg = reinterpret_cast<const T*>(a.x);
+    float xin[CIN][9];
+#pragma unroll
+    for (int r = 0; r < 3; ++r)
+#pragma unroll
+        for (int c = 0; c < 3; ++c) {
+            const int iy = oy * stride + r - 1, ix = ox * stride + c - 1;
+            const bool ok = iy >= 0 && iy < a.H && ix >= 0 && ix < a.W;
+#pragma unroll
+            for (int ci = 0; ci < CIN; ++ci) {
+                const size_t idx = a.layout == RTOSS_NCHW ? (((size_t)n * CIN + ci) * a.H + iy) * a.W + ix
+                                                          : (((size_t)n * a.H + iy) * a.W + ix) * CIN + ci;
+                xin[ci][r * 3 + c] = ok ? to_f32<T>(xg[idx]) : 0.f;
+            }
+        }
+    T* __restrict__ yg = reinterpret_cast<T*>(a.y);
+    const int Cs = a.y_c_stride;
+    const bool vec = a.layout == RTOSS_NHWC && (Cs * sizeof(T)) % 16 == 0 && ((a.y_c_off + co0) * sizeof(T)) % 16 == 0 &&
+                     co0 + kStemCo <= a.Cout;
+    constexpr int PER16 = 16 / (int)sizeof(T);
+    for (int c8 = 0; c8 < kStemCo; c8 += PER16) {
+        __align__(16) T o[PER16];
+#pragma unroll
+        for (int q = 0; q < PER16; ++q) {
+            const float* wr = sWd[c8 + q];
+            float acc = wr[CIN * 9];
+#pragma unroll
+            for (int i = 0; i < CIN * 9; ++i) acc = fmaf(wr[i], xin[i / 9][i % 9], acc);
+            o[q] = from_f32<T>(activate(acc, a.act));
+        }
+        if (vec) {
+            *reinterpret_cast<uint4*>(yg + (((size_t)n * a.Ho + oy) * a.Wo + ox) * Cs + a.y_c_off + co0 + c8) =
+                *reinterpret_cast<const uint4*>(o);
+        } else {
+#pragma unroll
+            for (int q = 0; q < PER16; ++q) {
+                const int co = co0 + c8 + q;
+                if (co < a.Cout) {
+                    const size_t idx = a.layout == RTOSS_NCHW ? (((size_t)n * Cs + a.y_c_off + co) * a.Ho + oy) * a.Wo + ox
+                                                              : (((size_t)n * a.Ho + oy) * a.Wo + ox) * Cs + a.y_c_off + co;
+                    yg[idx] = o[q];
+                }
+            }
+        }
+    }
+}
+
+template <typename T>
+int launch_small_cin(const Conv3Args& a, int stride, cudaStream_t stream) {
+    const long long total = (long long)a.N * a.Ho * a.Wo;
+    dim3 grid((unsigned)((total + 255) / 256), (unsigned)((a.Cout + kStemCo - 1) / kStemCo));
+    switch (a.Cin) {
+        case 1: conv3x3_small_cin_kernel<T, 1><<<grid, 256, 0, stream>>>(a, stride); break;
+        case 2: conv3x3_small_cin_kernel<T, 2><<<grid, 256, 0, stream>>>(a, stride); break;
+        case 3: conv3x3_small_cin_kernel<T, 3><<<grid, 256, 0, stream>>>(a, stride); break;
+        default: conv3x3_small_cin_kernel<T, 4><<<grid, 256, 0, stream>>>(a, stride); break;
+    }
+    return (int)cudaGetLastError();
+}
+
 // Pick the lane arrangement that wastes the fewest lanes and pixels.
 void choose_lanes(int Ho, int Wo, int PH, int PW, int* LX, int* LY) {
     double best = -1.0;
@@ -465,6 +565,7 @@ int launch_variant(Conv3Args& a, cudaStream_t stream) {
 
 template <typename T>
 int launch_typed(Conv3Args& a, int stride, cudaStream_t stream) {
+    if (a.Cin <= 4) return launch_small_cin<T>(a, stride, stream);
     if (stride == 1) return launch_variant<T, 1, 4, 8, 4>(a, stream);
     return launch_variant<T, 2, 2, 8, 4>(a, stream);
 }

@@ -93,6 +93,9 @@ SHAPES_3x3 = [
     (1, 8, 16, 11, 6, 1, 3, "f32", "none", "nchw", True),       # fp32 rows of 24 bytes
     (1, 16, 24, 30, 22, 1, 4, "f32", "silu", "nhwc", True),     # fp32 NHWC, two 16-byte vectors per pixel
     (1, 40, 36, 200, 272, 2, 4, "bf16", "relu", "nchw", False), # large image, stride 2, many tiles
+    (2, 3, 40, 20, 22, 1, 3, "f16", "silu", "nhwc", True),      # 3-channel stem kernel, NHWC, ragged filter block
+    (1, 4, 64, 16, 16, 2, 2, "bf16", "relu", "nhwc", False),    # 4-channel stem kernel, vector stores
+    (1, 2, 32, 9, 9, 1, 4, "f32", "none", "nchw", True),
 ]
 
 
