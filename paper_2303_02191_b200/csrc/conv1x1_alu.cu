@@ -4,10 +4,12 @@
 // nine and each run pruned to the k taps of its pattern (Section IV.D,
 // Algorithm 3 of arXiv 2303.02191).  Row co of the [Cout][Cin] matrix therefore
 // keeps about Cin*k/9 entries at irregular positions: a sparse-matrix x
-// dense-matrix product.  A thread keeps CO_T x 32 accumulators (CO_T filters,
-// 32 pixels); per input channel it loads its 32 activations once and, for each
-// of its filters, issues the 32 FMAs only when the (co,ci) weight survived
-// (warp-uniform keep bit, uniform branch).
+// dense-matrix product.  A thread keeps 8 x 16 accumulators (8 filters, 16
+// pixels); per input channel it loads its 16 activations and the 8 weights
+// (pruned ones are zeros) and issues all 128 FMAs.  Skipping the pruned
+// weights with a uniform branch per (filter, channel) was measured and lost: a
+// branch every 16-32 FMAs costs more than the zeros it avoids.  This is the
+// path for fp32 and for what the tensor path does not take.
 #include "conv_common.cuh"
 
 namespace {
@@ -17,10 +19,10 @@ using namespace rtoss_dev;
 constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
 constexpr int kCiChunk = 8;
-constexpr int kCoT = 4;
-constexpr int kCoBlock = kWarps * kCoT;  // 32
-constexpr int kPxThread = 32;
-constexpr int kPxTile = 32 * kPxThread;  // 1024 output pixels per CTA
+constexpr int kCoT = 8;
+constexpr int kCoBlock = kWarps * kCoT;  // 64
+constexpr int kPxThread = 16;
+constexpr int kPxTile = 32 * kPxThread;  // 512 output pixels per CTA
 
 struct Conv1Args {
     const void* x;
@@ -40,8 +42,7 @@ struct Conv1Args {
 template <typename T>
 __global__ void __launch_bounds__(kThreads, 1) conv1x1_alu_kernel(const Conv1Args a) {
     __shared__ __align__(16) float sX[kCiChunk][kPxTile];
-    __shared__ float sW[kCiChunk][kCoBlock];
-    __shared__ unsigned sBits[kCoBlock];
+    __shared__ __align__(16) float sW[kCiChunk][kCoBlock];
     __shared__ int tabG[kPxTile];
     __shared__ uint16_t smask[256];
 
@@ -110,34 +111,25 @@ __global__ void __launch_bounds__(kThreads, 1) conv1x1_alu_kernel(const Conv1Arg
                 sX[cl][e] = (g >= 0 && ci < a.Cin) ? to_f32<T>(img[(size_t)g * a.Cin + ci]) : 0.f;
             }
         }
-        // weights of this chunk: thread i -> (filter i/8, channel i%8); keep bits gathered by ballot
-        {
-            const int cl = tid & (kCiChunk - 1), col = tid >> 3;
+        // weights of this chunk, dense-expanded: position (co, ci) holds its value or 0
+        for (int i = tid; i < kCoBlock * kCiChunk; i += kThreads) {
+            const int cl = i & (kCiChunk - 1), col = i >> 3;
             const int co = co0 + col, ci = ci0 + cl;
             float w = 0.f;
-            bool keep = false;
             if (co < a.Cout && ci < a.Cin) {
                 const long long e = (long long)co * a.Cin + ci;
                 const long long g = e / 9;
                 const int t = (int)(e - 9 * g);
                 if (g < a.G) {
                     const unsigned m = smask[a.pid[g]];
-                    if (m & (1u << t)) {
-                        keep = true;
-                        w = load_val(a.val, (size_t)(g * a.k + __popc(m & ((1u << t) - 1u))), a.val_dtype);
-                    }
+                    if (m & (1u << t)) w = load_val(a.val, (size_t)(g * a.k + __popc(m & ((1u << t) - 1u))), a.val_dtype);
                 }
             }
             sW[cl][col] = w;
-            const unsigned ballot = __ballot_sync(0xFFFFFFFFu, keep);
-            if (cl == 0) sBits[col] = (ballot >> ((lane >> 3) * 8)) & 0xFFu;
         }
         __syncthreads();
 
-        unsigned bits[kCoT];
-#pragma unroll
-        for (int c = 0; c < kCoT; ++c) bits[c] = sBits[warp * kCoT + c];
-#pragma unroll 1
+#pragma unroll 2
         for (int cl = 0; cl < kCiChunk; ++cl) {
             float xv[kPxThread];
 #pragma unroll
@@ -145,14 +137,13 @@ __global__ void __launch_bounds__(kThreads, 1) conv1x1_alu_kernel(const Conv1Arg
                 const float4 v = *reinterpret_cast<const float4*>(&sX[cl][j * 128 + lane * 4]);
                 xv[4 * j] = v.x; xv[4 * j + 1] = v.y; xv[4 * j + 2] = v.z; xv[4 * j + 3] = v.w;
             }
+            const float4 wa = *reinterpret_cast<const float4*>(&sW[cl][warp * kCoT]);
+            const float4 wb = *reinterpret_cast<const float4*>(&sW[cl][warp * kCoT + 4]);
+            const float wv[kCoT] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
 #pragma unroll
-            for (int c = 0; c < kCoT; ++c) {
-                if ((bits[c] >> cl) & 1u) {
-                    const float w = sW[cl][warp * kCoT + c];
+            for (int c = 0; c < kCoT; ++c)
 #pragma unroll
-                    for (int i = 0; i < kPxThread; ++i) acc[c][i] = fmaf(w, xv[i], acc[c][i]);
-                }
-            }
+                for (int i = 0; i < kPxThread; ++i) acc[c][i] = fmaf(wv[c], xv[i], acc[c][i]);
         }
     }
 

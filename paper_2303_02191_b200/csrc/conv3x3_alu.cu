@@ -4,11 +4,11 @@
 // inference cost model of Section II.B of arXiv 2303.02191 (work proportional
 // to the non-zero weights).  Because every kernel (co,ci) picks its own
 // pattern, the kept (ci,tap) positions differ from filter to filter: this is a
-// gather of k taps per kernel, not a dense contraction, and it runs on the
-// plain FMA pipes.
+// gather of k taps per kernel, not a dense contraction.  This path runs it on
+// the plain FMA pipes (any dtype, layout and stride; the only path for fp32).
 //
 // Shape of the kernel
-//   * A CTA owns a spatial tile of one image and a block of kWarps*CO_T output
+//   * A CTA owns a spatial tile of one image and a block of WARPS*CO_T output
 //     channels.  All warps share the staged input tile; warp w owns CO_T
 //     consecutive filters, so the weights and the pattern a warp works on are
 //     warp-uniform (one broadcast shared-memory read, uniform branches).
@@ -17,10 +17,10 @@
 //     of PH x PW output pixels and keeps its (PH-1)S+3 x (PW-1)S+3 input window
 //     of the current input channel in registers.  That window is reused by the
 //     CO_T filters of the warp.
-//   * Per (filter, channel): the 9 dense-expanded weights and the pattern mask
-//     are read once; each tap whose mask bit is set runs PH*PW FMAs with static
-//     register indices; cleared taps are skipped by a uniform branch.  Only
-//     k*PH*PW FMAs are issued per kernel.
+//   * Per (filter, channel): the 9 dense-expanded weights (pruned taps = 0) are
+//     read once and all nine taps run PH*PW FMAs with static register indices.
+//     The sparsity is not skipped here (see the note in the compute loop); it
+//     pays through the packed weights' smaller HBM footprint only.
 //   * Input channels are processed kCiChunk at a time through a two-stage
 //     pipeline: while chunk i is being computed, the raw bytes of chunk i+1
 //     (activations in their storage type, packed values and pattern ids) arrive
@@ -37,8 +37,6 @@ namespace {
 
 using namespace rtoss_dev;
 
-constexpr int kWarps = 8;
-constexpr int kThreads = kWarps * 32;
 constexpr int kCiChunk = 8;
 constexpr int kWSlots = 12;  // 9 weights, mask, 2 pad: three float4 per kernel
 
@@ -82,11 +80,63 @@ __device__ __forceinline__ void fma_tap(float (&acc)[PH][PW], const float (&win)
         for (int px = 0; px < PW; ++px) acc[py][px] = fmaf(w, win[py * S + R][px * S + C], acc[py][px]);
 }
 
-template <typename T, int S, int PH, int PW, int CO_T>
-__global__ void __launch_bounds__(kThreads, 1) conv3x3_alu_kernel(const Conv3Args a) {
+template <int VB>
+__device__ __forceinline__ void cp_async_fixed(void* smem_dst, const void* gsrc) {
+    const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
+    if (VB == 16) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gsrc) : "memory");
+    else if (VB == 8) asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(s), "l"(gsrc) : "memory");
+    else asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(s), "l"(gsrc) : "memory");
+}
+
+// NCHW activations of one chunk: a thread owns raw vector e of EVERY channel of the chunk, so the table
+// entry is read once and the eight copies are independent of one another.
+template <typename T, int VB, int NTHREADS>
+__device__ __forceinline__ void issue_nchw(const T* chunk_base, size_t HW, int n_ch, const int* tab_g, int EV,
+                                           unsigned char* dst, int tid) {
+    for (int e = tid; e < EV; e += NTHREADS) {
+        const int g = tab_g[e];
+        if (g < 0) continue;
+        const T* src = chunk_base + g;
+        unsigned char* d = dst + (size_t)e * VB;
+#pragma unroll
+        for (int cl = 0; cl < kCiChunk; ++cl)
+            if (cl < n_ch) cp_async_fixed<VB>(d + (size_t)cl * EV * VB, src + (size_t)cl * HW);
+    }
+}
+
+// Conversion of the raw vectors into the fp32 tile, same ownership: table entries and the destination
+// bounds are worked out once per vector, then applied to the eight channels.
+template <typename T, int VB, int NTHREADS>
+__device__ __forceinline__ void convert_nchw(const unsigned char* src, int n_ch, const int* tab_g, const int* tab_s, int EV,
+                                             float* sX, int plane, int TWP, int tid) {
+    constexpr int VEQ = VB / (int)sizeof(T);
+    for (int e = tid; e < EV; e += NTHREADS) {
+        const bool inside = tab_g[e] >= 0;
+        const int s = tab_s[e];
+        const int r = s >> 16, c0 = (s & 0xFFFF) - 16;  // destination row, column of element 0 (>= -(VEQ-1))
+        float* drow = sX + r * TWP + c0;
+#pragma unroll
+        for (int cl = 0; cl < kCiChunk; ++cl) {
+            const bool ok = inside && cl < n_ch;
+            __align__(16) T v[VEQ];
+            if (VB == 16) *reinterpret_cast<uint4*>(v) = *reinterpret_cast<const uint4*>(src + ((size_t)cl * EV + e) * VB);
+            else if (VB == 8) *reinterpret_cast<uint2*>(v) = *reinterpret_cast<const uint2*>(src + ((size_t)cl * EV + e) * VB);
+            else *reinterpret_cast<unsigned*>(v) = *reinterpret_cast<const unsigned*>(src + ((size_t)cl * EV + e) * VB);
+#pragma unroll
+            for (int q = 0; q < VEQ; ++q) {
+                const int c = c0 + q;
+                if (c >= 0 && c < TWP) drow[cl * plane + q] = ok ? to_f32<T>(v[q]) : 0.f;
+            }
+        }
+    }
+}
+
+template <typename T, int S, int PH, int PW, int CO_T, int WARPS, int MINB>
+__global__ void __launch_bounds__(WARPS * 32, MINB) conv3x3_alu_kernel(const Conv3Args a) {
+    constexpr int kThreads = WARPS * 32;
     constexpr int WIN_H = (PH - 1) * S + 3;
     constexpr int WIN_W = (PW - 1) * S + 3;
-    constexpr int CO_BLOCK = kWarps * CO_T;
+    constexpr int CO_BLOCK = WARPS * CO_T;
 
     constexpr int VE16 = 16 / (int)sizeof(T);
     static_assert(kCiChunk == 8, "index arithmetic below assumes chunks of 8 channels");
@@ -159,15 +209,12 @@ __global__ void __launch_bounds__(kThreads, 1) conv3x3_alu_kernel(const Conv3Arg
     // ---- asynchronous part of staging chunk ci0 into raw buffer `buf`
     auto issue = [&](int ci0, int buf) {
         if (a.xmode == X_NCHW_VEC) {
-            const int ci = ci0 + warp;  // one warp per channel of the chunk
-            if (ci < a.Cin) {
-                const T* plane_ptr = xg + ((size_t)n * a.Cin + ci) * HW;
-                unsigned char* dst = rawX + (size_t)buf * a.rawX_bytes + (size_t)warp * a.EV * a.vb;
-                for (int e = lane; e < a.EV; e += 32) {
-                    const int g = tab_g[e];
-                    if (g >= 0) cp_async(dst + (size_t)e * a.vb, plane_ptr + g, a.vb);
-                }
-            }
+            const int n_ch = a.Cin - ci0 < kCiChunk ? a.Cin - ci0 : kCiChunk;
+            const T* chunk_base = xg + ((size_t)n * a.Cin + ci0) * HW;
+            unsigned char* dst = rawX + (size_t)buf * a.rawX_bytes;
+            if (a.vb == 16) issue_nchw<T, 16, kThreads>(chunk_base, HW, n_ch, tab_g, a.EV, dst, tid);
+            else if (a.vb == 8) issue_nchw<T, 8, kThreads>(chunk_base, HW, n_ch, tab_g, a.EV, dst, tid);
+            else issue_nchw<T, 4, kThreads>(chunk_base, HW, n_ch, tab_g, a.EV, dst, tid);
         } else if (a.xmode == X_NHWC_VEC) {
             constexpr int VPP = 8 / VE16;  // 16-byte vectors per pixel for 8 channels
             const T* img = xg + (size_t)n * HW * a.Cin + ci0;
@@ -198,21 +245,13 @@ __global__ void __launch_bounds__(kThreads, 1) conv3x3_alu_kernel(const Conv3Arg
     // ---- conversion of chunk ci0 (raw buffer `buf`, or straight from global memory) into sX / sW
     auto convert = [&](int ci0, int buf) {
         if (a.xmode == X_NCHW_VEC) {
-            const int ci = ci0 + warp;
-            const unsigned char* src = rawX + (size_t)buf * a.rawX_bytes + (size_t)warp * a.EV * a.vb;
-            float* dst = sX + warp * a.plane;
-            for (int e = lane; e < a.EV; e += 32) {
-                const bool ok = tab_g[e] >= 0 && ci < a.Cin;
-                const int s = tab_s[e];
-                const int r = s >> 16, c0 = (s & 0xFFFF) - 16;  // destination row, column of element 0 (>= -(veq-1))
-                const T* rv = reinterpret_cast<const T*>(src + (size_t)e * a.vb);
-#pragma unroll
-                for (int q = 0; q < VE16; ++q) {
-                    if (q < veq) {
-                        const int c = c0 + q;
-                        if (c >= 0 && c < a.TWP) dst[r * a.TWP + c] = ok ? to_f32<T>(rv[q]) : 0.f;
-                    }
-                }
+            const int n_ch = a.Cin - ci0 < kCiChunk ? a.Cin - ci0 : kCiChunk;
+            const unsigned char* src = rawX + (size_t)buf * a.rawX_bytes;
+            if (a.vb == 16) convert_nchw<T, 16, kThreads>(src, n_ch, tab_g, tab_s, a.EV, sX, a.plane, a.TWP, tid);
+            else if (a.vb == 8) {
+                if (sizeof(T) <= 4) convert_nchw<T, 8, kThreads>(src, n_ch, tab_g, tab_s, a.EV, sX, a.plane, a.TWP, tid);
+            } else {
+                if (sizeof(T) <= 4) convert_nchw<T, 4, kThreads>(src, n_ch, tab_g, tab_s, a.EV, sX, a.plane, a.TWP, tid);
             }
         } else if (a.xmode == X_NHWC_VEC) {
             const unsigned char* src = rawX + (size_t)buf * a.rawX_bytes;
@@ -313,16 +352,19 @@ __global__ void __launch_bounds__(kThreads, 1) conv3x3_alu_kernel(const Conv3Arg
                     n1 = wp[(c + 1) * 3 + 1];
                     n2 = wp[(c + 1) * 3 + 2];
                 }
-                const unsigned m = __float_as_uint(w2.y);
-                if (m & 0x001) fma_tap<S, PH, PW, 0, 0>(acc[c], win, w0.x);
-                if (m & 0x002) fma_tap<S, PH, PW, 0, 1>(acc[c], win, w0.y);
-                if (m & 0x004) fma_tap<S, PH, PW, 0, 2>(acc[c], win, w0.z);
-                if (m & 0x008) fma_tap<S, PH, PW, 1, 0>(acc[c], win, w0.w);
-                if (m & 0x010) fma_tap<S, PH, PW, 1, 1>(acc[c], win, w1.x);
-                if (m & 0x020) fma_tap<S, PH, PW, 1, 2>(acc[c], win, w1.y);
-                if (m & 0x040) fma_tap<S, PH, PW, 2, 0>(acc[c], win, w1.z);
-                if (m & 0x080) fma_tap<S, PH, PW, 2, 1>(acc[c], win, w1.w);
-                if (m & 0x100) fma_tap<S, PH, PW, 2, 2>(acc[c], win, w2.x);
+                // All nine taps, no branch: the pruned taps of a kernel are zeros in its expanded weights.
+                // Skipping them was measured and lost: with one pattern per (filter, channel) a skip is a
+                // branch every few dozen FMAs, and the dispatch instructions plus the instruction-fetch
+                // stalls after taken branches cost as much as the multiplications they avoid.
+                fma_tap<S, PH, PW, 0, 0>(acc[c], win, w0.x);
+                fma_tap<S, PH, PW, 0, 1>(acc[c], win, w0.y);
+                fma_tap<S, PH, PW, 0, 2>(acc[c], win, w0.z);
+                fma_tap<S, PH, PW, 1, 0>(acc[c], win, w0.w);
+                fma_tap<S, PH, PW, 1, 1>(acc[c], win, w1.x);
+                fma_tap<S, PH, PW, 1, 2>(acc[c], win, w1.y);
+                fma_tap<S, PH, PW, 2, 0>(acc[c], win, w1.z);
+                fma_tap<S, PH, PW, 2, 1>(acc[c], win, w1.w);
+                fma_tap<S, PH, PW, 2, 2>(acc[c], win, w2.x);
             }
         }
     }
@@ -473,14 +515,15 @@ int launch_small_cin(const Conv3Args& a, int stride, cudaStream_t stream) {
 }
 
 // Pick the lane arrangement that wastes the fewest lanes and pixels.
-void choose_lanes(int Ho, int Wo, int PH, int PW, int* LX, int* LY) {
+void choose_lanes(int Ho, int Wo, int PH, int PW, int S, int* LX, int* LY) {
     double best = -1.0;
     for (int lx = 1; lx <= 16; ++lx)
         for (int ly = 1; ly * lx <= 32; ++ly) {
             const int tw = lx * PW, th = ly * PH;
             const double cover = (double)((Wo + tw - 1) / tw * tw) * ((Ho + th - 1) / th * th);
             double util = (double)Wo * Ho / cover * (lx * ly) / 32.0;
-            util -= 1e-3 * (double)(tw + th) / (tw * th);  // tie-break: less halo per pixel
+            // staging cost grows with the halo: staged input pixels per output pixel
+            util /= 1.0 + 0.25 * ((double)((tw * S + 2) * (th * S + 2)) / (double)(tw * th * S * S) - 1.0);
             if (util > best) {
                 best = util;
                 *LX = lx;
@@ -491,11 +534,12 @@ void choose_lanes(int Ho, int Wo, int PH, int PW, int* LX, int* LY) {
 
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
-template <typename T, int S, int PH, int PW, int CO_T>
+template <typename T, int S, int PH, int PW, int CO_T, int WARPS, int MINB>
 int launch_variant(Conv3Args& a, cudaStream_t stream) {
-    constexpr int CO_BLOCK = kWarps * CO_T;
+    constexpr int CO_BLOCK = WARPS * CO_T;
+    constexpr int kThreads = WARPS * 32;
     const int es = (int)sizeof(T);
-    choose_lanes(a.Ho, a.Wo, PH, PW, &a.LX, &a.LY);
+    choose_lanes(a.Ho, a.Wo, PH, PW, S, &a.LX, &a.LY);
     a.tiles_x = (a.Wo + a.LX * PW - 1) / (a.LX * PW);
     a.tiles_y = (a.Ho + a.LY * PH - 1) / (a.LY * PH);
     a.TW_in = (a.LX * PW - 1) * S + 3;
@@ -507,7 +551,7 @@ int launch_variant(Conv3Args& a, cudaStream_t stream) {
     a.rawV_bytes = a.w_async ? CO_BLOCK * 8 * a.k * a.val_esize : 0;
     const int fixed_bytes = (int)sizeof(float) * kCiChunk * (a.plane + CO_BLOCK * kWSlots) + 2 * a.rawV_bytes +
                             (a.w_async ? 2 * CO_BLOCK * 8 : 0);
-    const int smem_cap = 200 * 1024;
+    const int smem_cap = (MINB > 1 ? 227 * 1024 / MINB - 1024 : 200 * 1024);  // leave room for MINB CTAs per SM
 
     // how the activations travel: cp.async where rows are aligned and the raw buffers fit, else plain loads
     a.xmode = X_SYNC;
@@ -555,7 +599,7 @@ int launch_variant(Conv3Args& a, cudaStream_t stream) {
     off += 2 * (int)sizeof(int) * n_tab;
     const size_t smem = (size_t)off;
     if (smem > 220 * 1024) return (int)cudaErrorInvalidConfiguration;
-    auto kern = conv3x3_alu_kernel<T, S, PH, PW, CO_T>;
+    auto kern = conv3x3_alu_kernel<T, S, PH, PW, CO_T, WARPS, MINB>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return (int)e;
     dim3 grid((unsigned)((size_t)a.tiles_x * a.tiles_y * a.N), (unsigned)((a.Cout + CO_BLOCK - 1) / CO_BLOCK));
@@ -566,8 +610,9 @@ int launch_variant(Conv3Args& a, cudaStream_t stream) {
 template <typename T>
 int launch_typed(Conv3Args& a, int stride, cudaStream_t stream) {
     if (a.Cin <= 4) return launch_small_cin<T>(a, stride, stream);
-    if (stride == 1) return launch_variant<T, 1, 4, 8, 4>(a, stream);
-    return launch_variant<T, 2, 2, 8, 4>(a, stream);
+    // one output row of eight pixels per lane, eight filters per warp, two CTAs per SM
+    if (stride == 1) return launch_variant<T, 1, 1, 8, 8, 8, 2>(a, stream);
+    return launch_variant<T, 2, 1, 8, 8, 8, 2>(a, stream);
 }
 
 }  // namespace
