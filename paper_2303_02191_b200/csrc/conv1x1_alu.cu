@@ -18,7 +18,8 @@ using namespace rtoss_dev;
 
 constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
-constexpr int kCiChunk = 8;
+constexpr int kCiChunk = 32;  // channels per staging round: long enough to amortise the two barriers and the load latency
+constexpr int kCiShift = 5;
 constexpr int kCoT = 8;
 constexpr int kCoBlock = kWarps * kCoT;  // 64
 constexpr int kPxThread = 16;
@@ -41,8 +42,9 @@ struct Conv1Args {
 
 template <typename T>
 __global__ void __launch_bounds__(kThreads, 1) conv1x1_alu_kernel(const Conv1Args a) {
-    __shared__ __align__(16) float sX[kCiChunk][kPxTile];
-    __shared__ __align__(16) float sW[kCiChunk][kCoBlock];
+    extern __shared__ __align__(16) unsigned char smem_dyn[];
+    float (*sX)[kPxTile] = reinterpret_cast<float (*)[kPxTile]>(smem_dyn);                                              // [kCiChunk][kPxTile]
+    float (*sW)[kCoBlock] = reinterpret_cast<float (*)[kCoBlock]>(smem_dyn + sizeof(float) * kCiChunk * kPxTile);  // [kCiChunk][kCoBlock]
     __shared__ int tabG[kPxTile];
     __shared__ uint16_t smask[256];
 
@@ -105,7 +107,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv1x1_alu_kernel(const Conv1Arg
         } else {
             const T* img = xg + (size_t)n * HW * a.Cin;
             for (int i = tid; i < kPxTile * kCiChunk; i += kThreads) {
-                const int cl = i & (kCiChunk - 1), e = i >> 3;
+                const int cl = i & (kCiChunk - 1), e = i >> kCiShift;
                 const int ci = ci0 + cl;
                 const int g = tabG[e];
                 sX[cl][e] = (g >= 0 && ci < a.Cin) ? to_f32<T>(img[(size_t)g * a.Cin + ci]) : 0.f;
@@ -113,7 +115,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv1x1_alu_kernel(const Conv1Arg
         }
         // weights of this chunk, dense-expanded: position (co, ci) holds its value or 0
         for (int i = tid; i < kCoBlock * kCiChunk; i += kThreads) {
-            const int cl = i & (kCiChunk - 1), col = i >> 3;
+            const int cl = i & (kCiChunk - 1), col = i >> kCiShift;
             const int co = co0 + col, ci = ci0 + cl;
             float w = 0.f;
             if (co < a.Cout && ci < a.Cin) {
@@ -213,10 +215,19 @@ int rtoss_launch_conv1x1(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     a.y_c_stride = d->y_channel_stride ? d->y_channel_stride : p->Cout;
     dim3 grid((unsigned)((size_t)a.tiles * a.N), (unsigned)((a.Cout + kCoBlock - 1) / kCoBlock));
     cudaStream_t s = (cudaStream_t)stream;
+    const int smem = (int)sizeof(float) * kCiChunk * (kPxTile + kCoBlock);
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(conv1x1_alu_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(conv1x1_alu_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(conv1x1_alu_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return (int)e;
+        attr_set = true;
+    }
     switch (d->io_dtype) {
-        case RTOSS_F32: conv1x1_alu_kernel<float><<<grid, kThreads, 0, s>>>(a); break;
-        case RTOSS_BF16: conv1x1_alu_kernel<__nv_bfloat16><<<grid, kThreads, 0, s>>>(a); break;
-        case RTOSS_F16: conv1x1_alu_kernel<__half><<<grid, kThreads, 0, s>>>(a); break;
+        case RTOSS_F32: conv1x1_alu_kernel<float><<<grid, kThreads, smem, s>>>(a); break;
+        case RTOSS_BF16: conv1x1_alu_kernel<__nv_bfloat16><<<grid, kThreads, smem, s>>>(a); break;
+        case RTOSS_F16: conv1x1_alu_kernel<__half><<<grid, kThreads, smem, s>>>(a); break;
     }
     return (int)cudaGetLastError();
 }
