@@ -19,11 +19,12 @@ using namespace rtoss_dev;
 constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
 constexpr int kCiChunk = 32;  // channels per staging round: long enough to amortise the two barriers and the load latency
-constexpr int kCiShift = 5;
 constexpr int kCoT = 8;
 constexpr int kCoBlock = kWarps * kCoT;  // 64
 constexpr int kPxThread = 16;
 constexpr int kPxTile = 32 * kPxThread;  // 512 output pixels per CTA
+constexpr int kXPitch = kPxTile + 4;     // floats per staged channel row: +4 keeps 16-byte alignment and spreads
+                                         // eight consecutive channels over distinct banks
 
 struct Conv1Args {
     const void* x;
@@ -43,8 +44,8 @@ struct Conv1Args {
 template <typename T>
 __global__ void __launch_bounds__(kThreads, 1) conv1x1_alu_kernel(const Conv1Args a) {
     extern __shared__ __align__(16) unsigned char smem_dyn[];
-    float (*sX)[kPxTile] = reinterpret_cast<float (*)[kPxTile]>(smem_dyn);                                              // [kCiChunk][kPxTile]
-    float (*sW)[kCoBlock] = reinterpret_cast<float (*)[kCoBlock]>(smem_dyn + sizeof(float) * kCiChunk * kPxTile);  // [kCiChunk][kCoBlock]
+    float (*sX)[kXPitch] = reinterpret_cast<float (*)[kXPitch]>(smem_dyn);                                              // [kCiChunk][kXPitch]
+    float (*sW)[kCoBlock] = reinterpret_cast<float (*)[kCoBlock]>(smem_dyn + sizeof(float) * kCiChunk * kXPitch);  // [kCiChunk][kCoBlock]
     __shared__ int tabG[kPxTile];
     __shared__ uint16_t smask[256];
 
@@ -105,17 +106,21 @@ __global__ void __launch_bounds__(kThreads, 1) conv1x1_alu_kernel(const Conv1Arg
                 }
             }
         } else {
+            // NHWC: a warp takes eight consecutive channels of four pixels per step (16-byte runs in memory,
+            // 32 distinct banks in shared memory)
             const T* img = xg + (size_t)n * HW * a.Cin;
-            for (int i = tid; i < kPxTile * kCiChunk; i += kThreads) {
-                const int cl = i & (kCiChunk - 1), e = i >> kCiShift;
-                const int ci = ci0 + cl;
-                const int g = tabG[e];
-                sX[cl][e] = (g >= 0 && ci < a.Cin) ? to_f32<T>(img[(size_t)g * a.Cin + ci]) : 0.f;
+            for (int cg = 0; cg < kCiChunk; cg += 8) {
+                for (int i = tid; i < kPxTile * 8; i += kThreads) {
+                    const int cl = cg + (i & 7), e = i >> 3;
+                    const int ci = ci0 + cl;
+                    const int g = tabG[e];
+                    sX[cl][e] = (g >= 0 && ci < a.Cin) ? to_f32<T>(img[(size_t)g * a.Cin + ci]) : 0.f;
+                }
             }
         }
         // weights of this chunk, dense-expanded: position (co, ci) holds its value or 0
         for (int i = tid; i < kCoBlock * kCiChunk; i += kThreads) {
-            const int cl = i & (kCiChunk - 1), col = i >> kCiShift;
+            const int cl = i & (kCiChunk - 1), col = i / kCiChunk;
             const int co = co0 + col, ci = ci0 + cl;
             float w = 0.f;
             if (co < a.Cout && ci < a.Cin) {
@@ -215,7 +220,7 @@ int rtoss_launch_conv1x1(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     a.y_c_stride = d->y_channel_stride ? d->y_channel_stride : p->Cout;
     dim3 grid((unsigned)((size_t)a.tiles * a.N), (unsigned)((a.Cout + kCoBlock - 1) / kCoBlock));
     cudaStream_t s = (cudaStream_t)stream;
-    const int smem = (int)sizeof(float) * kCiChunk * (kPxTile + kCoBlock);
+    const int smem = (int)sizeof(float) * kCiChunk * (kXPitch + kCoBlock);
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(conv1x1_alu_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
