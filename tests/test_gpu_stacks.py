@@ -64,3 +64,41 @@ def test_retinanet_stack_unique_layers_batch4_sampled():
         packed.close()
         del x, y
     assert gu.ctx().rtoss_device_status() == 0
+
+
+SWEEP_SUBSET = [(dt, C, HW, k) for dt in ("bf16", "f32") for C in (64, 256) for HW in (20, 40) for k in (2, 3, 4, 9)]
+
+
+@pytest.mark.parametrize("dt,C,HW,k", SWEEP_SUBSET, ids=lambda v: str(v))
+def test_sweep_points_batch1_full_tensor(dt, C, HW, k):
+    """Points of the isolated-3x3 sweep the oracle finishes quickly, in the sweep's own launch configuration:
+    bf16 NHWC (automatic path) and fp32 NCHW."""
+    preset = {2: orc.PRESET_CONN4, 3: orc.PRESET_CONN4, 4: orc.PRESET_CENTRE8, 9: orc.PRESET_DENSE}[k]
+    masks = orc.pattern_preset(k, preset)
+    gu.check_layer(42, 800 + C + HW + k, 3, 1, C, C, HW, HW, 1, k, masks, dt, "silu", "nhwc" if dt == "bf16" else "nchw")
+
+
+def test_sweep_large_point_sampled():
+    """The largest point of the sweep (C = 512, 160 x 160, batch 32 is cut to batch 2 to bound memory and time)
+    on sampled outputs, both dtypes."""
+    rng = np.random.default_rng(12)
+    masks = orc.pattern_preset(4, orc.PRESET_CENTRE8)
+    N, C, HW = 2, 512, 160
+    w = synth.kaiming_weights(43, 1, C, C, 3)
+    b = synth.bias(43, 1, C)
+    for dt, layout in (("bf16", "nhwc"), ("f32", "nchw")):
+        x = synth.round_like(synth.activations(43, 1, N, C, HW, HW), dt)
+        pid_g, packed = gu.select_pack(w, 3, masks, 4, dt)
+        pid_o, wd, _ = gu.oracle_weights(w, 3, masks, 4, dt)
+        assert np.array_equal(pid_g, pid_o.ravel())
+        y = gu.run_conv(packed, 3, x, dt, 1, "silu", b, layout)
+        npts = 2000
+        idx = np.stack([rng.integers(0, N, npts), rng.integers(0, C, npts), rng.integers(0, HW, npts),
+                        rng.integers(0, HW, npts)], axis=1).astype(np.int32)
+        idx[:3] = [[0, 0, 0, 0], [N - 1, C - 1, HW - 1, HW - 1], [0, C - 1, 0, HW - 1]]
+        ref = orc.conv_points(3, x, wd, b, 1, orc.ACT_SILU, gu.ORC_DT[dt], idx)
+        got = y[idx[:, 0], idx[:, 1], idx[:, 2], idx[:, 3]]
+        rms = float(np.sqrt(np.mean(ref.astype(np.float64) ** 2)))
+        assert np.max(np.abs(got - ref) / np.maximum(np.abs(ref), rms)) <= gu.TOL[dt]
+        packed.close()
+    assert gu.ctx().rtoss_device_status() == 0
