@@ -231,7 +231,9 @@ rtoss_status rtoss_device_status(rtoss_ctx* ctx, int* code);
 
 /* Same convolutions with HOST buffers: copies x to the device, runs the
  * kernel for the handle's ksize, copies y back and waits for it.  x_host and
- * y_host are dense tensors in desc's layout and dtype (y_channel_* apply).
+ * y_host are dense tensors in desc's layout and dtype (y_channel_* apply).  The batch is cut into chunks of
+ * images whose copies and kernels overlap on three internal streams; pinned host memory is needed for
+ * the copies to be asynchronous.
  * Uses (and grows on demand) the context's device workspace, so concurrent
  * calls on one context are not allowed.  bias_dev stays a device pointer. */
 rtoss_status rtoss_conv_pattern_host(rtoss_ctx* ctx, const rtoss_packed* p, const void* x_host, void* y_host,

@@ -134,8 +134,14 @@ void rtoss_destroy(rtoss_ctx* ctx) {
     cudaGetDevice(&prev);
     cudaSetDevice(ctx->device);
     if (ctx->h_stream) {
-        cudaStreamSynchronize((cudaStream_t)ctx->h_stream);
+        cudaDeviceSynchronize();
         cudaStreamDestroy((cudaStream_t)ctx->h_stream);
+        cudaStreamDestroy((cudaStream_t)ctx->h_stream2);
+        cudaStreamDestroy((cudaStream_t)ctx->h_stream3);
+        for (int i = 0; i < kHostChunks; ++i) {
+            if (ctx->h_ev_in[i]) cudaEventDestroy((cudaEvent_t)ctx->h_ev_in[i]);
+            if (ctx->h_ev_run[i]) cudaEventDestroy((cudaEvent_t)ctx->h_ev_run[i]);
+        }
     }
     if (ctx->ws_x) cudaFree(ctx->ws_x);
     if (ctx->ws_y) cudaFree(ctx->ws_y);
@@ -361,10 +367,19 @@ rtoss_status rtoss_conv_pattern_host(rtoss_ctx* ctx, const rtoss_packed* p, cons
     const size_t yb = (size_t)desc->N * cs * Ho * Wo * es;
     cudaError_t e = cudaSuccess;
     if (!ctx->h_stream) {
-        cudaStream_t s;
-        e = cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking);
-        if (e != cudaSuccess) return cuda_fail(ctx, "host path stream", (int)e);
-        ctx->h_stream = s;
+        cudaStream_t st3[3] = {nullptr, nullptr, nullptr};
+        for (int i = 0; i < 3 && e == cudaSuccess; ++i) e = cudaStreamCreateWithFlags(&st3[i], cudaStreamNonBlocking);
+        for (int i = 0; i < kHostChunks && e == cudaSuccess; ++i) {
+            cudaEvent_t ev;
+            e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+            ctx->h_ev_in[i] = ev;
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+            ctx->h_ev_run[i] = ev;
+        }
+        if (e != cudaSuccess) return cuda_fail(ctx, "host path streams", (int)e);
+        ctx->h_stream = st3[0];
+        ctx->h_stream2 = st3[1];
+        ctx->h_stream3 = st3[2];
     }
     if (ctx->ws_x_bytes < xb) {
         if (ctx->ws_x) cudaFree(ctx->ws_x);
@@ -388,18 +403,48 @@ rtoss_status rtoss_conv_pattern_host(rtoss_ctx* ctx, const rtoss_packed* p, cons
         }
         ctx->ws_y_bytes = yb;
     }
-    cudaStream_t s = (cudaStream_t)ctx->h_stream;
+    // Three streams, the batch cut into image chunks: the copy-in of chunk c+1, the kernel of chunk c and the
+    // copy-out of chunk c-1 overlap (PCIe is full duplex), so a call costs about max(copy in, copy out).
     const bool slice = cs != p->Cout;
-    e = cudaMemcpyAsync(ctx->ws_x, x_host, xb, cudaMemcpyHostToDevice, s);
-    // a channel slice leaves the other channels of y untouched: bring the caller's y over first
-    if (e == cudaSuccess && slice) e = cudaMemcpyAsync(ctx->ws_y, y_host, yb, cudaMemcpyHostToDevice, s);
-    if (e != cudaSuccess) return cuda_fail(ctx, "host path copy in", (int)e);
-    int le = dispatch_conv(ctx, p, ctx->ws_x, ctx->ws_y, desc, s, &st);
-    if (st != RTOSS_OK) return st;
-    if (le) return cuda_fail(ctx, "host path launch", le);
-    e = cudaMemcpyAsync(y_host, ctx->ws_y, yb, cudaMemcpyDeviceToHost, s);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
-    return e == cudaSuccess ? RTOSS_OK : cuda_fail(ctx, "host path copy out", (int)e);
+    const size_t x_img = (size_t)p->Cin * desc->H * desc->W * es, y_img = (size_t)cs * Ho * Wo * es;
+    int n_chunks = desc->N < kHostChunks ? desc->N : kHostChunks;
+    while (n_chunks > 1 && (xb + yb) / n_chunks < ((size_t)1 << 20)) --n_chunks;  // not below ~1 MB per chunk
+    cudaStream_t s_in = (cudaStream_t)ctx->h_stream, s_run = (cudaStream_t)ctx->h_stream2, s_out = (cudaStream_t)ctx->h_stream3;
+    rtoss_conv_desc dc = *desc;
+    int done = 0;
+    for (int c = 0; c < n_chunks && e == cudaSuccess; ++c) {
+        const int n_c = (desc->N - done + (n_chunks - c) - 1) / (n_chunks - c);
+        char* xd = static_cast<char*>(ctx->ws_x) + (size_t)done * x_img;
+        char* yd = static_cast<char*>(ctx->ws_y) + (size_t)done * y_img;
+        e = cudaMemcpyAsync(xd, static_cast<const char*>(x_host) + (size_t)done * x_img, (size_t)n_c * x_img,
+                            cudaMemcpyHostToDevice, s_in);
+        // a channel slice leaves the other channels of y untouched: bring the caller's y over first
+        if (e == cudaSuccess && slice)
+            e = cudaMemcpyAsync(yd, static_cast<const char*>(y_host) + (size_t)done * y_img, (size_t)n_c * y_img,
+                                cudaMemcpyHostToDevice, s_in);
+        if (e == cudaSuccess) e = cudaEventRecord((cudaEvent_t)ctx->h_ev_in[c], s_in);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s_run, (cudaEvent_t)ctx->h_ev_in[c], 0);
+        if (e != cudaSuccess) break;
+        dc.N = n_c;
+        int le = dispatch_conv(ctx, p, xd, yd, &dc, s_run, &st);
+        if (st != RTOSS_OK || le) {
+            cudaDeviceSynchronize();
+            if (st != RTOSS_OK) return st;
+            return cuda_fail(ctx, "host path launch", le);
+        }
+        e = cudaEventRecord((cudaEvent_t)ctx->h_ev_run[c], s_run);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s_out, (cudaEvent_t)ctx->h_ev_run[c], 0);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(static_cast<char*>(y_host) + (size_t)done * y_img, yd, (size_t)n_c * y_img,
+                                cudaMemcpyDeviceToHost, s_out);
+        done += n_c;
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s_out);
+    if (e != cudaSuccess) {
+        cudaDeviceSynchronize();
+        return cuda_fail(ctx, "host path", (int)e);
+    }
+    return RTOSS_OK;
 }
 
 }  // extern "C"

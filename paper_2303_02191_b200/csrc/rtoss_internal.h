@@ -15,6 +15,8 @@ struct rtoss_tmap_entry {
     alignas(64) unsigned char map[128];
 };
 
+constexpr int kHostChunks = 8;  // the host-buffer path cuts a batch into at most this many chunks
+
 struct rtoss_ctx {
     int device;
     int sm_count;
@@ -24,7 +26,11 @@ struct rtoss_ctx {
     size_t ws_x_bytes;
     void* ws_y;
     size_t ws_y_bytes;
-    void* h_stream;  // cudaStream_t owned by the context, used by the host-buffer path
+    void* h_stream;  // cudaStream_t owned by the context: copies in of the host-buffer path
+    void* h_stream2;  // its kernels
+    void* h_stream3;  // its copies out
+    void* h_ev_in[8];   // cudaEvent_t per batch chunk: copy in done
+    void* h_ev_run[8];  // kernel done
     int* dev_status;  // device word: 0, or the code of a bounded device-side wait that ran out
     mutable rtoss_tmap_entry tmap_cache[32];  // activation descriptors of the tensor path, round robin
     mutable int tmap_next;

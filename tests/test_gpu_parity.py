@@ -210,6 +210,22 @@ def test_host_buffer_entry_point(ksize):
     gu.check_layer(9, 300 + ksize, ksize, 2, 32, 48, 20, 24, 1, 4, _table(4), "bf16", "silu", host=True)
 
 
+def test_host_buffer_entry_point_chunked_batch():
+    """A batch large enough to be cut into overlapping chunks (uneven: 7 images), both layouts, and a channel slice."""
+    gu.check_layer(9, 310, 3, 7, 64, 64, 48, 40, 1, 4, _table(4), "bf16", "relu", layout="nhwc", host=True)
+    gu.check_layer(9, 311, 1, 7, 64, 96, 48, 40, 2, 3, _table(3), "f32", "silu", layout="nchw", host=True)
+    masks = _table(4)
+    x = synth.round_like(synth.activations(9, 312, 6, 32, 40, 40), "bf16")
+    w = synth.kaiming_weights(9, 312, 48, 32, 3)
+    _, packed = gu.select_pack(w, 3, masks, 4, "bf16")
+    _, wd, _ = gu.oracle_weights(w, 3, masks, 4, "bf16")
+    y = gu.run_conv(packed, 3, x, "bf16", 1, "none", None, "nhwc", y_off=8, y_stride=64, host=True)
+    ref = gu.oracle_conv(3, x, wd, None, 1, "none", "bf16")
+    assert orc.rel_err(y[:, 8:56], ref) <= 2e-2
+    assert (y[:, :8] == 7.0).all() and (y[:, 56:] == 7.0).all()
+    packed.close()
+
+
 def test_argument_errors_return_status_codes():
     c = gu.ctx()
     masks = _table(4)
