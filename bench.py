@@ -260,7 +260,8 @@ def run_gpu(args):
         for wt in weights.values():
             ctx.rtoss_select_patterns(wt["w"], wt["ksize"], wt["masks"], wt["k"], pid=wt["pid"])
             wt["packed"] = ctx.rtoss_pack(wt["w"], wt["ksize"], wt["masks"], wt["k"], wt["pid"], cdt, into=wt["packed"])
-            launches += 3 if wt["ksize"] == 3 else 2
+            # select, pack values, (3x3: pack order), and for handles the tensor path can use the dense expansion
+            launches += (3 if wt["ksize"] == 3 else 2) + (1 if (dtype != "f32" and wt["w"].shape[1] % 8 == 0) else 0)
         return launches
 
     def conv(st, ev=None):
