@@ -256,3 +256,27 @@ def test_argument_errors_return_status_codes():
     c.rtoss_conv3x3_pattern(packed, x, y, 1, 6, 6)                            # the context stays usable
     torch.cuda.synchronize()
     packed.close()
+
+
+def test_children_inherit_the_parent_layers_patterns():
+    """Layer grouping (Algorithm 1) lets the layers of a group share kernel patterns: a child is packed with its
+    PARENT's pattern ids (same shape, identity mapping of (co, ci)) instead of being re-selected."""
+    masks = _table(3)
+    nodes = [dict(kind="conv", cin=24, cout=24, ksize=3, inputs=[]), dict(kind="conv", cin=24, cout=24, ksize=3, inputs=[0]),
+             dict(kind="op", inputs=[0, 1]), dict(kind="conv", cin=24, cout=24, ksize=3, inputs=[2])]
+    parent, group, ng = rt.rtoss_group_layers(nodes)
+    assert ng == 1 and parent.tolist() == [0, 0, -1, 0]
+    c = gu.ctx()
+    w_parent = synth.kaiming_weights(50, 1, 24, 24, 3)
+    pid_parent = c.rtoss_select_patterns(torch.from_numpy(w_parent).cuda(), 3, masks, 3)
+    pid_o = orc.select_3x3(w_parent, masks)
+    assert np.array_equal(pid_parent.cpu().numpy(), pid_o.ravel())
+    for child in (1, 3):
+        w_child = synth.kaiming_weights(50, 1 + child, 24, 24, 3)
+        packed = c.rtoss_pack(torch.from_numpy(w_child).cuda(), 3, masks, 3, pid_parent, rt.F32)
+        dense = packed.to_dense().cpu().numpy()
+        assert np.array_equal(dense, orc.mask_3x3(w_child, masks, pid_o))          # the parent's masks on the child's weights
+        x = synth.activations(50, 9, 1, 24, 10, 10)
+        y = gu.run_conv(packed, 3, x, "f32", 1, "none", None)
+        assert orc.rel_err(y, gu.oracle_conv(3, x, dense, None, 1, "none", "f32")) <= 1e-4
+        packed.close()
