@@ -209,6 +209,58 @@ def whole_job_value(images_per_rank, world, ms_per_step):
 
 # --------------------------------------------------------------------------- GPU arm
 
+def run_network(args):
+    """Whole-network replay of the YOLOv5s-shaped backbone + neck (convolutions + glue) as one CUDA graph."""
+    import torch
+    from paper_2303_02191_b200 import binding as rt
+    from paper_2303_02191_b200.yolov5s_net import GpuNet
+    N = 1 if args.workload.endswith("b1") else 16
+    torch.cuda.set_device(0)
+    ctx = rt.Context(0)
+    net = GpuNet(ctx, N)
+    xh = synth.round_like(synth.activations(0, 1, N, 3, 640, 640), "bf16")
+    net.set_input(xh)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for _ in range(max(args.warmup, 3)):
+            net.run()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        net.run()
+    graph.replay()
+    torch.cuda.synchronize()
+    if ctx.rtoss_device_status() != 0:
+        raise SystemExit("a device-side wait of the tensor path ran out")
+    sampler = ClockSampler(physical_gpu_index(0))
+    sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for s in range(args.steps):
+        flush.zero_()
+        ev[s][0].record()
+        graph.replay()
+        ev[s][1].record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = float(np.mean([a.elapsed_time(b) for a, b in ev]))
+    flops = sum(synth.layer_nnz_flops(L, N, 4) for L in net.layers)
+    n_glue = sum(1 for op in net.ops if op[0] != "conv")
+    print(json.dumps({
+        "metric": "pattern-sparse conv images/sec", "value": N / (ms * 1e-3), "unit": "images/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "batch": N, "layout": "NHWC", "l2": "flushed between steps (256 MB write)",
+                   "launch": "one CUDA graph per step", "convs": len(net.layers), "glue_kernels": n_glue,
+                   "note": "chained network: every layer consumes the previous layer's output"},
+        "nnz_gflops_per_s": flops / (ms * 1e-3) / 1e9, "clocks": clocks, "gpu_launches": (len(net.layers) + n_glue) * args.steps,
+    }))
+    net.close()
+    ctx.close()
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -447,6 +499,9 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.workload in ("yolov5s_net_b1", "yolov5s_net_b16"):
+        run_network(args)
         return
     if int(os.environ.get("WORLD_SIZE", "1")) > 1 or args.gpus == 1:
         if int(os.environ.get("WORLD_SIZE", "1")) > 1:

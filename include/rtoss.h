@@ -239,6 +239,25 @@ rtoss_status rtoss_device_status(rtoss_ctx* ctx, int* code);
 rtoss_status rtoss_conv_pattern_host(rtoss_ctx* ctx, const rtoss_packed* p, const void* x_host, void* y_host,
                                      const rtoss_conv_desc* desc);
 
+/* ---- glue between the convolutions of a whole network ---------------------- */
+/* Not part of the paper's method (Table 3 and Fig. 6 time whole models, whose graphs need these between the
+ * pruned convolutions).  Element-wise, bandwidth-bound; x and y in the given layout and dtype; y may be a
+ * channel slice [offset, offset + C) of a tensor with y_channel_stride channels (0 = C), which makes a
+ * concatenation a write.  Errors: RTOSS_ERR_INVALID_ARG, RTOSS_ERR_CUDA. */
+
+/* k x k max-pooling, given stride and padding (pad <= k/2; padded positions never win):
+ * Ho = (H + 2*pad - k)/stride + 1. */
+rtoss_status rtoss_maxpool2d(const void* x_dev, void* y_dev, int N, int C, int H, int W, int k, int stride, int pad,
+                             rtoss_layout layout, rtoss_dtype dtype, int y_channel_offset, int y_channel_stride,
+                             void* cuda_stream);
+/* Nearest-neighbour up-sampling by 2: y[n,c,oh,ow] = x[n,c,oh/2,ow/2], output 2H x 2W. */
+rtoss_status rtoss_upsample2x(const void* x_dev, void* y_dev, int N, int C, int H, int W, rtoss_layout layout,
+                              rtoss_dtype dtype, int y_channel_offset, int y_channel_stride, void* cuda_stream);
+/* y = act(a + b) over n_elements contiguous elements (residual connections); the sum is formed in fp32 and
+ * rounded once.  y may alias a or b. */
+rtoss_status rtoss_add_act(const void* a_dev, const void* b_dev, void* y_dev, int64_t n_elements, rtoss_dtype dtype,
+                           rtoss_act act, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -472,3 +472,35 @@ int oracle_group_layers(int L, const int *kind, const int *cout, const int *cin,
     }
     return ngroups;
 }
+
+/* ---- glue operations of a whole network (outside the paper's method; NCHW) ---- */
+
+/* k x k max-pooling with stride; padded positions are ignored (they count as minus infinity). */
+void oracle_maxpool2d(const float *x, int N, int C, int H, int W, int k, int stride, int pad, float *y) {
+    int Ho = (H + 2 * pad - k) / stride + 1, Wo = (W + 2 * pad - k) / stride + 1;
+    for (long nc = 0; nc < (long)N * C; ++nc)
+        for (int oh = 0; oh < Ho; ++oh)
+            for (int ow = 0; ow < Wo; ++ow) {
+                float m = -INFINITY;
+                for (int dy = 0; dy < k; ++dy)
+                    for (int dx = 0; dx < k; ++dx) {
+                        int ih = oh * stride + dy - pad, iw = ow * stride + dx - pad;
+                        if (ih < 0 || ih >= H || iw < 0 || iw >= W) continue;
+                        float v = x[(nc * H + ih) * W + iw];
+                        if (v > m) m = v;
+                    }
+                y[(nc * Ho + oh) * Wo + ow] = m;
+            }
+}
+
+/* nearest-neighbour up-sampling by two */
+void oracle_upsample2x(const float *x, int N, int C, int H, int W, float *y) {
+    for (long nc = 0; nc < (long)N * C; ++nc)
+        for (int oh = 0; oh < 2 * H; ++oh)
+            for (int ow = 0; ow < 2 * W; ++ow) y[(nc * 2 * H + oh) * 2 * W + ow] = x[(nc * H + oh / 2) * W + ow / 2];
+}
+
+/* y = act(a + b), sum in double, one rounding to the storage type */
+void oracle_add_act(const float *a, const float *b, long n, int act, int out_dtype, float *y) {
+    for (long i = 0; i < n; ++i) y[i] = oracle_round_to((float)activate((double)a[i] + (double)b[i], act), out_dtype);
+}

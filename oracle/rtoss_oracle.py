@@ -249,3 +249,27 @@ def rel_err(y, y_ref):
     rms = float(np.sqrt(np.mean(r * r))) if r.size else 0.0
     den = np.maximum(np.abs(r), max(rms, 1e-30))
     return float(np.max(np.abs(y - r) / den)) if r.size else 0.0
+
+
+def maxpool2d(x, k, stride, pad):
+    x = _f32(x)
+    N, C, H, W = x.shape
+    Ho, Wo = (H + 2 * pad - k) // stride + 1, (W + 2 * pad - k) // stride + 1
+    y = np.empty((N, C, Ho, Wo), dtype=np.float32)
+    lib().oracle_maxpool2d(_p(x), N, C, H, W, int(k), int(stride), int(pad), _p(y))
+    return y
+
+
+def upsample2x(x):
+    x = _f32(x)
+    N, C, H, W = x.shape
+    y = np.empty((N, C, 2 * H, 2 * W), dtype=np.float32)
+    lib().oracle_upsample2x(_p(x), N, C, H, W, _p(y))
+    return y
+
+
+def add_act(a, b, act, out_dtype):
+    a, b = _f32(a), _f32(b)
+    y = np.empty_like(a)
+    lib().oracle_add_act(_p(a), _p(b), ctypes.c_long(a.size), int(act), int(out_dtype), _p(y))
+    return y

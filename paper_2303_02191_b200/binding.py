@@ -26,7 +26,7 @@ SYMBOLS = [
     "rtoss_create", "rtoss_destroy", "rtoss_status_string", "rtoss_last_error", "rtoss_pattern_preset",
     "rtoss_pattern_table_validate", "rtoss_group_layers", "rtoss_select_patterns", "rtoss_pack",
     "rtoss_packed_info_get", "rtoss_packed_export", "rtoss_packed_to_dense", "rtoss_packed_destroy",
-    "rtoss_conv3x3_pattern", "rtoss_conv1x1_pattern", "rtoss_conv_pattern_host", "rtoss_device_status", "rtoss_prune_dense_static",
+    "rtoss_conv3x3_pattern", "rtoss_conv1x1_pattern", "rtoss_conv_pattern_host", "rtoss_device_status", "rtoss_prune_dense_static", "rtoss_maxpool2d", "rtoss_upsample2x", "rtoss_add_act",
 ]
 
 
@@ -82,6 +82,9 @@ def _load():
     lib.rtoss_conv_pattern_host.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ConvDesc)]
     lib.rtoss_device_status.argtypes = [vp, ctypes.POINTER(ci)]
     lib.rtoss_prune_dense_static.argtypes = [vp, ci, ci, ci, ci, vp, ci, ci, vp, vp]
+    lib.rtoss_maxpool2d.argtypes = [vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, vp]
+    lib.rtoss_upsample2x.argtypes = [vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, vp]
+    lib.rtoss_add_act.argtypes = [vp, vp, vp, ctypes.c_int64, ci, ci, vp]
     return lib
 
 
@@ -133,6 +136,28 @@ def rtoss_group_layers(nodes):
     if st != OK:
         raise RtossError(st, status_string(st))
     return parent[:L], group[:L], ng.value
+
+
+def _glue_check(st):
+    if st != OK:
+        raise RtossError(st, status_string(st))
+
+
+def rtoss_maxpool2d(x, y, N, C, H, W, k, stride, pad, layout=NCHW, y_channel_offset=0, y_channel_stride=0):
+    _glue_check(lib.rtoss_maxpool2d(x.data_ptr(), y.data_ptr(), N, C, H, W, k, stride, pad, layout, _torch_dtype_code(x),
+                                    y_channel_offset, y_channel_stride, _stream()))
+    return y
+
+
+def rtoss_upsample2x(x, y, N, C, H, W, layout=NCHW, y_channel_offset=0, y_channel_stride=0):
+    _glue_check(lib.rtoss_upsample2x(x.data_ptr(), y.data_ptr(), N, C, H, W, layout, _torch_dtype_code(x), y_channel_offset,
+                                     y_channel_stride, _stream()))
+    return y
+
+
+def rtoss_add_act(a, b, y, act=ACT_NONE):
+    _glue_check(lib.rtoss_add_act(a.data_ptr(), b.data_ptr(), y.data_ptr(), a.numel(), _torch_dtype_code(a), act, _stream()))
+    return y
 
 
 def rtoss_prune_dense_static(w, ksize, masks, k, out=None):

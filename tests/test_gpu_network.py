@@ -1,0 +1,50 @@
+"""Whole-network replay: the YOLOv5s-shaped backbone + neck chained on the GPU (57 pattern convolutions and the
+glue kernels, all through the C ABI) against the same program in the CPU oracle on a small input.  Every layer
+rounds to bf16, and a one-ulp difference early on changes later roundings, so the chained error is reported and
+held to a looser bound than the per-layer tests."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    from oracle import rtoss_oracle as orc
+    from paper_2303_02191_b200 import synth
+    from paper_2303_02191_b200.yolov5s_net import GpuNet
+    import gpu_util as gu
+    import net_oracle
+
+
+def test_chained_yolov5s_shaped_network_small_input():
+    N, H0 = 2, 96
+    x = synth.activations(70, 1, N, 3, H0, H0)
+    net = GpuNet(gu.ctx(), N, H0, H0, k=4, seed=3)
+    net.set_input(synth.round_like(x, "bf16"))
+    net.run()
+    torch.cuda.synchronize()
+    assert gu.ctx().rtoss_device_status() == 0
+    got = net.outputs()
+    ref = net_oracle.oracle_forward(x, H0, H0, k=4, seed=3)
+    for name in ("o3", "o4", "o5"):
+        err = orc.rel_err(got[name], ref[name])
+        print(name, got[name].shape, "chained relative error %.4f" % err)
+        assert got[name].shape == ref[name].shape
+        assert err <= 0.1
+        assert np.mean(np.abs(got[name] - ref[name])) <= 0.01 * np.sqrt(np.mean(ref[name] ** 2)) + 1e-6
+    # replay through a CUDA graph gives the same bits as the eager run
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        net.run()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    with torch.cuda.graph(g):
+        net.run()
+    g.replay()
+    torch.cuda.synchronize()
+    again = net.outputs()
+    for name in ("o3", "o4", "o5"):
+        assert np.array_equal(again[name], got[name])
+    net.close()

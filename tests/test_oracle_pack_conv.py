@@ -276,3 +276,19 @@ def test_grouping_invariants_on_the_yolov5s_graph():
         shapes = {(nodes[i]["cin"], nodes[i]["cout"], nodes[i]["ksize"]) for i in convs if group[i] == g}
         assert len(shapes) == 1
     assert all(group[i] == -1 and parent[i] == -1 for i in range(len(nodes)) if nodes[i]["kind"] != "conv")
+
+
+# ---------------------------------------------------------------- glue operations (library routines as pins)
+
+def test_glue_oracle_against_torch():
+    x = synth.activations(60, 1, 2, 3, 9, 11)
+    for k, s, p in ((5, 1, 2), (3, 2, 1), (2, 2, 0)):
+        ref = F.max_pool2d(torch.from_numpy(x), k, s, p).numpy()
+        assert np.array_equal(orc.maxpool2d(x, k, s, p), ref)
+    assert np.array_equal(orc.upsample2x(x), np.repeat(np.repeat(x, 2, axis=2), 2, axis=3))
+    y = synth.activations(60, 2, 2, 3, 9, 11)
+    s_ = (x.astype(np.float64) + y.astype(np.float64))
+    assert np.abs(orc.add_act(x, y, orc.ACT_NONE, orc.DT_F32) - s_).max() < 1e-6
+    silu = orc.add_act(x, y, orc.ACT_SILU, orc.DT_BF16)
+    want = torch.from_numpy((s_ / (1 + np.exp(-s_))).astype(np.float32)).to(torch.bfloat16).float().numpy()
+    assert (silu != want).mean() < 0.01
