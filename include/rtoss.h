@@ -126,6 +126,16 @@ rtoss_status rtoss_select_patterns(rtoss_ctx* ctx, const void* w_dev, rtoss_dtyp
                                    int ksize, const uint16_t* masks_host, int P, int k, uint8_t* pid_dev,
                                    void* cuda_stream);
 
+/* Pattern usage over a sample of kernels (Section IV.B, criterion 2: keep the most used patterns, judged by the
+ * L2 norm on random kernels in [-1, 1]).  kernels_dev holds n_kernels 3x3 kernels (9 values each, the caller's
+ * random sample); every kernel is matched against the candidate table exactly as rtoss_select_patterns does and
+ * counts_dev[p] (P entries, uint64, zeroed by the call) receives how many kernels chose pattern p.  Ranking the
+ * counts and cutting the table is left to the caller (ties: lower pattern id first).  pid_scratch_dev is a
+ * caller-owned buffer of n_kernels bytes. */
+rtoss_status rtoss_pattern_usage(rtoss_ctx* ctx, const void* kernels_dev, rtoss_dtype dtype, int64_t n_kernels,
+                                 const uint16_t* masks_host, int P, int k, uint8_t* pid_scratch_dev, uint64_t* counts_dev,
+                                 void* cuda_stream);
+
 /* ---- packing (Section IV.C: "kernels with similar patterns are grouped") --- */
 
 /* Build the packed form of one layer from its weights and pattern ids:

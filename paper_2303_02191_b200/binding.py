@@ -26,7 +26,7 @@ SYMBOLS = [
     "rtoss_create", "rtoss_destroy", "rtoss_status_string", "rtoss_last_error", "rtoss_pattern_preset",
     "rtoss_pattern_table_validate", "rtoss_group_layers", "rtoss_select_patterns", "rtoss_pack",
     "rtoss_packed_info_get", "rtoss_packed_export", "rtoss_packed_to_dense", "rtoss_packed_destroy",
-    "rtoss_conv3x3_pattern", "rtoss_conv1x1_pattern", "rtoss_conv_pattern_host", "rtoss_device_status", "rtoss_prune_dense_static", "rtoss_maxpool2d", "rtoss_upsample2x", "rtoss_add_act",
+    "rtoss_conv3x3_pattern", "rtoss_conv1x1_pattern", "rtoss_conv_pattern_host", "rtoss_device_status", "rtoss_prune_dense_static", "rtoss_maxpool2d", "rtoss_upsample2x", "rtoss_add_act", "rtoss_pattern_usage",
 ]
 
 
@@ -85,6 +85,7 @@ def _load():
     lib.rtoss_maxpool2d.argtypes = [vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, vp]
     lib.rtoss_upsample2x.argtypes = [vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, vp]
     lib.rtoss_add_act.argtypes = [vp, vp, vp, ctypes.c_int64, ci, ci, vp]
+    lib.rtoss_pattern_usage.argtypes = [vp, vp, ci, ctypes.c_int64, vp, ci, ci, vp, vp, vp]
     return lib
 
 
@@ -222,6 +223,17 @@ class Context:
         self._check(lib.rtoss_select_patterns(self.h, w.data_ptr(), _torch_dtype_code(w), Cout, Cin, int(ksize),
                                               _np_ptr(m), len(m), int(k), pid.data_ptr(), _stream()))
         return pid[:n]
+
+    def rtoss_pattern_usage(self, kernels, masks, k):
+        """kernels: CUDA tensor [n, 9] (or [n,3,3]) -> numpy uint64 win counts per pattern of the table."""
+        import torch
+        m = _masks_arr(masks)
+        n = kernels.numel() // 9
+        scratch = torch.empty(n, dtype=torch.uint8, device=kernels.device)
+        counts = torch.zeros(len(m), dtype=torch.int64, device=kernels.device)
+        self._check(lib.rtoss_pattern_usage(self.h, kernels.data_ptr(), _torch_dtype_code(kernels), n, _np_ptr(m), len(m),
+                                            int(k), scratch.data_ptr(), counts.data_ptr(), _stream()))
+        return counts.cpu().numpy().astype(np.uint64)
 
     def rtoss_pack(self, w, ksize, masks, k, pid, compute_dtype, into=None):
         """New packed handle, or re-pack `into` (an existing handle of the same layer) without allocating."""

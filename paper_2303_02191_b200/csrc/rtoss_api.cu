@@ -265,6 +265,31 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
     return RTOSS_OK;
 }
 
+rtoss_status rtoss_pattern_usage(rtoss_ctx* ctx, const void* kernels_dev, rtoss_dtype dtype, int64_t n_kernels,
+                                 const uint16_t* masks_host, int P, int k, uint8_t* pid_scratch_dev, uint64_t* counts_dev,
+                                 void* cuda_stream) {
+    if (!ctx) return RTOSS_ERR_INVALID_ARG;
+    if (!kernels_dev || !masks_host || !pid_scratch_dev || !counts_dev || n_kernels < 1 || !dtype_ok(dtype)) {
+        set_err(ctx, "pattern usage", "null argument, bad dtype or no kernels");
+        return RTOSS_ERR_INVALID_ARG;
+    }
+    if (!rtoss_table_ok(masks_host, P, k)) {
+        set_err(ctx, "pattern usage", "pattern table invalid");
+        return RTOSS_ERR_BAD_PATTERN_TABLE;
+    }
+    if (!aligned16(kernels_dev)) {
+        set_err(ctx, "pattern usage", "kernels must be 16-byte aligned");
+        return RTOSS_ERR_ALIGNMENT;
+    }
+    cudaSetDevice(ctx->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaMemsetAsync(counts_dev, 0, sizeof(uint64_t) * (size_t)P, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, "pattern usage", (int)e);
+    int le = rtoss_launch_select(kernels_dev, dtype, n_kernels, make_table(masks_host, P), P, pid_scratch_dev, cuda_stream);
+    if (!le) le = rtoss_launch_pid_histogram(pid_scratch_dev, n_kernels, P, reinterpret_cast<unsigned long long*>(counts_dev), cuda_stream);
+    return le ? cuda_fail(ctx, "pattern usage launch", le) : RTOSS_OK;
+}
+
 rtoss_status rtoss_packed_info_get(const rtoss_packed* p, rtoss_packed_info* info) {
     if (!p || !info) return RTOSS_ERR_INVALID_ARG;
     info->Cout = p->Cout;

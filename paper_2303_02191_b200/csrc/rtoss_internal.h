@@ -68,6 +68,7 @@ int rtoss_launch_pack_values(const void* w, rtoss_dtype wdt, int64_t n_kernels, 
 int rtoss_launch_pack_order(const uint8_t* pid, int Cout, int Cin, int P, uint32_t* perm, uint32_t* bucket_off,
                             void* stream);
 int rtoss_launch_to_dense(const rtoss_packed* p, void* w_out, void* stream);
+int rtoss_launch_pid_histogram(const uint8_t* pid, int64_t n, int P, unsigned long long* counts, void* stream);
 int rtoss_launch_conv3x3(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y,
                          const rtoss_conv_desc* d, void* stream);
 int rtoss_launch_conv1x1(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y,

@@ -362,3 +362,28 @@ extern "C" rtoss_status rtoss_prune_dense_static(const void* w_dev, rtoss_dtype 
     }
     return cudaGetLastError() == cudaSuccess ? RTOSS_OK : RTOSS_ERR_CUDA;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Pattern usage ranking (Section IV.B, criterion 2): how often each pattern of a candidate table is the
+// best fit over a sample of kernels.  The sample (random kernels in [-1, 1]) is the caller's input; this
+// is the selection of Algorithm 2 followed by a histogram of the winning ids.
+namespace {
+
+__global__ void __launch_bounds__(256) pid_histogram_kernel(const uint8_t* __restrict__ pid, int64_t n, int P,
+                                                            unsigned long long* __restrict__ counts) {
+    __shared__ unsigned int local[256];
+    local[threadIdx.x] = 0;
+    __syncthreads();
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        atomicAdd(&local[pid[i]], 1u);
+    __syncthreads();
+    if ((int)threadIdx.x < P && local[threadIdx.x]) atomicAdd(&counts[threadIdx.x], (unsigned long long)local[threadIdx.x]);
+}
+
+}  // namespace
+
+int rtoss_launch_pid_histogram(const uint8_t* pid, int64_t n, int P, unsigned long long* counts, void* stream) {
+    if (n <= 0) return 0;
+    pid_histogram_kernel<<<grid_for((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(pid, n, P, counts);
+    return (int)cudaGetLastError();
+}

@@ -25,6 +25,11 @@ def normal(seed, tensor_id, shape, std=1.0):
     return a
 
 
+def uniform_kernels(seed, n):
+    """n random 3x3 kernels with entries uniform in [-1, 1) (the sample of the pattern usage ranking)."""
+    return (_rng(seed, 424242).random(size=(n, 9), dtype=np.float32) * np.float32(2.0) - np.float32(1.0)).astype(np.float32)
+
+
 def activations(seed, tensor_id, N, C, H, W):
     """NCHW float32 activations ~N(0,1)."""
     return normal(seed, 2 * tensor_id, (N, C, H, W))

@@ -280,3 +280,16 @@ def test_children_inherit_the_parent_layers_patterns():
         y = gu.run_conv(packed, 3, x, "f32", 1, "none", None)
         assert orc.rel_err(y, gu.oracle_conv(3, x, dense, None, 1, "none", "f32")) <= 1e-4
         packed.close()
+
+
+@pytest.mark.parametrize("k", [2, 3])
+def test_pattern_usage_counts_match_oracle(k):
+    """Criterion 2 of Section IV.B: win counts of every candidate pattern over a seeded sample of random kernels in
+    [-1, 1); the oracle is its selection followed by a plain count.  Counts are integers: exact."""
+    masks = orc.pattern_preset(k, orc.PRESET_CONN4)
+    sample = synth.uniform_kernels(5, 1 << 18)
+    counts = gu.ctx().rtoss_pattern_usage(torch.from_numpy(sample).cuda(), masks, k)
+    want = np.bincount(orc.select_kernels(sample, masks), minlength=len(masks)).astype(np.uint64)
+    assert np.array_equal(counts, want)
+    assert int(counts.sum()) == sample.shape[0]
+    assert (counts > 0).all()            # every edge-connected pattern wins somewhere in a quarter million kernels
