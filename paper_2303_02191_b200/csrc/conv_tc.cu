@@ -31,7 +31,7 @@
 //     beyond Cout are zero-filled by TMA.
 //   * Persistent CTAs, one per SM, each walking a strided list of tiles.  Warp
 //     roles: warp 0 issues TMA, warp 1 issues tcgen05.mma and owns the TMEM
-//     allocation, warps 2..9 run the epilogue (tcgen05.ld, bias, activation,
+//     allocation, warps 2..17 run the epilogue (tcgen05.ld, bias, activation,
 //     rounding, NHWC stores: a warp holds 32 consecutive filters of one
 //     position, i.e. 64 contiguous bytes per store instruction).  Activation
 //     and weight stages form rings that run on across tiles; two accumulator
@@ -50,8 +50,9 @@ namespace {
 
 using namespace rtoss_dev;
 
-constexpr int kTcThreads = 320;    // TMA warp, MMA warp, eight epilogue warps
-constexpr int kEpiWarps = 8;
+constexpr int kEpiWarps = 16;
+constexpr int kTcThreads = (2 + kEpiWarps) * 32;  // TMA warp, MMA warp, sixteen epilogue warps
+constexpr int kPatchRows = 16;       // positions an epilogue warp turns at a time
 constexpr int kMaxA = 4, kMaxB = 8;  // most activation stages / weight slots
 constexpr int kMTile = 128;          // filters per tile = TMEM lanes
 constexpr int kPatchPitch = 80;      // bytes per position row of an epilogue transpose patch (64 + pad)
@@ -165,12 +166,13 @@ __device__ __forceinline__ void tmem_ld32(unsigned taddr, unsigned (&r)[32]) {
         : "memory");
 }
 
-// One 32-position chunk of one filter: bias, activation, rounding, into the transpose patch.
-template <typename T, int ACT>
+// Sixteen positions (registers J0 .. J0+15 of a 32-position chunk) of one filter: bias, activation,
+// rounding, into the transpose patch.
+template <typename T, int ACT, int J0>
 __device__ __forceinline__ void act_to_patch(const unsigned (&r)[32], float bv, unsigned char* col) {
 #pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        float v = __uint_as_float(r[j]) + bv;
+    for (int j = 0; j < kPatchRows; ++j) {
+        float v = __uint_as_float(r[J0 + j]) + bv;
         if (ACT == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
         if (ACT == RTOSS_ACT_SILU) {
             // v * sigmoid(v) with sigmoid(v) = 0.5 * tanh(v / 2) + 0.5: one special-function op per element
@@ -210,7 +212,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const unsigned bar_accFull = bar_emptyB + 8 * kMaxB, bar_accEmpty = bar_accFull + 16;
     const unsigned s_tmem_ptr = bar_accEmpty + 16;
     volatile unsigned* tmem_ptr_gen = reinterpret_cast<volatile unsigned*>(smem_dyn + (s_tmem_ptr - smem_u32(smem_dyn)));
-    unsigned char* epi_patch = smem_dyn + (s_tmem_ptr + 16 - smem_u32(smem_dyn));  // [kEpiWarps][32][kPatchPitch], 16-byte aligned
+    unsigned char* epi_patch = smem_dyn + (s_tmem_ptr + 16 - smem_u32(smem_dyn));  // [kEpiWarps][kPatchRows][kPatchPitch], 16-byte aligned
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = a.N * a.tiles_y * a.tiles_x * a.co_tiles;
@@ -331,7 +333,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else {
         // ---------------- epilogue: TMEM -> registers -> bias / activation -> NHWC global
         const int quarter = warp & 3;      // TMEM lanes a warp may read: 32 * (warp id mod 4)
-        const int half = (warp - 2) >> 2;  // two warps share a lane quarter and alternate 32-column chunks
+        const int sub = (warp - 2) >> 2;   // four warps share a lane quarter and take every fourth 32-column chunk
         T* __restrict__ yg = reinterpret_cast<T*>(a.y);
         bool ok = true;
         int gt = 0;
@@ -355,44 +357,54 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // position side by side.  The chunk is turned through a private shared-memory patch
             // (position-major rows of 64 + 16 pad bytes) so that global stores are 16 bytes per lane,
             // four lanes covering the 64 contiguous bytes of one position.
-            unsigned char* patch = epi_patch + (warp - 2) * (32 * kPatchPitch);
+            unsigned char* patch = epi_patch + (warp - 2) * (kPatchRows * kPatchPitch);
             const bool vec_ok = (a.y_c_stride % 8 == 0) && ((a.y_c_off + co0) % 8 == 0) && (co0 + quarter * 32 + 32 <= a.Cout);
-            for (int c0 = half * 32; c0 < a.N_px; c0 += 64) {
+            for (int c0 = sub * 32; c0 < a.N_px; c0 += 128) {
                 unsigned r[32];
                 tmem_ld32(d_base + (unsigned)c0, r);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                // the activation is picked outside the loop: 32 independent, branch-free chains
-                if (a.act == RTOSS_ACT_SILU) act_to_patch<T, RTOSS_ACT_SILU>(r, bv, patch + lane * 2);
-                else if (a.act == RTOSS_ACT_RELU) act_to_patch<T, RTOSS_ACT_RELU>(r, bv, patch + lane * 2);
-                else act_to_patch<T, RTOSS_ACT_NONE>(r, bv, patch + lane * 2);
-                __syncwarp();
-                if (vec_ok) {
 #pragma unroll
-                    for (int it = 0; it < 4; ++it) {
-                        const int i = it * 32 + lane, j = i >> 2, v = i & 3;  // position j of the chunk, 8-filter group v
-                        const int pos = c0 + j;
-                        const int oyl = pos / a.Wq, oxl = pos - oyl * a.Wq, oy = y0 + oyl, ox = x0 + oxl;
-                        if (oyl < a.TH && oxl < a.TW && ox < a.Wo && oy < a.Ho) {
-                            const uint4 o = *reinterpret_cast<const uint4*>(patch + j * kPatchPitch + v * 16);
-                            *reinterpret_cast<uint4*>(yg + (((size_t)n * a.Ho + oy) * a.Wo + ox) * a.y_c_stride + a.y_c_off + co0 +
-                                                      quarter * 32 + v * 8) = o;
+                for (int h = 0; h < 2; ++h) {
+                    // the activation is picked outside the element loop: independent, branch-free chains
+                    if (h == 0) {
+                        if (a.act == RTOSS_ACT_SILU) act_to_patch<T, RTOSS_ACT_SILU, 0>(r, bv, patch + lane * 2);
+                        else if (a.act == RTOSS_ACT_RELU) act_to_patch<T, RTOSS_ACT_RELU, 0>(r, bv, patch + lane * 2);
+                        else act_to_patch<T, RTOSS_ACT_NONE, 0>(r, bv, patch + lane * 2);
+                    } else {
+                        if (a.act == RTOSS_ACT_SILU) act_to_patch<T, RTOSS_ACT_SILU, 16>(r, bv, patch + lane * 2);
+                        else if (a.act == RTOSS_ACT_RELU) act_to_patch<T, RTOSS_ACT_RELU, 16>(r, bv, patch + lane * 2);
+                        else act_to_patch<T, RTOSS_ACT_NONE, 16>(r, bv, patch + lane * 2);
+                    }
+                    __syncwarp();
+                    const int p0 = c0 + h * kPatchRows;
+                    if (vec_ok) {
+#pragma unroll
+                        for (int it = 0; it < 2; ++it) {
+                            const int i = it * 32 + lane, j = i >> 2, v = i & 3;  // position j of the patch, 8-filter group v
+                            const int pos = p0 + j;
+                            const int oyl = pos / a.Wq, oxl = pos - oyl * a.Wq, oy = y0 + oyl, ox = x0 + oxl;
+                            if (oyl < a.TH && oxl < a.TW && ox < a.Wo && oy < a.Ho) {
+                                const uint4 o = *reinterpret_cast<const uint4*>(patch + j * kPatchPitch + v * 16);
+                                *reinterpret_cast<uint4*>(yg + (((size_t)n * a.Ho + oy) * a.Wo + ox) * a.y_c_stride + a.y_c_off +
+                                                          co0 + quarter * 32 + v * 8) = o;
+                            }
+                        }
+                    } else {
+                        // ragged filter counts or unaligned channel slices: element stores, lane = filter
+                        int oyl = p0 / a.Wq, oxl = p0 - oyl * a.Wq;
+                        for (int j = 0; j < kPatchRows; ++j) {
+                            const int oy = y0 + oyl, ox = x0 + oxl;
+                            if (co_ok && oyl < a.TH && oxl < a.TW && ox < a.Wo && oy < a.Ho)
+                                yg[(((size_t)n * a.Ho + oy) * a.Wo + ox) * a.y_c_stride + a.y_c_off + co] =
+                                    *reinterpret_cast<const T*>(patch + j * kPatchPitch + lane * 2);
+                            if (++oxl == a.Wq) {
+                                oxl = 0;
+                                ++oyl;
+                            }
                         }
                     }
-                } else {
-                    // ragged filter counts or unaligned channel slices: element stores, lane = filter
-                    int oyl = c0 / a.Wq, oxl = c0 - oyl * a.Wq;
-                    for (int j = 0; j < 32; ++j) {
-                        const int oy = y0 + oyl, ox = x0 + oxl;
-                        if (co_ok && oyl < a.TH && oxl < a.TW && ox < a.Wo && oy < a.Ho)
-                            yg[(((size_t)n * a.Ho + oy) * a.Wo + ox) * a.y_c_stride + a.y_c_off + co] =
-                                *reinterpret_cast<const T*>(patch + j * kPatchPitch + lane * 2);
-                        if (++oxl == a.Wq) {
-                            oxl = 0;
-                            ++oyl;
-                        }
-                    }
+                    __syncwarp();
                 }
-                __syncwarp();
             }
             // this warp has read everything it needs from the accumulator stage
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -461,7 +473,7 @@ bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count
     const int halo = ksize == 3 ? (S == 1 ? 2 : 1) : 0;
     const int n_sub = (ksize == 3 && S == 2) ? 4 : 1;
     const int max_pitch = S == 1 ? 256 : 128;  // TMA box: at most 256 elements traversed per dimension
-    const int fixed = 1024 /*alignment slack*/ + 512 /*barriers*/ + kEpiWarps * 32 * kPatchPitch /*epilogue patches*/;
+    const int fixed = 1024 /*alignment slack*/ + 512 /*barriers*/ + kEpiWarps * kPatchRows * kPatchPitch /*epilogue patches*/;
     const int cap = 227 * 1024 - 64;
     double best = -1;
     for (int nseg = 1; nseg <= 16; ++nseg) {
