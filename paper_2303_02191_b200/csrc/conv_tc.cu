@@ -36,6 +36,8 @@
 //     position, i.e. 64 contiguous bytes per store instruction).  Activation
 //     and weight stages form rings that run on across tiles; two accumulator
 //     stages in TMEM let the epilogue of a tile run under the MMAs of the next.
+//   * Launched with programmatic stream serialization: barrier set-up, TMEM allocation and descriptor
+//     prefetch run before griddepcontrol.wait, i.e. possibly under the tail of the previous kernel.
 //   * Every mbarrier wait is bounded; a wait that runs out records a code in
 //     the context's status word and the CTA leaves through the normal exit
 //     (TMEM is always released).
@@ -216,6 +218,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = a.N * a.tiles_y * a.tiles_x * a.co_tiles;
+    // Programmatic dependent launch: the next kernel of the stream may start its own prologue now (on SMs this
+    // grid leaves free); it reads or writes nothing before its own griddepcontrol.wait.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < a.NA; ++i) {
@@ -243,6 +248,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const unsigned tmem_base = *tmem_ptr_gen;
+    // Everything above (barriers, TMEM, descriptor prefetch) touched no tensor.  From here on the kernel reads x,
+    // the weights and the bias and writes y: wait until the kernels before it in the stream have completed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // Every role walks the same list of tiles: tile = blockIdx.x, + gridDim.x, ...  A tile is (image,
     // row band, filter tile) with the filter tile fastest, so CTAs working side by side read the same
@@ -684,7 +692,20 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
         if (e != cudaSuccess) return (int)e;
         attr_set = true;
     }
-    if (a.is_bf16) conv_tc_kernel<__nv_bfloat16><<<grid, kTcThreads, smem, (cudaStream_t)stream>>>(tmA, tmB, a);
-    else conv_tc_kernel<__half><<<grid, kTcThreads, smem, (cudaStream_t)stream>>>(tmA, tmB, a);
+    // launched with programmatic stream serialization: its prologue may overlap the tail of the previous kernel
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = (cudaStream_t)stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t le = a.is_bf16 ? cudaLaunchKernelEx(&cfg, conv_tc_kernel<__nv_bfloat16>, tmA, tmB, a)
+                               : cudaLaunchKernelEx(&cfg, conv_tc_kernel<__half>, tmA, tmB, a);
+    if (le != cudaSuccess) return (int)le;
     return (int)cudaGetLastError();
 }
