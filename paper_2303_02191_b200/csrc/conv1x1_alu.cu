@@ -43,6 +43,7 @@ struct Conv1Args {
 
 template <typename T>
 __global__ void __launch_bounds__(kThreads, 1) conv1x1_alu_kernel(const Conv1Args a) {
+    rtoss_dev::pdl_enter();
     extern __shared__ __align__(16) unsigned char smem_dyn[];
     float (*sX)[kXPitch] = reinterpret_cast<float (*)[kXPitch]>(smem_dyn);                                              // [kCiChunk][kXPitch]
     float (*sW)[kCoBlock] = reinterpret_cast<float (*)[kCoBlock]>(smem_dyn + sizeof(float) * kCiChunk * kXPitch);  // [kCiChunk][kCoBlock]
@@ -230,9 +231,9 @@ int rtoss_launch_conv1x1(const rtoss_ctx* ctx, const rtoss_packed* p, const void
         attr_set = true;
     }
     switch (d->io_dtype) {
-        case RTOSS_F32: conv1x1_alu_kernel<float><<<grid, kThreads, smem, s>>>(a); break;
-        case RTOSS_BF16: conv1x1_alu_kernel<__nv_bfloat16><<<grid, kThreads, smem, s>>>(a); break;
-        case RTOSS_F16: conv1x1_alu_kernel<__half><<<grid, kThreads, smem, s>>>(a); break;
+        case RTOSS_F32: rtoss_dev::launch_pdl(conv1x1_alu_kernel<float>, grid, kThreads, smem, s, a); break;
+        case RTOSS_BF16: rtoss_dev::launch_pdl(conv1x1_alu_kernel<__nv_bfloat16>, grid, kThreads, smem, s, a); break;
+        case RTOSS_F16: rtoss_dev::launch_pdl(conv1x1_alu_kernel<__half>, grid, kThreads, smem, s, a); break;
     }
     return (int)cudaGetLastError();
 }

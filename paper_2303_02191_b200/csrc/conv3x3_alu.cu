@@ -133,6 +133,7 @@ __device__ __forceinline__ void convert_nchw(const unsigned char* src, int n_ch,
 
 template <typename T, int S, int PH, int PW, int CO_T, int WARPS, int MINB>
 __global__ void __launch_bounds__(WARPS * 32, MINB) conv3x3_alu_kernel(const Conv3Args a) {
+    rtoss_dev::pdl_enter();
     constexpr int kThreads = WARPS * 32;
     constexpr int WIN_H = (PH - 1) * S + 3;
     constexpr int WIN_W = (PW - 1) * S + 3;
@@ -424,6 +425,7 @@ constexpr int kStemCo = 32;
 
 template <typename T, int CIN>
 __global__ void __launch_bounds__(256) conv3x3_small_cin_kernel(const Conv3Args a, int stride) {
+    rtoss_dev::pdl_enter();
     __shared__ float sWd[kStemCo][CIN * 9 + 1];  // [filter][ci*9 + tap], last = bias
     __shared__ uint16_t smask[256];
     const int co0 = blockIdx.y * kStemCo;
@@ -506,10 +508,10 @@ int launch_small_cin(const Conv3Args& a, int stride, cudaStream_t stream) {
     const long long total = (long long)a.N * a.Ho * a.Wo;
     dim3 grid((unsigned)((total + 255) / 256), (unsigned)((a.Cout + kStemCo - 1) / kStemCo));
     switch (a.Cin) {
-        case 1: conv3x3_small_cin_kernel<T, 1><<<grid, 256, 0, stream>>>(a, stride); break;
-        case 2: conv3x3_small_cin_kernel<T, 2><<<grid, 256, 0, stream>>>(a, stride); break;
-        case 3: conv3x3_small_cin_kernel<T, 3><<<grid, 256, 0, stream>>>(a, stride); break;
-        default: conv3x3_small_cin_kernel<T, 4><<<grid, 256, 0, stream>>>(a, stride); break;
+        case 1: rtoss_dev::launch_pdl(conv3x3_small_cin_kernel<T, 1>, grid, 256, 0, stream, a, stride); break;
+        case 2: rtoss_dev::launch_pdl(conv3x3_small_cin_kernel<T, 2>, grid, 256, 0, stream, a, stride); break;
+        case 3: rtoss_dev::launch_pdl(conv3x3_small_cin_kernel<T, 3>, grid, 256, 0, stream, a, stride); break;
+        default: rtoss_dev::launch_pdl(conv3x3_small_cin_kernel<T, 4>, grid, 256, 0, stream, a, stride); break;
     }
     return (int)cudaGetLastError();
 }
@@ -603,7 +605,7 @@ int launch_variant(Conv3Args& a, cudaStream_t stream) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return (int)e;
     dim3 grid((unsigned)((size_t)a.tiles_x * a.tiles_y * a.N), (unsigned)((a.Cout + CO_BLOCK - 1) / CO_BLOCK));
-    kern<<<grid, kThreads, smem, stream>>>(a);
+    rtoss_dev::launch_pdl(kern, grid, kThreads, smem, stream, a);
     return (int)cudaGetLastError();
 }
 

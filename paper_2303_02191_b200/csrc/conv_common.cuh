@@ -34,6 +34,32 @@ __device__ __forceinline__ float activate(float v, int act) {
     return v;
 }
 
+// Programmatic dependent launch.  Every kernel of the library is launched with programmatic stream
+// serialization and begins with pdl_enter(): it lets the NEXT kernel of the stream be scheduled already (launch
+// latency and block start-up then overlap this kernel's run) and then waits until every kernel before it in the
+// stream has completed and its writes are visible.  No kernel touches memory before that wait, so the stream's
+// order of reads and writes is unchanged.
+__device__ __forceinline__ void pdl_enter() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<Args&&>(args)...);
+}
+
 }  // namespace rtoss_dev
 
 #endif

@@ -434,6 +434,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 template <typename V>
 __global__ void expand_taps_kernel(const V* __restrict__ val, const uint8_t* __restrict__ pid,
                                    const uint16_t* __restrict__ masks, int k, int Cout, int Cin, V* __restrict__ out) {
+    rtoss_dev::pdl_enter();
     const size_t n = (size_t)Cout * Cin;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         const unsigned m = masks[pid[i]];
@@ -548,10 +549,10 @@ int rtoss_launch_expand_taps(const rtoss_packed* p, void* out, void* stream) {
     size_t g = (n + threads - 1) / threads;
     if (g > 148 * 8) g = 148 * 8;
     if (p->dtype == RTOSS_BF16)
-        expand_taps_kernel<__nv_bfloat16><<<(int)g, threads, 0, (cudaStream_t)stream>>>(
+        rtoss_dev::launch_pdl(expand_taps_kernel<__nv_bfloat16>, (int)g, threads, 0, (cudaStream_t)stream,
             (const __nv_bfloat16*)p->val, p->pid, p->masks_dev, p->k, p->Cout, p->Cin, (__nv_bfloat16*)out);
     else
-        expand_taps_kernel<__half><<<(int)g, threads, 0, (cudaStream_t)stream>>>((const __half*)p->val, p->pid, p->masks_dev,
+        rtoss_dev::launch_pdl(expand_taps_kernel<__half>, (int)g, threads, 0, (cudaStream_t)stream, (const __half*)p->val, p->pid, p->masks_dev,
                                                                                  p->k, p->Cout, p->Cin, (__half*)out);
     return (int)cudaGetLastError();
 }
@@ -692,20 +693,8 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
         if (e != cudaSuccess) return (int)e;
         attr_set = true;
     }
-    // launched with programmatic stream serialization: its prologue may overlap the tail of the previous kernel
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof(cfg));
-    cfg.gridDim = grid;
-    cfg.blockDim = dim3(kTcThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = (cudaStream_t)stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t le = a.is_bf16 ? cudaLaunchKernelEx(&cfg, conv_tc_kernel<__nv_bfloat16>, tmA, tmB, a)
-                               : cudaLaunchKernelEx(&cfg, conv_tc_kernel<__half>, tmA, tmB, a);
+    const cudaError_t le = a.is_bf16 ? rtoss_dev::launch_pdl(conv_tc_kernel<__nv_bfloat16>, grid, kTcThreads, smem, (cudaStream_t)stream, tmA, tmB, a)
+                                     : rtoss_dev::launch_pdl(conv_tc_kernel<__half>, grid, kTcThreads, smem, (cudaStream_t)stream, tmA, tmB, a);
     if (le != cudaSuccess) return (int)le;
     return (int)cudaGetLastError();
 }

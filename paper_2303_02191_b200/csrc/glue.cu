@@ -25,6 +25,7 @@ __device__ __forceinline__ size_t idx_of(int layout, int n, int c, int h, int w,
 // One thread per output element, channel fastest for NHWC and column fastest for NCHW (coalesced both ways).
 template <typename T>
 __global__ void maxpool_kernel(const GlueArgs a) {
+    rtoss_dev::pdl_enter();
     const size_t total = (size_t)a.N * a.C * a.Ho * a.Wo;
     const T* __restrict__ x = reinterpret_cast<const T*>(a.x);
     T* __restrict__ y = reinterpret_cast<T*>(a.y);
@@ -58,6 +59,7 @@ __global__ void maxpool_kernel(const GlueArgs a) {
 
 template <typename T>
 __global__ void upsample2x_kernel(const GlueArgs a) {
+    rtoss_dev::pdl_enter();
     const size_t total = (size_t)a.N * a.C * a.Ho * a.Wo;
     const T* __restrict__ x = reinterpret_cast<const T*>(a.x);
     T* __restrict__ y = reinterpret_cast<T*>(a.y);
@@ -82,6 +84,7 @@ __global__ void upsample2x_kernel(const GlueArgs a) {
 
 template <typename T>
 __global__ void add_act_kernel(const T* __restrict__ p, const T* __restrict__ q, T* __restrict__ y, size_t n, int act) {
+    rtoss_dev::pdl_enter();
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
         y[i] = from_f32<T>(activate(to_f32<T>(p[i]) + to_f32<T>(q[i]), act));
 }
@@ -112,9 +115,9 @@ rtoss_status rtoss_maxpool2d(const void* x_dev, void* y_dev, int N, int C, int H
     GlueArgs a{x_dev, nullptr, y_dev, N, C, H, W, Ho, Wo, k, stride, pad, (int)layout, 0, y_channel_offset, cs};
     const int grid = grid_for((size_t)N * C * Ho * Wo);
     cudaStream_t s = (cudaStream_t)cuda_stream;
-    if (dtype == RTOSS_F32) maxpool_kernel<float><<<grid, 256, 0, s>>>(a);
-    else if (dtype == RTOSS_BF16) maxpool_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(a);
-    else maxpool_kernel<__half><<<grid, 256, 0, s>>>(a);
+    if (dtype == RTOSS_F32) rtoss_dev::launch_pdl(maxpool_kernel<float>, grid, 256, 0, s, a);
+    else if (dtype == RTOSS_BF16) rtoss_dev::launch_pdl(maxpool_kernel<__nv_bfloat16>, grid, 256, 0, s, a);
+    else rtoss_dev::launch_pdl(maxpool_kernel<__half>, grid, 256, 0, s, a);
     return cudaGetLastError() == cudaSuccess ? RTOSS_OK : RTOSS_ERR_CUDA;
 }
 
@@ -128,9 +131,9 @@ rtoss_status rtoss_upsample2x(const void* x_dev, void* y_dev, int N, int C, int 
     GlueArgs a{x_dev, nullptr, y_dev, N, C, H, W, 2 * H, 2 * W, 0, 0, 0, (int)layout, 0, y_channel_offset, cs};
     const int grid = grid_for((size_t)N * C * 4 * H * W);
     cudaStream_t s = (cudaStream_t)cuda_stream;
-    if (dtype == RTOSS_F32) upsample2x_kernel<float><<<grid, 256, 0, s>>>(a);
-    else if (dtype == RTOSS_BF16) upsample2x_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(a);
-    else upsample2x_kernel<__half><<<grid, 256, 0, s>>>(a);
+    if (dtype == RTOSS_F32) rtoss_dev::launch_pdl(upsample2x_kernel<float>, grid, 256, 0, s, a);
+    else if (dtype == RTOSS_BF16) rtoss_dev::launch_pdl(upsample2x_kernel<__nv_bfloat16>, grid, 256, 0, s, a);
+    else rtoss_dev::launch_pdl(upsample2x_kernel<__half>, grid, 256, 0, s, a);
     return cudaGetLastError() == cudaSuccess ? RTOSS_OK : RTOSS_ERR_CUDA;
 }
 
@@ -142,12 +145,12 @@ rtoss_status rtoss_add_act(const void* a_dev, const void* b_dev, void* y_dev, in
     const int grid = grid_for((size_t)n_elements);
     cudaStream_t s = (cudaStream_t)cuda_stream;
     if (dtype == RTOSS_F32)
-        add_act_kernel<float><<<grid, 256, 0, s>>>((const float*)a_dev, (const float*)b_dev, (float*)y_dev, (size_t)n_elements, (int)act);
+        rtoss_dev::launch_pdl(add_act_kernel<float>, grid, 256, 0, s, (const float*)a_dev, (const float*)b_dev, (float*)y_dev, (size_t)n_elements, (int)act);
     else if (dtype == RTOSS_BF16)
-        add_act_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16*)a_dev, (const __nv_bfloat16*)b_dev,
+        rtoss_dev::launch_pdl(add_act_kernel<__nv_bfloat16>, grid, 256, 0, s, (const __nv_bfloat16*)a_dev, (const __nv_bfloat16*)b_dev,
                                                             (__nv_bfloat16*)y_dev, (size_t)n_elements, (int)act);
     else
-        add_act_kernel<__half><<<grid, 256, 0, s>>>((const __half*)a_dev, (const __half*)b_dev, (__half*)y_dev, (size_t)n_elements, (int)act);
+        rtoss_dev::launch_pdl(add_act_kernel<__half>, grid, 256, 0, s, (const __half*)a_dev, (const __half*)b_dev, (__half*)y_dev, (size_t)n_elements, (int)act);
     return cudaGetLastError() == cudaSuccess ? RTOSS_OK : RTOSS_ERR_CUDA;
 }
 

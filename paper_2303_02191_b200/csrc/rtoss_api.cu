@@ -246,11 +246,9 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
     int le = 0;
     // the mask table is copied from the handle's own (pageable) storage: the copy is staged before return
     if (masks_changed) e = cudaMemcpyAsync(p->masks_dev, p->masks, sizeof(uint16_t) * 256, cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess && p->n_kernels > 0)
-        e = cudaMemcpyAsync(p->pid, pid_dev, (size_t)p->n_kernels, cudaMemcpyDeviceToDevice, s);
-    if (e == cudaSuccess)
+    if (e == cudaSuccess)  // also writes the handle's own copy of the ids
         le = rtoss_launch_pack_values(w_dev, w_dtype, p->n_kernels, make_table(masks_host, P), pid_dev, k, p->val,
-                                      compute_dtype, cuda_stream);
+                                      compute_dtype, p->pid, cuda_stream);
     if (e == cudaSuccess && !le && ksize == 3)
         le = rtoss_launch_pack_order(pid_dev, Cout, Cin, P, p->perm, p->bucket_off, cuda_stream);
     // the tensor path reads dense-expanded weights: built here from the packed arrays just written

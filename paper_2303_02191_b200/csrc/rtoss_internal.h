@@ -64,7 +64,7 @@ static inline size_t rtoss_dtype_size(rtoss_dtype d) { return d == RTOSS_F32 ? 4
 int rtoss_launch_select(const void* w, rtoss_dtype wdt, int64_t n_kernels, const MaskTable& t, int P, uint8_t* pid,
                         void* stream);
 int rtoss_launch_pack_values(const void* w, rtoss_dtype wdt, int64_t n_kernels, const MaskTable& t, const uint8_t* pid,
-                             int k, void* val, rtoss_dtype vdt, void* stream);
+                             int k, void* val, rtoss_dtype vdt, uint8_t* pid_copy, void* stream);
 int rtoss_launch_pack_order(const uint8_t* pid, int Cout, int Cin, int P, uint32_t* perm, uint32_t* bucket_off,
                             void* stream);
 int rtoss_launch_to_dense(const rtoss_packed* p, void* w_out, void* stream);

@@ -7,6 +7,7 @@
 
 #include <cstring>
 
+#include "conv_common.cuh"
 #include "rtoss_internal.h"
 
 namespace {
@@ -47,6 +48,7 @@ __device__ __forceinline__ void stage_kernels(const T* __restrict__ w, int64_t f
 template <typename T>
 __global__ void __launch_bounds__(kSelThreads) select_kernel(const T* __restrict__ w, int64_t n_kernels, MaskTable table,
                                                              int P, uint8_t* __restrict__ pid) {
+    rtoss_dev::pdl_enter();
     __shared__ __align__(16) T sw[kSelThreads * 9];
     const int64_t n_chunks = (n_kernels + kSelThreads - 1) / kSelThreads;
     for (int64_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
@@ -83,11 +85,12 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const T* __restrict
 }
 
 // Gather the k kept values of each kernel (ascending tap order) and round them
-// to the packed type.
+// to the packed type; the handle's own copy of the pattern ids is written on the way.
 template <typename T, typename V>
 __global__ void __launch_bounds__(kSelThreads) pack_values_kernel(const T* __restrict__ w, int64_t n_kernels,
-                                                                  MaskTable table, const uint8_t* __restrict__ pid, int k,
-                                                                  V* __restrict__ val) {
+                                                                  MaskTable table, const uint8_t* pid, int k,
+                                                                  V* __restrict__ val, uint8_t* pid_copy) {
+    rtoss_dev::pdl_enter();
     __shared__ __align__(16) T sw[kSelThreads * 9];
     const int64_t n_chunks = (n_kernels + kSelThreads - 1) / kSelThreads;
     for (int64_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
@@ -98,7 +101,9 @@ __global__ void __launch_bounds__(kSelThreads) pack_values_kernel(const T* __res
         __syncthreads();
         if ((int)threadIdx.x < count) {
             const int64_t i = first + threadIdx.x;
-            const unsigned m = table.m[pid[i]];
+            const uint8_t id = pid[i];
+            pid_copy[i] = id;
+            const unsigned m = table.m[id];
             V* out = val + i * k;
             int j = 0;
 #pragma unroll
@@ -115,6 +120,7 @@ constexpr int kOrderWarps = 4;
 __global__ void __launch_bounds__(kOrderWarps * 32) pack_order_kernel(const uint8_t* __restrict__ pid, int Cout, int Cin,
                                                                       int P, uint32_t* __restrict__ perm,
                                                                       uint32_t* __restrict__ bucket_off) {
+    rtoss_dev::pdl_enter();
     __shared__ uint32_t fill_all[kOrderWarps][256];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint32_t* fill = fill_all[warp];
@@ -175,6 +181,7 @@ template <typename V>
 __global__ void to_dense_kernel(const V* __restrict__ val, const uint8_t* __restrict__ pid,
                                 const uint16_t* __restrict__ masks, int k, int64_t n_kernels, int64_t n_dense,
                                 V* __restrict__ out) {
+    rtoss_dev::pdl_enter();
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n_dense; e += (int64_t)gridDim.x * blockDim.x) {
         const int64_t g = e / 9;
         const int t = (int)(e - 9 * g);
@@ -201,38 +208,38 @@ int rtoss_launch_select(const void* w, rtoss_dtype wdt, int64_t n_kernels, const
     cudaStream_t s = (cudaStream_t)stream;
     const int grid = grid_for((n_kernels + kSelThreads - 1) / kSelThreads);
     switch (wdt) {
-        case RTOSS_F32: select_kernel<float><<<grid, kSelThreads, 0, s>>>((const float*)w, n_kernels, t, P, pid); break;
+        case RTOSS_F32: rtoss_dev::launch_pdl(select_kernel<float>, grid, kSelThreads, 0, s, (const float*)w, n_kernels, t, P, pid); break;
         case RTOSS_BF16:
-            select_kernel<__nv_bfloat16><<<grid, kSelThreads, 0, s>>>((const __nv_bfloat16*)w, n_kernels, t, P, pid);
+            rtoss_dev::launch_pdl(select_kernel<__nv_bfloat16>, grid, kSelThreads, 0, s, (const __nv_bfloat16*)w, n_kernels, t, P, pid);
             break;
-        case RTOSS_F16: select_kernel<__half><<<grid, kSelThreads, 0, s>>>((const __half*)w, n_kernels, t, P, pid); break;
+        case RTOSS_F16: rtoss_dev::launch_pdl(select_kernel<__half>, grid, kSelThreads, 0, s, (const __half*)w, n_kernels, t, P, pid); break;
     }
     return (int)cudaGetLastError();
 }
 
 template <typename T>
 static int launch_pack_values_t(const T* w, int64_t n, const MaskTable& t, const uint8_t* pid, int k, void* val,
-                                rtoss_dtype vdt, cudaStream_t s) {
+                                rtoss_dtype vdt, uint8_t* pid_copy, cudaStream_t s) {
     const int grid = grid_for((n + kSelThreads - 1) / kSelThreads);
     switch (vdt) {
-        case RTOSS_F32: pack_values_kernel<T, float><<<grid, kSelThreads, 0, s>>>(w, n, t, pid, k, (float*)val); break;
+        case RTOSS_F32: rtoss_dev::launch_pdl(pack_values_kernel<T, float>, grid, kSelThreads, 0, s, w, n, t, pid, k, (float*)val, pid_copy); break;
         case RTOSS_BF16:
-            pack_values_kernel<T, __nv_bfloat16><<<grid, kSelThreads, 0, s>>>(w, n, t, pid, k, (__nv_bfloat16*)val);
+            rtoss_dev::launch_pdl(pack_values_kernel<T, __nv_bfloat16>, grid, kSelThreads, 0, s, w, n, t, pid, k, (__nv_bfloat16*)val, pid_copy);
             break;
-        case RTOSS_F16: pack_values_kernel<T, __half><<<grid, kSelThreads, 0, s>>>(w, n, t, pid, k, (__half*)val); break;
+        case RTOSS_F16: rtoss_dev::launch_pdl(pack_values_kernel<T, __half>, grid, kSelThreads, 0, s, w, n, t, pid, k, (__half*)val, pid_copy); break;
     }
     return (int)cudaGetLastError();
 }
 
 int rtoss_launch_pack_values(const void* w, rtoss_dtype wdt, int64_t n_kernels, const MaskTable& t, const uint8_t* pid,
-                             int k, void* val, rtoss_dtype vdt, void* stream) {
+                             int k, void* val, rtoss_dtype vdt, uint8_t* pid_copy, void* stream) {
     if (n_kernels <= 0) return 0;
     cudaStream_t s = (cudaStream_t)stream;
     switch (wdt) {
-        case RTOSS_F32: return launch_pack_values_t<float>((const float*)w, n_kernels, t, pid, k, val, vdt, s);
+        case RTOSS_F32: return launch_pack_values_t<float>((const float*)w, n_kernels, t, pid, k, val, vdt, pid_copy, s);
         case RTOSS_BF16:
-            return launch_pack_values_t<__nv_bfloat16>((const __nv_bfloat16*)w, n_kernels, t, pid, k, val, vdt, s);
-        case RTOSS_F16: return launch_pack_values_t<__half>((const __half*)w, n_kernels, t, pid, k, val, vdt, s);
+            return launch_pack_values_t<__nv_bfloat16>((const __nv_bfloat16*)w, n_kernels, t, pid, k, val, vdt, pid_copy, s);
+        case RTOSS_F16: return launch_pack_values_t<__half>((const __half*)w, n_kernels, t, pid, k, val, vdt, pid_copy, s);
     }
     return (int)cudaErrorInvalidValue;
 }
@@ -240,7 +247,7 @@ int rtoss_launch_pack_values(const void* w, rtoss_dtype wdt, int64_t n_kernels, 
 int rtoss_launch_pack_order(const uint8_t* pid, int Cout, int Cin, int P, uint32_t* perm, uint32_t* bucket_off,
                             void* stream) {
     const int grid = (Cin + kOrderWarps - 1) / kOrderWarps;
-    pack_order_kernel<<<grid, kOrderWarps * 32, 0, (cudaStream_t)stream>>>(pid, Cout, Cin, P, perm, bucket_off);
+    rtoss_dev::launch_pdl(pack_order_kernel, grid, kOrderWarps * 32, 0, (cudaStream_t)stream, pid, Cout, Cin, P, perm, bucket_off);
     return (int)cudaGetLastError();
 }
 
@@ -252,15 +259,15 @@ int rtoss_launch_to_dense(const rtoss_packed* p, void* w_out, void* stream) {
     const int grid = grid_for((n_dense + threads - 1) / threads);
     switch (p->dtype) {
         case RTOSS_F32:
-            to_dense_kernel<float><<<grid, threads, 0, s>>>((const float*)p->val, p->pid, p->masks_dev, p->k, p->n_kernels,
+            rtoss_dev::launch_pdl(to_dense_kernel<float>, grid, threads, 0, s, (const float*)p->val, p->pid, p->masks_dev, p->k, p->n_kernels,
                                                             n_dense, (float*)w_out);
             break;
         case RTOSS_BF16:
-            to_dense_kernel<__nv_bfloat16><<<grid, threads, 0, s>>>((const __nv_bfloat16*)p->val, p->pid, p->masks_dev,
+            rtoss_dev::launch_pdl(to_dense_kernel<__nv_bfloat16>, grid, threads, 0, s, (const __nv_bfloat16*)p->val, p->pid, p->masks_dev,
                                                                     p->k, p->n_kernels, n_dense, (__nv_bfloat16*)w_out);
             break;
         case RTOSS_F16:
-            to_dense_kernel<__half><<<grid, threads, 0, s>>>((const __half*)p->val, p->pid, p->masks_dev, p->k,
+            rtoss_dev::launch_pdl(to_dense_kernel<__half>, grid, threads, 0, s, (const __half*)p->val, p->pid, p->masks_dev, p->k,
                                                              p->n_kernels, n_dense, (__half*)w_out);
             break;
     }
@@ -290,6 +297,7 @@ namespace {
 template <typename T>
 __global__ void mask_dense_kernel(const T* __restrict__ w, const uint8_t* __restrict__ pid, MaskTable table,
                                   int64_t n_kernels, int64_t n_dense, T* __restrict__ out) {
+    rtoss_dev::pdl_enter();
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n_dense; e += (int64_t)gridDim.x * blockDim.x) {
         const int64_t g = e / 9;
         const int t = (int)(e - 9 * g);
@@ -349,14 +357,14 @@ extern "C" rtoss_status rtoss_prune_dense_static(const void* w_dev, rtoss_dtype 
     cudaStream_t s = (cudaStream_t)cuda_stream;
     switch (w_dtype) {
         case RTOSS_F32:
-            mask_dense_kernel<float><<<grid, threads, 0, s>>>((const float*)w_dev, pid, table, n_kernels, n_dense, (float*)w_pruned_dev);
+            rtoss_dev::launch_pdl(mask_dense_kernel<float>, grid, threads, 0, s, (const float*)w_dev, pid, table, n_kernels, n_dense, (float*)w_pruned_dev);
             break;
         case RTOSS_BF16:
-            mask_dense_kernel<__nv_bfloat16><<<grid, threads, 0, s>>>((const __nv_bfloat16*)w_dev, pid, table, n_kernels, n_dense,
+            rtoss_dev::launch_pdl(mask_dense_kernel<__nv_bfloat16>, grid, threads, 0, s, (const __nv_bfloat16*)w_dev, pid, table, n_kernels, n_dense,
                                                                       (__nv_bfloat16*)w_pruned_dev);
             break;
         case RTOSS_F16:
-            mask_dense_kernel<__half><<<grid, threads, 0, s>>>((const __half*)w_dev, pid, table, n_kernels, n_dense,
+            rtoss_dev::launch_pdl(mask_dense_kernel<__half>, grid, threads, 0, s, (const __half*)w_dev, pid, table, n_kernels, n_dense,
                                                                (__half*)w_pruned_dev);
             break;
     }
@@ -371,6 +379,7 @@ namespace {
 
 __global__ void __launch_bounds__(256) pid_histogram_kernel(const uint8_t* __restrict__ pid, int64_t n, int P,
                                                             unsigned long long* __restrict__ counts) {
+    rtoss_dev::pdl_enter();
     __shared__ unsigned int local[256];
     local[threadIdx.x] = 0;
     __syncthreads();
@@ -384,6 +393,6 @@ __global__ void __launch_bounds__(256) pid_histogram_kernel(const uint8_t* __res
 
 int rtoss_launch_pid_histogram(const uint8_t* pid, int64_t n, int P, unsigned long long* counts, void* stream) {
     if (n <= 0) return 0;
-    pid_histogram_kernel<<<grid_for((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(pid, n, P, counts);
+    rtoss_dev::launch_pdl(pid_histogram_kernel, grid_for((n + 255) / 256), 256, 0, (cudaStream_t)stream, pid, n, P, counts);
     return (int)cudaGetLastError();
 }
