@@ -177,6 +177,40 @@ rtoss_status rtoss_packed_export(rtoss_ctx* ctx, const rtoss_packed* p, uint8_t*
 rtoss_status rtoss_packed_to_dense(rtoss_ctx* ctx, const rtoss_packed* p, void* w_masked_dev, void* cuda_stream);
 void rtoss_packed_destroy(rtoss_packed* p);
 
+/* ---- whole-model pruning pass ------------------------------------------------ */
+
+/* The pruning pass visits every convolution layer of the model (the outer loop of Algorithm 1 calling Algorithm 2,
+ * or Algorithm 3 for 1x1 layers); a batch runs selection and packing of ALL its layers in two kernel launches.
+ * Results are bit-identical to rtoss_select_patterns + rtoss_pack called layer by layer.
+ *
+ * One item per layer.  `packed` is an existing handle for that layer (made once by rtoss_pack; it owns the
+ * device arrays the batch re-writes, so a batch call allocates nothing and may be captured into a CUDA graph).
+ * `pid_dev` (nullable, device, Cout*Cin or floor(Cout*Cin/9) bytes) also receives the ids.  `pid_from`: -1, or
+ * the index of an EARLIER item of the same shape and table whose patterns this layer inherits (Section IV.A:
+ * the layers of a group share the parent's kernel patterns): the selection is then evaluated on that item's
+ * weights (on the root of the chain, if that item inherits too) and applied to this layer's own.
+ * The arrays w_dev, pid_dev and the handles must stay valid, and the tables unchanged, for the batch's life:
+ * rtoss_batch_create copies pointers and tables to the device once (it synchronises); the handles take the
+ * batch's tables.  Weights may change between calls -- that is the point: call again after every update.
+ * Errors: RTOSS_ERR_INVALID_ARG (null, shape mismatch with the handle, handle used twice, bad pid_from),
+ * RTOSS_ERR_BAD_PATTERN_TABLE, RTOSS_ERR_ALIGNMENT (w_dev not 16-byte aligned), RTOSS_ERR_ALLOC. */
+typedef struct {
+    const void* w_dev; /* [Cout][Cin][3][3] or [Cout][Cin], device */
+    rtoss_dtype w_dtype;
+    int Cout, Cin, ksize;
+    const uint16_t* masks_host; /* P masks of k taps, host */
+    int P, k;
+    uint8_t* pid_dev;     /* nullable */
+    rtoss_packed* packed; /* existing handle of this layer */
+    int pid_from;         /* -1 or index of an earlier item */
+} rtoss_batch_item;
+typedef struct rtoss_batch rtoss_batch;
+rtoss_status rtoss_batch_create(rtoss_ctx* ctx, const rtoss_batch_item* items, int L, rtoss_batch** out);
+/* Enqueue the pass on the stream: ids, packed values, filter order and the tensor path's weights of every layer. */
+rtoss_status rtoss_batch_select_pack(rtoss_ctx* ctx, const rtoss_batch* batch, void* cuda_stream);
+/* Frees the batch's own tables (not the handles).  The caller makes sure no call is still running. */
+void rtoss_batch_destroy(rtoss_batch* batch);
+
 /* Pruned dense weights with no allocation anywhere (the paper has no counterpart: this entry point
  * exists for deployment, not for the method).  Same result as rtoss_select_patterns followed by
  * rtoss_pack (compute type = w_dtype) and rtoss_packed_to_dense: w_pruned_dev receives W (.) mask,

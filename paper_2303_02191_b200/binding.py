@@ -27,6 +27,7 @@ SYMBOLS = [
     "rtoss_pattern_table_validate", "rtoss_group_layers", "rtoss_select_patterns", "rtoss_pack",
     "rtoss_packed_info_get", "rtoss_packed_export", "rtoss_packed_to_dense", "rtoss_packed_destroy",
     "rtoss_conv3x3_pattern", "rtoss_conv1x1_pattern", "rtoss_conv_pattern_host", "rtoss_device_status", "rtoss_prune_dense_static", "rtoss_maxpool2d", "rtoss_upsample2x", "rtoss_add_act", "rtoss_pattern_usage",
+    "rtoss_batch_create", "rtoss_batch_select_pack", "rtoss_batch_destroy",
 ]
 
 
@@ -45,6 +46,12 @@ class PackedInfo(ctypes.Structure):
     _fields_ = [("Cout", ctypes.c_int), ("Cin", ctypes.c_int), ("ksize", ctypes.c_int), ("P", ctypes.c_int),
                 ("k", ctypes.c_int), ("dtype", ctypes.c_int), ("n_kernels", ctypes.c_int64),
                 ("n_values", ctypes.c_int64)]
+
+
+class BatchItem(ctypes.Structure):
+    _fields_ = [("w_dev", ctypes.c_void_p), ("w_dtype", ctypes.c_int), ("Cout", ctypes.c_int), ("Cin", ctypes.c_int),
+                ("ksize", ctypes.c_int), ("masks_host", ctypes.c_void_p), ("P", ctypes.c_int), ("k", ctypes.c_int),
+                ("pid_dev", ctypes.c_void_p), ("packed", ctypes.c_void_p), ("pid_from", ctypes.c_int)]
 
 
 class ConvDesc(ctypes.Structure):
@@ -86,6 +93,10 @@ def _load():
     lib.rtoss_upsample2x.argtypes = [vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, vp]
     lib.rtoss_add_act.argtypes = [vp, vp, vp, ctypes.c_int64, ci, ci, vp]
     lib.rtoss_pattern_usage.argtypes = [vp, vp, ci, ctypes.c_int64, vp, ci, ci, vp, vp, vp]
+    lib.rtoss_batch_create.argtypes = [vp, ctypes.POINTER(BatchItem), ci, ctypes.POINTER(vp)]
+    lib.rtoss_batch_select_pack.argtypes = [vp, vp, vp]
+    lib.rtoss_batch_destroy.argtypes = [vp]
+    lib.rtoss_batch_destroy.restype = None
     return lib
 
 
@@ -244,6 +255,10 @@ class Context:
                                    len(m), int(k), pid.data_ptr(), int(compute_dtype), ctypes.byref(h), _stream()))
         return into if into is not None else Packed(self, h)
 
+    def rtoss_batch_create(self, items):
+        """items: list of dict(w, ksize, masks, k, packed, pid=None, pid_from=-1) -> Batch (whole-model pass)."""
+        return Batch(self, items)
+
     def _desc(self, x_shape_nchw, stride, layout, io_dtype, act, bias, y_off, y_stride, path=PATH_AUTO):
         N, _, H, W = x_shape_nchw
         return ConvDesc(int(N), int(H), int(W), int(stride), int(layout), int(io_dtype), int(act),
@@ -278,6 +293,33 @@ class Context:
                        y_channel_stride, path)
         self._check(lib.rtoss_conv_pattern_host(self.h, packed.h, x_host.data_ptr(), y_host.data_ptr(), ctypes.byref(d)))
         return y_host
+
+
+class Batch:
+    """Owns an rtoss_batch: selection + packing of every layer of a model in two launches."""
+
+    def __init__(self, ctx, items):
+        self.ctx = ctx
+        self._keep = []   # tensors, tables and handles the batch points at
+        arr = (BatchItem * max(len(items), 1))()
+        for i, it in enumerate(items):
+            w, m = it["w"], _masks_arr(it["masks"])
+            pid = it.get("pid")
+            self._keep.append((w, m, pid, it["packed"]))
+            arr[i] = BatchItem(w.data_ptr(), _torch_dtype_code(w), int(w.shape[0]), int(w.shape[1]), int(it["ksize"]),
+                               m.ctypes.data, len(m), int(it["k"]),
+                               pid.data_ptr() if pid is not None and pid.numel() else None, it["packed"].h,
+                               int(it.get("pid_from", -1)))
+        self.h = ctypes.c_void_p()
+        ctx._check(lib.rtoss_batch_create(ctx.h, arr, len(items), ctypes.byref(self.h)))
+
+    def rtoss_batch_select_pack(self):
+        self.ctx._check(lib.rtoss_batch_select_pack(self.ctx.h, self.h, _stream()))
+
+    def close(self):
+        if self.h:
+            lib.rtoss_batch_destroy(self.h)
+            self.h = ctypes.c_void_p()
 
 
 class Packed:

@@ -430,24 +430,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
 }
 
-// Dense-expanded weights for the tensor path: out[t][co][ci] = kept value or +0.
-template <typename V>
-__global__ void expand_taps_kernel(const V* __restrict__ val, const uint8_t* __restrict__ pid,
-                                   const uint16_t* __restrict__ masks, int k, int Cout, int Cin, V* __restrict__ out) {
-    rtoss_dev::pdl_enter();
-    const size_t n = (size_t)Cout * Cin;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        const unsigned m = masks[pid[i]];
-        size_t j = i * k;
-#pragma unroll
-        for (int t = 0; t < 9; ++t) {
-            V v = from_f32<V>(0.f);
-            if (m & (1u << t)) v = val[j++];
-            out[(size_t)t * n + i] = v;
-        }
-    }
-}
-
 PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
     static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
     static bool tried = false;
@@ -541,20 +523,6 @@ bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count
 
 bool rtoss_tc_weights_eligible(const rtoss_packed* p) {
     return (p->dtype == RTOSS_BF16 || p->dtype == RTOSS_F16) && p->Cin % 8 == 0;  // 16-byte rows for TMA
-}
-
-int rtoss_launch_expand_taps(const rtoss_packed* p, void* out, void* stream) {
-    const size_t n = (size_t)p->Cout * p->Cin;
-    const int threads = 256;
-    size_t g = (n + threads - 1) / threads;
-    if (g > 148 * 8) g = 148 * 8;
-    if (p->dtype == RTOSS_BF16)
-        rtoss_dev::launch_pdl(expand_taps_kernel<__nv_bfloat16>, (int)g, threads, 0, (cudaStream_t)stream,
-            (const __nv_bfloat16*)p->val, p->pid, p->masks_dev, p->k, p->Cout, p->Cin, (__nv_bfloat16*)out);
-    else
-        rtoss_dev::launch_pdl(expand_taps_kernel<__half>, (int)g, threads, 0, (cudaStream_t)stream, (const __half*)p->val, p->pid, p->masks_dev,
-                                                                                 p->k, p->Cout, p->Cin, (__half*)out);
-    return (int)cudaGetLastError();
 }
 
 // Can this call run on the tensor path?

@@ -234,8 +234,13 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
             e = cudaMalloc((void**)&p->perm, sizeof(uint32_t) * (size_t)Cin * Cout);
             if (e == cudaSuccess) e = cudaMalloc((void**)&p->bucket_off, sizeof(uint32_t) * (size_t)Cin * (P + 1));
         }
-        if (e == cudaSuccess && rtoss_tc_weights_eligible(p))
-            e = cudaMalloc(&p->wtc, (size_t)(ksize == 3 ? 9 : 1) * Cout * Cin * rtoss_dtype_size(compute_dtype));
+        if (e == cudaSuccess && rtoss_tc_weights_eligible(p)) {
+            // dense-expanded weights of the tensor path; zeroed once: the trailing Cout*Cin mod 9 weights of a 1x1
+            // layer are pruned for good and no later pack writes them
+            const size_t wtc_bytes = (size_t)(ksize == 3 ? 9 : 1) * Cout * Cin * rtoss_dtype_size(compute_dtype);
+            e = cudaMalloc(&p->wtc, wtc_bytes);
+            if (e == cudaSuccess) e = cudaMemsetAsync(p->wtc, 0, wtc_bytes, s);
+        }
         if (e != cudaSuccess) {
             cudaGetLastError();
             rtoss_packed_destroy(p);
@@ -246,14 +251,11 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
     int le = 0;
     // the mask table is copied from the handle's own (pageable) storage: the copy is staged before return
     if (masks_changed) e = cudaMemcpyAsync(p->masks_dev, p->masks, sizeof(uint16_t) * 256, cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess)  // also writes the handle's own copy of the ids
+    if (e == cudaSuccess)  // also writes the handle's own copy of the ids and the tensor path's dense-expanded weights
         le = rtoss_launch_pack_values(w_dev, w_dtype, p->n_kernels, make_table(masks_host, P), pid_dev, k, p->val,
-                                      compute_dtype, p->pid, cuda_stream);
+                                      compute_dtype, p->pid, p->wtc, ksize, (int64_t)Cout * Cin, cuda_stream);
     if (e == cudaSuccess && !le && ksize == 3)
         le = rtoss_launch_pack_order(pid_dev, Cout, Cin, P, p->perm, p->bucket_off, cuda_stream);
-    // the tensor path reads dense-expanded weights: built here from the packed arrays just written
-    if (e == cudaSuccess && !le && p->wtc)
-        le = ksize == 3 ? rtoss_launch_expand_taps(p, p->wtc, cuda_stream) : rtoss_launch_to_dense(p, p->wtc, cuda_stream);
     if (e != cudaSuccess || le) {
         rtoss_status r = cuda_fail(ctx, "pack launch", e != cudaSuccess ? (int)e : le);
         if (!reuse) rtoss_packed_destroy(p);

@@ -64,7 +64,8 @@ static inline size_t rtoss_dtype_size(rtoss_dtype d) { return d == RTOSS_F32 ? 4
 int rtoss_launch_select(const void* w, rtoss_dtype wdt, int64_t n_kernels, const MaskTable& t, int P, uint8_t* pid,
                         void* stream);
 int rtoss_launch_pack_values(const void* w, rtoss_dtype wdt, int64_t n_kernels, const MaskTable& t, const uint8_t* pid,
-                             int k, void* val, rtoss_dtype vdt, uint8_t* pid_copy, void* stream);
+                             int k, void* val, rtoss_dtype vdt, uint8_t* pid_copy, void* wtc, int ksize, int64_t n_dense,
+                             void* stream);
 int rtoss_launch_pack_order(const uint8_t* pid, int Cout, int Cin, int P, uint32_t* perm, uint32_t* bucket_off,
                             void* stream);
 int rtoss_launch_to_dense(const rtoss_packed* p, void* w_out, void* stream);
@@ -75,7 +76,6 @@ int rtoss_launch_conv1x1(const rtoss_ctx* ctx, const rtoss_packed* p, const void
                          const rtoss_conv_desc* d, void* stream);
 // tensor path (conv_tc.cu)
 bool rtoss_tc_weights_eligible(const rtoss_packed* p);
-int rtoss_launch_expand_taps(const rtoss_packed* p, void* out, void* stream);
 bool rtoss_tc_eligible(const rtoss_packed* p, const rtoss_conv_desc* d, const void* x, const void* y);
 int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y,
                          const rtoss_conv_desc* d, void* stream);

@@ -1,0 +1,124 @@
+// Per-kernel arithmetic of pattern selection and packing (Algorithm 2; Algorithm 3 after regrouping), shared by
+// the single-layer kernels and the whole-model batch so that both give the same bits.
+#ifndef RTOSS_SELECT_CORE_CUH
+#define RTOSS_SELECT_CORE_CUH
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+namespace rtoss_dev {
+
+// Squares in fp32, pattern sums in fp32 over ascending taps, first strictly larger sum wins (ties -> lowest id,
+// a NaN sum never wins).  __fmul_rn / __fadd_rn keep the compiler from contracting or reordering the arithmetic.
+// `tab[p]` is the 9-bit mask of pattern p.
+template <typename Tab>
+__device__ __forceinline__ int select_best(const float (&w)[9], const Tab& tab, int P) {
+    float q[9];
+#pragma unroll
+    for (int t = 0; t < 9; ++t) q[t] = __fmul_rn(w[t], w[t]);
+    int best = 0;
+    float best_s = 0.f;
+    for (int p = 0; p < P; ++p) {
+        const unsigned m = tab[p];
+        float s = 0.f;
+#pragma unroll
+        for (int t = 0; t < 9; ++t)
+            if (m & (1u << t)) s = __fadd_rn(s, q[t]);
+        if (p == 0) {
+            best_s = s;
+        } else if (s > best_s || (best_s != best_s && s == s)) {
+            best = p;
+            best_s = s;
+        }
+    }
+    return best;
+}
+
+template <typename V> __device__ __forceinline__ V narrow_to(float v);
+template <> __device__ __forceinline__ float narrow_to<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 narrow_to<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+template <> __device__ __forceinline__ __half narrow_to<__half>(float v) { return __float2half_rn(v); }
+
+// Writes of one kernel (3x3) or run of nine (1x1) with mask m: its k kept values, ascending taps, rounded to V, to
+// val[i*k ...]; and, where the handle carries dense-expanded weights for the tensor path (wtc != nullptr), all nine
+// taps, pruned ones as +0:  3x3 -> wtc[t][co][ci] (i = co*Cin+ci, n = Cout*Cin);  1x1 -> wtc[9*i + t].
+template <typename V>
+__device__ __forceinline__ void pack_one(const float (&w)[9], unsigned m, int64_t i, int k, V* __restrict__ val,
+                                         V* __restrict__ wtc, int ksize, int64_t n) {
+    V* out = val + i * k;
+    int j = 0;
+#pragma unroll
+    for (int t = 0; t < 9; ++t)
+        if (m & (1u << t)) out[j++] = narrow_to<V>(w[t]);
+    if (wtc) {
+#pragma unroll
+        for (int t = 0; t < 9; ++t) {
+            const V v = (m & (1u << t)) ? narrow_to<V>(w[t]) : narrow_to<V>(0.f);
+            if (ksize == 3) wtc[(int64_t)t * n + i] = v;
+            else wtc[i * 9 + t] = v;
+        }
+    }
+}
+
+// Stable counting sort of the Cout filters of input channel ci by pattern id, by one warp: perm[ci*Cout + j] lists
+// the filters by ascending id (ties by ascending filter), bucket_off[ci*(P+1) + p] is where pattern p starts.
+// Ranks inside a group of 32 filters come from __match_any_sync; `fill` is 256 words of shared memory of this warp.
+__device__ __forceinline__ void order_channel(const uint8_t* __restrict__ pid, int Cout, int Cin, int P, int ci,
+                                              uint32_t* __restrict__ perm, uint32_t* __restrict__ bucket_off,
+                                              uint32_t* fill, int lane) {
+    for (int p = lane; p < 256; p += 32) fill[p] = 0;
+    __syncwarp();
+    // pass 1: histogram
+    for (int base = 0; base < Cout; base += 32) {
+        const int co = base + lane;
+        const unsigned key = co < Cout ? pid[(size_t)co * Cin + ci] : 0xFFFFu;
+        const unsigned peers = __match_any_sync(0xFFFFFFFFu, key);
+        if (co < Cout && lane == __ffs(peers) - 1) fill[key] += __popc(peers);
+        __syncwarp();
+    }
+    // exclusive scan over the P buckets (P <= 255: eight per lane, then a warp scan of lane totals)
+    uint32_t local[8];
+    uint32_t sum = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int p = lane * 8 + j;
+        local[j] = sum;
+        sum += (p < P) ? fill[p] : 0;
+    }
+    uint32_t incl = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= d) incl += o;
+    }
+    const uint32_t excl = incl - sum;
+    __syncwarp();
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int p = lane * 8 + j;
+        if (p < P) {
+            fill[p] = excl + local[j];
+            bucket_off[(size_t)ci * (P + 1) + p] = excl + local[j];
+        }
+    }
+    if (lane == 0) bucket_off[(size_t)ci * (P + 1) + P] = (uint32_t)Cout;
+    __syncwarp();
+    // pass 2: placement, filters in ascending order inside each bucket
+    for (int base = 0; base < Cout; base += 32) {
+        const int co = base + lane;
+        const unsigned key = co < Cout ? pid[(size_t)co * Cin + ci] : 0xFFFFu;
+        const unsigned peers = __match_any_sync(0xFFFFFFFFu, key);
+        const unsigned before = peers & ((1u << lane) - 1u);
+        if (co < Cout) perm[(size_t)ci * Cout + fill[key] + __popc(before)] = (uint32_t)co;
+        __syncwarp();
+        if (co < Cout && before == 0) fill[key] += __popc(peers);
+        __syncwarp();
+    }
+}
+
+}  // namespace rtoss_dev
+
+#endif

@@ -9,6 +9,7 @@
 
 #include "conv_common.cuh"
 #include "rtoss_internal.h"
+#include "select_core.cuh"
 
 namespace {
 
@@ -58,38 +59,23 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const T* __restrict
         stage_kernels<T>(w, first, count, sw);
         __syncthreads();
         if ((int)threadIdx.x < count) {
-            float q[9];
+            float v[9];
 #pragma unroll
-            for (int t = 0; t < 9; ++t) {
-                float v = widen<T>(sw[threadIdx.x * 9 + t]);
-                q[t] = __fmul_rn(v, v);
-            }
-            int best = 0;
-            float best_s = 0.f;
-            for (int p = 0; p < P; ++p) {
-                const unsigned m = table.m[p];
-                float s = 0.f;
-#pragma unroll
-                for (int t = 0; t < 9; ++t)
-                    if (m & (1u << t)) s = __fadd_rn(s, q[t]);
-                if (p == 0) {
-                    best_s = s;
-                } else if (s > best_s || (best_s != best_s && s == s)) {
-                    best = p;
-                    best_s = s;
-                }
-            }
+            for (int t = 0; t < 9; ++t) v[t] = widen<T>(sw[threadIdx.x * 9 + t]);
+            const int best = rtoss_dev::select_best(v, table.m, P);
             pid[first + threadIdx.x] = (uint8_t)best;
         }
     }
 }
 
-// Gather the k kept values of each kernel (ascending tap order) and round them
-// to the packed type; the handle's own copy of the pattern ids is written on the way.
+// Gather the k kept values of each kernel (ascending tap order) and round them to the packed type; the handle's
+// own copy of the pattern ids and, where it has them, the dense-expanded weights of the tensor path are written
+// on the way.
 template <typename T, typename V>
 __global__ void __launch_bounds__(kSelThreads) pack_values_kernel(const T* __restrict__ w, int64_t n_kernels,
                                                                   MaskTable table, const uint8_t* pid, int k,
-                                                                  V* __restrict__ val, uint8_t* pid_copy) {
+                                                                  V* __restrict__ val, uint8_t* pid_copy,
+                                                                  V* __restrict__ wtc, int ksize, int64_t n_dense) {
     rtoss_dev::pdl_enter();
     __shared__ __align__(16) T sw[kSelThreads * 9];
     const int64_t n_chunks = (n_kernels + kSelThreads - 1) / kSelThreads;
@@ -103,19 +89,15 @@ __global__ void __launch_bounds__(kSelThreads) pack_values_kernel(const T* __res
             const int64_t i = first + threadIdx.x;
             const uint8_t id = pid[i];
             pid_copy[i] = id;
-            const unsigned m = table.m[id];
-            V* out = val + i * k;
-            int j = 0;
+            float v[9];
 #pragma unroll
-            for (int t = 0; t < 9; ++t)
-                if (m & (1u << t)) out[j++] = narrow<V>(widen<T>(sw[threadIdx.x * 9 + t]));
+            for (int t = 0; t < 9; ++t) v[t] = widen<T>(sw[threadIdx.x * 9 + t]);
+            rtoss_dev::pack_one<V>(v, table.m[id], i, k, val, wtc, ksize, n_dense);
         }
     }
 }
 
-// Per input channel: stable counting sort of the filters by pattern id.  One
-// warp per channel; ranks inside a group of 32 filters come from
-// __match_any_sync, running bucket fill levels live in shared memory.
+// Per input channel: stable counting sort of the filters by pattern id, one warp per channel.
 constexpr int kOrderWarps = 4;
 __global__ void __launch_bounds__(kOrderWarps * 32) pack_order_kernel(const uint8_t* __restrict__ pid, int Cout, int Cin,
                                                                       int P, uint32_t* __restrict__ perm,
@@ -123,57 +105,9 @@ __global__ void __launch_bounds__(kOrderWarps * 32) pack_order_kernel(const uint
     rtoss_dev::pdl_enter();
     __shared__ uint32_t fill_all[kOrderWarps][256];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    uint32_t* fill = fill_all[warp];
     const int ci = blockIdx.x * kOrderWarps + warp;
     if (ci >= Cin) return;  // whole warp leaves together; no block-wide barrier below
-    for (int p = lane; p < 256; p += 32) fill[p] = 0;
-    __syncwarp();
-    // pass 1: histogram
-    for (int base = 0; base < Cout; base += 32) {
-        const int co = base + lane;
-        const unsigned key = co < Cout ? pid[(size_t)co * Cin + ci] : 0xFFFFu;
-        const unsigned peers = __match_any_sync(0xFFFFFFFFu, key);
-        if (co < Cout && lane == __ffs(peers) - 1) fill[key] += __popc(peers);
-        __syncwarp();
-    }
-    // exclusive scan over the P buckets (P <= 255: eight per lane, then a warp scan of lane totals)
-    uint32_t local[8];
-    uint32_t sum = 0;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const int p = lane * 8 + j;
-        local[j] = sum;
-        sum += (p < P) ? fill[p] : 0;
-    }
-    uint32_t incl = sum;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-        if (lane >= d) incl += o;
-    }
-    const uint32_t excl = incl - sum;
-    __syncwarp();
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const int p = lane * 8 + j;
-        if (p < P) {
-            fill[p] = excl + local[j];
-            bucket_off[(size_t)ci * (P + 1) + p] = excl + local[j];
-        }
-    }
-    if (lane == 0) bucket_off[(size_t)ci * (P + 1) + P] = (uint32_t)Cout;
-    __syncwarp();
-    // pass 2: placement, filters in ascending order inside each bucket
-    for (int base = 0; base < Cout; base += 32) {
-        const int co = base + lane;
-        const unsigned key = co < Cout ? pid[(size_t)co * Cin + ci] : 0xFFFFu;
-        const unsigned peers = __match_any_sync(0xFFFFFFFFu, key);
-        const unsigned before = peers & ((1u << lane) - 1u);
-        if (co < Cout) perm[(size_t)ci * Cout + fill[key] + __popc(before)] = (uint32_t)co;
-        __syncwarp();
-        if (co < Cout && before == 0) fill[key] += __popc(peers);
-        __syncwarp();
-    }
+    rtoss_dev::order_channel(pid, Cout, Cin, P, ci, perm, bucket_off, fill_all[warp], lane);
 }
 
 // Dense masked weights from the packed form, one thread per dense element.
@@ -219,27 +153,28 @@ int rtoss_launch_select(const void* w, rtoss_dtype wdt, int64_t n_kernels, const
 
 template <typename T>
 static int launch_pack_values_t(const T* w, int64_t n, const MaskTable& t, const uint8_t* pid, int k, void* val,
-                                rtoss_dtype vdt, uint8_t* pid_copy, cudaStream_t s) {
+                                rtoss_dtype vdt, uint8_t* pid_copy, void* wtc, int ksize, int64_t n_dense, cudaStream_t s) {
     const int grid = grid_for((n + kSelThreads - 1) / kSelThreads);
     switch (vdt) {
-        case RTOSS_F32: rtoss_dev::launch_pdl(pack_values_kernel<T, float>, grid, kSelThreads, 0, s, w, n, t, pid, k, (float*)val, pid_copy); break;
+        case RTOSS_F32: rtoss_dev::launch_pdl(pack_values_kernel<T, float>, grid, kSelThreads, 0, s, w, n, t, pid, k, (float*)val, pid_copy, (float*)wtc, ksize, n_dense); break;
         case RTOSS_BF16:
-            rtoss_dev::launch_pdl(pack_values_kernel<T, __nv_bfloat16>, grid, kSelThreads, 0, s, w, n, t, pid, k, (__nv_bfloat16*)val, pid_copy);
+            rtoss_dev::launch_pdl(pack_values_kernel<T, __nv_bfloat16>, grid, kSelThreads, 0, s, w, n, t, pid, k, (__nv_bfloat16*)val, pid_copy, (__nv_bfloat16*)wtc, ksize, n_dense);
             break;
-        case RTOSS_F16: rtoss_dev::launch_pdl(pack_values_kernel<T, __half>, grid, kSelThreads, 0, s, w, n, t, pid, k, (__half*)val, pid_copy); break;
+        case RTOSS_F16: rtoss_dev::launch_pdl(pack_values_kernel<T, __half>, grid, kSelThreads, 0, s, w, n, t, pid, k, (__half*)val, pid_copy, (__half*)wtc, ksize, n_dense); break;
     }
     return (int)cudaGetLastError();
 }
 
 int rtoss_launch_pack_values(const void* w, rtoss_dtype wdt, int64_t n_kernels, const MaskTable& t, const uint8_t* pid,
-                             int k, void* val, rtoss_dtype vdt, uint8_t* pid_copy, void* stream) {
+                             int k, void* val, rtoss_dtype vdt, uint8_t* pid_copy, void* wtc, int ksize, int64_t n_dense,
+                             void* stream) {
     if (n_kernels <= 0) return 0;
     cudaStream_t s = (cudaStream_t)stream;
     switch (wdt) {
-        case RTOSS_F32: return launch_pack_values_t<float>((const float*)w, n_kernels, t, pid, k, val, vdt, pid_copy, s);
+        case RTOSS_F32: return launch_pack_values_t<float>((const float*)w, n_kernels, t, pid, k, val, vdt, pid_copy, wtc, ksize, n_dense, s);
         case RTOSS_BF16:
-            return launch_pack_values_t<__nv_bfloat16>((const __nv_bfloat16*)w, n_kernels, t, pid, k, val, vdt, pid_copy, s);
-        case RTOSS_F16: return launch_pack_values_t<__half>((const __half*)w, n_kernels, t, pid, k, val, vdt, pid_copy, s);
+            return launch_pack_values_t<__nv_bfloat16>((const __nv_bfloat16*)w, n_kernels, t, pid, k, val, vdt, pid_copy, wtc, ksize, n_dense, s);
+        case RTOSS_F16: return launch_pack_values_t<__half>((const __half*)w, n_kernels, t, pid, k, val, vdt, pid_copy, wtc, ksize, n_dense, s);
     }
     return (int)cudaErrorInvalidValue;
 }
