@@ -307,14 +307,17 @@ def run_gpu(args):
         L_state.append(st)
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)   # larger than the 126 MB L2
 
+    # handles are made once, layer by layer (this allocates); every step then re-selects and re-packs ALL layers
+    # with the whole-model pass: two launches, whatever the number of layers
+    for wt in weights.values():
+        ctx.rtoss_select_patterns(wt["w"], wt["ksize"], wt["masks"], wt["k"], pid=wt["pid"])
+        wt["packed"] = ctx.rtoss_pack(wt["w"], wt["ksize"], wt["masks"], wt["k"], wt["pid"], cdt)
+    batch = ctx.rtoss_batch_create(list(weights.values()))
+    any3 = any(wt["ksize"] == 3 for wt in weights.values())
+
     def prune_weights():
-        launches = 0
-        for wt in weights.values():
-            ctx.rtoss_select_patterns(wt["w"], wt["ksize"], wt["masks"], wt["k"], pid=wt["pid"])
-            wt["packed"] = ctx.rtoss_pack(wt["w"], wt["ksize"], wt["masks"], wt["k"], wt["pid"], cdt, into=wt["packed"])
-            # select, pack values, (3x3: pack order), and for handles the tensor path can use the dense expansion
-            launches += (3 if wt["ksize"] == 3 else 2) + (1 if (dtype != "f32" and wt["w"].shape[1] % 8 == 0) else 0)
-        return launches
+        batch.rtoss_batch_select_pack()
+        return 2 if any3 else 1
 
     def conv(st, ev=None):
         L = st["L"]
@@ -477,6 +480,8 @@ def run_gpu(args):
                                    "sample": "%d image(s) of the batch of %d, the first %.3f of every layer's output channels, "
                                              "one pass of %.1f s; images/s = images x fraction / seconds" % (n_cpu, N, f_cpu, t_cpu)}
         print(json.dumps(out))
+    torch.cuda.synchronize()
+    batch.close()
     for wt in weights.values():
         if wt["packed"] is not None:
             wt["packed"].close()
