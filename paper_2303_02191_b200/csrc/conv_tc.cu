@@ -57,6 +57,7 @@ constexpr int kTcThreads = (2 + kEpiWarps) * 32;  // TMA warp, MMA warp, sixteen
 constexpr int kPatchRows = 16;       // positions an epilogue warp turns at a time
 constexpr int kMaxA = 4, kMaxB = 8;  // most activation stages / weight slots
 constexpr int kMTile = 128;          // filters per tile = TMEM lanes
+constexpr int kPxmMaxCout = 64;      // layers this narrow run with positions as the M operand
 constexpr int kPatchPitch = 80;      // bytes per position row of an epilogue transpose patch (64 + pad)
 constexpr int kKBlock = 64;       // channels per staged block: 128 bytes of bf16 / fp16
 constexpr int kRowBytes = 128;    // one padded pixel, one channel block
@@ -81,6 +82,8 @@ struct TcArgs {
     int act, y_c_off, y_c_stride, is_bf16;
     unsigned idesc;
     int tmem_cols;
+    int w_rows;           // filter rows per staged weight tile (128; fewer with positions as the M operand)
+    int pxm, MH, n_cols;  // positions as the M operand: M halves of 128 positions per tile, filters per tile (the MMA's N)
 };
 
 __device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -168,6 +171,50 @@ __device__ __forceinline__ void tmem_ld32(unsigned taddr, unsigned (&r)[32]) {
         : "memory");
 }
 
+template <typename T>
+__device__ __forceinline__ unsigned pack2(float a, float b);
+template <>
+__device__ __forceinline__ unsigned pack2<__nv_bfloat16>(float a, float b) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<unsigned*>(&v);
+}
+template <>
+__device__ __forceinline__ unsigned pack2<__half>(float a, float b) {
+    __half2 v = __floats2half2_rn(a, b);
+    return *reinterpret_cast<unsigned*>(&v);
+}
+
+__device__ __forceinline__ void tmem_ld16(unsigned taddr, unsigned (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+
+// Sixteen consecutive filters of one position (positions as the M operand): bias, activation, rounding, packed
+// two to a register in memory order.
+template <typename T, int ACT>
+__device__ __forceinline__ void act_pack16(const unsigned (&r)[16], const float* bias16, unsigned (&o)[8]) {
+#pragma unroll
+    for (int j = 0; j < 16; j += 2) {
+        float v[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            v[e] = __uint_as_float(r[j + e]) + bias16[j + e];
+            if (ACT == RTOSS_ACT_RELU) v[e] = fmaxf(v[e], 0.f);
+            if (ACT == RTOSS_ACT_SILU) {
+                float th;
+                asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(0.5f * v[e]));
+                v[e] = v[e] * fmaf(0.5f, th, 0.5f);
+            }
+        }
+        o[j >> 1] = pack2<T>(v[0], v[1]);
+    }
+}
+
 // Sixteen positions (registers J0 .. J0+15 of a 32-position chunk) of one filter: bias, activation,
 // rounding, into the transpose patch.
 template <typename T, int ACT, int J0>
@@ -187,18 +234,6 @@ __device__ __forceinline__ void act_to_patch(const unsigned (&r)[32], float bv, 
     }
 }
 
-template <typename T>
-__device__ __forceinline__ unsigned pack2(float a, float b);
-template <>
-__device__ __forceinline__ unsigned pack2<__nv_bfloat16>(float a, float b) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
-    return *reinterpret_cast<unsigned*>(&v);
-}
-template <>
-__device__ __forceinline__ unsigned pack2<__half>(float a, float b) {
-    __half2 v = __floats2half2_rn(a, b);
-    return *reinterpret_cast<unsigned*>(&v);
-}
 
 template <typename T>
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -284,7 +319,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         if (!ok) break;
                         mbar_expect_tx(bar_fullB + 8 * sb, a.b_tx_bytes * a.G);
                         for (int i = 0; i < a.G; ++i)
-                            tma_load_3d(sB + sb * a.b_stage_bytes + i * (kMTile * kRowBytes), &tmB, cb * kKBlock, co0, t0 + i,
+                            tma_load_3d(sB + sb * a.b_stage_bytes + i * (a.w_rows * kRowBytes), &tmB, cb * kKBlock, co0, t0 + i,
                                         bar_fullB + 8 * sb);
                     }
                 }
@@ -309,6 +344,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const unsigned a_tile = sA + sa * a.a_stage_bytes;
+                    // 16-channel slabs of this block that hold channels (the rest of the 64 is TMA zero fill)
+                    const int left = a.Cin - cb * kKBlock;
+                    const int nk4 = left >= kKBlock ? kKBlock / 16 : (left + 15) >> 4;
                     for (int t0 = 0; t0 < a.taps; t0 += a.G, ++gb) {
                         const int sb = gb % a.NB;
                         ok = mbar_wait(bar_fullB + 8 * sb, (gb / a.NB) & 1);
@@ -316,12 +354,27 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                         for (int i = 0; i < a.G; ++i) {
                             const int t = t0 + i;
-                            const unsigned w_tile = sB + sb * a.b_stage_bytes + i * (kMTile * kRowBytes);  // M operand: 128 filters
+                            const unsigned w_tile = sB + sb * a.b_stage_bytes + i * (a.w_rows * kRowBytes);
                             const unsigned x_rows = a_tile + (unsigned)(a.tap_sub[t] * a.sub_bytes + a.tap_shift[t] * kRowBytes);  // N operand
+                            // One thread issues everything, so the instructions between two tcgen05.mma are the budget:
+                            // the descriptors of a tap are built once and stepped by adding to their address field
+                            // (+2 = 32 bytes = 16 channels; +1024 = 128 rows), the loops are unrolled and predicated.
+                            const unsigned long long wd = make_sw128_desc(w_tile), xd = make_sw128_desc(x_rows);
+                            if (a.pxm) {
+                                // positions are the M operand: one instruction per half of 128 positions; the halves
+                                // accumulate side by side in TMEM
+                                const unsigned d_hi = d_base + (unsigned)a.n_cols;
 #pragma unroll
-                            for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
-                                umma_f16(d_base, make_sw128_desc(w_tile + k4 * 32), make_sw128_desc(x_rows + k4 * 32), a.idesc,
-                                         (cb | t | k4) != 0);
+                                for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
+                                    if (k4 < nk4) {
+                                        umma_f16(d_base, xd + 2 * k4, wd + 2 * k4, a.idesc, (cb | t | k4) != 0);
+                                        if (a.MH == 2) umma_f16(d_hi, xd + 1024 + 2 * k4, wd + 2 * k4, a.idesc, (cb | t | k4) != 0);
+                                    }
+                                }
+                            } else {
+#pragma unroll
+                                for (int k4 = 0; k4 < kKBlock / 16; ++k4)
+                                    if (k4 < nk4) umma_f16(d_base, wd + 2 * k4, xd + 2 * k4, a.idesc, (cb | t | k4) != 0);
                             }
                         }
                         umma_commit(bar_emptyB + 8 * sb);  // this weight stage may be refilled once the MMAs have read it
@@ -345,6 +398,58 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         T* __restrict__ yg = reinterpret_cast<T*>(a.y);
         bool ok = true;
         int gt = 0;
+        if (a.pxm) {
+            // Positions are the TMEM lanes: a thread owns one position and reads its filters sixteen at a time, which
+            // are contiguous in NHWC -- no transpose.  One filter tile covers the layer, so the bias is staged once.
+            float* bias_s = reinterpret_cast<float*>(epi_patch);
+            for (int i = threadIdx.x - 64; i < a.n_cols; i += kEpiWarps * 32)
+                bias_s[i] = (a.bias && i < a.Cout) ? __ldg(a.bias + i) : 0.f;
+            asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
+            const int n_chunks = a.n_cols >> 4, items = a.MH * n_chunks;
+            const bool vec_ok = (a.y_c_stride % 8 == 0) && (a.y_c_off % 8 == 0);
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++gt) {
+                int rest = tile;
+                const int tx = rest % a.tiles_x;
+                rest /= a.tiles_x;
+                const int ty = rest % a.tiles_y, n = rest / a.tiles_y;
+                const int y0 = ty * a.TH, x0 = tx * a.TW;
+                const int as = gt % a.AS;
+                ok = mbar_wait(bar_accFull + 8 * as, (gt / a.AS) & 1);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const unsigned d_base = tmem_base + (unsigned)(as * a.acc_cols) + ((unsigned)(quarter * 32) << 16);
+                for (int item = sub; item < items; item += 4) {
+                    const int h = item / n_chunks, c = item - h * n_chunks;
+                    unsigned r[16];
+                    tmem_ld16(d_base + (unsigned)(h * a.n_cols + c * 16), r);
+                    const int pos = h * 128 + quarter * 32 + lane;
+                    const int oyl = pos / a.Wq, oxl = pos - oyl * a.Wq, oy = y0 + oyl, ox = x0 + oxl;
+                    const bool px_ok = pos < a.N_px && oyl < a.TH && oxl < a.TW && ox < a.Wo && oy < a.Ho;
+                    const float* b16 = bias_s + c * 16;
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    unsigned o[8];
+                    if (a.act == RTOSS_ACT_SILU) act_pack16<T, RTOSS_ACT_SILU>(r, b16, o);
+                    else if (a.act == RTOSS_ACT_RELU) act_pack16<T, RTOSS_ACT_RELU>(r, b16, o);
+                    else act_pack16<T, RTOSS_ACT_NONE>(r, b16, o);
+                    if (px_ok) {
+                        T* dst = yg + (((size_t)n * a.Ho + oy) * a.Wo + ox) * a.y_c_stride + a.y_c_off + c * 16;
+                        if (vec_ok && c * 16 + 16 <= a.Cout) {
+                            reinterpret_cast<uint4*>(dst)[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                            reinterpret_cast<uint4*>(dst)[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                        } else {
+                            // ragged filter count or unaligned channel slice: element stores
+                            const T* ov = reinterpret_cast<const T*>(o);
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (c * 16 + j < a.Cout) dst[j] = ov[j];
+                        }
+                    }
+                }
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_accEmpty + 8 * as) : "memory");
+            }
+        } else
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++gt) {
             int rest = tile;
             const int cot = rest % a.co_tiles;
@@ -446,6 +551,13 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
 
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
+// Which operand the positions are.  A tcgen05.mma costs about the same whatever its N, so the wide operand should be
+// N: with the filters as M and up to 256 positions as N a layer of 128 filters per tile runs near the tensor peak.
+// A narrow layer wastes most of M that way and, worse, leaves three of four epilogue warps without TMEM lanes to
+// read; with the positions as M every lane carries an output and a thread's filters are contiguous in NHWC.  The
+// price is one instruction per 128 positions instead of per 256: taken where few instructions are needed anyway.
+bool use_pxm(const rtoss_packed* p) { return p->Cout <= kPxmMaxCout && (p->ksize == 1 || p->Cin <= 64); }
+
 struct TcPlan {
     int TH, TW, Wq, N_px, NA, NB, G, n_sub, sub_rows, rows_staged, tiles_x, smem;
 };
@@ -460,7 +572,7 @@ struct TcPlan {
 //                 the even rows for r = 1, one staged row further down for r = 1, 2; columns alike.
 // The plan picks TH, the column segment TW (images wider than a TMA box are cut into segments), the
 // ring depths, and how many taps share a weight stage.
-bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count, TcPlan* out) {
+bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count, bool pxm, int w_rows, TcPlan* out) {
     const int halo = ksize == 3 ? (S == 1 ? 2 : 1) : 0;
     const int n_sub = (ksize == 3 && S == 2) ? 4 : 1;
     const int max_pitch = S == 1 ? 256 : 128;  // TMA box: at most 256 elements traversed per dimension
@@ -476,11 +588,14 @@ bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count
             if (th * wq > 256 || rows_staged * S > 256) break;
             const int n_px = round_up(th * wq, 16);
             const int max_shift = ksize == 3 ? (S == 1 ? 2 * wq + 2 : wq + 1) : 0;
-            const int need_rows = n_px + max_shift > rows_staged * wq ? n_px + max_shift : rows_staged * wq;
+            int need_rows = n_px + max_shift > rows_staged * wq ? n_px + max_shift : rows_staged * wq;
+            // positions as the M operand: every instruction reads 128 rows, also where the tile's list ends earlier
+            const int halves = n_px > 128 ? 2 : 1;
+            if (pxm && max_shift + 128 * halves > need_rows) need_rows = max_shift + 128 * halves;
             const int sub_rows = round_up(need_rows, 8);
             const int a_bytes = n_sub * sub_rows * kRowBytes;
             for (int G = (ksize == 3 ? 3 : 1); G >= 1; G -= 2) {
-                const int b_bytes = G * kMTile * kRowBytes;
+                const int b_bytes = G * w_rows * kRowBytes;
                 int na = (cap - fixed - 2 * b_bytes) / a_bytes;
                 if (na < 1) continue;
                 if (na > kMaxA) na = kMaxA;
@@ -492,7 +607,7 @@ bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count
                 const double waves = (double)tiles / sm_count;
                 const double balance = waves / (double)((tiles + sm_count - 1) / sm_count);  // 1 = SMs equally loaded
                 // an instruction costs about the same for any N: what counts is useful positions per instruction
-                const double eff = (double)(th * tw) / 256.0 * Ho / (double)((Ho + th - 1) / th * th) * Wo / (double)(tw * nseg);
+                const double eff = (double)(th * tw) / (pxm ? 128.0 * halves : 256.0) * Ho / (double)((Ho + th - 1) / th * th) * Wo / (double)(tw * nseg);
                 const double halo_cost = (double)(th * tw) / (double)(rows_staged * wq);  // staged pixels that are outputs
                 const double score = eff * (0.5 + 0.5 * balance) * (G == 3 || ksize == 1 ? 1.0 : 0.8) * (na >= 2 ? 1.0 : 0.8) *
                                          (0.8 + 0.2 * halo_cost) +
@@ -533,7 +648,9 @@ bool rtoss_tc_eligible(const rtoss_packed* p, const rtoss_conv_desc* d, const vo
     if (!encode_fn()) return false;
     const int Ho = (d->H - 1) / d->stride + 1, Wo = (d->W - 1) / d->stride + 1;
     TcPlan plan;
-    return plan_tc(d->N, Ho, Wo, p->ksize, d->stride, (p->Cout + kMTile - 1) / kMTile, 148, &plan);
+    const bool pxm = use_pxm(p);
+    return plan_tc(d->N, Ho, Wo, p->ksize, d->stride, (p->Cout + kMTile - 1) / kMTile, 148, pxm, pxm ? round_up(p->Cout, 16) : kMTile,
+                   &plan);
 }
 
 int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y, const rtoss_conv_desc* d,
@@ -544,7 +661,10 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     const int N_T = kMTile;
     const int sms = ctx->sm_count > 0 ? ctx->sm_count : 148;
     TcPlan plan;
-    if (!plan_tc(d->N, Ho, Wo, p->ksize, S, (p->Cout + kMTile - 1) / kMTile, sms, &plan))
+    // narrow layers put the positions on the M operand (all 128 TMEM lanes carry outputs whatever Cout is)
+    const bool pxm = use_pxm(p);
+    const int w_rows = pxm ? round_up(p->Cout, 16) : kMTile;
+    if (!plan_tc(d->N, Ho, Wo, p->ksize, S, (p->Cout + kMTile - 1) / kMTile, sms, pxm, w_rows, &plan))
         return (int)cudaErrorInvalidConfiguration;
 
     TcArgs a;
@@ -586,14 +706,15 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     a.tiles_y = (Ho + plan.TH - 1) / plan.TH;
     a.co_tiles = (p->Cout + N_T - 1) / N_T;
     a.a_stage_bytes = plan.n_sub * plan.sub_rows * kRowBytes;
-    a.b_stage_bytes = plan.G * N_T * kRowBytes;
+    a.w_rows = w_rows;
+    a.b_stage_bytes = plan.G * w_rows * kRowBytes;
     a.G = plan.G;
     a.NA = plan.NA;
     a.NB = plan.NB;
     a.AS = 2;
     a.acc_cols = round_up(plan.N_px, 32);  // the epilogue reads 32 columns at a time
     a.a_tx_bytes = (unsigned)(kKBlock * 2 * plan.Wq * plan.rows_staged);  // per sub-tile
-    a.b_tx_bytes = (unsigned)(kKBlock * 2 * N_T);
+    a.b_tx_bytes = (unsigned)(kKBlock * 2 * w_rows);
     a.act = (int)d->act;
     a.y_c_off = d->y_channel_offset;
     a.y_c_stride = d->y_channel_stride ? d->y_channel_stride : p->Cout;
@@ -601,6 +722,13 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     // instruction descriptor: fp32 accumulate, A and B of the io type, both K-major, N/8 and M/16
     const unsigned fmt = a.is_bf16 ? 1u : 0u;
     a.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((unsigned)(plan.N_px >> 3) << 17) | ((unsigned)(kMTile >> 4) << 24);
+    a.pxm = pxm ? 1 : 0;
+    a.MH = plan.N_px > 128 ? 2 : 1;
+    a.n_cols = round_up(p->Cout, 16);
+    if (pxm) {
+        a.acc_cols = round_up(a.MH * a.n_cols, 32);
+        a.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((unsigned)(a.n_cols >> 3) << 17) | ((unsigned)(128 >> 4) << 24);
+    }
     const int cols = a.AS * a.acc_cols;
     int alloc = 32;
     while (alloc < cols) alloc <<= 1;
@@ -633,10 +761,10 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     }
     // weights: one descriptor per handle
     rtoss_tmap_entry* eb = &p->wtc_map;
-    if (!eb->valid || eb->base != p->wtc || eb->dims[0] != N_T) {
+    if (!eb->valid || eb->base != p->wtc || eb->dims[0] != w_rows) {
         cuuint64_t dims[3] = {(cuuint64_t)p->Cin, (cuuint64_t)p->Cout, (cuuint64_t)taps};
         cuuint64_t strides[2] = {(cuuint64_t)p->Cin * 2, (cuuint64_t)p->Cout * p->Cin * 2};
-        cuuint32_t box[3] = {(cuuint32_t)kKBlock, (cuuint32_t)N_T, 1};
+        cuuint32_t box[3] = {(cuuint32_t)kKBlock, (cuuint32_t)w_rows, 1};
         cuuint32_t es[3] = {1, 1, 1};
         eb->valid = 0;
         CUresult r = enc(reinterpret_cast<CUtensorMap*>(eb->map), dt, 3, p->wtc, dims, strides, box, es,
@@ -644,7 +772,7 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return (int)cudaErrorInvalidValue;
         eb->base = p->wtc;
-        eb->dims[0] = N_T;
+        eb->dims[0] = w_rows;
         eb->valid = 1;
     }
     const CUtensorMap& tmA = *reinterpret_cast<const CUtensorMap*>(ea->map);
