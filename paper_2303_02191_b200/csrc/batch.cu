@@ -40,7 +40,7 @@ struct BatchLayer {
     uint32_t* perm;
     uint32_t* bucket_off;
     long long n_kernels;
-    long long n_dense;  // Cout*Cin
+    rtoss_wtc_layout lay;  // layout of wtc
     int Cout, Cin, ksize, P, k;
     int w_dtype, sel_dtype, v_dtype;
     unsigned chunk0;  // first chunk of this layer
@@ -106,12 +106,14 @@ __global__ void __launch_bounds__(kChunk) batch_select_pack_kernel(const BatchLa
             }
             const unsigned m = s_masks[best];
             if (L.v_dtype == RTOSS_F32)
-                rtoss_dev::pack_one<float>(v, m, i, L.k, (float*)L.val, (float*)L.wtc, L.ksize, L.n_dense);
+                rtoss_dev::pack_one<float>(v, m, i, L.k, (float*)L.val, (float*)L.wtc, L.ksize, L.Cin, L.lay.rows, L.lay.rep_rows,
+                                           L.lay.copies);
             else if (L.v_dtype == RTOSS_BF16)
-                rtoss_dev::pack_one<__nv_bfloat16>(v, m, i, L.k, (__nv_bfloat16*)L.val, (__nv_bfloat16*)L.wtc, L.ksize,
-                                                   L.n_dense);
+                rtoss_dev::pack_one<__nv_bfloat16>(v, m, i, L.k, (__nv_bfloat16*)L.val, (__nv_bfloat16*)L.wtc, L.ksize, L.Cin,
+                                                   L.lay.rows, L.lay.rep_rows, L.lay.copies);
             else
-                rtoss_dev::pack_one<__half>(v, m, i, L.k, (__half*)L.val, (__half*)L.wtc, L.ksize, L.n_dense);
+                rtoss_dev::pack_one<__half>(v, m, i, L.k, (__half*)L.val, (__half*)L.wtc, L.ksize, L.Cin, L.lay.rows, L.lay.rep_rows,
+                                            L.lay.copies);
         }
     }
 }
@@ -212,7 +214,7 @@ rtoss_status rtoss_batch_create(rtoss_ctx* ctx, const rtoss_batch_item* items, i
         B.perm = p->perm;
         B.bucket_off = p->bucket_off;
         B.n_kernels = p->n_kernels;
-        B.n_dense = (long long)it.Cout * it.Cin;
+        B.lay = rtoss_wtc_layout_of(it.Cout, it.ksize);
         B.Cout = it.Cout;
         B.Cin = it.Cin;
         B.ksize = it.ksize;

@@ -83,6 +83,7 @@ struct TcArgs {
     unsigned idesc;
     int tmem_cols;
     int w_rows;           // filter rows per staged weight tile (128; fewer with positions as the M operand)
+    int rep_rows, R;      // filters as M, narrow layer: the tile holds R copies of rep_rows filter rows (else 128, 1)
     int pxm, MH, n_cols;  // positions as the M operand: M halves of 128 positions per tile, filters per tile (the MMA's N)
 };
 
@@ -463,7 +464,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const unsigned d_base = tmem_base + (unsigned)(as * a.acc_cols) + ((unsigned)(quarter * 32) << 16);
-            const int co = co0 + quarter * 32 + lane;  // this thread's filter: TMEM lane = filter
+            // TMEM lane = filter.  A narrow layer's filters are repeated down the lanes (R copies): every lane quarter
+            // then holds outputs, and the copies share the tile's columns between them.
+            const int row0 = (quarter * 32) % a.rep_rows, copy = (quarter * 32) / a.rep_rows;
+            const int co = co0 + row0 + lane;
             const bool co_ok = co < a.Cout;
             const float bv = (a.bias && co_ok) ? __ldg(a.bias + co) : 0.f;
             // A warp holds 32 filters (lanes) x 32 positions (registers); NHWC wants the filters of one
@@ -471,8 +475,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // (position-major rows of 64 + 16 pad bytes) so that global stores are 16 bytes per lane,
             // four lanes covering the 64 contiguous bytes of one position.
             unsigned char* patch = epi_patch + (warp - 2) * (kPatchRows * kPatchPitch);
-            const bool vec_ok = (a.y_c_stride % 8 == 0) && ((a.y_c_off + co0) % 8 == 0) && (co0 + quarter * 32 + 32 <= a.Cout);
-            for (int c0 = sub * 32; c0 < a.N_px; c0 += 128) {
+            const bool vec_ok = (a.y_c_stride % 8 == 0) && ((a.y_c_off + co0) % 8 == 0) && (co0 + row0 + 32 <= a.Cout);
+            for (int c0 = (sub + 4 * copy) * 32; c0 < a.N_px; c0 += 128 * a.R) {
                 unsigned r[32];
                 tmem_ld32(d_base + (unsigned)c0, r);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -499,7 +503,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             if (oyl < a.TH && oxl < a.TW && ox < a.Wo && oy < a.Ho) {
                                 const uint4 o = *reinterpret_cast<const uint4*>(patch + j * kPatchPitch + v * 16);
                                 *reinterpret_cast<uint4*>(yg + (((size_t)n * a.Ho + oy) * a.Wo + ox) * a.y_c_stride + a.y_c_off +
-                                                          co0 + quarter * 32 + v * 8) = o;
+                                                          co0 + row0 + v * 8) = o;
                             }
                         }
                     } else {
@@ -556,7 +560,7 @@ inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 // A narrow layer wastes most of M that way and, worse, leaves three of four epilogue warps without TMEM lanes to
 // read; with the positions as M every lane carries an output and a thread's filters are contiguous in NHWC.  The
 // price is one instruction per 128 positions instead of per 256: taken where few instructions are needed anyway.
-bool use_pxm(const rtoss_packed* p) { return p->Cout <= kPxmMaxCout && (p->ksize == 1 || p->Cin <= 64); }
+bool use_pxm(const rtoss_packed* p) { return p->Cout <= kPxmMaxCout && p->ksize == 1; }
 
 struct TcPlan {
     int TH, TW, Wq, N_px, NA, NB, G, n_sub, sub_rows, rows_staged, tiles_x, smem;
@@ -707,6 +711,10 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     a.co_tiles = (p->Cout + N_T - 1) / N_T;
     a.a_stage_bytes = plan.n_sub * plan.sub_rows * kRowBytes;
     a.w_rows = w_rows;
+    // narrow 3x3 layers keep the filters on M and repeat them down the 128 rows of the tile
+    const rtoss_wtc_layout lay = rtoss_wtc_layout_of(p->Cout, p->ksize);  // how rtoss_pack laid the weights out
+    a.rep_rows = lay.copies > 1 ? lay.rep_rows : 128;
+    a.R = lay.copies;
     a.b_stage_bytes = plan.G * w_rows * kRowBytes;
     a.G = plan.G;
     a.NA = plan.NA;
@@ -762,8 +770,8 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     // weights: one descriptor per handle
     rtoss_tmap_entry* eb = &p->wtc_map;
     if (!eb->valid || eb->base != p->wtc || eb->dims[0] != w_rows) {
-        cuuint64_t dims[3] = {(cuuint64_t)p->Cin, (cuuint64_t)p->Cout, (cuuint64_t)taps};
-        cuuint64_t strides[2] = {(cuuint64_t)p->Cin * 2, (cuuint64_t)p->Cout * p->Cin * 2};
+        cuuint64_t dims[3] = {(cuuint64_t)p->Cin, (cuuint64_t)lay.rows, (cuuint64_t)taps};
+        cuuint64_t strides[2] = {(cuuint64_t)p->Cin * 2, (cuuint64_t)lay.rows * p->Cin * 2};
         cuuint32_t box[3] = {(cuuint32_t)kKBlock, (cuuint32_t)w_rows, 1};
         cuuint32_t es[3] = {1, 1, 1};
         eb->valid = 0;

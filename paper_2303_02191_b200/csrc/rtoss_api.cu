@@ -237,7 +237,8 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
         if (e == cudaSuccess && rtoss_tc_weights_eligible(p)) {
             // dense-expanded weights of the tensor path; zeroed once: the trailing Cout*Cin mod 9 weights of a 1x1
             // layer are pruned for good and no later pack writes them
-            const size_t wtc_bytes = (size_t)(ksize == 3 ? 9 : 1) * Cout * Cin * rtoss_dtype_size(compute_dtype);
+            const size_t wtc_bytes =
+                (size_t)(ksize == 3 ? 9 : 1) * rtoss_wtc_layout_of(Cout, ksize).rows * Cin * rtoss_dtype_size(compute_dtype);
             e = cudaMalloc(&p->wtc, wtc_bytes);
             if (e == cudaSuccess) e = cudaMemsetAsync(p->wtc, 0, wtc_bytes, s);
         }
@@ -253,7 +254,7 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
     if (masks_changed) e = cudaMemcpyAsync(p->masks_dev, p->masks, sizeof(uint16_t) * 256, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess)  // also writes the handle's own copy of the ids and the tensor path's dense-expanded weights
         le = rtoss_launch_pack_values(w_dev, w_dtype, p->n_kernels, make_table(masks_host, P), pid_dev, k, p->val,
-                                      compute_dtype, p->pid, p->wtc, ksize, (int64_t)Cout * Cin, cuda_stream);
+                                      compute_dtype, p->pid, p->wtc, ksize, Cout, Cin, cuda_stream);
     if (e == cudaSuccess && !le && ksize == 3)
         le = rtoss_launch_pack_order(pid_dev, Cout, Cin, P, p->perm, p->bucket_off, cuda_stream);
     if (e != cudaSuccess || le) {

@@ -60,11 +60,32 @@ bool rtoss_table_ok(const uint16_t* masks, int P, int k);
 
 static inline size_t rtoss_dtype_size(rtoss_dtype d) { return d == RTOSS_F32 ? 4 : 2; }
 
+// Layout of the tensor path's dense-expanded weights wtc[tap][row][ci].  Normally row = filter (rows = Cout).  A
+// narrow 3x3 layer (Cout <= 64) stores its filters `copies` times down 128 rows, copy c of filter co at row
+// c*rep_rows + co (rows in between stay zero): the MMA then fills all 128 accumulator lanes with outputs and every
+// epilogue warp has lanes to read.
+struct rtoss_wtc_layout {
+    int rows, rep_rows, copies;
+};
+static inline rtoss_wtc_layout rtoss_wtc_layout_of(int Cout, int ksize) {
+    rtoss_wtc_layout l;
+    if (ksize == 3 && Cout <= 64) {
+        l.rep_rows = Cout <= 32 ? 32 : 64;
+        l.rows = 128;
+        l.copies = 128 / l.rep_rows;
+    } else {
+        l.rows = Cout;
+        l.rep_rows = Cout;
+        l.copies = 1;
+    }
+    return l;
+}
+
 // kernel launchers (select_pack.cu, conv3x3_alu.cu, conv1x1_alu.cu); each returns a cudaError_t as int
 int rtoss_launch_select(const void* w, rtoss_dtype wdt, int64_t n_kernels, const MaskTable& t, int P, uint8_t* pid,
                         void* stream);
 int rtoss_launch_pack_values(const void* w, rtoss_dtype wdt, int64_t n_kernels, const MaskTable& t, const uint8_t* pid,
-                             int k, void* val, rtoss_dtype vdt, uint8_t* pid_copy, void* wtc, int ksize, int64_t n_dense,
+                             int k, void* val, rtoss_dtype vdt, uint8_t* pid_copy, void* wtc, int ksize, int Cout, int Cin,
                              void* stream);
 int rtoss_launch_pack_order(const uint8_t* pid, int Cout, int Cin, int P, uint32_t* perm, uint32_t* bucket_off,
                             void* stream);

@@ -44,21 +44,26 @@ template <> __device__ __forceinline__ __half narrow_to<__half>(float v) { retur
 
 // Writes of one kernel (3x3) or run of nine (1x1) with mask m: its k kept values, ascending taps, rounded to V, to
 // val[i*k ...]; and, where the handle carries dense-expanded weights for the tensor path (wtc != nullptr), all nine
-// taps, pruned ones as +0:  3x3 -> wtc[t][co][ci] (i = co*Cin+ci, n = Cout*Cin);  1x1 -> wtc[9*i + t].
+// taps, pruned ones as +0:  3x3 -> wtc[t][row][ci] with `rows` rows per tap, filter co = i / Cin at rows
+// c*rep_rows + co for c < copies (one copy at row co in the plain layout);  1x1 -> wtc[9*i + t].
 template <typename V>
 __device__ __forceinline__ void pack_one(const float (&w)[9], unsigned m, int64_t i, int k, V* __restrict__ val,
-                                         V* __restrict__ wtc, int ksize, int64_t n) {
+                                         V* __restrict__ wtc, int ksize, int Cin, int rows, int rep_rows, int copies) {
     V* out = val + i * k;
     int j = 0;
 #pragma unroll
     for (int t = 0; t < 9; ++t)
         if (m & (1u << t)) out[j++] = narrow_to<V>(w[t]);
     if (wtc) {
+        const int64_t co = i / Cin, ci = i - co * Cin;
 #pragma unroll
         for (int t = 0; t < 9; ++t) {
             const V v = (m & (1u << t)) ? narrow_to<V>(w[t]) : narrow_to<V>(0.f);
-            if (ksize == 3) wtc[(int64_t)t * n + i] = v;
-            else wtc[i * 9 + t] = v;
+            if (ksize == 3) {
+                for (int c = 0; c < copies; ++c) wtc[((int64_t)t * rows + c * rep_rows + co) * Cin + ci] = v;
+            } else {
+                wtc[i * 9 + t] = v;
+            }
         }
     }
 }

@@ -75,7 +75,8 @@ template <typename T, typename V>
 __global__ void __launch_bounds__(kSelThreads) pack_values_kernel(const T* __restrict__ w, int64_t n_kernels,
                                                                   MaskTable table, const uint8_t* pid, int k,
                                                                   V* __restrict__ val, uint8_t* pid_copy,
-                                                                  V* __restrict__ wtc, int ksize, int64_t n_dense) {
+                                                                  V* __restrict__ wtc, int ksize, int Cin,
+                                                                  rtoss_wtc_layout lay) {
     rtoss_dev::pdl_enter();
     __shared__ __align__(16) T sw[kSelThreads * 9];
     const int64_t n_chunks = (n_kernels + kSelThreads - 1) / kSelThreads;
@@ -92,7 +93,7 @@ __global__ void __launch_bounds__(kSelThreads) pack_values_kernel(const T* __res
             float v[9];
 #pragma unroll
             for (int t = 0; t < 9; ++t) v[t] = widen<T>(sw[threadIdx.x * 9 + t]);
-            rtoss_dev::pack_one<V>(v, table.m[id], i, k, val, wtc, ksize, n_dense);
+            rtoss_dev::pack_one<V>(v, table.m[id], i, k, val, wtc, ksize, Cin, lay.rows, lay.rep_rows, lay.copies);
         }
     }
 }
@@ -153,28 +154,29 @@ int rtoss_launch_select(const void* w, rtoss_dtype wdt, int64_t n_kernels, const
 
 template <typename T>
 static int launch_pack_values_t(const T* w, int64_t n, const MaskTable& t, const uint8_t* pid, int k, void* val,
-                                rtoss_dtype vdt, uint8_t* pid_copy, void* wtc, int ksize, int64_t n_dense, cudaStream_t s) {
+                                rtoss_dtype vdt, uint8_t* pid_copy, void* wtc, int ksize, int Cin, rtoss_wtc_layout lay, cudaStream_t s) {
     const int grid = grid_for((n + kSelThreads - 1) / kSelThreads);
     switch (vdt) {
-        case RTOSS_F32: rtoss_dev::launch_pdl(pack_values_kernel<T, float>, grid, kSelThreads, 0, s, w, n, t, pid, k, (float*)val, pid_copy, (float*)wtc, ksize, n_dense); break;
+        case RTOSS_F32: rtoss_dev::launch_pdl(pack_values_kernel<T, float>, grid, kSelThreads, 0, s, w, n, t, pid, k, (float*)val, pid_copy, (float*)wtc, ksize, Cin, lay); break;
         case RTOSS_BF16:
-            rtoss_dev::launch_pdl(pack_values_kernel<T, __nv_bfloat16>, grid, kSelThreads, 0, s, w, n, t, pid, k, (__nv_bfloat16*)val, pid_copy, (__nv_bfloat16*)wtc, ksize, n_dense);
+            rtoss_dev::launch_pdl(pack_values_kernel<T, __nv_bfloat16>, grid, kSelThreads, 0, s, w, n, t, pid, k, (__nv_bfloat16*)val, pid_copy, (__nv_bfloat16*)wtc, ksize, Cin, lay);
             break;
-        case RTOSS_F16: rtoss_dev::launch_pdl(pack_values_kernel<T, __half>, grid, kSelThreads, 0, s, w, n, t, pid, k, (__half*)val, pid_copy, (__half*)wtc, ksize, n_dense); break;
+        case RTOSS_F16: rtoss_dev::launch_pdl(pack_values_kernel<T, __half>, grid, kSelThreads, 0, s, w, n, t, pid, k, (__half*)val, pid_copy, (__half*)wtc, ksize, Cin, lay); break;
     }
     return (int)cudaGetLastError();
 }
 
 int rtoss_launch_pack_values(const void* w, rtoss_dtype wdt, int64_t n_kernels, const MaskTable& t, const uint8_t* pid,
-                             int k, void* val, rtoss_dtype vdt, uint8_t* pid_copy, void* wtc, int ksize, int64_t n_dense,
+                             int k, void* val, rtoss_dtype vdt, uint8_t* pid_copy, void* wtc, int ksize, int Cout, int Cin,
                              void* stream) {
+    const rtoss_wtc_layout lay = rtoss_wtc_layout_of(Cout, ksize);
     if (n_kernels <= 0) return 0;
     cudaStream_t s = (cudaStream_t)stream;
     switch (wdt) {
-        case RTOSS_F32: return launch_pack_values_t<float>((const float*)w, n_kernels, t, pid, k, val, vdt, pid_copy, wtc, ksize, n_dense, s);
+        case RTOSS_F32: return launch_pack_values_t<float>((const float*)w, n_kernels, t, pid, k, val, vdt, pid_copy, wtc, ksize, Cin, lay, s);
         case RTOSS_BF16:
-            return launch_pack_values_t<__nv_bfloat16>((const __nv_bfloat16*)w, n_kernels, t, pid, k, val, vdt, pid_copy, wtc, ksize, n_dense, s);
-        case RTOSS_F16: return launch_pack_values_t<__half>((const __half*)w, n_kernels, t, pid, k, val, vdt, pid_copy, wtc, ksize, n_dense, s);
+            return launch_pack_values_t<__nv_bfloat16>((const __nv_bfloat16*)w, n_kernels, t, pid, k, val, vdt, pid_copy, wtc, ksize, Cin, lay, s);
+        case RTOSS_F16: return launch_pack_values_t<__half>((const __half*)w, n_kernels, t, pid, k, val, vdt, pid_copy, wtc, ksize, Cin, lay, s);
     }
     return (int)cudaErrorInvalidValue;
 }

@@ -140,3 +140,44 @@ def test_tensor_path_refuses_what_it_cannot_take():
         gu.run_conv(packed, 3, x8, "bf16", 1, "none", None, "nhwc", path=rt.PATH_TENSOR)
     assert e.value.status == 3
     packed.close()
+
+
+# Narrow layers run with the positions as the M operand of the MMA (filters as N): cases that differ there --
+# filter counts around the 16-column read, one or two halves of 128 positions per tile, many tiles per CTA
+NARROW = [
+    # ksize, stride, N, Cin, Cout, H, W, k, dt, act, bias
+    (1, 1, 1, 64, 8, 12, 10, 4, "bf16", "silu", True),       # one 16-filter read, half of it real; 120 positions: one half
+    (1, 1, 1, 32, 64, 9, 16, 3, "f16", "none", False),       # 144 positions: two halves, the second nearly empty
+    (1, 1, 4, 64, 32, 160, 160, 4, "bf16", "silu", True),    # several tiles per CTA, both accumulator stages in turn
+    (3, 1, 2, 32, 32, 64, 64, 4, "bf16", "relu", True),      # half-filled channel block: two of four K slabs issued
+    (3, 1, 1, 48, 40, 33, 21, 2, "f16", "silu", True),       # ragged filter count (40 of 48 columns), ragged channels
+    (3, 2, 3, 16, 64, 31, 45, 3, "bf16", "silu", True),      # stride 2, odd sizes
+    (1, 2, 2, 256, 48, 40, 40, 4, "bf16", "relu", False),    # deep K, strided 1x1
+]
+
+
+@pytest.mark.parametrize("case", NARROW, ids=lambda c: "-".join(str(v) for v in c))
+def test_tensor_path_narrow_layers(case):
+    ks, s, N, Cin, Cout, H, W, k, dt, act, use_bias = case
+    gu.check_layer(26, 900 + Cin + Cout + W, ks, N, Cin, Cout, H, W, s, k, _table(k), dt, act, "nhwc", use_bias=use_bias,
+                   path=rt.PATH_TENSOR)
+    _no_timeout()
+
+
+@pytest.mark.parametrize("y_off,y_stride", [(8, 96), (5, 77)])
+def test_tensor_path_narrow_channel_slice(y_off, y_stride):
+    """Output written into a channel slice: aligned (16-byte stores) and unaligned (element stores); the rest of
+    the buffer keeps its fill value."""
+    masks = _table(4)
+    N, Cin, Cout, H, W = 2, 64, 32, 19, 23
+    x = synth.round_like(synth.activations(27, 1, N, Cin, H, W), "bf16")
+    w = synth.kaiming_weights(27, 1, Cout, Cin, 3)
+    b = synth.bias(27, 1, Cout)
+    _, packed = gu.select_pack(w, 3, masks, 4, "bf16")
+    _, wd, _ = gu.oracle_weights(w, 3, masks, 4, "bf16")
+    y = gu.run_conv(packed, 3, x, "bf16", 1, "silu", b, "nhwc", y_off=y_off, y_stride=y_stride, path=rt.PATH_TENSOR)
+    assert (y[:, :y_off] == 7.0).all() and (y[:, y_off + Cout:] == 7.0).all()
+    ref = gu.oracle_conv(3, x, wd, b, 1, "silu", "bf16")
+    assert orc.rel_err(y[:, y_off:y_off + Cout], ref) <= gu.TOL["bf16"]
+    _no_timeout()
+    packed.close()
