@@ -331,63 +331,115 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else if (warp == 1) {
         // ---------------- MMA issuer
         if (lane == 0) {
+            // One thread issues every tcgen05.mma, so the instructions between two of them are the budget: with one or
+            // two instructions per tap (few channels, or few filters with the positions as M) the tensor pipe waits
+            // for this thread.  Hence: ring positions and phases are carried as counters (no division), a descriptor
+            // is a constant high word plus address / 16 in the low word (addresses stay below 2^18: adding never
+            // carries out of the field), a tap's offset is a register picked by a compile-time index (the taps of
+            // a 3x3 layer are unrolled), and K steps (+2 = 32 bytes = 16 channels) or the second half of the
+            // positions (+1024 = 128 rows) are additions.
             bool ok = true;
-            int ga = 0, gb = 0, gt = 0;
-            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++gt) {
-                const int as = gt % a.AS;
-                ok = mbar_wait(bar_accEmpty + 8 * as, ((gt / a.AS) & 1) ^ 1);  // epilogue has drained this stage
+            const unsigned long long d0 = make_sw128_desc(0);
+            const unsigned desc_hi = (unsigned)(d0 >> 32), desc_lo0 = (unsigned)d0;
+            unsigned tap16[9];
+#pragma unroll
+            for (int t = 0; t < 9; ++t) tap16[t] = (unsigned)(a.tap_sub[t] * a.sub_bytes + a.tap_shift[t] * kRowBytes) >> 4;
+            const unsigned wtile16 = (unsigned)(a.w_rows * kRowBytes) >> 4;
+            const unsigned astage16 = (unsigned)a.a_stage_bytes >> 4, bstage16 = (unsigned)a.b_stage_bytes >> 4;
+            const unsigned idesc = a.idesc, hi_cols = (unsigned)a.n_cols;
+            const bool pxm = a.pxm != 0, two = a.MH == 2, unrolled9 = a.taps == 9 && a.G == 3;
+            int sa = 0, sb = 0, as = 0, n_done = 0;
+            unsigned pa = 0, pb = 0, pacc = 0;  // phase parities of the three rings
+            auto mk = [desc_hi](unsigned lo) { return ((unsigned long long)desc_hi << 32) | lo; };
+            // all instructions of one tap: nk4 K slabs (times two halves of positions with the positions as M)
+            auto issue_tap = [&](unsigned d_base, unsigned wl, unsigned xl, int nk4, unsigned& acc) {
+                if (pxm) {
+#pragma unroll
+                    for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
+                        if (k4 < nk4) {
+                            umma_f16(d_base, mk(xl + 2 * k4), mk(wl + 2 * k4), idesc, acc);
+                            if (two) umma_f16(d_base + hi_cols, mk(xl + 1024 + 2 * k4), mk(wl + 2 * k4), idesc, acc);
+                            acc = 1;
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
+                        if (k4 < nk4) {
+                            umma_f16(d_base, mk(wl + 2 * k4), mk(xl + 2 * k4), idesc, acc);
+                            acc = 1;
+                        }
+                    }
+                }
+            };
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++n_done) {
+                ok = mbar_wait(bar_accEmpty + 8 * as, pacc ^ 1);  // epilogue has drained this stage
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const unsigned d_base = tmem_base + (unsigned)(as * a.acc_cols);
-                for (int cb = 0; cb < a.ncb && ok; ++cb, ++ga) {
-                    const int sa = ga % a.NA;
-                    ok = mbar_wait(bar_fullA + 8 * sa, (ga / a.NA) & 1);
+                unsigned acc = 0;  // the first instruction of a tile overwrites the accumulator
+                int left = a.Cin;
+                for (int cb = 0; cb < a.ncb && ok; ++cb, left -= kKBlock) {
+                    ok = mbar_wait(bar_fullA + 8 * sa, pa);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const unsigned a_tile = sA + sa * a.a_stage_bytes;
+                    const unsigned xl0 = desc_lo0 + (sA >> 4) + (unsigned)sa * astage16;
                     // 16-channel slabs of this block that hold channels (the rest of the 64 is TMA zero fill)
-                    const int left = a.Cin - cb * kKBlock;
                     const int nk4 = left >= kKBlock ? kKBlock / 16 : (left + 15) >> 4;
-                    for (int t0 = 0; t0 < a.taps; t0 += a.G, ++gb) {
-                        const int sb = gb % a.NB;
-                        ok = mbar_wait(bar_fullB + 8 * sb, (gb / a.NB) & 1);
-                        if (!ok) break;
-                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                        for (int i = 0; i < a.G; ++i) {
-                            const int t = t0 + i;
-                            const unsigned w_tile = sB + sb * a.b_stage_bytes + i * (a.w_rows * kRowBytes);
-                            const unsigned x_rows = a_tile + (unsigned)(a.tap_sub[t] * a.sub_bytes + a.tap_shift[t] * kRowBytes);  // N operand
-                            // One thread issues everything, so the instructions between two tcgen05.mma are the budget:
-                            // the descriptors of a tap are built once and stepped by adding to their address field
-                            // (+2 = 32 bytes = 16 channels; +1024 = 128 rows), the loops are unrolled and predicated.
-                            const unsigned long long wd = make_sw128_desc(w_tile), xd = make_sw128_desc(x_rows);
-                            if (a.pxm) {
-                                // positions are the M operand: one instruction per half of 128 positions; the halves
-                                // accumulate side by side in TMEM
-                                const unsigned d_hi = d_base + (unsigned)a.n_cols;
+                    if (unrolled9) {
 #pragma unroll
-                                for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
-                                    if (k4 < nk4) {
-                                        umma_f16(d_base, xd + 2 * k4, wd + 2 * k4, a.idesc, (cb | t | k4) != 0);
-                                        if (a.MH == 2) umma_f16(d_hi, xd + 1024 + 2 * k4, wd + 2 * k4, a.idesc, (cb | t | k4) != 0);
-                                    }
+                        for (int s3 = 0; s3 < 3; ++s3) {
+                            ok = ok && mbar_wait(bar_fullB + 8 * sb, pb);
+                            if (ok) {
+                                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                                const unsigned wl0 = desc_lo0 + (sB >> 4) + (unsigned)sb * bstage16;
+#pragma unroll
+                                for (int i = 0; i < 3; ++i) issue_tap(d_base, wl0 + i * wtile16, xl0 + tap16[s3 * 3 + i], nk4, acc);
+                                umma_commit(bar_emptyB + 8 * sb);  // this weight stage may be refilled once the MMAs have read it
+                                if (++sb == a.NB) {
+                                    sb = 0;
+                                    pb ^= 1;
                                 }
-                            } else {
-#pragma unroll
-                                for (int k4 = 0; k4 < kKBlock / 16; ++k4)
-                                    if (k4 < nk4) umma_f16(d_base, wd + 2 * k4, xd + 2 * k4, a.idesc, (cb | t | k4) != 0);
                             }
                         }
-                        umma_commit(bar_emptyB + 8 * sb);  // this weight stage may be refilled once the MMAs have read it
+                    } else {
+                        for (int t0 = 0; t0 < a.taps && ok; t0 += a.G) {
+                            ok = mbar_wait(bar_fullB + 8 * sb, pb);
+                            if (!ok) break;
+                            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                            const unsigned wl0 = desc_lo0 + (sB >> 4) + (unsigned)sb * bstage16;
+                            for (int i = 0; i < a.G; ++i) {
+                                const unsigned off =
+                                    (unsigned)(a.tap_sub[t0 + i] * a.sub_bytes + a.tap_shift[t0 + i] * kRowBytes) >> 4;
+                                issue_tap(d_base, wl0 + i * wtile16, xl0 + off, nk4, acc);
+                            }
+                            umma_commit(bar_emptyB + 8 * sb);
+                            if (++sb == a.NB) {
+                                sb = 0;
+                                pb ^= 1;
+                            }
+                        }
                     }
                     if (ok) umma_commit(bar_emptyA + 8 * sa);
+                    if (++sa == a.NA) {
+                        sa = 0;
+                        pa ^= 1;
+                    }
                 }
                 if (ok) umma_commit(bar_accFull + 8 * as);
+                if (++as == a.AS) {
+                    as = 0;
+                    pacc ^= 1;
+                }
             }
-            // TMEM may only be released after the epilogue has drained the last tiles
-            for (int i = 0; i < a.AS && i < gt && ok; ++i) {
-                const int g = gt - 1 - i;
-                ok = mbar_wait(bar_accEmpty + 8 * (g % a.AS), (g / a.AS) & 1);
+            // TMEM may only be released after the epilogue has drained the last tiles: the last min(AS, tiles done)
+            // stages used, walking backwards from the ring position
+            for (int i = 0; i < a.AS && i < n_done && ok; ++i) {
+                if (--as < 0) {
+                    as = a.AS - 1;
+                    pacc ^= 1;
+                }
+                ok = mbar_wait(bar_accEmpty + 8 * as, pacc);
             }
             if (!ok) atomicExch(a.status, 2);
         }
