@@ -474,6 +474,18 @@ def run_gpu(args):
             "e2e": {"value": world * N / e2e_s, "unit": "images/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": launches,
         }
+        if args.layers_csv:
+            # per-layer table: cold-L2 kernel time next to the two roofline terms at non-zero FLOPs
+            with open(args.layers_csv, "w") as f:
+                f.write("layer,ksize,cin,cout,H,W,stride,k,path,kernel_us,hbm_us,pipe_us,frac\n")
+                for st, ms, fl, by in zip(L_state, conv_ms, flops, bytes_):
+                    L = st["L"]
+                    tc = st["path"] == rt.PATH_TENSOR
+                    pipe_us = fl / ((tc_peak if tc else ALU_PEAK_TFLOPS) * 1e12) * 1e6
+                    hbm_us = by / (hbm_peak * 1e9) * 1e6
+                    f.write("%s,%d,%d,%d,%d,%d,%d,%d,%s,%.2f,%.2f,%.2f,%.3f\n" % (
+                        L["name"], L["ksize"], L["cin"], L["cout"], L["H"], L["W"], L["stride"], st["k"],
+                        "tensor" if tc else "fma", ms * 1e3, hbm_us, pipe_us, max(hbm_us, pipe_us) / (ms * 1e3)))
         if args.cpu_baseline:
             v_cpu, t_cpu, f_cpu, n_cpu = cpu_baseline_sample(layers_k, dtype, N, 15.0)
             out["cpu_baseline"] = {"value": v_cpu, "unit": "images/s", "cores": os.cpu_count(), "kind": "oracle",
@@ -500,6 +512,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--no-graph", dest="graph", action="store_false", help="time eager launches instead of a CUDA graph")
     ap.add_argument("--path", default="auto", choices=["auto", "fma"], help="fma: keep every layer on the FMA path")
+    ap.add_argument("--layers-csv", default=None, help="write the per-layer kernel times and roofline terms to this file")
     ap.add_argument("--layout", default="auto", choices=["auto", "nchw"], help="nchw: NCHW activations also for 16-bit types")
     args = ap.parse_args()
     if args.impl == "reference":

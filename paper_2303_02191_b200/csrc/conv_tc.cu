@@ -59,6 +59,9 @@ constexpr int kMaxA = 4, kMaxB = 8;  // most activation stages / weight slots
 constexpr int kMTile = 128;          // filters per tile = TMEM lanes
 constexpr int kPxmMaxCout = 64;      // layers this narrow run with positions as the M operand
 constexpr int kPatchPitch = 80;      // bytes per position row of an epilogue transpose patch (64 + pad)
+constexpr int kMaxPx = 256;          // most positions in a tile's list
+constexpr int kPairPitch = 144;      // bytes per row (a pair of positions x 32 filters, + 16 pad) of the packed patch
+static_assert(kPatchRows / 2 * kPairPitch <= kPatchRows * kPatchPitch, "the packed patch must fit the warp's patch");
 constexpr int kKBlock = 64;       // channels per staged block: 128 bytes of bf16 / fp16
 constexpr int kRowBytes = 128;    // one padded pixel, one channel block
 constexpr long long kWaitCycles = 2000000000LL;  // about one second
@@ -216,25 +219,119 @@ __device__ __forceinline__ void act_pack16(const unsigned (&r)[16], const float*
     }
 }
 
-// Sixteen positions (registers J0 .. J0+15 of a 32-position chunk) of one filter: bias, activation,
-// rounding, into the transpose patch.
-template <typename T, int ACT, int J0>
-__device__ __forceinline__ void act_to_patch(const unsigned (&r)[32], float bv, unsigned char* col) {
-#pragma unroll
-    for (int j = 0; j < kPatchRows; ++j) {
-        float v = __uint_as_float(r[J0 + j]) + bv;
-        if (ACT == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
-        if (ACT == RTOSS_ACT_SILU) {
-            // v * sigmoid(v) with sigmoid(v) = 0.5 * tanh(v / 2) + 0.5: one special-function op per element
-            // (tanh.approx, relative error about 2^-11: below half an ulp of bf16, about one ulp of fp16)
-            float th;
-            asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(0.5f * v));
-            v = v * fmaf(0.5f, th, 0.5f);
-        }
-        *reinterpret_cast<T*>(col + j * kPatchPitch) = from_f32<T>(v);
-    }
+// Two fp32 values rounded to the 16-bit output type and packed (lo in the low half), with the ReLU folded into
+// the conversion where asked for.
+template <typename T, bool RELU>
+__device__ __forceinline__ unsigned round_pack(float lo, float hi);
+template <>
+__device__ __forceinline__ unsigned round_pack<__nv_bfloat16, false>(float lo, float hi) {
+    return pack2<__nv_bfloat16>(lo, hi);
+}
+template <>
+__device__ __forceinline__ unsigned round_pack<__half, false>(float lo, float hi) {
+    return pack2<__half>(lo, hi);
+}
+template <>
+__device__ __forceinline__ unsigned round_pack<__nv_bfloat16, true>(float lo, float hi) {
+    unsigned d;
+    asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+template <>
+__device__ __forceinline__ unsigned round_pack<__half, true>(float lo, float hi) {
+    unsigned d;
+    asm("cvt.rn.relu.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
 }
 
+// Bias and activation of one accumulator value.  bs is the bias, for SiLU half the bias:
+//   v * sigmoid(v) = h + h * tanh(h) with h = v / 2 = fma(acc, 0.5, b / 2): two fused multiply-adds around one
+//   special-function op (tanh.approx, relative error about 2^-11: below half an ulp of bf16, about one ulp of
+//   fp16).  ReLU is left to the conversion.
+template <int ACT>
+__device__ __forceinline__ float bias_act(unsigned acc_bits, float bs) {
+    const float acc = __uint_as_float(acc_bits);
+    if (ACT == RTOSS_ACT_SILU) {
+        const float h = fmaf(acc, 0.5f, bs);
+        float th;
+        asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(h));
+        return fmaf(h, th, h);
+    }
+    return acc + bs;
+}
+
+// One tile of the filters-as-M epilogue for one warp: its lane quarter of the accumulator stage at d_base, the
+// 32-column chunks c0, c0 + c_step, ...  A warp holds 32 filters (lanes) x 32 positions (registers); NHWC wants
+// the filters of one position side by side.  The shared-memory pipe (one 128-byte wavefront a cycle, which the
+// tensor cores' operand reads also use) is what bounds this, so the transpose moves full wavefronts:
+//   * a lane rounds two neighbouring positions of its filter into one 32-bit word and stores it to row
+//     (position pair), column (filter) of the warp's patch: eight conflict-free 128-byte stores per 16 positions;
+//   * lane (pair jp = lane / 4, filter group v = lane % 4) reads the eight words of its group (two 16-byte
+//     loads; rows are 36 words apart, so the two rows a quarter warp touches fall on disjoint banks), splits
+//     them into the low halves (position 2 jp) and the high halves (position 2 jp + 1) and writes each as one
+//     16-byte store: four lanes cover the 64 contiguous bytes of a position.
+// Where a position goes comes from the table built in the prologue (no division here): tab[p] = {element offset
+// inside the tile, row << 16 | column}.  patch and tab are shared-memory addresses (32 bits: the accesses are
+// spelled out so that none is compiled as a generic one).
+// Sixteen positions of one filter (a half chunk): round, transpose through the patch, store.  See epilogue_chunks.
+template <typename T, int ACT>
+__device__ __forceinline__ void epilogue_half(const unsigned (&r)[16], float bs, unsigned wr, unsigned rd, unsigned tab_at,
+                                              T* ybv, unsigned ry, unsigned rx) {
+#pragma unroll
+    for (int jp = 0; jp < kPatchRows / 2; ++jp) {
+        const unsigned w = round_pack<T, ACT == RTOSS_ACT_RELU>(bias_act<ACT>(r[2 * jp], bs), bias_act<ACT>(r[2 * jp + 1], bs));
+        asm volatile("st.shared.u32 [%0], %1;" ::"r"(wr + jp * kPairPitch), "r"(w) : "memory");
+    }
+    __syncwarp();
+    unsigned w[8], e[4];
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(rd));
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "r"(rd + 16));
+    // table entries of positions 2 jp and 2 jp + 1 (an even position: 16-byte aligned)
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(e[0]), "=r"(e[1]), "=r"(e[2]), "=r"(e[3]) : "r"(tab_at));
+    if ((e[1] >> 16) < ry && (e[1] & 0xFFFFu) < rx)
+        *reinterpret_cast<uint4*>(ybv + e[0]) = make_uint4(__byte_perm(w[0], w[1], 0x5410), __byte_perm(w[2], w[3], 0x5410),
+                                                           __byte_perm(w[4], w[5], 0x5410), __byte_perm(w[6], w[7], 0x5410));
+    if ((e[3] >> 16) < ry && (e[3] & 0xFFFFu) < rx)
+        *reinterpret_cast<uint4*>(ybv + e[2]) = make_uint4(__byte_perm(w[0], w[1], 0x7632), __byte_perm(w[2], w[3], 0x7632),
+                                                           __byte_perm(w[4], w[5], 0x7632), __byte_perm(w[6], w[7], 0x7632));
+    __syncwarp();
+}
+
+// One tile of the filters-as-M epilogue for one warp: its lane quarter of the accumulator stage at d_base, the
+// 32-column chunks c0, c0 + c_step, ...  A warp holds 32 filters (lanes) x 16 positions (registers) at a time;
+// NHWC wants the filters of one position side by side.  The shared-memory pipe (one 128-byte wavefront a cycle,
+// which the tensor cores' operand reads also use) is what bounds the transpose, so it moves full wavefronts:
+//   * a lane rounds two neighbouring positions of its filter into one 32-bit word and stores it to row
+//     (position pair), column (filter) of the warp's patch: eight conflict-free 128-byte stores per 16 positions;
+//   * lane (pair jp = lane / 4, filter group v = lane % 4) reads the eight words of its group (two 16-byte
+//     loads; rows are 36 words apart, so the two rows a quarter warp touches fall on disjoint banks), splits
+//     them into the low halves (position 2 jp) and the high halves (position 2 jp + 1) and writes each as one
+//     16-byte store: four lanes cover the 64 contiguous bytes of a position.
+// The accumulator is read sixteen columns at a time into two register sets: the load of the next sixteen is in
+// flight while the current ones are processed (a load takes a few hundred cycles when all warps read at once).
+// Where a position goes comes from the table built in the prologue (no division here): tab[p] = {element offset
+// inside the tile, row << 16 | column}.  patch and tab are shared-memory addresses (32 bits: the accesses are
+// spelled out so that none is compiled as a generic one).
+template <typename T, int ACT>
+__device__ __forceinline__ void epilogue_chunks(unsigned d_base, int c0, int c_step, int n_px, float bs,
+                                                unsigned patch, unsigned tab, T* yb, unsigned ry, unsigned rx,
+                                                int lane) {
+    const unsigned wr = patch + lane * 4;                                       // this lane's column of the patch
+    const unsigned rd = patch + (lane >> 2) * kPairPitch + (lane & 3) * 32;   // row lane / 4, filter group lane % 4
+    const unsigned tab_l = tab + (unsigned)(2 * (lane >> 2)) * 8;
+    T* ybv = yb + (lane & 3) * 8;
+    if (c0 >= n_px) return;
+    unsigned ra[16], rb[16];
+    tmem_ld16(d_base + (unsigned)c0, ra);
+    for (; c0 < n_px; c0 += c_step) {
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        tmem_ld16(d_base + (unsigned)(c0 + kPatchRows), rb);
+        epilogue_half<T, ACT>(ra, bs, wr, rd, tab_l + (unsigned)c0 * 8, ybv, ry, rx);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (c0 + c_step < n_px) tmem_ld16(d_base + (unsigned)(c0 + c_step), ra);
+        epilogue_half<T, ACT>(rb, bs, wr, rd, tab_l + (unsigned)(c0 + kPatchRows) * 8, ybv, ry, rx);
+    }
+}
 
 template <typename T>
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -251,6 +348,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const unsigned s_tmem_ptr = bar_accEmpty + 16;
     volatile unsigned* tmem_ptr_gen = reinterpret_cast<volatile unsigned*>(smem_dyn + (s_tmem_ptr - smem_u32(smem_dyn)));
     unsigned char* epi_patch = smem_dyn + (s_tmem_ptr + 16 - smem_u32(smem_dyn));  // [kEpiWarps][kPatchRows][kPatchPitch], 16-byte aligned
+    uint2* pos_tab = reinterpret_cast<uint2*>(epi_patch + kEpiWarps * kPatchRows * kPatchPitch);  // [kMaxPx]
+    const unsigned s_tab = s_tmem_ptr + 16 + kEpiWarps * kPatchRows * kPatchPitch;                // the same, as a shared address
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = a.N * a.tiles_y * a.tiles_x * a.co_tiles;
@@ -274,6 +373,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+    }
+    // Where position p of a tile's list lies: the same for every tile (the tile's origin and the image's edges
+    // come in per tile), so the epilogue looks it up instead of dividing.  {element offset from the tile's first
+    // output, row << 16 | column}; positions that are no output (pitch padding, the list's tail) get 0xFFFFFFFF.
+    for (int p = threadIdx.x; p < kMaxPx; p += kTcThreads) {
+        const int oyl = p / a.Wq, oxl = p - oyl * a.Wq;
+        const bool is_out = p < a.N_px && oyl < a.TH && oxl < a.TW;
+        pos_tab[p] = make_uint2((unsigned)((oyl * a.Wo + oxl) * a.y_c_stride), is_out ? (unsigned)(oyl << 16 | oxl) : 0xFFFFFFFFu);
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s_tmem_ptr), "r"(a.tmem_cols)
@@ -471,13 +578,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const unsigned d_base = tmem_base + (unsigned)(as * a.acc_cols) + ((unsigned)(quarter * 32) << 16);
+                T* yb = yg + (((size_t)n * a.Ho + y0) * a.Wo + x0) * a.y_c_stride + a.y_c_off;
+                const unsigned ry = (unsigned)min(a.TH, a.Ho - y0), rx = (unsigned)min(a.TW, a.Wo - x0);
                 for (int item = sub; item < items; item += 4) {
                     const int h = item / n_chunks, c = item - h * n_chunks;
                     unsigned r[16];
                     tmem_ld16(d_base + (unsigned)(h * a.n_cols + c * 16), r);
-                    const int pos = h * 128 + quarter * 32 + lane;
-                    const int oyl = pos / a.Wq, oxl = pos - oyl * a.Wq, oy = y0 + oyl, ox = x0 + oxl;
-                    const bool px_ok = pos < a.N_px && oyl < a.TH && oxl < a.TW && ox < a.Wo && oy < a.Ho;
+                    const uint2 e = pos_tab[h * 128 + quarter * 32 + lane];
+                    const bool px_ok = (e.y >> 16) < ry && (e.y & 0xFFFFu) < rx;
                     const float* b16 = bias_s + c * 16;
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                     unsigned o[8];
@@ -485,7 +593,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     else if (a.act == RTOSS_ACT_RELU) act_pack16<T, RTOSS_ACT_RELU>(r, b16, o);
                     else act_pack16<T, RTOSS_ACT_NONE>(r, b16, o);
                     if (px_ok) {
-                        T* dst = yg + (((size_t)n * a.Ho + oy) * a.Wo + ox) * a.y_c_stride + a.y_c_off + c * 16;
+                        T* dst = yb + e.x + c * 16;
                         if (vec_ok && c * 16 + 16 <= a.Cout) {
                             reinterpret_cast<uint4*>(dst)[0] = make_uint4(o[0], o[1], o[2], o[3]);
                             reinterpret_cast<uint4*>(dst)[1] = make_uint4(o[4], o[5], o[6], o[7]);
@@ -512,67 +620,49 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int ty = rest % a.tiles_y, n = rest / a.tiles_y;
             const int y0 = ty * a.TH, x0 = tx * a.TW, co0 = cot * kMTile;
             const int as = gt % a.AS;
-            ok = mbar_wait(bar_accFull + 8 * as, (gt / a.AS) & 1);
-            if (!ok) break;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const unsigned d_base = tmem_base + (unsigned)(as * a.acc_cols) + ((unsigned)(quarter * 32) << 16);
+            // Everything that does not need the accumulator comes before the wait for it: the bias is a global load
+            // (a cold one costs more than a thousand cycles) and would otherwise sit on the path of every tile.
             // TMEM lane = filter.  A narrow layer's filters are repeated down the lanes (R copies): every lane quarter
             // then holds outputs, and the copies share the tile's columns between them.
             const int row0 = (quarter * 32) % a.rep_rows, copy = (quarter * 32) / a.rep_rows;
             const int co = co0 + row0 + lane;
             const bool co_ok = co < a.Cout;
             const float bv = (a.bias && co_ok) ? __ldg(a.bias + co) : 0.f;
-            // A warp holds 32 filters (lanes) x 32 positions (registers); NHWC wants the filters of one
-            // position side by side.  The chunk is turned through a private shared-memory patch
-            // (position-major rows of 64 + 16 pad bytes) so that global stores are 16 bytes per lane,
-            // four lanes covering the 64 contiguous bytes of one position.
-            unsigned char* patch = epi_patch + (warp - 2) * (kPatchRows * kPatchPitch);
+            const unsigned patch = s_tmem_ptr + 16 + (unsigned)(warp - 2) * (kPatchRows * kPatchPitch);  // shared address
             const bool vec_ok = (a.y_c_stride % 8 == 0) && ((a.y_c_off + co0) % 8 == 0) && (co0 + row0 + 32 <= a.Cout);
-            for (int c0 = (sub + 4 * copy) * 32; c0 < a.N_px; c0 += 128 * a.R) {
-                unsigned r[32];
-                tmem_ld32(d_base + (unsigned)c0, r);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            T* yb = yg + (((size_t)n * a.Ho + y0) * a.Wo + x0) * a.y_c_stride + a.y_c_off + co0 + row0;
+            const unsigned ry = (unsigned)min(a.TH, a.Ho - y0), rx = (unsigned)min(a.TW, a.Wo - x0);  // rows / columns inside the image
+            const int c_first = (sub + 4 * copy) * 32, c_step = 128 * a.R;
+            const float bs = a.act == RTOSS_ACT_SILU ? 0.5f * bv : bv;
+            ok = mbar_wait(bar_accFull + 8 * as, (gt / a.AS) & 1);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const unsigned d_base = tmem_base + (unsigned)(as * a.acc_cols) + ((unsigned)(quarter * 32) << 16);
+            if (vec_ok) {
+                if (a.act == RTOSS_ACT_SILU)
+                    epilogue_chunks<T, RTOSS_ACT_SILU>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane);
+                else if (a.act == RTOSS_ACT_RELU)
+                    epilogue_chunks<T, RTOSS_ACT_RELU>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane);
+                else
+                    epilogue_chunks<T, RTOSS_ACT_NONE>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane);
+            } else {
+                // ragged filter counts or unaligned channel slices: element stores, lane = filter
+                for (int c0 = c_first; c0 < a.N_px; c0 += c_step) {
+                    unsigned r[32];
+                    tmem_ld32(d_base + (unsigned)c0, r);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    // the activation is picked outside the element loop: independent, branch-free chains
-                    if (h == 0) {
-                        if (a.act == RTOSS_ACT_SILU) act_to_patch<T, RTOSS_ACT_SILU, 0>(r, bv, patch + lane * 2);
-                        else if (a.act == RTOSS_ACT_RELU) act_to_patch<T, RTOSS_ACT_RELU, 0>(r, bv, patch + lane * 2);
-                        else act_to_patch<T, RTOSS_ACT_NONE, 0>(r, bv, patch + lane * 2);
-                    } else {
-                        if (a.act == RTOSS_ACT_SILU) act_to_patch<T, RTOSS_ACT_SILU, 16>(r, bv, patch + lane * 2);
-                        else if (a.act == RTOSS_ACT_RELU) act_to_patch<T, RTOSS_ACT_RELU, 16>(r, bv, patch + lane * 2);
-                        else act_to_patch<T, RTOSS_ACT_NONE, 16>(r, bv, patch + lane * 2);
-                    }
-                    __syncwarp();
-                    const int p0 = c0 + h * kPatchRows;
-                    if (vec_ok) {
-#pragma unroll
-                        for (int it = 0; it < 2; ++it) {
-                            const int i = it * 32 + lane, j = i >> 2, v = i & 3;  // position j of the patch, 8-filter group v
-                            const int pos = p0 + j;
-                            const int oyl = pos / a.Wq, oxl = pos - oyl * a.Wq, oy = y0 + oyl, ox = x0 + oxl;
-                            if (oyl < a.TH && oxl < a.TW && ox < a.Wo && oy < a.Ho) {
-                                const uint4 o = *reinterpret_cast<const uint4*>(patch + j * kPatchPitch + v * 16);
-                                *reinterpret_cast<uint4*>(yg + (((size_t)n * a.Ho + oy) * a.Wo + ox) * a.y_c_stride + a.y_c_off +
-                                                          co0 + row0 + v * 8) = o;
-                            }
+                    for (int j = 0; j < 32; ++j) {
+                        const uint2 e = pos_tab[c0 + j];
+                        float v = __uint_as_float(r[j]) + bv;
+                        if (a.act == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
+                        if (a.act == RTOSS_ACT_SILU) {
+                            float th;
+                            asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(0.5f * v));
+                            v = v * fmaf(0.5f, th, 0.5f);
                         }
-                    } else {
-                        // ragged filter counts or unaligned channel slices: element stores, lane = filter
-                        int oyl = p0 / a.Wq, oxl = p0 - oyl * a.Wq;
-                        for (int j = 0; j < kPatchRows; ++j) {
-                            const int oy = y0 + oyl, ox = x0 + oxl;
-                            if (co_ok && oyl < a.TH && oxl < a.TW && ox < a.Wo && oy < a.Ho)
-                                yg[(((size_t)n * a.Ho + oy) * a.Wo + ox) * a.y_c_stride + a.y_c_off + co] =
-                                    *reinterpret_cast<const T*>(patch + j * kPatchPitch + lane * 2);
-                            if (++oxl == a.Wq) {
-                                oxl = 0;
-                                ++oyl;
-                            }
-                        }
+                        if (co_ok && (e.y >> 16) < ry && (e.y & 0xFFFFu) < rx) yb[e.x + lane] = from_f32<T>(v);
                     }
-                    __syncwarp();
                 }
             }
             // this warp has read everything it needs from the accumulator stage
@@ -632,7 +722,7 @@ bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count
     const int halo = ksize == 3 ? (S == 1 ? 2 : 1) : 0;
     const int n_sub = (ksize == 3 && S == 2) ? 4 : 1;
     const int max_pitch = S == 1 ? 256 : 128;  // TMA box: at most 256 elements traversed per dimension
-    const int fixed = 1024 /*alignment slack*/ + 512 /*barriers*/ + kEpiWarps * kPatchRows * kPatchPitch /*epilogue patches*/;
+    const int fixed = 1024 /*alignment slack*/ + 512 /*barriers*/ + kEpiWarps * kPatchRows * kPatchPitch /*epilogue patches*/ + kMaxPx * 8 /*position table*/;
     const int cap = 227 * 1024 - 64;
     double best = -1;
     for (int nseg = 1; nseg <= 16; ++nseg) {
