@@ -53,7 +53,8 @@ namespace {
 using namespace rtoss_dev;
 
 constexpr int kEpiWarps = 16;
-constexpr int kTcThreads = (2 + kEpiWarps) * 32;  // TMA warp, MMA warp, sixteen epilogue warps
+constexpr int kTcThreads = (3 + kEpiWarps) * 32;  // activation TMA warp, MMA warp, sixteen epilogue warps, weight TMA warp
+constexpr int kWeightWarp = 2 + kEpiWarps;        // the last warp loads the weights
 constexpr int kPatchRows = 16;       // positions an epilogue warp turns at a time
 constexpr int kMaxA = 4, kMaxB = 8;  // most activation stages / weight slots
 constexpr int kMTile = 128;          // filters per tile = TMEM lanes
@@ -401,40 +402,63 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // tile's operands while the current one is still being multiplied, and the two accumulator stages
     // let the epilogue of one tile run under the MMAs of the next.
     if (warp == 0) {
-        // ---------------- TMA producer
+        // ---------------- TMA producer of the activations.  Issuing a bulk copy keeps its thread busy for some
+        // hundred cycles whatever the size, so the activations and the weights have a producer thread each, and a
+        // weight stage (G taps) is ONE copy.
         if (lane == 0) {
             bool ok = true;
-            int ga = 0, gb = 0;
+            int sa = 0;
+            unsigned pa = 0;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-                int rest = tile;
-                const int cot = rest % a.co_tiles;
-                rest /= a.co_tiles;
+                int rest = tile / a.co_tiles;
                 const int tx = rest % a.tiles_x;
                 rest /= a.tiles_x;
                 const int ty = rest % a.tiles_y, n = rest / a.tiles_y;
-                const int y0 = ty * a.TH, x0 = tx * a.TW, co0 = cot * kMTile;
-                for (int cb = 0; cb < a.ncb && ok; ++cb, ++ga) {
-                    const int sa = ga % a.NA;
-                    ok = mbar_wait(bar_emptyA + 8 * sa, ((ga / a.NA) & 1) ^ 1);
+                const int y0 = ty * a.TH, x0 = tx * a.TW;
+                for (int cb = 0; cb < a.ncb; ++cb) {
+                    ok = mbar_wait(bar_emptyA + 8 * sa, pa ^ 1);
                     if (!ok) break;
                     mbar_expect_tx(bar_fullA + 8 * sa, a.a_tx_bytes * a.n_sub);
                     for (int sub = 0; sub < a.n_sub; ++sub)
                         tma_load_4d(sA + sa * a.a_stage_bytes + sub * a.sub_bytes, &tmA, cb * kKBlock, x0 * a.S + a.x_add[sub],
                                     y0 * a.S + a.y_add[sub], n, bar_fullA + 8 * sa);
-                    for (int t0 = 0; t0 < a.taps; t0 += a.G, ++gb) {
-                        const int sb = gb % a.NB;
-                        ok = mbar_wait(bar_emptyB + 8 * sb, ((gb / a.NB) & 1) ^ 1);
-                        if (!ok) break;
-                        mbar_expect_tx(bar_fullB + 8 * sb, a.b_tx_bytes * a.G);
-                        for (int i = 0; i < a.G; ++i)
-                            tma_load_3d(sB + sb * a.b_stage_bytes + i * (a.w_rows * kRowBytes), &tmB, cb * kKBlock, co0, t0 + i,
-                                        bar_fullB + 8 * sb);
+                    if (++sa == a.NA) {
+                        sa = 0;
+                        pa ^= 1;
                     }
                 }
             }
             if (!ok) atomicExch(a.status, 1);
         }
         __syncwarp();  // lanes 1..31 wait here for lane 0: the warp reaches the final barrier as one
+    } else if (warp == kWeightWarp) {
+        // ---------------- TMA producer of the weights: per tile and channel block, taps / G stages of G taps each
+        if (lane == 0) {
+            bool ok = true;
+            int sb = 0;
+            unsigned pb = 0;
+            const int cstep = (int)gridDim.x % a.co_tiles;   // the filter tile moves by this from one of the CTA's tiles to the next
+            int cot = (int)blockIdx.x % a.co_tiles;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                const int co0 = cot * (a.pxm ? a.n_cols : kMTile);
+                for (int cb = 0; cb < a.ncb && ok; ++cb) {
+                    for (int t0 = 0; t0 < a.taps; t0 += a.G) {
+                        ok = mbar_wait(bar_emptyB + 8 * sb, pb ^ 1);
+                        if (!ok) break;
+                        mbar_expect_tx(bar_fullB + 8 * sb, a.b_tx_bytes * a.G);
+                        tma_load_3d(sB + sb * a.b_stage_bytes, &tmB, cb * kKBlock, co0, t0, bar_fullB + 8 * sb);
+                        if (++sb == a.NB) {
+                            sb = 0;
+                            pb ^= 1;
+                        }
+                    }
+                }
+                cot += cstep;
+                if (cot >= a.co_tiles) cot -= a.co_tiles;
+            }
+            if (!ok) atomicExch(a.status, 4);
+        }
+        __syncwarp();
     } else if (warp == 1) {
         // ---------------- MMA issuer
         if (lane == 0) {
@@ -911,10 +935,10 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     }
     // weights: one descriptor per handle
     rtoss_tmap_entry* eb = &p->wtc_map;
-    if (!eb->valid || eb->base != p->wtc || eb->dims[0] != w_rows) {
+    if (!eb->valid || eb->base != p->wtc || eb->dims[0] != w_rows || eb->dims[1] != plan.G) {
         cuuint64_t dims[3] = {(cuuint64_t)p->Cin, (cuuint64_t)lay.rows, (cuuint64_t)taps};
         cuuint64_t strides[2] = {(cuuint64_t)p->Cin * 2, (cuuint64_t)lay.rows * p->Cin * 2};
-        cuuint32_t box[3] = {(cuuint32_t)kKBlock, (cuuint32_t)w_rows, 1};
+        cuuint32_t box[3] = {(cuuint32_t)kKBlock, (cuuint32_t)w_rows, (cuuint32_t)plan.G};  // a weight stage is one copy
         cuuint32_t es[3] = {1, 1, 1};
         eb->valid = 0;
         CUresult r = enc(reinterpret_cast<CUtensorMap*>(eb->map), dt, 3, p->wtc, dims, strides, box, es,
@@ -923,6 +947,7 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
         if (r != CUDA_SUCCESS) return (int)cudaErrorInvalidValue;
         eb->base = p->wtc;
         eb->dims[0] = w_rows;
+        eb->dims[1] = plan.G;
         eb->valid = 1;
     }
     const CUtensorMap& tmA = *reinterpret_cast<const CUtensorMap*>(ea->map);
