@@ -59,10 +59,9 @@ constexpr int kPatchRows = 16;       // positions an epilogue warp turns at a ti
 constexpr int kMaxA = 4, kMaxB = 8;  // most activation stages / weight slots
 constexpr int kMTile = 128;          // filters per tile = TMEM lanes
 constexpr int kPxmMaxCout = 64;      // layers this narrow run with positions as the M operand
-constexpr int kPatchPitch = 80;      // bytes per position row of an epilogue transpose patch (64 + pad)
 constexpr int kMaxPx = 256;          // most positions in a tile's list
 constexpr int kPairPitch = 144;      // bytes per row (a pair of positions x 32 filters, + 16 pad) of the packed patch
-static_assert(kPatchRows / 2 * kPairPitch <= kPatchRows * kPatchPitch, "the packed patch must fit the warp's patch");
+constexpr int kPatchBytes = kPatchRows / 2 * kPairPitch;  // an epilogue warp's transpose patch
 constexpr int kKBlock = 64;       // channels per staged block: 128 bytes of bf16 / fp16
 constexpr int kRowBytes = 128;    // one padded pixel, one channel block
 constexpr long long kWaitCycles = 2000000000LL;  // about one second
@@ -89,6 +88,11 @@ struct TcArgs {
     int w_rows;           // filter rows per staged weight tile (128; fewer with positions as the M operand)
     int rep_rows, R;      // filters as M, narrow layer: the tile holds R copies of rep_rows filter rows (else 128, 1)
     int pxm, MH, n_cols;  // positions as the M operand: M halves of 128 positions per tile, filters per tile (the MMA's N)
+    // Split K: a tile's channel blocks are shared out to KS units (CTAs), cb_per blocks each; every unit leaves its
+    // partial sums in sk_scratch and the unit that arrives last at the tile's counter adds them up and finishes.
+    int KS, cb_per;
+    float* sk_scratch;  // [units][kMaxPx columns][128 lanes] fp32
+    int* sk_count;      // [tiles], zero between launches
 };
 
 __device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -334,6 +338,42 @@ __device__ __forceinline__ void epilogue_chunks(unsigned d_base, int c0, int c_s
     }
 }
 
+// Split K, the unit that arrived last: add up the KS partial sums of the tile (src points at this thread's lane
+// of the first one; partial sums are kMaxPx * 128 floats apart, columns 128 floats apart) and finish as usual.
+template <typename T, int ACT>
+__device__ __forceinline__ void epilogue_from_scratch(const float* src, int KS, int c0, int c_step, int n_px, float bs, bool vec_ok,
+                                                      bool co_ok, unsigned patch, unsigned tab, const uint2* pos_tab, T* yb,
+                                                      unsigned ry, unsigned rx, int lane) {
+    const unsigned wr = patch + lane * 4;
+    const unsigned rd = patch + (lane >> 2) * kPairPitch + (lane & 3) * 32;
+    const unsigned tab_l = tab + (unsigned)(2 * (lane >> 2)) * 8;
+    T* ybv = yb + (lane & 3) * 8;
+    for (; c0 < n_px; c0 += c_step) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            unsigned r[16];
+#pragma unroll
+            for (int j = 0; j < kPatchRows; ++j) {
+                const float* q = src + (size_t)(c0 + h * kPatchRows + j) * 128;
+                float acc = 0.f;
+                for (int i = 0; i < KS; ++i) acc += __ldcg(q + (size_t)i * (kMaxPx * 128));
+                r[j] = __float_as_uint(acc);
+            }
+            if (vec_ok) {
+                epilogue_half<T, ACT>(r, bs, wr, rd, tab_l + (unsigned)(c0 + h * kPatchRows) * 8, ybv, ry, rx);
+            } else {
+#pragma unroll
+                for (int j = 0; j < kPatchRows; ++j) {
+                    const uint2 e = pos_tab[c0 + h * kPatchRows + j];
+                    float v = bias_act<ACT>(r[j], bs);
+                    if (ACT == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
+                    if (co_ok && (e.y >> 16) < ry && (e.y & 0xFFFFu) < rx) yb[e.x + lane] = from_f32<T>(v);
+                }
+            }
+        }
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kTcThreads, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcArgs a) {
@@ -348,12 +388,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const unsigned bar_accFull = bar_emptyB + 8 * kMaxB, bar_accEmpty = bar_accFull + 16;
     const unsigned s_tmem_ptr = bar_accEmpty + 16;
     volatile unsigned* tmem_ptr_gen = reinterpret_cast<volatile unsigned*>(smem_dyn + (s_tmem_ptr - smem_u32(smem_dyn)));
-    unsigned char* epi_patch = smem_dyn + (s_tmem_ptr + 16 - smem_u32(smem_dyn));  // [kEpiWarps][kPatchRows][kPatchPitch], 16-byte aligned
-    uint2* pos_tab = reinterpret_cast<uint2*>(epi_patch + kEpiWarps * kPatchRows * kPatchPitch);  // [kMaxPx]
-    const unsigned s_tab = s_tmem_ptr + 16 + kEpiWarps * kPatchRows * kPatchPitch;                // the same, as a shared address
+    unsigned char* epi_patch = smem_dyn + (s_tmem_ptr + 16 - smem_u32(smem_dyn));  // [kEpiWarps][kPatchBytes], 16-byte aligned
+    uint2* pos_tab = reinterpret_cast<uint2*>(epi_patch + kEpiWarps * kPatchBytes);  // [kMaxPx]
+    const unsigned s_tab = s_tmem_ptr + 16 + kEpiWarps * kPatchBytes;                // the same, as a shared address
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_tiles = a.N * a.tiles_y * a.tiles_x * a.co_tiles;
+    const int n_tiles = a.N * a.tiles_y * a.tiles_x * a.co_tiles * a.KS;  // units of work: (tile, share of the channel blocks)
     // Programmatic dependent launch: the next kernel of the stream may start its own prologue now (on SMs this
     // grid leaves free); it reads or writes nothing before its own griddepcontrol.wait.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -409,13 +449,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             bool ok = true;
             int sa = 0;
             unsigned pa = 0;
-            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-                int rest = tile / a.co_tiles;
+            for (int unit = blockIdx.x; unit < n_tiles && ok; unit += gridDim.x) {
+                const int ks = unit % a.KS;
+                int rest = unit / a.KS / a.co_tiles;
                 const int tx = rest % a.tiles_x;
                 rest /= a.tiles_x;
                 const int ty = rest % a.tiles_y, n = rest / a.tiles_y;
                 const int y0 = ty * a.TH, x0 = tx * a.TW;
-                for (int cb = 0; cb < a.ncb; ++cb) {
+                const int cb_end = min(a.ncb, (ks + 1) * a.cb_per);
+                for (int cb = ks * a.cb_per; cb < cb_end; ++cb) {
                     ok = mbar_wait(bar_emptyA + 8 * sa, pa ^ 1);
                     if (!ok) break;
                     mbar_expect_tx(bar_fullA + 8 * sa, a.a_tx_bytes * a.n_sub);
@@ -437,11 +479,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             bool ok = true;
             int sb = 0;
             unsigned pb = 0;
-            const int cstep = (int)gridDim.x % a.co_tiles;   // the filter tile moves by this from one of the CTA's tiles to the next
-            int cot = (int)blockIdx.x % a.co_tiles;
-            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+            for (int unit = blockIdx.x; unit < n_tiles && ok; unit += gridDim.x) {
+                const int ks = unit % a.KS, cot = (unit / a.KS) % a.co_tiles;
                 const int co0 = cot * (a.pxm ? a.n_cols : kMTile);
-                for (int cb = 0; cb < a.ncb && ok; ++cb) {
+                const int cb_end = min(a.ncb, (ks + 1) * a.cb_per);
+                for (int cb = ks * a.cb_per; cb < cb_end && ok; ++cb) {
                     for (int t0 = 0; t0 < a.taps; t0 += a.G) {
                         ok = mbar_wait(bar_emptyB + 8 * sb, pb ^ 1);
                         if (!ok) break;
@@ -453,8 +495,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                     }
                 }
-                cot += cstep;
-                if (cot >= a.co_tiles) cot -= a.co_tiles;
             }
             if (!ok) atomicExch(a.status, 4);
         }
@@ -509,8 +549,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const unsigned d_base = tmem_base + (unsigned)(as * a.acc_cols);
                 unsigned acc = 0;  // the first instruction of a tile overwrites the accumulator
-                int left = a.Cin;
-                for (int cb = 0; cb < a.ncb && ok; ++cb, left -= kKBlock) {
+                const int ks = tile % a.KS, cb_end = min(a.ncb, (ks + 1) * a.cb_per);
+                int left = a.Cin - ks * a.cb_per * kKBlock;
+                for (int cb = ks * a.cb_per; cb < cb_end && ok; ++cb, left -= kKBlock) {
                     ok = mbar_wait(bar_fullA + 8 * sa, pa);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -636,7 +677,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
         } else
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++gt) {
-            int rest = tile;
+            int rest = tile / a.KS;   // tile counts units: (tile proper, share of the channel blocks)
+            const int t_idx = rest;
             const int cot = rest % a.co_tiles;
             rest /= a.co_tiles;
             const int tx = rest % a.tiles_x;
@@ -652,7 +694,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int co = co0 + row0 + lane;
             const bool co_ok = co < a.Cout;
             const float bv = (a.bias && co_ok) ? __ldg(a.bias + co) : 0.f;
-            const unsigned patch = s_tmem_ptr + 16 + (unsigned)(warp - 2) * (kPatchRows * kPatchPitch);  // shared address
+            const unsigned patch = s_tmem_ptr + 16 + (unsigned)(warp - 2) * kPatchBytes;  // shared address
             const bool vec_ok = (a.y_c_stride % 8 == 0) && ((a.y_c_off + co0) % 8 == 0) && (co0 + row0 + 32 <= a.Cout);
             T* yb = yg + (((size_t)n * a.Ho + y0) * a.Wo + x0) * a.y_c_stride + a.y_c_off + co0 + row0;
             const unsigned ry = (unsigned)min(a.TH, a.Ho - y0), rx = (unsigned)min(a.TW, a.Wo - x0);  // rows / columns inside the image
@@ -662,6 +704,38 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const unsigned d_base = tmem_base + (unsigned)(as * a.acc_cols) + ((unsigned)(quarter * 32) << 16);
+            if (a.KS > 1) {
+                // ---- split K: leave the partial sums, count in, and finish the tile if this unit is the last one
+                float* slot = a.sk_scratch + (size_t)tile * (kMaxPx * 128) + quarter * 32 + lane;
+                for (int c0 = c_first; c0 < a.N_px; c0 += c_step) {
+                    unsigned r[32];
+                    tmem_ld32(d_base + (unsigned)c0, r);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) slot[(size_t)(c0 + j) * 128] = __uint_as_float(r[j]);   // 128 contiguous bytes per warp
+                }
+                __threadfence();
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_accEmpty + 8 * as) : "memory");
+                volatile int* sk_flag = reinterpret_cast<volatile int*>(tmem_ptr_gen + 2);
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");   // every epilogue warp has written and fenced
+                if (threadIdx.x == 64) *sk_flag = atomicAdd(a.sk_count + t_idx, 1);
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
+                if (*sk_flag == a.KS - 1) {
+                    __threadfence();
+                    const float* src = a.sk_scratch + (size_t)(t_idx * a.KS) * (kMaxPx * 128) + quarter * 32 + lane;
+                    if (a.act == RTOSS_ACT_SILU)
+                        epilogue_from_scratch<T, RTOSS_ACT_SILU>(src, a.KS, c_first, c_step, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
+                    else if (a.act == RTOSS_ACT_RELU)
+                        epilogue_from_scratch<T, RTOSS_ACT_RELU>(src, a.KS, c_first, c_step, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
+                    else
+                        epilogue_from_scratch<T, RTOSS_ACT_NONE>(src, a.KS, c_first, c_step, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
+                    if (threadIdx.x == 64) a.sk_count[t_idx] = 0;   // ready for the next launch
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");   // the flag word is free again
+                continue;
+            }
             if (vec_ok) {
                 if (a.act == RTOSS_ACT_SILU)
                     epilogue_chunks<T, RTOSS_ACT_SILU>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane);
@@ -746,7 +820,7 @@ bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count
     const int halo = ksize == 3 ? (S == 1 ? 2 : 1) : 0;
     const int n_sub = (ksize == 3 && S == 2) ? 4 : 1;
     const int max_pitch = S == 1 ? 256 : 128;  // TMA box: at most 256 elements traversed per dimension
-    const int fixed = 1024 /*alignment slack*/ + 512 /*barriers*/ + kEpiWarps * kPatchRows * kPatchPitch /*epilogue patches*/ + kMaxPx * 8 /*position table*/;
+    const int fixed = 1024 /*alignment slack*/ + 512 /*barriers*/ + kEpiWarps * kPatchBytes /*epilogue patches*/ + kMaxPx * 8 /*position table*/;
     const int cap = 227 * 1024 - 64;
     double best = -1;
     for (int nseg = 1; nseg <= 16; ++nseg) {
@@ -903,6 +977,25 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
         a.acc_cols = round_up(a.MH * a.n_cols, 32);
         a.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((unsigned)(a.n_cols >> 3) << 17) | ((unsigned)(128 >> 4) << 24);
     }
+    // Split K where the layer has too few tiles for the SMs and several channel blocks: a tile's MMAs are one serial
+    // chain (an instruction costs the same however few positions it covers), so the blocks go to several CTAs.
+    a.KS = 1;
+    a.cb_per = a.ncb;
+    a.sk_scratch = ctx->sk_scratch;
+    a.sk_count = ctx->sk_count;
+    {
+        const long tiles = (long)d->N * a.tiles_y * a.tiles_x * a.co_tiles;
+        const int min_cb = p->ksize == 3 ? 1 : 4;   // at least this many blocks per share (36 resp. 16 instructions)
+        if (!pxm && ctx->sk_scratch && tiles * 2 <= sms && a.ncb >= 2 * min_cb) {
+            int want = (int)(sms / tiles);
+            if (want > a.ncb / min_cb) want = a.ncb / min_cb;
+            if (want > 8) want = 8;
+            if (want > 1) {
+                a.cb_per = (a.ncb + want - 1) / want;
+                a.KS = (a.ncb + a.cb_per - 1) / a.cb_per;
+            }
+        }
+    }
     const int cols = a.AS * a.acc_cols;
     int alloc = 32;
     while (alloc < cols) alloc <<= 1;
@@ -954,7 +1047,7 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     const CUtensorMap& tmB = *reinterpret_cast<const CUtensorMap*>(eb->map);
     // at least half an SM's shared memory, so that a second CTA (which would wait for TMEM) never shares the SM
     const size_t smem = (size_t)(plan.smem > 116 * 1024 ? plan.smem : 116 * 1024);
-    const size_t n_tiles = (size_t)d->N * a.tiles_y * a.tiles_x * a.co_tiles;
+    const size_t n_tiles = (size_t)d->N * a.tiles_y * a.tiles_x * a.co_tiles * a.KS;
     dim3 grid((unsigned)(n_tiles < (size_t)sms ? n_tiles : (size_t)sms));
     static bool attr_set = false;  // both instantiations may use up to the whole shared memory of an SM
     if (!attr_set) {

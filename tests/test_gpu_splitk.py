@@ -1,0 +1,47 @@
+"""Tensor path on layers with few tiles and many channel blocks: the channel blocks of a tile are shared out to
+several CTAs (split K) and the CTA that arrives last adds up the partial sums.  Parity against the CPU oracle,
+twice in a row on the same context (the arrival counters must be back at zero), with every activation, a channel
+slice of a wider output, a ragged filter count and both kernel sizes."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    from oracle import rtoss_oracle as orc
+    from paper_2303_02191_b200 import binding as rt
+    from paper_2303_02191_b200 import synth
+    import gpu_util as G
+
+CASES = [
+    # ksize, Cin, Cout, N, H, W, stride, act, (y_off, y_stride)
+    (3, 256, 256, 2, 13, 17, 1, "relu", (0, 0)),
+    (3, 256, 256, 1, 7, 9, 1, "none", (0, 0)),
+    (3, 512, 128, 1, 20, 20, 1, "silu", (0, 0)),
+    (3, 192, 100, 1, 9, 11, 1, "silu", (0, 0)),       # ragged filter count: element stores
+    (3, 256, 128, 1, 12, 12, 2, "silu", (64, 256)),   # stride 2, channel slice of a wider tensor
+    (1, 2048, 512, 1, 7, 9, 1, "relu", (0, 0)),
+    (1, 1024, 128, 2, 10, 10, 1, "silu", (0, 0)),
+]
+
+
+@pytest.mark.parametrize("ksize,cin,cout,N,H,W,stride,act,ysl", CASES)
+def test_split_k_parity(ksize, cin, cout, N, H, W, stride, act, ysl):
+    masks = orc.pattern_preset(4, orc.PRESET_CENTRE8)
+    w = synth.kaiming_weights(3, 11, cout, cin, ksize)
+    b = synth.bias(3, 11, cout)
+    x = synth.round_like(synth.activations(3, 11, N, cin, H, W), "bf16")
+    pid, packed = G.select_pack(w, ksize, masks, 4, "bf16")
+    pid_o, wd, _ = G.oracle_weights(w, ksize, masks, 4, "bf16")
+    assert np.array_equal(pid, pid_o.ravel())
+    conv = orc.conv3x3 if ksize == 3 else orc.conv1x1
+    ref = conv(x, wd, b, stride, {"none": orc.ACT_NONE, "relu": orc.ACT_RELU, "silu": orc.ACT_SILU}[act], orc.DT_BF16)
+    for _ in range(2):
+        y = G.run_conv(packed, ksize, x, "bf16", stride, act, b, layout="nhwc", y_off=ysl[0], y_stride=ysl[1], path=rt.PATH_TENSOR)
+        if ysl[1]:
+            y = y[:, ysl[0]:ysl[0] + cout]
+        err = orc.rel_err(y, ref)
+        assert err <= G.TOL["bf16"], "relative error %g" % err
+    assert G.ctx().rtoss_device_status() == 0
+    packed.close()
