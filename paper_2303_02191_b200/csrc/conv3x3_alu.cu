@@ -31,6 +31,8 @@
 //     4, 8 or 16 bytes (the widest that divides W*elem is used); NHWC: Cin a
 //     multiple of 8.  Weights: Cin a multiple of 8.  Anything else takes a plain
 //     load-convert-store path inside the same kernel.
+#include <cstring>
+
 #include "conv_common.cuh"
 
 namespace {
@@ -416,18 +418,46 @@ struct Variant {
 };
 
 // ---------------------------------------------------------------------------------------------
-// Layers with very few input channels (the 3-channel stem of a detector): one thread per output
-// pixel, its 3x3xCIN input neighbourhood in registers, 32 filters per thread in sequence with the
-// dense-expanded weights (pruned taps are zeros) broadcast from shared memory.  The layer is bound
-// by its output traffic; with 9*CIN <= 36 multiply-adds per output the zeros cost less than
-// skipping them would.
+// Layers with very few input channels (the 3-channel stem of a detector).  A thread computes kStemPx
+// neighbouring output pixels of one row for 32 filters: its input window (3 rows x ((kStemPx-1)*S+3)
+// columns x CIN) sits in registers, the dense-expanded weights (pruned taps are zeros: with 9*CIN <= 36
+// multiply-adds per output the zeros cost less than skipping them) are read from shared memory once per
+// filter as 16-byte loads and used for all kStemPx pixels.  The layer's bound is its traffic, so loads and
+// stores must be whole segments:
+//   * the detector stem proper (three 16-bit channels, NHWC, stride 2, rows of a multiple of 8 pixels): a
+//     thread's window of 9 pixels x 3 channels is 54 contiguous bytes that start 6 bytes before a 16-byte
+//     boundary, so it comes in as four aligned 16-byte loads per row and every value sits at a position
+//     known at compile time (81 separate 2-byte loads a thread, each lane in its own sector, were what
+//     bounded the kernel before);
+//   * with 16-bit NHWC outputs a block's 512 pixels x 32 filters are gathered in shared memory and written
+//     out with consecutive lanes on consecutive 16 bytes.
+// A block walks the pixel groups in steps of the grid, so the weight table is built once per block.
 constexpr int kStemCo = 32;
+constexpr int kStemPx = 4;
+constexpr int kStemThreads = 128;
 
-template <typename T, int CIN>
-__global__ void __launch_bounds__(256) conv3x3_small_cin_kernel(const Conv3Args a, int stride) {
+// SiLU of a 16-bit output through tanh.approx (relative error about 2^-11, below half an ulp of bf16);
+// fp32 outputs keep the exponential form (the tolerance there is 1e-4).
+template <typename T>
+__device__ __forceinline__ float stem_act(float v, int act) {
+    if (sizeof(T) == 2 && act == RTOSS_ACT_SILU) {
+        const float h = 0.5f * v;
+        float th;
+        asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(h));
+        return fmaf(h, th, h);
+    }
+    return activate(v, act);
+}
+
+template <typename T, int CIN, int S>
+__global__ void __launch_bounds__(kStemThreads) conv3x3_small_cin_kernel(const Conv3Args a) {
     rtoss_dev::pdl_enter();
-    __shared__ float sWd[kStemCo][CIN * 9 + 1];  // [filter][ci*9 + tap], last = bias
+    constexpr int KW = (CIN * 9 + 1 + 3) / 4 * 4;          // a filter's row: CIN*9 weights, the bias, padding to 16 bytes
+    constexpr int WIN = (kStemPx - 1) * S + 3;              // input columns a thread needs
+    constexpr int kStageRow = kStemPx * 4 + 1;              // 16-byte pieces a thread stages (+1: lanes on different banks)
+    __shared__ __align__(16) float sWd[kStemCo][KW];         // [filter][ci*9 + tap], then the bias
     __shared__ uint16_t smask[256];
+    __shared__ uint4 sOut[sizeof(T) == 2 ? kStemThreads * kStageRow : 1];
     const int co0 = blockIdx.y * kStemCo;
     for (int p = threadIdx.x; p < 256; p += blockDim.x) smask[p] = p < a.P ? a.masks[p] : 0;
     __syncthreads();
@@ -446,74 +476,163 @@ __global__ void __launch_bounds__(256) conv3x3_small_cin_kernel(const Conv3Args 
         }
 #pragma unroll
         for (int t = 0; t < 9; ++t) sWd[col][ci * 9 + t] = wv[t];
-        if (ci == 0) sWd[col][CIN * 9] = (a.bias && co < a.Cout) ? a.bias[co] : 0.f;
+        if (ci == 0) {
+            sWd[col][CIN * 9] = (a.bias && co < a.Cout) ? a.bias[co] : 0.f;
+            for (int t = CIN * 9 + 1; t < KW; ++t) sWd[col][t] = 0.f;
+        }
     }
     __syncthreads();
 
-    const long long total = (long long)a.N * a.Ho * a.Wo;
-    const long long pix = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (pix >= total) return;
-    const int ox = (int)(pix % a.Wo);
-    const long long r1 = pix / a.Wo;
-    const int oy = (int)(r1 % a.Ho), n = (int)(r1 / a.Ho);
     const T* __restrict__ xg = reinterpret_cast<const T*>(a.x);
-    float xin[CIN][9];
-#pragma unroll
-    for (int r = 0; r < 3; ++r)
-#pragma unroll
-        for (int c = 0; c < 3; ++c) {
-            const int iy = oy * stride + r - 1, ix = ox * stride + c - 1;
-            const bool ok = iy >= 0 && iy < a.H && ix >= 0 && ix < a.W;
-#pragma unroll
-            for (int ci = 0; ci < CIN; ++ci) {
-                const size_t idx = a.layout == RTOSS_NCHW ? (((size_t)n * CIN + ci) * a.H + iy) * a.W + ix
-                                                          : (((size_t)n * a.H + iy) * a.W + ix) * CIN + ci;
-                xin[ci][r * 3 + c] = ok ? to_f32<T>(xg[idx]) : 0.f;
-            }
-        }
     T* __restrict__ yg = reinterpret_cast<T*>(a.y);
     const int Cs = a.y_c_stride;
+    constexpr int PER16 = 16 / (int)sizeof(T);
     const bool vec = a.layout == RTOSS_NHWC && (Cs * sizeof(T)) % 16 == 0 && ((a.y_c_off + co0) * sizeof(T)) % 16 == 0 &&
                      co0 + kStemCo <= a.Cout;
-    constexpr int PER16 = 16 / (int)sizeof(T);
-    for (int c8 = 0; c8 < kStemCo; c8 += PER16) {
-        __align__(16) T o[PER16];
+    // 16-bit NHWC outputs whose rows hold whole groups: pixel index = kStemPx * group index + px, the pixels of a
+    // round of the block are consecutive, and the stores go through the staging buffer
+    const bool staged = sizeof(T) == 2 && vec && a.Wo % kStemPx == 0;
+    const bool fast_in = sizeof(T) == 2 && CIN == 3 && S == 2 && kStemPx == 4 && a.layout == RTOSS_NHWC && a.W % 8 == 0;
+    const int groups = (a.Wo + kStemPx - 1) / kStemPx;      // groups of kStemPx output columns per row
+    const long long total = (long long)a.N * a.Ho * groups;
+    const long long px_total = (long long)a.N * a.Ho * a.Wo;
+
+    for (long long blk = blockIdx.x; blk * kStemThreads < total; blk += gridDim.x) {
+        const long long gi_raw = blk * kStemThreads + threadIdx.x;
+        const bool active = gi_raw < total;
+        const long long gi = active ? gi_raw : total - 1;   // idle threads recompute the last group and store nothing
+        const int ox0 = (int)(gi % groups) * kStemPx;
+        const long long r1 = gi / groups;
+        const int oy = (int)(r1 % a.Ho), n = (int)(r1 / a.Ho);
+        float xin[CIN][3][WIN];
+        if (fast_in) {
 #pragma unroll
-        for (int q = 0; q < PER16; ++q) {
-            const float* wr = sWd[c8 + q];
-            float acc = wr[CIN * 9];
+            for (int r = 0; r < 3; ++r) {
+                const int iy = oy * S + r - 1;
+                const bool row_ok = iy >= 0 && iy < a.H;
+                // 16-byte piece 3 * (ox0 / 4) of the row holds input pixel 2 * ox0; the window starts one pixel earlier
+                const uint4* rowp = reinterpret_cast<const uint4*>(xg + ((size_t)n * a.H + (row_ok ? iy : 0)) * a.W * CIN) + (ox0 / kStemPx) * 3;
+                const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+                uint4 ch[4];
+                ch[0] = (row_ok && ox0 > 0) ? __ldg(rowp - 1) : zero;
 #pragma unroll
-            for (int i = 0; i < CIN * 9; ++i) acc = fmaf(wr[i], xin[i / 9][i % 9], acc);
-            o[q] = from_f32<T>(activate(acc, a.act));
-        }
-        if (vec) {
-            *reinterpret_cast<uint4*>(yg + (((size_t)n * a.Ho + oy) * a.Wo + ox) * Cs + a.y_c_off + co0 + c8) =
-                *reinterpret_cast<const uint4*>(o);
+                for (int i = 1; i < 4; ++i) ch[i] = row_ok ? __ldg(rowp + i - 1) : zero;
+                const unsigned wds[16] = {ch[0].x, ch[0].y, ch[0].z, ch[0].w, ch[1].x, ch[1].y, ch[1].z, ch[1].w,
+                                          ch[2].x, ch[2].y, ch[2].z, ch[2].w, ch[3].x, ch[3].y, ch[3].z, ch[3].w};
+#pragma unroll
+                for (int c = 0; c < WIN; ++c)
+#pragma unroll
+                    for (int ci = 0; ci < CIN; ++ci) {
+                        const int hi = (5 + c * CIN + ci) & 31;   // 16-bit index inside the 64 bytes: the window starts at byte 10
+                        const unsigned short bits = (hi & 1) ? (unsigned short)(wds[hi >> 1] >> 16) : (unsigned short)(wds[hi >> 1] & 0xFFFFu);
+                        T v;
+                        memcpy(&v, &bits, sizeof(bits));
+                        xin[ci][r][c] = to_f32<T>(v);
+                    }
+            }
         } else {
 #pragma unroll
-            for (int q = 0; q < PER16; ++q) {
-                const int co = co0 + c8 + q;
-                if (co < a.Cout) {
-                    const size_t idx = a.layout == RTOSS_NCHW ? (((size_t)n * Cs + a.y_c_off + co) * a.Ho + oy) * a.Wo + ox
-                                                              : (((size_t)n * a.Ho + oy) * a.Wo + ox) * Cs + a.y_c_off + co;
-                    yg[idx] = o[q];
+            for (int r = 0; r < 3; ++r) {
+                const int iy = oy * S + r - 1;
+                const bool row_ok = iy >= 0 && iy < a.H;
+#pragma unroll
+                for (int c = 0; c < WIN; ++c) {
+                    const int ix = ox0 * S + c - 1;
+                    const bool ok = row_ok && ix >= 0 && ix < a.W;
+#pragma unroll
+                    for (int ci = 0; ci < CIN; ++ci) {
+                        const size_t idx = a.layout == RTOSS_NCHW ? (((size_t)n * CIN + ci) * a.H + iy) * a.W + ix
+                                                                  : (((size_t)n * a.H + iy) * a.W + ix) * CIN + ci;
+                        xin[ci][r][c] = ok ? to_f32<T>(xg[idx]) : 0.f;
+                    }
                 }
             }
+        }
+        for (int c8 = 0; c8 < kStemCo; c8 += PER16) {
+            __align__(16) T o[kStemPx][PER16];
+#pragma unroll
+            for (int q = 0; q < PER16; ++q) {
+                float w[KW];
+                const float4* wr = reinterpret_cast<const float4*>(sWd[c8 + q]);
+#pragma unroll
+                for (int i = 0; i < KW / 4; ++i) {
+                    const float4 v = wr[i];
+                    w[4 * i] = v.x;
+                    w[4 * i + 1] = v.y;
+                    w[4 * i + 2] = v.z;
+                    w[4 * i + 3] = v.w;
+                }
+#pragma unroll
+                for (int px = 0; px < kStemPx; ++px) {
+                    float acc = w[CIN * 9];
+#pragma unroll
+                    for (int ci = 0; ci < CIN; ++ci)
+#pragma unroll
+                        for (int r = 0; r < 3; ++r)
+#pragma unroll
+                            for (int c = 0; c < 3; ++c) acc = fmaf(w[ci * 9 + r * 3 + c], xin[ci][r][px * S + c], acc);
+                    o[px][q] = from_f32<T>(stem_act<T>(acc, a.act));
+                }
+            }
+#pragma unroll
+            for (int px = 0; px < kStemPx; ++px) {
+                const int ox = ox0 + px;
+                if (staged) {
+                    sOut[threadIdx.x * kStageRow + px * 4 + c8 / PER16] = *reinterpret_cast<const uint4*>(o[px]);
+                    continue;
+                }
+                if (ox >= a.Wo || !active) continue;
+                if (vec) {
+                    *reinterpret_cast<uint4*>(yg + (((size_t)n * a.Ho + oy) * a.Wo + ox) * Cs + a.y_c_off + co0 + c8) =
+                        *reinterpret_cast<const uint4*>(o[px]);
+                } else {
+#pragma unroll
+                    for (int q = 0; q < PER16; ++q) {
+                        const int co = co0 + c8 + q;
+                        if (co < a.Cout) {
+                            const size_t idx = a.layout == RTOSS_NCHW ? (((size_t)n * Cs + a.y_c_off + co) * a.Ho + oy) * a.Wo + ox
+                                                                      : (((size_t)n * a.Ho + oy) * a.Wo + ox) * Cs + a.y_c_off + co;
+                            yg[idx] = o[px][q];
+                        }
+                    }
+                }
+            }
+        }
+        if (staged) {
+            __syncthreads();
+            const long long px_first = blk * kStemThreads * kStemPx;   // first pixel of this round of the block
+#pragma unroll 4
+            for (int it = 0; it < kStemPx * 4; ++it) {
+                const int q = it * kStemThreads + threadIdx.x;        // 16-byte piece of the round's outputs, in memory order
+                const int pl = q >> 2, part = q & 3;                   // pixel inside the round, 8-filter group
+                const long long pg = px_first + pl;
+                if (pg < px_total)
+                    *reinterpret_cast<uint4*>(yg + (size_t)pg * Cs + a.y_c_off + co0 + part * PER16) =
+                        sOut[(pl / kStemPx) * kStageRow + (pl % kStemPx) * 4 + part];
+            }
+            __syncthreads();   // the staging buffer is free for the next round
         }
     }
 }
 
-template <typename T>
-int launch_small_cin(const Conv3Args& a, int stride, cudaStream_t stream) {
-    const long long total = (long long)a.N * a.Ho * a.Wo;
-    dim3 grid((unsigned)((total + 255) / 256), (unsigned)((a.Cout + kStemCo - 1) / kStemCo));
+template <typename T, int S>
+int launch_small_cin_s(const Conv3Args& a, cudaStream_t stream) {
+    const long long total = (long long)a.N * a.Ho * ((a.Wo + kStemPx - 1) / kStemPx);
+    long long blocks = (total + kStemThreads - 1) / kStemThreads;
+    if (blocks > 148 * 6) blocks = 148 * 6;   // a few rounds per block
+    dim3 grid((unsigned)blocks, (unsigned)((a.Cout + kStemCo - 1) / kStemCo));
     switch (a.Cin) {
-        case 1: rtoss_dev::launch_pdl(conv3x3_small_cin_kernel<T, 1>, grid, 256, 0, stream, a, stride); break;
-        case 2: rtoss_dev::launch_pdl(conv3x3_small_cin_kernel<T, 2>, grid, 256, 0, stream, a, stride); break;
-        case 3: rtoss_dev::launch_pdl(conv3x3_small_cin_kernel<T, 3>, grid, 256, 0, stream, a, stride); break;
-        default: rtoss_dev::launch_pdl(conv3x3_small_cin_kernel<T, 4>, grid, 256, 0, stream, a, stride); break;
+        case 1: rtoss_dev::launch_pdl(conv3x3_small_cin_kernel<T, 1, S>, grid, kStemThreads, 0, stream, a); break;
+        case 2: rtoss_dev::launch_pdl(conv3x3_small_cin_kernel<T, 2, S>, grid, kStemThreads, 0, stream, a); break;
+        case 3: rtoss_dev::launch_pdl(conv3x3_small_cin_kernel<T, 3, S>, grid, kStemThreads, 0, stream, a); break;
+        default: rtoss_dev::launch_pdl(conv3x3_small_cin_kernel<T, 4, S>, grid, kStemThreads, 0, stream, a); break;
     }
     return (int)cudaGetLastError();
+}
+
+template <typename T>
+int launch_small_cin(const Conv3Args& a, int stride, cudaStream_t stream) {
+    return stride == 1 ? launch_small_cin_s<T, 1>(a, stream) : launch_small_cin_s<T, 2>(a, stream);
 }
 
 // Pick the lane arrangement that wastes the fewest lanes and pixels.

@@ -351,14 +351,18 @@ __device__ __forceinline__ void epilogue_from_scratch(const float* src, int KS, 
     for (; c0 < n_px; c0 += c_step) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
+            // sixteen independent loads in flight per partial sum (the shares' loop is the outer one)
+            float sum[kPatchRows];
+#pragma unroll
+            for (int j = 0; j < kPatchRows; ++j) sum[j] = 0.f;
+            const float* q = src + (size_t)(c0 + h * kPatchRows) * 128;
+            for (int i = 0; i < KS; ++i, q += kMaxPx * 128) {
+#pragma unroll
+                for (int j = 0; j < kPatchRows; ++j) sum[j] += __ldcg(q + j * 128);
+            }
             unsigned r[16];
 #pragma unroll
-            for (int j = 0; j < kPatchRows; ++j) {
-                const float* q = src + (size_t)(c0 + h * kPatchRows + j) * 128;
-                float acc = 0.f;
-                for (int i = 0; i < KS; ++i) acc += __ldcg(q + (size_t)i * (kMaxPx * 128));
-                r[j] = __float_as_uint(acc);
-            }
+            for (int j = 0; j < kPatchRows; ++j) r[j] = __float_as_uint(sum[j]);
             if (vec_ok) {
                 epilogue_half<T, ACT>(r, bs, wr, rd, tab_l + (unsigned)(c0 + h * kPatchRows) * 8, ybv, ry, rx);
             } else {
@@ -985,7 +989,11 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     a.sk_count = ctx->sk_count;
     {
         const long tiles = (long)d->N * a.tiles_y * a.tiles_x * a.co_tiles;
-        const int min_cb = p->ksize == 3 ? 1 : 4;   // at least this many blocks per share (36 resp. 16 instructions)
+        // The round trip of the partial sums (a store, a fence, a counter, and the last CTA reading every share back
+        // through one SM) costs about as much as 70 instructions of the chain: measured on 256-channel layers at
+        // 25x34 and 13x17, halving a chain of 144 gained nothing, while stride-2 layers (four staged input phases
+        // per channel block) and chains of 288 and more came out ahead.  Hence the shares stay long.
+        const int min_cb = p->ksize == 3 ? (S == 2 ? 2 : 4) : 32;
         if (!pxm && ctx->sk_scratch && tiles * 2 <= sms && a.ncb >= 2 * min_cb) {
             int want = (int)(sms / tiles);
             if (want > a.ncb / min_cb) want = a.ncb / min_cb;

@@ -96,6 +96,12 @@ SHAPES_3x3 = [
     (2, 3, 40, 20, 22, 1, 3, "f16", "silu", "nhwc", True),      # 3-channel stem kernel, NHWC, ragged filter block
     (1, 4, 64, 16, 16, 2, 2, "bf16", "relu", "nhwc", False),    # 4-channel stem kernel, vector stores
     (1, 2, 32, 9, 9, 1, 4, "f32", "none", "nchw", True),
+    (2, 3, 32, 32, 48, 2, 4, "bf16", "silu", "nhwc", True),     # detector stem: 16-byte window loads, staged stores, 2 blocks
+    (1, 3, 32, 24, 40, 2, 4, "f16", "relu", "nhwc", True),      # the same in fp16
+    (1, 3, 64, 16, 16, 2, 4, "bf16", "silu", "nhwc", True),     # two filter blocks: staged stores into 128-byte pixels
+    (1, 3, 32, 18, 20, 2, 4, "bf16", "silu", "nhwc", True),     # rows of 20 pixels: element loads, 10 outputs a row: direct stores
+    (1, 3, 32, 12, 16, 1, 4, "bf16", "none", "nhwc", True),     # stride 1: element loads, staged stores
+    (8, 3, 32, 480, 480, 2, 4, "bf16", "silu", "nhwc", True),   # more groups than one round of the grid
 ]
 
 
