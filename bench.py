@@ -397,19 +397,44 @@ def run_gpu(args):
     step_ms = np.array([a.elapsed_time(b) for a, b in step_ev])
     total_ms = float(step_ms.sum())
 
-    # Per-kernel durations for the roofline: the same K steps again, launched one by one, every convolution
-    # between its own pair of events.  The 256 MB flush write queued right before each launch both empties
-    # L2 and keeps the GPU busy while the host enqueues the launch, so the interval is the kernel alone.
-    conv_ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in L_state]
-               for _ in range(args.steps)]
-    for s in range(args.steps):
-        prune_weights()
-        for i, st in enumerate(L_state):
-            flush.zero_()
-            conv(st, conv_ev[s][i])
+    # Per-kernel durations for the roofline: the same K steps again, every convolution between its own pair of
+    # events right after a 256 MB flush write (cold L2).  The pass is captured once into a CUDA graph whose event
+    # records are graph nodes (external events) and replayed K times, so the host's enqueue time cannot leak into
+    # an interval; if the capture is not available the launches are issued one by one (the flush write queued
+    # before each launch then keeps the GPU busy while the host enqueues it).
+    conv_ms = None
+    if args.graph:
+        try:
+            gev = [(torch.cuda.Event(enable_timing=True, external=True), torch.cuda.Event(enable_timing=True, external=True))
+                   for _ in L_state]
+            kgraph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(kgraph):
+                prune_weights()
+                for i, st in enumerate(L_state):
+                    flush.zero_()
+                    conv(st, gev[i])
+            acc = np.zeros(len(L_state))
+            for s in range(args.steps):
+                kgraph.replay()
+                torch.cuda.synchronize()
+                acc += np.array([a.elapsed_time(b) for a, b in gev])
+            conv_ms = acc / args.steps
+        except Exception as err:
+            sys.stderr.write("per-kernel timing graph not available, timing eager launches: %r\n" % (err,))
+            torch.cuda.synchronize()
+            conv_ms = None
+    if conv_ms is None:
+        conv_ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in L_state]
+                   for _ in range(args.steps)]
+        for s in range(args.steps):
+            prune_weights()
+            for i, st in enumerate(L_state):
+                flush.zero_()
+                conv(st, conv_ev[s][i])
+        barrier()
+        conv_ms = np.array([[a.elapsed_time(b) for a, b in row] for row in conv_ev]).mean(axis=0)
     barrier()
     clocks = sampler.stop()
-    conv_ms = np.array([[a.elapsed_time(b) for a, b in row] for row in conv_ev]).mean(axis=0)
 
     # ---- end to end through the host-buffer entry point (pinned host tensors, copies inside the timed region)
     torch.cuda.synchronize()
