@@ -210,15 +210,22 @@ def whole_job_value(images_per_rank, world, ms_per_step):
 # --------------------------------------------------------------------------- GPU arm
 
 def run_network(args):
-    """Whole-network replay of the YOLOv5s-shaped backbone + neck (convolutions + glue) as one CUDA graph."""
+    """Whole-network replay (convolutions + glue) as one CUDA graph: the YOLOv5s-shaped backbone + neck, or the
+    RetinaNet ResNet-50-FPN-shaped network behind its 7x7 stem."""
     import torch
     from paper_2303_02191_b200 import binding as rt
-    from paper_2303_02191_b200.yolov5s_net import GpuNet
-    N = 1 if args.workload.endswith("b1") else 16
     torch.cuda.set_device(0)
     ctx = rt.Context(0)
-    net = GpuNet(ctx, N)
-    xh = synth.round_like(synth.activations(0, 1, N, 3, 640, 640), "bf16")
+    if args.workload.startswith("retinanet"):
+        from paper_2303_02191_b200.retinanet_net import GpuNet
+        N = 4
+        net = GpuNet(ctx, N)
+        xh = synth.round_like(synth.activations(0, 1, N, 64, 200, 272), "bf16")
+    else:
+        from paper_2303_02191_b200.yolov5s_net import GpuNet
+        N = 1 if args.workload.endswith("b1") else 16
+        net = GpuNet(ctx, N)
+        xh = synth.round_like(synth.activations(0, 1, N, 3, 640, 640), "bf16")
     net.set_input(xh)
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
     side = torch.cuda.Stream()
@@ -543,7 +550,7 @@ def main():
     if args.impl == "reference":
         run_reference(args)
         return
-    if args.workload in ("yolov5s_net_b1", "yolov5s_net_b16"):
+    if args.workload in ("yolov5s_net_b1", "yolov5s_net_b16", "retinanet_net_b4"):
         run_network(args)
         return
     if int(os.environ.get("WORLD_SIZE", "1")) > 1 or args.gpus == 1:

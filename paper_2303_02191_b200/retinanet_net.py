@@ -1,0 +1,138 @@
+"""RetinaNet ResNet-50-FPN-shaped network as ONE chained program over the library's calls.
+
+The 100 pattern-pruned convolution calls of `synth.retinanet_r50fpn_stack()` (68 weight tensors: the two towers
+share theirs across the five pyramid levels) plus the glue a whole network needs: the residual add + ReLU that
+closes every bottleneck, the top-down pathway of the pyramid (2x up-sampling + add), the ReLU in front of P7.
+The program starts at the 64-channel tensor behind the 7x7 stem and its max-pool (those are outside the 3x3 / 1x1
+pattern set).  The same description drives `GpuNet` here (the C-ABI library, NHWC bf16, suitable for CUDA-graph
+capture) and the tests' CPU-oracle executor.  Only shapes come from the model family; weights are seeded and
+synthetic.
+"""
+from . import synth
+
+
+def program(H0, W0):
+    """-> (ops, bufs, layers).  bufs: name -> (C, H, W).  ops in execution order:
+    ('conv', layer_index, src, dst, act) | ('add', a, b, dst, act) | ('up', src, dst) | ('relu', src, dst)."""
+    layers = synth.retinanet_r50fpn_stack(H0, W0)
+    ops, bufs = [], {}
+    li = [0]
+
+    def buf(name, C, H, W):
+        bufs[name] = (C, H, W)
+        return name
+
+    def conv(src, dst, act):
+        L = layers[li[0]]
+        assert bufs[src] == (L["cin"], L["H"], L["W"]), (L["name"], bufs[src])
+        Ho, Wo = synth.out_hw(L["H"], L["W"], L["stride"])
+        assert bufs[dst] == (L["cout"], Ho, Wo), (L["name"], bufs[dst])
+        ops.append(("conv", li[0], src, dst, act))
+        li[0] += 1
+
+    H, W = H0 // 4, W0 // 4
+    cur = buf("in", 64, H, W)
+    cin = 64
+    feats = {}
+    for si, (nblk, w) in enumerate(zip([3, 4, 6, 3], [64, 128, 256, 512])):
+        for b in range(nblk):
+            s = 2 if (b == 0 and si > 0) else 1
+            tag = "layer%d.%d" % (si + 1, b)
+            Ho, Wo = synth.out_hw(H, W, s)
+            conv(cur, buf(tag + ".t1", w, H, W), "relu")
+            conv(tag + ".t1", buf(tag + ".t2", w, Ho, Wo), "relu")
+            conv(tag + ".t2", buf(tag + ".t3", 4 * w, Ho, Wo), "none")     # the ReLU comes after the residual add
+            idn = cur
+            if b == 0:
+                conv(cur, buf(tag + ".idn", 4 * w, Ho, Wo), "none")
+                idn = tag + ".idn"
+            ops.append(("add", tag + ".t3", idn, buf(tag + ".out", 4 * w, Ho, Wo), "relu"))
+            cur, cin, H, W = tag + ".out", 4 * w, Ho, Wo
+        feats[si] = (cur, cin, H, W)
+    # pyramid: laterals, top-down sums, 3x3 outputs, P6 from P5, P7 from ReLU(P6)
+    for si in (1, 2, 3):
+        src, c, h, w_ = feats[si]
+        conv(src, buf("lat%d" % (si + 2), 256, h, w_), "none")
+    for si in (2, 1):   # m5 = lat5; m4 = lat4 + up(m5); m3 = lat3 + up(m4)
+        _, _, h, w_ = feats[si]
+        top = "lat5" if si == 2 else "m4"
+        ops.append(("up", top, buf("up%d" % (si + 2), 256, h, w_)))
+        ops.append(("add", "lat%d" % (si + 2), "up%d" % (si + 2), buf("m%d" % (si + 2), 256, h, w_), "none"))
+    levels = []
+    for si in (1, 2, 3):
+        _, _, h, w_ = feats[si]
+        conv("lat5" if si == 3 else "m%d" % (si + 2), buf("p%d" % (si + 2), 256, h, w_), "none")
+        levels.append(("p%d" % (si + 2), h, w_))
+    _, h, w_ = levels[-1]
+    h6, w6 = synth.out_hw(h, w_, 2)
+    conv("p5", buf("p6", 256, h6, w6), "none")
+    levels.append(("p6", h6, w6))
+    ops.append(("relu", "p6", buf("p6.relu", 256, h6, w6)))
+    h7, w7 = synth.out_hw(h6, w6, 2)
+    conv("p6.relu", buf("p7", 256, h7, w7), "none")
+    levels.append(("p7", h7, w7))
+    outputs = []
+    for tower in ("cls", "box"):
+        for (feat, h, w_) in levels:
+            src = feat
+            for i in range(4):
+                dst = buf("%s.%s.%d" % (tower, feat, i), 256, h, w_)
+                conv(src, dst, "relu")
+                src = dst
+            outputs.append(src)
+    assert li[0] == len(layers) == 100
+    return ops, bufs, layers, tuple(outputs)
+
+
+class GpuNet:
+    """The program on the GPU through the C-ABI library: NHWC, bf16 (or fp16), k-entry patterns."""
+
+    def __init__(self, ctx, N, H0=800, W0=1088, k=4, seed=0, dtype="bf16"):
+        import torch
+        from . import binding as rt
+        self.rt, self.ctx, self.N, self.torch = rt, ctx, N, torch
+        self.ops, self.bufs, self.layers, self.output_names = program(H0, W0)
+        tdt = {"bf16": torch.bfloat16, "f16": torch.float16}[dtype]
+        self.t = {n: torch.zeros((N, H, W, C), dtype=tdt, device="cuda") for n, (C, H, W) in self.bufs.items()}
+        self.zero = {}   # all-zero operands of the ReLU glue op, one per shape
+        for op in self.ops:
+            if op[0] == "relu" and self.bufs[op[1]] not in self.zero:
+                C, H, W = self.bufs[op[1]]
+                self.zero[self.bufs[op[1]]] = torch.zeros((N, H, W, C), dtype=tdt, device="cuda")
+        masks = rt.rtoss_pattern_preset(k, rt.PRESET_CENTRE8 if k == 4 else rt.PRESET_CONN4)
+        self.packed, self.bias = {}, {}
+        for L in self.layers:
+            if L["wid"] in self.packed:
+                continue
+            w = torch.from_numpy(synth.kaiming_weights(seed, 3000 + L["wid"], L["cout"], L["cin"], L["ksize"])).cuda()
+            pid = ctx.rtoss_select_patterns(w, L["ksize"], masks, k)
+            self.packed[L["wid"]] = ctx.rtoss_pack(w, L["ksize"], masks, k, pid, rt.DTYPE_NAMES[dtype])
+            self.bias[L["wid"]] = torch.from_numpy(synth.bias(seed, 3000 + L["wid"], L["cout"])).cuda()
+        torch.cuda.synchronize()
+
+    def set_input(self, x_nchw):
+        self.t["in"].copy_(self.torch.from_numpy(x_nchw).permute(0, 2, 3, 1).to(self.t["in"].dtype))
+
+    def run(self):
+        rt, N, t = self.rt, self.N, self.t
+        for op in self.ops:
+            if op[0] == "conv":
+                _, i, src, dst, act = op
+                L = self.layers[i]
+                fn = self.ctx.rtoss_conv3x3_pattern if L["ksize"] == 3 else self.ctx.rtoss_conv1x1_pattern
+                fn(self.packed[L["wid"]], t[src], t[dst], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_NAMES[act],
+                   self.bias[L["wid"]])
+            elif op[0] == "add":
+                rt.rtoss_add_act(t[op[1]], t[op[2]], t[op[3]], rt.ACT_NAMES[op[4]])
+            elif op[0] == "up":
+                C, H, W = self.bufs[op[1]]
+                rt.rtoss_upsample2x(t[op[1]], t[op[2]], N, C, H, W, rt.NHWC)
+            elif op[0] == "relu":
+                rt.rtoss_add_act(t[op[1]], self.zero[self.bufs[op[1]]], t[op[2]], rt.ACT_RELU)
+
+    def outputs(self):
+        return {n: self.t[n].float().permute(0, 3, 1, 2).cpu().numpy() for n in self.output_names}
+
+    def close(self):
+        for p in self.packed.values():
+            p.close()

@@ -48,3 +48,26 @@ def test_chained_yolov5s_shaped_network_small_input():
     for name in ("o3", "o4", "o5"):
         assert np.array_equal(again[name], got[name])
     net.close()
+
+
+def test_chained_retinanet_shaped_network_small_input():
+    """The RetinaNet ResNet-50-FPN-shaped program (100 convolution calls on 68 weight tensors, residual adds,
+    top-down pyramid, towers with weights shared across the levels) against the same program in the CPU oracle."""
+    from paper_2303_02191_b200 import retinanet_net
+    N, H0, W0 = 1, 64, 96
+    x = synth.activations(71, 1, N, 64, H0 // 4, W0 // 4)
+    net = retinanet_net.GpuNet(gu.ctx(), N, H0, W0, k=4, seed=5)
+    net.set_input(synth.round_like(x, "bf16"))
+    net.run()
+    torch.cuda.synchronize()
+    assert gu.ctx().rtoss_device_status() == 0
+    got = net.outputs()
+    ref = net_oracle.oracle_forward_retinanet(x, H0, W0, k=4, seed=5)
+    assert len(got) == 10
+    for name in net.output_names:
+        err = orc.rel_err(got[name], ref[name])
+        print(name, got[name].shape, "chained relative error %.4f" % err)
+        assert got[name].shape == ref[name].shape
+        assert err <= 0.1
+        assert np.mean(np.abs(got[name] - ref[name])) <= 0.01 * np.sqrt(np.mean(ref[name] ** 2)) + 1e-6
+    net.close()
