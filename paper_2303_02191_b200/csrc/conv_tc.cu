@@ -338,41 +338,44 @@ __device__ __forceinline__ void epilogue_chunks(unsigned d_base, int c0, int c_s
     }
 }
 
-// Split K, the unit that arrived last: add up the KS partial sums of the tile (src points at this thread's lane
-// of the first one; partial sums are kMaxPx * 128 floats apart, columns 128 floats apart) and finish as usual.
+// Split K, second half: once every share of the tile has left its partial sums, each of the KS CTAs finishes its
+// own part of the tile's columns: the 32-column chunks c with c % KS == ks, as half chunks of 16 columns dealt to
+// the four warps of a lane quarter (sub = 0..3).  src points at this thread's lane of the first share; shares are
+// kMaxPx * 128 floats apart, columns 128 floats apart.
 template <typename T, int ACT>
-__device__ __forceinline__ void epilogue_from_scratch(const float* src, int KS, int c0, int c_step, int n_px, float bs, bool vec_ok,
+__device__ __forceinline__ void epilogue_from_scratch(const float* src, int KS, int ks, int sub, int n_px, float bs, bool vec_ok,
                                                       bool co_ok, unsigned patch, unsigned tab, const uint2* pos_tab, T* yb,
                                                       unsigned ry, unsigned rx, int lane) {
     const unsigned wr = patch + lane * 4;
     const unsigned rd = patch + (lane >> 2) * kPairPitch + (lane & 3) * 32;
     const unsigned tab_l = tab + (unsigned)(2 * (lane >> 2)) * 8;
     T* ybv = yb + (lane & 3) * 8;
-    for (; c0 < n_px; c0 += c_step) {
+    int mine = 0;
+    for (int h = 0; h * kPatchRows < n_px; ++h) {
+        if ((h >> 1) % KS != ks) continue;
+        if ((mine++ & 3) != sub) continue;
+        const int c0 = h * kPatchRows;
+        // sixteen independent loads in flight per share (the shares' loop is the outer one)
+        float sum[kPatchRows];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            // sixteen independent loads in flight per partial sum (the shares' loop is the outer one)
-            float sum[kPatchRows];
+        for (int j = 0; j < kPatchRows; ++j) sum[j] = 0.f;
+        const float* q = src + (size_t)c0 * 128;
+        for (int i = 0; i < KS; ++i, q += kMaxPx * 128) {
 #pragma unroll
-            for (int j = 0; j < kPatchRows; ++j) sum[j] = 0.f;
-            const float* q = src + (size_t)(c0 + h * kPatchRows) * 128;
-            for (int i = 0; i < KS; ++i, q += kMaxPx * 128) {
+            for (int j = 0; j < kPatchRows; ++j) sum[j] += __ldcg(q + j * 128);
+        }
+        unsigned r[16];
 #pragma unroll
-                for (int j = 0; j < kPatchRows; ++j) sum[j] += __ldcg(q + j * 128);
-            }
-            unsigned r[16];
+        for (int j = 0; j < kPatchRows; ++j) r[j] = __float_as_uint(sum[j]);
+        if (vec_ok) {
+            epilogue_half<T, ACT>(r, bs, wr, rd, tab_l + (unsigned)c0 * 8, ybv, ry, rx);
+        } else {
 #pragma unroll
-            for (int j = 0; j < kPatchRows; ++j) r[j] = __float_as_uint(sum[j]);
-            if (vec_ok) {
-                epilogue_half<T, ACT>(r, bs, wr, rd, tab_l + (unsigned)(c0 + h * kPatchRows) * 8, ybv, ry, rx);
-            } else {
-#pragma unroll
-                for (int j = 0; j < kPatchRows; ++j) {
-                    const uint2 e = pos_tab[c0 + h * kPatchRows + j];
-                    float v = bias_act<ACT>(r[j], bs);
-                    if (ACT == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
-                    if (co_ok && (e.y >> 16) < ry && (e.y & 0xFFFFu) < rx) yb[e.x + lane] = from_f32<T>(v);
-                }
+            for (int j = 0; j < kPatchRows; ++j) {
+                const uint2 e = pos_tab[c0 + j];
+                float v = bias_act<ACT>(r[j], bs);
+                if (ACT == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
+                if (co_ok && (e.y >> 16) < ry && (e.y & 0xFFFFu) < rx) yb[e.x + lane] = from_f32<T>(v);
             }
         }
     }
@@ -709,7 +712,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const unsigned d_base = tmem_base + (unsigned)(as * a.acc_cols) + ((unsigned)(quarter * 32) << 16);
             if (a.KS > 1) {
-                // ---- split K: leave the partial sums, count in, and finish the tile if this unit is the last one
+                // ---- split K.  Leave the partial sums, count in, wait (bounded) until the tile's other shares have
+                // counted in too, then finish this share's part of the columns.  All shares of a tile are resident
+                // together: the host makes one CTA per share and never more shares than SMs.
                 float* slot = a.sk_scratch + (size_t)tile * (kMaxPx * 128) + quarter * 32 + lane;
                 for (int c0 = c_first; c0 < a.N_px; c0 += c_step) {
                     unsigned r[32];
@@ -723,21 +728,45 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 __syncwarp();
                 if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_accEmpty + 8 * as) : "memory");
                 volatile int* sk_flag = reinterpret_cast<volatile int*>(tmem_ptr_gen + 2);
+                int* arrived = a.sk_count + t_idx;
+                int* finished = a.sk_count + 128 + t_idx;
                 asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");   // every epilogue warp has written and fenced
-                if (threadIdx.x == 64) *sk_flag = atomicAdd(a.sk_count + t_idx, 1);
-                asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
-                if (*sk_flag == a.KS - 1) {
-                    __threadfence();
-                    const float* src = a.sk_scratch + (size_t)(t_idx * a.KS) * (kMaxPx * 128) + quarter * 32 + lane;
-                    if (a.act == RTOSS_ACT_SILU)
-                        epilogue_from_scratch<T, RTOSS_ACT_SILU>(src, a.KS, c_first, c_step, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
-                    else if (a.act == RTOSS_ACT_RELU)
-                        epilogue_from_scratch<T, RTOSS_ACT_RELU>(src, a.KS, c_first, c_step, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
-                    else
-                        epilogue_from_scratch<T, RTOSS_ACT_NONE>(src, a.KS, c_first, c_step, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
-                    if (threadIdx.x == 64) a.sk_count[t_idx] = 0;   // ready for the next launch
+                if (threadIdx.x == 64) {
+                    atomicAdd(arrived, 1);
+                    const long long t0 = clock64();
+                    int seen = 0, good = 1;
+                    for (;;) {
+                        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(arrived) : "memory");
+                        if (seen >= a.KS) break;
+                        if (clock64() - t0 > kWaitCycles) {
+                            good = 0;
+                            break;
+                        }
+                    }
+                    *sk_flag = good;
                 }
-                asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");   // the flag word is free again
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
+                if (!*sk_flag) {   // a share never arrived: every epilogue warp leaves, the status word says why
+                    ok = false;
+                    if (threadIdx.x == 64) atomicExch(a.status, 5);
+                    break;
+                }
+                {
+                    const float* src = a.sk_scratch + (size_t)(t_idx * a.KS) * (kMaxPx * 128) + quarter * 32 + lane;
+                    const int ks = tile % a.KS;
+                    if (a.act == RTOSS_ACT_SILU)
+                        epilogue_from_scratch<T, RTOSS_ACT_SILU>(src, a.KS, ks, sub, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
+                    else if (a.act == RTOSS_ACT_RELU)
+                        epilogue_from_scratch<T, RTOSS_ACT_RELU>(src, a.KS, ks, sub, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
+                    else
+                        epilogue_from_scratch<T, RTOSS_ACT_NONE>(src, a.KS, ks, sub, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");   // all reads of the shares done; the flag word is free again
+                // the share that finishes last leaves both counters at zero for the next launch
+                if (threadIdx.x == 64 && atomicAdd(finished, 1) == a.KS - 1) {
+                    *arrived = 0;
+                    *finished = 0;
+                }
                 continue;
             }
             if (vec_ok) {
@@ -989,12 +1018,12 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     a.sk_count = ctx->sk_count;
     {
         const long tiles = (long)d->N * a.tiles_y * a.tiles_x * a.co_tiles;
-        // The round trip of the partial sums (a store, a fence, a counter, and the last CTA reading every share back
-        // through one SM) costs about as much as 70 instructions of the chain: measured on 256-channel layers at
-        // 25x34 and 13x17, halving a chain of 144 gained nothing, while stride-2 layers (four staged input phases
-        // per channel block) and chains of 288 and more came out ahead.  Hence the shares stay long.
-        const int min_cb = p->ksize == 3 ? (S == 2 ? 2 : 4) : 32;
-        if (!pxm && ctx->sk_scratch && tiles * 2 <= sms && a.ncb >= 2 * min_cb) {
+        // The round trip of the partial sums costs about 6 K cycles (a 128 KB store, a fence, the counter, a 128 KB
+        // read), as much as 45 instructions of the chain: chains of 144 and more are cut (3x3 layers from four
+        // channel blocks, 1x1 layers from 32), and a share keeps at least one block resp. eight.
+        const int min_cb = p->ksize == 3 ? 1 : 8;
+        const int min_ncb = p->ksize == 3 ? 4 : 32;
+        if (!pxm && a.R == 1 && ctx->sk_scratch && tiles * 2 <= sms && tiles <= 128 && a.ncb >= min_ncb) {
             int want = (int)(sms / tiles);
             if (want > a.ncb / min_cb) want = a.ncb / min_cb;
             if (want > 8) want = 8;

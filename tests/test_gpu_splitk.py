@@ -1,5 +1,5 @@
 """Tensor path on layers with few tiles and many channel blocks: the channel blocks of a tile are shared out to
-several CTAs (split K) and the CTA that arrives last adds up the partial sums.  Parity against the CPU oracle,
+several CTAs (split K), every share leaves its partial sums, and each CTA finishes a part of the tile once all have arrived.  Parity against the CPU oracle,
 twice in a row on the same context (the arrival counters must be back at zero), with every activation, a channel
 slice of a wider output, a ragged filter count and both kernel sizes."""
 import numpy as np
@@ -19,10 +19,11 @@ CASES = [
     (3, 256, 256, 2, 13, 17, 1, "relu", (0, 0)),
     (3, 256, 256, 1, 7, 9, 1, "none", (0, 0)),
     (3, 512, 128, 1, 20, 20, 1, "silu", (0, 0)),
-    (3, 192, 100, 1, 9, 11, 1, "silu", (0, 0)),       # ragged filter count: element stores
+    (3, 320, 100, 1, 9, 11, 1, "silu", (0, 0)),       # ragged filter count: element stores; five channel blocks in four shares
     (3, 256, 128, 1, 12, 12, 2, "silu", (64, 256)),   # stride 2, channel slice of a wider tensor
     (1, 2048, 512, 1, 7, 9, 1, "relu", (0, 0)),
-    (1, 1024, 128, 2, 10, 10, 1, "silu", (0, 0)),
+    (1, 2048, 128, 2, 10, 10, 1, "silu", (0, 0)),
+    (3, 256, 256, 4, 25, 34, 1, "relu", (0, 0)),      # sixteen tiles x four shares: 64 CTAs
 ]
 
 
