@@ -253,10 +253,7 @@ typedef struct {
  * II.B: work proportional to the non-zero weights).  x: N x Cin x H x W in the
  * given layout, y: N x Cs x Ho x Wo with Cs = y_channel_stride (or Cout),
  * written at channels [offset, offset+Cout).  x and y must not overlap.  The
- * packed handle must come from rtoss_pack with ksize 3.  The tensor path may
- * use the context's device workspace (partial sums of layers it cuts along
- * the channels): convolutions of one context must not overlap on the GPU;
- * callers that run two streams at once create one context per stream. */
+ * packed handle must come from rtoss_pack with ksize 3. */
 rtoss_status rtoss_conv3x3_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const void* x_dev, void* y_dev,
                                    const rtoss_conv_desc* desc, void* cuda_stream);
 

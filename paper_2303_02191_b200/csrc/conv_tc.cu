@@ -88,11 +88,9 @@ struct TcArgs {
     int w_rows;           // filter rows per staged weight tile (128; fewer with positions as the M operand)
     int rep_rows, R;      // filters as M, narrow layer: the tile holds R copies of rep_rows filter rows (else 128, 1)
     int pxm, MH, n_cols;  // positions as the M operand: M halves of 128 positions per tile, filters per tile (the MMA's N)
-    // Split K: a tile's channel blocks are shared out to KS units (CTAs), cb_per blocks each; every unit leaves its
-    // partial sums in sk_scratch and the unit that arrives last at the tile's counter adds them up and finishes.
+    // Split K: a tile's channel blocks are shared out to the KS CTAs of a thread-block cluster, cb_per blocks each;
+    // the partial sums are exchanged through distributed shared memory and every CTA finishes a part of the tile.
     int KS, cb_per;
-    float* sk_scratch;  // [units][kMaxPx columns][128 lanes] fp32
-    int* sk_count;      // [tiles], zero between launches
 };
 
 __device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -122,6 +120,26 @@ __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
         if (mbar_try(bar, parity)) return true;
         if (clock64() - t0 > kWaitCycles) return false;
     }
+}
+
+// Thread-block cluster primitives (split K): rank of this CTA, the address of a peer's shared memory, a store to it,
+// and the cluster-wide barrier (release / acquire: stores to peers before it are visible after it).
+__device__ __forceinline__ unsigned cluster_rank() {
+    unsigned r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ unsigned peer_smem(unsigned local_addr, unsigned rank) {
+    unsigned r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_peer_f32(unsigned addr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
 }
 
 __device__ __forceinline__ void tma_load_4d(unsigned dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
@@ -338,31 +356,32 @@ __device__ __forceinline__ void epilogue_chunks(unsigned d_base, int c0, int c_s
     }
 }
 
-// Split K, second half: once every share of the tile has left its partial sums, each of the KS CTAs finishes its
-// own part of the tile's columns: the 32-column chunks c with c % KS == ks, as half chunks of 16 columns dealt to
-// the four warps of a lane quarter (sub = 0..3).  src points at this thread's lane of the first share; shares are
-// kMaxPx * 128 floats apart, columns 128 floats apart.
+// Split K, second half.  Every CTA of the cluster owns the 32-column chunks c of the tile with c % KS == its rank
+// (its local chunk lc = c / KS) and holds, in its own shared memory at `buf`, what each of the KS shares summed
+// for them: share i, local chunk lc, column col, accumulator lane row at ((i * n_lc + lc) * 32 + col) * 128 + row
+// floats.  The owned chunks are finished as half chunks of 16 columns dealt to the four warps of a lane quarter.
 template <typename T, int ACT>
-__device__ __forceinline__ void epilogue_from_scratch(const float* src, int KS, int ks, int sub, int n_px, float bs, bool vec_ok,
-                                                      bool co_ok, unsigned patch, unsigned tab, const uint2* pos_tab, T* yb,
-                                                      unsigned ry, unsigned rx, int lane) {
+__device__ __forceinline__ void epilogue_from_shares(unsigned buf, int KS, int rank, int n_lc, int sub, int row, int n_px, float bs,
+                                                     bool vec_ok, bool co_ok, unsigned patch, unsigned tab, const uint2* pos_tab,
+                                                     T* yb, unsigned ry, unsigned rx, int lane) {
     const unsigned wr = patch + lane * 4;
     const unsigned rd = patch + (lane >> 2) * kPairPitch + (lane & 3) * 32;
     const unsigned tab_l = tab + (unsigned)(2 * (lane >> 2)) * 8;
     T* ybv = yb + (lane & 3) * 8;
-    int mine = 0;
-    for (int h = 0; h * kPatchRows < n_px; ++h) {
-        if ((h >> 1) % KS != ks) continue;
-        if ((mine++ & 3) != sub) continue;
-        const int c0 = h * kPatchRows;
-        // sixteen independent loads in flight per share (the shares' loop is the outer one)
+    for (int t = sub; t < 2 * n_lc; t += 4) {
+        const int lc = t >> 1, c0 = (lc * KS + rank) * 32 + (t & 1) * kPatchRows;   // first column of the half chunk
+        if (c0 >= n_px) continue;
         float sum[kPatchRows];
 #pragma unroll
         for (int j = 0; j < kPatchRows; ++j) sum[j] = 0.f;
-        const float* q = src + (size_t)c0 * 128;
-        for (int i = 0; i < KS; ++i, q += kMaxPx * 128) {
+        for (int i = 0; i < KS; ++i) {
+            const unsigned q = buf + (unsigned)((((i * n_lc + lc) * 32 + (t & 1) * kPatchRows) * 128 + row) * 4);
 #pragma unroll
-            for (int j = 0; j < kPatchRows; ++j) sum[j] += __ldcg(q + j * 128);
+            for (int j = 0; j < kPatchRows; ++j) {
+                float v;
+                asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(q + j * 512));
+                sum[j] += v;
+            }
         }
         unsigned r[16];
 #pragma unroll
@@ -613,7 +632,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             // TMEM may only be released after the epilogue has drained the last tiles: the last min(AS, tiles done)
             // stages used, walking backwards from the ring position
-            for (int i = 0; i < a.AS && i < n_done && ok; ++i) {
+            for (int i = 0; i < a.AS && i < n_done && ok && a.KS == 1; ++i) {   // (split K: the cluster barriers below order it)
                 if (--as < 0) {
                     as = a.AS - 1;
                     pacc ^= 1;
@@ -708,64 +727,39 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int c_first = (sub + 4 * copy) * 32, c_step = 128 * a.R;
             const float bs = a.act == RTOSS_ACT_SILU ? 0.5f * bv : bv;
             ok = mbar_wait(bar_accFull + 8 * as, (gt / a.AS) & 1);
-            if (!ok) break;
+            if (!ok && a.KS == 1) break;   // (split K: the cluster barriers below must still be passed)
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const unsigned d_base = tmem_base + (unsigned)(as * a.acc_cols) + ((unsigned)(quarter * 32) << 16);
             if (a.KS > 1) {
-                // ---- split K.  Leave the partial sums, count in, wait (bounded) until the tile's other shares have
-                // counted in too, then finish this share's part of the columns.  All shares of a tile are resident
-                // together: the host makes one CTA per share and never more shares than SMs.
-                float* slot = a.sk_scratch + (size_t)tile * (kMaxPx * 128) + quarter * 32 + lane;
-                for (int c0 = c_first; c0 < a.N_px; c0 += c_step) {
-                    unsigned r[32];
-                    tmem_ld32(d_base + (unsigned)c0, r);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                // ---- split K.  The KS CTAs of the cluster hold the partial sums of one tile.  Barrier 1: every CTA's
+                // MMAs have completed, so the operand rings of all of them are free; each CTA then stores its partial
+                // sums of chunk c into the shared memory of the chunk's owner (rank c % KS); barrier 2: all stores have
+                // landed; every CTA adds up and finishes the chunks it owns.  Every thread of the cluster passes both
+                // barriers, whatever happened to its waits (the other roles pass them at the end of the kernel).
+                const int rank = (int)cluster_rank(), n_chunks = (a.N_px + 31) >> 5, n_lc = (n_chunks + a.KS - 1) / a.KS;
+                cluster_sync_all();
+                if (ok) {
+                    for (int c0 = c_first; c0 < a.N_px; c0 += c_step) {
+                        unsigned r[32];
+                        tmem_ld32(d_base + (unsigned)c0, r);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                        const int c = c0 >> 5;
+                        const unsigned dst = peer_smem(sA + (unsigned)((((rank * n_lc + c / a.KS) * 32) * 128 + quarter * 32 + lane) * 4),
+                                                       (unsigned)(c % a.KS));
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) slot[(size_t)(c0 + j) * 128] = __uint_as_float(r[j]);   // 128 contiguous bytes per warp
-                }
-                __threadfence();
-                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_accEmpty + 8 * as) : "memory");
-                volatile int* sk_flag = reinterpret_cast<volatile int*>(tmem_ptr_gen + 2);
-                int* arrived = a.sk_count + t_idx;
-                int* finished = a.sk_count + 128 + t_idx;
-                asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");   // every epilogue warp has written and fenced
-                if (threadIdx.x == 64) {
-                    atomicAdd(arrived, 1);
-                    const long long t0 = clock64();
-                    int seen = 0, good = 1;
-                    for (;;) {
-                        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(arrived) : "memory");
-                        if (seen >= a.KS) break;
-                        if (clock64() - t0 > kWaitCycles) {
-                            good = 0;
-                            break;
-                        }
+                        for (int j = 0; j < 32; ++j) st_peer_f32(dst + j * 512, __uint_as_float(r[j]));   // 128 contiguous bytes per warp
                     }
-                    *sk_flag = good;
                 }
-                asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
-                if (!*sk_flag) {   // a share never arrived: every epilogue warp leaves, the status word says why
-                    ok = false;
-                    if (threadIdx.x == 64) atomicExch(a.status, 5);
-                    break;
-                }
-                {
-                    const float* src = a.sk_scratch + (size_t)(t_idx * a.KS) * (kMaxPx * 128) + quarter * 32 + lane;
-                    const int ks = tile % a.KS;
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                cluster_sync_all();
+                if (ok) {
+                    const int row = quarter * 32 + lane;
                     if (a.act == RTOSS_ACT_SILU)
-                        epilogue_from_scratch<T, RTOSS_ACT_SILU>(src, a.KS, ks, sub, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
+                        epilogue_from_shares<T, RTOSS_ACT_SILU>(sA, a.KS, rank, n_lc, sub, row, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
                     else if (a.act == RTOSS_ACT_RELU)
-                        epilogue_from_scratch<T, RTOSS_ACT_RELU>(src, a.KS, ks, sub, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
+                        epilogue_from_shares<T, RTOSS_ACT_RELU>(sA, a.KS, rank, n_lc, sub, row, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
                     else
-                        epilogue_from_scratch<T, RTOSS_ACT_NONE>(src, a.KS, ks, sub, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
-                }
-                asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");   // all reads of the shares done; the flag word is free again
-                // the share that finishes last leaves both counters at zero for the next launch
-                if (threadIdx.x == 64 && atomicAdd(finished, 1) == a.KS - 1) {
-                    *arrived = 0;
-                    *finished = 0;
+                        epilogue_from_shares<T, RTOSS_ACT_NONE>(sA, a.KS, rank, n_lc, sub, row, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
                 }
                 continue;
             }
@@ -804,6 +798,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (!ok && lane == 0) atomicExch(a.status, 3);
     }
 
+    if (a.KS > 1 && (warp < 2 || warp >= kWeightWarp)) {   // split K: the barriers the epilogue warps pass around the exchange
+        cluster_sync_all();
+        cluster_sync_all();
+    }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 1) {
@@ -1014,22 +1012,27 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     // chain (an instruction costs the same however few positions it covers), so the blocks go to several CTAs.
     a.KS = 1;
     a.cb_per = a.ncb;
-    a.sk_scratch = ctx->sk_scratch;
-    a.sk_count = ctx->sk_count;
     {
         const long tiles = (long)d->N * a.tiles_y * a.tiles_x * a.co_tiles;
-        // The round trip of the partial sums costs about 6 K cycles (a 128 KB store, a fence, the counter, a 128 KB
-        // read), as much as 45 instructions of the chain: chains of 144 and more are cut (3x3 layers from four
-        // channel blocks, 1x1 layers from 32), and a share keeps at least one block resp. eight.
-        const int min_cb = p->ksize == 3 ? 1 : 8;
-        const int min_ncb = p->ksize == 3 ? 4 : 32;
-        if (!pxm && a.R == 1 && ctx->sk_scratch && tiles * 2 <= sms && tiles <= 128 && a.ncb >= min_ncb) {
+        // The exchange costs a few thousand cycles (two cluster barriers, 128 KB through distributed shared memory):
+        // chains of 72 instructions and more are cut; a share keeps at least one channel block (1x1: four).  The
+        // CTAs of a tile form one cluster (at most 8), one CTA per share, and all clusters must be resident.
+        const int min_cb = p->ksize == 3 ? 1 : 4;
+        const int min_ncb = p->ksize == 3 ? 2 : 16;
+        const int n_lc_max = 8;   // a tile has at most 8 chunks of 32 columns: the owner's buffers take KS * ceil(chunks / KS) * 16 KB
+        if (!pxm && a.R == 1 && tiles * 2 <= sms && a.ncb >= min_ncb) {
             int want = (int)(sms / tiles);
             if (want > a.ncb / min_cb) want = a.ncb / min_cb;
             if (want > 8) want = 8;
-            if (want > 1) {
-                a.cb_per = (a.ncb + want - 1) / want;
-                a.KS = (a.ncb + a.cb_per - 1) / a.cb_per;
+            while (want > 1) {
+                const int cb_per = (a.ncb + want - 1) / want, ks = (a.ncb + cb_per - 1) / cb_per;
+                const int n_chunks = (plan.N_px + 31) / 32, n_lc = (n_chunks + ks - 1) / ks;
+                if (ks > 1 && ks * n_lc <= 2 * n_lc_max && (size_t)ks * n_lc * 16384 <= (size_t)a.NA * a.a_stage_bytes + (size_t)a.NB * a.b_stage_bytes) {
+                    a.cb_per = cb_per;
+                    a.KS = ks;
+                    break;
+                }
+                --want;
             }
         }
     }
@@ -1094,8 +1097,20 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
         if (e != cudaSuccess) return (int)e;
         attr_set = true;
     }
-    const cudaError_t le = a.is_bf16 ? rtoss_dev::launch_pdl(conv_tc_kernel<__nv_bfloat16>, grid, kTcThreads, smem, (cudaStream_t)stream, tmA, tmB, a)
-                                     : rtoss_dev::launch_pdl(conv_tc_kernel<__half>, grid, kTcThreads, smem, (cudaStream_t)stream, tmA, tmB, a);
+    cudaError_t le;
+    if (a.KS > 1) {
+        // one cluster per tile; if the device cannot place the clusters the layer runs uncut
+        le = a.is_bf16 ? rtoss_dev::launch_pdl(conv_tc_kernel<__nv_bfloat16>, grid, kTcThreads, smem, (cudaStream_t)stream, a.KS, tmA, tmB, a)
+                       : rtoss_dev::launch_pdl(conv_tc_kernel<__half>, grid, kTcThreads, smem, (cudaStream_t)stream, a.KS, tmA, tmB, a);
+        if (le == cudaSuccess) return (int)cudaGetLastError();
+        cudaGetLastError();
+        a.KS = 1;
+        a.cb_per = a.ncb;
+        const size_t uncut = (size_t)d->N * a.tiles_y * a.tiles_x * a.co_tiles;
+        grid = dim3((unsigned)(uncut < (size_t)sms ? uncut : (size_t)sms));
+    }
+    le = a.is_bf16 ? rtoss_dev::launch_pdl(conv_tc_kernel<__nv_bfloat16>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, tmA, tmB, a)
+                   : rtoss_dev::launch_pdl(conv_tc_kernel<__half>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, tmA, tmB, a);
     if (le != cudaSuccess) return (int)le;
     return (int)cudaGetLastError();
 }

@@ -118,14 +118,6 @@ rtoss_status rtoss_create(int device, rtoss_ctx** out) {
     cudaSetDevice(device);
     cudaError_t se = cudaMalloc((void**)&c->dev_status, sizeof(int));
     if (se == cudaSuccess) se = cudaMemset(c->dev_status, 0, sizeof(int));
-    if (se == cudaSuccess) se = cudaMalloc((void**)&c->sk_scratch, (size_t)c->sm_count * 256 * 128 * sizeof(float));
-    if (se == cudaSuccess) se = cudaMalloc((void**)&c->sk_count, 256 * sizeof(int));
-    if (se == cudaSuccess) se = cudaMemset(c->sk_count, 0, 256 * sizeof(int));
-    if (se != cudaSuccess) {
-        if (c->dev_status) cudaFree(c->dev_status);
-        if (c->sk_scratch) cudaFree(c->sk_scratch);
-        if (c->sk_count) cudaFree(c->sk_count);
-    }
     cudaSetDevice(prev);
     if (se != cudaSuccess) {
         cudaGetLastError();
@@ -154,8 +146,6 @@ void rtoss_destroy(rtoss_ctx* ctx) {
     if (ctx->ws_x) cudaFree(ctx->ws_x);
     if (ctx->ws_y) cudaFree(ctx->ws_y);
     if (ctx->dev_status) cudaFree(ctx->dev_status);
-    if (ctx->sk_scratch) cudaFree(ctx->sk_scratch);
-    if (ctx->sk_count) cudaFree(ctx->sk_count);
     cudaSetDevice(prev);
     delete ctx;
 }

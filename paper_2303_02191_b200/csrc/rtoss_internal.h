@@ -32,11 +32,6 @@ struct rtoss_ctx {
     void* h_ev_in[8];   // cudaEvent_t per batch chunk: copy in done
     void* h_ev_run[8];  // kernel done
     int* dev_status;  // device word: 0, or the code of a bounded device-side wait that ran out
-    // split-K workspace of the tensor path: partial sums of up to sm_count units (256 columns x 128 lanes of fp32
-    // each) and one arrival counter per tile.  Shared by every convolution of the context: calls that overlap on
-    // the GPU (two streams) must use two contexts.
-    float* sk_scratch;
-    int* sk_count;
     mutable rtoss_tmap_entry tmap_cache[32];  // activation descriptors of the tensor path, round robin
     mutable int tmap_next;
 };
