@@ -435,6 +435,7 @@ struct Variant {
 constexpr int kStemCo = 32;
 constexpr int kStemPx = 4;
 constexpr int kStemThreads = 128;
+constexpr int kStemNf = 4;   // filters per trip of the filter loop
 
 // SiLU of a 16-bit output through tanh.approx (relative error about 2^-11, below half an ulp of bf16);
 // fp32 outputs keep the exponential form (the tolerance there is 1e-4).
@@ -548,12 +549,15 @@ __global__ void __launch_bounds__(kStemThreads) conv3x3_small_cin_kernel(const C
                 }
             }
         }
-        for (int c8 = 0; c8 < kStemCo; c8 += PER16) {
-            __align__(16) T o[kStemPx][PER16];
+        // kStemNf filters per trip of a loop that is NOT unrolled: with all 32 filters unrolled the body was 17 KB of
+        // instructions and the warps waited for instruction fetch more than for anything else
+#pragma unroll 1
+        for (int q0 = 0; q0 < kStemCo; q0 += kStemNf) {
+            __align__(8) T o[kStemPx][kStemNf];
 #pragma unroll
-            for (int q = 0; q < PER16; ++q) {
+            for (int q = 0; q < kStemNf; ++q) {
                 float w[KW];
-                const float4* wr = reinterpret_cast<const float4*>(sWd[c8 + q]);
+                const float4* wr = reinterpret_cast<const float4*>(sWd[q0 + q]);
 #pragma unroll
                 for (int i = 0; i < KW / 4; ++i) {
                     const float4 v = wr[i];
@@ -578,22 +582,19 @@ __global__ void __launch_bounds__(kStemThreads) conv3x3_small_cin_kernel(const C
             for (int px = 0; px < kStemPx; ++px) {
                 const int ox = ox0 + px;
                 if (staged) {
-                    sOut[threadIdx.x * kStageRow + px * 4 + c8 / PER16] = *reinterpret_cast<const uint4*>(o[px]);
+                    // 8 bytes (four 16-bit filters) into the thread's 64 bytes of pixel px
+                    reinterpret_cast<uint2*>(sOut)[(threadIdx.x * kStageRow + px * 4) * 2 + q0 / kStemNf] =
+                        *reinterpret_cast<const uint2*>(o[px]);
                     continue;
                 }
                 if (ox >= a.Wo || !active) continue;
-                if (vec) {
-                    *reinterpret_cast<uint4*>(yg + (((size_t)n * a.Ho + oy) * a.Wo + ox) * Cs + a.y_c_off + co0 + c8) =
-                        *reinterpret_cast<const uint4*>(o[px]);
-                } else {
 #pragma unroll
-                    for (int q = 0; q < PER16; ++q) {
-                        const int co = co0 + c8 + q;
-                        if (co < a.Cout) {
-                            const size_t idx = a.layout == RTOSS_NCHW ? (((size_t)n * Cs + a.y_c_off + co) * a.Ho + oy) * a.Wo + ox
-                                                                      : (((size_t)n * a.Ho + oy) * a.Wo + ox) * Cs + a.y_c_off + co;
-                            yg[idx] = o[px][q];
-                        }
+                for (int q = 0; q < kStemNf; ++q) {
+                    const int co = co0 + q0 + q;
+                    if (co < a.Cout) {
+                        const size_t idx = a.layout == RTOSS_NCHW ? (((size_t)n * Cs + a.y_c_off + co) * a.Ho + oy) * a.Wo + ox
+                                                                  : (((size_t)n * a.Ho + oy) * a.Wo + ox) * Cs + a.y_c_off + co;
+                        yg[idx] = o[px][q];
                     }
                 }
             }
