@@ -1,4 +1,4 @@
-// Tensor-core path of the pattern convolutions (bf16 / fp16, NHWC, stride 1).
+// Tensor-core path of the pattern convolutions (bf16 / fp16, NHWC, stride 1 or 2).
 //
 // Per-kernel patterns cannot be compacted into a dense contraction (every
 // filter keeps different (channel, tap) positions), so this path evaluates the
@@ -23,19 +23,25 @@
 //   * Operand roles: the weights are the M operand (128 filters = the 128 TMEM
 //     lanes), the positions are the N operand (up to 256 per instruction), K =
 //     16 channels per instruction.  One instruction costs about 140 cycles
-//     whatever N is (the 128-row M operand is fetched at a row per cycle), so N
+//     whatever N is, and with M = 64 as with M = 128 (measured), so N
 //     must be wide: 128 x 256 x 16 per instruction runs near the tensor peak,
 //     128 x 128 x 16 at half of it (measured on this kernel with both roles).
 //   * Weights are the dense-expanded form Wt[t][co][ci] that rtoss_pack builds
-//     next to the packed arrays; one TMA box per (tap, channel block); filters
+//     next to the packed arrays; one TMA box per (kernel row of three taps,
+//     channel block); filters
 //     beyond Cout are zero-filled by TMA.
 //   * Persistent CTAs, one per SM, each walking a strided list of tiles.  Warp
-//     roles: warp 0 issues TMA, warp 1 issues tcgen05.mma and owns the TMEM
-//     allocation, warps 2..17 run the epilogue (tcgen05.ld, bias, activation,
-//     rounding, NHWC stores: a warp holds 32 consecutive filters of one
-//     position, i.e. 64 contiguous bytes per store instruction).  Activation
-//     and weight stages form rings that run on across tiles; two accumulator
-//     stages in TMEM let the epilogue of a tile run under the MMAs of the next.
+//     roles: warp 0 issues the TMA copies of the activations, warp 1 issues
+//     tcgen05.mma and owns the TMEM allocation, warps 2..17 run the epilogue
+//     (tcgen05.ld, bias, activation, rounding, a transpose through shared memory,
+//     16-byte NHWC stores), warp 18 issues the TMA copies of the weights (a stage
+//     of three taps is one copy: issuing a copy occupies its thread for hundreds
+//     of cycles whatever the size).  Activation and weight stages form rings
+//     that run on across tiles; two accumulator stages in TMEM let the epilogue
+//     of a tile run under the MMAs of the next.
+//   * Layers with few tiles and long channel loops are cut along the channel
+//     blocks: the CTAs that share a tile form a thread-block cluster and exchange
+//     their partial sums through distributed shared memory (split K).
 //   * Launched with programmatic stream serialization: barrier set-up, TMEM allocation and descriptor
 //     prefetch run before griddepcontrol.wait, i.e. possibly under the tail of the previous kernel.
 //   * Every mbarrier wait is bounded; a wait that runs out records a code in
