@@ -5,7 +5,7 @@ For every point: cold-L2 and warm kernel time (CUDA events), algorithmic GB/s, n
 fraction of the point's roofline max(bytes / HBM peak, nnz FLOP / pipe peak).  bf16 runs NHWC (tensor path
 where it applies), fp32 runs NCHW (FMA path).  Writes a CSV and prints a short summary.
 
-    python -m paper_2303_02191_b200.sweep --out gpurun_out/sweep.csv [--quick]
+    python -m paper_2303_02191_b200.sweep --out sweep.csv [--quick]
 """
 import argparse
 import csv
@@ -45,7 +45,7 @@ def main():
     from . import binding as rt
 
     ap = argparse.ArgumentParser()
-    ap.add_argument("--out", default="gpurun_out/sweep.csv")
+    ap.add_argument("--out", default="sweep.csv")
     ap.add_argument("--quick", action="store_true")
     ap.add_argument("--reps", type=int, default=10)
     args = ap.parse_args()
