@@ -1021,10 +1021,11 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     {
         const long tiles = (long)d->N * a.tiles_y * a.tiles_x * a.co_tiles;
         // The exchange costs a few thousand cycles (two cluster barriers, 128 KB through distributed shared memory):
-        // chains of 72 instructions and more are cut; a share keeps at least one channel block (1x1: four).  The
-        // CTAs of a tile form one cluster (at most 8), one CTA per share, and all clusters must be resident.
-        const int min_cb = p->ksize == 3 ? 1 : 4;
-        const int min_ncb = p->ksize == 3 ? 2 : 16;
+        // chains of 72 instructions (3x3: two channel blocks) resp. 32 (1x1: eight blocks) and more are cut, a share
+        // keeps at least one block (1x1: two); cutting shorter 1x1 chains was measured and lost.  The CTAs of a tile
+        // form one cluster (at most 8), one CTA per share.
+        const int min_cb = p->ksize == 3 ? 1 : 2;
+        const int min_ncb = p->ksize == 3 ? 2 : 8;
         const int n_lc_max = 8;   // a tile has at most 8 chunks of 32 columns: the owner's buffers take KS * ceil(chunks / KS) * 16 KB
         if (!pxm && a.R == 1 && tiles * 2 <= sms && a.ncb >= min_ncb) {
             int want = (int)(sms / tiles);
