@@ -27,6 +27,44 @@ CASES = [
 ]
 
 
+def test_split_k_fp16_and_graph_replay():
+    """fp16 data, and the cluster launch captured into a CUDA graph: the replay gives the bits of the eager run."""
+    masks = orc.pattern_preset(3, orc.PRESET_CONN4)
+    w = synth.kaiming_weights(4, 12, 256, 256, 3)
+    b = synth.bias(4, 12, 256)
+    x = synth.round_like(synth.activations(4, 12, 2, 256, 13, 17), "f16")
+    pid, packed = G.select_pack(w, 3, masks, 3, "f16")
+    _, wd, _ = G.oracle_weights(w, 3, masks, 3, "f16")
+    ref = orc.conv3x3(x, wd, b, 1, orc.ACT_SILU, orc.DT_F16)
+    c = G.ctx()
+    xd = G.to_dev(x, "f16", "nhwc")
+    bd = torch.from_numpy(b).cuda()
+    y = torch.zeros((2, 13, 17, 256), dtype=torch.float16, device="cuda")
+
+    def run():
+        c.rtoss_conv3x3_pattern(packed, xd, y, 2, 13, 17, 1, rt.NHWC, rt.ACT_SILU, bd, path=rt.PATH_TENSOR)
+
+    run()
+    torch.cuda.synchronize()
+    eager = y.clone()
+    assert orc.rel_err(G.from_dev(eager, "nhwc"), ref) <= G.TOL["f16"]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        run()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        run()
+    y.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(y, eager)
+    assert c.rtoss_device_status() == 0
+    packed.close()
+
+
 @pytest.mark.parametrize("ksize,cin,cout,N,H,W,stride,act,ysl", CASES)
 def test_split_k_parity(ksize, cin, cout, N, H, W, stride, act, ysl):
     masks = orc.pattern_preset(4, orc.PRESET_CENTRE8)
