@@ -178,7 +178,13 @@ def cpu_baseline_sample(layers_k, dtype, N, budget_s):
     frac = min(1.0, max(1.0 / 64, budget_s / max(t_image, 1e-6)))
     n = min(N, max(1, int(budget_s / t_image))) if frac >= 1.0 else 1
     t, f = oracle_step(layers_k, dtype, n, frac)
-    return n * f / t, t, f, n
+    # a workload the oracle finishes in a second or two is passed over several times (about ten seconds in all)
+    passes = 1
+    if t < 5.0:
+        extra = min(20, int(10.0 / max(t, 1e-3)))
+        ts = [t] + [oracle_step(layers_k, dtype, n, frac)[0] for _ in range(extra)]
+        t, passes = float(np.mean(ts)), len(ts)
+    return n * f / t, t, f, n, passes
 
 
 def run_reference(args):
@@ -541,10 +547,11 @@ def run_gpu(args):
                         L["name"], L["ksize"], L["cin"], L["cout"], L["H"], L["W"], L["stride"], st["k"],
                         "tensor" if tc else "fma", ms * 1e3, hbm_us, pipe_us, max(hbm_us, pipe_us) / (ms * 1e3)))
         if args.cpu_baseline:
-            v_cpu, t_cpu, f_cpu, n_cpu = cpu_baseline_sample(layers_k, dtype, N, 15.0)
+            v_cpu, t_cpu, f_cpu, n_cpu, p_cpu = cpu_baseline_sample(layers_k, dtype, N, 15.0)
             out["cpu_baseline"] = {"value": v_cpu, "unit": "images/s", "cores": os.cpu_count(), "kind": "oracle",
                                    "sample": "%d image(s) of the batch of %d, the first %.3f of every layer's output channels, "
-                                             "one pass of %.1f s; images/s = images x fraction / seconds" % (n_cpu, N, f_cpu, t_cpu)}
+                                             "%d pass(es) of %.1f s each (mean); images/s = images x fraction / seconds"
+                                             % (n_cpu, N, f_cpu, p_cpu, t_cpu)}
         print(json.dumps(out))
     torch.cuda.synchronize()
     batch.close()
