@@ -244,6 +244,16 @@ typedef struct {
     int y_channel_offset;   /* y may be a channel slice of a wider tensor: */
     int y_channel_stride;   /*   channels of that tensor, 0 = Cout */
     rtoss_path path;        /* which kernel family runs the call */
+    const void* residual_dev; /* NULL, or a tensor laid out exactly like y (same type, layout, channel stride and
+                               * offset: element (n,co,oy,ox) at the index it has in y) that is added before the
+                               * activation: y = act(round(conv + bias) + residual), the sum formed in fp32 and
+                               * rounded once more -- for act none and ReLU bit for bit what the convolution with
+                               * act = none followed by rtoss_add_act gives, in one pass; for SiLU the same up to
+                               * the rounding of the two SiLU evaluations (the residual connection that closes a
+                               * bottleneck block; not part of the paper's method).  May be y itself.  Tensor
+                               * path only (16-bit NHWC, more than 64 filters or a 3x3 kernel, pointer 16-byte
+                               * aligned): other calls return RTOSS_ERR_UNSUPPORTED before anything is launched
+                               * and the caller adds separately. */
 } rtoss_conv_desc;
 
 /* y[n,co,oy,ox] = act( bias[co] + sum_ci sum_{t in mask(pid[co,ci])}

@@ -67,6 +67,7 @@ constexpr int kMTile = 128;          // filters per tile = TMEM lanes
 constexpr int kPxmMaxCout = 64;      // layers this narrow run with positions as the M operand
 constexpr int kMaxPx = 256;          // most positions in a tile's list
 constexpr int kPairPitch = 144;      // bytes per row (a pair of positions x 32 filters, + 16 pad) of the packed patch
+constexpr int kResStage = 2048;   // per epilogue warp: two buffers of 2 x 32 residual pieces of 16 bytes
 constexpr int kPatchBytes = kPatchRows / 2 * kPairPitch;  // an epilogue warp's transpose patch
 constexpr int kKBlock = 64;       // channels per staged block: 128 bytes of bf16 / fp16
 constexpr int kRowBytes = 128;    // one padded pixel, one channel block
@@ -74,6 +75,7 @@ constexpr long long kWaitCycles = 2000000000LL;  // about one second
 
 struct TcArgs {
     void* y;
+    const void* resid;   // residual operand laid out like y, or null
     const float* bias;
     int* status;
     int N, Ho, Wo, Cin, Cout;    // output image size
@@ -302,13 +304,42 @@ __device__ __forceinline__ float bias_act(unsigned acc_bits, float bs) {
 // Where a position goes comes from the table built in the prologue (no division here): tab[p] = {element offset
 // inside the tile, row << 16 | column}.  patch and tab are shared-memory addresses (32 bits: the accesses are
 // spelled out so that none is compiled as a generic one).
+// Eight outputs of one position (four words of two 16-bit values, already rounded without activation) plus the eight
+// residual values at the same place: sum in fp32, activation, one more rounding -- what a convolution without
+// activation followed by an element-wise add + activation gives, bit for bit.
+template <typename T, int ACT>
+__device__ __forceinline__ uint4 add_residual8(uint4 o, const uint4 rv) {
+    const T* oe = reinterpret_cast<const T*>(&o);
+    const T* re = reinterpret_cast<const T*>(&rv);
+    unsigned w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float v[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            v[e] = to_f32<T>(oe[2 * i + e]) + to_f32<T>(re[2 * i + e]);
+            if (ACT == RTOSS_ACT_SILU) {
+                const float h = 0.5f * v[e];
+                float th;
+                asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(h));
+                v[e] = fmaf(h, th, h);
+            }
+        }
+        w[i] = round_pack<T, ACT == RTOSS_ACT_RELU>(v[0], v[1]);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
 // Sixteen positions of one filter (a half chunk): round, transpose through the patch, store.  See epilogue_chunks.
+// With a residual operand (rbv, laid out like the output) the activation moves behind the residual add.
 template <typename T, int ACT>
 __device__ __forceinline__ void epilogue_half(const unsigned (&r)[16], float bs, unsigned wr, unsigned rd, unsigned tab_at,
-                                              T* ybv, unsigned ry, unsigned rx) {
+                                              T* ybv, unsigned ry, unsigned rx, const T* rbv = nullptr) {
+    const bool res = rbv != nullptr;   // then bs is the plain bias and nothing is activated before the add
 #pragma unroll
     for (int jp = 0; jp < kPatchRows / 2; ++jp) {
-        const unsigned w = round_pack<T, ACT == RTOSS_ACT_RELU>(bias_act<ACT>(r[2 * jp], bs), bias_act<ACT>(r[2 * jp + 1], bs));
+        const unsigned w = res ? round_pack<T, false>(__uint_as_float(r[2 * jp]) + bs, __uint_as_float(r[2 * jp + 1]) + bs)
+                               : round_pack<T, ACT == RTOSS_ACT_RELU>(bias_act<ACT>(r[2 * jp], bs), bias_act<ACT>(r[2 * jp + 1], bs));
         asm volatile("st.shared.u32 [%0], %1;" ::"r"(wr + jp * kPairPitch), "r"(w) : "memory");
     }
     __syncwarp();
@@ -317,12 +348,18 @@ __device__ __forceinline__ void epilogue_half(const unsigned (&r)[16], float bs,
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "r"(rd + 16));
     // table entries of positions 2 jp and 2 jp + 1 (an even position: 16-byte aligned)
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(e[0]), "=r"(e[1]), "=r"(e[2]), "=r"(e[3]) : "r"(tab_at));
-    if ((e[1] >> 16) < ry && (e[1] & 0xFFFFu) < rx)
-        *reinterpret_cast<uint4*>(ybv + e[0]) = make_uint4(__byte_perm(w[0], w[1], 0x5410), __byte_perm(w[2], w[3], 0x5410),
-                                                           __byte_perm(w[4], w[5], 0x5410), __byte_perm(w[6], w[7], 0x5410));
-    if ((e[3] >> 16) < ry && (e[3] & 0xFFFFu) < rx)
-        *reinterpret_cast<uint4*>(ybv + e[2]) = make_uint4(__byte_perm(w[0], w[1], 0x7632), __byte_perm(w[2], w[3], 0x7632),
-                                                           __byte_perm(w[4], w[5], 0x7632), __byte_perm(w[6], w[7], 0x7632));
+    if ((e[1] >> 16) < ry && (e[1] & 0xFFFFu) < rx) {
+        uint4 o = make_uint4(__byte_perm(w[0], w[1], 0x5410), __byte_perm(w[2], w[3], 0x5410), __byte_perm(w[4], w[5], 0x5410),
+                             __byte_perm(w[6], w[7], 0x5410));
+        if (res) o = add_residual8<T, ACT>(o, *reinterpret_cast<const uint4*>(rbv + e[0]));
+        *reinterpret_cast<uint4*>(ybv + e[0]) = o;
+    }
+    if ((e[3] >> 16) < ry && (e[3] & 0xFFFFu) < rx) {
+        uint4 o = make_uint4(__byte_perm(w[0], w[1], 0x7632), __byte_perm(w[2], w[3], 0x7632), __byte_perm(w[4], w[5], 0x7632),
+                             __byte_perm(w[6], w[7], 0x7632));
+        if (res) o = add_residual8<T, ACT>(o, *reinterpret_cast<const uint4*>(rbv + e[2]));
+        *reinterpret_cast<uint4*>(ybv + e[2]) = o;
+    }
     __syncwarp();
 }
 
@@ -344,22 +381,103 @@ __device__ __forceinline__ void epilogue_half(const unsigned (&r)[16], float bs,
 template <typename T, int ACT>
 __device__ __forceinline__ void epilogue_chunks(unsigned d_base, int c0, int c_step, int n_px, float bs,
                                                 unsigned patch, unsigned tab, T* yb, unsigned ry, unsigned rx,
-                                                int lane) {
+                                                int lane, const T* rb) {
     const unsigned wr = patch + lane * 4;                                       // this lane's column of the patch
     const unsigned rd = patch + (lane >> 2) * kPairPitch + (lane & 3) * 32;   // row lane / 4, filter group lane % 4
     const unsigned tab_l = tab + (unsigned)(2 * (lane >> 2)) * 8;
     T* ybv = yb + (lane & 3) * 8;
+    const T* rbv = rb ? rb + (lane & 3) * 8 : nullptr;
     if (c0 >= n_px) return;
-    unsigned ra[16], rb[16];
+    unsigned ra[16], rb2[16];
     tmem_ld16(d_base + (unsigned)c0, ra);
     for (; c0 < n_px; c0 += c_step) {
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        tmem_ld16(d_base + (unsigned)(c0 + kPatchRows), rb);
-        epilogue_half<T, ACT>(ra, bs, wr, rd, tab_l + (unsigned)c0 * 8, ybv, ry, rx);
+        tmem_ld16(d_base + (unsigned)(c0 + kPatchRows), rb2);
+        epilogue_half<T, ACT>(ra, bs, wr, rd, tab_l + (unsigned)c0 * 8, ybv, ry, rx, rbv);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         if (c0 + c_step < n_px) tmem_ld16(d_base + (unsigned)(c0 + c_step), ra);
-        epilogue_half<T, ACT>(rb, bs, wr, rd, tab_l + (unsigned)(c0 + kPatchRows) * 8, ybv, ry, rx);
+        epilogue_half<T, ACT>(rb2, bs, wr, rd, tab_l + (unsigned)(c0 + kPatchRows) * 8, ybv, ry, rx, rbv);
     }
+}
+
+// The same with a residual operand.  Its values arrive by asynchronous 16-byte copies (global -> shared, no
+// registers held while they fly): every lane fetches the two pieces it will add (positions 2 jp and 2 jp + 1, its
+// eight filters) into its own slots of the warp's staging area, one half chunk ahead of the one being finished, so a
+// load from memory has a whole half chunk of work to hide behind.  A lane reads back only what it fetched itself:
+// cp.async.wait_group is all the ordering needed.  stage: shared address of the warp's kResStage bytes, two buffers
+// of [2 pieces][32 lanes] x 16 bytes.
+template <typename T>
+__device__ __forceinline__ void fetch_residual(unsigned tab_at, const T* rbv, unsigned ry, unsigned rx, unsigned slot) {
+    unsigned e[4];
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(e[0]), "=r"(e[1]), "=r"(e[2]), "=r"(e[3]) : "r"(tab_at));
+    if ((e[1] >> 16) < ry && (e[1] & 0xFFFFu) < rx)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot), "l"(rbv + e[0]) : "memory");
+    if ((e[3] >> 16) < ry && (e[3] & 0xFFFFu) < rx)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot + 512u), "l"(rbv + e[2]) : "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+template <typename T, int ACT>
+__device__ __forceinline__ void epilogue_half_res(const unsigned (&r)[16], float bias, unsigned wr, unsigned rd, unsigned tab_at,
+                                                  T* ybv, unsigned ry, unsigned rx, unsigned slot) {
+#pragma unroll
+    for (int jp = 0; jp < kPatchRows / 2; ++jp) {
+        const unsigned w = round_pack<T, false>(__uint_as_float(r[2 * jp]) + bias, __uint_as_float(r[2 * jp + 1]) + bias);
+        asm volatile("st.shared.u32 [%0], %1;" ::"r"(wr + jp * kPairPitch), "r"(w) : "memory");
+    }
+    __syncwarp();
+    unsigned w[8], e[4];
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(rd));
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "r"(rd + 16));
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(e[0]), "=r"(e[1]), "=r"(e[2]), "=r"(e[3]) : "r"(tab_at));
+    if ((e[1] >> 16) < ry && (e[1] & 0xFFFFu) < rx) {
+        uint4 rv;
+        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(rv.x), "=r"(rv.y), "=r"(rv.z), "=r"(rv.w) : "r"(slot));
+        const uint4 o = make_uint4(__byte_perm(w[0], w[1], 0x5410), __byte_perm(w[2], w[3], 0x5410),
+                                   __byte_perm(w[4], w[5], 0x5410), __byte_perm(w[6], w[7], 0x5410));
+        *reinterpret_cast<uint4*>(ybv + e[0]) = add_residual8<T, ACT>(o, rv);
+    }
+    if ((e[3] >> 16) < ry && (e[3] & 0xFFFFu) < rx) {
+        uint4 rv;
+        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(rv.x), "=r"(rv.y), "=r"(rv.z), "=r"(rv.w) : "r"(slot + 512u));
+        const uint4 o = make_uint4(__byte_perm(w[0], w[1], 0x7632), __byte_perm(w[2], w[3], 0x7632),
+                                   __byte_perm(w[4], w[5], 0x7632), __byte_perm(w[6], w[7], 0x7632));
+        *reinterpret_cast<uint4*>(ybv + e[2]) = add_residual8<T, ACT>(o, rv);
+    }
+    __syncwarp();
+}
+
+template <typename T, int ACT>
+__device__ __forceinline__ void epilogue_chunks_res(unsigned d_base, int c0, int c_step, int n_px, float bias,
+                                                    unsigned patch, unsigned tab, T* yb, unsigned ry, unsigned rx,
+                                                    int lane, const T* rb, unsigned stage) {
+    const unsigned wr = patch + lane * 4;
+    const unsigned rd = patch + (lane >> 2) * kPairPitch + (lane & 3) * 32;
+    const unsigned tab_l = tab + (unsigned)(2 * (lane >> 2)) * 8;
+    T* ybv = yb + (lane & 3) * 8;
+    const T* rbv = rb + (lane & 3) * 8;
+    if (c0 >= n_px) return;
+    const unsigned slot0 = stage + (unsigned)lane * 16, slot1 = slot0 + 1024u;
+    unsigned ra[16], rb2[16];
+    fetch_residual<T>(tab_l + (unsigned)c0 * 8, rbv, ry, rx, slot0);
+    tmem_ld16(d_base + (unsigned)c0, ra);
+    for (; c0 < n_px; c0 += c_step) {
+        fetch_residual<T>(tab_l + (unsigned)(c0 + kPatchRows) * 8, rbv, ry, rx, slot1);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        tmem_ld16(d_base + (unsigned)(c0 + kPatchRows), rb2);
+        asm volatile("cp.async.wait_group 1;" ::: "memory");   // the pieces of this half are in
+        epilogue_half_res<T, ACT>(ra, bias, wr, rd, tab_l + (unsigned)c0 * 8, ybv, ry, rx, slot0);
+        const bool more = c0 + c_step < n_px;
+        if (more)
+            fetch_residual<T>(tab_l + (unsigned)(c0 + c_step) * 8, rbv, ry, rx, slot0);
+        else
+            asm volatile("cp.async.commit_group;" ::: "memory");   // keeps the group count in step
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (more) tmem_ld16(d_base + (unsigned)(c0 + c_step), ra);
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
+        epilogue_half_res<T, ACT>(rb2, bias, wr, rd, tab_l + (unsigned)(c0 + kPatchRows) * 8, ybv, ry, rx, slot1);
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
 // Split K, second half.  Every CTA of the cluster owns the 32-column chunks c of the tile with c % KS == its rank
@@ -369,11 +487,12 @@ __device__ __forceinline__ void epilogue_chunks(unsigned d_base, int c0, int c_s
 template <typename T, int ACT>
 __device__ __forceinline__ void epilogue_from_shares(unsigned buf, int KS, int rank, int n_lc, int sub, int row, int n_px, float bs,
                                                      bool vec_ok, bool co_ok, unsigned patch, unsigned tab, const uint2* pos_tab,
-                                                     T* yb, unsigned ry, unsigned rx, int lane) {
+                                                     T* yb, unsigned ry, unsigned rx, int lane, const T* rb) {
     const unsigned wr = patch + lane * 4;
     const unsigned rd = patch + (lane >> 2) * kPairPitch + (lane & 3) * 32;
     const unsigned tab_l = tab + (unsigned)(2 * (lane >> 2)) * 8;
     T* ybv = yb + (lane & 3) * 8;
+    const T* rbv = rb ? rb + (lane & 3) * 8 : nullptr;
     for (int t = sub; t < 2 * n_lc; t += 4) {
         const int lc = t >> 1, c0 = (lc * KS + rank) * 32 + (t & 1) * kPatchRows;   // first column of the half chunk
         if (c0 >= n_px) continue;
@@ -393,14 +512,27 @@ __device__ __forceinline__ void epilogue_from_shares(unsigned buf, int KS, int r
 #pragma unroll
         for (int j = 0; j < kPatchRows; ++j) r[j] = __float_as_uint(sum[j]);
         if (vec_ok) {
-            epilogue_half<T, ACT>(r, bs, wr, rd, tab_l + (unsigned)c0 * 8, ybv, ry, rx);
+            epilogue_half<T, ACT>(r, bs, wr, rd, tab_l + (unsigned)c0 * 8, ybv, ry, rx, rbv);
         } else {
 #pragma unroll
             for (int j = 0; j < kPatchRows; ++j) {
                 const uint2 e = pos_tab[c0 + j];
-                float v = bias_act<ACT>(r[j], bs);
-                if (ACT == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
-                if (co_ok && (e.y >> 16) < ry && (e.y & 0xFFFFu) < rx) yb[e.x + lane] = from_f32<T>(v);
+                if (co_ok && (e.y >> 16) < ry && (e.y & 0xFFFFu) < rx) {
+                    float v;
+                    if (rb) {   // round, add the residual, activate, round
+                        v = to_f32<T>(from_f32<T>(__uint_as_float(r[j]) + bs)) + to_f32<T>(rb[e.x + lane]);
+                        if (ACT == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
+                        if (ACT == RTOSS_ACT_SILU) {
+                            float th;
+                            asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(0.5f * v));
+                            v = fmaf(0.5f * v, th, 0.5f * v);
+                        }
+                    } else {
+                        v = bias_act<ACT>(r[j], bs);
+                        if (ACT == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
+                    }
+                    yb[e.x + lane] = from_f32<T>(v);
+                }
             }
         }
     }
@@ -423,6 +555,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     unsigned char* epi_patch = smem_dyn + (s_tmem_ptr + 16 - smem_u32(smem_dyn));  // [kEpiWarps][kPatchBytes], 16-byte aligned
     uint2* pos_tab = reinterpret_cast<uint2*>(epi_patch + kEpiWarps * kPatchBytes);  // [kMaxPx]
     const unsigned s_tab = s_tmem_ptr + 16 + kEpiWarps * kPatchBytes;                // the same, as a shared address
+    const unsigned s_res = s_tab + kMaxPx * 8;   // [kEpiWarps][kResStage], present when the call has a residual operand
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = a.N * a.tiles_y * a.tiles_x * a.co_tiles * a.KS;  // units of work: (tile, share of the channel blocks)
@@ -731,7 +864,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             T* yb = yg + (((size_t)n * a.Ho + y0) * a.Wo + x0) * a.y_c_stride + a.y_c_off + co0 + row0;
             const unsigned ry = (unsigned)min(a.TH, a.Ho - y0), rx = (unsigned)min(a.TW, a.Wo - x0);  // rows / columns inside the image
             const int c_first = (sub + 4 * copy) * 32, c_step = 128 * a.R;
-            const float bs = a.act == RTOSS_ACT_SILU ? 0.5f * bv : bv;
+            const T* rb = a.resid ? reinterpret_cast<const T*>(a.resid) + (yb - yg) : nullptr;   // laid out like y
+            const float bs = (a.act == RTOSS_ACT_SILU && !rb) ? 0.5f * bv : bv;   // (with a residual the bias is added plain)
             ok = mbar_wait(bar_accFull + 8 * as, (gt / a.AS) & 1);
             if (!ok && a.KS == 1) break;   // (split K: the cluster barriers below must still be passed)
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -761,21 +895,29 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (ok) {
                     const int row = quarter * 32 + lane;
                     if (a.act == RTOSS_ACT_SILU)
-                        epilogue_from_shares<T, RTOSS_ACT_SILU>(sA, a.KS, rank, n_lc, sub, row, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
+                        epilogue_from_shares<T, RTOSS_ACT_SILU>(sA, a.KS, rank, n_lc, sub, row, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane, rb);
                     else if (a.act == RTOSS_ACT_RELU)
-                        epilogue_from_shares<T, RTOSS_ACT_RELU>(sA, a.KS, rank, n_lc, sub, row, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
+                        epilogue_from_shares<T, RTOSS_ACT_RELU>(sA, a.KS, rank, n_lc, sub, row, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane, rb);
                     else
-                        epilogue_from_shares<T, RTOSS_ACT_NONE>(sA, a.KS, rank, n_lc, sub, row, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane);
+                        epilogue_from_shares<T, RTOSS_ACT_NONE>(sA, a.KS, rank, n_lc, sub, row, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane, rb);
                 }
                 continue;
             }
             if (vec_ok) {
-                if (a.act == RTOSS_ACT_SILU)
-                    epilogue_chunks<T, RTOSS_ACT_SILU>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane);
+                if (rb) {
+                    const unsigned stage = s_res + (unsigned)(warp - 2) * kResStage;
+                    if (a.act == RTOSS_ACT_SILU)
+                        epilogue_chunks_res<T, RTOSS_ACT_SILU>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb, stage);
+                    else if (a.act == RTOSS_ACT_RELU)
+                        epilogue_chunks_res<T, RTOSS_ACT_RELU>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb, stage);
+                    else
+                        epilogue_chunks_res<T, RTOSS_ACT_NONE>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb, stage);
+                } else if (a.act == RTOSS_ACT_SILU)
+                    epilogue_chunks<T, RTOSS_ACT_SILU>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb);
                 else if (a.act == RTOSS_ACT_RELU)
-                    epilogue_chunks<T, RTOSS_ACT_RELU>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane);
+                    epilogue_chunks<T, RTOSS_ACT_RELU>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb);
                 else
-                    epilogue_chunks<T, RTOSS_ACT_NONE>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane);
+                    epilogue_chunks<T, RTOSS_ACT_NONE>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb);
             } else {
                 // ragged filter counts or unaligned channel slices: element stores, lane = filter
                 for (int c0 = c_first; c0 < a.N_px; c0 += c_step) {
@@ -785,7 +927,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         const uint2 e = pos_tab[c0 + j];
+                        const bool in_img = co_ok && (e.y >> 16) < ry && (e.y & 0xFFFFu) < rx;
                         float v = __uint_as_float(r[j]) + bv;
+                        if (rb && in_img) v = to_f32<T>(from_f32<T>(v)) + to_f32<T>(rb[e.x + lane]);   // round, then add the residual
                         if (a.act == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
                         if (a.act == RTOSS_ACT_SILU) {
                             float th;
@@ -853,11 +997,12 @@ struct TcPlan {
 //                 the even rows for r = 1, one staged row further down for r = 1, 2; columns alike.
 // The plan picks TH, the column segment TW (images wider than a TMA box are cut into segments), the
 // ring depths, and how many taps share a weight stage.
-bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count, bool pxm, int w_rows, TcPlan* out) {
+bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count, bool pxm, int w_rows, bool resid, TcPlan* out) {
     const int halo = ksize == 3 ? (S == 1 ? 2 : 1) : 0;
     const int n_sub = (ksize == 3 && S == 2) ? 4 : 1;
     const int max_pitch = S == 1 ? 256 : 128;  // TMA box: at most 256 elements traversed per dimension
-    const int fixed = 1024 /*alignment slack*/ + 512 /*barriers*/ + kEpiWarps * kPatchBytes /*epilogue patches*/ + kMaxPx * 8 /*position table*/;
+    const int fixed = 1024 /*alignment slack*/ + 512 /*barriers*/ + kEpiWarps * kPatchBytes /*epilogue patches*/ + kMaxPx * 8 /*position table*/ +
+                      (resid ? kEpiWarps * kResStage : 0) /*staging of the residual operand*/;
     const int cap = 227 * 1024 - 64;
     double best = -1;
     for (int nseg = 1; nseg <= 16; ++nseg) {
@@ -927,11 +1072,13 @@ bool rtoss_tc_eligible(const rtoss_packed* p, const rtoss_conv_desc* d, const vo
     if (d->layout != RTOSS_NHWC || (int)d->io_dtype != (int)p->dtype) return false;
     if ((reinterpret_cast<uintptr_t>(x) & 15) || (reinterpret_cast<uintptr_t>(y) & 15)) return false;
     if (!encode_fn()) return false;
+    // a residual operand: 16-byte aligned, and not for the positions-as-M form (narrow 1x1 layers)
+    if (d->residual_dev && (use_pxm(p) || (reinterpret_cast<uintptr_t>(d->residual_dev) & 15))) return false;
     const int Ho = (d->H - 1) / d->stride + 1, Wo = (d->W - 1) / d->stride + 1;
     TcPlan plan;
     const bool pxm = use_pxm(p);
     return plan_tc(d->N, Ho, Wo, p->ksize, d->stride, (p->Cout + kMTile - 1) / kMTile, 148, pxm, pxm ? round_up(p->Cout, 16) : kMTile,
-                   &plan);
+                   d->residual_dev != nullptr, &plan);
 }
 
 int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y, const rtoss_conv_desc* d,
@@ -945,11 +1092,12 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     // narrow layers put the positions on the M operand (all 128 TMEM lanes carry outputs whatever Cout is)
     const bool pxm = use_pxm(p);
     const int w_rows = pxm ? round_up(p->Cout, 16) : kMTile;
-    if (!plan_tc(d->N, Ho, Wo, p->ksize, S, (p->Cout + kMTile - 1) / kMTile, sms, pxm, w_rows, &plan))
+    if (!plan_tc(d->N, Ho, Wo, p->ksize, S, (p->Cout + kMTile - 1) / kMTile, sms, pxm, w_rows, d->residual_dev != nullptr, &plan))
         return (int)cudaErrorInvalidConfiguration;
 
     TcArgs a;
     a.y = y;
+    a.resid = d->residual_dev;
     a.bias = d->bias_dev;
     a.status = ctx->dev_status;
     a.N = d->N;

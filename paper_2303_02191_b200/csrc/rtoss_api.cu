@@ -86,6 +86,11 @@ int dispatch_conv(rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y,
                   rtoss_status* st) {
     *st = RTOSS_OK;
     const bool tc_ok = d->path != RTOSS_PATH_FMA && rtoss_tc_eligible(p, d, x, y);
+    if (d->residual_dev && !tc_ok) {
+        set_err(ctx, "conv", "a residual operand is only taken by the tensor path (see rtoss.h)");
+        *st = RTOSS_ERR_UNSUPPORTED;
+        return 0;
+    }
     if (d->path == RTOSS_PATH_TENSOR && !tc_ok) {
         set_err(ctx, "conv", "the tensor path does not take this call (see rtoss.h for its conditions)");
         *st = RTOSS_ERR_UNSUPPORTED;
@@ -385,6 +390,10 @@ rtoss_status rtoss_conv_pattern_host(rtoss_ctx* ctx, const rtoss_packed* p, cons
     if (!ctx || !p) return RTOSS_ERR_INVALID_ARG;
     rtoss_status st = check_conv(ctx, p, x_host, y_host, desc, p->ksize, false);
     if (st != RTOSS_OK) return st;
+    if (desc->residual_dev) {
+        set_err(ctx, "conv", "the host-buffer entry point takes no residual operand");
+        return RTOSS_ERR_UNSUPPORTED;
+    }
     cudaSetDevice(ctx->device);
     const size_t es = rtoss_dtype_size(desc->io_dtype);
     const int Ho = (desc->H - 1) / desc->stride + 1, Wo = (desc->W - 1) / desc->stride + 1;

@@ -84,14 +84,45 @@ def program(H0, W0):
     return ops, bufs, layers, tuple(outputs)
 
 
+def fuse_adds(ops, outputs):
+    """Every 'add' one of whose operands comes from a convolution without activation and is read by nothing else
+    becomes ('convres', layer_index, src, tmp, other, dst, act) at the add's place: the convolution moves there (each
+    buffer of the program is written once, so moving a producer later changes nothing) and adds the other operand in
+    its epilogue.  tmp is the buffer the convolution would have written, used when the fused call is declined."""
+    reads = {}
+    for op in ops:
+        srcs = (op[2],) if op[0] == "conv" else (op[1], op[2]) if op[0] == "add" else (op[1],)
+        for s_ in srcs:
+            reads[s_] = reads.get(s_, 0) + 1
+    for name in outputs:
+        reads[name] = reads.get(name, 0) + 1
+    producer = {op[3]: j for j, op in enumerate(ops) if op[0] == "conv" and op[4] == "none"}
+    moved, out = {}, []
+    for j, op in enumerate(ops):
+        if op[0] == "add":
+            for tmp, other in ((op[1], op[2]), (op[2], op[1])):
+                if tmp in producer and reads[tmp] == 1 and tmp != other:
+                    moved[producer[tmp]] = ("convres", ops[producer[tmp]][1], ops[producer[tmp]][2], tmp, other, op[3], op[4])
+                    break
+    by_add = {v[5]: v for v in moved.values()}
+    for j, op in enumerate(ops):
+        if j in moved:
+            continue
+        out.append(by_add[op[3]] if op[0] == "add" and op[3] in by_add else op)
+    return out
+
+
 class GpuNet:
     """The program on the GPU through the C-ABI library: NHWC, bf16 (or fp16), k-entry patterns."""
 
-    def __init__(self, ctx, N, H0=800, W0=1088, k=4, seed=0, dtype="bf16"):
+    def __init__(self, ctx, N, H0=800, W0=1088, k=4, seed=0, dtype="bf16", fuse_residual=True):
         import torch
         from . import binding as rt
         self.rt, self.ctx, self.N, self.torch = rt, ctx, N, torch
         self.ops, self.bufs, self.layers, self.output_names = program(H0, W0)
+        if fuse_residual:
+            self.ops = fuse_adds(self.ops, self.output_names)
+        self.unfused = set()   # layers whose fused call the library declined: convolution and add run separately
         tdt = {"bf16": torch.bfloat16, "f16": torch.float16}[dtype]
         self.t = {n: torch.zeros((N, H, W, C), dtype=tdt, device="cuda") for n, (C, H, W) in self.bufs.items()}
         self.zero = {}   # all-zero operands of the ReLU glue op, one per shape
@@ -122,6 +153,21 @@ class GpuNet:
                 fn = self.ctx.rtoss_conv3x3_pattern if L["ksize"] == 3 else self.ctx.rtoss_conv1x1_pattern
                 fn(self.packed[L["wid"]], t[src], t[dst], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_NAMES[act],
                    self.bias[L["wid"]])
+            elif op[0] == "convres":   # convolution (no activation) + residual + activation in one call
+                _, i, src, tmp, other, dst, act = op
+                L = self.layers[i]
+                fn = self.ctx.rtoss_conv3x3_pattern if L["ksize"] == 3 else self.ctx.rtoss_conv1x1_pattern
+                args = (self.packed[L["wid"]], t[src], None, N, L["H"], L["W"], L["stride"], rt.NHWC)
+                if i not in self.unfused:
+                    try:
+                        fn(*args[:2], t[dst], *args[3:], rt.ACT_NAMES[act], self.bias[L["wid"]], residual=t[other])
+                        continue
+                    except rt.RtossError as err:
+                        if err.status != rt.ERR_UNSUPPORTED:
+                            raise
+                        self.unfused.add(i)
+                fn(*args[:2], t[tmp], *args[3:], rt.ACT_NONE, self.bias[L["wid"]])
+                rt.rtoss_add_act(t[tmp], t[other], t[dst], rt.ACT_NAMES[act])
             elif op[0] == "add":
                 rt.rtoss_add_act(t[op[1]], t[op[2]], t[op[3]], rt.ACT_NAMES[op[4]])
             elif op[0] == "up":

@@ -104,3 +104,30 @@ def test_create_fails_loudly_without_a_device(rt):
         pytest.skip("a CUDA device is present")
     with pytest.raises(rt.RtossError):
         rt.Context(0)
+
+
+def test_retinanet_program_add_fusion_keeps_a_valid_order():
+    """Host logic of the chained RetinaNet-shaped runner: every add fed by an activation-free convolution that
+    nothing else reads is folded into that convolution (16 block ends, 2 pyramid sums), each buffer is still
+    written before it is read, and the same buffers are produced."""
+    from paper_2303_02191_b200 import retinanet_net as rn
+    ops, bufs, layers, outs = rn.program(800, 1088)
+    fused = rn.fuse_adds(ops, outs)
+    assert sum(op[0] == "add" for op in ops) == 18
+    assert sum(op[0] == "convres" for op in fused) == 18 and not any(op[0] == "add" for op in fused)
+    assert len(fused) == len(ops) - 18
+    assert sorted(op[1] for op in fused if op[0] in ("conv", "convres")) == list(range(100))
+    written = {"in"}
+    for op in fused:
+        srcs = op[2:3] if op[0] == "conv" else (op[2], op[4]) if op[0] == "convres" else op[1:2]
+        dst = op[3] if op[0] == "conv" else op[5] if op[0] == "convres" else op[2]
+        assert all(s in written for s in srcs), op
+        assert dst not in written
+        written.add(dst)
+        if op[0] == "convres":
+            assert bufs[op[3]] == bufs[op[4]] == bufs[op[5]]
+            assert op[3] not in written
+    assert all(o in written for o in outs)
+    original = {op[3] if op[0] in ("conv", "add") else op[2] for op in ops}
+    skipped = {op[3] for op in fused if op[0] == "convres"}
+    assert written - {"in"} == original - skipped
