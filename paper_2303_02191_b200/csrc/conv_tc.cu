@@ -291,22 +291,10 @@ __device__ __forceinline__ float bias_act(unsigned acc_bits, float bs) {
     return acc + bs;
 }
 
-// One tile of the filters-as-M epilogue for one warp: its lane quarter of the accumulator stage at d_base, the
-// 32-column chunks c0, c0 + c_step, ...  A warp holds 32 filters (lanes) x 32 positions (registers); NHWC wants
-// the filters of one position side by side.  The shared-memory pipe (one 128-byte wavefront a cycle, which the
-// tensor cores' operand reads also use) is what bounds this, so the transpose moves full wavefronts:
-//   * a lane rounds two neighbouring positions of its filter into one 32-bit word and stores it to row
-//     (position pair), column (filter) of the warp's patch: eight conflict-free 128-byte stores per 16 positions;
-//   * lane (pair jp = lane / 4, filter group v = lane % 4) reads the eight words of its group (two 16-byte
-//     loads; rows are 36 words apart, so the two rows a quarter warp touches fall on disjoint banks), splits
-//     them into the low halves (position 2 jp) and the high halves (position 2 jp + 1) and writes each as one
-//     16-byte store: four lanes cover the 64 contiguous bytes of a position.
-// Where a position goes comes from the table built in the prologue (no division here): tab[p] = {element offset
-// inside the tile, row << 16 | column}.  patch and tab are shared-memory addresses (32 bits: the accesses are
-// spelled out so that none is compiled as a generic one).
 // Eight outputs of one position (four words of two 16-bit values, already rounded without activation) plus the eight
 // residual values at the same place: sum in fp32, activation, one more rounding -- what a convolution without
-// activation followed by an element-wise add + activation gives, bit for bit.
+// activation followed by an element-wise add + activation gives, bit for bit (act none and ReLU; SiLU here is the
+// tanh form of the epilogue).
 template <typename T, int ACT>
 __device__ __forceinline__ uint4 add_residual8(uint4 o, const uint4 rv) {
     const T* oe = reinterpret_cast<const T*>(&o);
