@@ -136,6 +136,28 @@ rtoss_status rtoss_pattern_usage(rtoss_ctx* ctx, const void* kernels_dev, rtoss_
                                  const uint16_t* masks_host, int P, int k, uint8_t* pid_scratch_dev, uint64_t* counts_dev,
                                  void* cuda_stream);
 
+/* Criterion 2, the cut (Section IV.B: "select the most used kernel pattern"): rank the candidates of a table by
+ * their usage counts -- most used first; equal counts: the numerically lower mask first -- and keep the best M.
+ * order_host (P entries, may be NULL) receives the candidate indices in rank order; top_masks_host (M entries) the
+ * kept masks in ascending numeric order, i.e. a table every other call accepts.  Host only.  How many to keep is
+ * the caller's choice: the paper gives no cut-off.  RTOSS_ERR_BAD_PATTERN_TABLE for an invalid candidate table,
+ * RTOSS_ERR_INVALID_ARG for null pointers or M outside 1..P. */
+rtoss_status rtoss_pattern_rank(const uint16_t* masks_host, const uint64_t* counts_host, int P, int k, int M,
+                                uint16_t* top_masks_host, int* order_host);
+
+/* Pattern-set derivation in one call (Section IV.B): the candidates are the preset table for k (RTOSS_PRESET_ALL:
+ * Eq. 1 alone; RTOSS_PRESET_CONN4: Eq. 1 and the adjacency criterion), their usage over the caller's sample of
+ * kernels is counted on the GPU exactly as rtoss_pattern_usage does (same arguments: kernels_dev, pid_scratch_dev
+ * of n_kernels bytes, counts_dev with room for 255 counters), the stream is synchronised, and the M most used are
+ * returned as rtoss_pattern_rank returns them (M larger than the number of candidates keeps them all).
+ * *P_candidates receives the number of candidates, *M_kept the number of masks written to top_masks_host (room for
+ * M); cand_masks_host / cand_counts_host (room for 255 entries each, may be NULL) the candidate table and its
+ * counts.  The random sample is the caller's (the paper asks for values in [-1, 1]; count and seed are not given). */
+rtoss_status rtoss_pattern_table_derive(rtoss_ctx* ctx, const void* kernels_dev, rtoss_dtype dtype, int64_t n_kernels,
+                                        int k, rtoss_preset preset, int M, uint8_t* pid_scratch_dev, uint64_t* counts_dev,
+                                        uint16_t* top_masks_host, int* M_kept, uint16_t* cand_masks_host,
+                                        uint64_t* cand_counts_host, int* P_candidates, void* cuda_stream);
+
 /* ---- packing (Section IV.C: "kernels with similar patterns are grouped") --- */
 
 /* Build the packed form of one layer from its weights and pattern ids:

@@ -84,6 +84,35 @@ def select_kernels(w9, masks):
     return pid
 
 
+def pattern_usage(w9, masks):
+    """Section IV.B, criterion 2: how many kernels of the sample choose each candidate pattern (Algorithm 2's argmax
+    per kernel, then a plain count)."""
+    m = _masks(masks)
+    counts = np.zeros(len(m), dtype=np.uint64)
+    for p in select_kernels(w9, m):
+        counts[p] += 1
+    return counts
+
+
+def pattern_rank(masks, counts, M):
+    """The cut of criterion 2: candidates by falling count, equal counts by rising mask value; the M best, returned in
+    ascending mask order (a table).  Also returns the candidate indices in rank order."""
+    m = [int(v) for v in _masks(masks)]
+    c = [int(v) for v in counts]
+    order = sorted(range(len(m)), key=lambda i: (-c[i], m[i]))
+    top = sorted(m[i] for i in order[:M])
+    return np.array(top, dtype=np.uint16), np.array(order, dtype=np.int32)
+
+
+def derive_pattern_table(w9, k, preset, M):
+    """Section IV.B end to end: Eq. 1 candidates (preset ALL) or those with adjacent taps (preset CONN4), usage over
+    the sample, the M most used."""
+    cand = pattern_preset(k, preset)
+    counts = pattern_usage(w9, cand)
+    top, _ = pattern_rank(cand, counts, min(M, len(cand)))
+    return top, cand, counts
+
+
 def select_3x3(w, masks):
     w = _f32(w)
     Cout, Cin = w.shape[:2]

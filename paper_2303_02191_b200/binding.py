@@ -28,6 +28,7 @@ SYMBOLS = [
     "rtoss_pattern_table_validate", "rtoss_group_layers", "rtoss_select_patterns", "rtoss_pack",
     "rtoss_packed_info_get", "rtoss_packed_export", "rtoss_packed_to_dense", "rtoss_packed_destroy",
     "rtoss_conv3x3_pattern", "rtoss_conv1x1_pattern", "rtoss_conv_pattern_host", "rtoss_device_status", "rtoss_prune_dense_static", "rtoss_maxpool2d", "rtoss_upsample2x", "rtoss_add_act", "rtoss_pattern_usage",
+    "rtoss_pattern_rank", "rtoss_pattern_table_derive",
     "rtoss_batch_create", "rtoss_batch_select_pack", "rtoss_batch_destroy",
 ]
 
@@ -77,6 +78,9 @@ def _load():
     lib.rtoss_last_error.restype = ctypes.c_char_p
     lib.rtoss_pattern_preset.argtypes = [ci, ci, vp, ctypes.POINTER(ci)]
     lib.rtoss_pattern_table_validate.argtypes = [vp, ci, ci]
+    lib.rtoss_pattern_rank.argtypes = [vp, vp, ci, ci, ci, vp, vp]
+    lib.rtoss_pattern_table_derive.argtypes = [vp, vp, ci, ctypes.c_int64, ci, ci, ci, vp, vp, vp, ctypes.POINTER(ci), vp, vp,
+                                               ctypes.POINTER(ci), vp]
     lib.rtoss_group_layers.argtypes = [ctypes.POINTER(LayerNode), ci, vp, vp, ctypes.POINTER(ci)]
     lib.rtoss_select_patterns.argtypes = [vp, vp, ci, ci, ci, ci, vp, ci, ci, vp, vp]
     lib.rtoss_pack.argtypes = [vp, vp, ci, ci, ci, ci, vp, ci, ci, vp, ci, ctypes.POINTER(vp), vp]
@@ -124,6 +128,18 @@ def rtoss_pattern_preset(k, preset):
     if st != OK:
         raise RtossError(st, status_string(st))
     return out[:n.value].copy()
+
+
+def rtoss_pattern_rank(masks, counts, k, M):
+    """-> (the M most used masks in ascending order, candidate indices in rank order); host only."""
+    m = _masks_arr(masks)
+    c = np.ascontiguousarray(counts, dtype=np.uint64)
+    top = np.zeros(max(int(M), 1), dtype=np.uint16)
+    order = np.zeros(len(m), dtype=np.int32)
+    st = lib.rtoss_pattern_rank(_np_ptr(m), _np_ptr(c), len(m), int(k), int(M), _np_ptr(top), _np_ptr(order))
+    if st != OK:
+        raise RtossError(st, status_string(st))
+    return top[:int(M)].copy(), order
 
 
 def rtoss_pattern_table_validate(masks, k):
@@ -246,6 +262,21 @@ class Context:
         self._check(lib.rtoss_pattern_usage(self.h, kernels.data_ptr(), _torch_dtype_code(kernels), n, _np_ptr(m), len(m),
                                             int(k), scratch.data_ptr(), counts.data_ptr(), _stream()))
         return counts.cpu().numpy().astype(np.uint64)
+
+    def rtoss_pattern_table_derive(self, kernels, k, preset, M):
+        """kernels: CUDA tensor [n, 9] -> (kept masks ascending, candidate masks, candidate counts)."""
+        import torch
+        n = kernels.numel() // 9
+        scratch = torch.empty(n, dtype=torch.uint8, device=kernels.device)
+        counts_dev = torch.zeros(255, dtype=torch.int64, device=kernels.device)
+        top = np.zeros(max(int(M), 1), dtype=np.uint16)
+        cand = np.zeros(255, dtype=np.uint16)
+        cnt = np.zeros(255, dtype=np.uint64)
+        kept, P = ctypes.c_int(0), ctypes.c_int(0)
+        self._check(lib.rtoss_pattern_table_derive(self.h, kernels.data_ptr(), _torch_dtype_code(kernels), n, int(k), int(preset),
+                                                   int(M), scratch.data_ptr(), counts_dev.data_ptr(), _np_ptr(top),
+                                                   ctypes.byref(kept), _np_ptr(cand), _np_ptr(cnt), ctypes.byref(P), _stream()))
+        return top[:kept.value].copy(), cand[:P.value].copy(), cnt[:P.value].copy()
 
     def rtoss_pack(self, w, ksize, masks, k, pid, compute_dtype, into=None):
         """New packed handle, or re-pack `into` (an existing handle of the same layer) without allocating."""

@@ -296,6 +296,39 @@ rtoss_status rtoss_pattern_usage(rtoss_ctx* ctx, const void* kernels_dev, rtoss_
     return le ? cuda_fail(ctx, "pattern usage launch", le) : RTOSS_OK;
 }
 
+rtoss_status rtoss_pattern_table_derive(rtoss_ctx* ctx, const void* kernels_dev, rtoss_dtype dtype, int64_t n_kernels,
+                                        int k, rtoss_preset preset, int M, uint8_t* pid_scratch_dev, uint64_t* counts_dev,
+                                        uint16_t* top_masks_host, int* M_kept, uint16_t* cand_masks_host,
+                                        uint64_t* cand_counts_host, int* P_candidates, void* cuda_stream) {
+    if (!ctx) return RTOSS_ERR_INVALID_ARG;
+    if (!top_masks_host || !M_kept || M < 1 || (preset != RTOSS_PRESET_ALL && preset != RTOSS_PRESET_CONN4)) {
+        set_err(ctx, "pattern table derive", "null argument, M < 1 or a preset that is not a candidate family");
+        return RTOSS_ERR_INVALID_ARG;
+    }
+    uint16_t cand[255];
+    int P = 255;
+    rtoss_status st = rtoss_pattern_preset(k, preset, cand, &P);
+    if (st != RTOSS_OK) {
+        set_err(ctx, "pattern table derive", "bad k for the preset");
+        return st;
+    }
+    st = rtoss_pattern_usage(ctx, kernels_dev, dtype, n_kernels, cand, P, k, pid_scratch_dev, counts_dev, cuda_stream);
+    if (st != RTOSS_OK) return st;
+    uint64_t counts[255];
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaMemcpyAsync(counts, counts_dev, sizeof(uint64_t) * (size_t)P, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(ctx, "pattern table derive", (int)e);
+    const int keep = M < P ? M : P;
+    st = rtoss_pattern_rank(cand, counts, P, k, keep, top_masks_host, nullptr);
+    if (st != RTOSS_OK) return st;
+    *M_kept = keep;
+    if (P_candidates) *P_candidates = P;
+    if (cand_masks_host) memcpy(cand_masks_host, cand, sizeof(uint16_t) * (size_t)P);
+    if (cand_counts_host) memcpy(cand_counts_host, counts, sizeof(uint64_t) * (size_t)P);
+    return RTOSS_OK;
+}
+
 rtoss_status rtoss_packed_info_get(const rtoss_packed* p, rtoss_packed_info* info) {
     if (!p || !info) return RTOSS_ERR_INVALID_ARG;
     info->Cout = p->Cout;

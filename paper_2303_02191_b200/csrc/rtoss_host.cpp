@@ -1,6 +1,7 @@
 // Host-only parts of librtoss: status text, pattern-table presets and
 // validation (Section IV.B of arXiv 2303.02191), layer grouping by depth-first
 // search (Section IV.A, Algorithm 1).  Plain C++, no CUDA.
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 #include <vector>
@@ -99,6 +100,26 @@ rtoss_status rtoss_pattern_preset(int k, rtoss_preset preset, uint16_t* masks_ho
 
 rtoss_status rtoss_pattern_table_validate(const uint16_t* masks_host, int P, int k) {
     return rtoss_table_ok(masks_host, P, k) ? RTOSS_OK : RTOSS_ERR_BAD_PATTERN_TABLE;
+}
+
+rtoss_status rtoss_pattern_rank(const uint16_t* masks_host, const uint64_t* counts_host, int P, int k, int M,
+                                uint16_t* top_masks_host, int* order_host) {
+    if (!masks_host || !counts_host || !top_masks_host) return RTOSS_ERR_INVALID_ARG;
+    if (!rtoss_table_ok(masks_host, P, k)) return RTOSS_ERR_BAD_PATTERN_TABLE;
+    if (M < 1 || M > P) return RTOSS_ERR_INVALID_ARG;
+    std::vector<int> order(P);
+    for (int i = 0; i < P; ++i) order[i] = i;
+    std::sort(order.begin(), order.end(), [&](int a, int b) {
+        if (counts_host[a] != counts_host[b]) return counts_host[a] > counts_host[b];
+        return masks_host[a] < masks_host[b];
+    });
+    if (order_host)
+        for (int i = 0; i < P; ++i) order_host[i] = order[i];
+    std::vector<uint16_t> top(M);
+    for (int i = 0; i < M; ++i) top[i] = masks_host[order[i]];
+    std::sort(top.begin(), top.end());
+    for (int i = 0; i < M; ++i) top_masks_host[i] = top[i];
+    return RTOSS_OK;
 }
 
 rtoss_status rtoss_group_layers(const rtoss_layer_node* nodes, int L, int* parent, int* group, int* n_groups) {

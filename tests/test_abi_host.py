@@ -131,3 +131,22 @@ def test_retinanet_program_add_fusion_keeps_a_valid_order():
     original = {op[3] if op[0] in ("conv", "add") else op[2] for op in ops}
     skipped = {op[3] for op in fused if op[0] == "convres"}
     assert written - {"in"} == original - skipped
+
+
+def test_pattern_rank_matches_the_oracle_on_ties_and_cuts(rt):
+    """rtoss_pattern_rank is host code: counts with many ties, every cut size."""
+    rng = np.random.default_rng(3)
+    for k, preset in ((2, orc.PRESET_CONN4), (3, orc.PRESET_CONN4), (4, orc.PRESET_ALL)):
+        masks = orc.pattern_preset(k, preset)
+        counts = rng.integers(0, 6, size=len(masks)).astype(np.uint64)     # few distinct values: many ties
+        for M in (1, 2, len(masks) // 2, len(masks)):
+            top, order = rt.rtoss_pattern_rank(masks, counts, k, M)
+            want_top, want_order = orc.pattern_rank(masks, counts, M)
+            assert np.array_equal(top, want_top) and np.array_equal(order, want_order)
+    masks = orc.pattern_preset(2, orc.PRESET_CONN4)
+    with pytest.raises(rt.RtossError):
+        rt.rtoss_pattern_rank(masks, np.zeros(len(masks), dtype=np.uint64), 2, 0)
+    with pytest.raises(rt.RtossError):
+        rt.rtoss_pattern_rank(masks, np.zeros(len(masks), dtype=np.uint64), 2, len(masks) + 1)
+    with pytest.raises(rt.RtossError):
+        rt.rtoss_pattern_rank(masks, np.zeros(len(masks), dtype=np.uint64), 3, 2)      # table is not a 3-entry table

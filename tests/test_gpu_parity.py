@@ -299,3 +299,22 @@ def test_pattern_usage_counts_match_oracle(k):
     assert np.array_equal(counts, want)
     assert int(counts.sum()) == sample.shape[0]
     assert (counts > 0).all()            # every edge-connected pattern wins somewhere in a quarter million kernels
+
+
+@pytest.mark.parametrize("k,preset,M", [(3, "conn4", 8), (2, "conn4", 12), (4, "all", 21), (5, "conn4", 16)])
+def test_pattern_table_derivation_matches_oracle(k, preset, M):
+    """Section IV.B end to end: candidates from Eq. 1 (with or without the adjacency criterion), usage over a seeded
+    sample in [-1, 1), the M most used.  Integers throughout: candidate table, counts and kept table are exact."""
+    pre_g = {"conn4": rt.PRESET_CONN4, "all": rt.PRESET_ALL}[preset]
+    pre_o = {"conn4": orc.PRESET_CONN4, "all": orc.PRESET_ALL}[preset]
+    sample = synth.uniform_kernels(6, 1 << 17)
+    top, cand, counts = gu.ctx().rtoss_pattern_table_derive(torch.from_numpy(sample).cuda(), k, pre_g, M)
+    want_top, want_cand, want_counts = orc.derive_pattern_table(sample, k, pre_o, M)
+    assert np.array_equal(cand, want_cand)
+    assert np.array_equal(counts, want_counts)
+    assert np.array_equal(top, want_top)
+    assert rt.rtoss_pattern_table_validate(top, k) == rt.OK
+    # the derived table is usable by the next step of the path
+    w = synth.kaiming_weights(6, 2, 16, 8, 3)
+    pid = gu.ctx().rtoss_select_patterns(torch.from_numpy(w).cuda(), 3, top, k)
+    assert np.array_equal(pid.cpu().numpy().ravel(), orc.select_3x3(w, want_top).ravel())

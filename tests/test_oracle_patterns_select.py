@@ -267,3 +267,87 @@ def test_1x1_flat_order_is_filter_major():
     masks = orc.pattern_preset(2, orc.PRESET_CONN4).tolist()
     pid1 = orc.select_1x1(w, masks)
     assert masks[pid1[0]] == 0x003 and masks[pid1[1]] == 0x180
+
+
+# ---------------------------------------------------------------- criterion 2: usage ranking and the cut
+
+def test_usage_of_one_tap_and_eight_tap_patterns_is_uniform():
+    """Closed form: for nine i.i.d. values every tap is equally likely to be the largest (1-entry patterns keep it)
+    and equally likely to be the smallest (8-entry patterns drop it): each of the nine patterns wins 1/9 of the
+    sample, within five standard deviations of the binomial count."""
+    n = 90000
+    sample = synth.uniform_kernels(11, n)
+    sd = math.sqrt(n * (1 / 9) * (8 / 9))
+    for k in (1, 8):
+        masks = orc.pattern_preset(k, orc.PRESET_ALL)
+        counts = orc.pattern_usage(sample, masks)
+        assert int(counts.sum()) == n and len(counts) == 9
+        assert np.all(np.abs(counts.astype(float) - n / 9) < 5 * sd)
+
+
+def test_usage_counts_against_a_pure_python_argmax():
+    masks = orc.pattern_preset(3, orc.PRESET_CONN4)
+    sample = synth.uniform_kernels(12, 500)
+    want = np.zeros(len(masks), dtype=np.uint64)
+    for kern in sample.reshape(-1, 9):
+        sq = [float(np.float32(v) * np.float32(v)) for v in kern]
+        best, best_e = 0, -1.0
+        for p, m in enumerate(masks):
+            e = np.float32(0)
+            for t in range(9):
+                if (int(m) >> t) & 1:
+                    e = np.float32(e + np.float32(sq[t]))
+            if float(e) > best_e:
+                best, best_e = p, float(e)
+        want[best] += 1
+    assert np.array_equal(orc.pattern_usage(sample, masks), want)
+
+
+def test_usage_is_symmetric_under_the_squares_symmetries():
+    """A uniform sample has no preferred direction: patterns that are rotations / reflections of one another (one
+    orbit of the square's symmetry group) are used equally often up to sampling noise.  The twelve dominoes fall into
+    two orbits: eight touching a corner, four touching the centre."""
+    def image(mask, f):
+        out = 0
+        for t in range(9):
+            if (mask >> t) & 1:
+                r, c = divmod(t, 3)
+                r2, c2 = f(r, c)
+                out |= 1 << (3 * r2 + c2)
+        return out
+    syms = [lambda r, c: (r, c), lambda r, c: (c, 2 - r), lambda r, c: (2 - r, 2 - c), lambda r, c: (2 - c, r),
+            lambda r, c: (r, 2 - c), lambda r, c: (2 - r, c), lambda r, c: (c, r), lambda r, c: (2 - c, 2 - r)]
+    masks = [int(m) for m in orc.pattern_preset(2, orc.PRESET_CONN4)]
+    counts = orc.pattern_usage(synth.uniform_kernels(13, 120000), masks).astype(float)
+    orbits = {}
+    for m, c in zip(masks, counts):
+        orbits.setdefault(min(image(m, f) for f in syms), []).append(c)
+    assert sorted(len(v) for v in orbits.values()) == [4, 8]
+    for v in orbits.values():
+        assert max(v) / min(v) < 1.1
+
+
+def test_rank_orders_by_count_then_mask_and_returns_a_table():
+    masks = np.array([0x003, 0x006, 0x009, 0x012, 0x018, 0x024], dtype=np.uint16)
+    counts = np.array([5, 9, 5, 0, 9, 7], dtype=np.uint64)
+    top, order = orc.pattern_rank(masks, counts, 4)
+    assert list(order) == [1, 4, 5, 0, 2, 3]                 # 9 (mask 0x006), 9 (0x018), 7, 5 (0x003), 5 (0x009), 0
+    assert list(top) == [0x003, 0x006, 0x018, 0x024]         # the four best, ascending
+    assert orc.pattern_table_valid(top, 2)
+    full, _ = orc.pattern_rank(masks, counts, 6)
+    assert np.array_equal(full, masks)                       # keeping all candidates returns the table itself
+    one, _ = orc.pattern_rank(masks, counts, 1)
+    assert list(one) == [0x006]                              # the tie at 9 goes to the lower mask
+
+
+def test_derive_keeps_a_subset_with_the_largest_counts():
+    sample = synth.uniform_kernels(14, 40000)
+    top, cand, counts = orc.derive_pattern_table(sample, 3, orc.PRESET_CONN4, 8)
+    assert len(top) == 8 and set(top) <= set(cand) and orc.pattern_table_valid(top, 3)
+    kept = np.isin(cand, top)
+    assert counts[kept].min() >= counts[~kept].max()
+    everything, _, _ = orc.derive_pattern_table(sample, 3, orc.PRESET_CONN4, 1000)
+    assert np.array_equal(everything, cand)
+    # Eq. 1 alone as the candidate family: the most used 4-entry patterns over all 126
+    top4, cand4, _ = orc.derive_pattern_table(sample, 4, orc.PRESET_ALL, 21)
+    assert len(cand4) == math.comb(9, 4) and len(top4) == 21
