@@ -188,6 +188,39 @@ __device__ __forceinline__ void umma_f16(unsigned d_tmem, unsigned long long ade
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// 1x1 layers: the MMAs of one channel block (nk4 <= 4 slabs of 16 channels; filters on M), with a look at the "full"
+// barriers of the NEXT activation and weight stage started in front of them (mbarrier.test_wait: the answer comes
+// back while the MMAs are being issued).  A wait costs the issuing thread a round trip of a few hundred cycles through
+// a memory pipe the epilogue warps keep busy, and with four MMAs per wait nothing hides two of those per channel
+// block; the stages ahead are normally full already, so the look usually replaces both waits of the next block.
+// Returns bit 0: next activation stage full, bit 1: next weight stage full.
+__device__ __forceinline__ unsigned umma_block_peek(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc,
+                                                    unsigned idesc, unsigned accumulate, int nk4, unsigned barA,
+                                                    unsigned parA, unsigned barB, unsigned parB) {
+    unsigned res;
+    asm volatile(
+        "{\n\t.reg .pred pa, pb, q, p1, p2, p3, pt;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t.reg .b32 ta, tb;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 pa, [%7], %8;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 pb, [%9], %10;\n\t"
+        "setp.ne.b32 q, %5, 0;\n\t"
+        "setp.gt.s32 p1, %6, 1;\n\t"
+        "setp.gt.s32 p2, %6, 2;\n\t"
+        "setp.gt.s32 p3, %6, 3;\n\t"
+        "setp.eq.s32 pt, %6, %6;\n\t"
+        "add.u64 a1, %2, 2;\n\tadd.u64 a2, %2, 4;\n\tadd.u64 a3, %2, 6;\n\t"
+        "add.u64 b1, %3, 2;\n\tadd.u64 b2, %3, 4;\n\tadd.u64 b3, %3, 6;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %3, %4, q;\n\t"
+        "@p1 tcgen05.mma.cta_group::1.kind::f16 [%1], a1, b1, %4, pt;\n\t"
+        "@p2 tcgen05.mma.cta_group::1.kind::f16 [%1], a2, b2, %4, pt;\n\t"
+        "@p3 tcgen05.mma.cta_group::1.kind::f16 [%1], a3, b3, %4, pt;\n\t"
+        "selp.u32 ta, 1, 0, pa;\n\t"
+        "selp.u32 tb, 2, 0, pb;\n\t"
+        "or.b32 %0, ta, tb;\n\t}"
+        : "=r"(res)
+        : "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(nk4), "r"(barA), "r"(parA), "r"(barB), "r"(parB)
+        : "memory");
+    return res;
+}
 // Arrive on an mbarrier once all tcgen05.mma issued so far by this thread have completed.
 __device__ __forceinline__ void umma_commit(unsigned bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -674,6 +707,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const bool pxm = a.pxm != 0, two = a.MH == 2, unrolled9 = a.taps == 9 && a.G == 3;
             int sa = 0, sb = 0, as = 0, n_done = 0;
             unsigned pa = 0, pb = 0, pacc = 0;  // phase parities of the three rings
+            unsigned peek = 0;                  // 1x1: what umma_block_peek saw of the stages now current
             auto mk = [desc_hi](unsigned lo) { return ((unsigned long long)desc_hi << 32) | lo; };
             // all instructions of one tap: nk4 K slabs (times two halves of positions with the positions as M)
             auto issue_tap = [&](unsigned d_base, unsigned wl, unsigned xl, int nk4, unsigned& acc) {
@@ -705,21 +739,67 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int ks = tile % a.KS, cb_end = min(a.ncb, (ks + 1) * a.cb_per);
                 int left = a.Cin - ks * a.cb_per * kKBlock;
                 for (int cb = ks * a.cb_per; cb < cb_end && ok; ++cb, left -= kKBlock) {
-                    ok = mbar_wait(bar_fullA + 8 * sa, pa);
+                    if (a.taps == 1) {
+                        if (!(peek & 1u)) ok = mbar_wait(bar_fullA + 8 * sa, pa);
+                        if (ok && !(peek & 2u)) ok = mbar_wait(bar_fullB + 8 * sb, pb);
+                        if (!ok) break;
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        const int nk4 = left >= kKBlock ? kKBlock / 16 : (left + 15) >> 4;
+                        const int sa_n = sa + 1 == a.NA ? 0 : sa + 1, sb_n = sb + 1 == a.NB ? 0 : sb + 1;
+                        const unsigned pa_n = sa_n ? pa : pa ^ 1, pb_n = sb_n ? pb : pb ^ 1;
+                        const unsigned wl0 = desc_lo0 + (sB >> 4) + (unsigned)sb * bstage16;
+                        const unsigned xl0 = desc_lo0 + (sA >> 4) + (unsigned)sa * astage16;
+                        if (!pxm) {
+                            peek = umma_block_peek(d_base, mk(wl0), mk(xl0), idesc, acc, nk4, bar_fullA + 8 * sa_n, pa_n,
+                                                   bar_fullB + 8 * sb_n, pb_n);
+                        } else {
+                            // positions on M: the first 128 positions with the look ahead, then the second 128
+                            peek = umma_block_peek(d_base, mk(xl0), mk(wl0), idesc, acc, nk4, bar_fullA + 8 * sa_n, pa_n,
+                                                   bar_fullB + 8 * sb_n, pb_n);
+                            if (two) {
+                                unsigned acc2 = acc;
+#pragma unroll
+                                for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
+                                    if (k4 < nk4) {
+                                        umma_f16(d_base + hi_cols, mk(xl0 + 1024 + 2 * k4), mk(wl0 + 2 * k4), idesc, acc2);
+                                        acc2 = 1;
+                                    }
+                                }
+                            }
+                        }
+                        acc = 1;
+                        umma_commit(bar_emptyB + 8 * sb);
+                        umma_commit(bar_emptyA + 8 * sa);
+                        sa = sa_n, pa = pa_n, sb = sb_n, pb = pb_n;
+                        continue;
+                    }
+                    if (!(peek & 1u)) ok = mbar_wait(bar_fullA + 8 * sa, pa);   // (peek stays 0 on the paths that do not look ahead)
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const unsigned xl0 = desc_lo0 + (sA >> 4) + (unsigned)sa * astage16;
                     // 16-channel slabs of this block that hold channels (the rest of the 64 is TMA zero fill)
                     const int nk4 = left >= kKBlock ? kKBlock / 16 : (left + 15) >> 4;
                     if (unrolled9) {
+                        const int sa_n = sa + 1 == a.NA ? 0 : sa + 1;
+                        const unsigned pa_n = sa_n ? pa : pa ^ 1;
 #pragma unroll
                         for (int s3 = 0; s3 < 3; ++s3) {
-                            ok = ok && mbar_wait(bar_fullB + 8 * sb, pb);
+                            if (!(peek & 2u)) ok = ok && mbar_wait(bar_fullB + 8 * sb, pb);
                             if (ok) {
                                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                                 const unsigned wl0 = desc_lo0 + (sB >> 4) + (unsigned)sb * bstage16;
+                                if (!pxm) {
+                                    // the first tap of the stage goes out together with a look at the next stages
+                                    const int sb_n = sb + 1 == a.NB ? 0 : sb + 1;
+                                    peek = umma_block_peek(d_base, mk(wl0), mk(xl0 + tap16[s3 * 3]), idesc, acc, nk4,
+                                                           bar_fullA + 8 * sa_n, pa_n, bar_fullB + 8 * sb_n, sb_n ? pb : pb ^ 1);
+                                    acc = 1;
 #pragma unroll
-                                for (int i = 0; i < 3; ++i) issue_tap(d_base, wl0 + i * wtile16, xl0 + tap16[s3 * 3 + i], nk4, acc);
+                                    for (int i = 1; i < 3; ++i) issue_tap(d_base, wl0 + i * wtile16, xl0 + tap16[s3 * 3 + i], nk4, acc);
+                                } else {
+#pragma unroll
+                                    for (int i = 0; i < 3; ++i) issue_tap(d_base, wl0 + i * wtile16, xl0 + tap16[s3 * 3 + i], nk4, acc);
+                                }
                                 umma_commit(bar_emptyB + 8 * sb);  // this weight stage may be refilled once the MMAs have read it
                                 if (++sb == a.NB) {
                                     sb = 0;
