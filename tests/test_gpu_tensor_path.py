@@ -181,3 +181,20 @@ def test_tensor_path_narrow_channel_slice(y_off, y_stride):
     assert orc.rel_err(y[:, y_off:y_off + Cout], ref) <= gu.TOL["bf16"]
     _no_timeout()
     packed.close()
+
+
+MANY_TILES = [
+    # ks, stride, N, Cin, Cout, H, W, k, dtype, act: several tiles per CTA, so the operand rings wrap and their phase
+    # parities flip inside one CTA while the MMA thread's early look at the next stages crosses tile boundaries
+    (1, 1, 2, 320, 192, 120, 136, 4, "bf16", "silu"),    # five channel blocks per tile, ragged last block, two filter tiles
+    (1, 1, 2, 136, 48, 150, 200, 3, "bf16", "relu"),     # positions on M, three channel blocks (the last one 8 channels)
+    (3, 1, 2, 64, 64, 200, 272, 4, "bf16", "silu"),      # 3x3, one channel block per tile, about three tiles per CTA
+    (3, 2, 2, 128, 128, 160, 200, 4, "f16", "none"),     # stride 2: four staged sub-tiles per activation stage
+]
+
+
+@pytest.mark.parametrize("case", MANY_TILES, ids=lambda c: "-".join(str(v) for v in c))
+def test_tensor_path_many_tiles_per_cta(case):
+    ks, s, N, Cin, Cout, H, W, k, dt, act = case
+    gu.check_layer(27, 900 + Cin + W, ks, N, Cin, Cout, H, W, s, k, _table(k), dt, act, "nhwc", path=rt.PATH_TENSOR)
+    _no_timeout()
