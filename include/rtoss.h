@@ -276,6 +276,10 @@ typedef struct {
                                * path only (16-bit NHWC, more than 64 filters or a 3x3 kernel, pointer 16-byte
                                * aligned): other calls return RTOSS_ERR_UNSUPPORTED before anything is launched
                                * and the caller adds separately. */
+    int residual_after_act;   /* 0: as above.  1: the residual is added behind the activation instead,
+                               * y = round(act(conv + bias)) + residual, rounded once more: bit for bit (every
+                               * activation) what the convolution followed by rtoss_add_act with act = none gives
+                               * (the shortcut of a bottleneck block whose last convolution carries the activation). */
 } rtoss_conv_desc;
 
 /* y[n,co,oy,ox] = act( bias[co] + sum_ci sum_{t in mask(pid[co,ci])}

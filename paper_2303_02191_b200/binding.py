@@ -60,7 +60,7 @@ class ConvDesc(ctypes.Structure):
     _fields_ = [("N", ctypes.c_int), ("H", ctypes.c_int), ("W", ctypes.c_int), ("stride", ctypes.c_int),
                 ("layout", ctypes.c_int), ("io_dtype", ctypes.c_int), ("act", ctypes.c_int),
                 ("bias_dev", ctypes.c_void_p), ("y_channel_offset", ctypes.c_int), ("y_channel_stride", ctypes.c_int),
-                ("path", ctypes.c_int), ("residual_dev", ctypes.c_void_p)]
+                ("path", ctypes.c_int), ("residual_dev", ctypes.c_void_p), ("residual_after_act", ctypes.c_int)]
 
 
 def _load():
@@ -291,11 +291,12 @@ class Context:
         """items: list of dict(w, ksize, masks, k, packed, pid=None, pid_from=-1) -> Batch (whole-model pass)."""
         return Batch(self, items)
 
-    def _desc(self, x_shape_nchw, stride, layout, io_dtype, act, bias, y_off, y_stride, path=PATH_AUTO, residual=None):
+    def _desc(self, x_shape_nchw, stride, layout, io_dtype, act, bias, y_off, y_stride, path=PATH_AUTO, residual=None,
+              residual_after_act=False):
         N, _, H, W = x_shape_nchw
         return ConvDesc(int(N), int(H), int(W), int(stride), int(layout), int(io_dtype), int(act),
                         bias.data_ptr() if bias is not None else None, int(y_off), int(y_stride), int(path),
-                        residual.data_ptr() if residual is not None else None)
+                        residual.data_ptr() if residual is not None else None, 1 if residual_after_act else 0)
 
     def rtoss_device_status(self):
         """Synchronise the device and return the code a timed-out device wait left (0 = none)."""
@@ -306,16 +307,16 @@ class Context:
         return code.value
 
     def rtoss_conv3x3_pattern(self, packed, x, y, N, H, W, stride=1, layout=NCHW, act=ACT_NONE, bias=None,
-                              y_channel_offset=0, y_channel_stride=0, path=PATH_AUTO, residual=None):
+                              y_channel_offset=0, y_channel_stride=0, path=PATH_AUTO, residual=None, residual_after_act=False):
         d = self._desc((N, 0, H, W), stride, layout, _torch_dtype_code(x), act, bias, y_channel_offset, y_channel_stride,
-                       path, residual)
+                       path, residual, residual_after_act)
         self._check(lib.rtoss_conv3x3_pattern(self.h, packed.h, x.data_ptr(), y.data_ptr(), ctypes.byref(d), _stream()))
         return y
 
     def rtoss_conv1x1_pattern(self, packed, x, y, N, H, W, stride=1, layout=NCHW, act=ACT_NONE, bias=None,
-                              y_channel_offset=0, y_channel_stride=0, path=PATH_AUTO, residual=None):
+                              y_channel_offset=0, y_channel_stride=0, path=PATH_AUTO, residual=None, residual_after_act=False):
         d = self._desc((N, 0, H, W), stride, layout, _torch_dtype_code(x), act, bias, y_channel_offset, y_channel_stride,
-                       path, residual)
+                       path, residual, residual_after_act)
         self._check(lib.rtoss_conv1x1_pattern(self.h, packed.h, x.data_ptr(), y.data_ptr(), ctypes.byref(d), _stream()))
         return y
 

@@ -76,6 +76,7 @@ constexpr long long kWaitCycles = 2000000000LL;  // about one second
 struct TcArgs {
     void* y;
     const void* resid;   // residual operand laid out like y, or null
+    int resid_post;      // 1: the residual is added behind the activation (y = act(conv) + residual), 0: in front of it
     const float* bias;
     int* status;
     int N, Ho, Wo, Cin, Cout;    // output image size
@@ -355,11 +356,11 @@ __device__ __forceinline__ uint4 add_residual8(uint4 o, const uint4 rv) {
 // With a residual operand (rbv, laid out like the output) the activation moves behind the residual add.
 template <typename T, int ACT>
 __device__ __forceinline__ void epilogue_half(const unsigned (&r)[16], float bs, unsigned wr, unsigned rd, unsigned tab_at,
-                                              T* ybv, unsigned ry, unsigned rx, const T* rbv = nullptr) {
-    const bool res = rbv != nullptr;   // then bs is the plain bias and nothing is activated before the add
+                                              T* ybv, unsigned ry, unsigned rx, const T* rbv = nullptr, bool post = false) {
+    const bool res = rbv != nullptr;   // then (unless post) bs is the plain bias and nothing is activated before the add
 #pragma unroll
     for (int jp = 0; jp < kPatchRows / 2; ++jp) {
-        const unsigned w = res ? round_pack<T, false>(__uint_as_float(r[2 * jp]) + bs, __uint_as_float(r[2 * jp + 1]) + bs)
+        const unsigned w = (res && !post) ? round_pack<T, false>(__uint_as_float(r[2 * jp]) + bs, __uint_as_float(r[2 * jp + 1]) + bs)
                                : round_pack<T, ACT == RTOSS_ACT_RELU>(bias_act<ACT>(r[2 * jp], bs), bias_act<ACT>(r[2 * jp + 1], bs));
         asm volatile("st.shared.u32 [%0], %1;" ::"r"(wr + jp * kPairPitch), "r"(w) : "memory");
     }
@@ -372,13 +373,19 @@ __device__ __forceinline__ void epilogue_half(const unsigned (&r)[16], float bs,
     if ((e[1] >> 16) < ry && (e[1] & 0xFFFFu) < rx) {
         uint4 o = make_uint4(__byte_perm(w[0], w[1], 0x5410), __byte_perm(w[2], w[3], 0x5410), __byte_perm(w[4], w[5], 0x5410),
                              __byte_perm(w[6], w[7], 0x5410));
-        if (res) o = add_residual8<T, ACT>(o, *reinterpret_cast<const uint4*>(rbv + e[0]));
+        if (res) {
+            const uint4 rv = *reinterpret_cast<const uint4*>(rbv + e[0]);
+            o = post ? add_residual8<T, RTOSS_ACT_NONE>(o, rv) : add_residual8<T, ACT>(o, rv);
+        }
         *reinterpret_cast<uint4*>(ybv + e[0]) = o;
     }
     if ((e[3] >> 16) < ry && (e[3] & 0xFFFFu) < rx) {
         uint4 o = make_uint4(__byte_perm(w[0], w[1], 0x7632), __byte_perm(w[2], w[3], 0x7632), __byte_perm(w[4], w[5], 0x7632),
                              __byte_perm(w[6], w[7], 0x7632));
-        if (res) o = add_residual8<T, ACT>(o, *reinterpret_cast<const uint4*>(rbv + e[2]));
+        if (res) {
+            const uint4 rv = *reinterpret_cast<const uint4*>(rbv + e[2]);
+            o = post ? add_residual8<T, RTOSS_ACT_NONE>(o, rv) : add_residual8<T, ACT>(o, rv);
+        }
         *reinterpret_cast<uint4*>(ybv + e[2]) = o;
     }
     __syncwarp();
@@ -438,12 +445,14 @@ __device__ __forceinline__ void fetch_residual(unsigned tab_at, const T* rbv, un
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
 
-template <typename T, int ACT>
+template <typename T, int ACT, bool POST>
 __device__ __forceinline__ void epilogue_half_res(const unsigned (&r)[16], float bias, unsigned wr, unsigned rd, unsigned tab_at,
                                                   T* ybv, unsigned ry, unsigned rx, unsigned slot) {
 #pragma unroll
     for (int jp = 0; jp < kPatchRows / 2; ++jp) {
-        const unsigned w = round_pack<T, false>(__uint_as_float(r[2 * jp]) + bias, __uint_as_float(r[2 * jp + 1]) + bias);
+        // POST: activated and rounded as without a residual (bias is then what bias_act expects); else the plain sum
+        const unsigned w = POST ? round_pack<T, ACT == RTOSS_ACT_RELU>(bias_act<ACT>(r[2 * jp], bias), bias_act<ACT>(r[2 * jp + 1], bias))
+                                : round_pack<T, false>(__uint_as_float(r[2 * jp]) + bias, __uint_as_float(r[2 * jp + 1]) + bias);
         asm volatile("st.shared.u32 [%0], %1;" ::"r"(wr + jp * kPairPitch), "r"(w) : "memory");
     }
     __syncwarp();
@@ -456,19 +465,19 @@ __device__ __forceinline__ void epilogue_half_res(const unsigned (&r)[16], float
         asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(rv.x), "=r"(rv.y), "=r"(rv.z), "=r"(rv.w) : "r"(slot));
         const uint4 o = make_uint4(__byte_perm(w[0], w[1], 0x5410), __byte_perm(w[2], w[3], 0x5410),
                                    __byte_perm(w[4], w[5], 0x5410), __byte_perm(w[6], w[7], 0x5410));
-        *reinterpret_cast<uint4*>(ybv + e[0]) = add_residual8<T, ACT>(o, rv);
+        *reinterpret_cast<uint4*>(ybv + e[0]) = add_residual8<T, POST ? RTOSS_ACT_NONE : ACT>(o, rv);
     }
     if ((e[3] >> 16) < ry && (e[3] & 0xFFFFu) < rx) {
         uint4 rv;
         asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(rv.x), "=r"(rv.y), "=r"(rv.z), "=r"(rv.w) : "r"(slot + 512u));
         const uint4 o = make_uint4(__byte_perm(w[0], w[1], 0x7632), __byte_perm(w[2], w[3], 0x7632),
                                    __byte_perm(w[4], w[5], 0x7632), __byte_perm(w[6], w[7], 0x7632));
-        *reinterpret_cast<uint4*>(ybv + e[2]) = add_residual8<T, ACT>(o, rv);
+        *reinterpret_cast<uint4*>(ybv + e[2]) = add_residual8<T, POST ? RTOSS_ACT_NONE : ACT>(o, rv);
     }
     __syncwarp();
 }
 
-template <typename T, int ACT>
+template <typename T, int ACT, bool POST>
 __device__ __forceinline__ void epilogue_chunks_res(unsigned d_base, int c0, int c_step, int n_px, float bias,
                                                     unsigned patch, unsigned tab, T* yb, unsigned ry, unsigned rx,
                                                     int lane, const T* rb, unsigned stage) {
@@ -487,7 +496,7 @@ __device__ __forceinline__ void epilogue_chunks_res(unsigned d_base, int c0, int
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         tmem_ld16(d_base + (unsigned)(c0 + kPatchRows), rb2);
         asm volatile("cp.async.wait_group 1;" ::: "memory");   // the pieces of this half are in
-        epilogue_half_res<T, ACT>(ra, bias, wr, rd, tab_l + (unsigned)c0 * 8, ybv, ry, rx, slot0);
+        epilogue_half_res<T, ACT, POST>(ra, bias, wr, rd, tab_l + (unsigned)c0 * 8, ybv, ry, rx, slot0);
         const bool more = c0 + c_step < n_px;
         if (more)
             fetch_residual<T>(tab_l + (unsigned)(c0 + c_step) * 8, rbv, ry, rx, slot0);
@@ -496,7 +505,7 @@ __device__ __forceinline__ void epilogue_chunks_res(unsigned d_base, int c0, int
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         if (more) tmem_ld16(d_base + (unsigned)(c0 + c_step), ra);
         asm volatile("cp.async.wait_group 1;" ::: "memory");
-        epilogue_half_res<T, ACT>(rb2, bias, wr, rd, tab_l + (unsigned)(c0 + kPatchRows) * 8, ybv, ry, rx, slot1);
+        epilogue_half_res<T, ACT, POST>(rb2, bias, wr, rd, tab_l + (unsigned)(c0 + kPatchRows) * 8, ybv, ry, rx, slot1);
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
@@ -508,7 +517,7 @@ __device__ __forceinline__ void epilogue_chunks_res(unsigned d_base, int c0, int
 template <typename T, int ACT>
 __device__ __forceinline__ void epilogue_from_shares(unsigned buf, int KS, int rank, int n_lc, int sub, int row, int n_px, float bs,
                                                      bool vec_ok, bool co_ok, unsigned patch, unsigned tab, const uint2* pos_tab,
-                                                     T* yb, unsigned ry, unsigned rx, int lane, const T* rb) {
+                                                     T* yb, unsigned ry, unsigned rx, int lane, const T* rb, bool post) {
     const unsigned wr = patch + lane * 4;
     const unsigned rd = patch + (lane >> 2) * kPairPitch + (lane & 3) * 32;
     const unsigned tab_l = tab + (unsigned)(2 * (lane >> 2)) * 8;
@@ -533,14 +542,18 @@ __device__ __forceinline__ void epilogue_from_shares(unsigned buf, int KS, int r
 #pragma unroll
         for (int j = 0; j < kPatchRows; ++j) r[j] = __float_as_uint(sum[j]);
         if (vec_ok) {
-            epilogue_half<T, ACT>(r, bs, wr, rd, tab_l + (unsigned)c0 * 8, ybv, ry, rx, rbv);
+            epilogue_half<T, ACT>(r, bs, wr, rd, tab_l + (unsigned)c0 * 8, ybv, ry, rx, rbv, post);
         } else {
 #pragma unroll
             for (int j = 0; j < kPatchRows; ++j) {
                 const uint2 e = pos_tab[c0 + j];
                 if (co_ok && (e.y >> 16) < ry && (e.y & 0xFFFFu) < rx) {
                     float v;
-                    if (rb) {   // round, add the residual, activate, round
+                    if (rb && post) {   // activate, round, add the residual, round
+                        v = bias_act<ACT>(r[j], bs);
+                        if (ACT == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
+                        v = to_f32<T>(from_f32<T>(v)) + to_f32<T>(rb[e.x + lane]);
+                    } else if (rb) {   // round, add the residual, activate, round
                         v = to_f32<T>(from_f32<T>(__uint_as_float(r[j]) + bs)) + to_f32<T>(rb[e.x + lane]);
                         if (ACT == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
                         if (ACT == RTOSS_ACT_SILU) {
@@ -933,7 +946,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const unsigned ry = (unsigned)min(a.TH, a.Ho - y0), rx = (unsigned)min(a.TW, a.Wo - x0);  // rows / columns inside the image
             const int c_first = (sub + 4 * copy) * 32, c_step = 128 * a.R;
             const T* rb = a.resid ? reinterpret_cast<const T*>(a.resid) + (yb - yg) : nullptr;   // laid out like y
-            const float bs = (a.act == RTOSS_ACT_SILU && !rb) ? 0.5f * bv : bv;   // (with a residual the bias is added plain)
+            const bool post = a.resid_post != 0;
+            const float bs = (a.act == RTOSS_ACT_SILU && (!rb || post)) ? 0.5f * bv : bv;   // (a residual in front of the activation: plain bias)
             ok = mbar_wait(bar_accFull + 8 * as, (gt / a.AS) & 1);
             if (!ok && a.KS == 1) break;   // (split K: the cluster barriers below must still be passed)
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -963,23 +977,29 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (ok) {
                     const int row = quarter * 32 + lane;
                     if (a.act == RTOSS_ACT_SILU)
-                        epilogue_from_shares<T, RTOSS_ACT_SILU>(sA, a.KS, rank, n_lc, sub, row, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane, rb);
+                        epilogue_from_shares<T, RTOSS_ACT_SILU>(sA, a.KS, rank, n_lc, sub, row, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane, rb, post);
                     else if (a.act == RTOSS_ACT_RELU)
-                        epilogue_from_shares<T, RTOSS_ACT_RELU>(sA, a.KS, rank, n_lc, sub, row, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane, rb);
+                        epilogue_from_shares<T, RTOSS_ACT_RELU>(sA, a.KS, rank, n_lc, sub, row, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane, rb, post);
                     else
-                        epilogue_from_shares<T, RTOSS_ACT_NONE>(sA, a.KS, rank, n_lc, sub, row, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane, rb);
+                        epilogue_from_shares<T, RTOSS_ACT_NONE>(sA, a.KS, rank, n_lc, sub, row, a.N_px, bs, vec_ok, co_ok, patch, s_tab, pos_tab, yb, ry, rx, lane, rb, post);
                 }
                 continue;
             }
             if (vec_ok) {
                 if (rb) {
                     const unsigned stage = s_res + (unsigned)(warp - 2) * kResStage;
-                    if (a.act == RTOSS_ACT_SILU)
-                        epilogue_chunks_res<T, RTOSS_ACT_SILU>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb, stage);
-                    else if (a.act == RTOSS_ACT_RELU)
-                        epilogue_chunks_res<T, RTOSS_ACT_RELU>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb, stage);
-                    else
-                        epilogue_chunks_res<T, RTOSS_ACT_NONE>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb, stage);
+#define RTOSS_RES_CALL(ACT_, POST_) \
+    epilogue_chunks_res<T, ACT_, POST_>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb, stage)
+                    if (post) {
+                        if (a.act == RTOSS_ACT_SILU) RTOSS_RES_CALL(RTOSS_ACT_SILU, true);
+                        else if (a.act == RTOSS_ACT_RELU) RTOSS_RES_CALL(RTOSS_ACT_RELU, true);
+                        else RTOSS_RES_CALL(RTOSS_ACT_NONE, false);   // no activation: both orders are the same sum
+                    } else {
+                        if (a.act == RTOSS_ACT_SILU) RTOSS_RES_CALL(RTOSS_ACT_SILU, false);
+                        else if (a.act == RTOSS_ACT_RELU) RTOSS_RES_CALL(RTOSS_ACT_RELU, false);
+                        else RTOSS_RES_CALL(RTOSS_ACT_NONE, false);
+                    }
+#undef RTOSS_RES_CALL
                 } else if (a.act == RTOSS_ACT_SILU)
                     epilogue_chunks<T, RTOSS_ACT_SILU>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb);
                 else if (a.act == RTOSS_ACT_RELU)
@@ -997,13 +1017,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         const uint2 e = pos_tab[c0 + j];
                         const bool in_img = co_ok && (e.y >> 16) < ry && (e.y & 0xFFFFu) < rx;
                         float v = __uint_as_float(r[j]) + bv;
-                        if (rb && in_img) v = to_f32<T>(from_f32<T>(v)) + to_f32<T>(rb[e.x + lane]);   // round, then add the residual
+                        if (rb && in_img && !post) v = to_f32<T>(from_f32<T>(v)) + to_f32<T>(rb[e.x + lane]);   // round, then add the residual
                         if (a.act == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
                         if (a.act == RTOSS_ACT_SILU) {
                             float th;
                             asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(0.5f * v));
                             v = v * fmaf(0.5f, th, 0.5f);
                         }
+                        if (rb && in_img && post) v = to_f32<T>(from_f32<T>(v)) + to_f32<T>(rb[e.x + lane]);   // behind the activation
                         if (co_ok && (e.y >> 16) < ry && (e.y & 0xFFFFu) < rx) yb[e.x + lane] = from_f32<T>(v);
                     }
                 }
@@ -1166,6 +1187,7 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     TcArgs a;
     a.y = y;
     a.resid = d->residual_dev;
+    a.resid_post = (d->residual_dev && d->residual_after_act) ? 1 : 0;
     a.bias = d->bias_dev;
     a.status = ctx->dev_status;
     a.N = d->N;

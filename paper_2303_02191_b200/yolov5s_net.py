@@ -100,14 +100,35 @@ def program(H0, W0):
 OUTPUTS = ("o3", "o4", "o5")
 
 
+def fuse_shortcuts(ops):
+    """A bottleneck's shortcut add directly behind its second convolution, whose output nothing else reads, becomes
+    ('convres', layer_index, src, tmp, other, dst): the convolution adds the block input behind its activation."""
+    reads = {}
+    for op in ops:
+        for s_ in ((op[2],) if op[0] == "conv" else (op[1], op[2]) if op[0] == "add" else (op[1],)):
+            reads[s_] = reads.get(s_, 0) + 1
+    out = []
+    for op in ops:
+        prev = out[-1] if out else None
+        if (op[0] == "add" and prev is not None and prev[0] == "conv" and prev[4] == 0 and prev[3] == op[2]
+                and reads[op[2]] == 1 and op[1] != op[2]):
+            out[-1] = ("convres", prev[1], prev[2], prev[3], op[1], op[3])
+        else:
+            out.append(op)
+    return out
+
+
 class GpuNet:
     """The program on the GPU through the C-ABI library: NHWC, bf16 (or fp16), k-entry patterns."""
 
-    def __init__(self, ctx, N, H0=640, W0=640, k=4, seed=0, dtype="bf16"):
+    def __init__(self, ctx, N, H0=640, W0=640, k=4, seed=0, dtype="bf16", fuse_residual=True):
         import torch
         from . import binding as rt
         self.rt, self.ctx, self.N, self.torch = rt, ctx, N, torch
         self.ops, self.bufs, self.layers = program(H0, W0)
+        if fuse_residual:
+            self.ops = fuse_shortcuts(self.ops)
+        self.unfused = set()   # layers whose fused call the library declined: convolution and add run separately
         tdt = {"bf16": torch.bfloat16, "f16": torch.float16}[dtype]
         self.t = {n: torch.zeros((N, H, W, C), dtype=tdt, device="cuda") for n, (C, H, W) in self.bufs.items()}
         masks = rt.rtoss_pattern_preset(k, rt.PRESET_CENTRE8 if k == 4 else rt.PRESET_CONN4)
@@ -131,6 +152,21 @@ class GpuNet:
                 fn = self.ctx.rtoss_conv3x3_pattern if L["ksize"] == 3 else self.ctx.rtoss_conv1x1_pattern
                 fn(self.packed[i], t[src], t[dst], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_SILU, self.bias[i],
                    off, self.bufs[dst][0])
+            elif op[0] == "convres":   # second convolution of a bottleneck + its shortcut in one call
+                _, i, src, tmp, other, dst = op
+                L = self.layers[i]
+                fn = self.ctx.rtoss_conv3x3_pattern if L["ksize"] == 3 else self.ctx.rtoss_conv1x1_pattern
+                if i not in self.unfused:
+                    try:
+                        fn(self.packed[i], t[src], t[dst], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_SILU, self.bias[i],
+                           residual=t[other], residual_after_act=True)
+                        continue
+                    except rt.RtossError as err:
+                        if err.status != rt.ERR_UNSUPPORTED:
+                            raise
+                        self.unfused.add(i)
+                fn(self.packed[i], t[src], t[tmp], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_SILU, self.bias[i])
+                rt.rtoss_add_act(t[other], t[tmp], t[dst], rt.ACT_NONE)
             elif op[0] == "add":
                 rt.rtoss_add_act(t[op[1]], t[op[2]], t[op[3]], rt.ACT_NONE)
             elif op[0] == "pool5":

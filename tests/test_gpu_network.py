@@ -47,6 +47,16 @@ def test_chained_yolov5s_shaped_network_small_input():
     again = net.outputs()
     for name in ("o3", "o4", "o5"):
         assert np.array_equal(again[name], got[name])
+    # the runs above add the seven bottleneck shortcuts inside the convolutions; separate adds give the same bits
+    assert sum(op[0] == "convres" for op in net.ops) == 7 and len(net.unfused) == 0
+    plain = GpuNet(gu.ctx(), N, H0, H0, k=4, seed=3, fuse_residual=False)
+    plain.set_input(synth.round_like(x, "bf16"))
+    plain.run()
+    torch.cuda.synchronize()
+    sep = plain.outputs()
+    for name in ("o3", "o4", "o5"):
+        assert np.array_equal(sep[name], got[name]), name
+    plain.close()
     net.close()
 
 

@@ -2,7 +2,9 @@
 against the CPU oracle (convolution without activation, then its element-wise add + activation) and, bit for bit for
 act none and ReLU, against the library's own two-call form; on uncut tiles, tiles shared out over a cluster (split K),
 the element-store form of ragged filter counts, a channel slice of a wider tensor, stride 2, both 16-bit types, and
-with the output aliasing the residual.  Calls the tensor path cannot take must be declined, not computed elsewhere."""
+with the output aliasing the residual; and the other order, y = round(act(conv + bias)) + residual, bit for bit
+against the two-call form for every activation.  Calls the tensor path cannot take must be declined, not computed
+elsewhere."""
 import numpy as np
 import pytest
 import torch
@@ -120,4 +122,46 @@ def test_residual_is_declined_off_the_tensor_path():
     with pytest.raises(rt.RtossError) as e:
         c.rtoss_conv3x3_pattern(packed, x, y, 1, 8, 8, 1, rt.NHWC, rt.ACT_RELU, None, residual=r)
     assert e.value.status == rt.ERR_UNSUPPORTED
+    packed.close()
+
+
+POST_CASES = [
+    # ksize, Cin, Cout, N, H, W, stride, act, (y_off, y_stride), dtype: the residual behind the activation
+    (3, 32, 32, 2, 40, 40, 1, "silu", (0, 0), "bf16"),         # narrow 3x3: the filters are repeated down the lanes
+    (3, 64, 64, 1, 23, 31, 1, "silu", (0, 0), "bf16"),
+    (3, 128, 128, 2, 40, 40, 1, "silu", (0, 0), "f16"),
+    (3, 128, 128, 1, 24, 24, 2, "relu", (128, 384), "bf16"),
+    (3, 256, 256, 1, 13, 17, 1, "silu", (0, 0), "bf16"),       # split K over a cluster
+    (3, 320, 100, 1, 9, 11, 1, "silu", (0, 0), "bf16"),        # split K, element stores
+    (3, 96, 100, 1, 17, 18, 1, "silu", (0, 0), "bf16"),        # element stores
+    (1, 256, 256, 2, 20, 28, 1, "silu", (0, 0), "bf16"),
+    (1, 2048, 512, 1, 7, 9, 1, "none", (0, 0), "bf16"),
+]
+
+
+@pytest.mark.parametrize("ksize,cin,cout,N,H,W,stride,act,ysl,dt", POST_CASES)
+def test_residual_behind_the_activation(ksize, cin, cout, N, H, W, stride, act, ysl, dt):
+    """y = round(act(conv + bias)) + residual: against the oracle (its convolution with the activation, then its add
+    without one) and, bit for bit for every activation, against the library's two-call form."""
+    _, b, x, res, packed, wd, (Ho, Wo, Cs) = _setup(ksize, cin, cout, N, H, W, stride, ysl, dt)
+    a = {"none": orc.ACT_NONE, "relu": orc.ACT_RELU, "silu": orc.ACT_SILU}[act]
+    conv = orc.conv3x3 if ksize == 3 else orc.conv1x1
+    ref = orc.add_act(conv(x, wd, b, stride, a, G.ORC_DT[dt]), res[:, ysl[0]:ysl[0] + cout], orc.ACT_NONE, G.ORC_DT[dt])
+    c = G.ctx()
+    fn = c.rtoss_conv3x3_pattern if ksize == 3 else c.rtoss_conv1x1_pattern
+    xd, bd, rd = G.to_dev(x, dt, "nhwc"), torch.from_numpy(b).cuda(), G.to_dev(res, dt, "nhwc")
+    sl = slice(ysl[0], ysl[0] + cout)
+    y = torch.full((N, Ho, Wo, Cs), 7.0, dtype=G.TORCH_DT[dt], device="cuda")
+    fn(packed, xd, y, N, H, W, stride, rt.NHWC, rt.ACT_NAMES[act], bd, ysl[0], ysl[1], rt.PATH_TENSOR, residual=rd,
+       residual_after_act=True)
+    torch.cuda.synchronize()
+    err = orc.rel_err(G.from_dev(y, "nhwc")[:, sl], ref)
+    assert err <= G.TOL[dt], "relative error %g" % err
+    t = torch.zeros((N, Ho, Wo, Cs), dtype=G.TORCH_DT[dt], device="cuda")
+    fn(packed, xd, t, N, H, W, stride, rt.NHWC, rt.ACT_NAMES[act], bd, ysl[0], ysl[1], rt.PATH_TENSOR)
+    two = torch.empty_like(t)
+    rt.rtoss_add_act(t, rd, two, rt.ACT_NONE)
+    torch.cuda.synchronize()
+    assert torch.equal(two[..., sl], y[..., sl])
+    assert c.rtoss_device_status() == 0
     packed.close()
