@@ -4,10 +4,11 @@
 A step is one pass of the whole hot path over one batch of synthetic input:
 pattern selection (Algorithm 2 / 3 of arXiv 2303.02191), packing, and the
 pattern-sparse convolution, for each layer of the workload.  Default workload
-"layer128": batch 8, bf16 --
-  3x3 128->128 @80x80 with 3-entry patterns, the same layer with 2-entry
-  patterns, and a 1x1 256->128 @80x80 whose weights are regrouped into 3x3
-  blocks and pruned with the 3-entry patterns.
+"retinanet_b4": the RetinaNet ResNet-50-FPN-shaped stack (100 convolution calls
+on 68 weight tensors behind the 7x7 stem), batch 4 of 800x1088 frames, bf16,
+4-entry patterns -- the largest configuration that fits one GPU.  The smaller
+configurations ("layer32", "layer128", "yolov5s_b1", "yolov5s_b16") are measured
+in the same run with fewer steps and reported as sub-records under "others".
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
 """
 import argparse
@@ -46,7 +47,7 @@ def workload_layers(name):
 
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of a workload's dominant kernel from one
-# ncu capture (caches flushed before every pass; the commands are in profiles/conv_tc_layer128.md), valid
+# ncu capture (caches flushed before every pass; the command is recorded with the capture's summary), valid
 # for the kernel source whose hash is recorded with it: once conv_tc.cu changes the figure is withheld (null).
 # 13.5 MB = the activations and the weights once; the 13.1 MB of outputs are still dirty in the 126 MB L2 when the
 # kernel ends, so the capture sees no write.
@@ -136,6 +137,26 @@ def physical_gpu_index(local_rank):
 
 # --------------------------------------------------------------------------- CPU oracle legs
 
+_PREPARED = {}
+
+
+def oracle_inputs(layers_k, dtype, n_sample, seed=0):
+    """Seeded inputs of every layer for the oracle legs, generated once per (workload, sample size)."""
+    key = (id(layers_k), dtype, n_sample, seed)
+    if key not in _PREPARED:
+        from oracle import rtoss_oracle as orc
+        prepared = []
+        for (L, k, preset) in layers_k:
+            masks = orc.pattern_preset(k, orc.PRESET_CENTRE8 if preset == "centre8" else orc.PRESET_CONN4)
+            x = synth.round_like(synth.activations(seed, L["wid"], n_sample, L["cin"], L["H"], L["W"]), dtype)
+            w = synth.kaiming_weights(seed, L["wid"], L["cout"], L["cin"], L["ksize"])
+            b = synth.bias(seed, L["wid"], L["cout"])
+            prepared.append((L, k, masks, x, w, b))
+        _PREPARED.clear()   # one sample at a time is kept
+        _PREPARED[key] = prepared
+    return _PREPARED[key]
+
+
 def oracle_step(layers_k, dtype, n_sample, frac=1.0, seed=0):
     """One pass of the hot path in the CPU oracle on n_sample images.  With frac < 1 each convolution
     computes only the first ceil(frac*Cout) output channels (selection and packing always see the whole
@@ -144,11 +165,7 @@ def oracle_step(layers_k, dtype, n_sample, frac=1.0, seed=0):
     odt = {"f32": orc.DT_F32, "bf16": orc.DT_BF16, "f16": orc.DT_F16}[dtype]
     act = {"none": orc.ACT_NONE, "relu": orc.ACT_RELU, "silu": orc.ACT_SILU}
     prepared, done, full = [], 0.0, 0.0
-    for (L, k, preset) in layers_k:
-        masks = orc.pattern_preset(k, orc.PRESET_CENTRE8 if preset == "centre8" else orc.PRESET_CONN4)
-        x = synth.round_like(synth.activations(seed, L["wid"], n_sample, L["cin"], L["H"], L["W"]), dtype)
-        w = synth.kaiming_weights(seed, L["wid"], L["cout"], L["cin"], L["ksize"])
-        b = synth.bias(seed, L["wid"], L["cout"])
+    for (L, k, masks, x, w, b) in oracle_inputs(layers_k, dtype, n_sample, seed):
         cs = max(1, min(L["cout"], int(np.ceil(frac * L["cout"]))))
         fl = synth.layer_nnz_flops(L, 1, k)
         full += fl
@@ -209,7 +226,8 @@ def run_reference(args):
         "impl": "reference", "metric": "pattern-sparse conv images/sec", "value": value, "unit": "images/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
-        "config": {"workload": args.workload, "batch": N},
+        "config": {"workload": args.workload, "batch": N, "layout": "NCHW" if dtype == "f32" else "NHWC", "layers": len(layers_k),
+                   "l2": "not applicable (CPU oracle)", "multi_gpu": "rank 0 only", "launch": "host cores"},
         "cpu_baseline": {"value": value, "unit": "images/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -298,24 +316,14 @@ def run_network(args):
     ctx.close()
 
 
-def run_gpu(args):
+def measure_workload(ctx, rt, dev, name, steps, warmup, args, world, rank, full):
+    """One workload on this rank's GPU: the graph-replayed step (select + pack of every weight tensor, then every
+    convolution), the cold-L2 per-launch pass for the roofline, and -- with `full` -- the end-to-end leg through the
+    host-buffer entry point.  Returns a dict of raw figures (times of this rank; the caller reduces over ranks)."""
     import torch
     import torch.distributed as dist
-    from paper_2303_02191_b200 import binding as rt
-
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    dev = torch.device("cuda", local_rank)
-    ctx = rt.Context(local_rank)
     tdt = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}
-
-    N, dtype, layers_k = workload_layers(args.workload)
+    N, dtype, layers_k = workload_layers(name)
     elem = 4 if dtype == "f32" else 2
     cdt = rt.DTYPE_NAMES[dtype]
     preset_of = {"centre8": rt.PRESET_CENTRE8, "conn4": rt.PRESET_CONN4}
@@ -331,16 +339,18 @@ def run_gpu(args):
             b = torch.from_numpy(synth.bias(rank, L["wid"], L["cout"])).to(dev)
             n_k = L["cout"] * L["cin"] if L["ksize"] == 3 else (L["cout"] * L["cin"]) // 9
             pid = torch.empty(max(n_k, 1), dtype=torch.uint8, device=dev)
-            weights[L["wid"]] = dict(w=w, b=b, pid=pid, packed=None, masks=masks, k=k, ksize=L["ksize"])
+            weights[L["wid"]] = dict(w=w, b=b, pid=pid, packed=None, masks=masks, k=k, ksize=L["ksize"], n_k=n_k)
         Ho, Wo = synth.out_hw(L["H"], L["W"], L["stride"])
         xh = torch.from_numpy(synth.activations(rank, len(L_state), N, L["cin"], L["H"], L["W"])).to(tdt[dtype])
         yshape = (N, L["cout"], Ho, Wo)
         if layout == rt.NHWC:
             xh = xh.permute(0, 2, 3, 1).contiguous()
             yshape = (N, Ho, Wo, L["cout"])
-        st = dict(L=L, k=k, x=xh.to(dev), y=torch.empty(yshape, dtype=tdt[dtype], device=dev),
-                  xh=xh.pin_memory(), yh=torch.empty(yshape, dtype=tdt[dtype]).pin_memory(),
-                  Ho=Ho, Wo=Wo, wt=weights[L["wid"]], path=rt.PATH_FMA)
+        st = dict(L=L, k=k, x=xh.to(dev), y=torch.empty(yshape, dtype=tdt[dtype], device=dev), Ho=Ho, Wo=Wo,
+                  wt=weights[L["wid"]], path=rt.PATH_FMA)
+        if full:
+            st["xh"] = xh.pin_memory()
+            st["yh"] = torch.empty(yshape, dtype=tdt[dtype]).pin_memory()
         L_state.append(st)
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)   # larger than the 126 MB L2
 
@@ -391,14 +401,15 @@ def run_gpu(args):
     torch.cuda.synchronize()
     if ctx.rtoss_device_status() != 0:
         raise SystemExit("a device-side wait of the tensor path ran out")
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(max(warmup, 3)):
         step()
         flush.zero_()
     barrier()
 
-    # The step is launch-bound when driven call by call from Python (about twenty small launches for
-    # ~100 us of GPU work), so the timed region replays it as ONE CUDA graph, as a deployment would.
+    # The step is launch-bound when driven call by call from Python, so the timed region replays it as ONE CUDA
+    # graph, as a deployment would.
     graph = None
+    launches_per_step = 0
     if args.graph:
         try:
             side = torch.cuda.Stream()
@@ -416,12 +427,12 @@ def run_gpu(args):
             sys.stderr.write("graph capture failed, timing eager launches: %r\n" % (err,))
             graph = None
             torch.cuda.synchronize()
-    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler = ClockSampler(physical_gpu_index(int(os.environ.get("LOCAL_RANK", "0"))))
     sampler.start()
-    step_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    step_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     launches = 0
     barrier()
-    for s in range(args.steps):
+    for s in range(steps):
         flush.zero_()                       # L2 flush between timed iterations, outside the step's events
         step_ev[s][0].record()
         if graph is not None:
@@ -431,124 +442,233 @@ def run_gpu(args):
             launches += step()
         step_ev[s][1].record()
     barrier()
-    step_ms = np.array([a.elapsed_time(b) for a, b in step_ev])
-    total_ms = float(step_ms.sum())
+    total_ms = float(np.array([a.elapsed_time(b) for a, b in step_ev]).sum())
 
-    # Per-kernel durations for the roofline: the same K steps again, every convolution between its own pair of
-    # events right after a 256 MB flush write (cold L2).  The pass is captured once into a CUDA graph whose event
-    # records are graph nodes (external events) and replayed K times, so the host's enqueue time cannot leak into
-    # an interval; if the capture is not available the launches are issued one by one (the flush write queued
-    # before each launch then keeps the GPU busy while the host enqueues it).
-    conv_ms = None
+    # Per-launch durations for the roofline: the same K steps again, the whole-model select + pack and every
+    # convolution each between its own pair of events right after a 256 MB flush write (cold L2).  The pass is
+    # captured once into a CUDA graph whose event records are graph nodes (external events) and replayed K times,
+    # so the host's enqueue time cannot leak into an interval; if the capture is not available the launches are
+    # issued one by one (the flush write queued before each launch then keeps the GPU busy while the host enqueues).
+    conv_ms, prune_ms = None, None
     if args.graph:
         try:
             gev = [(torch.cuda.Event(enable_timing=True, external=True), torch.cuda.Event(enable_timing=True, external=True))
-                   for _ in L_state]
+                   for _ in range(len(L_state) + 1)]
             kgraph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(kgraph):
+                flush.zero_()
+                gev[-1][0].record()
                 prune_weights()
+                gev[-1][1].record()
                 for i, st in enumerate(L_state):
                     flush.zero_()
                     conv(st, gev[i])
-            acc = np.zeros(len(L_state))
-            for s in range(args.steps):
+            acc = np.zeros(len(L_state) + 1)
+            for s in range(steps):
                 kgraph.replay()
                 torch.cuda.synchronize()
                 acc += np.array([a.elapsed_time(b) for a, b in gev])
-            conv_ms = acc / args.steps
+            conv_ms, prune_ms = acc[:-1] / steps, float(acc[-1] / steps)
         except Exception as err:
             sys.stderr.write("per-kernel timing graph not available, timing eager launches: %r\n" % (err,))
             torch.cuda.synchronize()
             conv_ms = None
     if conv_ms is None:
-        conv_ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in L_state]
-                   for _ in range(args.steps)]
-        for s in range(args.steps):
+        conv_ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(len(L_state) + 1)]
+                   for _ in range(steps)]
+        for s in range(steps):
+            flush.zero_()
+            conv_ev[s][-1][0].record()
             prune_weights()
+            conv_ev[s][-1][1].record()
             for i, st in enumerate(L_state):
                 flush.zero_()
                 conv(st, conv_ev[s][i])
         barrier()
-        conv_ms = np.array([[a.elapsed_time(b) for a, b in row] for row in conv_ev]).mean(axis=0)
+        allms = np.array([[a.elapsed_time(b) for a, b in row] for row in conv_ev]).mean(axis=0)
+        conv_ms, prune_ms = allms[:-1], float(allms[-1])
     barrier()
     clocks = sampler.stop()
 
-    # ---- end to end through the host-buffer entry point (pinned host tensors, copies inside the timed region)
-    torch.cuda.synchronize()
-    h2d = sum(st["xh"].numel() * elem for st in L_state)
-    d2h = sum(st["yh"].numel() * elem for st in L_state)
-    e2e_steps = max(2, min(args.steps, 20, int(2e10 / (h2d + d2h))))   # bounded: about 20 GB over PCIe at most
-    for st in L_state[:1]:
-        ctx.rtoss_conv_pattern_host(st["wt"]["packed"], st["xh"], st["yh"], N, st["L"]["H"], st["L"]["W"], st["L"]["stride"],
-                                    layout, rt.ACT_NAMES[st["L"]["act"]], st["wt"]["b"], path=st["path"])
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        prune_weights()
-        torch.cuda.synchronize()
-        for st in L_state:
-            L = st["L"]
-            ctx.rtoss_conv_pattern_host(st["wt"]["packed"], st["xh"], st["yh"], N, L["H"], L["W"], L["stride"], layout,
-                                        rt.ACT_NAMES[L["act"]], st["wt"]["b"], path=st["path"])
-    torch.cuda.synchronize()
-    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    res = dict(name=name, N=N, dtype=dtype, elem=elem, layout="NHWC" if layout == rt.NHWC else "NCHW", total_ms=total_ms,
+               steps=steps, launches=launches, graph=graph is not None, conv_ms=conv_ms, prune_ms=prune_ms, clocks=clocks,
+               layers=[st["L"] for st in L_state], ks=[st["k"] for st in L_state],
+               on_tc=[st["path"] == rt.PATH_TENSOR for st in L_state],
+               weights=[dict(n_k=wt["n_k"], k=wt["k"], ksize=wt["ksize"]) for wt in weights.values()], e2e_s=None)
 
-    total_ms, e2e_s = max_over_ranks([total_ms, e2e_s], dev, world)
+    # ---- end to end through the host-buffer entry point (pinned host tensors, copies inside the timed region)
+    if full:
+        torch.cuda.synchronize()
+        res["h2d"] = sum(st["xh"].numel() * elem for st in L_state)
+        res["d2h"] = sum(st["yh"].numel() * elem for st in L_state)
+        e2e_steps = max(2, min(steps, 20, int(2e10 / (res["h2d"] + res["d2h"]))))   # bounded: about 20 GB over PCIe at most
+        for st in L_state[:1]:
+            ctx.rtoss_conv_pattern_host(st["wt"]["packed"], st["xh"], st["yh"], N, st["L"]["H"], st["L"]["W"], st["L"]["stride"],
+                                        layout, rt.ACT_NAMES[st["L"]["act"]], st["wt"]["b"], path=st["path"])
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            prune_weights()
+            torch.cuda.synchronize()   # the host-buffer call runs on the context's own streams: packing must be complete
+            for st in L_state:
+                L = st["L"]
+                ctx.rtoss_conv_pattern_host(st["wt"]["packed"], st["xh"], st["yh"], N, L["H"], L["W"], L["stride"], layout,
+                                            rt.ACT_NAMES[L["act"]], st["wt"]["b"], path=st["path"])
+        torch.cuda.synchronize()
+        res["e2e_s"] = (time.perf_counter() - t0) / e2e_steps
+
+    torch.cuda.synchronize()
+    batch.close()
+    for wt in weights.values():
+        if wt["packed"] is not None:
+            wt["packed"].close()
+    del L_state, weights, flush
+    torch.cuda.empty_cache()
+    return res
+
+
+def roofline_of(res, hbm_peak, tc_peak, peak_kind):
+    """Roofline figures of one measured workload.  Per launch: T_roof = max(algorithmic bytes / HBM copy peak,
+    non-zero FLOP / peak of the pipe the kernel uses); the stack's fraction is sum(T_roof) / sum(T_measured) over the
+    cold-L2 per-launch pass; the dominant kernel (largest share of that pass) gets its own record."""
+    N, elem = res["N"], res["elem"]
+    flops = np.array([synth.layer_nnz_flops(L, N, k) for L, k in zip(res["layers"], res["ks"])])
+    bytes_ = np.array([synth.layer_bytes(L, N, k, elem) for L, k in zip(res["layers"], res["ks"])], dtype=np.float64)
+    pipe = np.array([tc_peak if tc else ALU_PEAK_TFLOPS for tc in res["on_tc"]]) * 1e12
+    t_pipe, t_hbm = flops / pipe, bytes_ / (hbm_peak * 1e9)
+    t_roof = np.maximum(t_pipe, t_hbm)
+    t_meas = res["conv_ms"] * 1e-3
+    stack_frac = float(t_roof.sum() / t_meas.sum())
+    # the dominant kernel shape: layers of one shape share a kernel configuration; the shape with the largest share
+    shape_of = lambda L: (L["ksize"], L["stride"], L["cin"], L["cout"], L["H"], L["W"])
+    share = {}
+    for i, L in enumerate(res["layers"]):
+        share.setdefault(shape_of(L), []).append(i)
+    top_shape = max(share, key=lambda sh: t_meas[share[sh]].sum())
+    idx = share[top_shape]
+    top = idx[int(np.argmax(t_meas[idx]))]
+    on_tc = res["on_tc"][top]
+    t_top = float(np.mean(t_meas[idx]))
+    if t_pipe[top] >= t_hbm[top]:
+        dom = {"bound": "tensor" if on_tc else "alu", "achieved": flops[top] / t_top / 1e12, "peak": pipe[top] / 1e12, "unit": "TFLOP/s",
+               "peak_kind": ("of %s (bf16 cuBLAS, sustained)" % peak_kind) if on_tc
+               else "nominal, not measured: 148 SM x 128 FMA lanes x 2 x 1.965 GHz"}
+    else:
+        dom = {"bound": "hbm", "achieved": bytes_[top] / t_top / 1e9, "peak": hbm_peak, "unit": "GB/s", "peak_kind": "of " + peak_kind}
+    dom["frac"] = dom["achieved"] / dom["peak"]
+    L = res["layers"][top]
+    dom["kernel"] = ("conv_tc_kernel " if on_tc else "conv_alu_kernel ") + L["name"] + " k=%d" % res["ks"][top]
+    dom["launches_of_this_shape"] = len(idx)
+    dom["share_of_cold_pass"] = float(t_meas[idx].sum() / t_meas.sum())
+    dom["kernel_ms"] = t_top * 1e3
+    dom["nnz_flop_per_launch"] = float(flops[top])
+    dom["algorithmic_bytes_per_launch"] = float(bytes_[top])
+    dom["traffic"] = ncu_traffic(res["name"], L["name"], res["ks"][top])
+    # whole-model selection + packing: 36 B read per kernel (nine fp32 weights), k values + the id + the order entry written
+    sp_bytes = float(sum(w["n_k"] * (36 + w["k"] * elem + (5 if w["ksize"] == 3 else 1)) for w in res["weights"]))
+    sp = {"kernels": int(sum(w["n_k"] for w in res["weights"])), "launches": 2 if any(w["ksize"] == 3 for w in res["weights"]) else 1,
+          "algorithmic_bytes": sp_bytes, "us": res["prune_ms"] * 1e3, "bound": "hbm",
+          "achieved_gbs": sp_bytes / (res["prune_ms"] * 1e-3) / 1e9, "peak_gbs": hbm_peak,
+          "frac": sp_bytes / (res["prune_ms"] * 1e-3) / 1e9 / hbm_peak,
+          "note": "cold L2; besides the algorithmic bytes the pass writes the tensor path's 9-tap weight expansion"}
+    tensor_share = float(t_roof[t_pipe >= t_hbm].sum() / t_roof.sum())
+    return dict(stack_frac=stack_frac, sum_roof_ms=float(t_roof.sum() * 1e3), sum_cold_ms=float(t_meas.sum() * 1e3),
+                tensor_share=tensor_share, dominant=dom, select_pack=sp, flops=flops, bytes=bytes_, t_roof=t_roof,
+                t_pipe=t_pipe, t_hbm=t_hbm)
+
+
+OTHER_WORKLOADS = ("layer32", "layer128", "yolov5s_b1", "yolov5s_b16")
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2303_02191_b200 import binding as rt
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+    ctx = rt.Context(local_rank)
+
+    res = measure_workload(ctx, rt, dev, args.workload, args.steps, args.warmup, args, world, rank, full=True)
+    total_ms, e2e_s = max_over_ranks([res["total_ms"], res["e2e_s"]], dev, world)
+    others = {}
+    if args.others and world == 1:
+        for name in OTHER_WORKLOADS:
+            if name != args.workload:
+                others[name] = measure_workload(ctx, rt, dev, name, min(args.steps, 20), 3, args, 1, rank, full=False)
 
     if rank == 0:
+        N, dtype = res["N"], res["dtype"]
         ms_per_step = total_ms / args.steps
         value = whole_job_value(N, world, ms_per_step)
-        flops = [synth.layer_nnz_flops(st["L"], N, st["k"]) for st in L_state]
-        bytes_ = [synth.layer_bytes(st["L"], N, st["k"], elem) for st in L_state]
-        top = int(np.argmax(conv_ms))
         hbm_peak, tc_peak, peak_kind = read_peaks()
-        t_top = conv_ms[top] * 1e-3
-        on_tc = L_state[top]["path"] == rt.PATH_TENSOR
-        pipe_peak = tc_peak if on_tc else ALU_PEAK_TFLOPS          # TFLOP/s of the pipe the kernel uses
-        pipe_t, hbm_t = flops[top] / (pipe_peak * 1e12), bytes_[top] / (hbm_peak * 1e9)
-        if pipe_t >= hbm_t:
-            roof = {"bound": "tensor" if on_tc else "alu", "achieved": flops[top] / t_top / 1e12, "peak": pipe_peak,
-                    "unit": "TFLOP/s",
-                    "peak_kind": ("of %s (bf16 cuBLAS, sustained)" % peak_kind) if on_tc
-                    else "derived: 148 SM x 128 FMA lanes x 2 x 1.965 GHz"}
-        else:
-            roof = {"bound": "hbm", "achieved": bytes_[top] / t_top / 1e9, "peak": hbm_peak, "unit": "GB/s",
-                    "peak_kind": "of " + peak_kind}
-        roof["frac"] = roof["achieved"] / roof["peak"]
-        roof["traffic"] = ncu_traffic(args.workload, L_state[top]["L"]["name"], L_state[top]["k"])
-        roof["kernel"] = ("conv_tc_kernel " if on_tc else "conv_alu_kernel ") + L_state[top]["L"]["name"] + " k=%d" % L_state[top]["k"]
-        roof["kernel_ms"] = float(conv_ms[top])
-        roof["nnz_flop_per_launch"] = flops[top]
-        roof["algorithmic_bytes_per_launch"] = bytes_[top]
+        rf = roofline_of(res, hbm_peak, tc_peak, peak_kind)
+        dom = rf["dominant"]
+        tensor_led = rf["tensor_share"] >= 0.5
+        roof = {
+            "bound": "tensor" if tensor_led else "hbm",
+            "frac": rf["stack_frac"],
+            # the stack's fraction expressed in the unit of the bound that holds most of the roofline time
+            "achieved": rf["stack_frac"] * (tc_peak if tensor_led else hbm_peak), "peak": tc_peak if tensor_led else hbm_peak,
+            "unit": "TFLOP/s" if tensor_led else "GB/s",
+            "peak_kind": "of %s (%s)" % (peak_kind, "bf16 cuBLAS, sustained" if tensor_led else "copy"),
+            "traffic": dom.pop("traffic"),
+            "definition": "stack figure: sum over launches of max(algorithmic bytes / HBM copy peak, non-zero FLOP / pipe peak) "
+                          "divided by the sum of the cold-L2 CUDA-event times of the same launches; 'achieved' = frac x peak; "
+                          "share of the roofline time that is tensor-bound: %.2f" % rf["tensor_share"],
+            "sum_roofline_ms": rf["sum_roof_ms"], "sum_cold_kernel_ms": rf["sum_cold_ms"],
+            "dominant_kernel": dom, "select_pack": rf["select_pack"],
+            "notes": ["both convolution paths multiply the pruned taps as zeros: a tensor-bound layer cannot exceed k/9 of its "
+                      "non-zero roofline",
+                      "the tensor path reads the 9-tap dense expansion of the weights (9/k x the packed bytes the roofline counts)",
+                      "the FMA-pipe peak is the nominal 148 x 128 x 2 x 1.965 GHz, not a measured one"],
+        }
         out = {
             "metric": "pattern-sparse conv images/sec", "value": value, "unit": "images/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
-            "config": {"workload": args.workload, "batch": N, "layout": "NHWC" if layout == rt.NHWC else "NCHW",
-                       "l2": "flushed between steps (256 MB write)", "layers": len(L_state), "multi_gpu": "replicas only",
-                       "launch": "one CUDA graph per step" if graph is not None else "eager",
-                       "tensor_path_layers": sum(1 for st in L_state if st["path"] == rt.PATH_TENSOR),
-                       "fma_path_layers": sum(1 for st in L_state if st["path"] == rt.PATH_FMA)},
-            "nnz_gflops_per_s": sum(flops) / (ms_per_step * 1e-3) / 1e9 * world,
-            "conv_ms": [float(v) for v in conv_ms] if len(conv_ms) <= 8 else None,
-            "conv_ms_sum": float(conv_ms.sum()),
-            "roofline": roof, "clocks": clocks,
-            "e2e": {"value": world * N / e2e_s, "unit": "images/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            "gpu_launches": launches,
+            "config": {"workload": args.workload, "batch": N, "layout": res["layout"], "layers": len(res["layers"]),
+                       "l2": "flushed between steps (256 MB write)", "multi_gpu": "replicas only",
+                       "launch": "one CUDA graph per step" if res["graph"] else "eager"},
+            "paths": {"tensor_path_layers": int(sum(res["on_tc"])), "fma_path_layers": int(len(res["on_tc"]) - sum(res["on_tc"]))},
+            "nnz_gflops_per_s": float(rf["flops"].sum()) / (ms_per_step * 1e-3) / 1e9 * world,
+            "conv_ms": [float(v) for v in res["conv_ms"]] if len(res["conv_ms"]) <= 8 else None,
+            "conv_ms_sum": float(res["conv_ms"].sum()),
+            "roofline": roof, "clocks": res["clocks"],
+            "e2e": {"value": world * N / e2e_s, "unit": "images/s", "h2d_bytes_per_step": res["h2d"], "d2h_bytes_per_step": res["d2h"]},
+            "gpu_launches": res["launches"],
         }
+        if others:
+            out["others"] = {}
+            for name, r in others.items():
+                orf = roofline_of(r, hbm_peak, tc_peak, peak_kind)
+                ms = r["total_ms"] / r["steps"]
+                d = orf["dominant"]
+                out["others"][name] = {
+                    "batch": r["N"], "dtype": r["dtype"], "steps": r["steps"], "ms_per_step": ms, "images_per_s": r["N"] / (ms * 1e-3),
+                    "nnz_gflops_per_s": float(orf["flops"].sum()) / (ms * 1e-3) / 1e9, "roofline_frac": orf["stack_frac"],
+                    "sum_roofline_ms": orf["sum_roof_ms"], "sum_cold_kernel_ms": orf["sum_cold_ms"],
+                    "dominant_kernel": {"kernel": d["kernel"], "bound": d["bound"], "frac": d["frac"], "kernel_ms": d["kernel_ms"]},
+                    "select_pack_us": orf["select_pack"]["us"], "select_pack_frac": orf["select_pack"]["frac"],
+                    "tensor_path_layers": int(sum(r["on_tc"])), "fma_path_layers": int(len(r["on_tc"]) - sum(r["on_tc"])),
+                    "clocks": r["clocks"], "gpu_launches": r["launches"]}
         if args.layers_csv:
             # per-layer table: cold-L2 kernel time next to the two roofline terms at non-zero FLOPs
             with open(args.layers_csv, "w") as f:
                 f.write("layer,ksize,cin,cout,H,W,stride,k,path,kernel_us,hbm_us,pipe_us,frac\n")
-                for st, ms, fl, by in zip(L_state, conv_ms, flops, bytes_):
-                    L = st["L"]
-                    tc = st["path"] == rt.PATH_TENSOR
-                    pipe_us = fl / ((tc_peak if tc else ALU_PEAK_TFLOPS) * 1e12) * 1e6
-                    hbm_us = by / (hbm_peak * 1e9) * 1e6
+                for L, k, tc, ms, hu, pu in zip(res["layers"], res["ks"], res["on_tc"], res["conv_ms"], rf["t_hbm"], rf["t_pipe"]):
                     f.write("%s,%d,%d,%d,%d,%d,%d,%d,%s,%.2f,%.2f,%.2f,%.3f\n" % (
-                        L["name"], L["ksize"], L["cin"], L["cout"], L["H"], L["W"], L["stride"], st["k"],
-                        "tensor" if tc else "fma", ms * 1e3, hbm_us, pipe_us, max(hbm_us, pipe_us) / (ms * 1e3)))
+                        L["name"], L["ksize"], L["cin"], L["cout"], L["H"], L["W"], L["stride"], k,
+                        "tensor" if tc else "fma", ms * 1e3, hu * 1e6, pu * 1e6, max(hu, pu) * 1e3 / ms))
         if args.cpu_baseline:
+            _, _, layers_k = workload_layers(args.workload)
             v_cpu, t_cpu, f_cpu, n_cpu, p_cpu = cpu_baseline_sample(layers_k, dtype, N, 15.0)
             out["cpu_baseline"] = {"value": v_cpu, "unit": "images/s", "cores": os.cpu_count(), "kind": "oracle",
                                    "sample": "%d image(s) of the batch of %d, the first %.3f of every layer's output channels, "
@@ -556,10 +676,6 @@ def run_gpu(args):
                                              % (n_cpu, N, f_cpu, p_cpu, t_cpu)}
         print(json.dumps(out))
     torch.cuda.synchronize()
-    batch.close()
-    for wt in weights.values():
-        if wt["packed"] is not None:
-            wt["packed"].close()
     ctx.close()
     if world > 1:
         dist.destroy_process_group()
@@ -568,10 +684,12 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="layer128")
+    ap.add_argument("--workload", default="retinanet_b4")
+    ap.add_argument("--no-others", dest="others", action="store_false",
+                    help="skip the sub-records of the other configurations (layer32, layer128, yolov5s_b1, yolov5s_b16)")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--no-graph", dest="graph", action="store_false", help="time eager launches instead of a CUDA graph")
     ap.add_argument("--path", default="auto", choices=["auto", "fma"], help="fma: keep every layer on the FMA path")

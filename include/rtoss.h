@@ -55,7 +55,7 @@ typedef enum {
 
 typedef enum {
     RTOSS_PATH_AUTO = 0,   /* tensor path where the call qualifies, FMA path otherwise */
-    RTOSS_PATH_FMA = 1,    /* gather of the k kept taps on the FP32 FMA pipes (any dtype, layout, stride) */
+    RTOSS_PATH_FMA = 1,    /* FP32 FMA pipes (any dtype, layout, stride); the pruned taps are multiplied as zeros */
     RTOSS_PATH_TENSOR = 2  /* masked dense implicit GEMM on tcgen05; RTOSS_ERR_UNSUPPORTED if the call does not qualify */
 } rtoss_path;
 
@@ -136,7 +136,7 @@ rtoss_status rtoss_pattern_usage(rtoss_ctx* ctx, const void* kernels_dev, rtoss_
                                  const uint16_t* masks_host, int P, int k, uint8_t* pid_scratch_dev, uint64_t* counts_dev,
                                  void* cuda_stream);
 
-/* Criterion 2, the cut (Section IV.B: "select the most used kernel pattern"): rank the candidates of a table by
+/* Criterion 2, the cut (Section IV.B: only the most frequently chosen patterns stay): rank the candidates of a table by
  * their usage counts -- most used first; equal counts: the numerically lower mask first -- and keep the best M.
  * order_host (P entries, may be NULL) receives the candidate indices in rank order; top_masks_host (M entries) the
  * kept masks in ascending numeric order, i.e. a table every other call accepts.  Host only.  How many to keep is
@@ -158,7 +158,7 @@ rtoss_status rtoss_pattern_table_derive(rtoss_ctx* ctx, const void* kernels_dev,
                                         uint16_t* top_masks_host, int* M_kept, uint16_t* cand_masks_host,
                                         uint64_t* cand_counts_host, int* P_candidates, void* cuda_stream);
 
-/* ---- packing (Section IV.C: "kernels with similar patterns are grouped") --- */
+/* ---- packing (Section IV.C, last sentence: kernels of like pattern are put together) --- */
 
 /* Build the packed form of one layer from its weights and pattern ids:
  *   val  [n_kernels*k]  kept weights, ascending tap order inside a kernel,
@@ -168,6 +168,9 @@ rtoss_status rtoss_pattern_table_derive(rtoss_ctx* ctx, const void* kernels_dev,
  *   filters by pattern id: perm[ci*Cout+i] = filter at position i,
  *   bucket_off[ci*(P+1)+p] = first position of pattern p (entry P = Cout).
  * n_kernels = Cout*Cin (ksize 3) or floor(Cout*Cin/9) (ksize 1).
+ * Precondition: every id in pid_dev is < P (what rtoss_select_patterns writes for the same table).  An id
+ * outside the table keeps none of its kernel's weights and its filter is left out of perm (the call stays
+ * inside its arrays; the result is then not a valid packed layer).
  * *out must be NULL or an existing handle.  NULL: a new handle is created and
  * its device memory allocated (RTOSS_ERR_ALLOC on failure).  Existing handle
  * of the same layer shape, P, k and dtype: it is re-packed in place without
@@ -246,6 +249,8 @@ void rtoss_batch_destroy(rtoss_batch* batch);
  *     RTOSS_ERR_UNSUPPORTED.
  *   - The first call on a device looks the array's address up (cudaGetSymbolAddress); make that first
  *     call outside any stream capture.
+ *   - w_pruned_dev may be w_dev itself (pruning in place, W <- W (.) mask); two different arrays that overlap
+ *     are refused with RTOSS_ERR_INVALID_ARG.
  *   - All calls on a device share the array and it keeps the last call's ids.  Each call overwrites
  *     what it reads, so nothing needs clearing, but two calls whose kernels overlap on the GPU (two
  *     streams, two host threads) race on it: keep calls on one device in stream order.
@@ -284,9 +289,11 @@ typedef struct {
 
 /* y[n,co,oy,ox] = act( bias[co] + sum_ci sum_{t in mask(pid[co,ci])}
  *                      w[co,ci,t] * x[n,ci,oy*s+r-1,ox*s+c-1] ),  t = 3r+c,
- * zero outside the image (padding 1); Ho = (H-1)/s+1, Wo = (W-1)/s+1.  Only
- * the k kept taps of each kernel are multiplied (the cost model of Section
- * II.B: work proportional to the non-zero weights).  x: N x Cin x H x W in the
+ * zero outside the image (padding 1); Ho = (H-1)/s+1, Wo = (W-1)/s+1.  The
+ * result is that of the k kept taps per kernel (the cost model of Section II.B
+ * counts the non-zero weights).  Both kernel families evaluate it over the
+ * dense-expanded weights, pruned taps as zeros: the sparsity saves weight
+ * bytes, not multiplications.  x: N x Cin x H x W in the
  * given layout, y: N x Cs x Ho x Wo with Cs = y_channel_stride (or Cout),
  * written at channels [offset, offset+Cout).  x and y must not overlap.  The
  * packed handle must come from rtoss_pack with ksize 3. */
@@ -315,7 +322,10 @@ rtoss_status rtoss_device_status(rtoss_ctx* ctx, int* code);
  * images whose copies and kernels overlap on three internal streams; pinned host memory is needed for
  * the copies to be asynchronous.
  * Uses (and grows on demand) the context's device workspace, so concurrent
- * calls on one context are not allowed.  bias_dev stays a device pointer. */
+ * calls on one context are not allowed.  bias_dev stays a device pointer.
+ * The kernels run on the context's own (non-blocking) streams, which are not ordered after the stream
+ * rtoss_pack was given: the handle's packing must have COMPLETED (synchronise that stream, or an event)
+ * before this call. */
 rtoss_status rtoss_conv_pattern_host(rtoss_ctx* ctx, const rtoss_packed* p, const void* x_host, void* y_host,
                                      const rtoss_conv_desc* desc);
 

@@ -180,22 +180,10 @@ void oracle_select_3x3(const float *w, int Cout, int Cin, const uint16_t *masks,
  * Cout*Cin - 9G left-over weights at the end of the list are pruned.
  */
 long oracle_select_1x1(const float *w, int Cout, int Cin, const uint16_t *masks, int P, uint8_t *pid1) {
-    long len = (long)Cout * Cin;
-    float *fl = (float *)malloc(sizeof(float) * (size_t)(len > 0 ? len : 1));
-    long n = 0;
-    for (int co = 0; co < Cout; ++co)
-        for (int ci = 0; ci < Cin; ++ci) fl[n++] = w[(long)co * Cin + ci];
-    long G = 0;
-    float *temp_array = (float *)malloc(sizeof(float) * (size_t)(len > 0 ? len : 1));
-    for (long i = 0; i < len; i += 9) {
-        if (len - i >= 9) {
-            for (int t = 0; t < 9; ++t) temp_array[9 * G + t] = fl[i + t];
-            ++G;
-        }
-    }
-    oracle_select_kernels(temp_array, G, masks, P, pid1);
-    free(temp_array);
-    free(fl);
+    /* w is [Cout][Cin] contiguous, so the filter-major flat list is w itself: weight e = co*Cin + ci.
+     * Run g is w[9g .. 9g+8], already in the order of a row-major 3x3; only full runs are selected on. */
+    const long G = ((long)Cout * Cin) / 9;
+    oracle_select_kernels(w, G, masks, P, pid1);
     return G;
 }
 

@@ -276,7 +276,7 @@ rtoss_status rtoss_batch_select_pack(rtoss_ctx* ctx, const rtoss_batch* b, void*
         set_err(ctx, "null batch or batch of another device");
         return RTOSS_ERR_INVALID_ARG;
     }
-    cudaSetDevice(ctx->device);
+    rtoss_device_guard on_device(ctx->device);   // the caller's current device comes back when the call returns
     cudaStream_t s = (cudaStream_t)cuda_stream;
     cudaError_t e = cudaSuccess;
     const unsigned cap = (unsigned)ctx->sm_count * 8u;

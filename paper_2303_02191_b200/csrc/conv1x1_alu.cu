@@ -10,6 +10,8 @@
 // weights with a uniform branch per (filter, channel) was measured and lost: a
 // branch every 16-32 FMAs costs more than the zeros it avoids.  This is the
 // path for fp32 and for what the tensor path does not take.
+#include <atomic>
+
 #include "conv_common.cuh"
 
 namespace {
@@ -222,13 +224,15 @@ int rtoss_launch_conv1x1(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     dim3 grid((unsigned)((size_t)a.tiles * a.N), (unsigned)((a.Cout + kCoBlock - 1) / kCoBlock));
     cudaStream_t s = (cudaStream_t)stream;
     const int smem = (int)sizeof(float) * kCiChunk * (kXPitch + kCoBlock);
-    static bool attr_set = false;
-    if (!attr_set) {
+    // the attribute belongs to the (function, device) pair: one flag per device
+    static std::atomic<bool> attr_set[64];
+    const int dev_slot = ctx->device >= 0 && ctx->device < 64 ? ctx->device : -1;
+    if (dev_slot < 0 || !attr_set[dev_slot].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(conv1x1_alu_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(conv1x1_alu_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(conv1x1_alu_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return (int)e;
-        attr_set = true;
+        if (dev_slot >= 0) attr_set[dev_slot].store(true, std::memory_order_release);
     }
     switch (d->io_dtype) {
         case RTOSS_F32: rtoss_dev::launch_pdl(conv1x1_alu_kernel<float>, grid, kThreads, smem, s, a); break;

@@ -10,8 +10,8 @@
 // Shape of the kernel
 //   * A CTA owns a spatial tile of one image and a block of WARPS*CO_T output
 //     channels.  All warps share the staged input tile; warp w owns CO_T
-//     consecutive filters, so the weights and the pattern a warp works on are
-//     warp-uniform (one broadcast shared-memory read, uniform branches).
+//     consecutive filters, so the weights a warp works on are warp-uniform
+//     (one broadcast shared-memory read; no branch depends on the pattern).
 //   * Inside a warp, lane (lx,ly) of an LX x LY arrangement (LX*LY <= 32, picked
 //     per layer by the host to waste the fewest lanes and pixels) owns a patch
 //     of PH x PW output pixels and keeps its (PH-1)S+3 x (PW-1)S+3 input window

@@ -50,6 +50,7 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
+#include <atomic>
 #include <cstring>
 
 #include "conv_common.cuh"
@@ -1334,13 +1335,16 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     const size_t smem = (size_t)(plan.smem > 116 * 1024 ? plan.smem : 116 * 1024);
     const size_t n_tiles = (size_t)d->N * a.tiles_y * a.tiles_x * a.co_tiles * a.KS;
     dim3 grid((unsigned)(n_tiles < (size_t)sms ? n_tiles : (size_t)sms));
-    static bool attr_set = false;  // both instantiations may use up to the whole shared memory of an SM
-    if (!attr_set) {
+    // both instantiations may use up to the whole shared memory of an SM; the attribute belongs to the
+    // (function, device) pair, so there is one flag per device
+    static std::atomic<bool> attr_set[64];
+    const int dev_slot = ctx->device >= 0 && ctx->device < 64 ? ctx->device : -1;
+    if (dev_slot < 0 || !attr_set[dev_slot].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(conv_tc_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return (int)e;
-        attr_set = true;
+        if (dev_slot >= 0) attr_set[dev_slot].store(true, std::memory_order_release);
     }
     cudaError_t le;
     if (a.KS > 1) {

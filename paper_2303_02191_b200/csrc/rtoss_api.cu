@@ -102,6 +102,13 @@ int dispatch_conv(rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y,
 
 }  // namespace
 
+rtoss_device_guard::rtoss_device_guard(int device) : prev(device), switched(false) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != device) switched = cudaSetDevice(device) == cudaSuccess;
+}
+rtoss_device_guard::~rtoss_device_guard() {
+    if (switched) cudaSetDevice(prev);
+}
+
 extern "C" {
 
 rtoss_status rtoss_create(int device, rtoss_ctx** out) {
@@ -176,7 +183,7 @@ rtoss_status rtoss_select_patterns(rtoss_ctx* ctx, const void* w_dev, rtoss_dtyp
         return RTOSS_ERR_ALIGNMENT;
     }
     const int64_t n = ksize == 3 ? (int64_t)Cout * Cin : ((int64_t)Cout * Cin) / 9;
-    cudaSetDevice(ctx->device);
+    rtoss_device_guard on_device(ctx->device);   // the caller's current device comes back when the call returns
     int e = rtoss_launch_select(w_dev, w_dtype, n, make_table(masks_host, P), P, pid_dev, cuda_stream);
     return e ? cuda_fail(ctx, "select launch", e) : RTOSS_OK;
 }
@@ -200,7 +207,7 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
         set_err(ctx, "pack", "weights must be 16-byte aligned");
         return RTOSS_ERR_ALIGNMENT;
     }
-    cudaSetDevice(ctx->device);
+    rtoss_device_guard on_device(ctx->device);   // the caller's current device comes back when the call returns
     cudaStream_t s = (cudaStream_t)cuda_stream;
     cudaError_t e = cudaSuccess;
     rtoss_packed* p = *out;
@@ -287,7 +294,7 @@ rtoss_status rtoss_pattern_usage(rtoss_ctx* ctx, const void* kernels_dev, rtoss_
         set_err(ctx, "pattern usage", "kernels must be 16-byte aligned");
         return RTOSS_ERR_ALIGNMENT;
     }
-    cudaSetDevice(ctx->device);
+    rtoss_device_guard on_device(ctx->device);   // the caller's current device comes back when the call returns
     cudaStream_t s = (cudaStream_t)cuda_stream;
     cudaError_t e = cudaMemsetAsync(counts_dev, 0, sizeof(uint64_t) * (size_t)P, s);
     if (e != cudaSuccess) return cuda_fail(ctx, "pattern usage", (int)e);
@@ -345,7 +352,7 @@ rtoss_status rtoss_packed_info_get(const rtoss_packed* p, rtoss_packed_info* inf
 rtoss_status rtoss_packed_export(rtoss_ctx* ctx, const rtoss_packed* p, uint8_t* pid_host, void* val_host,
                                  uint32_t* perm_host, uint32_t* bucket_off_host, void* cuda_stream) {
     if (!ctx || !p) return RTOSS_ERR_INVALID_ARG;
-    cudaSetDevice(p->device);
+    rtoss_device_guard on_device(p->device);   // the caller's current device comes back when the call returns
     cudaStream_t s = (cudaStream_t)cuda_stream;
     cudaError_t e = cudaSuccess;
     if (pid_host && p->n_kernels > 0) e = cudaMemcpyAsync(pid_host, p->pid, (size_t)p->n_kernels, cudaMemcpyDeviceToHost, s);
@@ -363,7 +370,7 @@ rtoss_status rtoss_packed_export(rtoss_ctx* ctx, const rtoss_packed* p, uint8_t*
 
 rtoss_status rtoss_packed_to_dense(rtoss_ctx* ctx, const rtoss_packed* p, void* w_masked_dev, void* cuda_stream) {
     if (!ctx || !p || !w_masked_dev) return RTOSS_ERR_INVALID_ARG;
-    cudaSetDevice(p->device);
+    rtoss_device_guard on_device(p->device);   // the caller's current device comes back when the call returns
     int e = rtoss_launch_to_dense(p, w_masked_dev, cuda_stream);
     return e ? cuda_fail(ctx, "to_dense launch", e) : RTOSS_OK;
 }
@@ -388,7 +395,7 @@ rtoss_status rtoss_conv3x3_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const 
                                    const rtoss_conv_desc* desc, void* cuda_stream) {
     rtoss_status st = check_conv(ctx, p, x_dev, y_dev, desc, 3, true);
     if (st != RTOSS_OK) return st;
-    cudaSetDevice(ctx->device);
+    rtoss_device_guard on_device(ctx->device);   // the caller's current device comes back when the call returns
     int e = dispatch_conv(ctx, p, x_dev, y_dev, desc, cuda_stream, &st);
     if (st != RTOSS_OK) return st;
     return e ? cuda_fail(ctx, "conv3x3 launch", e) : RTOSS_OK;
@@ -398,7 +405,7 @@ rtoss_status rtoss_conv1x1_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const 
                                    const rtoss_conv_desc* desc, void* cuda_stream) {
     rtoss_status st = check_conv(ctx, p, x_dev, y_dev, desc, 1, true);
     if (st != RTOSS_OK) return st;
-    cudaSetDevice(ctx->device);
+    rtoss_device_guard on_device(ctx->device);   // the caller's current device comes back when the call returns
     int e = dispatch_conv(ctx, p, x_dev, y_dev, desc, cuda_stream, &st);
     if (st != RTOSS_OK) return st;
     return e ? cuda_fail(ctx, "conv1x1 launch", e) : RTOSS_OK;
@@ -406,7 +413,7 @@ rtoss_status rtoss_conv1x1_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const 
 
 rtoss_status rtoss_device_status(rtoss_ctx* ctx, int* code) {
     if (!ctx || !code) return RTOSS_ERR_INVALID_ARG;
-    cudaSetDevice(ctx->device);
+    rtoss_device_guard on_device(ctx->device);   // the caller's current device comes back when the call returns
     cudaError_t e = cudaDeviceSynchronize();
     if (e == cudaSuccess) e = cudaMemcpy(code, ctx->dev_status, sizeof(int), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail(ctx, "device status", (int)e);
@@ -427,7 +434,7 @@ rtoss_status rtoss_conv_pattern_host(rtoss_ctx* ctx, const rtoss_packed* p, cons
         set_err(ctx, "conv", "the host-buffer entry point takes no residual operand");
         return RTOSS_ERR_UNSUPPORTED;
     }
-    cudaSetDevice(ctx->device);
+    rtoss_device_guard on_device(ctx->device);   // the caller's current device comes back when the call returns
     const size_t es = rtoss_dtype_size(desc->io_dtype);
     const int Ho = (desc->H - 1) / desc->stride + 1, Wo = (desc->W - 1) / desc->stride + 1;
     const int cs = desc->y_channel_stride ? desc->y_channel_stride : p->Cout;

@@ -58,6 +58,18 @@ struct MaskTable {
 
 bool rtoss_table_ok(const uint16_t* masks, int P, int k);
 
+// Makes `device` current for the life of the object and gives the caller its own current device back afterwards:
+// an entry point must not leave another GPU selected behind the back of the caller (or of torch).  Defined in
+// rtoss_api.cu (host code, CUDA runtime).
+struct rtoss_device_guard {
+    explicit rtoss_device_guard(int device);
+    ~rtoss_device_guard();
+    rtoss_device_guard(const rtoss_device_guard&) = delete;
+    rtoss_device_guard& operator=(const rtoss_device_guard&) = delete;
+    int prev;
+    bool switched;
+};
+
 static inline size_t rtoss_dtype_size(rtoss_dtype d) { return d == RTOSS_F32 ? 4 : 2; }
 
 // Layout of the tensor path's dense-expanded weights wtc[tap][row][ci].  Normally row = filter (rows = Cout).  A

@@ -71,6 +71,8 @@ __device__ __forceinline__ void pack_one(const float (&w)[9], unsigned m, int64_
 // Stable counting sort of the Cout filters of input channel ci by pattern id, by one warp: perm[ci*Cout + j] lists
 // the filters by ascending id (ties by ascending filter), bucket_off[ci*(P+1) + p] is where pattern p starts.
 // Ranks inside a group of 32 filters come from __match_any_sync; `fill` is 256 words of shared memory of this warp.
+// Ids must be < P; a filter whose id is not is left out of perm (the channel's list is then short by it, the last
+// bucket ends before bucket_off's closing entry Cout) rather than written past the channel's slice.
 __device__ __forceinline__ void order_channel(const uint8_t* __restrict__ pid, int Cout, int Cin, int P, int ci,
                                               uint32_t* __restrict__ perm, uint32_t* __restrict__ bucket_off,
                                               uint32_t* fill, int lane) {
@@ -79,9 +81,10 @@ __device__ __forceinline__ void order_channel(const uint8_t* __restrict__ pid, i
     // pass 1: histogram
     for (int base = 0; base < Cout; base += 32) {
         const int co = base + lane;
-        const unsigned key = co < Cout ? pid[(size_t)co * Cin + ci] : 0xFFFFu;
+        unsigned key = co < Cout ? pid[(size_t)co * Cin + ci] : 0xFFFFu;
+        if (key >= (unsigned)P) key = 0xFFFFu;   // an id outside the table is not placed (nothing is written for it)
         const unsigned peers = __match_any_sync(0xFFFFFFFFu, key);
-        if (co < Cout && lane == __ffs(peers) - 1) fill[key] += __popc(peers);
+        if (key != 0xFFFFu && lane == __ffs(peers) - 1) fill[key] += __popc(peers);
         __syncwarp();
     }
     // exclusive scan over the P buckets (P <= 255: eight per lane, then a warp scan of lane totals)
@@ -114,12 +117,13 @@ __device__ __forceinline__ void order_channel(const uint8_t* __restrict__ pid, i
     // pass 2: placement, filters in ascending order inside each bucket
     for (int base = 0; base < Cout; base += 32) {
         const int co = base + lane;
-        const unsigned key = co < Cout ? pid[(size_t)co * Cin + ci] : 0xFFFFu;
+        unsigned key = co < Cout ? pid[(size_t)co * Cin + ci] : 0xFFFFu;
+        if (key >= (unsigned)P) key = 0xFFFFu;
         const unsigned peers = __match_any_sync(0xFFFFFFFFu, key);
         const unsigned before = peers & ((1u << lane) - 1u);
-        if (co < Cout) perm[(size_t)ci * Cout + fill[key] + __popc(before)] = (uint32_t)co;
+        if (key != 0xFFFFu) perm[(size_t)ci * Cout + fill[key] + __popc(before)] = (uint32_t)co;
         __syncwarp();
-        if (co < Cout && before == 0) fill[key] += __popc(peers);
+        if (key != 0xFFFFu && before == 0) fill[key] += __popc(peers);
         __syncwarp();
     }
 }

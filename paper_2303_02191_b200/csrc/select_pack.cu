@@ -1,6 +1,7 @@
 // Pattern selection (Algorithm 2 / Algorithm 3 of arXiv 2303.02191) and the
 // packing kernels.  All three are bandwidth-bound streaming passes over the
 // weights: 9 values read per kernel, one byte (pid) or k values written.
+#include <atomic>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -231,9 +232,11 @@ namespace {
 
 // Dense masked weights straight from the weights and the pattern ids: out[e] = w[e] if position e is
 // kept by the pattern of its kernel (or run of nine), else +0.
+// w and out may be the same array (pruning in place): a thread reads element e and writes element e, nothing else,
+// so neither pointer is declared restrict.
 template <typename T>
-__global__ void mask_dense_kernel(const T* __restrict__ w, const uint8_t* __restrict__ pid, MaskTable table,
-                                  int64_t n_kernels, int64_t n_dense, T* __restrict__ out) {
+__global__ void mask_dense_kernel(const T* w, const uint8_t* __restrict__ pid, MaskTable table,
+                                  int64_t n_kernels, int64_t n_dense, T* out) {
     rtoss_dev::pdl_enter();
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n_dense; e += (int64_t)gridDim.x * blockDim.x) {
         const int64_t g = e / 9;
@@ -248,7 +251,7 @@ __global__ void mask_dense_kernel(const T* __restrict__ w, const uint8_t* __rest
 // handle for the runtime, never a pointer a kernel could use: the address has to be asked for, once
 // per device, with that device current.
 unsigned char* static_pid_address(cudaError_t* err) {
-    static unsigned char* cached[64] = {nullptr};
+    static std::atomic<unsigned char*> cached[64];   // two host threads may ask at once: both store the same address
     int dev = -1;
     *err = cudaGetDevice(&dev);
     if (*err != cudaSuccess) return nullptr;
@@ -256,13 +259,15 @@ unsigned char* static_pid_address(cudaError_t* err) {
         *err = cudaErrorInvalidDevice;
         return nullptr;
     }
-    if (!cached[dev]) {
+    unsigned char* at = cached[dev].load(std::memory_order_acquire);
+    if (!at) {
         void* p = nullptr;
         *err = cudaGetSymbolAddress(&p, g_static_pid);
         if (*err != cudaSuccess) return nullptr;
-        cached[dev] = static_cast<unsigned char*>(p);
+        at = static_cast<unsigned char*>(p);
+        cached[dev].store(at, std::memory_order_release);
     }
-    return cached[dev];
+    return at;
 }
 
 }  // namespace
@@ -279,6 +284,12 @@ extern "C" rtoss_status rtoss_prune_dense_static(const void* w_dev, rtoss_dtype 
     const int64_t total = (int64_t)Cout * Cin;
     const int64_t n_kernels = ksize == 3 ? total : total / 9;
     if (n_kernels > (int64_t)kStaticPidBytes) return RTOSS_ERR_UNSUPPORTED;  // more kernels than the fixed array holds
+    {
+        // in place (same array) is fine; two different arrays that overlap are not
+        const size_t bytes = (size_t)(ksize == 3 ? total * 9 : total) * rtoss_dtype_size(w_dtype);
+        const uintptr_t a = reinterpret_cast<uintptr_t>(w_dev), b = reinterpret_cast<uintptr_t>(w_pruned_dev);
+        if (a != b && a < b + bytes && b < a + bytes) return RTOSS_ERR_INVALID_ARG;
+    }
     cudaError_t ce;
     unsigned char* pid = static_pid_address(&ce);
     if (!pid) return RTOSS_ERR_CUDA;
@@ -292,20 +303,21 @@ extern "C" rtoss_status rtoss_prune_dense_static(const void* w_dev, rtoss_dtype 
     const int threads = 256;
     const int grid = grid_for((n_dense + threads - 1) / threads);
     cudaStream_t s = (cudaStream_t)cuda_stream;
+    cudaError_t le = cudaSuccess;   // this launch's own result (not the thread's last error, which may be older)
     switch (w_dtype) {
         case RTOSS_F32:
-            rtoss_dev::launch_pdl(mask_dense_kernel<float>, grid, threads, 0, s, (const float*)w_dev, pid, table, n_kernels, n_dense, (float*)w_pruned_dev);
+            le = rtoss_dev::launch_pdl(mask_dense_kernel<float>, grid, threads, 0, s, (const float*)w_dev, pid, table, n_kernels, n_dense, (float*)w_pruned_dev);
             break;
         case RTOSS_BF16:
-            rtoss_dev::launch_pdl(mask_dense_kernel<__nv_bfloat16>, grid, threads, 0, s, (const __nv_bfloat16*)w_dev, pid, table, n_kernels, n_dense,
-                                                                      (__nv_bfloat16*)w_pruned_dev);
+            le = rtoss_dev::launch_pdl(mask_dense_kernel<__nv_bfloat16>, grid, threads, 0, s, (const __nv_bfloat16*)w_dev, pid, table, n_kernels, n_dense,
+                                       (__nv_bfloat16*)w_pruned_dev);
             break;
         case RTOSS_F16:
-            rtoss_dev::launch_pdl(mask_dense_kernel<__half>, grid, threads, 0, s, (const __half*)w_dev, pid, table, n_kernels, n_dense,
-                                                               (__half*)w_pruned_dev);
+            le = rtoss_dev::launch_pdl(mask_dense_kernel<__half>, grid, threads, 0, s, (const __half*)w_dev, pid, table, n_kernels, n_dense,
+                                       (__half*)w_pruned_dev);
             break;
     }
-    return cudaGetLastError() == cudaSuccess ? RTOSS_OK : RTOSS_ERR_CUDA;
+    return le == cudaSuccess ? RTOSS_OK : RTOSS_ERR_CUDA;
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -318,3 +318,34 @@ def test_pattern_table_derivation_matches_oracle(k, preset, M):
     w = synth.kaiming_weights(6, 2, 16, 8, 3)
     pid = gu.ctx().rtoss_select_patterns(torch.from_numpy(w).cuda(), 3, top, k)
     assert np.array_equal(pid.cpu().numpy().ravel(), orc.select_3x3(w, want_top).ravel())
+
+
+def test_pack_with_ids_outside_the_table_stays_inside_its_arrays():
+    """rtoss_pack's precondition is pid < P.  Ids that break it (here: ids chosen with a larger table) must not make the
+    ordering pass write outside the channel's slice of perm: the other channels' slices and bucket offsets equal the
+    oracle's, the offending filters are simply not listed, and the device reports no fault."""
+    c = gu.ctx()
+    masks = orc.pattern_preset(3, orc.PRESET_CONN4)[:6]          # P = 6
+    Cout, Cin = 40, 24
+    w = synth.kaiming_weights(51, 1, Cout, Cin, 3)
+    pid_o = orc.select_3x3(w, masks)
+    bad = pid_o.copy()
+    bad[5, Cin - 1] = 9        # the last channel: the out-of-range slot would lie behind the end of perm
+    bad[17, Cin - 1] = 200
+    bad[3, 2] = 6              # an inner channel: the slot would lie in the next channel's slice
+    wd = torch.from_numpy(w).cuda()
+    packed = c.rtoss_pack(wd, 3, masks, 3, torch.from_numpy(bad).cuda().reshape(-1), rt.F32)
+    torch.cuda.synchronize()
+    ex = packed.export()
+    _, perm_o, off_o = orc.pack_3x3(w, masks, 3, pid_o, orc.DT_F32)
+    perm, off = ex["perm"].reshape(Cin, Cout), ex["bucket_off"].reshape(Cin, len(masks) + 1)
+    perm_o, off_o = perm_o.reshape(Cin, Cout), off_o.reshape(Cin, len(masks) + 1)
+    untouched = [ci for ci in range(Cin) if ci not in (2, Cin - 1)]
+    assert np.array_equal(perm[untouched], perm_o[untouched]) and np.array_equal(off[untouched], off_o[untouched])
+    for ci, dropped in ((2, {3}), (Cin - 1, {5, 17})):
+        n_ok = Cout - len(dropped)
+        listed = perm[ci][:n_ok]
+        assert sorted(listed.tolist()) == sorted(set(range(Cout)) - dropped)
+        assert off[ci][-1] == Cout and np.all(np.diff(off[ci][:-1].astype(np.int64)) >= 0)
+    assert c.rtoss_device_status() == 0
+    packed.close()

@@ -1,7 +1,8 @@
 """Tensor path on layers with few tiles and many channel blocks: the channel blocks of a tile are shared out to
-several CTAs (split K), every share leaves its partial sums, and each CTA finishes a part of the tile once all have arrived.  Parity against the CPU oracle,
-twice in a row on the same context (the arrival counters must be back at zero), with every activation, a channel
-slice of a wider output, a ragged filter count and both kernel sizes."""
+the CTAs of a thread-block cluster (split K); every CTA leaves its partial sums in the shared memory of the chunk's
+owner (distributed shared memory, between two cluster barriers) and finishes the chunks it owns.  Parity against the
+CPU oracle, twice in a row on the same context (nothing of the first call may linger), with every activation, a
+channel slice of a wider output, a ragged filter count and both kernel sizes."""
 import numpy as np
 import pytest
 import torch

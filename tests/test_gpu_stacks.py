@@ -1,6 +1,6 @@
 """Per-layer parity of the two model-shaped stacks, in the layout and path selection the benchmark uses
-(bf16, NHWC, automatic path): YOLOv5s-shaped layers in full at batch 1, RetinaNet-R50-FPN-shaped layers at
-the benchmark's batch 4 on sampled outputs (corners included)."""
+(bf16, NHWC, automatic path): YOLOv5s-shaped layers in full at batch 1 and on sampled outputs at the benchmark's
+batch 16, RetinaNet-R50-FPN-shaped layers at the benchmark's batch 4 on sampled outputs (corners included)."""
 import numpy as np
 import pytest
 import torch
@@ -37,15 +37,13 @@ def test_yolov5s_stack_every_unique_layer_full_tensor():
     assert worst <= 2e-2
 
 
-def test_retinanet_stack_unique_layers_batch4_sampled():
+def _sampled_stack(layers, N, seed, tid0, rng):
     masks = orc.pattern_preset(4, orc.PRESET_CENTRE8)
-    rng = np.random.default_rng(11)
-    N = 4
-    for i, L in enumerate(_unique(synth.retinanet_r50fpn_stack())):
+    for i, L in enumerate(_unique(layers)):
         ks, s, Cin, Cout, H, W = L["ksize"], L["stride"], L["cin"], L["cout"], L["H"], L["W"]
-        x = synth.round_like(synth.activations(41, 600 + i, N, Cin, H, W), "bf16")
-        w = synth.kaiming_weights(41, 600 + i, Cout, Cin, ks)
-        b = synth.bias(41, 600 + i, Cout)
+        x = synth.round_like(synth.activations(seed, tid0 + i, N, Cin, H, W), "bf16")
+        w = synth.kaiming_weights(seed, tid0 + i, Cout, Cin, ks)
+        b = synth.bias(seed, tid0 + i, Cout)
         pid_g, packed = gu.select_pack(w, ks, masks, 4, "bf16")
         pid_o, wd, _ = gu.oracle_weights(w, ks, masks, 4, "bf16")
         assert np.array_equal(pid_g, pid_o.ravel()), L["name"]
@@ -64,6 +62,15 @@ def test_retinanet_stack_unique_layers_batch4_sampled():
         packed.close()
         del x, y
     assert gu.ctx().rtoss_device_status() == 0
+
+
+def test_retinanet_stack_unique_layers_batch4_sampled():
+    _sampled_stack(synth.retinanet_r50fpn_stack(), 4, 41, 600, np.random.default_rng(11))
+
+
+def test_yolov5s_stack_unique_layers_batch16_sampled():
+    """The batch the benchmark times: the tile walk over sixteen images of every layer shape of the stack."""
+    _sampled_stack(synth.yolov5s_stack(), 16, 44, 700, np.random.default_rng(13))
 
 
 SWEEP_SUBSET = [(dt, C, HW, k) for dt in ("bf16", "f32") for C in (64, 256) for HW in (20, 40) for k in (2, 3, 4, 9)]

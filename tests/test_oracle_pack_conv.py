@@ -292,3 +292,23 @@ def test_glue_oracle_against_torch():
     silu = orc.add_act(x, y, orc.ACT_SILU, orc.DT_BF16)
     want = torch.from_numpy((s_ / (1 + np.exp(-s_))).astype(np.float32)).to(torch.bfloat16).float().numpy()
     assert (silu != want).mean() < 0.01
+
+
+def test_rel_err_on_hand_computed_cases():
+    """The metric every convolution verdict rests on: max |y - ref| / max(|ref|, rms(ref)).
+    ref = (6, -8, 0, 0): rms = sqrt((36 + 64) / 4) = 5 exactly.
+      y = (6.3, -8.8, 1, 0): 0.3 / 6 = 0.05, 0.8 / 8 = 0.1, 1 / max(0, 5) = 0.2 (the element below the floor decides),
+                             0 -> 0.2;
+      y = (6, -10, 0.5, 0):  0, 2 / 8 = 0.25 (an element above the floor decides), 0.5 / 5 = 0.1 -> 0.25.
+    A sum instead of the max in the denominator, the rms of y instead of ref's, a mean instead of the max over the
+    elements, or no floor at all each miss at least one of the two."""
+    ref = np.array([6.0, -8.0, 0.0, 0.0])
+    assert abs(orc.rel_err(np.array([6.3, -8.8, 1.0, 0.0]), ref) - 0.2) < 1e-12
+    assert abs(orc.rel_err(np.array([6.0, -10.0, 0.5, 0.0]), ref) - 0.25) < 1e-12
+    assert orc.rel_err(ref, ref) == 0.0
+    # shape does not matter, the floor is the rms of the whole reference tensor
+    assert abs(orc.rel_err(np.array([[6.3, -8.8], [1.0, 0.0]]), ref.reshape(2, 2)) - 0.2) < 1e-12
+    # the sampled-point form the large-layer tests spell out inline is the same formula
+    got, r = np.array([6.3, -8.8, 1.0, 0.0]), ref
+    rms = float(np.sqrt(np.mean(r ** 2)))
+    assert abs(np.max(np.abs(got - r) / np.maximum(np.abs(r), max(rms, 1e-30))) - 0.2) < 1e-12

@@ -2,9 +2,10 @@
 
 It serves callers that cannot call cudaMalloc (all device memory already given to their own arena, or
 no tolerance for cudaMalloc's device-wide synchronisation): the pattern ids live in a fixed array inside
-the library.  Checked here through the C ABI against the allocating chain select -> pack -> to_dense,
-bit for bit, on two calls in a row (the second must not see anything of the first in the shared array),
-for both kernel sizes, and the size limit must be refused.  Collected last on purpose."""
+the library.  Checked here through the C ABI against the allocating chain select -> pack -> to_dense
+and against the CPU oracle's W (.) mask, bit for bit, on consecutive calls (a call must not see anything of
+the one before in the shared array), for both kernel sizes, also in place (output = input); the size limit
+and overlapping arrays must be refused.  Collected last on purpose."""
 import numpy as np
 import pytest
 import torch
@@ -12,8 +13,18 @@ import torch
 pytestmark = pytest.mark.gpu
 
 if torch.cuda.is_available():
+    from oracle import rtoss_oracle as orc
     from paper_2303_02191_b200 import binding as rt
     from paper_2303_02191_b200 import synth
+
+
+def _oracle_pruned(w, ksize, masks):
+    """W (.) mask from the CPU oracle; w's values are exact in fp32 whatever its storage type."""
+    wf = w.float().cpu().numpy()
+    if ksize == 3:
+        return orc.mask_3x3(wf, masks, orc.select_3x3(wf, masks))
+    w2 = wf.reshape(wf.shape[0], wf.shape[1])
+    return orc.mask_1x1(w2, masks, orc.select_1x1(w2, masks)).reshape(wf.shape)
 
 
 def _chain(ctx, w, ksize, masks, k):
@@ -44,6 +55,13 @@ def test_static_pruning_matches_the_allocating_chain_twice_in_a_row():
         a = out.float().cpu().numpy().view(np.uint32)
         b = want.float().cpu().numpy().view(np.uint32)
         assert np.array_equal(a, b)
+        assert np.array_equal(a, _oracle_pruned(w, ksize, masks).view(np.uint32))
+        # in place: the output array is the input array
+        w2 = w.clone()
+        st, same = rt.rtoss_prune_dense_static(w2, ksize, masks, k, w2)
+        assert st == rt.OK
+        torch.cuda.synchronize()
+        assert np.array_equal(w2.float().cpu().numpy().view(np.uint32), b)
         kept = np.count_nonzero(out.float().cpu().numpy().reshape(-1))
         n_k = w.shape[0] * w.shape[1] if ksize == 3 else (w.shape[0] * w.shape[1]) // 9
         assert kept == n_k * k
@@ -61,3 +79,9 @@ def test_static_pruning_refuses_layers_beyond_its_fixed_array():
     assert st == rt.OK and not out.any()
     st, _ = rt.rtoss_prune_dense_static(ok, 3, [3, 3], 2, torch.empty_like(ok))  # duplicate mask
     assert st == 2
+    # two different arrays that overlap: refused before anything is launched
+    flat = torch.zeros(2 * 16 * 16 * 9 + 64, device="cuda")
+    a = flat[:16 * 16 * 9].view(16, 16, 3, 3)
+    b = flat[64:64 + 16 * 16 * 9].view(16, 16, 3, 3)
+    st, _ = rt.rtoss_prune_dense_static(a, 3, masks, 2, b)
+    assert st == 1
