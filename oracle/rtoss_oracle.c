@@ -4,7 +4,7 @@
  * A plain, slow, obviously-correct restatement of what the R-TOSS hot path
  * computes (arXiv 2303.02191): pattern table construction (Section IV.B,
  * Eq. 1 and criterion 1), per-kernel pattern selection (Section IV.C,
- * Algorithm 2), the 1x1 -> 3x3 regrouping (Section IV.D, Algorithm 3), mask
+ * Algorithm 2; and a block-shared variant of it), the 1x1 -> 3x3 regrouping (Section IV.D, Algorithm 3), mask
  * application (Section II.B, "semi-structured pruning"), a canonical packed
  * form of the pruned weights (Section IV.C, last sentence), the layer
  * grouping (Section IV.A, Algorithm 1) and the inference convolution over
@@ -185,6 +185,61 @@ long oracle_select_1x1(const float *w, int Cout, int Cin, const uint16_t *masks,
     const long G = ((long)Cout * Cin) / 9;
     oracle_select_kernels(w, G, masks, P, pid1);
     return G;
+}
+
+/* ---- selection with one pattern per block of kernels (a variant, not the paper's per-kernel rule) ---- */
+
+/*
+ * Section IV.C lets the kernels of a layer group take over one kernel mask; this variant applies that idea
+ * inside a layer: the kernels (co, ci) with co in a block of FB consecutive filters and ci in a block of CB
+ * consecutive input channels all get ONE pattern, the one that retains the most energy of the whole block.
+ * (It changes which weights survive, so it is a different pruning result from Algorithm 2; it exists because a
+ * pattern shared by a block lets a matrix unit skip the pruned taps of the whole block.)
+ *
+ *   q[co][ci][t]  = w*w rounded to float (as in Algorithm 2's restatement above), then widened to double
+ *   r[co][t]      = sum over the block's channels ci, ascending, in double
+ *   E[t]          = sum over the block's filters co, ascending, of r[co][t], in double
+ *   S_p           = sum over the taps t of mask p, ascending, of E[t], in double
+ *   pattern       = first p with a strictly larger S_p (ties -> lowest id; a NaN sum never wins)
+ *
+ * FB = CB = 1 is Algorithm 2 with double instead of float pattern sums.  Blocks at the ragged end of the
+ * filter or channel range are simply smaller.  pid gets Cout*Cin entries, constant inside a block.
+ */
+void oracle_select_shared(const float *w, int Cout, int Cin, int FB, int CB, const uint16_t *masks, int P, uint8_t *pid) {
+    for (int co0 = 0; co0 < Cout; co0 += FB)
+        for (int ci0 = 0; ci0 < Cin; ci0 += CB) {
+            int co1 = co0 + FB < Cout ? co0 + FB : Cout;
+            int ci1 = ci0 + CB < Cin ? ci0 + CB : Cin;
+            double E[9];
+            for (int t = 0; t < 9; ++t) E[t] = 0.0;
+            for (int co = co0; co < co1; ++co) {
+                double r[9];
+                for (int t = 0; t < 9; ++t) r[t] = 0.0;
+                for (int ci = ci0; ci < ci1; ++ci) {
+                    const float *kw = w + 9 * ((long)co * Cin + ci);
+                    for (int t = 0; t < 9; ++t) {
+                        volatile float sq = kw[t] * kw[t];
+                        r[t] = r[t] + (double)sq;
+                    }
+                }
+                for (int t = 0; t < 9; ++t) E[t] = E[t] + r[t];
+            }
+            int best = 0;
+            double best_s = 0.0;
+            for (int p = 0; p < P; ++p) {
+                double sv = 0.0;
+                for (int t = 0; t < 9; ++t)
+                    if ((masks[p] >> t) & 1u) sv = sv + E[t];
+                if (p == 0) {
+                    best_s = sv;
+                } else if (sv > best_s || (best_s != best_s && sv == sv)) {
+                    best = p;
+                    best_s = sv;
+                }
+            }
+            for (int co = co0; co < co1; ++co)
+                for (int ci = ci0; ci < ci1; ++ci) pid[(long)co * Cin + ci] = (uint8_t)best;
+        }
 }
 
 /* ---- mask application ---------------------------------------------------- */

@@ -122,6 +122,17 @@ def select_3x3(w, masks):
     return pid
 
 
+def select_shared(w, masks, FB, CB):
+    """One pattern per block of FB filters x CB input channels: the pattern retaining the most energy of the block
+    (a variant of Algorithm 2, see the C source).  w [Cout, Cin, 3, 3] -> pid [Cout, Cin], constant per block."""
+    w = _f32(w)
+    Cout, Cin = w.shape[:2]
+    m = _masks(masks)
+    pid = np.zeros((Cout, Cin), dtype=np.uint8)
+    lib().oracle_select_shared(_p(w), Cout, Cin, int(FB), int(CB), _p(m), len(m), _p(pid))
+    return pid
+
+
 def select_1x1(w, masks):
     """w: [Cout, Cin] -> pid1[G], G = floor(Cout*Cin/9) (Algorithm 3)."""
     w = _f32(w).reshape(w.shape[0], -1)
