@@ -316,10 +316,14 @@ def run_network(args):
     ctx.close()
 
 
-def measure_workload(ctx, rt, dev, name, steps, warmup, args, world, rank, full):
+def measure_workload(ctx, rt, dev, name, steps, warmup, args, world, rank, full, shared=False):
     """One workload on this rank's GPU: the graph-replayed step (select + pack of every weight tensor, then every
     convolution), the cold-L2 per-launch pass for the roofline, and -- with `full` -- the end-to-end leg through the
-    host-buffer entry point.  Returns a dict of raw figures (times of this rank; the caller reduces over ranks)."""
+    host-buffer entry point.  Convolutions that do not depend on one another in the network (synth.independent_sets)
+    go out as one rtoss_conv_group call.  `shared`: the variant with one pattern per block of 128 filters x 16
+    channels for the 3x3 layers (rtoss_select_patterns_shared); its step is the convolutions alone, selection and
+    packing of the variant run once, layer by layer, outside the timed region.
+    Returns a dict of raw figures (times of this rank; the caller reduces over ranks)."""
     import torch
     import torch.distributed as dist
     tdt = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}
@@ -357,12 +361,17 @@ def measure_workload(ctx, rt, dev, name, steps, warmup, args, world, rank, full)
     # handles are made once, layer by layer (this allocates); every step then re-selects and re-packs ALL layers
     # with the whole-model pass: two launches, whatever the number of layers
     for wt in weights.values():
-        ctx.rtoss_select_patterns(wt["w"], wt["ksize"], wt["masks"], wt["k"], pid=wt["pid"])
+        if shared and wt["ksize"] == 3:
+            ctx.rtoss_select_patterns_shared(wt["w"], wt["masks"], wt["k"], 128, 16, pid=wt["pid"])
+        else:
+            ctx.rtoss_select_patterns(wt["w"], wt["ksize"], wt["masks"], wt["k"], pid=wt["pid"])
         wt["packed"] = ctx.rtoss_pack(wt["w"], wt["ksize"], wt["masks"], wt["k"], wt["pid"], cdt)
     batch = ctx.rtoss_batch_create(list(weights.values()))
     any3 = any(wt["ksize"] == 3 for wt in weights.values())
 
     def prune_weights():
+        if shared:
+            return 0
         batch.rtoss_batch_select_pack()
         return 2 if any3 else 1
 
@@ -376,11 +385,35 @@ def measure_workload(ctx, rt, dev, name, steps, warmup, args, world, rank, full)
         if ev:
             ev[1].record()
 
+    # launch units: convolutions that are independent in the network share one grouped call
+    units = synth.independent_sets([st["L"] for st in L_state]) if args.group else [[i] for i in range(len(L_state))]
+    unit_launches = [1] * len(units)
+
+    def run_unit(u, ev=None):
+        """-> kernel launches made."""
+        idx = units[u]
+        if len(idx) == 1:
+            conv(L_state[idx[0]], ev)
+            return 1
+        items = []
+        for i in idx:
+            st = L_state[i]
+            L = st["L"]
+            items.append(ctx.conv_item(st["wt"]["packed"], st["x"], st["y"], N, L["H"], L["W"], L["stride"], layout,
+                                       rt.ACT_NAMES[L["act"]], st["wt"]["b"], path=st["path"]))
+        if ev:
+            ev[0].record()
+        n = ctx.rtoss_conv_group(items)
+        if ev:
+            ev[1].record()
+        return n
+
     def step(evs=None):
         n = prune_weights()
-        for i, st in enumerate(L_state):
-            conv(st, evs[i] if evs else None)
-        return n + len(L_state)
+        for u in range(len(units)):
+            unit_launches[u] = run_unit(u, evs[u] if evs else None)
+            n += unit_launches[u]
+        return n
 
     def barrier():
         if world > 1:
@@ -453,17 +486,17 @@ def measure_workload(ctx, rt, dev, name, steps, warmup, args, world, rank, full)
     if args.graph:
         try:
             gev = [(torch.cuda.Event(enable_timing=True, external=True), torch.cuda.Event(enable_timing=True, external=True))
-                   for _ in range(len(L_state) + 1)]
+                   for _ in range(len(units) + 1)]
             kgraph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(kgraph):
                 flush.zero_()
                 gev[-1][0].record()
                 prune_weights()
                 gev[-1][1].record()
-                for i, st in enumerate(L_state):
+                for u in range(len(units)):
                     flush.zero_()
-                    conv(st, gev[i])
-            acc = np.zeros(len(L_state) + 1)
+                    run_unit(u, gev[u])
+            acc = np.zeros(len(units) + 1)
             for s in range(steps):
                 kgraph.replay()
                 torch.cuda.synchronize()
@@ -474,16 +507,16 @@ def measure_workload(ctx, rt, dev, name, steps, warmup, args, world, rank, full)
             torch.cuda.synchronize()
             conv_ms = None
     if conv_ms is None:
-        conv_ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(len(L_state) + 1)]
+        conv_ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(len(units) + 1)]
                    for _ in range(steps)]
         for s in range(steps):
             flush.zero_()
             conv_ev[s][-1][0].record()
             prune_weights()
             conv_ev[s][-1][1].record()
-            for i, st in enumerate(L_state):
+            for u in range(len(units)):
                 flush.zero_()
-                conv(st, conv_ev[s][i])
+                run_unit(u, conv_ev[s][u])
         barrier()
         allms = np.array([[a.elapsed_time(b) for a, b in row] for row in conv_ev]).mean(axis=0)
         conv_ms, prune_ms = allms[:-1], float(allms[-1])
@@ -492,6 +525,7 @@ def measure_workload(ctx, rt, dev, name, steps, warmup, args, world, rank, full)
 
     res = dict(name=name, N=N, dtype=dtype, elem=elem, layout="NHWC" if layout == rt.NHWC else "NCHW", total_ms=total_ms,
                steps=steps, launches=launches, graph=graph is not None, conv_ms=conv_ms, prune_ms=prune_ms, clocks=clocks,
+               units=units, unit_launches=list(unit_launches), shared=shared,
                layers=[st["L"] for st in L_state], ks=[st["k"] for st in L_state],
                on_tc=[st["path"] == rt.PATH_TENSOR for st in L_state],
                weights=[dict(n_k=wt["n_k"], k=wt["k"], ksize=wt["ksize"]) for wt in weights.values()], e2e_s=None)
@@ -537,33 +571,42 @@ def roofline_of(res, hbm_peak, tc_peak, peak_kind):
     pipe = np.array([tc_peak if tc else ALU_PEAK_TFLOPS for tc in res["on_tc"]]) * 1e12
     t_pipe, t_hbm = flops / pipe, bytes_ / (hbm_peak * 1e9)
     t_roof = np.maximum(t_pipe, t_hbm)
-    t_meas = res["conv_ms"] * 1e-3
+    t_meas = res["conv_ms"] * 1e-3          # one entry per launch unit (a unit of several layers is one grouped call)
+    units = res["units"]
+    u_roof = np.array([t_roof[u].sum() for u in units])
+    u_flops = np.array([flops[u].sum() for u in units])
+    u_bytes = np.array([bytes_[u].sum() for u in units])
     stack_frac = float(t_roof.sum() / t_meas.sum())
-    # the dominant kernel shape: layers of one shape share a kernel configuration; the shape with the largest share
+    # the dominant kernel: units of one composition (the shapes of their layers) share a kernel configuration; the
+    # composition with the largest share of the cold pass
     shape_of = lambda L: (L["ksize"], L["stride"], L["cin"], L["cout"], L["H"], L["W"])
     share = {}
-    for i, L in enumerate(res["layers"]):
-        share.setdefault(shape_of(L), []).append(i)
+    for ui, u in enumerate(units):
+        share.setdefault(tuple(shape_of(res["layers"][i]) for i in u), []).append(ui)
     top_shape = max(share, key=lambda sh: t_meas[share[sh]].sum())
     idx = share[top_shape]
     top = idx[int(np.argmax(t_meas[idx]))]
-    on_tc = res["on_tc"][top]
+    members = units[top]
+    on_tc = res["on_tc"][members[0]]
     t_top = float(np.mean(t_meas[idx]))
-    if t_pipe[top] >= t_hbm[top]:
-        dom = {"bound": "tensor" if on_tc else "alu", "achieved": flops[top] / t_top / 1e12, "peak": pipe[top] / 1e12, "unit": "TFLOP/s",
+    if t_pipe[members].sum() >= t_hbm[members].sum():
+        dom = {"bound": "tensor" if on_tc else "alu", "achieved": u_flops[top] / t_top / 1e12, "peak": pipe[members[0]] / 1e12,
+               "unit": "TFLOP/s",
                "peak_kind": ("of %s (bf16 cuBLAS, sustained)" % peak_kind) if on_tc
                else "nominal, not measured: 148 SM x 128 FMA lanes x 2 x 1.965 GHz"}
     else:
-        dom = {"bound": "hbm", "achieved": bytes_[top] / t_top / 1e9, "peak": hbm_peak, "unit": "GB/s", "peak_kind": "of " + peak_kind}
-    dom["frac"] = dom["achieved"] / dom["peak"]
-    L = res["layers"][top]
-    dom["kernel"] = ("conv_tc_kernel " if on_tc else "conv_alu_kernel ") + L["name"] + " k=%d" % res["ks"][top]
-    dom["launches_of_this_shape"] = len(idx)
+        dom = {"bound": "hbm", "achieved": u_bytes[top] / t_top / 1e9, "peak": hbm_peak, "unit": "GB/s", "peak_kind": "of " + peak_kind}
+    dom["frac"] = float(u_roof[top] / t_top)   # sum of the members' roofline times / the launch's time
+    L = res["layers"][members[0]]
+    dom["kernel"] = ("conv_tc_kernel " if on_tc else "conv_alu_kernel ") + L["name"] + " k=%d" % res["ks"][members[0]] + \
+                    ("" if len(members) == 1 else " + %d more convolutions in the same launch" % (len(members) - 1))
+    dom["convolutions_per_launch"] = len(members)
+    dom["launches_of_this_kind"] = len(idx)
     dom["share_of_cold_pass"] = float(t_meas[idx].sum() / t_meas.sum())
     dom["kernel_ms"] = t_top * 1e3
-    dom["nnz_flop_per_launch"] = float(flops[top])
-    dom["algorithmic_bytes_per_launch"] = float(bytes_[top])
-    dom["traffic"] = ncu_traffic(res["name"], L["name"], res["ks"][top])
+    dom["nnz_flop_per_launch"] = float(u_flops[top])
+    dom["algorithmic_bytes_per_launch"] = float(u_bytes[top])
+    dom["traffic"] = ncu_traffic(res["name"], L["name"], res["ks"][members[0]]) if len(members) == 1 else None
     # whole-model selection + packing: 36 B read per kernel (nine fp32 weights), k values + the id + the order entry written
     sp_bytes = float(sum(w["n_k"] * (36 + w["k"] * elem + (5 if w["ksize"] == 3 else 1)) for w in res["weights"]))
     sp = {"kernels": int(sum(w["n_k"] for w in res["weights"])), "launches": 2 if any(w["ksize"] == 3 for w in res["weights"]) else 1,
@@ -574,7 +617,7 @@ def roofline_of(res, hbm_peak, tc_peak, peak_kind):
     tensor_share = float(t_roof[t_pipe >= t_hbm].sum() / t_roof.sum())
     return dict(stack_frac=stack_frac, sum_roof_ms=float(t_roof.sum() * 1e3), sum_cold_ms=float(t_meas.sum() * 1e3),
                 tensor_share=tensor_share, dominant=dom, select_pack=sp, flops=flops, bytes=bytes_, t_roof=t_roof,
-                t_pipe=t_pipe, t_hbm=t_hbm)
+                t_pipe=t_pipe, t_hbm=t_hbm, u_roof=u_roof)
 
 
 OTHER_WORKLOADS = ("layer32", "layer128", "yolov5s_b1", "yolov5s_b16")
@@ -598,11 +641,13 @@ def run_gpu(args):
 
     res = measure_workload(ctx, rt, dev, args.workload, args.steps, args.warmup, args, world, rank, full=True)
     total_ms, e2e_s = max_over_ranks([res["total_ms"], res["e2e_s"]], dev, world)
-    others = {}
+    others, variant = {}, None
     if args.others and world == 1:
         for name in OTHER_WORKLOADS:
             if name != args.workload:
                 others[name] = measure_workload(ctx, rt, dev, name, min(args.steps, 20), 3, args, 1, rank, full=False)
+        if res["dtype"] != "f32":
+            variant = measure_workload(ctx, rt, dev, args.workload, min(args.steps, 20), 3, args, 1, rank, full=False, shared=True)
 
     if rank == 0:
         N, dtype = res["N"], res["dtype"]
@@ -636,7 +681,9 @@ def run_gpu(args):
             "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
             "config": {"workload": args.workload, "batch": N, "layout": res["layout"], "layers": len(res["layers"]),
                        "l2": "flushed between steps (256 MB write)", "multi_gpu": "replicas only",
-                       "launch": "one CUDA graph per step" if res["graph"] else "eager"},
+                       "launch": "one CUDA graph per step" if res["graph"] else "eager",
+                       "grouping": ("independent convolutions share a launch: %d launches for %d convolutions"
+                                    % (sum(res["unit_launches"]), len(res["layers"]))) if args.group else "one launch per convolution"},
             "paths": {"tensor_path_layers": int(sum(res["on_tc"])), "fma_path_layers": int(len(res["on_tc"]) - sum(res["on_tc"]))},
             "nnz_gflops_per_s": float(rf["flops"].sum()) / (ms_per_step * 1e-3) / 1e9 * world,
             "conv_ms": [float(v) for v in res["conv_ms"]] if len(res["conv_ms"]) <= 8 else None,
@@ -659,14 +706,32 @@ def run_gpu(args):
                     "select_pack_us": orf["select_pack"]["us"], "select_pack_frac": orf["select_pack"]["frac"],
                     "tensor_path_layers": int(sum(r["on_tc"])), "fma_path_layers": int(len(r["on_tc"]) - sum(r["on_tc"])),
                     "clocks": r["clocks"], "gpu_launches": r["launches"]}
+        if variant is not None:
+            vrf = roofline_of(variant, hbm_peak, tc_peak, peak_kind)
+            vms = variant["total_ms"] / variant["steps"]
+            vd = vrf["dominant"]
+            out["shared_pattern_variant"] = {
+                "what": "the 3x3 layers pruned with ONE pattern per block of 128 filters x 16 input channels "
+                        "(rtoss_select_patterns_shared) instead of one per kernel: a different, coarser pruning result (its "
+                        "effect on detection accuracy is not measured here); the tensor path then issues only the k kept taps",
+                "step": "the convolutions only (selection and packing of the variant run once, outside the timed region)",
+                "steps": variant["steps"], "ms_per_step": vms, "images_per_s": variant["N"] / (vms * 1e-3),
+                "nnz_gflops_per_s": float(vrf["flops"].sum()) / (vms * 1e-3) / 1e9,
+                "roofline_frac": vrf["stack_frac"], "sum_roofline_ms": vrf["sum_roof_ms"], "sum_cold_kernel_ms": vrf["sum_cold_ms"],
+                "dominant_kernel": {k_: vd[k_] for k_ in ("kernel", "bound", "achieved", "peak", "unit", "frac", "kernel_ms",
+                                                          "convolutions_per_launch", "share_of_cold_pass")},
+                "clocks": variant["clocks"], "gpu_launches": variant["launches"]}
         if args.layers_csv:
             # per-layer table: cold-L2 kernel time next to the two roofline terms at non-zero FLOPs
             with open(args.layers_csv, "w") as f:
-                f.write("layer,ksize,cin,cout,H,W,stride,k,path,kernel_us,hbm_us,pipe_us,frac\n")
-                for L, k, tc, ms, hu, pu in zip(res["layers"], res["ks"], res["on_tc"], res["conv_ms"], rf["t_hbm"], rf["t_pipe"]):
-                    f.write("%s,%d,%d,%d,%d,%d,%d,%d,%s,%.2f,%.2f,%.2f,%.3f\n" % (
-                        L["name"], L["ksize"], L["cin"], L["cout"], L["H"], L["W"], L["stride"], k,
-                        "tensor" if tc else "fma", ms * 1e3, hu * 1e6, pu * 1e6, max(hu, pu) * 1e3 / ms))
+                f.write("launch,convolutions,launches,ksize,cin,cout,H,W,stride,k,path,kernel_us,hbm_us,pipe_us,roofline_us,frac\n")
+                for ui, u in enumerate(res["units"]):
+                    L, k, tc = res["layers"][u[0]], res["ks"][u[0]], res["on_tc"][u[0]]
+                    ms = res["conv_ms"][ui]
+                    f.write("%s,%d,%d,%d,%d,%d,%d,%d,%d,%d,%s,%.2f,%.2f,%.2f,%.2f,%.3f\n" % (
+                        L["name"], len(u), res["unit_launches"][ui], L["ksize"], L["cin"], L["cout"], L["H"], L["W"], L["stride"], k,
+                        "tensor" if tc else "fma", ms * 1e3, rf["t_hbm"][u].sum() * 1e6, rf["t_pipe"][u].sum() * 1e6,
+                        rf["u_roof"][ui] * 1e6, rf["u_roof"][ui] * 1e3 / ms))
         if args.cpu_baseline:
             _, _, layers_k = workload_layers(args.workload)
             v_cpu, t_cpu, f_cpu, n_cpu, p_cpu = cpu_baseline_sample(layers_k, dtype, N, 15.0)
@@ -692,6 +757,7 @@ def main():
                     help="skip the sub-records of the other configurations (layer32, layer128, yolov5s_b1, yolov5s_b16)")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--no-graph", dest="graph", action="store_false", help="time eager launches instead of a CUDA graph")
+    ap.add_argument("--no-group", dest="group", action="store_false", help="one launch per convolution (no rtoss_conv_group)")
     ap.add_argument("--path", default="auto", choices=["auto", "fma"], help="fma: keep every layer on the FMA path")
     ap.add_argument("--layers-csv", default=None, help="write the per-layer kernel times and roofline terms to this file")
     ap.add_argument("--layout", default="auto", choices=["auto", "nchw"], help="nchw: NCHW activations also for 16-bit types")

@@ -158,6 +158,22 @@ rtoss_status rtoss_pattern_table_derive(rtoss_ctx* ctx, const void* kernels_dev,
                                         uint16_t* top_masks_host, int* M_kept, uint16_t* cand_masks_host,
                                         uint64_t* cand_counts_host, int* P_candidates, void* cuda_stream);
 
+/* A variant of the selection, not the paper's per-kernel rule: ONE pattern for every block of `filter_block`
+ * consecutive filters x `channel_block` consecutive input channels of a 3x3 layer, namely the pattern that retains the
+ * largest sum of squared weights of the whole block (Section IV.C shares kernel masks inside layer groups; this
+ * shares them inside a layer).  pid_dev gets Cout*Cin ids as rtoss_select_patterns writes them, constant inside a
+ * block, so rtoss_pack and the convolutions take them unchanged.  Why: with filter_block = 128 and channel_block a
+ * multiple of 16 the tensor path multiplies only the k kept taps of every block (9/k fewer matrix instructions), which
+ * per-kernel patterns never allow.  The price is retained norm: the result is a different (coarser) pruning than
+ * Algorithm 2's, whose effect on detection accuracy this library cannot measure.
+ * Arithmetic (fixed, so that ids are reproducible): squares rounded to fp32, then summed in double over the block's
+ * channels (ascending) per filter, over the block's filters (ascending), over the pattern's taps (ascending); first
+ * strictly larger sum wins.  Blocks at the ragged end of a range are smaller.  1 <= filter_block <= 256,
+ * channel_block >= 1; ksize 3 only.  Errors as rtoss_select_patterns. */
+rtoss_status rtoss_select_patterns_shared(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, int Cout, int Cin,
+                                          int filter_block, int channel_block, const uint16_t* masks_host, int P, int k,
+                                          uint8_t* pid_dev, void* cuda_stream);
+
 /* ---- packing (Section IV.C, last sentence: kernels of like pattern are put together) --- */
 
 /* Build the packed form of one layer from its weights and pattern ids:
@@ -307,14 +323,42 @@ rtoss_status rtoss_conv3x3_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const 
 rtoss_status rtoss_conv1x1_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const void* x_dev, void* y_dev,
                                    const rtoss_conv_desc* desc, void* cuda_stream);
 
+/* Several INDEPENDENT convolutions at once (no item reads or overwrites what another item writes): the pyramid levels
+ * a detection tower is applied to (Section V evaluates RetinaNet, whose towers share their weights across five
+ * levels), the two towers, the two 1x1 branches that open a block.  Results are those of the single calls.  Items
+ * that qualify for the tensor path with more than 64 filters or a 3x3 kernel, and agree in kernel size, data type
+ * and (3x3) stride, share ONE launch, up to ten at a time: small items then fill the SMs the large ones leave idle
+ * instead of paying a launch each.  The other items run as single launches inside the same call.  *launches
+ * (nullable) receives the number of kernel launches made.  Errors: those of the single calls; nothing is launched
+ * when an argument check fails. */
+typedef struct {
+    const rtoss_packed* packed; /* ksize 3 or 1 */
+    const void* x_dev;
+    void* y_dev;
+    rtoss_conv_desc desc;
+} rtoss_conv_item;
+rtoss_status rtoss_conv_group(rtoss_ctx* ctx, const rtoss_conv_item* items, int n, int* launches, void* cuda_stream);
+
 /* The tensor path (RTOSS_PATH_TENSOR, or RTOSS_PATH_AUTO when it applies) takes: bf16 / fp16 NHWC,
- * stride 1 or 2, io_dtype equal to the packed dtype, Cin a multiple of 8.  It multiplies the pruned
- * taps as zeros on the tensor cores; results agree with the FMA path to fp32 summation order.
+ * stride 1 or 2, io_dtype equal to the packed dtype, Cin a multiple of 8.  It multiplies blocks of 128 filters x 16
+ * channels per tap on the tensor cores and leaves out the blocks in which every weight is pruned (none with
+ * per-kernel patterns on ordinary weights; 9 - k of every 9 with rtoss_select_patterns_shared); inside a block the
+ * pruned taps are multiplied as zeros.  Results agree with the FMA path to fp32 summation order.
  *
  * Device-side waits of that path are bounded.  If one runs out, the kernel records a non-zero code in
  * the context and returns; rtoss_device_status synchronises the device, reports the code
  * (RTOSS_ERR_TIMEOUT when non-zero) and clears it. */
 rtoss_status rtoss_device_status(rtoss_ctx* ctx, int* code);
+
+/* Limit of those waits in SM clock cycles (default 2e9, about a second; at least 1000). */
+rtoss_status rtoss_set_wait_limit(rtoss_ctx* ctx, long long sm_cycles);
+
+/* Failure-detection aid: the NEXT tensor-path launch of this context withholds its first weight copy, so that the
+ * waits that depend on it run out and the timeout path above can be exercised.  Nothing illegal happens on the
+ * device: every role of the kernel gives up after the wait limit and the kernel ends normally; the output of that
+ * call is undefined.  Only a launch of a single CTA (one tile) is accepted -- any other returns RTOSS_ERR_CUDA
+ * without launching -- and the request is consumed either way.  Lower the wait limit first. */
+rtoss_status rtoss_inject_lost_copy(rtoss_ctx* ctx);
 
 /* Same convolutions with HOST buffers: copies x to the device, runs the
  * kernel for the handle's ksize, copies y back and waits for it.  x_host and

@@ -30,6 +30,7 @@ SYMBOLS = [
     "rtoss_conv3x3_pattern", "rtoss_conv1x1_pattern", "rtoss_conv_pattern_host", "rtoss_device_status", "rtoss_prune_dense_static", "rtoss_maxpool2d", "rtoss_upsample2x", "rtoss_add_act", "rtoss_pattern_usage",
     "rtoss_pattern_rank", "rtoss_pattern_table_derive",
     "rtoss_batch_create", "rtoss_batch_select_pack", "rtoss_batch_destroy",
+    "rtoss_select_patterns_shared", "rtoss_conv_group", "rtoss_set_wait_limit", "rtoss_inject_lost_copy",
 ]
 
 
@@ -63,6 +64,10 @@ class ConvDesc(ctypes.Structure):
                 ("path", ctypes.c_int), ("residual_dev", ctypes.c_void_p), ("residual_after_act", ctypes.c_int)]
 
 
+class ConvItem(ctypes.Structure):
+    _fields_ = [("packed", ctypes.c_void_p), ("x_dev", ctypes.c_void_p), ("y_dev", ctypes.c_void_p), ("desc", ConvDesc)]
+
+
 def _load():
     if not os.path.exists(LIB_PATH):
         raise RuntimeError("librtoss.so not built (%s): run `python -m paper_2303_02191_b200._build`; "
@@ -93,6 +98,10 @@ def _load():
     lib.rtoss_conv1x1_pattern.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ConvDesc), vp]
     lib.rtoss_conv_pattern_host.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ConvDesc)]
     lib.rtoss_device_status.argtypes = [vp, ctypes.POINTER(ci)]
+    lib.rtoss_conv_group.argtypes = [vp, ctypes.POINTER(ConvItem), ci, ctypes.POINTER(ci), vp]
+    lib.rtoss_set_wait_limit.argtypes = [vp, ctypes.c_longlong]
+    lib.rtoss_inject_lost_copy.argtypes = [vp]
+    lib.rtoss_select_patterns_shared.argtypes = [vp, vp, ci, ci, ci, ci, ci, vp, ci, ci, vp, vp]
     lib.rtoss_prune_dense_static.argtypes = [vp, ci, ci, ci, ci, vp, ci, ci, vp, vp]
     lib.rtoss_maxpool2d.argtypes = [vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, vp]
     lib.rtoss_upsample2x.argtypes = [vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, vp]
@@ -252,6 +261,17 @@ class Context:
                                               _np_ptr(m), len(m), int(k), pid.data_ptr(), _stream()))
         return pid[:n]
 
+    def rtoss_select_patterns_shared(self, w, masks, k, filter_block, channel_block, pid=None):
+        """w: CUDA tensor [Cout,Cin,3,3] -> uint8 ids [Cout*Cin], one pattern per block of filters x channels."""
+        import torch
+        Cout, Cin = int(w.shape[0]), int(w.shape[1])
+        m = _masks_arr(masks)
+        if pid is None:
+            pid = torch.empty(Cout * Cin, dtype=torch.uint8, device=w.device)
+        self._check(lib.rtoss_select_patterns_shared(self.h, w.data_ptr(), _torch_dtype_code(w), Cout, Cin, int(filter_block),
+                                                     int(channel_block), _np_ptr(m), len(m), int(k), pid.data_ptr(), _stream()))
+        return pid
+
     def rtoss_pattern_usage(self, kernels, masks, k):
         """kernels: CUDA tensor [n, 9] (or [n,3,3]) -> numpy uint64 win counts per pattern of the table."""
         import torch
@@ -319,6 +339,26 @@ class Context:
                        path, residual, residual_after_act)
         self._check(lib.rtoss_conv1x1_pattern(self.h, packed.h, x.data_ptr(), y.data_ptr(), ctypes.byref(d), _stream()))
         return y
+
+    def conv_item(self, packed, x, y, N, H, W, stride=1, layout=NCHW, act=ACT_NONE, bias=None, y_channel_offset=0,
+                  y_channel_stride=0, path=PATH_AUTO, residual=None, residual_after_act=False):
+        """One entry for rtoss_conv_group (arguments as rtoss_conv3x3_pattern / rtoss_conv1x1_pattern)."""
+        d = self._desc((N, 0, H, W), stride, layout, _torch_dtype_code(x), act, bias, y_channel_offset, y_channel_stride,
+                       path, residual, residual_after_act)
+        return ConvItem(packed.h.value, x.data_ptr(), y.data_ptr(), d)
+
+    def rtoss_conv_group(self, items):
+        """items: list of conv_item(...) -> number of kernel launches made."""
+        arr = (ConvItem * len(items))(*items)
+        n = ctypes.c_int(0)
+        self._check(lib.rtoss_conv_group(self.h, arr, len(items), ctypes.byref(n), _stream()))
+        return n.value
+
+    def rtoss_set_wait_limit(self, sm_cycles):
+        self._check(lib.rtoss_set_wait_limit(self.h, int(sm_cycles)))
+
+    def rtoss_inject_lost_copy(self):
+        self._check(lib.rtoss_inject_lost_copy(self.h))
 
     def rtoss_conv_pattern_host(self, packed, x_host, y_host, N, H, W, stride=1, layout=NCHW, act=ACT_NONE, bias=None,
                                 y_channel_offset=0, y_channel_stride=0, path=PATH_AUTO):

@@ -39,6 +39,8 @@ struct BatchLayer {
     void* wtc;
     uint32_t* perm;
     uint32_t* bucket_off;
+    unsigned long long* issue;  // the handle's issue words (tensor path, 3x3), or null
+    int issue_n;
     long long n_kernels;
     rtoss_wtc_layout lay;  // layout of wtc
     int Cout, Cin, ksize, P, k;
@@ -87,6 +89,9 @@ __global__ void __launch_bounds__(kChunk) batch_select_pack_kernel(const BatchLa
         const long long left = L.n_kernels - first;
         const int count = (int)(left < kChunk ? left : kChunk);
         const bool inherits = L.w_sel != L.w;
+        // the layer's first chunk clears its issue words: the ordering kernel (next launch) ORs the bits in
+        if (chunk == L.chunk0 && L.issue)
+            for (int i = threadIdx.x; i < L.issue_n; i += kChunk) L.issue[i] = 0ull;
         __syncthreads();  // the previous step's readers are done
         stage_raw(L.w_sel, first, count, L.sel_dtype == RTOSS_F32 ? 4 : 2, s_sel);
         if (inherits) stage_raw(L.w, first, count, L.w_dtype == RTOSS_F32 ? 4 : 2, s_own);
@@ -127,7 +132,7 @@ __global__ void __launch_bounds__(kOrderWarps * 32) batch_order_kernel(const Bat
     for (unsigned task = blockIdx.x * kOrderWarps + warp; task < n_tasks; task += gridDim.x * kOrderWarps) {
         const BatchLayer& L = layers[task_layer[task]];
         rtoss_dev::order_channel(L.pid, L.Cout, L.Cin, L.P, (int)(task - L.task0), L.perm, L.bucket_off, fill_all[warp],
-                                 lane);
+                                 lane, L.masks, L.issue);
         __syncwarp();
     }
 }
@@ -213,6 +218,8 @@ rtoss_status rtoss_batch_create(rtoss_ctx* ctx, const rtoss_batch_item* items, i
         B.wtc = p->wtc;
         B.perm = p->perm;
         B.bucket_off = p->bucket_off;
+        B.issue = p->issue;
+        B.issue_n = p->issue_n;
         B.n_kernels = p->n_kernels;
         B.lay = rtoss_wtc_layout_of(it.Cout, it.ksize);
         B.Cout = it.Cout;

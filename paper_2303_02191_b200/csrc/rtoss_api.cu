@@ -4,6 +4,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <vector>
 #include <new>
 
 #include "rtoss.h"
@@ -188,6 +189,34 @@ rtoss_status rtoss_select_patterns(rtoss_ctx* ctx, const void* w_dev, rtoss_dtyp
     return e ? cuda_fail(ctx, "select launch", e) : RTOSS_OK;
 }
 
+rtoss_status rtoss_select_patterns_shared(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, int Cout, int Cin,
+                                          int filter_block, int channel_block, const uint16_t* masks_host, int P, int k,
+                                          uint8_t* pid_dev, void* cuda_stream) {
+    if (!ctx) return RTOSS_ERR_INVALID_ARG;
+    if (!w_dev || !pid_dev || !masks_host || !dtype_ok(w_dtype)) {
+        set_err(ctx, "select shared", "null argument or bad dtype");
+        return RTOSS_ERR_INVALID_ARG;
+    }
+    rtoss_status st = check_layer(ctx, Cout, Cin, 3);
+    if (st != RTOSS_OK) return st;
+    if (filter_block < 1 || filter_block > 256 || channel_block < 1) {
+        set_err(ctx, "select shared", "filter_block must be 1..256, channel_block at least 1");
+        return RTOSS_ERR_INVALID_ARG;
+    }
+    if (!rtoss_table_ok(masks_host, P, k)) {
+        set_err(ctx, "select shared", "pattern table invalid");
+        return RTOSS_ERR_BAD_PATTERN_TABLE;
+    }
+    if (!aligned16(w_dev)) {
+        set_err(ctx, "select shared", "weights must be 16-byte aligned");
+        return RTOSS_ERR_ALIGNMENT;
+    }
+    rtoss_device_guard on_device(ctx->device);
+    int e = rtoss_launch_select_shared(w_dev, w_dtype, Cout, Cin, filter_block, channel_block, make_table(masks_host, P), P,
+                                       pid_dev, cuda_stream);
+    return e ? cuda_fail(ctx, "select shared launch", e) : RTOSS_OK;
+}
+
 rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, int Cout, int Cin, int ksize,
                         const uint16_t* masks_host, int P, int k, const uint8_t* pid_dev, rtoss_dtype compute_dtype,
                         rtoss_packed** out, void* cuda_stream) {
@@ -253,6 +282,10 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
                 (size_t)(ksize == 3 ? 9 : 1) * rtoss_wtc_layout_of(Cout, ksize).rows * Cin * rtoss_dtype_size(compute_dtype);
             e = cudaMalloc(&p->wtc, wtc_bytes);
             if (e == cudaSuccess) e = cudaMemsetAsync(p->wtc, 0, wtc_bytes, s);
+            if (e == cudaSuccess && ksize == 3) {
+                p->issue_n = rtoss_issue_words(Cout, Cin, ksize);
+                e = cudaMalloc((void**)&p->issue, sizeof(unsigned long long) * (size_t)p->issue_n);
+            }
         }
         if (e != cudaSuccess) {
             cudaGetLastError();
@@ -267,8 +300,10 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
     if (e == cudaSuccess)  // also writes the handle's own copy of the ids and the tensor path's dense-expanded weights
         le = rtoss_launch_pack_values(w_dev, w_dtype, p->n_kernels, make_table(masks_host, P), pid_dev, k, p->val,
                                       compute_dtype, p->pid, p->wtc, ksize, Cout, Cin, cuda_stream);
+    // the ordering pass also gathers which (tap, channel slab) pairs of every filter tile hold kept weights; its words start at zero
+    if (e == cudaSuccess && !le && p->issue) e = cudaMemsetAsync(p->issue, 0, sizeof(unsigned long long) * (size_t)p->issue_n, s);
     if (e == cudaSuccess && !le && ksize == 3)
-        le = rtoss_launch_pack_order(pid_dev, Cout, Cin, P, p->perm, p->bucket_off, cuda_stream);
+        le = rtoss_launch_pack_order(pid_dev, Cout, Cin, P, p->perm, p->bucket_off, p->masks_dev, p->issue, cuda_stream);
     if (e != cudaSuccess || le) {
         rtoss_status r = cuda_fail(ctx, "pack launch", e != cudaSuccess ? (int)e : le);
         if (!reuse) rtoss_packed_destroy(p);
@@ -387,6 +422,7 @@ void rtoss_packed_destroy(rtoss_packed* p) {
     if (p->bucket_off) cudaFree(p->bucket_off);
     if (p->masks_dev) cudaFree(p->masks_dev);
     if (p->wtc) cudaFree(p->wtc);
+    if (p->issue) cudaFree(p->issue);
     cudaSetDevice(prev);
     delete p;
 }
@@ -409,6 +445,75 @@ rtoss_status rtoss_conv1x1_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const 
     int e = dispatch_conv(ctx, p, x_dev, y_dev, desc, cuda_stream, &st);
     if (st != RTOSS_OK) return st;
     return e ? cuda_fail(ctx, "conv1x1 launch", e) : RTOSS_OK;
+}
+
+rtoss_status rtoss_conv_group(rtoss_ctx* ctx, const rtoss_conv_item* items, int n, int* launches, void* cuda_stream) {
+    if (!ctx) return RTOSS_ERR_INVALID_ARG;
+    if (launches) *launches = 0;
+    if (!items || n < 1) {
+        set_err(ctx, "conv group", "null argument or no items");
+        return RTOSS_ERR_INVALID_ARG;
+    }
+    for (int i = 0; i < n; ++i) {
+        if (!items[i].packed) {
+            set_err(ctx, "conv group", "item without a packed handle");
+            return RTOSS_ERR_INVALID_ARG;
+        }
+        rtoss_status st = check_conv(ctx, items[i].packed, items[i].x_dev, items[i].y_dev, &items[i].desc, items[i].packed->ksize, true);
+        if (st != RTOSS_OK) return st;
+    }
+    rtoss_device_guard on_device(ctx->device);
+    // Items that can share a launch are collected class by class (kernel size, data type, stride for 3x3; tensor path,
+    // filters on M), at most ten to a launch; whatever is left over, or declined by the launcher, runs as single calls.
+    std::vector<char> done((size_t)n, 0);
+    int count = 0;
+    for (int i = 0; i < n; ++i) {
+        if (done[(size_t)i]) continue;
+        const rtoss_packed* ps[10];
+        const void* xs[10];
+        void* ys[10];
+        const rtoss_conv_desc* ds[10];
+        int idx[10], m = 0;
+        for (int j = i; j < n && m < 10; ++j) {
+            if (done[(size_t)j]) continue;
+            const rtoss_conv_item& a = items[j];
+            const rtoss_conv_item& b = items[i];
+            if (a.desc.path == RTOSS_PATH_FMA || !rtoss_tc_groupable(a.packed, &a.desc, a.x_dev, a.y_dev)) continue;
+            if (a.packed->ksize != b.packed->ksize || a.packed->dtype != b.packed->dtype) continue;
+            if (a.packed->ksize == 3 && a.desc.stride != b.desc.stride) continue;
+            ps[m] = a.packed, xs[m] = a.x_dev, ys[m] = a.y_dev, ds[m] = &a.desc, idx[m] = j;
+            ++m;
+        }
+        if (m >= 2 && items[i].desc.path != RTOSS_PATH_FMA) {
+            const int e = rtoss_launch_conv_tc_group(ctx, m, ps, xs, ys, ds, cuda_stream);
+            if (e == 0) {
+                for (int q = 0; q < m; ++q) done[(size_t)idx[q]] = 1;
+                ++count;
+                continue;
+            }
+            if (e > 0) return cuda_fail(ctx, "conv group launch", e);
+        }
+        rtoss_status st = RTOSS_OK;
+        const int e = dispatch_conv(ctx, items[i].packed, items[i].x_dev, items[i].y_dev, &items[i].desc, cuda_stream, &st);
+        if (st != RTOSS_OK) return st;
+        if (e) return cuda_fail(ctx, "conv launch", e);
+        done[(size_t)i] = 1;
+        ++count;
+    }
+    if (launches) *launches = count;
+    return RTOSS_OK;
+}
+
+rtoss_status rtoss_set_wait_limit(rtoss_ctx* ctx, long long sm_cycles) {
+    if (!ctx || sm_cycles < 1000) return RTOSS_ERR_INVALID_ARG;
+    ctx->wait_cycles = sm_cycles;
+    return RTOSS_OK;
+}
+
+rtoss_status rtoss_inject_lost_copy(rtoss_ctx* ctx) {
+    if (!ctx) return RTOSS_ERR_INVALID_ARG;
+    ctx->inject_next = 1;
+    return RTOSS_OK;
 }
 
 rtoss_status rtoss_device_status(rtoss_ctx* ctx, int* code) {

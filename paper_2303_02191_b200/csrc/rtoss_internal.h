@@ -32,6 +32,8 @@ struct rtoss_ctx {
     void* h_ev_in[8];   // cudaEvent_t per batch chunk: copy in done
     void* h_ev_run[8];  // kernel done
     int* dev_status;  // device word: 0, or the code of a bounded device-side wait that ran out
+    long long wait_cycles;     // limit of every device-side wait of the tensor path, in SM clock cycles
+    mutable int inject_next;   // failure-detection test hook: the next tensor-path launch withholds its first weight copy
     mutable rtoss_tmap_entry tmap_cache[32];  // activation descriptors of the tensor path, round robin
     mutable int tmap_next;
 };
@@ -47,6 +49,9 @@ struct rtoss_packed {
     uint32_t* bucket_off;  // [Cin*(P+1)]     (ksize 3)
     uint16_t* masks_dev;   // [256]
     void* wtc;             // tensor path: dense-expanded weights [taps][Cout][Cin] in dtype, or NULL
+    unsigned long long* issue;  // tensor path, ksize 3: per (tile of 128 filters, block of 64 channels) which (tap, 16-channel
+                                // slab) pairs hold any kept weight (bit 4*tap + slab); [issue_n] words, or NULL
+    int issue_n;
     mutable rtoss_tmap_entry wtc_map;  // its TMA descriptor, encoded at first use
     uint16_t masks[256];
 };
@@ -100,17 +105,28 @@ int rtoss_launch_pack_values(const void* w, rtoss_dtype wdt, int64_t n_kernels, 
                              int k, void* val, rtoss_dtype vdt, uint8_t* pid_copy, void* wtc, int ksize, int Cout, int Cin,
                              void* stream);
 int rtoss_launch_pack_order(const uint8_t* pid, int Cout, int Cin, int P, uint32_t* perm, uint32_t* bucket_off,
-                            void* stream);
+                            const uint16_t* masks_dev, unsigned long long* issue, void* stream);
+int rtoss_launch_select_shared(const void* w, rtoss_dtype wdt, int Cout, int Cin, int FB, int CB, const MaskTable& t, int P,
+                               uint8_t* pid, void* stream);
 int rtoss_launch_to_dense(const rtoss_packed* p, void* w_out, void* stream);
 int rtoss_launch_pid_histogram(const uint8_t* pid, int64_t n, int P, unsigned long long* counts, void* stream);
 int rtoss_launch_conv3x3(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y,
                          const rtoss_conv_desc* d, void* stream);
 int rtoss_launch_conv1x1(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y,
                          const rtoss_conv_desc* d, void* stream);
+// Number of issue words of a layer (tiles of 128 filter rows x blocks of 64 channels).
+static inline int rtoss_issue_words(int Cout, int Cin, int ksize) {
+    return ((rtoss_wtc_layout_of(Cout, ksize).rows + 127) / 128) * ((Cin + 63) / 64);
+}
+
 // tensor path (conv_tc.cu)
 bool rtoss_tc_weights_eligible(const rtoss_packed* p);
 bool rtoss_tc_eligible(const rtoss_packed* p, const rtoss_conv_desc* d, const void* x, const void* y);
 int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y,
                          const rtoss_conv_desc* d, void* stream);
+bool rtoss_tc_groupable(const rtoss_packed* p, const rtoss_conv_desc* d, const void* x, const void* y);
+// several independent convolutions in one launch: 0 = launched, -1 = the set cannot share a launch (nothing launched)
+int rtoss_launch_conv_tc_group(const rtoss_ctx* ctx, int n, const rtoss_packed* const* ps, const void* const* xs,
+                               void* const* ys, const rtoss_conv_desc* const* ds, void* stream);
 
 #endif

@@ -73,18 +73,40 @@ __device__ __forceinline__ void pack_one(const float (&w)[9], unsigned m, int64_
 // Ranks inside a group of 32 filters come from __match_any_sync; `fill` is 256 words of shared memory of this warp.
 // Ids must be < P; a filter whose id is not is left out of perm (the channel's list is then short by it, the last
 // bucket ends before bucket_off's closing entry Cout) rather than written past the channel's slice.
+//
+// On the way the warp also records which taps the tensor path has to multiply at all: `issue` (nullable) holds one
+// 64-bit word per (tile of 128 filters, block of 64 input channels), bit 4 t + s set when some kernel of the tile
+// with its channel in 16-channel slab s of the block keeps tap t (the union of the kept taps over the tile, from
+// `masks`, the table as the device sees it).  The words must be zero before the pass; channels add their bits with
+// atomicOr.  A (tile, slab, tap) whose bit stays clear holds only pruned weights: its matrix instruction is skipped.
 __device__ __forceinline__ void order_channel(const uint8_t* __restrict__ pid, int Cout, int Cin, int P, int ci,
                                               uint32_t* __restrict__ perm, uint32_t* __restrict__ bucket_off,
-                                              uint32_t* fill, int lane) {
+                                              uint32_t* fill, int lane, const uint16_t* __restrict__ masks = nullptr,
+                                              unsigned long long* __restrict__ issue = nullptr) {
     for (int p = lane; p < 256; p += 32) fill[p] = 0;
     __syncwarp();
     // pass 1: histogram
+    unsigned used = 0;   // taps kept by any filter of the current tile of 128
+    const int ncb = (Cin + 63) >> 6;
     for (int base = 0; base < Cout; base += 32) {
         const int co = base + lane;
         unsigned key = co < Cout ? pid[(size_t)co * Cin + ci] : 0xFFFFu;
         if (key >= (unsigned)P) key = 0xFFFFu;   // an id outside the table is not placed (nothing is written for it)
         const unsigned peers = __match_any_sync(0xFFFFFFFFu, key);
         if (key != 0xFFFFu && lane == __ffs(peers) - 1) fill[key] += __popc(peers);
+        if (issue) {
+            used |= __reduce_or_sync(0xFFFFFFFFu, key != 0xFFFFu ? (unsigned)masks[key] : 0u);
+            if (((base + 32) & 127) == 0 || base + 32 >= Cout) {
+                if (lane == 0 && used) {
+                    unsigned long long bits = 0;
+#pragma unroll
+                    for (int t = 0; t < 9; ++t)
+                        if (used & (1u << t)) bits |= 1ull << (4 * t + ((ci & 63) >> 4));
+                    atomicOr(issue + (size_t)(base >> 7) * ncb + (ci >> 6), bits);
+                }
+                used = 0;
+            }
+        }
         __syncwarp();
     }
     // exclusive scan over the P buckets (P <= 255: eight per lane, then a warp scan of lane totals)

@@ -103,13 +103,82 @@ __global__ void __launch_bounds__(kSelThreads) pack_values_kernel(const T* __res
 constexpr int kOrderWarps = 4;
 __global__ void __launch_bounds__(kOrderWarps * 32) pack_order_kernel(const uint8_t* __restrict__ pid, int Cout, int Cin,
                                                                       int P, uint32_t* __restrict__ perm,
-                                                                      uint32_t* __restrict__ bucket_off) {
+                                                                      uint32_t* __restrict__ bucket_off,
+                                                                      const uint16_t* __restrict__ masks,
+                                                                      unsigned long long* __restrict__ issue) {
     rtoss_dev::pdl_enter();
     __shared__ uint32_t fill_all[kOrderWarps][256];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ci = blockIdx.x * kOrderWarps + warp;
     if (ci >= Cin) return;  // whole warp leaves together; no block-wide barrier below
-    rtoss_dev::order_channel(pid, Cout, Cin, P, ci, perm, bucket_off, fill_all[warp], lane);
+    rtoss_dev::order_channel(pid, Cout, Cin, P, ci, perm, bucket_off, fill_all[warp], lane, masks, issue);
+}
+
+// Selection with one pattern per block of FB filters x CB input channels (a variant of Algorithm 2 in the spirit of
+// Section IV.C's shared kernel masks): the pattern that retains the most energy of the whole block.  One CTA per
+// block, one thread per filter of the block.  Arithmetic, fixed so that the ids are reproducible:
+//   q = w*w rounded to fp32, widened to double;  r[co][t] = sum over the block's channels, ascending, in double;
+//   E[t] = sum over the block's filters, ascending, of r[co][t];  S_p = sum over the taps of mask p, ascending, of E[t];
+//   first strictly larger S_p wins (ties -> lowest id, a NaN sum never wins).
+constexpr int kSharedMaxFB = 256;
+template <typename T>
+__global__ void __launch_bounds__(kSharedMaxFB) select_shared_kernel(const T* __restrict__ w, int Cout, int Cin, int FB, int CB,
+                                                                      MaskTable table, int P, uint8_t* __restrict__ pid) {
+    rtoss_dev::pdl_enter();
+    __shared__ double r[kSharedMaxFB][9];
+    __shared__ double E[9];
+    __shared__ int s_best;
+    const int nbc = (Cin + CB - 1) / CB, nbf = (Cout + FB - 1) / FB;
+    for (int blk = blockIdx.x; blk < nbc * nbf; blk += gridDim.x) {
+        const int co0 = (blk / nbc) * FB, ci0 = (blk % nbc) * CB;
+        const int co1 = min(co0 + FB, Cout), ci1 = min(ci0 + CB, Cin);
+        const int co = co0 + (int)threadIdx.x;
+        if (co < co1) {
+            double acc[9];
+#pragma unroll
+            for (int t = 0; t < 9; ++t) acc[t] = 0.0;
+            const T* kw = w + ((size_t)co * Cin + ci0) * 9;
+            for (int ci = ci0; ci < ci1; ++ci, kw += 9) {
+#pragma unroll
+                for (int t = 0; t < 9; ++t) {
+                    const float v = widen<T>(kw[t]);
+                    acc[t] = __dadd_rn(acc[t], (double)__fmul_rn(v, v));
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < 9; ++t) r[threadIdx.x][t] = acc[t];
+        }
+        __syncthreads();
+        if (threadIdx.x < 9) {
+            double e = 0.0;
+            for (int f = 0; f < co1 - co0; ++f) e = __dadd_rn(e, r[f][threadIdx.x]);
+            E[threadIdx.x] = e;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int best = 0;
+            double best_s = 0.0;
+            for (int p = 0; p < P; ++p) {
+                const unsigned m = table.m[p];
+                double sv = 0.0;
+                for (int t = 0; t < 9; ++t)
+                    if (m & (1u << t)) sv = __dadd_rn(sv, E[t]);
+                if (p == 0) {
+                    best_s = sv;
+                } else if (sv > best_s || (best_s != best_s && sv == sv)) {
+                    best = p;
+                    best_s = sv;
+                }
+            }
+            s_best = best;
+        }
+        __syncthreads();
+        if (co < co1) {
+            const uint8_t b = (uint8_t)s_best;
+            for (int ci = ci0; ci < ci1; ++ci) pid[(size_t)co * Cin + ci] = b;
+        }
+        __syncthreads();
+    }
 }
 
 // Dense masked weights from the packed form, one thread per dense element.
@@ -183,10 +252,28 @@ int rtoss_launch_pack_values(const void* w, rtoss_dtype wdt, int64_t n_kernels, 
 }
 
 int rtoss_launch_pack_order(const uint8_t* pid, int Cout, int Cin, int P, uint32_t* perm, uint32_t* bucket_off,
-                            void* stream) {
+                            const uint16_t* masks_dev, unsigned long long* issue, void* stream) {
     const int grid = (Cin + kOrderWarps - 1) / kOrderWarps;
-    rtoss_dev::launch_pdl(pack_order_kernel, grid, kOrderWarps * 32, 0, (cudaStream_t)stream, pid, Cout, Cin, P, perm, bucket_off);
+    rtoss_dev::launch_pdl(pack_order_kernel, grid, kOrderWarps * 32, 0, (cudaStream_t)stream, pid, Cout, Cin, P, perm, bucket_off,
+                          masks_dev, issue);
     return (int)cudaGetLastError();
+}
+
+int rtoss_launch_select_shared(const void* w, rtoss_dtype wdt, int Cout, int Cin, int FB, int CB, const MaskTable& t, int P,
+                               uint8_t* pid, void* stream) {
+    cudaStream_t s = (cudaStream_t)stream;
+    const int64_t blocks = (int64_t)((Cout + FB - 1) / FB) * ((Cin + CB - 1) / CB);
+    const int grid = grid_for(blocks);
+    const int threads = ((FB < Cout ? FB : Cout) + 31) / 32 * 32;
+    cudaError_t e = cudaErrorInvalidValue;
+    switch (wdt) {
+        case RTOSS_F32: e = rtoss_dev::launch_pdl(select_shared_kernel<float>, grid, threads, 0, s, (const float*)w, Cout, Cin, FB, CB, t, P, pid); break;
+        case RTOSS_BF16:
+            e = rtoss_dev::launch_pdl(select_shared_kernel<__nv_bfloat16>, grid, threads, 0, s, (const __nv_bfloat16*)w, Cout, Cin, FB, CB, t, P, pid);
+            break;
+        case RTOSS_F16: e = rtoss_dev::launch_pdl(select_shared_kernel<__half>, grid, threads, 0, s, (const __half*)w, Cout, Cin, FB, CB, t, P, pid); break;
+    }
+    return (int)e;
 }
 
 int rtoss_launch_to_dense(const rtoss_packed* p, void* w_out, void* stream) {

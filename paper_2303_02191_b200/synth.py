@@ -165,6 +165,42 @@ def retinanet_r50fpn_stack(H0=800, W0=1088):
     return layers
 
 
+def independent_sets(layers):
+    """Launch units of a layer table: lists of layer indices, in execution order, whose members do not depend on one
+    another in the network the table was taken from, so that they may run side by side (one grouped launch).
+      YOLOv5s-shaped: the two 1x1 branches (cv1, cv2) that open a C3 block read the same input.
+      RetinaNet-shaped: tower layer i of both towers on all five pyramid levels (each needs only tower layer i-1 of
+      its own tower and level); the three 3x3 pyramid outputs; the three 1x1 laterals; the first 1x1 of a stage's first
+      bottleneck and that block's 1x1 projection (both read the block input).
+    Every other layer is a unit of its own."""
+    import re
+    key_of = {}
+    for i, L in enumerate(layers):
+        n = L["name"]
+        m = re.match(r"(cls|box)_tower(\d)\.p\d$", n)
+        if m:
+            key_of[i] = "tower%s" % m.group(2)
+        elif re.match(r"fpn\.output\d$", n):
+            key_of[i] = "fpn.output"
+        elif re.match(r"fpn\.lateral\d$", n):
+            key_of[i] = "fpn.lateral"
+        elif re.match(r"layer\d\.0\.(conv1|downsample)$", n):
+            key_of[i] = n.rsplit(".", 1)[0] + ".in"
+        elif re.match(r".*c3_\d\.cv[12]$", n):
+            key_of[i] = n.rsplit(".", 1)[0] + ".in"
+    units, at = [], {}
+    for i in range(len(layers)):
+        k = key_of.get(i)
+        if k is None:
+            units.append([i])
+        elif k in at:
+            units[at[k]].append(i)
+        else:
+            at[k] = len(units)
+            units.append([i])
+    return units
+
+
 def layer_nnz_flops(layer, N, k):
     """2 * (kept multiply-adds) of one call at batch N with k kept taps."""
     Ho, Wo = out_hw(layer["H"], layer["W"], layer["stride"])
