@@ -112,20 +112,25 @@ struct TcArgs {
     int KS, cb_per;
 };
 
-// A launch: up to kMaxProb convolutions sharing the CTA's rings (stage sizes are the largest any of them needs).
-struct TcLaunch {
+// A launch: up to NP convolutions sharing the CTA's rings (stage sizes are the largest any of them needs).  The struct
+// travels as the kernel's parameter: a launch of one convolution carries the small instantiation (a large parameter
+// block costs launch time).
+template <int NP>
+struct TcLaunchT {
     int n_prob;
-    int unit_end[kMaxProb];   // units (tile x share of the channel blocks) of problems 0..i
+    int unit_end[NP];   // units (tile x share of the channel blocks) of problems 0..i
     int* status;
     long long wait_cycles;    // limit of every wait
     int inject;               // test hook: 1 = the first weight copy of the launch is withheld (the wait for it must run out)
     int a_stage_bytes, b_stage_bytes, NA, NB;  // stage sizes, activation stages, weight stages
     int AS, acc_stride;                        // accumulator stages in TMEM and columns per stage
     int tmem_cols;
-    TcArgs prob[kMaxProb];
-    CUtensorMap tmA[kMaxProb], tmB[kMaxProb];
+    TcArgs prob[NP];
+    CUtensorMap tmA[NP], tmB[NP];
 };
-static_assert(sizeof(TcLaunch) <= 8192, "kernel parameters: well inside the 32 KB a launch may carry");
+using TcLaunch1 = TcLaunchT<1>;
+using TcLaunchN = TcLaunchT<kMaxProb>;
+static_assert(sizeof(TcLaunchN) <= 8192, "kernel parameters: well inside the 32 KB a launch may carry");
 
 __device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
 
@@ -602,16 +607,22 @@ __device__ __forceinline__ void epilogue_from_shares(unsigned buf, int KS, int r
 }
 
 // Which problem a unit of the launch's list belongs to, and its index inside that problem.
-__device__ __forceinline__ int find_problem(const TcLaunch& g, int unit, int& local) {
+template <bool kMulti, typename G>
+__device__ __forceinline__ int find_problem(const G& g, int unit, int& local) {
+    if (!kMulti) {   // a launch of one problem: the index is a compile-time constant
+        local = unit;
+        return 0;
+    }
     int pi = 0;
     while (pi + 1 < g.n_prob && unit >= g.unit_end[pi]) ++pi;
     local = unit - (pi ? g.unit_end[pi - 1] : 0);
     return pi;
 }
 
-template <typename T>
+template <typename T, typename G>
 __global__ void __launch_bounds__(kTcThreads, 1)
-conv_tc_kernel(const __grid_constant__ TcLaunch g) {
+conv_tc_kernel(const __grid_constant__ G g) {
+    constexpr bool kMulti = sizeof(G) > sizeof(TcLaunch1);
     extern __shared__ unsigned char smem_dyn[];
     // tiles need 1024-byte alignment for the 128-byte swizzle pattern
     const unsigned base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -691,7 +702,7 @@ conv_tc_kernel(const __grid_constant__ TcLaunch g) {
             unsigned pa = 0;
             for (int unit = blockIdx.x; unit < n_tiles && ok; unit += gridDim.x) {
                 int local;
-                const int pi = find_problem(g, unit, local);
+                const int pi = find_problem<kMulti>(g, unit, local);
                 const TcArgs& a = g.prob[pi];
                 const int ks = local % a.KS;
                 int rest = local / a.KS / a.co_tiles;
@@ -724,7 +735,7 @@ conv_tc_kernel(const __grid_constant__ TcLaunch g) {
             unsigned pb = 0;
             for (int unit = blockIdx.x; unit < n_tiles && ok; unit += gridDim.x) {
                 int local;
-                const int pi = find_problem(g, unit, local);
+                const int pi = find_problem<kMulti>(g, unit, local);
                 const TcArgs& a = g.prob[pi];
                 const int ks = local % a.KS, cot = (local / a.KS) % a.co_tiles;
                 const int co0 = cot * (a.pxm ? a.n_cols : kMTile);
@@ -793,7 +804,7 @@ conv_tc_kernel(const __grid_constant__ TcLaunch g) {
             };
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++n_done) {
                 int local;
-                const int pi = find_problem(g, tile, local);
+                const int pi = find_problem<kMulti>(g, tile, local);
                 const TcArgs& a = g.prob[pi];
                 if (pi != cur_pi) {
                     cur_pi = pi;
@@ -1000,7 +1011,7 @@ conv_tc_kernel(const __grid_constant__ TcLaunch g) {
         } else
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++gt) {
             int local;
-            const int pi = find_problem(g, tile, local);
+            const int pi = find_problem<kMulti>(g, tile, local);
             const TcArgs& a = g.prob[pi];
             T* __restrict__ yg = reinterpret_cast<T*>(a.y);
             const uint2* pos_tab = pos_tab_all + pi * kMaxPx;
@@ -1373,16 +1384,21 @@ int ensure_smem_attr(const rtoss_ctx* ctx) {
     static std::atomic<bool> attr_set[64];
     const int dev_slot = ctx->device >= 0 && ctx->device < 64 ? ctx->device : -1;
     if (dev_slot < 0 || !attr_set[dev_slot].load(std::memory_order_acquire)) {
-        cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel<__nv_bfloat16, TcLaunch1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(conv_tc_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+            e = cudaFuncSetAttribute(conv_tc_kernel<__half, TcLaunch1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(conv_tc_kernel<__nv_bfloat16, TcLaunchN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(conv_tc_kernel<__half, TcLaunchN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return (int)e;
         if (dev_slot >= 0) attr_set[dev_slot].store(true, std::memory_order_release);
     }
     return 0;
 }
 
-void launch_common(const rtoss_ctx* ctx, TcLaunch* g) {
+template <typename G>
+void launch_common(const rtoss_ctx* ctx, G* g) {
     g->status = ctx->dev_status;
     g->wait_cycles = ctx->wait_cycles > 0 ? ctx->wait_cycles : kWaitCycles;
     g->inject = 0;
@@ -1421,7 +1437,7 @@ bool rtoss_tc_groupable(const rtoss_packed* p, const rtoss_conv_desc* d, const v
 int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y, const rtoss_conv_desc* d,
                          void* stream) {
     const int sms = ctx->sm_count > 0 ? ctx->sm_count : 148;
-    static thread_local TcLaunch g;   // several KB: kept off the stack
+    static thread_local TcLaunch1 g;   // several KB: kept off the stack
     ProbPlan pp;
     g.n_prob = 1;
     int e = build_problem(ctx, p, x, y, d, 1, sms, &g.prob[0], &pp, &g.tmA[0], &g.tmB[0]);
@@ -1478,8 +1494,8 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     cudaError_t le;
     if (a.KS > 1) {
         // one cluster per tile; if the device cannot place the clusters the layer runs uncut
-        le = a.is_bf16 ? rtoss_dev::launch_pdl(conv_tc_kernel<__nv_bfloat16>, grid, kTcThreads, smem, (cudaStream_t)stream, a.KS, g)
-                       : rtoss_dev::launch_pdl(conv_tc_kernel<__half>, grid, kTcThreads, smem, (cudaStream_t)stream, a.KS, g);
+        le = a.is_bf16 ? rtoss_dev::launch_pdl(conv_tc_kernel<__nv_bfloat16, TcLaunch1>, grid, kTcThreads, smem, (cudaStream_t)stream, a.KS, g)
+                       : rtoss_dev::launch_pdl(conv_tc_kernel<__half, TcLaunch1>, grid, kTcThreads, smem, (cudaStream_t)stream, a.KS, g);
         if (le == cudaSuccess) return 0;
         cudaGetLastError();
         a.KS = 1;
@@ -1488,8 +1504,8 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
         g.unit_end[0] = (int)n_units;
         grid = dim3((unsigned)(n_units < (size_t)sms ? n_units : (size_t)sms));
     }
-    le = a.is_bf16 ? rtoss_dev::launch_pdl(conv_tc_kernel<__nv_bfloat16>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g)
-                   : rtoss_dev::launch_pdl(conv_tc_kernel<__half>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g);
+    le = a.is_bf16 ? rtoss_dev::launch_pdl(conv_tc_kernel<__nv_bfloat16, TcLaunch1>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g)
+                   : rtoss_dev::launch_pdl(conv_tc_kernel<__half, TcLaunch1>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g);
     return (int)le;
 }
 
@@ -1506,7 +1522,7 @@ int rtoss_launch_conv_tc_group(const rtoss_ctx* ctx, int n, const rtoss_packed* 
         if (ps[i]->ksize == 3 && ds[i]->stride != ds[0]->stride) return -1;   // (3x3: stride 2 stages four sub-tiles per block)
         if (!rtoss_tc_eligible(ps[i], ds[i], xs[i], ys[i])) return -1;
     }
-    static thread_local TcLaunch g;
+    static thread_local TcLaunchN g;
     ProbPlan pp[kMaxProb];
     bool resid = false;
     for (int i = 0; i < n; ++i) resid = resid || ds[i]->residual_dev != nullptr;
@@ -1568,7 +1584,7 @@ int rtoss_launch_conv_tc_group(const rtoss_ctx* ctx, int n, const rtoss_packed* 
     int e = ensure_smem_attr(ctx);
     if (e) return e;
     const bool bf = ps[0]->dtype == RTOSS_BF16;
-    cudaError_t le = bf ? rtoss_dev::launch_pdl(conv_tc_kernel<__nv_bfloat16>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g)
-                        : rtoss_dev::launch_pdl(conv_tc_kernel<__half>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g);
+    cudaError_t le = bf ? rtoss_dev::launch_pdl(conv_tc_kernel<__nv_bfloat16, TcLaunchN>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g)
+                        : rtoss_dev::launch_pdl(conv_tc_kernel<__half, TcLaunchN>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g);
     return (int)le;
 }
