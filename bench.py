@@ -278,12 +278,12 @@ def run_network(args):
     side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
         for _ in range(max(args.warmup, 3)):
-            net.run()
+            net.run(grouped=args.group)
     torch.cuda.current_stream().wait_stream(side)
     torch.cuda.synchronize()
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
-        net.run()
+        net.run(grouped=args.group)
     graph.replay()
     torch.cuda.synchronize()
     if ctx.rtoss_device_status() != 0:
@@ -308,9 +308,10 @@ def run_network(args):
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.workload, "batch": N, "layout": "NHWC", "l2": "flushed between steps (256 MB write)",
                    "launch": "one CUDA graph per step", "convs": len(net.layers), "glue_kernels": n_glue,
+                   "launches_per_step": net.launches,
                    "residual_adds_inside_convs": sum(1 for op in net.ops if op[0] == "convres") - len(getattr(net, "unfused", ())),
                    "note": "chained network: every layer consumes the previous layer's output"},
-        "nnz_gflops_per_s": flops / (ms * 1e-3) / 1e9, "clocks": clocks, "gpu_launches": (len(net.layers) + n_glue) * args.steps,
+        "nnz_gflops_per_s": flops / (ms * 1e-3) / 1e9, "clocks": clocks, "gpu_launches": net.launches * args.steps,
     }))
     net.close()
     ctx.close()

@@ -8,7 +8,7 @@ pattern set).  The same description drives `GpuNet` here (the C-ABI library, NHW
 capture) and the tests' CPU-oracle executor.  Only shapes come from the model family; weights are seeded and
 synthetic.
 """
-from . import synth
+from . import schedule, synth
 
 
 def program(H0, W0):
@@ -123,6 +123,7 @@ class GpuNet:
         if fuse_residual:
             self.ops = fuse_adds(self.ops, self.output_names)
         self.unfused = set()   # layers whose fused call the library declined: convolution and add run separately
+        self.rounds, self.probed = None, False
         tdt = {"bf16": torch.bfloat16, "f16": torch.float16}[dtype]
         self.t = {n: torch.zeros((N, H, W, C), dtype=tdt, device="cuda") for n, (C, H, W) in self.bufs.items()}
         self.zero = {}   # all-zero operands of the ReLU glue op, one per shape
@@ -144,37 +145,84 @@ class GpuNet:
     def set_input(self, x_nchw):
         self.t["in"].copy_(self.torch.from_numpy(x_nchw).permute(0, 2, 3, 1).to(self.t["in"].dtype))
 
-    def run(self):
+    def _reads(self, op):
+        if op[0] == "conv":
+            return (op[2],)
+        if op[0] == "convres":
+            return (op[2], op[4])
+        if op[0] == "add":
+            return (op[1], op[2])
+        return (op[1],)
+
+    def _write(self, op):
+        return op[{"conv": 3, "convres": 5, "add": 3, "up": 2, "relu": 2}[op[0]]]
+
+    def run(self, grouped=True):
+        """One pass.  grouped: operations are issued round by round (schedule.levels) and the convolutions of a round go
+        out through rtoss_conv_group; else one call per operation in program order."""
+        self.launches = 0      # kernel launches of this pass
+        if not grouped or not self.probed:
+            for op in self.ops:
+                self._run_op(op)
+            self.probed = True     # the first pass finds out which fused residual calls the library declines
+            return
+        if self.rounds is None:
+            # as late as possible: tower layer i of every pyramid level then shares a round (and a launch)
+            self.rounds = schedule.levels(self.ops, self._reads, self._write, late=True)
+        for rnd in self.rounds:
+            convs = [self.ops[i] for i in rnd if self.ops[i][0] == "conv" or (self.ops[i][0] == "convres" and self.ops[i][1] not in self.unfused)]
+            rest = [self.ops[i] for i in rnd if not (self.ops[i][0] == "conv" or (self.ops[i][0] == "convres" and self.ops[i][1] not in self.unfused))]
+            if len(convs) >= 2:
+                self.launches += self.ctx.rtoss_conv_group([self._item(op) for op in convs])
+            else:
+                rest = convs + rest
+            for op in rest:
+                self._run_op(op)
+
+    def _item(self, op):
         rt, N, t = self.rt, self.N, self.t
-        for op in self.ops:
-            if op[0] == "conv":
-                _, i, src, dst, act = op
-                L = self.layers[i]
-                fn = self.ctx.rtoss_conv3x3_pattern if L["ksize"] == 3 else self.ctx.rtoss_conv1x1_pattern
-                fn(self.packed[L["wid"]], t[src], t[dst], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_NAMES[act],
-                   self.bias[L["wid"]])
-            elif op[0] == "convres":   # convolution (no activation) + residual + activation in one call
-                _, i, src, tmp, other, dst, act = op
-                L = self.layers[i]
-                fn = self.ctx.rtoss_conv3x3_pattern if L["ksize"] == 3 else self.ctx.rtoss_conv1x1_pattern
-                args = (self.packed[L["wid"]], t[src], None, N, L["H"], L["W"], L["stride"], rt.NHWC)
-                if i not in self.unfused:
-                    try:
-                        fn(*args[:2], t[dst], *args[3:], rt.ACT_NAMES[act], self.bias[L["wid"]], residual=t[other])
-                        continue
-                    except rt.RtossError as err:
-                        if err.status != rt.ERR_UNSUPPORTED:
-                            raise
-                        self.unfused.add(i)
-                fn(*args[:2], t[tmp], *args[3:], rt.ACT_NONE, self.bias[L["wid"]])
-                rt.rtoss_add_act(t[tmp], t[other], t[dst], rt.ACT_NAMES[act])
-            elif op[0] == "add":
-                rt.rtoss_add_act(t[op[1]], t[op[2]], t[op[3]], rt.ACT_NAMES[op[4]])
-            elif op[0] == "up":
-                C, H, W = self.bufs[op[1]]
-                rt.rtoss_upsample2x(t[op[1]], t[op[2]], N, C, H, W, rt.NHWC)
-            elif op[0] == "relu":
-                rt.rtoss_add_act(t[op[1]], self.zero[self.bufs[op[1]]], t[op[2]], rt.ACT_RELU)
+        L = self.layers[op[1]]
+        if op[0] == "conv":
+            _, i, src, dst, act = op
+            return self.ctx.conv_item(self.packed[L["wid"]], t[src], t[dst], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_NAMES[act],
+                                      self.bias[L["wid"]])
+        _, i, src, tmp, other, dst, act = op
+        return self.ctx.conv_item(self.packed[L["wid"]], t[src], t[dst], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_NAMES[act],
+                                  self.bias[L["wid"]], residual=t[other])
+
+    def _run_op(self, op):
+        rt, N, t = self.rt, self.N, self.t
+        self.launches += 1
+        if op[0] == "conv":
+            _, i, src, dst, act = op
+            L = self.layers[i]
+            fn = self.ctx.rtoss_conv3x3_pattern if L["ksize"] == 3 else self.ctx.rtoss_conv1x1_pattern
+            fn(self.packed[L["wid"]], t[src], t[dst], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_NAMES[act],
+               self.bias[L["wid"]])
+        elif op[0] == "convres":   # convolution (no activation) + residual + activation in one call
+            _, i, src, tmp, other, dst, act = op
+            L = self.layers[i]
+            fn = self.ctx.rtoss_conv3x3_pattern if L["ksize"] == 3 else self.ctx.rtoss_conv1x1_pattern
+            args = (self.packed[L["wid"]], t[src], None, N, L["H"], L["W"], L["stride"], rt.NHWC)
+            if i not in self.unfused:
+                try:
+                    fn(*args[:2], t[dst], *args[3:], rt.ACT_NAMES[act], self.bias[L["wid"]], residual=t[other])
+                    return
+                except rt.RtossError as err:
+                    if err.status != rt.ERR_UNSUPPORTED:
+                        raise
+                    self.unfused.add(i)
+                    self.rounds = None
+            fn(*args[:2], t[tmp], *args[3:], rt.ACT_NONE, self.bias[L["wid"]])
+            rt.rtoss_add_act(t[tmp], t[other], t[dst], rt.ACT_NAMES[act])
+            self.launches += 1
+        elif op[0] == "add":
+            rt.rtoss_add_act(t[op[1]], t[op[2]], t[op[3]], rt.ACT_NAMES[op[4]])
+        elif op[0] == "up":
+            C, H, W = self.bufs[op[1]]
+            rt.rtoss_upsample2x(t[op[1]], t[op[2]], N, C, H, W, rt.NHWC)
+        elif op[0] == "relu":
+            rt.rtoss_add_act(t[op[1]], self.zero[self.bufs[op[1]]], t[op[2]], rt.ACT_RELU)
 
     def outputs(self):
         return {n: self.t[n].float().permute(0, 3, 1, 2).cpu().numpy() for n in self.output_names}

@@ -8,7 +8,7 @@ Only shapes come from the model family; weights are seeded and synthetic.
 """
 import numpy as np
 
-from . import synth
+from . import schedule, synth
 
 
 def program(H0, W0):
@@ -129,6 +129,7 @@ class GpuNet:
         if fuse_residual:
             self.ops = fuse_shortcuts(self.ops)
         self.unfused = set()   # layers whose fused call the library declined: convolution and add run separately
+        self.rounds, self.probed = None, False
         tdt = {"bf16": torch.bfloat16, "f16": torch.float16}[dtype]
         self.t = {n: torch.zeros((N, H, W, C), dtype=tdt, device="cuda") for n, (C, H, W) in self.bufs.items()}
         masks = rt.rtoss_pattern_preset(k, rt.PRESET_CENTRE8 if k == 4 else rt.PRESET_CONN4)
@@ -143,41 +144,91 @@ class GpuNet:
     def set_input(self, x_nchw):
         self.t["in"].copy_(self.torch.from_numpy(x_nchw).permute(0, 2, 3, 1).to(self.t["in"].dtype))
 
-    def run(self):
+    def _reads(self, op):
+        if op[0] == "conv":
+            return (op[2],)
+        if op[0] == "convres":
+            return (op[2], op[4])
+        if op[0] == "add":
+            return (op[1], op[2])
+        return (op[1],)
+
+    def _write(self, op):
+        return op[{"conv": 3, "convres": 5, "add": 3, "pool5": 2, "up": 2, "copy": 2}[op[0]]]
+
+    def run(self, grouped=True):
+        """One pass.  grouped: operations are issued round by round (schedule.levels: a buffer is ready when every slice
+        of it has been written) and the convolutions of a round go out through rtoss_conv_group; else one call per
+        operation in program order."""
+        self.launches = 0      # kernel launches of this pass
+        if not grouped or not self.probed:
+            for op in self.ops:
+                self._run_op(op)
+            self.probed = True     # the first pass finds out which fused shortcut calls the library declines
+            return
+        if self.rounds is None:
+            # as soon as possible: the two 1x1 branches that open a C3 block then share a round (and a launch)
+            self.rounds = schedule.levels(self.ops, self._reads, self._write, late=False)
+        for rnd in self.rounds:
+            is_conv = lambda op: op[0] == "conv" or (op[0] == "convres" and op[1] not in self.unfused)
+            convs = [self.ops[i] for i in rnd if is_conv(self.ops[i])]
+            rest = [self.ops[i] for i in rnd if not is_conv(self.ops[i])]
+            if len(convs) >= 2:
+                self.launches += self.ctx.rtoss_conv_group([self._item(op) for op in convs])
+            else:
+                rest = convs + rest
+            for op in rest:
+                self._run_op(op)
+
+    def _item(self, op):
         rt, N, t = self.rt, self.N, self.t
-        for op in self.ops:
-            if op[0] == "conv":
-                _, i, src, dst, off = op
-                L = self.layers[i]
-                fn = self.ctx.rtoss_conv3x3_pattern if L["ksize"] == 3 else self.ctx.rtoss_conv1x1_pattern
-                fn(self.packed[i], t[src], t[dst], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_SILU, self.bias[i],
-                   off, self.bufs[dst][0])
-            elif op[0] == "convres":   # second convolution of a bottleneck + its shortcut in one call
-                _, i, src, tmp, other, dst = op
-                L = self.layers[i]
-                fn = self.ctx.rtoss_conv3x3_pattern if L["ksize"] == 3 else self.ctx.rtoss_conv1x1_pattern
-                if i not in self.unfused:
-                    try:
-                        fn(self.packed[i], t[src], t[dst], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_SILU, self.bias[i],
-                           residual=t[other], residual_after_act=True)
-                        continue
-                    except rt.RtossError as err:
-                        if err.status != rt.ERR_UNSUPPORTED:
-                            raise
-                        self.unfused.add(i)
-                fn(self.packed[i], t[src], t[tmp], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_SILU, self.bias[i])
-                rt.rtoss_add_act(t[other], t[tmp], t[dst], rt.ACT_NONE)
-            elif op[0] == "add":
-                rt.rtoss_add_act(t[op[1]], t[op[2]], t[op[3]], rt.ACT_NONE)
-            elif op[0] == "pool5":
-                C, H, W = self.bufs[op[1]]
-                rt.rtoss_maxpool2d(t[op[1]], t[op[2]], N, C, H, W, 5, 1, 2, rt.NHWC, op[3], self.bufs[op[2]][0])
-            elif op[0] == "up":
-                C, H, W = self.bufs[op[1]]
-                rt.rtoss_upsample2x(t[op[1]], t[op[2]], N, C, H, W, rt.NHWC, op[3], self.bufs[op[2]][0])
-            elif op[0] == "copy":
-                C, H, W = self.bufs[op[1]]
-                rt.rtoss_maxpool2d(t[op[1]], t[op[2]], N, C, H, W, 1, 1, 0, rt.NHWC, op[3], self.bufs[op[2]][0])
+        i = op[1]
+        L = self.layers[i]
+        if op[0] == "conv":
+            _, _, src, dst, off = op
+            return self.ctx.conv_item(self.packed[i], t[src], t[dst], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_SILU, self.bias[i],
+                                      off, self.bufs[dst][0])
+        _, _, src, tmp, other, dst = op
+        return self.ctx.conv_item(self.packed[i], t[src], t[dst], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_SILU, self.bias[i],
+                                  residual=t[other], residual_after_act=True)
+
+    def _run_op(self, op):
+        rt, N, t = self.rt, self.N, self.t
+        self.launches += 1
+        if op[0] == "conv":
+            _, i, src, dst, off = op
+            L = self.layers[i]
+            fn = self.ctx.rtoss_conv3x3_pattern if L["ksize"] == 3 else self.ctx.rtoss_conv1x1_pattern
+            fn(self.packed[i], t[src], t[dst], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_SILU, self.bias[i],
+               off, self.bufs[dst][0])
+        elif op[0] == "convres":   # second convolution of a bottleneck + its shortcut in one call
+            _, i, src, tmp, other, dst = op
+            L = self.layers[i]
+            fn = self.ctx.rtoss_conv3x3_pattern if L["ksize"] == 3 else self.ctx.rtoss_conv1x1_pattern
+            if i not in self.unfused:
+                try:
+                    fn(self.packed[i], t[src], t[dst], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_SILU, self.bias[i],
+                       residual=t[other], residual_after_act=True)
+                    return
+                except rt.RtossError as err:
+                    if err.status != rt.ERR_UNSUPPORTED:
+                        raise
+                    self.unfused.add(i)
+                    self.rounds = None
+            fn(self.packed[i], t[src], t[tmp], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_SILU, self.bias[i])
+            rt.rtoss_add_act(t[other], t[tmp], t[dst], rt.ACT_NONE)
+            self.launches += 1
+        elif op[0] == "add":
+            rt.rtoss_add_act(t[op[1]], t[op[2]], t[op[3]], rt.ACT_NONE)
+        elif op[0] == "pool5":
+            C, H, W = self.bufs[op[1]]
+            rt.rtoss_maxpool2d(t[op[1]], t[op[2]], N, C, H, W, 5, 1, 2, rt.NHWC, op[3], self.bufs[op[2]][0])
+        elif op[0] == "up":
+            C, H, W = self.bufs[op[1]]
+            rt.rtoss_upsample2x(t[op[1]], t[op[2]], N, C, H, W, rt.NHWC, op[3], self.bufs[op[2]][0])
+        elif op[0] == "copy":
+            C, H, W = self.bufs[op[1]]
+            rt.rtoss_maxpool2d(t[op[1]], t[op[2]], N, C, H, W, 1, 1, 0, rt.NHWC, op[3], self.bufs[op[2]][0])
 
     def outputs(self):
         return {n: self.t[n].float().permute(0, 3, 1, 2).cpu().numpy() for n in OUTPUTS}
