@@ -43,6 +43,9 @@ def workload_layers(name):
         return (1 if name.endswith("b1") else 16), "bf16", [(L, 4, "centre8") for L in synth.yolov5s_stack()]
     if name == "retinanet_b4":
         return 4, "bf16", [(L, 4, "centre8") for L in synth.retinanet_r50fpn_stack()]
+    if name == "retinanet_tower":
+        # the launch that dominates retinanet_b4: the first layer of both towers on the five pyramid levels
+        return 4, "bf16", [(L, 4, "centre8") for L in synth.retinanet_r50fpn_stack() if "_tower0." in L["name"]]
     raise SystemExit("unknown workload " + name)
 
 
@@ -226,7 +229,7 @@ def run_reference(args):
         "impl": "reference", "metric": "pattern-sparse conv images/sec", "value": value, "unit": "images/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
-        "config": {"workload": args.workload, "batch": N, "layout": "NCHW" if dtype == "f32" else "NHWC", "layers": len(layers_k),
+        "config": {"workload": args.workload, "batch": N, "layout": "NCHW" if args.layout == "nchw" else "NHWC", "layers": len(layers_k),
                    "l2": "not applicable (CPU oracle)", "multi_gpu": "rank 0 only", "launch": "host cores"},
         "cpu_baseline": {"value": value, "unit": "images/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -332,8 +335,8 @@ def measure_workload(ctx, rt, dev, name, steps, warmup, args, world, rank, full,
     elem = 4 if dtype == "f32" else 2
     cdt = rt.DTYPE_NAMES[dtype]
     preset_of = {"centre8": rt.PRESET_CENTRE8, "conn4": rt.PRESET_CONN4}
-    # 16-bit activations travel NHWC (what the tensor path takes), fp32 NCHW
-    layout = rt.NCHW if (dtype == "f32" or args.layout == "nchw") else rt.NHWC
+    # activations travel NHWC (what the tensor path takes) unless NCHW is asked for (FMA path)
+    layout = rt.NCHW if args.layout == "nchw" else rt.NHWC
 
     # ---- resident inputs (replicas: every rank holds its own batch and weights; no data-path collective)
     weights, L_state = {}, []
@@ -569,7 +572,10 @@ def roofline_of(res, hbm_peak, tc_peak, peak_kind):
     N, elem = res["N"], res["elem"]
     flops = np.array([synth.layer_nnz_flops(L, N, k) for L, k in zip(res["layers"], res["ks"])])
     bytes_ = np.array([synth.layer_bytes(L, N, k, elem) for L, k in zip(res["layers"], res["ks"])], dtype=np.float64)
-    pipe = np.array([tc_peak if tc else ALU_PEAK_TFLOPS for tc in res["on_tc"]]) * 1e12
+    # pipe peak per layer: the measured bf16 tensor peak; fp32 on the tensor path issues tf32 instructions (half the bf16
+    # rate) three times per product (head x head, head x remainder, remainder x head); else the nominal FMA peak
+    tc_eff = tc_peak if res["dtype"] != "f32" else tc_peak / 6
+    pipe = np.array([tc_eff if tc else ALU_PEAK_TFLOPS for tc in res["on_tc"]]) * 1e12
     t_pipe, t_hbm = flops / pipe, bytes_ / (hbm_peak * 1e9)
     t_roof = np.maximum(t_pipe, t_hbm)
     t_meas = res["conv_ms"] * 1e-3          # one entry per launch unit (a unit of several layers is one grouped call)
@@ -591,9 +597,9 @@ def roofline_of(res, hbm_peak, tc_peak, peak_kind):
     on_tc = res["on_tc"][members[0]]
     t_top = float(np.mean(t_meas[idx]))
     if t_pipe[members].sum() >= t_hbm[members].sum():
-        dom = {"bound": "tensor" if on_tc else "alu", "achieved": u_flops[top] / t_top / 1e12, "peak": pipe[members[0]] / 1e12,
-               "unit": "TFLOP/s",
-               "peak_kind": ("of %s (bf16 cuBLAS, sustained)" % peak_kind) if on_tc
+        dom = {"bound": ("tensor (tf32 x3)" if res["dtype"] == "f32" else "tensor") if on_tc else "alu",
+               "achieved": u_flops[top] / t_top / 1e12, "peak": pipe[members[0]] / 1e12, "unit": "TFLOP/s",
+               "peak_kind": ("of %s (bf16 cuBLAS, sustained)%s" % (peak_kind, " / 2 (tf32) / 3 (products per tap)" if res["dtype"] == "f32" else "")) if on_tc
                else "nominal, not measured: 148 SM x 128 FMA lanes x 2 x 1.965 GHz"}
     else:
         dom = {"bound": "hbm", "achieved": u_bytes[top] / t_top / 1e9, "peak": hbm_peak, "unit": "GB/s", "peak_kind": "of " + peak_kind}

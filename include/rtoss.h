@@ -294,7 +294,7 @@ typedef struct {
                                * act = none followed by rtoss_add_act gives, in one pass; for SiLU the same up to
                                * the rounding of the two SiLU evaluations (the residual connection that closes a
                                * bottleneck block; not part of the paper's method).  May be y itself.  Tensor
-                               * path only (16-bit NHWC, more than 64 filters or a 3x3 kernel, pointer 16-byte
+                               * path only (NHWC; 16-bit data with more than 64 filters or a 3x3 kernel, or fp32 data; pointer 16-byte
                                * aligned): other calls return RTOSS_ERR_UNSUPPORTED before anything is launched
                                * and the caller adds separately. */
     int residual_after_act;   /* 0: as above.  1: the residual is added behind the activation instead,
@@ -339,8 +339,11 @@ typedef struct {
 } rtoss_conv_item;
 rtoss_status rtoss_conv_group(rtoss_ctx* ctx, const rtoss_conv_item* items, int n, int* launches, void* cuda_stream);
 
-/* The tensor path (RTOSS_PATH_TENSOR, or RTOSS_PATH_AUTO when it applies) takes: bf16 / fp16 NHWC,
- * stride 1 or 2, io_dtype equal to the packed dtype, Cin a multiple of 8.  It multiplies blocks of 128 filters x 16
+/* The tensor path (RTOSS_PATH_TENSOR, or RTOSS_PATH_AUTO when it applies) takes: NHWC, stride 1 or 2, io_dtype equal
+ * to the packed dtype; bf16 / fp16 with Cin a multiple of 8, or fp32 with Cin a multiple of 4.  fp32 data is computed
+ * with tf32 instructions on values split into a 19-bit head and a remainder (three products per tap, fp32
+ * accumulation): results stay within the fp32 bound of 1e-4 of max(|y|, rms(y)) and cost six times the tensor time of
+ * 16-bit data.  It multiplies blocks of 128 filters x 16
  * channels per tap on the tensor cores and leaves out the blocks in which every weight is pruned (none with
  * per-kernel patterns on ordinary weights; 9 - k of every 9 with rtoss_select_patterns_shared); inside a block the
  * pruned taps are multiplied as zeros.  Results agree with the FMA path to fp32 summation order.

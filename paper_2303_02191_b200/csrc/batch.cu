@@ -132,7 +132,7 @@ __global__ void __launch_bounds__(kOrderWarps * 32) batch_order_kernel(const Bat
     for (unsigned task = blockIdx.x * kOrderWarps + warp; task < n_tasks; task += gridDim.x * kOrderWarps) {
         const BatchLayer& L = layers[task_layer[task]];
         rtoss_dev::order_channel(L.pid, L.Cout, L.Cin, L.P, (int)(task - L.task0), L.perm, L.bucket_off, fill_all[warp],
-                                 lane, L.masks, L.issue);
+                                 lane, L.masks, L.issue, L.v_dtype == RTOSS_F32 ? 5 : 6);
         __syncwarp();
     }
 }

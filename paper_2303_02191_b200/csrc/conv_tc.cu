@@ -52,6 +52,11 @@
 //     is not issued.  With per-kernel patterns on dense random weights every such block holds kept weights; when a
 //     block of kernels shares one pattern (rtoss_select_patterns_shared) only k of the 9 taps of a slab are issued:
 //     the contraction is then compacted to the non-zero work.
+//   * fp32 data runs on the same pipeline with kind::tf32 instructions and three products per tap in place of one:
+//     every value is split into a tf32 head (19 leading bits) and the remainder, x = xh + xl, w = wh + wl, and
+//     wh*xh + wh*xl + wl*xh is accumulated in fp32 (the dropped wl*xl is below 2^-21 of the product).  The weights are
+//     split when they are packed; an activation block is split in shared memory by the warp that fetched it (head in
+//     place, remainder into the second half of the stage) before the MMA thread may read it.
 //   * One launch may carry several independent convolutions ("problems": the pyramid levels of a detection tower,
 //     the two branches of a block): the tile list runs over all of them, every role looks its tile's problem up.
 //     Small problems then fill the tail of the large ones' waves instead of paying a launch each.
@@ -110,6 +115,9 @@ struct TcArgs {
     // Split K: a tile's channel blocks are shared out to the KS CTAs of a thread-block cluster, cb_per blocks each;
     // the partial sums are exchanged through distributed shared memory and every CTA finishes a part of the tile.
     int KS, cb_per;
+    int cb_ch, slab_ch;   // channels per staged block (128 bytes) and per instruction (32 bytes): 64 / 16 for 16-bit data, 32 / 8 for fp32
+    int taps_real;        // 9 or 1; `taps` counts weight tiles per channel block: twice that for fp32 (heads, then remainders)
+    int lo_off;           // fp32: byte offset of the remainders inside an activation stage
 };
 
 // A launch: up to NP convolutions sharing the CTA's rings (stage sizes are the largest any of them needs).  The struct
@@ -210,14 +218,23 @@ __device__ __forceinline__ unsigned long long make_sw128_desc(unsigned addr) {
     return d;
 }
 
+template <bool TF32>
 __device__ __forceinline__ void umma_f16(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc,
                                          unsigned idesc, unsigned accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
+    if (TF32)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+            : "memory");
 }
 // The MMAs of one tap of one channel block (filters on M) for the 16-channel slabs named by the mask m4 (bit s = slab
 // s), with a look at the "full" barriers of the NEXT activation and weight stage started in front of them
@@ -226,35 +243,47 @@ __device__ __forceinline__ void umma_f16(unsigned d_tmem, unsigned long long ade
 // nothing hides two of those per channel block; the stages ahead are normally full already, so the look usually
 // replaces both waits of the next block.  The first instruction issued takes `accumulate` as its accumulate flag,
 // the later ones add.  Returns bit 0: next activation stage full, bit 1: next weight stage full.
+#define RTOSS_DEFINE_PEEK(NAME, KIND)                                                                                   \
+    __device__ __forceinline__ unsigned NAME(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc,     \
+                                             unsigned idesc, unsigned accumulate, unsigned m4, unsigned barA,          \
+                                             unsigned parA, unsigned barB, unsigned parB) {                            \
+        unsigned res;                                                                                                  \
+        asm volatile(                                                                                                  \
+            "{\n\t.reg .pred pa, pb, q, p0, p1, p2, p3;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t.reg .b32 ta, tb, tm;\n\t"     \
+            "mbarrier.test_wait.parity.shared::cta.b64 pa, [%7], %8;\n\t"                                              \
+            "mbarrier.test_wait.parity.shared::cta.b64 pb, [%9], %10;\n\t"                                             \
+            "setp.ne.b32 q, %5, 0;\n\t"                                                                                \
+            "and.b32 tm, %6, 1;\n\tsetp.ne.b32 p0, tm, 0;\n\t"                                                        \
+            "and.b32 tm, %6, 2;\n\tsetp.ne.b32 p1, tm, 0;\n\t"                                                        \
+            "and.b32 tm, %6, 4;\n\tsetp.ne.b32 p2, tm, 0;\n\t"                                                        \
+            "and.b32 tm, %6, 8;\n\tsetp.ne.b32 p3, tm, 0;\n\t"                                                        \
+            "add.u64 a1, %2, 2;\n\tadd.u64 a2, %2, 4;\n\tadd.u64 a3, %2, 6;\n\t"                                      \
+            "add.u64 b1, %3, 2;\n\tadd.u64 b2, %3, 4;\n\tadd.u64 b3, %3, 6;\n\t"                                      \
+            "@p0 tcgen05.mma.cta_group::1.kind::" KIND " [%1], %2, %3, %4, q;\n\t"                                     \
+            "or.pred q, q, p0;\n\t"                                                                                    \
+            "@p1 tcgen05.mma.cta_group::1.kind::" KIND " [%1], a1, b1, %4, q;\n\t"                                     \
+            "or.pred q, q, p1;\n\t"                                                                                    \
+            "@p2 tcgen05.mma.cta_group::1.kind::" KIND " [%1], a2, b2, %4, q;\n\t"                                     \
+            "or.pred q, q, p2;\n\t"                                                                                    \
+            "@p3 tcgen05.mma.cta_group::1.kind::" KIND " [%1], a3, b3, %4, q;\n\t"                                     \
+            "selp.u32 ta, 1, 0, pa;\n\t"                                                                               \
+            "selp.u32 tb, 2, 0, pb;\n\t"                                                                               \
+            "or.b32 %0, ta, tb;\n\t}"                                                                                  \
+            : "=r"(res)                                                                                                \
+            : "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(m4), "r"(barA), "r"(parA), "r"(barB), \
+              "r"(parB)                                                                                                \
+            : "memory");                                                                                               \
+        return res;                                                                                                    \
+    }
+RTOSS_DEFINE_PEEK(umma_block_peek_f16, "f16")
+RTOSS_DEFINE_PEEK(umma_block_peek_tf32, "tf32")
+#undef RTOSS_DEFINE_PEEK
+template <bool TF32>
 __device__ __forceinline__ unsigned umma_block_peek(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc,
                                                     unsigned idesc, unsigned accumulate, unsigned m4, unsigned barA,
                                                     unsigned parA, unsigned barB, unsigned parB) {
-    unsigned res;
-    asm volatile(
-        "{\n\t.reg .pred pa, pb, q, p0, p1, p2, p3;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t.reg .b32 ta, tb, tm;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 pa, [%7], %8;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 pb, [%9], %10;\n\t"
-        "setp.ne.b32 q, %5, 0;\n\t"
-        "and.b32 tm, %6, 1;\n\tsetp.ne.b32 p0, tm, 0;\n\t"
-        "and.b32 tm, %6, 2;\n\tsetp.ne.b32 p1, tm, 0;\n\t"
-        "and.b32 tm, %6, 4;\n\tsetp.ne.b32 p2, tm, 0;\n\t"
-        "and.b32 tm, %6, 8;\n\tsetp.ne.b32 p3, tm, 0;\n\t"
-        "add.u64 a1, %2, 2;\n\tadd.u64 a2, %2, 4;\n\tadd.u64 a3, %2, 6;\n\t"
-        "add.u64 b1, %3, 2;\n\tadd.u64 b2, %3, 4;\n\tadd.u64 b3, %3, 6;\n\t"
-        "@p0 tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %3, %4, q;\n\t"
-        "or.pred q, q, p0;\n\t"
-        "@p1 tcgen05.mma.cta_group::1.kind::f16 [%1], a1, b1, %4, q;\n\t"
-        "or.pred q, q, p1;\n\t"
-        "@p2 tcgen05.mma.cta_group::1.kind::f16 [%1], a2, b2, %4, q;\n\t"
-        "or.pred q, q, p2;\n\t"
-        "@p3 tcgen05.mma.cta_group::1.kind::f16 [%1], a3, b3, %4, q;\n\t"
-        "selp.u32 ta, 1, 0, pa;\n\t"
-        "selp.u32 tb, 2, 0, pb;\n\t"
-        "or.b32 %0, ta, tb;\n\t}"
-        : "=r"(res)
-        : "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(m4), "r"(barA), "r"(parA), "r"(barB), "r"(parB)
-        : "memory");
-    return res;
+    return TF32 ? umma_block_peek_tf32(d_tmem, adesc, bdesc, idesc, accumulate, m4, barA, parA, barB, parB)
+                : umma_block_peek_f16(d_tmem, adesc, bdesc, idesc, accumulate, m4, barA, parA, barB, parB);
 }
 // Arrive on an mbarrier once all tcgen05.mma issued so far by this thread have completed.
 __device__ __forceinline__ void umma_commit(unsigned bar) {
@@ -342,6 +371,10 @@ __device__ __forceinline__ unsigned round_pack<__half, true>(float lo, float hi)
     asm("cvt.rn.relu.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
     return d;
 }
+
+// SiLU of an fp32 output: v / (1 + e^-v) with the fast exponential (a few ulp: the tanh form below is good to 2^-11
+// only, enough for 16-bit outputs, not for the 1e-4 bound of fp32 ones).
+__device__ __forceinline__ float silu_f32(float v) { return v / (1.f + __expf(-v)); }
 
 // Bias and activation of one accumulator value.  bs is the bias, for SiLU half the bias:
 //   v * sigmoid(v) = h + h * tanh(h) with h = v / 2 = fma(acc, 0.5, b / 2): two fused multiply-adds around one
@@ -575,28 +608,38 @@ __device__ __forceinline__ void epilogue_from_shares(unsigned buf, int KS, int r
         unsigned r[16];
 #pragma unroll
         for (int j = 0; j < kPatchRows; ++j) r[j] = __float_as_uint(sum[j]);
-        if (vec_ok) {
-            epilogue_half<T, ACT>(r, bs, wr, rd, tab_l + (unsigned)c0 * 8, ybv, ry, rx, rbv, post);
-        } else {
+        bool done = false;
+        if constexpr (sizeof(T) == 2) {
+            if (vec_ok) {
+                epilogue_half<T, ACT>(r, bs, wr, rd, tab_l + (unsigned)c0 * 8, ybv, ry, rx, rbv, post);
+                done = true;
+            }
+        }
+        if (!done) {
+            constexpr bool f32 = sizeof(T) == 4;   // (fp32: bs is the plain bias and SiLU the exponential form)
 #pragma unroll
             for (int j = 0; j < kPatchRows; ++j) {
                 const uint2 e = pos_tab[c0 + j];
                 if (co_ok && (e.y >> 16) < ry && (e.y & 0xFFFFu) < rx) {
                     float v;
                     if (rb && post) {   // activate, round, add the residual, round
-                        v = bias_act<ACT>(r[j], bs);
+                        v = f32 ? (ACT == RTOSS_ACT_SILU ? silu_f32(__uint_as_float(r[j]) + bs) : __uint_as_float(r[j]) + bs) : bias_act<ACT>(r[j], bs);
                         if (ACT == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
                         v = to_f32<T>(from_f32<T>(v)) + to_f32<T>(rb[e.x + lane]);
                     } else if (rb) {   // round, add the residual, activate, round
                         v = to_f32<T>(from_f32<T>(__uint_as_float(r[j]) + bs)) + to_f32<T>(rb[e.x + lane]);
                         if (ACT == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
                         if (ACT == RTOSS_ACT_SILU) {
-                            float th;
-                            asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(0.5f * v));
-                            v = fmaf(0.5f * v, th, 0.5f * v);
+                            if (f32) {
+                                v = silu_f32(v);
+                            } else {
+                                float th;
+                                asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(0.5f * v));
+                                v = fmaf(0.5f * v, th, 0.5f * v);
+                            }
                         }
                     } else {
-                        v = bias_act<ACT>(r[j], bs);
+                        v = f32 ? (ACT == RTOSS_ACT_SILU ? silu_f32(__uint_as_float(r[j]) + bs) : __uint_as_float(r[j]) + bs) : bias_act<ACT>(r[j], bs);
                         if (ACT == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
                     }
                     yb[e.x + lane] = from_f32<T>(v);
@@ -623,6 +666,7 @@ template <typename T, typename G>
 __global__ void __launch_bounds__(kTcThreads, 1)
 conv_tc_kernel(const __grid_constant__ G g) {
     constexpr bool kMulti = sizeof(G) > sizeof(TcLaunch1);
+    constexpr bool kF32 = sizeof(T) == 4;   // fp32 data: tf32 instructions, three products per tap (see the head of the file)
     extern __shared__ unsigned char smem_dyn[];
     // tiles need 1024-byte alignment for the 128-byte swizzle pattern
     const unsigned base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -632,7 +676,8 @@ conv_tc_kernel(const __grid_constant__ G g) {
     const unsigned bar_fullA = sBar, bar_emptyA = sBar + 8 * kMaxA;
     const unsigned bar_fullB = bar_emptyA + 8 * kMaxA, bar_emptyB = bar_fullB + 8 * kMaxB;
     const unsigned bar_accFull = bar_emptyB + 8 * kMaxB, bar_accEmpty = bar_accFull + 16;
-    const unsigned s_tmem_ptr = bar_accEmpty + 16;
+    const unsigned bar_loFull = bar_accEmpty + 16;   // fp32: activation stage split into heads and remainders
+    const unsigned s_tmem_ptr = bar_loFull + 8 * kMaxA;
     volatile unsigned* tmem_ptr_gen = reinterpret_cast<volatile unsigned*>(smem_dyn + (s_tmem_ptr - smem_u32(smem_dyn)));
     unsigned char* epi_patch = smem_dyn + (s_tmem_ptr + 16 - smem_u32(smem_dyn));  // [kEpiWarps][kPatchBytes], 16-byte aligned
     uint2* pos_tab_all = reinterpret_cast<uint2*>(epi_patch + kEpiWarps * kPatchBytes);  // [n_prob][kMaxPx]
@@ -649,6 +694,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
         for (int i = 0; i < g.NA; ++i) {
             mbar_init(bar_fullA + 8 * i, 1);
             mbar_init(bar_emptyA + 8 * i, 1);
+            mbar_init(bar_loFull + 8 * i, 1);
         }
         for (int i = 0; i < g.NB; ++i) {
             mbar_init(bar_fullB + 8 * i, 1);
@@ -696,7 +742,8 @@ conv_tc_kernel(const __grid_constant__ G g) {
         // ---------------- TMA producer of the activations.  Issuing a bulk copy keeps its thread busy for some
         // hundred cycles whatever the size, so the activations and the weights have a producer thread each, and a
         // weight stage (G taps) is ONE copy.
-        if (lane == 0) {
+        if (kF32 || lane == 0) {
+            // (fp32: all 32 lanes walk the loop; lane 0 issues the copies, then the warp splits the block that arrived)
             bool ok = true;
             int sa = 0;
             unsigned pa = 0;
@@ -712,19 +759,53 @@ conv_tc_kernel(const __grid_constant__ G g) {
                 const int y0 = ty * a.TH, x0 = tx * a.TW;
                 const int cb_end = min(a.ncb, (ks + 1) * a.cb_per);
                 for (int cb = ks * a.cb_per; cb < cb_end; ++cb) {
-                    ok = mbar_wait(bar_emptyA + 8 * sa, pa ^ 1, g.wait_cycles);
+                    if (lane == 0) {
+                        ok = mbar_wait(bar_emptyA + 8 * sa, pa ^ 1, g.wait_cycles);
+                        if (ok) {
+                            mbar_expect_tx(bar_fullA + 8 * sa, a.a_tx_bytes * a.n_sub);
+                            for (int sub = 0; sub < a.n_sub; ++sub)
+                                tma_load_4d(sA + sa * g.a_stage_bytes + sub * a.sub_bytes, &g.tmA[pi], cb * a.cb_ch, x0 * a.S + a.x_add[sub],
+                                            y0 * a.S + a.y_add[sub], n, bar_fullA + 8 * sa);
+                        }
+                    }
+                    if (kF32) {
+                        // Split the block: x = head + remainder, head = the 19 leading bits (what a tf32 operand holds), in
+                        // place; the remainder (exact in fp32) goes to the second half of the stage.  Plain loads and stores
+                        // of this warp; the fence hands them to the proxy the tensor core reads through; then the stage is
+                        // announced to the MMA thread.  Any word may be split: rows the copy did not write are never outputs.
+                        ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+                        if (ok) {
+                            if (lane == 0) ok = mbar_wait(bar_fullA + 8 * sa, pa, g.wait_cycles);
+                            ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+                        }
+                        if (ok) {
+                            const unsigned src = sA + sa * g.a_stage_bytes, dst = src + (unsigned)a.lo_off;
+                            const int n16 = (a.n_sub * a.sub_bytes) >> 4;
+#pragma unroll 4
+                            for (int i = lane; i < n16; i += 32) {
+                                unsigned v[4], h[4], l[4];
+                                asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(src + 16u * i));
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    h[e] = v[e] & 0xFFFFE000u;
+                                    l[e] = __float_as_uint(__fsub_rn(__uint_as_float(v[e]), __uint_as_float(h[e])));
+                                }
+                                asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(src + 16u * i), "r"(h[0]), "r"(h[1]), "r"(h[2]), "r"(h[3]) : "memory");
+                                asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + 16u * i), "r"(l[0]), "r"(l[1]), "r"(l[2]), "r"(l[3]) : "memory");
+                            }
+                            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                            __syncwarp();
+                            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_loFull + 8 * sa) : "memory");
+                        }
+                    }
                     if (!ok) break;
-                    mbar_expect_tx(bar_fullA + 8 * sa, a.a_tx_bytes * a.n_sub);
-                    for (int sub = 0; sub < a.n_sub; ++sub)
-                        tma_load_4d(sA + sa * g.a_stage_bytes + sub * a.sub_bytes, &g.tmA[pi], cb * kKBlock, x0 * a.S + a.x_add[sub],
-                                    y0 * a.S + a.y_add[sub], n, bar_fullA + 8 * sa);
                     if (++sa == g.NA) {
                         sa = 0;
                         pa ^= 1;
                     }
                 }
             }
-            if (!ok) atomicExch(g.status, 1);
+            if (!ok && lane == 0) atomicExch(g.status, 1);
         }
         __syncwarp();  // lanes 1..31 wait here for lane 0: the warp reaches the final barrier as one
     } else if (warp == kWeightWarp) {
@@ -747,7 +828,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
                         // (failure-detection hook: the launch's very first weight copy is withheld, so the wait for it runs out)
                         if (!(g.inject == 1 && unit == (int)blockIdx.x && cb == ks * a.cb_per && t0 == 0)) {
                             mbar_expect_tx(bar_fullB + 8 * sb, a.b_tx_bytes * a.G);
-                            tma_load_3d(sB + sb * g.b_stage_bytes, &g.tmB[pi], cb * kKBlock, co0, t0, bar_fullB + 8 * sb);
+                            tma_load_3d(sB + sb * g.b_stage_bytes, &g.tmB[pi], cb * a.cb_ch, co0, t0, bar_fullB + 8 * sb);
                         }
                         if (++sb == g.NB) {
                             sb = 0;
@@ -777,6 +858,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
             unsigned tap16[9], wtile16 = 0, idesc = 0, hi_cols = 0;
             bool pxm = false, two = false, unrolled9 = false;
             int cur_pi = -1;
+            const unsigned bar_rdyA = kF32 ? bar_loFull : bar_fullA;   // the barrier that says an activation stage may be read
             int sa = 0, sb = 0, as = 0, n_done = 0;
             unsigned pa = 0, pb = 0, pacc = 0;  // phase parities of the three rings
             unsigned peek = 0;                  // what umma_block_peek saw of the stages now current
@@ -787,8 +869,8 @@ conv_tc_kernel(const __grid_constant__ G g) {
 #pragma unroll
                     for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
                         if (m4 & (1u << k4)) {
-                            umma_f16(d_base, mk(xl + 2 * k4), mk(wl + 2 * k4), idesc, acc);
-                            if (two) umma_f16(d_base + hi_cols, mk(xl + 1024 + 2 * k4), mk(wl + 2 * k4), idesc, acc);
+                            umma_f16<kF32>(d_base, mk(xl + 2 * k4), mk(wl + 2 * k4), idesc, acc);
+                            if (two) umma_f16<kF32>(d_base + hi_cols, mk(xl + 1024 + 2 * k4), mk(wl + 2 * k4), idesc, acc);
                             acc = 1;
                         }
                     }
@@ -796,7 +878,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
 #pragma unroll
                     for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
                         if (m4 & (1u << k4)) {
-                            umma_f16(d_base, mk(wl + 2 * k4), mk(xl + 2 * k4), idesc, acc);
+                            umma_f16<kF32>(d_base, mk(wl + 2 * k4), mk(xl + 2 * k4), idesc, acc);
                             acc = 1;
                         }
                     }
@@ -815,7 +897,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
                     hi_cols = (unsigned)a.n_cols;
                     pxm = a.pxm != 0;
                     two = a.MH == 2;
-                    unrolled9 = a.taps == 9 && a.G == 3;
+                    unrolled9 = !kF32 && a.taps == 9 && a.G == 3;
                 }
                 const int ks = local % a.KS, cb_end = min(a.ncb, (ks + 1) * a.cb_per);
                 // which (tap, slab) pairs of this filter tile hold kept weights: one word per channel block, the next
@@ -827,13 +909,13 @@ conv_tc_kernel(const __grid_constant__ G g) {
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const unsigned d_base = tmem_base + (unsigned)(as * g.acc_stride);
                 unsigned acc = 0;  // the first instruction of a tile overwrites the accumulator
-                int left = a.Cin - ks * a.cb_per * kKBlock;
-                for (int cb = ks * a.cb_per; cb < cb_end && ok; ++cb, left -= kKBlock) {
-                    // 16-channel slabs of this block that hold channels (the rest of the 64 is TMA zero fill)
-                    const int nk4 = left >= kKBlock ? kKBlock / 16 : (left + 15) >> 4;
+                int left = a.Cin - ks * a.cb_per * a.cb_ch;
+                for (int cb = ks * a.cb_per; cb < cb_end && ok; ++cb, left -= a.cb_ch) {
+                    // 32-byte slabs of this block that hold channels (the rest of the 128 bytes is TMA zero fill)
+                    const int nk4 = left >= a.cb_ch ? 4 : (left + a.slab_ch - 1) / a.slab_ch;
                     const unsigned nkmask = (1u << nk4) - 1u;
                     if (a.taps == 1) {
-                        if (!(peek & 1u)) ok = mbar_wait(bar_fullA + 8 * sa, pa, g.wait_cycles);
+                        if (!(peek & 1u)) ok = mbar_wait(bar_rdyA + 8 * sa, pa, g.wait_cycles);
                         if (ok && !(peek & 2u)) ok = mbar_wait(bar_fullB + 8 * sb, pb, g.wait_cycles);
                         if (!ok) break;
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -842,18 +924,18 @@ conv_tc_kernel(const __grid_constant__ G g) {
                         const unsigned wl0 = desc_lo0 + (sB >> 4) + (unsigned)sb * bstage16;
                         const unsigned xl0 = desc_lo0 + (sA >> 4) + (unsigned)sa * astage16;
                         if (!pxm) {
-                            peek = umma_block_peek(d_base, mk(wl0), mk(xl0), idesc, acc, nkmask, bar_fullA + 8 * sa_n, pa_n,
+                            peek = umma_block_peek<kF32>(d_base, mk(wl0), mk(xl0), idesc, acc, nkmask, bar_rdyA + 8 * sa_n, pa_n,
                                                    bar_fullB + 8 * sb_n, pb_n);
                         } else {
                             // positions on M: the first 128 positions with the look ahead, then the second 128
-                            peek = umma_block_peek(d_base, mk(xl0), mk(wl0), idesc, acc, nkmask, bar_fullA + 8 * sa_n, pa_n,
+                            peek = umma_block_peek<kF32>(d_base, mk(xl0), mk(wl0), idesc, acc, nkmask, bar_rdyA + 8 * sa_n, pa_n,
                                                    bar_fullB + 8 * sb_n, pb_n);
                             if (two) {
                                 unsigned acc2 = acc;
 #pragma unroll
                                 for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
                                     if (k4 < nk4) {
-                                        umma_f16(d_base + hi_cols, mk(xl0 + 1024 + 2 * k4), mk(wl0 + 2 * k4), idesc, acc2);
+                                        umma_f16<kF32>(d_base + hi_cols, mk(xl0 + 1024 + 2 * k4), mk(wl0 + 2 * k4), idesc, acc2);
                                         acc2 = 1;
                                     }
                                 }
@@ -866,7 +948,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
                         continue;
                     }
                     const unsigned long long bits_n = (iss && cb + 1 < cb_end) ? __ldg(iss + cb + 1) : ~0ull;
-                    if (!(peek & 1u)) ok = mbar_wait(bar_fullA + 8 * sa, pa, g.wait_cycles);   // (peek stays 0 on the paths that do not look ahead)
+                    if (!(peek & 1u)) ok = mbar_wait(bar_rdyA + 8 * sa, pa, g.wait_cycles);   // (peek stays 0 on the paths that do not look ahead)
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const unsigned xl0 = desc_lo0 + (sA >> 4) + (unsigned)sa * astage16;
@@ -883,8 +965,8 @@ conv_tc_kernel(const __grid_constant__ G g) {
                                 if (!pxm) {
                                     // the first tap of the stage goes out together with a look at the next stages
                                     const int sb_n = sb + 1 == g.NB ? 0 : sb + 1;
-                                    peek = umma_block_peek(d_base, mk(wl0), mk(xl0 + tap16[s3 * 3]), idesc, acc, m_first,
-                                                           bar_fullA + 8 * sa_n, pa_n, bar_fullB + 8 * sb_n, sb_n ? pb : pb ^ 1);
+                                    peek = umma_block_peek<kF32>(d_base, mk(wl0), mk(xl0 + tap16[s3 * 3]), idesc, acc, m_first,
+                                                           bar_rdyA + 8 * sa_n, pa_n, bar_fullB + 8 * sb_n, sb_n ? pb : pb ^ 1);
                                     if (m_first) acc = 1;
 #pragma unroll
                                     for (int i = 1; i < 3; ++i)
@@ -910,9 +992,14 @@ conv_tc_kernel(const __grid_constant__ G g) {
                             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                             const unsigned wl0 = desc_lo0 + (sB >> 4) + (unsigned)sb * bstage16;
                             for (int i = 0; i < a.G; ++i) {
-                                const unsigned off =
-                                    (unsigned)(a.tap_sub[t0 + i] * a.sub_bytes + a.tap_shift[t0 + i] * kRowBytes) >> 4;
-                                issue_tap(d_base, wl0 + i * wtile16, xl0 + off, (unsigned)(bits >> (4 * (t0 + i))) & nkmask, acc);
+                                // weight tile v of the block: tap v (16-bit data); fp32: the heads of tap v, then (v >= 9
+                                // resp. 1) the remainders of tap v - 9.  Heads meet the activations' heads and remainders,
+                                // remainders the heads only.
+                                const int v = t0 + i, t = v >= a.taps_real ? v - a.taps_real : v;
+                                const unsigned off = (unsigned)(a.tap_sub[t] * a.sub_bytes + a.tap_shift[t] * kRowBytes) >> 4;
+                                const unsigned m4 = (unsigned)(bits >> (4 * t)) & nkmask;
+                                issue_tap(d_base, wl0 + i * wtile16, xl0 + off, m4, acc);
+                                if (kF32 && v < a.taps_real) issue_tap(d_base, wl0 + i * wtile16, xl0 + off + ((unsigned)a.lo_off >> 4), m4, acc);
                             }
                             umma_commit(bar_emptyB + 8 * sb);
                             if (++sb == g.NB) {
@@ -952,8 +1039,8 @@ conv_tc_kernel(const __grid_constant__ G g) {
         const int sub = (warp - 2) >> 2;   // four warps share a lane quarter and take every fourth 32-column chunk
         bool ok = true;
         int gt = 0;
-        if (g.prob[0].pxm) {
-            // (a launch with the positions as M carries one problem)
+        if constexpr (!kF32) if (g.prob[0].pxm) {
+            // (a launch with the positions as M carries one problem; 16-bit data only)
             const TcArgs& a = g.prob[0];
             T* __restrict__ yg = reinterpret_cast<T*>(a.y);
             const uint2* pos_tab = pos_tab_all;
@@ -1008,8 +1095,9 @@ conv_tc_kernel(const __grid_constant__ G g) {
                 __syncwarp();
                 if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_accEmpty + 8 * as) : "memory");
             }
-        } else
-        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++gt) {
+            gt = -1;   // (done: the loop below does not run)
+        }
+        for (int tile = blockIdx.x; gt >= 0 && tile < n_tiles && ok; tile += gridDim.x, ++gt) {
             int local;
             const int pi = find_problem<kMulti>(g, tile, local);
             const TcArgs& a = g.prob[pi];
@@ -1033,13 +1121,14 @@ conv_tc_kernel(const __grid_constant__ G g) {
             const bool co_ok = co < a.Cout;
             const float bv = (a.bias && co_ok) ? __ldg(a.bias + co) : 0.f;
             const unsigned patch = s_tmem_ptr + 16 + (unsigned)(warp - 2) * kPatchBytes;  // shared address
-            const bool vec_ok = (a.y_c_stride % 8 == 0) && ((a.y_c_off + co0) % 8 == 0) && (co0 + row0 + 32 <= a.Cout);
+            // (fp32 outputs leave through the element stores below: a warp's 32 filters of one position are 128 contiguous bytes)
+            const bool vec_ok = !kF32 && (a.y_c_stride % 8 == 0) && ((a.y_c_off + co0) % 8 == 0) && (co0 + row0 + 32 <= a.Cout);
             T* yb = yg + (((size_t)n * a.Ho + y0) * a.Wo + x0) * a.y_c_stride + a.y_c_off + co0 + row0;
             const unsigned ry = (unsigned)min(a.TH, a.Ho - y0), rx = (unsigned)min(a.TW, a.Wo - x0);  // rows / columns inside the image
             const int c_first = (sub + 4 * copy) * 32, c_step = 128 * a.R;
             const T* rb = a.resid ? reinterpret_cast<const T*>(a.resid) + (yb - yg) : nullptr;   // laid out like y
             const bool post = a.resid_post != 0;
-            const float bs = (a.act == RTOSS_ACT_SILU && (!rb || post)) ? 0.5f * bv : bv;   // (a residual in front of the activation: plain bias)
+            const float bs = (!kF32 && a.act == RTOSS_ACT_SILU && (!rb || post)) ? 0.5f * bv : bv;   // (a residual in front of the activation, or fp32 data: plain bias)
             ok = mbar_wait(bar_accFull + 8 * as, (gt / g.AS) & 1, g.wait_cycles);
             if (!ok && a.KS == 1) break;   // (split K: the cluster barriers below must still be passed)
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -1077,29 +1166,34 @@ conv_tc_kernel(const __grid_constant__ G g) {
                 }
                 continue;
             }
-            if (vec_ok) {
-                if (rb) {
-                    const unsigned stage = s_res + (unsigned)(warp - 2) * kResStage;
+            bool stored = false;
+            if constexpr (!kF32) {
+                if (vec_ok) {
+                    stored = true;
+                    if (rb) {
+                        const unsigned stage = s_res + (unsigned)(warp - 2) * kResStage;
 #define RTOSS_RES_CALL(ACT_, POST_) \
-    epilogue_chunks_res<T, ACT_, POST_>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb, stage)
-                    if (post) {
-                        if (a.act == RTOSS_ACT_SILU) RTOSS_RES_CALL(RTOSS_ACT_SILU, true);
-                        else if (a.act == RTOSS_ACT_RELU) RTOSS_RES_CALL(RTOSS_ACT_RELU, true);
-                        else RTOSS_RES_CALL(RTOSS_ACT_NONE, false);   // no activation: both orders are the same sum
-                    } else {
-                        if (a.act == RTOSS_ACT_SILU) RTOSS_RES_CALL(RTOSS_ACT_SILU, false);
-                        else if (a.act == RTOSS_ACT_RELU) RTOSS_RES_CALL(RTOSS_ACT_RELU, false);
-                        else RTOSS_RES_CALL(RTOSS_ACT_NONE, false);
-                    }
+        epilogue_chunks_res<T, ACT_, POST_>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb, stage)
+                        if (post) {
+                            if (a.act == RTOSS_ACT_SILU) RTOSS_RES_CALL(RTOSS_ACT_SILU, true);
+                            else if (a.act == RTOSS_ACT_RELU) RTOSS_RES_CALL(RTOSS_ACT_RELU, true);
+                            else RTOSS_RES_CALL(RTOSS_ACT_NONE, false);   // no activation: both orders are the same sum
+                        } else {
+                            if (a.act == RTOSS_ACT_SILU) RTOSS_RES_CALL(RTOSS_ACT_SILU, false);
+                            else if (a.act == RTOSS_ACT_RELU) RTOSS_RES_CALL(RTOSS_ACT_RELU, false);
+                            else RTOSS_RES_CALL(RTOSS_ACT_NONE, false);
+                        }
 #undef RTOSS_RES_CALL
-                } else if (a.act == RTOSS_ACT_SILU)
-                    epilogue_chunks<T, RTOSS_ACT_SILU>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb);
-                else if (a.act == RTOSS_ACT_RELU)
-                    epilogue_chunks<T, RTOSS_ACT_RELU>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb);
-                else
-                    epilogue_chunks<T, RTOSS_ACT_NONE>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb);
-            } else {
-                // ragged filter counts or unaligned channel slices: element stores, lane = filter
+                    } else if (a.act == RTOSS_ACT_SILU)
+                        epilogue_chunks<T, RTOSS_ACT_SILU>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb);
+                    else if (a.act == RTOSS_ACT_RELU)
+                        epilogue_chunks<T, RTOSS_ACT_RELU>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb);
+                    else
+                        epilogue_chunks<T, RTOSS_ACT_NONE>(d_base, c_first, c_step, a.N_px, bs, patch, s_tab, yb, ry, rx, lane, rb);
+                }
+            }
+            if (!stored) {
+                // ragged filter counts, unaligned channel slices, fp32 data: element stores, lane = filter
                 for (int c0 = c_first; c0 < a.N_px; c0 += c_step) {
                     unsigned r[32];
                     tmem_ld32(d_base + (unsigned)c0, r);
@@ -1112,9 +1206,13 @@ conv_tc_kernel(const __grid_constant__ G g) {
                         if (rb && in_img && !post) v = to_f32<T>(from_f32<T>(v)) + to_f32<T>(rb[e.x + lane]);   // round, then add the residual
                         if (a.act == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
                         if (a.act == RTOSS_ACT_SILU) {
-                            float th;
-                            asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(0.5f * v));
-                            v = v * fmaf(0.5f, th, 0.5f);
+                            if (kF32) {
+                                v = silu_f32(v);
+                            } else {
+                                float th;
+                                asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(0.5f * v));
+                                v = v * fmaf(0.5f, th, 0.5f);
+                            }
                         }
                         if (rb && in_img && post) v = to_f32<T>(from_f32<T>(v)) + to_f32<T>(rb[e.x + lane]);   // behind the activation
                         if (co_ok && (e.y >> 16) < ry && (e.y & 0xFFFFu) < rx) yb[e.x + lane] = from_f32<T>(v);
@@ -1162,7 +1260,7 @@ inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 // A narrow layer wastes most of M that way and, worse, leaves three of four epilogue warps without TMEM lanes to
 // read; with the positions as M every lane carries an output and a thread's filters are contiguous in NHWC.  The
 // price is one instruction per 128 positions instead of per 256: taken where few instructions are needed anyway.
-bool use_pxm(const rtoss_packed* p) { return p->Cout <= kPxmMaxCout && p->ksize == 1; }
+bool use_pxm(const rtoss_packed* p) { return p->Cout <= kPxmMaxCout && p->ksize == 1 && p->dtype != RTOSS_F32; }
 
 struct TcPlan {
     int TH, TW, Wq, N_px, NA, NB, G, n_sub, sub_rows, rows_staged, tiles_x, smem;
@@ -1179,7 +1277,7 @@ struct TcPlan {
 // The plan picks TH, the column segment TW (images wider than a TMA box are cut into segments), the
 // ring depths, and how many taps share a weight stage.
 bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count, bool pxm, int w_rows, bool resid, TcPlan* out,
-             int n_prob = 1) {
+             int n_prob = 1, bool f32 = false) {
     const int halo = ksize == 3 ? (S == 1 ? 2 : 1) : 0;
     const int n_sub = (ksize == 3 && S == 2) ? 4 : 1;
     const int max_pitch = S == 1 ? 256 : 128;  // TMA box: at most 256 elements traversed per dimension
@@ -1202,7 +1300,7 @@ bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count
             const int halves = n_px > 128 ? 2 : 1;
             if (pxm && max_shift + 128 * halves > need_rows) need_rows = max_shift + 128 * halves;
             const int sub_rows = round_up(need_rows, 8);
-            const int a_bytes = n_sub * sub_rows * kRowBytes;
+            const int a_bytes = n_sub * sub_rows * kRowBytes * (f32 ? 2 : 1);   // (fp32: heads and remainders)
             for (int G = (ksize == 3 ? 3 : 1); G >= 1; G -= 2) {
                 const int b_bytes = G * w_rows * kRowBytes;
                 int na = (cap - fixed - 2 * b_bytes) / a_bytes;
@@ -1261,7 +1359,9 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
     // narrow layers put the positions on the M operand (all 128 TMEM lanes carry outputs whatever Cout is)
     const bool pxm = use_pxm(p);
     const int w_rows = pxm ? round_up(p->Cout, 16) : kMTile;
-    if (!plan_tc(d->N, Ho, Wo, p->ksize, S, (p->Cout + kMTile - 1) / kMTile, sms, pxm, w_rows, d->residual_dev != nullptr, &plan, n_prob))
+    const bool f32 = p->dtype == RTOSS_F32;
+    const int esize = f32 ? 4 : 2;
+    if (!plan_tc(d->N, Ho, Wo, p->ksize, S, (p->Cout + kMTile - 1) / kMTile, sms, pxm, w_rows, d->residual_dev != nullptr, &plan, n_prob, f32))
         return (int)cudaErrorInvalidConfiguration;
 
     TcArgs& a = *out;
@@ -1280,7 +1380,10 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
     a.Wq = plan.Wq;
     a.TH = plan.TH;
     a.TW = plan.TW;
-    a.taps = taps;
+    a.taps = taps * (f32 ? 2 : 1);   // weight tiles per channel block: fp32 has the heads, then the remainders
+    a.taps_real = taps;
+    a.cb_ch = kRowBytes / esize;
+    a.slab_ch = 32 / esize;
     a.tiles_x = plan.tiles_x;
     a.n_sub = plan.n_sub;
     a.sub_bytes = plan.sub_rows * kRowBytes;
@@ -1300,10 +1403,11 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
         }
     }
     a.N_px = plan.N_px;
-    a.ncb = (p->Cin + kKBlock - 1) / kKBlock;
+    a.ncb = (p->Cin + a.cb_ch - 1) / a.cb_ch;
     a.tiles_y = (Ho + plan.TH - 1) / plan.TH;
     a.co_tiles = (p->Cout + N_T - 1) / N_T;
-    pp->a_stage_bytes = plan.n_sub * plan.sub_rows * kRowBytes;
+    a.lo_off = f32 ? plan.n_sub * plan.sub_rows * kRowBytes : 0;
+    pp->a_stage_bytes = plan.n_sub * plan.sub_rows * kRowBytes * (f32 ? 2 : 1);
     a.w_rows = w_rows;
     // narrow 3x3 layers keep the filters on M and repeat them down the 128 rows of the tile
     const rtoss_wtc_layout lay = rtoss_wtc_layout_of(p->Cout, p->ksize);  // how rtoss_pack laid the weights out
@@ -1318,8 +1422,9 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
     a.y_c_off = d->y_channel_offset;
     a.y_c_stride = d->y_channel_stride ? d->y_channel_stride : p->Cout;
     a.is_bf16 = p->dtype == RTOSS_BF16;
-    // instruction descriptor: fp32 accumulate, A and B of the io type, both K-major, N/8 and M/16
-    const unsigned fmt = a.is_bf16 ? 1u : 0u;
+    // instruction descriptor: fp32 accumulate, A and B of the io type (f16 0, bf16 1; kind::tf32: tf32 2), both K-major,
+    // N/8 and M/16
+    const unsigned fmt = f32 ? 2u : a.is_bf16 ? 1u : 0u;
     a.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((unsigned)(plan.N_px >> 3) << 17) | ((unsigned)(kMTile >> 4) << 24);
     a.pxm = pxm ? 1 : 0;
     a.MH = plan.N_px > 128 ? 2 : 1;
@@ -1333,7 +1438,7 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
 
     PFN_cuTensorMapEncodeTiled_v12000 enc = encode_fn();
     if (!enc) return (int)cudaErrorNotSupported;
-    const CUtensorMapDataType dt = a.is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+    const CUtensorMapDataType dt = f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : a.is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
     // activations: descriptor cached per (pointer, shape, box)
     const int key[6] = {d->N, d->H, d->W, p->Cin, plan.rows_staged * 8 + S, plan.Wq * 4 + (int)p->dtype};
     rtoss_tmap_entry* ea = nullptr;
@@ -1343,9 +1448,9 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
         ea = &ctx->tmap_cache[ctx->tmap_next];
         ctx->tmap_next = (ctx->tmap_next + 1) % 32;
         cuuint64_t dims[4] = {(cuuint64_t)p->Cin, (cuuint64_t)d->W, (cuuint64_t)d->H, (cuuint64_t)d->N};
-        cuuint64_t strides[3] = {(cuuint64_t)p->Cin * 2, (cuuint64_t)d->W * p->Cin * 2, (cuuint64_t)d->H * d->W * p->Cin * 2};
+        cuuint64_t strides[3] = {(cuuint64_t)p->Cin * esize, (cuuint64_t)d->W * p->Cin * esize, (cuuint64_t)d->H * d->W * p->Cin * esize};
         // with element strides the box is counted in traversed elements: S*n covers n fetched pixels
-        cuuint32_t box[4] = {(cuuint32_t)kKBlock, (cuuint32_t)(plan.Wq * S), (cuuint32_t)(plan.rows_staged * S), 1};
+        cuuint32_t box[4] = {(cuuint32_t)a.cb_ch, (cuuint32_t)(plan.Wq * S), (cuuint32_t)(plan.rows_staged * S), 1};
         cuuint32_t es[4] = {1, (cuuint32_t)S, (cuuint32_t)S, 1};
         ea->valid = 0;
         CUresult r = enc(reinterpret_cast<CUtensorMap*>(ea->map), dt, 4, const_cast<void*>(x), dims, strides, box, es,
@@ -1359,9 +1464,9 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
     // weights: one descriptor per handle
     rtoss_tmap_entry* eb = &p->wtc_map;
     if (!eb->valid || eb->base != p->wtc || eb->dims[0] != w_rows || eb->dims[1] != plan.G) {
-        cuuint64_t dims[3] = {(cuuint64_t)p->Cin, (cuuint64_t)lay.rows, (cuuint64_t)taps};
-        cuuint64_t strides[2] = {(cuuint64_t)p->Cin * 2, (cuuint64_t)lay.rows * p->Cin * 2};
-        cuuint32_t box[3] = {(cuuint32_t)kKBlock, (cuuint32_t)w_rows, (cuuint32_t)plan.G};  // a weight stage is one copy
+        cuuint64_t dims[3] = {(cuuint64_t)p->Cin, (cuuint64_t)lay.rows, (cuuint64_t)a.taps};
+        cuuint64_t strides[2] = {(cuuint64_t)p->Cin * esize, (cuuint64_t)lay.rows * p->Cin * esize};
+        cuuint32_t box[3] = {(cuuint32_t)a.cb_ch, (cuuint32_t)w_rows, (cuuint32_t)plan.G};  // a weight stage is one copy
         cuuint32_t es[3] = {1, 1, 1};
         eb->valid = 0;
         CUresult r = enc(reinterpret_cast<CUtensorMap*>(eb->map), dt, 3, p->wtc, dims, strides, box, es,
@@ -1391,6 +1496,10 @@ int ensure_smem_attr(const rtoss_ctx* ctx) {
             e = cudaFuncSetAttribute(conv_tc_kernel<__nv_bfloat16, TcLaunchN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(conv_tc_kernel<__half, TcLaunchN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(conv_tc_kernel<float, TcLaunch1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(conv_tc_kernel<float, TcLaunchN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return (int)e;
         if (dev_slot >= 0) attr_set[dev_slot].store(true, std::memory_order_release);
     }
@@ -1411,7 +1520,7 @@ void launch_common(const rtoss_ctx* ctx, G* g) {
 }  // namespace
 
 bool rtoss_tc_weights_eligible(const rtoss_packed* p) {
-    return (p->dtype == RTOSS_BF16 || p->dtype == RTOSS_F16) && p->Cin % 8 == 0;  // 16-byte rows for TMA
+    return ((p->dtype == RTOSS_BF16 || p->dtype == RTOSS_F16) && p->Cin % 8 == 0) || (p->dtype == RTOSS_F32 && p->Cin % 4 == 0);  // 16-byte rows for TMA
 }
 
 // Can this call run on the tensor path?
@@ -1426,7 +1535,7 @@ bool rtoss_tc_eligible(const rtoss_packed* p, const rtoss_conv_desc* d, const vo
     TcPlan plan;
     const bool pxm = use_pxm(p);
     return plan_tc(d->N, Ho, Wo, p->ksize, d->stride, (p->Cout + kMTile - 1) / kMTile, 148, pxm, pxm ? round_up(p->Cout, 16) : kMTile,
-                   d->residual_dev != nullptr, &plan);
+                   d->residual_dev != nullptr, &plan, 1, p->dtype == RTOSS_F32);
 }
 
 // May this call be one of several in a launch?  (Tensor path with the filters on M.)
@@ -1444,6 +1553,7 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     if (e) return e;
     TcArgs& a = g.prob[0];
     const TcPlan& plan = pp.plan;
+    const bool f32 = p->dtype == RTOSS_F32;
     g.a_stage_bytes = pp.a_stage_bytes;
     g.b_stage_bytes = pp.b_stage_bytes;
     g.NA = plan.NA;
@@ -1494,8 +1604,9 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     cudaError_t le;
     if (a.KS > 1) {
         // one cluster per tile; if the device cannot place the clusters the layer runs uncut
-        le = a.is_bf16 ? rtoss_dev::launch_pdl(conv_tc_kernel<__nv_bfloat16, TcLaunch1>, grid, kTcThreads, smem, (cudaStream_t)stream, a.KS, g)
-                       : rtoss_dev::launch_pdl(conv_tc_kernel<__half, TcLaunch1>, grid, kTcThreads, smem, (cudaStream_t)stream, a.KS, g);
+        le = f32 ? rtoss_dev::launch_pdl(conv_tc_kernel<float, TcLaunch1>, grid, kTcThreads, smem, (cudaStream_t)stream, a.KS, g)
+             : a.is_bf16 ? rtoss_dev::launch_pdl(conv_tc_kernel<__nv_bfloat16, TcLaunch1>, grid, kTcThreads, smem, (cudaStream_t)stream, a.KS, g)
+                         : rtoss_dev::launch_pdl(conv_tc_kernel<__half, TcLaunch1>, grid, kTcThreads, smem, (cudaStream_t)stream, a.KS, g);
         if (le == cudaSuccess) return 0;
         cudaGetLastError();
         a.KS = 1;
@@ -1504,8 +1615,9 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
         g.unit_end[0] = (int)n_units;
         grid = dim3((unsigned)(n_units < (size_t)sms ? n_units : (size_t)sms));
     }
-    le = a.is_bf16 ? rtoss_dev::launch_pdl(conv_tc_kernel<__nv_bfloat16, TcLaunch1>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g)
-                   : rtoss_dev::launch_pdl(conv_tc_kernel<__half, TcLaunch1>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g);
+    le = f32 ? rtoss_dev::launch_pdl(conv_tc_kernel<float, TcLaunch1>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g)
+         : a.is_bf16 ? rtoss_dev::launch_pdl(conv_tc_kernel<__nv_bfloat16, TcLaunch1>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g)
+                     : rtoss_dev::launch_pdl(conv_tc_kernel<__half, TcLaunch1>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g);
     return (int)le;
 }
 
@@ -1583,8 +1695,9 @@ int rtoss_launch_conv_tc_group(const rtoss_ctx* ctx, int n, const rtoss_packed* 
     dim3 grid((unsigned)(units < sms ? units : sms));
     int e = ensure_smem_attr(ctx);
     if (e) return e;
-    const bool bf = ps[0]->dtype == RTOSS_BF16;
-    cudaError_t le = bf ? rtoss_dev::launch_pdl(conv_tc_kernel<__nv_bfloat16, TcLaunchN>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g)
-                        : rtoss_dev::launch_pdl(conv_tc_kernel<__half, TcLaunchN>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g);
+    const bool bf = ps[0]->dtype == RTOSS_BF16, f32 = ps[0]->dtype == RTOSS_F32;
+    cudaError_t le = f32 ? rtoss_dev::launch_pdl(conv_tc_kernel<float, TcLaunchN>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g)
+                     : bf ? rtoss_dev::launch_pdl(conv_tc_kernel<__nv_bfloat16, TcLaunchN>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g)
+                          : rtoss_dev::launch_pdl(conv_tc_kernel<__half, TcLaunchN>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g);
     return (int)le;
 }

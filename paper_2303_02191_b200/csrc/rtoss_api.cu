@@ -278,12 +278,12 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
         if (e == cudaSuccess && rtoss_tc_weights_eligible(p)) {
             // dense-expanded weights of the tensor path; zeroed once: the trailing Cout*Cin mod 9 weights of a 1x1
             // layer are pruned for good and no later pack writes them
-            const size_t wtc_bytes =
-                (size_t)(ksize == 3 ? 9 : 1) * rtoss_wtc_layout_of(Cout, ksize).rows * Cin * rtoss_dtype_size(compute_dtype);
+            const size_t wtc_bytes = (size_t)(ksize == 3 ? 9 : 1) * rtoss_wtc_layout_of(Cout, ksize).rows * Cin *
+                                     rtoss_dtype_size(compute_dtype) * (compute_dtype == RTOSS_F32 ? 2 : 1);   // fp32: heads + remainders
             e = cudaMalloc(&p->wtc, wtc_bytes);
             if (e == cudaSuccess) e = cudaMemsetAsync(p->wtc, 0, wtc_bytes, s);
             if (e == cudaSuccess && ksize == 3) {
-                p->issue_n = rtoss_issue_words(Cout, Cin, ksize);
+                p->issue_n = rtoss_issue_words(Cout, Cin, ksize, compute_dtype);
                 e = cudaMalloc((void**)&p->issue, sizeof(unsigned long long) * (size_t)p->issue_n);
             }
         }
@@ -303,7 +303,8 @@ rtoss_status rtoss_pack(rtoss_ctx* ctx, const void* w_dev, rtoss_dtype w_dtype, 
     // the ordering pass also gathers which (tap, channel slab) pairs of every filter tile hold kept weights; its words start at zero
     if (e == cudaSuccess && !le && p->issue) e = cudaMemsetAsync(p->issue, 0, sizeof(unsigned long long) * (size_t)p->issue_n, s);
     if (e == cudaSuccess && !le && ksize == 3)
-        le = rtoss_launch_pack_order(pid_dev, Cout, Cin, P, p->perm, p->bucket_off, p->masks_dev, p->issue, cuda_stream);
+        le = rtoss_launch_pack_order(pid_dev, Cout, Cin, P, p->perm, p->bucket_off, p->masks_dev, p->issue,
+                                     rtoss_issue_cb_log2(compute_dtype), cuda_stream);
     if (e != cudaSuccess || le) {
         rtoss_status r = cuda_fail(ctx, "pack launch", e != cudaSuccess ? (int)e : le);
         if (!reuse) rtoss_packed_destroy(p);

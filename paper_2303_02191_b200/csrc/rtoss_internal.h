@@ -105,7 +105,7 @@ int rtoss_launch_pack_values(const void* w, rtoss_dtype wdt, int64_t n_kernels, 
                              int k, void* val, rtoss_dtype vdt, uint8_t* pid_copy, void* wtc, int ksize, int Cout, int Cin,
                              void* stream);
 int rtoss_launch_pack_order(const uint8_t* pid, int Cout, int Cin, int P, uint32_t* perm, uint32_t* bucket_off,
-                            const uint16_t* masks_dev, unsigned long long* issue, void* stream);
+                            const uint16_t* masks_dev, unsigned long long* issue, int cb_log2, void* stream);
 int rtoss_launch_select_shared(const void* w, rtoss_dtype wdt, int Cout, int Cin, int FB, int CB, const MaskTable& t, int P,
                                uint8_t* pid, void* stream);
 int rtoss_launch_to_dense(const rtoss_packed* p, void* w_out, void* stream);
@@ -115,8 +115,10 @@ int rtoss_launch_conv3x3(const rtoss_ctx* ctx, const rtoss_packed* p, const void
 int rtoss_launch_conv1x1(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y,
                          const rtoss_conv_desc* d, void* stream);
 // Number of issue words of a layer (tiles of 128 filter rows x blocks of 64 channels).
-static inline int rtoss_issue_words(int Cout, int Cin, int ksize) {
-    return ((rtoss_wtc_layout_of(Cout, ksize).rows + 127) / 128) * ((Cin + 63) / 64);
+static inline int rtoss_issue_cb_log2(rtoss_dtype d) { return d == RTOSS_F32 ? 5 : 6; }   // channels per 128-byte block
+static inline int rtoss_issue_words(int Cout, int Cin, int ksize, rtoss_dtype d) {
+    const int cb = 1 << rtoss_issue_cb_log2(d);
+    return ((rtoss_wtc_layout_of(Cout, ksize).rows + 127) / 128) * ((Cin + cb - 1) / cb);
 }
 
 // tensor path (conv_tc.cu)

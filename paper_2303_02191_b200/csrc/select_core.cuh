@@ -45,7 +45,8 @@ template <> __device__ __forceinline__ __half narrow_to<__half>(float v) { retur
 // Writes of one kernel (3x3) or run of nine (1x1) with mask m: its k kept values, ascending taps, rounded to V, to
 // val[i*k ...]; and, where the handle carries dense-expanded weights for the tensor path (wtc != nullptr), all nine
 // taps, pruned ones as +0:  3x3 -> wtc[t][row][ci] with `rows` rows per tap, filter co = i / Cin at rows
-// c*rep_rows + co for c < copies (one copy at row co in the plain layout);  1x1 -> wtc[9*i + t].
+// c*rep_rows + co for c < copies (one copy at row co in the plain layout);  1x1 -> wtc[9*i + t].  fp32 handles hold
+// two such arrays back to back: tf32 heads, then remainders.
 template <typename V>
 __device__ __forceinline__ void pack_one(const float (&w)[9], unsigned m, int64_t i, int k, V* __restrict__ val,
                                          V* __restrict__ wtc, int ksize, int Cin, int rows, int rep_rows, int copies) {
@@ -56,13 +57,27 @@ __device__ __forceinline__ void pack_one(const float (&w)[9], unsigned m, int64_
         if (m & (1u << t)) out[j++] = narrow_to<V>(w[t]);
     if (wtc) {
         const int64_t co = i / Cin, ci = i - co * Cin;
+        // fp32: the tensor path multiplies tf32 operands, so every weight is stored as its tf32 head (the 19 leading bits)
+        // and, in a second copy of the array behind the first, the remainder (exact in fp32)
+        const int64_t lo_at = (int64_t)(ksize == 3 ? 9 : 1) * rows * Cin;
 #pragma unroll
         for (int t = 0; t < 9; ++t) {
-            const V v = (m & (1u << t)) ? narrow_to<V>(w[t]) : narrow_to<V>(0.f);
+            V v = (m & (1u << t)) ? narrow_to<V>(w[t]) : narrow_to<V>(0.f);
+            V lo = v;
+            if (sizeof(V) == 4) {
+                const float f = (m & (1u << t)) ? w[t] : 0.f;
+                const float head = __uint_as_float(__float_as_uint(f) & 0xFFFFE000u);
+                v = narrow_to<V>(head);
+                lo = narrow_to<V>(__fsub_rn(f, head));
+            }
             if (ksize == 3) {
-                for (int c = 0; c < copies; ++c) wtc[((int64_t)t * rows + c * rep_rows + co) * Cin + ci] = v;
+                for (int c = 0; c < copies; ++c) {
+                    wtc[((int64_t)t * rows + c * rep_rows + co) * Cin + ci] = v;
+                    if (sizeof(V) == 4) wtc[lo_at + ((int64_t)t * rows + c * rep_rows + co) * Cin + ci] = lo;
+                }
             } else {
                 wtc[i * 9 + t] = v;
+                if (sizeof(V) == 4) wtc[lo_at + i * 9 + t] = lo;
             }
         }
     }
@@ -75,19 +90,20 @@ __device__ __forceinline__ void pack_one(const float (&w)[9], unsigned m, int64_
 // bucket ends before bucket_off's closing entry Cout) rather than written past the channel's slice.
 //
 // On the way the warp also records which taps the tensor path has to multiply at all: `issue` (nullable) holds one
-// 64-bit word per (tile of 128 filters, block of 64 input channels), bit 4 t + s set when some kernel of the tile
-// with its channel in 16-channel slab s of the block keeps tap t (the union of the kept taps over the tile, from
+// 64-bit word per (tile of 128 filters, block of 2^cb_log2 input channels: 64 for 16-bit handles, 32 for fp32 ones --
+// 128 bytes of a row), bit 4 t + s set when some kernel of the tile with its channel in slab s (a quarter) of the
+// block keeps tap t (the union of the kept taps over the tile, from
 // `masks`, the table as the device sees it).  The words must be zero before the pass; channels add their bits with
 // atomicOr.  A (tile, slab, tap) whose bit stays clear holds only pruned weights: its matrix instruction is skipped.
 __device__ __forceinline__ void order_channel(const uint8_t* __restrict__ pid, int Cout, int Cin, int P, int ci,
                                               uint32_t* __restrict__ perm, uint32_t* __restrict__ bucket_off,
                                               uint32_t* fill, int lane, const uint16_t* __restrict__ masks = nullptr,
-                                              unsigned long long* __restrict__ issue = nullptr) {
+                                              unsigned long long* __restrict__ issue = nullptr, int cb_log2 = 6) {
     for (int p = lane; p < 256; p += 32) fill[p] = 0;
     __syncwarp();
     // pass 1: histogram
     unsigned used = 0;   // taps kept by any filter of the current tile of 128
-    const int ncb = (Cin + 63) >> 6;
+    const int cb_mask = (1 << cb_log2) - 1, ncb = (Cin + cb_mask) >> cb_log2;
     for (int base = 0; base < Cout; base += 32) {
         const int co = base + lane;
         unsigned key = co < Cout ? pid[(size_t)co * Cin + ci] : 0xFFFFu;
@@ -101,8 +117,8 @@ __device__ __forceinline__ void order_channel(const uint8_t* __restrict__ pid, i
                     unsigned long long bits = 0;
 #pragma unroll
                     for (int t = 0; t < 9; ++t)
-                        if (used & (1u << t)) bits |= 1ull << (4 * t + ((ci & 63) >> 4));
-                    atomicOr(issue + (size_t)(base >> 7) * ncb + (ci >> 6), bits);
+                        if (used & (1u << t)) bits |= 1ull << (4 * t + ((ci & cb_mask) >> (cb_log2 - 2)));
+                    atomicOr(issue + (size_t)(base >> 7) * ncb + (ci >> cb_log2), bits);
                 }
                 used = 0;
             }

@@ -105,13 +105,13 @@ __global__ void __launch_bounds__(kOrderWarps * 32) pack_order_kernel(const uint
                                                                       int P, uint32_t* __restrict__ perm,
                                                                       uint32_t* __restrict__ bucket_off,
                                                                       const uint16_t* __restrict__ masks,
-                                                                      unsigned long long* __restrict__ issue) {
+                                                                      unsigned long long* __restrict__ issue, int cb_log2) {
     rtoss_dev::pdl_enter();
     __shared__ uint32_t fill_all[kOrderWarps][256];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ci = blockIdx.x * kOrderWarps + warp;
     if (ci >= Cin) return;  // whole warp leaves together; no block-wide barrier below
-    rtoss_dev::order_channel(pid, Cout, Cin, P, ci, perm, bucket_off, fill_all[warp], lane, masks, issue);
+    rtoss_dev::order_channel(pid, Cout, Cin, P, ci, perm, bucket_off, fill_all[warp], lane, masks, issue, cb_log2);
 }
 
 // Selection with one pattern per block of FB filters x CB input channels (a variant of Algorithm 2 in the spirit of
@@ -252,10 +252,10 @@ int rtoss_launch_pack_values(const void* w, rtoss_dtype wdt, int64_t n_kernels, 
 }
 
 int rtoss_launch_pack_order(const uint8_t* pid, int Cout, int Cin, int P, uint32_t* perm, uint32_t* bucket_off,
-                            const uint16_t* masks_dev, unsigned long long* issue, void* stream) {
+                            const uint16_t* masks_dev, unsigned long long* issue, int cb_log2, void* stream) {
     const int grid = (Cin + kOrderWarps - 1) / kOrderWarps;
     rtoss_dev::launch_pdl(pack_order_kernel, grid, kOrderWarps * 32, 0, (cudaStream_t)stream, pid, Cout, Cin, P, perm, bucket_off,
-                          masks_dev, issue);
+                          masks_dev, issue, cb_log2);
     return (int)cudaGetLastError();
 }
 

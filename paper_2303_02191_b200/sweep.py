@@ -2,8 +2,9 @@
 Cin = Cout in {64, 256, 512} x H = W in {20, 40, 80, 160} x batch in {1, 32} x k in {2, 3, 4, 9} x {bf16, fp32}.
 
 For every point: cold-L2 and warm kernel time (CUDA events), algorithmic GB/s, non-zero GFLOP/s and the
-fraction of the point's roofline max(bytes / HBM peak, nnz FLOP / pipe peak).  bf16 runs NHWC (tensor path
-where it applies), fp32 runs NCHW (FMA path).  Writes a CSV and prints a short summary.
+fraction of the point's roofline max(bytes / HBM peak, nnz FLOP / pipe peak).  Both types run NHWC on the tensor
+path where it applies (fp32: kind::tf32 with three products per tap, pipe peak = bf16 peak / 2 / 3); `--fp32-nchw`
+runs fp32 in NCHW on the FMA pipes instead.  Writes a CSV and prints a short summary.
 
     python -m paper_2303_02191_b200.sweep --out sweep.csv [--quick]
 """
@@ -48,6 +49,8 @@ def main():
     ap.add_argument("--out", default="sweep.csv")
     ap.add_argument("--quick", action="store_true")
     ap.add_argument("--reps", type=int, default=10)
+    ap.add_argument("--fp32-nchw", action="store_true", help="fp32 points in NCHW on the FMA path")
+    ap.add_argument("--only", default=None, help="bf16 or f32: only that half of the sweep")
     args = ap.parse_args()
     hbm, tc_peak, kind = peaks()
     ctx = rt.Context(0)
@@ -55,8 +58,10 @@ def main():
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     rows = []
     for dt, C, H, N, k in points(args.quick):
+        if args.only and dt != args.only:
+            continue
         tdt = torch.bfloat16 if dt == "bf16" else torch.float32
-        layout = rt.NHWC if dt == "bf16" else rt.NCHW
+        layout = rt.NCHW if (dt == "f32" and args.fp32_nchw) else rt.NHWC
         preset = {2: rt.PRESET_CONN4, 3: rt.PRESET_CONN4, 4: rt.PRESET_CENTRE8, 9: rt.PRESET_DENSE}[k]
         masks = rt.rtoss_pattern_preset(k, preset)
         w = torch.from_numpy(synth.kaiming_weights(0, C + k, C, C, 3)).to(dev)
@@ -91,12 +96,14 @@ def main():
         L = dict(ksize=3, stride=1, cin=C, cout=C, H=H, W=H)
         flops = synth.layer_nnz_flops(L, N, k)
         nbytes = synth.layer_bytes(L, N, k, 2 if dt == "bf16" else 4)
-        pipe = tc_peak if path == rt.PATH_TENSOR else ALU_PEAK_TFLOPS
+        # tensor pipe: measured bf16 peak; fp32 runs tf32 instructions (half the rate) three times per product
+        pipe = (tc_peak if dt == "bf16" else tc_peak / 6) if path == rt.PATH_TENSOR else ALU_PEAK_TFLOPS
         t_roof = max(nbytes / (hbm * 1e9), flops / (pipe * 1e12))
         rows.append(dict(dtype=dt, C=C, HW=H, N=N, k=k, path="tensor" if path == rt.PATH_TENSOR else "fma",
                          cold_ms=round(cold, 5), warm_ms=round(warm, 5), gbs=round(nbytes / cold / 1e6, 1),
                          nnz_gflops=round(flops / cold / 1e6, 1), roofline_us=round(t_roof * 1e6, 2),
-                         bound="hbm" if nbytes / (hbm * 1e9) >= flops / (pipe * 1e12) else ("tensor" if path == rt.PATH_TENSOR else "alu"),
+                         bound="hbm" if nbytes / (hbm * 1e9) >= flops / (pipe * 1e12) else
+                         (("tensor" if dt == "bf16" else "tensor (tf32 x3)") if path == rt.PATH_TENSOR else "alu"),
                          frac=round(t_roof / (cold * 1e-3), 4)))
         packed.close()
         del x, y
@@ -108,6 +115,8 @@ def main():
         wr.writerows(rows)
     for dt in ("bf16", "f32"):
         sel = [r for r in rows if r["dtype"] == dt]
+        if not sel:
+            continue
         fr = np.array([r["frac"] for r in sel])
         best = max(sel, key=lambda r: r["frac"])
         print("%s: %d points, roofline fraction median %.3f, max %.3f (C=%d HW=%d N=%d k=%d, %.1f nnz GFLOP/s); peaks %s" %
