@@ -1277,7 +1277,7 @@ struct TcPlan {
 // The plan picks TH, the column segment TW (images wider than a TMA box are cut into segments), the
 // ring depths, and how many taps share a weight stage.
 bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count, bool pxm, int w_rows, bool resid, TcPlan* out,
-             int n_prob = 1, bool f32 = false) {
+             int n_prob = 1, bool f32 = false, int force_G = 0) {
     const int halo = ksize == 3 ? (S == 1 ? 2 : 1) : 0;
     const int n_sub = (ksize == 3 && S == 2) ? 4 : 1;
     const int max_pitch = S == 1 ? 256 : 128;  // TMA box: at most 256 elements traversed per dimension
@@ -1302,6 +1302,7 @@ bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count
             const int sub_rows = round_up(need_rows, 8);
             const int a_bytes = n_sub * sub_rows * kRowBytes * (f32 ? 2 : 1);   // (fp32: heads and remainders)
             for (int G = (ksize == 3 ? 3 : 1); G >= 1; G -= 2) {
+                if (force_G && G != force_G) continue;   // (the problems of one launch share the weight ring: one G for all)
                 const int b_bytes = G * w_rows * kRowBytes;
                 int na = (cap - fixed - 2 * b_bytes) / a_bytes;
                 if (na < 1) continue;
@@ -1316,8 +1317,10 @@ bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count
                 // an instruction costs about the same for any N: what counts is useful positions per instruction
                 const double eff = (double)(th * tw) / (pxm ? 128.0 * halves : 256.0) * Ho / (double)((Ho + th - 1) / th * th) * Wo / (double)(tw * nseg);
                 const double halo_cost = (double)(th * tw) / (double)(rows_staged * wq);  // staged pixels that are outputs
-                const double score = eff * (0.5 + 0.5 * balance) * (G == 3 || ksize == 1 ? 1.0 : 0.8) * (na >= 2 ? 1.0 : 0.8) *
-                                         (0.8 + 0.2 * halo_cost) +
+                // (fp32: a block feeds 108 instructions, twelve per tap, so a stage per tap costs little, while a single
+                // activation stage leaves the fetch and the split of the next block uncovered)
+                const double score = eff * (0.5 + 0.5 * balance) * (G == 3 || ksize == 1 ? 1.0 : (f32 ? 0.95 : 0.8)) *
+                                         (na >= 2 ? 1.0 : (f32 ? 0.7 : 0.8)) * (0.8 + 0.2 * halo_cost) +
                                      1e-4 * th;
                 if (score > best) {
                     best = score;
@@ -1334,7 +1337,7 @@ bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count
                     out->tiles_x = nseg;
                     out->smem = na * a_bytes + nb * b_bytes + fixed;
                 }
-                break;  // the largest G that fits is taken for this (th, tw)
+                if (!f32) break;  // 16-bit data: the largest G that fits is taken for this (th, tw); fp32 weighs both
             }
         }
     }
@@ -1350,7 +1353,7 @@ struct ProbPlan {
 // Geometry, operand roles and TMA descriptors of one convolution.  The rings' depths and the split along K are the
 // launch's business (the caller's).  Returns a cudaError_t as int.
 int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y, const rtoss_conv_desc* d, int n_prob, int sms,
-                  TcArgs* out, ProbPlan* pp, CUtensorMap* tmA_out, CUtensorMap* tmB_out) {
+                  TcArgs* out, ProbPlan* pp, CUtensorMap* tmA_out, CUtensorMap* tmB_out, int force_G = 0) {
     const int taps = p->ksize == 3 ? 9 : 1;
     const int S = d->stride;
     const int Ho = (d->H - 1) / S + 1, Wo = (d->W - 1) / S + 1;
@@ -1361,7 +1364,8 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
     const int w_rows = pxm ? round_up(p->Cout, 16) : kMTile;
     const bool f32 = p->dtype == RTOSS_F32;
     const int esize = f32 ? 4 : 2;
-    if (!plan_tc(d->N, Ho, Wo, p->ksize, S, (p->Cout + kMTile - 1) / kMTile, sms, pxm, w_rows, d->residual_dev != nullptr, &plan, n_prob, f32))
+    if (!plan_tc(d->N, Ho, Wo, p->ksize, S, (p->Cout + kMTile - 1) / kMTile, sms, pxm, w_rows, d->residual_dev != nullptr, &plan, n_prob, f32,
+                 force_G))
         return (int)cudaErrorInvalidConfiguration;
 
     TcArgs& a = *out;
@@ -1641,23 +1645,36 @@ int rtoss_launch_conv_tc_group(const rtoss_ctx* ctx, int n, const rtoss_packed* 
     g.n_prob = n;
     int a_max = 0, acc_max = 0, b_bytes = 0, units = 0;
     long n_tiles[kMaxProb];
-    for (int i = 0; i < n; ++i) {
-        // (every problem is planned with the launch's fixed shared memory: all position tables, the residual staging if any needs it)
-        rtoss_conv_desc dd = *ds[i];
-        static const int dummy = 0;
-        if (resid && !dd.residual_dev) dd.residual_dev = &dummy;   // only the plan's memory budget looks at it here
-        TcArgs tmp;
-        int e = build_problem(ctx, ps[i], xs[i], ys[i], &dd, n, sms, &tmp, &pp[i], &g.tmA[i], &g.tmB[i]);
-        if (e == (int)cudaErrorInvalidConfiguration) return -1;
-        if (e) return e;
-        tmp.resid = ds[i]->residual_dev;
-        tmp.resid_post = (ds[i]->residual_dev && ds[i]->residual_after_act) ? 1 : 0;
-        g.prob[i] = tmp;
-        if (i == 0) b_bytes = pp[i].b_stage_bytes;
-        if (pp[i].b_stage_bytes != b_bytes || tmp.G != g.prob[0].G || tmp.n_sub != g.prob[0].n_sub) return -1;
-        if (pp[i].a_stage_bytes > a_max) a_max = pp[i].a_stage_bytes;
-        if (pp[i].acc_cols > acc_max) acc_max = pp[i].acc_cols;
-        n_tiles[i] = (long)tmp.N * tmp.tiles_y * tmp.tiles_x * tmp.co_tiles;
+    // every problem is planned on its own first; where they disagree on the taps per weight stage, all are planned again
+    // with the smallest (a stage per tap fits whatever fits three)
+    int force_G = 0;
+    for (int pass = 0; pass < 2; ++pass) {
+        bool agree = true;
+        int g_min = 9;
+        a_max = acc_max = 0;
+        for (int i = 0; i < n; ++i) {
+            // (planned with the launch's fixed shared memory: all position tables, the residual staging if any needs it)
+            rtoss_conv_desc dd = *ds[i];
+            static const int dummy = 0;
+            if (resid && !dd.residual_dev) dd.residual_dev = &dummy;   // only the plan's memory budget looks at it here
+            TcArgs tmp;
+            int e = build_problem(ctx, ps[i], xs[i], ys[i], &dd, n, sms, &tmp, &pp[i], &g.tmA[i], &g.tmB[i], force_G);
+            if (e == (int)cudaErrorInvalidConfiguration) return -1;
+            if (e) return e;
+            tmp.resid = ds[i]->residual_dev;
+            tmp.resid_post = (ds[i]->residual_dev && ds[i]->residual_after_act) ? 1 : 0;
+            g.prob[i] = tmp;
+            if (i == 0) b_bytes = pp[i].b_stage_bytes;
+            if (tmp.n_sub != g.prob[0].n_sub) return -1;
+            if (pp[i].b_stage_bytes != b_bytes || tmp.G != g.prob[0].G) agree = false;
+            if (tmp.G < g_min) g_min = tmp.G;
+            if (pp[i].a_stage_bytes > a_max) a_max = pp[i].a_stage_bytes;
+            if (pp[i].acc_cols > acc_max) acc_max = pp[i].acc_cols;
+            n_tiles[i] = (long)tmp.N * tmp.tiles_y * tmp.tiles_x * tmp.co_tiles;
+        }
+        if (agree) break;
+        if (pass == 1) return -1;
+        force_G = g_min;
     }
     // insertion sort of the problems by falling tile count (stable), applied to every per-problem array
     for (int i = 1; i < n; ++i)
