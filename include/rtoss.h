@@ -376,6 +376,25 @@ rtoss_status rtoss_inject_lost_copy(rtoss_ctx* ctx);
 rtoss_status rtoss_conv_pattern_host(rtoss_ctx* ctx, const rtoss_packed* p, const void* x_host, void* y_host,
                                      const rtoss_conv_desc* desc);
 
+/* How the FMA path would tile a 3x3 call (host arithmetic only, nothing is launched; for Cin <= 4 only small_cin is
+ * set: that kernel has no staging plan).  staging: 0 = plain loads, 1 = NCHW rows as aligned vectors of vector_bytes
+ * through cp.async, 2 = NHWC pixels as 16-byte vectors through cp.async.  With staging 1 the address of every vector,
+ *   ((n*Cin + ci)*H*W + iy*W + tx*lanes_x*pixels_per_lane*stride - vector_bytes/es + j*vector_bytes/es) * es
+ * (es = bytes per activation, tx = tile column, j = vector inside the staged row), is a multiple of vector_bytes for a
+ * 16-byte aligned tensor: the plan guarantees it, and the CPU tests check it tile by tile.  Not part of the paper's
+ * method.  RTOSS_ERR_INVALID_ARG, RTOSS_ERR_UNSUPPORTED (no shape fits the shared memory). */
+typedef struct {
+    int small_cin;
+    int pixels_per_lane, filters_per_warp, warps, ctas_per_sm; /* kernel shape */
+    int lanes_x, lanes_y;                                      /* lane arrangement inside a warp */
+    int tiles_x, tiles_y, grid_x, grid_y;                      /* tiles per image, CTAs */
+    int staged_rows, staged_cols;                              /* input tile with halo */
+    int staging, vector_bytes, vectors_per_plane;
+    int shared_bytes;
+} rtoss_fma_plan;
+rtoss_status rtoss_fma_plan3x3(const rtoss_conv_desc* desc, int Cin, int Cout, int k, rtoss_dtype packed_dtype,
+                               rtoss_fma_plan* out);
+
 /* ---- glue between the convolutions of a whole network ---------------------- */
 /* Not part of the paper's method (Table 3 and Fig. 6 time whole models, whose graphs need these between the
  * pruned convolutions).  Element-wise, bandwidth-bound; x and y in the given layout and dtype; y may be a

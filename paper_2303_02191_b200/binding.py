@@ -31,6 +31,7 @@ SYMBOLS = [
     "rtoss_pattern_rank", "rtoss_pattern_table_derive",
     "rtoss_batch_create", "rtoss_batch_select_pack", "rtoss_batch_destroy",
     "rtoss_select_patterns_shared", "rtoss_conv_group", "rtoss_set_wait_limit", "rtoss_inject_lost_copy",
+    "rtoss_fma_plan3x3",
 ]
 
 
@@ -62,6 +63,12 @@ class ConvDesc(ctypes.Structure):
                 ("layout", ctypes.c_int), ("io_dtype", ctypes.c_int), ("act", ctypes.c_int),
                 ("bias_dev", ctypes.c_void_p), ("y_channel_offset", ctypes.c_int), ("y_channel_stride", ctypes.c_int),
                 ("path", ctypes.c_int), ("residual_dev", ctypes.c_void_p), ("residual_after_act", ctypes.c_int)]
+
+
+class FmaPlan(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in (
+        "small_cin", "pixels_per_lane", "filters_per_warp", "warps", "ctas_per_sm", "lanes_x", "lanes_y", "tiles_x", "tiles_y",
+        "grid_x", "grid_y", "staged_rows", "staged_cols", "staging", "vector_bytes", "vectors_per_plane", "shared_bytes")]
 
 
 class ConvItem(ctypes.Structure):
@@ -101,6 +108,7 @@ def _load():
     lib.rtoss_conv_group.argtypes = [vp, ctypes.POINTER(ConvItem), ci, ctypes.POINTER(ci), vp]
     lib.rtoss_set_wait_limit.argtypes = [vp, ctypes.c_longlong]
     lib.rtoss_inject_lost_copy.argtypes = [vp]
+    lib.rtoss_fma_plan3x3.argtypes = [ctypes.POINTER(ConvDesc), ci, ci, ci, ci, ctypes.POINTER(FmaPlan)]
     lib.rtoss_select_patterns_shared.argtypes = [vp, vp, ci, ci, ci, ci, ci, vp, ci, ci, vp, vp]
     lib.rtoss_prune_dense_static.argtypes = [vp, ci, ci, ci, ci, vp, ci, ci, vp, vp]
     lib.rtoss_maxpool2d.argtypes = [vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, vp]
@@ -196,6 +204,17 @@ def rtoss_upsample2x(x, y, N, C, H, W, layout=NCHW, y_channel_offset=0, y_channe
 def rtoss_add_act(a, b, y, act=ACT_NONE):
     _glue_check(lib.rtoss_add_act(a.data_ptr(), b.data_ptr(), y.data_ptr(), a.numel(), _torch_dtype_code(a), act, _stream()))
     return y
+
+
+def rtoss_fma_plan3x3(N, H, W, stride, layout, io_dtype, Cin, Cout, k, packed_dtype=None):
+    """The tiling the FMA path would use for a 3x3 call (host only) -> FmaPlan; raises on an argument error."""
+    d = ConvDesc(int(N), int(H), int(W), int(stride), int(layout), int(io_dtype), 0, None, 0, 0, 0, None, 0)
+    out = FmaPlan()
+    st = lib.rtoss_fma_plan3x3(ctypes.byref(d), int(Cin), int(Cout), int(k), int(io_dtype if packed_dtype is None else packed_dtype),
+                               ctypes.byref(out))
+    if st != OK:
+        raise RtossError(st, status_string(st))
+    return out
 
 
 def rtoss_prune_dense_static(w, ksize, masks, k, out=None):

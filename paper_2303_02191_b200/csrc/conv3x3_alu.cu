@@ -656,11 +656,17 @@ void choose_lanes(int Ho, int Wo, int PH, int PW, int S, int* LX, int* LY) {
 
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
-template <typename T, int S, int PH, int PW, int CO_T, int WARPS, int MINB>
-int launch_variant(Conv3Args& a, cudaStream_t stream) {
-    constexpr int CO_BLOCK = WARPS * CO_T;
-    constexpr int kThreads = WARPS * 32;
-    const int es = (int)sizeof(T);
+// Tiling and staging plan of one call for a kernel shape (PH x PW output pixels per lane, CO_T filters per warp, WARPS
+// warps, MINB CTAs per SM): lane arrangement, tile sizes, how the activations travel, shared-memory layout.  Host
+// arithmetic only.  Returns the dynamic shared memory in bytes, or 0 when the shape does not fit.
+//
+// NCHW activations travel as aligned vectors of vb bytes through cp.async.  A vector's address is
+//   base + ((n*Cin + ci)*H*W + iy*W + ox0*S - veq + j*veq) * es,   ox0 = tx * LX * PW,  veq = vb / es,
+// so vb has to divide the row pitch W*es AND the byte step between neighbouring tiles, LX*PW*S*es: with four pixels per
+// lane and an odd number of lane columns every second tile of a 16-bit image starts 8 bytes off a 16-byte boundary
+// (a misaligned-address fault on a 64-channel 40x40 bf16 layer once showed exactly that).
+size_t plan_variant(Conv3Args& a, int es, int S, int PH, int PW, int CO_T, int WARPS, int MINB) {
+    const int CO_BLOCK = WARPS * CO_T;
     choose_lanes(a.Ho, a.Wo, PH, PW, S, &a.LX, &a.LY);
     a.tiles_x = (a.Wo + a.LX * PW - 1) / (a.LX * PW);
     a.tiles_y = (a.Ho + a.LY * PH - 1) / (a.LY * PH);
@@ -683,8 +689,10 @@ int launch_variant(Conv3Args& a, cudaStream_t stream) {
     a.rawX_bytes = 0;
     const bool x16 = (reinterpret_cast<uintptr_t>(a.x) & 15) == 0;
     if (a.layout == RTOSS_NCHW && x16) {
-        const int row_bytes = a.W * es;
-        const int vb = row_bytes % 16 == 0 ? 16 : row_bytes % 8 == 0 ? 8 : row_bytes % 4 == 0 ? 4 : 0;
+        const int row_bytes = a.W * es, step_bytes = a.LX * PW * S * es;
+        int vb = 0;
+        for (int cand = 16; cand >= 4 && !vb; cand >>= 1)
+            if (row_bytes % cand == 0 && step_bytes % cand == 0) vb = cand;
         if (vb >= es && vb > 0) {
             const int veq = vb / es;
             const int nv = round_up(veq - 1 + a.TW_in, veq) / veq;
@@ -719,8 +727,15 @@ int launch_variant(Conv3Args& a, cudaStream_t stream) {
     off += a.w_async ? 2 * CO_BLOCK * 8 : 0;
     a.off_tab = off;
     off += 2 * (int)sizeof(int) * n_tab;
-    const size_t smem = (size_t)off;
-    if (smem > 220 * 1024) return (int)cudaErrorInvalidConfiguration;
+    return off > 220 * 1024 ? 0 : (size_t)off;
+}
+
+template <typename T, int S, int PH, int PW, int CO_T, int WARPS, int MINB>
+int launch_variant(Conv3Args& a, cudaStream_t stream) {
+    constexpr int CO_BLOCK = WARPS * CO_T;
+    constexpr int kThreads = WARPS * 32;
+    const size_t smem = plan_variant(a, (int)sizeof(T), S, PH, PW, CO_T, WARPS, MINB);
+    if (!smem) return (int)cudaErrorInvalidConfiguration;
     auto kern = conv3x3_alu_kernel<T, S, PH, PW, CO_T, WARPS, MINB>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return (int)e;
@@ -729,10 +744,28 @@ int launch_variant(Conv3Args& a, cudaStream_t stream) {
     return (int)cudaGetLastError();
 }
 
+// Which kernel shape takes a call: one output row of eight pixels per lane, eight filters per warp, eight warps, two
+// CTAs per SM; a layer that fills fewer than half the SMs that way takes the finer shape (four pixels per lane, four
+// filters per warp, four warps, four CTAs per SM: a quarter of the outputs per CTA).
+struct FmaShape {
+    int PH, PW, CO_T, WARPS, MINB;
+};
+FmaShape choose_shape(const Conv3Args& a0, int es, int S) {
+    Conv3Args a = a0;
+    const FmaShape big = {1, 8, 8, 8, 2}, fine = {1, 4, 4, 4, 4};
+    if (!plan_variant(a, es, S, big.PH, big.PW, big.CO_T, big.WARPS, big.MINB)) return big;
+    const long ctas = (long)a.tiles_x * a.tiles_y * a.N * ((a.Cout + 63) / 64);
+    return ctas < 74 ? fine : big;
+}
+
 template <typename T>
 int launch_typed(Conv3Args& a, int stride, cudaStream_t stream) {
     if (a.Cin <= 4) return launch_small_cin<T>(a, stride, stream);
-    // one output row of eight pixels per lane, eight filters per warp, two CTAs per SM
+    const FmaShape sh = choose_shape(a, (int)sizeof(T), stride);
+    if (sh.PW == 4) {
+        if (stride == 1) return launch_variant<T, 1, 1, 4, 4, 4, 4>(a, stream);
+        return launch_variant<T, 2, 1, 4, 4, 4, 4>(a, stream);
+    }
     if (stride == 1) return launch_variant<T, 1, 1, 8, 8, 8, 2>(a, stream);
     return launch_variant<T, 2, 1, 8, 8, 8, 2>(a, stream);
 }
@@ -771,4 +804,52 @@ int rtoss_launch_conv3x3(const rtoss_ctx* ctx, const rtoss_packed* p, const void
         case RTOSS_F16: return launch_typed<__half>(a, d->stride, s);
     }
     return (int)cudaErrorInvalidValue;
+}
+
+// The tiling the FMA path would use for a 3x3 call (host arithmetic only; see rtoss.h).
+extern "C" rtoss_status rtoss_fma_plan3x3(const rtoss_conv_desc* d, int Cin, int Cout, int k, rtoss_dtype packed_dtype,
+                                          rtoss_fma_plan* out) {
+    if (!d || !out || Cin < 1 || Cout < 1 || k < 1 || k > 9 || d->N < 1 || d->H < 1 || d->W < 1 || (d->stride != 1 && d->stride != 2) ||
+        (int)d->io_dtype < 0 || (int)d->io_dtype > 2 || (int)packed_dtype < 0 || (int)packed_dtype > 2)
+        return RTOSS_ERR_INVALID_ARG;
+    memset(out, 0, sizeof(*out));
+    if (Cin <= 4) {
+        out->small_cin = 1;   // the kernel for up to four input channels: no staging plan
+        return RTOSS_OK;
+    }
+    Conv3Args a;
+    memset(&a, 0, sizeof(a));
+    a.x = nullptr;   // (a 16-byte aligned pointer)
+    a.val_dtype = (int)packed_dtype;
+    a.val_esize = (int)rtoss_dtype_size(packed_dtype);
+    a.N = d->N;
+    a.Cin = Cin;
+    a.Cout = Cout;
+    a.H = d->H;
+    a.W = d->W;
+    a.Ho = (d->H - 1) / d->stride + 1;
+    a.Wo = (d->W - 1) / d->stride + 1;
+    a.k = k;
+    a.layout = (int)d->layout;
+    const int es = (int)rtoss_dtype_size(d->io_dtype);
+    const FmaShape sh = choose_shape(a, es, d->stride);
+    const size_t smem = plan_variant(a, es, d->stride, sh.PH, sh.PW, sh.CO_T, sh.WARPS, sh.MINB);
+    if (!smem) return RTOSS_ERR_UNSUPPORTED;
+    out->pixels_per_lane = sh.PW;
+    out->filters_per_warp = sh.CO_T;
+    out->warps = sh.WARPS;
+    out->ctas_per_sm = sh.MINB;
+    out->lanes_x = a.LX;
+    out->lanes_y = a.LY;
+    out->tiles_x = a.tiles_x;
+    out->tiles_y = a.tiles_y;
+    out->grid_x = a.tiles_x * a.tiles_y * a.N;
+    out->grid_y = (Cout + sh.WARPS * sh.CO_T - 1) / (sh.WARPS * sh.CO_T);
+    out->staged_rows = a.TH_in;
+    out->staged_cols = a.TW_in;
+    out->staging = a.xmode;
+    out->vector_bytes = a.vb;
+    out->vectors_per_plane = a.EV;
+    out->shared_bytes = (int)smem;
+    return RTOSS_OK;
 }

@@ -349,3 +349,23 @@ def test_pack_with_ids_outside_the_table_stays_inside_its_arrays():
         assert off[ci][-1] == Cout and np.all(np.diff(off[ci][:-1].astype(np.int64)) >= 0)
     assert c.rtoss_device_status() == 0
     packed.close()
+
+
+FINE_SHAPE = [
+    # N, Cin, Cout, H, W, stride, dt   -- layers small enough for the FMA path's finer kernel shape (four pixels per lane)
+    (1, 64, 64, 40, 40, 1, "bf16"),     # five lane columns: tiles 40 bytes apart, 8-byte activation vectors
+    (1, 32, 32, 32, 32, 1, "f32"),      # the 32-channel fp32 test layer
+    (1, 64, 48, 20, 20, 2, "f16"),
+    (2, 40, 24, 13, 16, 1, "bf16"),
+    (1, 128, 64, 25, 36, 2, "f32"),
+]
+
+
+@pytest.mark.parametrize("N,Cin,Cout,H,W,stride,dt", FINE_SHAPE)
+def test_fma_path_finer_shape_small_nchw_layers(N, Cin, Cout, H, W, stride, dt):
+    """The shape's staging plan is checked vector by vector on the host (test_fma_plan_cpu.py); here its results."""
+    p = rt.rtoss_fma_plan3x3(N, H, W, stride, rt.NCHW, rt.DTYPE_NAMES[dt], Cin, Cout, 4)
+    assert p.pixels_per_lane == 4
+    masks = orc.pattern_preset(4, orc.PRESET_CENTRE8)
+    gu.check_layer(52, Cin + Cout + H, 3, N, Cin, Cout, H, W, stride, 4, masks, dt, "silu", "nchw", path=rt.PATH_FMA)
+    assert gu.ctx().rtoss_device_status() == 0
