@@ -1314,8 +1314,13 @@ bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count
                 const long tiles = (long)N * ((Ho + th - 1) / th) * nseg * co_tiles;
                 const double waves = (double)tiles / sm_count;
                 const double balance = grouped ? 1.0 : waves / (double)((tiles + sm_count - 1) / sm_count);  // 1 = SMs equally loaded
-                // an instruction costs about the same for any N: what counts is useful positions per instruction
-                const double eff = (double)(th * tw) / (pxm ? 128.0 * halves : 256.0) * Ho / (double)((Ho + th - 1) / th * th) * Wo / (double)(tw * nseg);
+                // What counts is useful positions per tensor-pipe cycle.  An instruction with the filters on M and N positions
+                // takes N / 2 cycles, but never less than 76 (measured: 128.2 cycles at N = 256, 75.9 at every N <= 128).
+                // That is the measure for 3x3 layers of stride 1, whose tiles are bound by their instructions; the tiles of
+                // 1x1 and stride-2 layers are bound by what surrounds the instructions (fetches, barrier rounds, the
+                // epilogue) and do better with as many positions per tile as fit (measured both ways, layer by layer).
+                const double instr_cycles = pxm ? 128.0 * halves : (ksize == 3 && S == 1 && n_px / 2.0 < 128.0) ? (n_px / 2.0 > 76.0 ? n_px / 2.0 : 76.0) : 128.0;
+                const double eff = (double)(th * tw) / (2.0 * instr_cycles) * Ho / (double)((Ho + th - 1) / th * th) * Wo / (double)(tw * nseg);
                 const double halo_cost = (double)(th * tw) / (double)(rows_staged * wq);  // staged pixels that are outputs
                 // (fp32: a block feeds 108 instructions, twelve per tap, so a stage per tap costs little, while a single
                 // activation stage leaves the fetch and the split of the next block uncovered)
