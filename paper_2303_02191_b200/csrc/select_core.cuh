@@ -51,12 +51,30 @@ template <typename V>
 __device__ __forceinline__ void pack_one(const float (&w)[9], unsigned m, int64_t i, int k, V* __restrict__ val,
                                          V* __restrict__ wtc, int ksize, int Cin, int rows, int rep_rows, int copies) {
     V* out = val + i * k;
-    int j = 0;
+    if (k * (int)sizeof(V) == 8) {
+        // the k kept values of a kernel are 8 aligned bytes (four 16-bit or two 32-bit values): gathered in registers
+        // (the j-th set bit of the mask picks the j-th slot) and written with one store
+        V slot[8 / sizeof(V)];
+        unsigned rest = m;
 #pragma unroll
-    for (int t = 0; t < 9; ++t)
-        if (m & (1u << t)) out[j++] = narrow_to<V>(w[t]);
+        for (int j = 0; j < (int)(8 / sizeof(V)); ++j) {
+            const int t = __ffs(rest) - 1;   // (a valid mask has exactly k bits)
+            rest &= rest - 1;
+            float wt = 0.f;
+#pragma unroll
+            for (int u = 0; u < 9; ++u) wt = (u == t) ? w[u] : wt;
+            slot[j] = narrow_to<V>(wt);
+        }
+        *reinterpret_cast<uint2*>(out) = *reinterpret_cast<const uint2*>(slot);
+    } else {
+        int j = 0;
+#pragma unroll
+        for (int t = 0; t < 9; ++t)
+            if (m & (1u << t)) out[j++] = narrow_to<V>(w[t]);
+    }
     if (wtc) {
-        const int64_t co = i / Cin, ci = i - co * Cin;
+        // (layers hold fewer than 2^31 kernels: 32-bit division, several times cheaper than the 64-bit one)
+        const int64_t co = (int64_t)((unsigned)i / (unsigned)Cin), ci = i - co * Cin;
         // fp32: the tensor path multiplies tf32 operands, so every weight is stored as its tf32 head (the 19 leading bits)
         // and, in a second copy of the array behind the first, the remainder (exact in fp32)
         const int64_t lo_at = (int64_t)(ksize == 3 ? 9 : 1) * rows * Cin;
@@ -71,9 +89,10 @@ __device__ __forceinline__ void pack_one(const float (&w)[9], unsigned m, int64_
                 lo = narrow_to<V>(__fsub_rn(f, head));
             }
             if (ksize == 3) {
+                const int64_t at = ((int64_t)t * rows + co) * Cin + ci;   // copy 0; copy c lies c * rep_rows rows further down
                 for (int c = 0; c < copies; ++c) {
-                    wtc[((int64_t)t * rows + c * rep_rows + co) * Cin + ci] = v;
-                    if (sizeof(V) == 4) wtc[lo_at + ((int64_t)t * rows + c * rep_rows + co) * Cin + ci] = lo;
+                    wtc[at + (int64_t)c * rep_rows * Cin] = v;
+                    if (sizeof(V) == 4) wtc[lo_at + at + (int64_t)c * rep_rows * Cin] = lo;
                 }
             } else {
                 wtc[i * 9 + t] = v;
