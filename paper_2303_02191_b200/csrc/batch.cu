@@ -79,7 +79,7 @@ __device__ __forceinline__ void stage_raw(const void* w, long long first, int co
 __global__ void __launch_bounds__(kChunk) batch_select_pack_kernel(const BatchLayer* __restrict__ layers,
                                                                    const uint32_t* __restrict__ chunk_layer,
                                                                    unsigned n_chunks) {
-    rtoss_dev::pdl_enter();
+    rtoss_dev::pdl_enter_handle_writer();
     __shared__ __align__(16) unsigned char s_sel[kChunk * 9 * 4];
     __shared__ __align__(16) unsigned char s_own[kChunk * 9 * 4];
     __shared__ uint16_t s_masks[256];
@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(kChunk) batch_select_pack_kernel(const BatchLa
 __global__ void __launch_bounds__(kOrderWarps * 32) batch_order_kernel(const BatchLayer* __restrict__ layers,
                                                                        const uint32_t* __restrict__ task_layer,
                                                                        unsigned n_tasks) {
-    rtoss_dev::pdl_enter();
+    rtoss_dev::pdl_enter_handle_writer();
     __shared__ uint32_t fill_all[kOrderWarps][256];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (unsigned task = blockIdx.x * kOrderWarps + warp; task < n_tasks; task += gridDim.x * kOrderWarps) {

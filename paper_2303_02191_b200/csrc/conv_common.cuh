@@ -44,6 +44,12 @@ __device__ __forceinline__ void pdl_enter() {
     asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+// The kernels that WRITE a packed handle's arrays (values, ids, order, the tensor path's weights and issue words) begin
+// with this instead: they wait like every other kernel but never let the next kernel start early.  The tensor-path
+// convolution relies on it: it fetches its weights before its own wait (they are constant while a network runs), which is
+// safe because whatever may still be writing them -- one of these kernels -- has completed before the convolution starts.
+__device__ __forceinline__ void pdl_enter_handle_writer() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
                               Args&&... args) {

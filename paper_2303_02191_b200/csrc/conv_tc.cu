@@ -729,9 +729,12 @@ conv_tc_kernel(const __grid_constant__ G g) {
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const unsigned tmem_base = *tmem_ptr_gen;
-    // Everything above (barriers, TMEM, descriptor prefetch) touched no tensor.  From here on the kernel reads x,
-    // the weights and the bias and writes y: wait until the kernels before it in the stream have completed.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Everything above (barriers, TMEM, descriptor prefetch) touched no tensor.  What depends on the kernels before this
+    // one in the stream -- the activations, the bias, the residual operand, and y, which they may still read -- is only
+    // touched behind a griddepcontrol.wait, which the activation producer and the epilogue warps execute at the top of
+    // their roles.  The weights and the issue words are not: they are constant while a network runs, and the kernels
+    // that write them (packing) never let a successor start early, so the weight producer and the MMA thread begin at
+    // once and the weight ring is full by the time the activations may be fetched.
 
     // Every role walks the same list of tiles: tile = blockIdx.x, + gridDim.x, ...  A tile is (image,
     // row band, filter tile) with the filter tile fastest, so CTAs working side by side read the same
@@ -742,6 +745,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
         // ---------------- TMA producer of the activations.  Issuing a bulk copy keeps its thread busy for some
         // hundred cycles whatever the size, so the activations and the weights have a producer thread each, and a
         // weight stage (G taps) is ONE copy.
+        asm volatile("griddepcontrol.wait;" ::: "memory");   // the activations come from the kernels before this one
         if (kF32 || lane == 0) {
             // (fp32: all 32 lanes walk the loop; lane 0 issues the copies, then the warp splits the block that arrived)
             bool ok = true;
@@ -1035,6 +1039,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
         __syncwarp();
     } else {
         // ---------------- epilogue: TMEM -> registers -> bias / activation -> NHWC global
+        asm volatile("griddepcontrol.wait;" ::: "memory");   // bias, residual and y belong to the stream's order
         const int quarter = warp & 3;      // TMEM lanes a warp may read: 32 * (warp id mod 4)
         const int sub = (warp - 2) >> 2;   // four warps share a lane quarter and take every fourth 32-column chunk
         bool ok = true;
@@ -1319,7 +1324,10 @@ bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count
                 // That is the measure for 3x3 layers of stride 1, whose tiles are bound by their instructions; the tiles of
                 // 1x1 and stride-2 layers are bound by what surrounds the instructions (fetches, barrier rounds, the
                 // epilogue) and do better with as many positions per tile as fit (measured both ways, layer by layer).
-                const double instr_cycles = pxm ? 128.0 * halves : (ksize == 3 && S == 1 && n_px / 2.0 < 128.0) ? (n_px / 2.0 > 76.0 ? n_px / 2.0 : 76.0) : 128.0;
+                // (Nor does it pay where the smaller tiles would still fit one wave: such layers gain more from tiles of 256
+                // positions cut along the channel blocks.)
+                const bool by_cycles = ksize == 3 && S == 1 && n_px / 2.0 < 128.0 && (grouped || tiles > sm_count);
+                const double instr_cycles = pxm ? 128.0 * halves : by_cycles ? (n_px / 2.0 > 76.0 ? n_px / 2.0 : 76.0) : 128.0;
                 const double eff = (double)(th * tw) / (2.0 * instr_cycles) * Ho / (double)((Ho + th - 1) / th * th) * Wo / (double)(tw * nseg);
                 const double halo_cost = (double)(th * tw) / (double)(rows_staged * wq);  // staged pixels that are outputs
                 // (fp32: a block feeds 108 instructions, twelve per tap, so a stage per tap costs little, while a single

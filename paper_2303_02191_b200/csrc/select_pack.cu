@@ -78,7 +78,7 @@ __global__ void __launch_bounds__(kSelThreads) pack_values_kernel(const T* __res
                                                                   V* __restrict__ val, uint8_t* pid_copy,
                                                                   V* __restrict__ wtc, int ksize, int Cin,
                                                                   rtoss_wtc_layout lay) {
-    rtoss_dev::pdl_enter();
+    rtoss_dev::pdl_enter_handle_writer();
     __shared__ __align__(16) T sw[kSelThreads * 9];
     const int64_t n_chunks = (n_kernels + kSelThreads - 1) / kSelThreads;
     for (int64_t chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
@@ -106,7 +106,7 @@ __global__ void __launch_bounds__(kOrderWarps * 32) pack_order_kernel(const uint
                                                                       uint32_t* __restrict__ bucket_off,
                                                                       const uint16_t* __restrict__ masks,
                                                                       unsigned long long* __restrict__ issue, int cb_log2) {
-    rtoss_dev::pdl_enter();
+    rtoss_dev::pdl_enter_handle_writer();
     __shared__ uint32_t fill_all[kOrderWarps][256];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ci = blockIdx.x * kOrderWarps + warp;
