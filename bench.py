@@ -613,7 +613,7 @@ def roofline_of(res, hbm_peak, tc_peak, peak_kind):
     dom["kernel_ms"] = t_top * 1e3
     dom["nnz_flop_per_launch"] = float(u_flops[top])
     dom["algorithmic_bytes_per_launch"] = float(u_bytes[top])
-    dom["traffic"] = ncu_traffic(res["name"], L["name"], res["ks"][members[0]]) if len(members) == 1 else None
+    dom["traffic"] = ncu_traffic(res["name"], L["name"] + ("+%d" % (len(members) - 1) if len(members) > 1 else ""), res["ks"][members[0]])
     # whole-model selection + packing: 36 B read per kernel (nine fp32 weights), k values + the id + the order entry written
     sp_bytes = float(sum(w["n_k"] * (36 + w["k"] * elem + (5 if w["ksize"] == 3 else 1)) for w in res["weights"]))
     sp = {"kernels": int(sum(w["n_k"] for w in res["weights"])), "launches": 2 if any(w["ksize"] == 3 for w in res["weights"]) else 1,
@@ -676,6 +676,9 @@ def run_gpu(args):
                           "divided by the sum of the cold-L2 CUDA-event times of the same launches; 'achieved' = frac x peak; "
                           "share of the roofline time that is tensor-bound: %.2f" % rf["tensor_share"],
             "sum_roofline_ms": rf["sum_roof_ms"], "sum_cold_kernel_ms": rf["sum_cold_ms"],
+            # the same roofline time (convolutions + the select/pack pass at the copy peak) against the graph-replayed step,
+            # where a launch's latency and prologue overlap the kernel before it; the cold pass pays them once per launch
+            "frac_in_step": (rf["sum_roof_ms"] + rf["select_pack"]["algorithmic_bytes"] / (hbm_peak * 1e9) * 1e3) / ms_per_step,
             "dominant_kernel": dom, "select_pack": rf["select_pack"],
             "notes": ["both convolution paths multiply the pruned taps as zeros: a tensor-bound layer cannot exceed k/9 of its "
                       "non-zero roofline",
