@@ -52,9 +52,11 @@ def workload_layers(name):
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of a workload's dominant kernel from one
 # ncu capture (caches flushed before every pass; the command is recorded with the capture's summary), valid
 # for the kernel source whose hash is recorded with it: once conv_tc.cu changes the figure is withheld (null).
-# 13.5 MB = the activations and the weights once; the 13.1 MB of outputs are still dirty in the 126 MB L2 when the
-# kernel ends, so the capture sees no write.
-NCU_TRAFFIC = {("layer128", "conv3x3_128", 3): (13506304, "1977b3266a0d51c6")}
+# The launch is the first layer of both RetinaNet towers on the five pyramid levels (ten convolutions), captured in
+# the retinanet_tower workload, which issues exactly that launch: 76.9 MB read (both towers' inputs and the weights
+# once) + 33.5 MB written (the other 40 MB of outputs are still dirty in the 126 MB L2 when the kernel ends).
+NCU_TRAFFIC = {("retinanet_b4", "cls_tower0.p3+9", 4): (110400500, "76876d07a422ba62"),
+               ("retinanet_tower", "cls_tower0.p3+9", 4): (110400500, "76876d07a422ba62")}
 
 
 def ncu_traffic(workload, layer, k):
