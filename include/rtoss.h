@@ -327,7 +327,7 @@ rtoss_status rtoss_conv1x1_pattern(rtoss_ctx* ctx, const rtoss_packed* p, const 
  * a detection tower is applied to (Section V evaluates RetinaNet, whose towers share their weights across five
  * levels), the two towers, the two 1x1 branches that open a block.  Results are those of the single calls.  Items
  * that qualify for the tensor path with more than 64 filters or a 3x3 kernel, and agree in kernel size, data type
- * and (3x3) stride, share ONE launch, up to ten at a time: small items then fill the SMs the large ones leave idle
+ * and (3x3) stride, share ONE launch, up to twenty at a time: small items then fill the SMs the large ones leave idle
  * instead of paying a launch each.  The other items run as single launches inside the same call.  *launches
  * (nullable) receives the number of kernel launches made.  Errors: those of the single calls; nothing is launched
  * when an argument check fails. */
@@ -338,6 +338,38 @@ typedef struct {
     rtoss_conv_desc desc;
 } rtoss_conv_item;
 rtoss_status rtoss_conv_group(rtoss_ctx* ctx, const rtoss_conv_item* items, int n, int* launches, void* cuda_stream);
+
+/* Convolutions that DEPEND on one another, in one launch: the three convolutions of a bottleneck block, a whole
+ * stage of such blocks, successive layers of the towers (Section V's models are chains of such layers; every launch
+ * between two of them costs its start-up and its drain).  items[0..n) are given in an order in which they could run
+ * one after the other, n <= 32.  after (n words, or NULL) says which earlier items an item has to wait for: bit j of
+ * after[i], j < i, when item i reads what item j writes, or writes where item j reads or writes.  NULL: the library
+ * derives exactly that from the address ranges of the items' inputs, outputs and residual operands
+ * (rtoss_chain_deps).  The result is that of the single calls issued in the given order.
+ *
+ * When all items qualify for a shared launch (tensor path, more than 64 filters or a 3x3 kernel, one data type, at
+ * most 20 items) they go out as ONE kernel: its CTAs walk the items' tiles in order and, before the first tile of an
+ * item, wait until all tiles of the items it depends on are written (a counter per item in device memory; the wait is
+ * bounded like every device-side wait, see rtoss_set_wait_limit, and reports through rtoss_device_status).  Items
+ * that do not depend on one another run side by side as in rtoss_conv_group.  Such a launch relies on all its CTAs
+ * (at most one per SM) being on the device together: while it runs, no other work may occupy SMs without end, and two
+ * such launches must not run concurrently on different streams.  Otherwise the items run as single launches in the
+ * given order.  *launches (nullable) receives the number of kernel launches made.
+ * Errors: RTOSS_ERR_INVALID_ARG (null items, n outside 1..32, a bit of after[i] at or above i) and those of the single
+ * calls; nothing is launched when an argument check fails. */
+rtoss_status rtoss_conv_chain(rtoss_ctx* ctx, const rtoss_conv_item* items, int n, const uint32_t* after, int* launches,
+                              void* cuda_stream);
+
+/* The dependencies rtoss_conv_chain derives when it is given none (host arithmetic on the pointers; nothing is
+ * launched, no device is touched): after[i] gets bit j, j < i, when the input or residual operand of item i overlaps
+ * the output buffer of item j, or the output buffer of item i overlaps the input, residual operand or output buffer
+ * of item j.  An output buffer counts with its whole pixel pitch (y_channel_stride), so two items that write disjoint
+ * channel slices of one buffer are ordered too.  n <= 32. */
+rtoss_status rtoss_chain_deps(const rtoss_conv_item* items, int n, uint32_t* after);
+/* The same rule on plain byte ranges: spans holds, per item, {x_lo, x_hi, y_lo, y_hi, r_lo, r_hi} (half-open ranges;
+ * an absent residual operand is an empty range).  RTOSS_ERR_INVALID_ARG for a null pointer, n outside 1..32 or a
+ * range whose end lies before its start. */
+rtoss_status rtoss_chain_deps_spans(const uint64_t* spans, int n, uint32_t* after);
 
 /* The tensor path (RTOSS_PATH_TENSOR, or RTOSS_PATH_AUTO when it applies) takes: NHWC, stride 1 or 2, io_dtype equal
  * to the packed dtype; bf16 / fp16 with Cin a multiple of 8, or fp32 with Cin a multiple of 4.  fp32 data is computed

@@ -31,7 +31,7 @@ SYMBOLS = [
     "rtoss_pattern_rank", "rtoss_pattern_table_derive",
     "rtoss_batch_create", "rtoss_batch_select_pack", "rtoss_batch_destroy",
     "rtoss_select_patterns_shared", "rtoss_conv_group", "rtoss_set_wait_limit", "rtoss_inject_lost_copy",
-    "rtoss_fma_plan3x3",
+    "rtoss_fma_plan3x3", "rtoss_conv_chain", "rtoss_chain_deps", "rtoss_chain_deps_spans",
 ]
 
 
@@ -106,6 +106,9 @@ def _load():
     lib.rtoss_conv_pattern_host.argtypes = [vp, vp, vp, vp, ctypes.POINTER(ConvDesc)]
     lib.rtoss_device_status.argtypes = [vp, ctypes.POINTER(ci)]
     lib.rtoss_conv_group.argtypes = [vp, ctypes.POINTER(ConvItem), ci, ctypes.POINTER(ci), vp]
+    lib.rtoss_conv_chain.argtypes = [vp, ctypes.POINTER(ConvItem), ci, ctypes.POINTER(ctypes.c_uint32), ctypes.POINTER(ci), vp]
+    lib.rtoss_chain_deps.argtypes = [ctypes.POINTER(ConvItem), ci, ctypes.POINTER(ctypes.c_uint32)]
+    lib.rtoss_chain_deps_spans.argtypes = [ctypes.POINTER(ctypes.c_uint64), ci, ctypes.POINTER(ctypes.c_uint32)]
     lib.rtoss_set_wait_limit.argtypes = [vp, ctypes.c_longlong]
     lib.rtoss_inject_lost_copy.argtypes = [vp]
     lib.rtoss_fma_plan3x3.argtypes = [ctypes.POINTER(ConvDesc), ci, ci, ci, ci, ctypes.POINTER(FmaPlan)]
@@ -215,6 +218,26 @@ def rtoss_fma_plan3x3(N, H, W, stride, layout, io_dtype, Cin, Cout, k, packed_dt
     if st != OK:
         raise RtossError(st, status_string(st))
     return out
+
+
+def rtoss_chain_deps(items):
+    """Which earlier items each conv_item(...) entry has to wait for, from the operands' address ranges -> list of masks."""
+    arr = (ConvItem * len(items))(*items)
+    out = (ctypes.c_uint32 * len(items))()
+    st = lib.rtoss_chain_deps(arr, len(items), out)
+    if st != OK:
+        raise RtossError(st, status_string(st))
+    return list(out)
+
+
+def rtoss_chain_deps_spans(spans):
+    """spans: per item (x_lo, x_hi, y_lo, y_hi, r_lo, r_hi) byte ranges -> list of masks (host arithmetic only)."""
+    flat = (ctypes.c_uint64 * (6 * len(spans)))(*[int(v) for sp in spans for v in sp])
+    out = (ctypes.c_uint32 * len(spans))()
+    st = lib.rtoss_chain_deps_spans(flat, len(spans), out)
+    if st != OK:
+        raise RtossError(st, status_string(st))
+    return list(out)
 
 
 def rtoss_prune_dense_static(w, ksize, masks, k, out=None):
@@ -371,6 +394,15 @@ class Context:
         arr = (ConvItem * len(items))(*items)
         n = ctypes.c_int(0)
         self._check(lib.rtoss_conv_group(self.h, arr, len(items), ctypes.byref(n), _stream()))
+        return n.value
+
+    def rtoss_conv_chain(self, items, after=None):
+        """items: conv_item(...) entries in an order in which they could run one after the other; after: per item the
+        bit mask of earlier items it waits for (None: derived from the operands' addresses) -> kernel launches made."""
+        arr = (ConvItem * len(items))(*items)
+        aft = None if after is None else (ctypes.c_uint32 * len(items))(*[int(a) for a in after])
+        n = ctypes.c_int(0)
+        self._check(lib.rtoss_conv_chain(self.h, arr, len(items), aft, ctypes.byref(n), _stream()))
         return n.value
 
     def rtoss_set_wait_limit(self, sm_cycles):

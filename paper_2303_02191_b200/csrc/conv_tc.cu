@@ -88,7 +88,8 @@ constexpr int kKBlock = 64;       // channels per staged block: 128 bytes of bf1
 constexpr int kRowBytes = 128;    // one padded pixel, one channel block
 constexpr long long kWaitCycles = 2000000000LL;  // about one second
 
-constexpr int kMaxProb = 10;      // convolutions one launch may carry
+constexpr int kMaxProb = 20;      // convolutions one launch may carry
+constexpr int kMaxTabs = 8;       // distinct position tables of a launch (problems of equal tile geometry share one)
 
 // One convolution of a launch.
 struct TcArgs {
@@ -118,6 +119,17 @@ struct TcArgs {
     int cb_ch, slab_ch;   // channels per staged block (128 bytes) and per instruction (32 bytes): 64 / 16 for 16-bit data, 32 / 8 for fp32
     int taps_real;        // 9 or 1; `taps` counts weight tiles per channel block: twice that for fp32 (heads, then remainders)
     int lo_off;           // fp32: byte offset of the remainders inside an activation stage
+    // The operand rings this problem runs with: NA activation stages of a_stage bytes from the start of the ring area, NB
+    // weight stages of b_stage bytes from sB_off.  Problems of one launch with the same `geo` share all five; where a
+    // CTA passes to a problem of another geometry its rings run empty first (see bar_switch in the kernel).
+    int NA, NB;
+    unsigned a_stage, b_stage, sB_off;
+    int geo;
+    int tab;              // which of the launch's position tables
+    // Dependent problems of one launch: bit j of dep_mask = problem j (earlier in the launch's order) must be complete
+    // -- all its outputs written -- before this one reads an activation or writes an output; done_target = arrivals
+    // on this problem's counter that make it complete (epilogue warps x CTAs that hold units of it).
+    unsigned dep_mask, done_target;
 };
 
 // A launch: up to NP convolutions sharing the CTA's rings (stage sizes are the largest any of them needs).  The struct
@@ -130,7 +142,10 @@ struct TcLaunchT {
     int* status;
     long long wait_cycles;    // limit of every wait
     int inject;               // test hook: 1 = the first weight copy of the launch is withheld (the wait for it must run out)
-    int a_stage_bytes, b_stage_bytes, NA, NB;  // stage sizes, activation stages, weight stages
+    int ring_bytes;           // the ring area: the most any problem's activation + weight stages take
+    int max_na, max_nb;       // most activation / weight stages any problem uses (barriers to set up)
+    int n_tabs;               // position tables
+    unsigned* done;           // dependent problems: kMaxProb completion counters + one exit counter, all zero between launches; else null
     int AS, acc_stride;                        // accumulator stages in TMEM and columns per stage
     int tmem_cols;
     TcArgs prob[NP];
@@ -138,7 +153,8 @@ struct TcLaunchT {
 };
 using TcLaunch1 = TcLaunchT<1>;
 using TcLaunchN = TcLaunchT<kMaxProb>;
-static_assert(sizeof(TcLaunchN) <= 8192, "kernel parameters: well inside the 32 KB a launch may carry");
+static_assert(sizeof(TcLaunchN) <= 16384, "kernel parameters: well inside the 32 KB a launch may carry");
+static_assert(kMaxProb <= 32, "dependencies are a 32-bit mask");
 
 __device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
 
@@ -649,17 +665,54 @@ __device__ __forceinline__ void epilogue_from_shares(unsigned buf, int KS, int r
     }
 }
 
-// Which problem a unit of the launch's list belongs to, and its index inside that problem.
+// Which problem a unit of the launch's list belongs to, and its index inside that problem.  A CTA's units ascend, so
+// the search goes on from the problem of its previous unit (`from`).
 template <bool kMulti, typename G>
-__device__ __forceinline__ int find_problem(const G& g, int unit, int& local) {
+__device__ __forceinline__ int find_problem(const G& g, int unit, int& local, int from = 0) {
     if (!kMulti) {   // a launch of one problem: the index is a compile-time constant
         local = unit;
         return 0;
     }
-    int pi = 0;
+    int pi = from;
     while (pi + 1 < g.n_prob && unit >= g.unit_end[pi]) ++pi;
     local = unit - (pi ? g.unit_end[pi - 1] : 0);
     return pi;
+}
+
+// A ring of stages with one "full" and one "empty" mbarrier per stage: position s and, per stage, the parity of the
+// phase its next use belongs to (bit i of par = stage i).  The parities are kept per stage because the problems of a
+// launch may run with different ring depths: the stages then do not all have the same number of uses behind them.
+struct Ring {
+    int s = 0;
+    unsigned par = 0;
+    __device__ __forceinline__ unsigned parity() const { return (par >> s) & 1u; }
+    __device__ __forceinline__ void advance(int n) {
+        par ^= 1u << s;
+        if (++s == n) s = 0;
+    }
+};
+
+// Dependent problems of one launch: waits (bounded) until every problem named in dep_mask has all its outputs written,
+// then orders this thread's coming bulk copies behind what it has seen.  The writers' side is at the end of the
+// epilogue's tile loop.
+template <typename G>
+__device__ __forceinline__ bool wait_deps(const G& g, unsigned dep_mask) {
+    const long long t0 = clock64();
+    while (dep_mask) {
+        const int j = __ffs((int)dep_mask) - 1;
+        dep_mask &= dep_mask - 1;
+        const unsigned target = g.prob[j].done_target;
+        for (;;) {
+            unsigned seen;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(g.done + j) : "memory");
+            if (seen >= target) break;
+            if (clock64() - t0 > g.wait_cycles) return false;
+            __nanosleep(100);
+        }
+    }
+    // the outputs were written with ordinary stores; the copies that fetch them go through the asynchronous proxy
+    asm volatile("fence.proxy.async;" ::: "memory");
+    return true;
 }
 
 template <typename T, typename G>
@@ -670,19 +723,22 @@ conv_tc_kernel(const __grid_constant__ G g) {
     extern __shared__ unsigned char smem_dyn[];
     // tiles need 1024-byte alignment for the 128-byte swizzle pattern
     const unsigned base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
-    const unsigned sA = base;                                        // [NA][a_stage_bytes]
-    const unsigned sB = sA + (unsigned)g.NA * g.a_stage_bytes;       // [NB][b_stage_bytes]
-    const unsigned sBar = sB + (unsigned)g.NB * g.b_stage_bytes;     // barriers, 8 bytes each
+    const unsigned sA = base;                                        // the ring area: a problem's [NA][a_stage], then its [NB][b_stage]
+    const unsigned sBar = sA + (unsigned)g.ring_bytes;               // barriers, 8 bytes each
     const unsigned bar_fullA = sBar, bar_emptyA = sBar + 8 * kMaxA;
     const unsigned bar_fullB = bar_emptyA + 8 * kMaxA, bar_emptyB = bar_fullB + 8 * kMaxB;
     const unsigned bar_accFull = bar_emptyB + 8 * kMaxB, bar_accEmpty = bar_accFull + 16;
     const unsigned bar_loFull = bar_accEmpty + 16;   // fp32: activation stage split into heads and remainders
-    const unsigned s_tmem_ptr = bar_loFull + 8 * kMaxA;
+    // A CTA passing from a problem to one of another ring geometry: the MMA thread commits here once everything it
+    // issued for the old problem has completed, i.e. has read its operands; both producers wait for that before they
+    // write the first stage of the new layout over the old one.
+    const unsigned bar_switch = bar_loFull + 8 * kMaxA;
+    const unsigned s_tmem_ptr = bar_switch + 16;   // (what follows needs 16-byte alignment)
     volatile unsigned* tmem_ptr_gen = reinterpret_cast<volatile unsigned*>(smem_dyn + (s_tmem_ptr - smem_u32(smem_dyn)));
     unsigned char* epi_patch = smem_dyn + (s_tmem_ptr + 16 - smem_u32(smem_dyn));  // [kEpiWarps][kPatchBytes], 16-byte aligned
-    uint2* pos_tab_all = reinterpret_cast<uint2*>(epi_patch + kEpiWarps * kPatchBytes);  // [n_prob][kMaxPx]
+    uint2* pos_tab_all = reinterpret_cast<uint2*>(epi_patch + kEpiWarps * kPatchBytes);  // [n_tabs][kMaxPx]
     const unsigned s_tab_all = s_tmem_ptr + 16 + kEpiWarps * kPatchBytes;                // the same, as a shared address
-    const unsigned s_res = s_tab_all + (unsigned)g.n_prob * kMaxPx * 8;   // [kEpiWarps][kResStage], present when a call has a residual operand
+    const unsigned s_res = s_tab_all + (unsigned)g.n_tabs * kMaxPx * 8;   // [kEpiWarps][kResStage], present when a call has a residual operand
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = g.unit_end[g.n_prob - 1];  // units of work over all problems: (tile, share of the channel blocks)
@@ -691,15 +747,16 @@ conv_tc_kernel(const __grid_constant__ G g) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < g.NA; ++i) {
+        for (int i = 0; i < g.max_na; ++i) {
             mbar_init(bar_fullA + 8 * i, 1);
             mbar_init(bar_emptyA + 8 * i, 1);
             mbar_init(bar_loFull + 8 * i, 1);
         }
-        for (int i = 0; i < g.NB; ++i) {
+        for (int i = 0; i < g.max_nb; ++i) {
             mbar_init(bar_fullB + 8 * i, 1);
             mbar_init(bar_emptyB + 8 * i, 1);
         }
+        mbar_init(bar_switch, 1);
         for (int i = 0; i < g.AS; ++i) {
             mbar_init(bar_accFull + 8 * i, 1);
             mbar_init(bar_accEmpty + 8 * i, kEpiWarps);
@@ -713,8 +770,10 @@ conv_tc_kernel(const __grid_constant__ G g) {
     // Where position p of a tile's list lies: the same for every tile (the tile's origin and the image's edges
     // come in per tile), so the epilogue looks it up instead of dividing.  {element offset from the tile's first
     // output, row << 16 | column}; positions that are no output (pitch padding, the list's tail) get 0xFFFFFFFF.
-    for (int q = threadIdx.x; q < g.n_prob * kMaxPx; q += kTcThreads) {
-        const TcArgs& a = g.prob[q / kMaxPx];
+    for (int q = threadIdx.x; q < g.n_tabs * kMaxPx; q += kTcThreads) {
+        int owner = 0;   // (any problem that uses the table describes it)
+        while (owner + 1 < g.n_prob && g.prob[owner].tab != q / kMaxPx) ++owner;
+        const TcArgs& a = g.prob[owner];
         const int p = q % kMaxPx;
         const int oyl = p / a.Wq, oxl = p - oyl * a.Wq;
         const bool is_out = p < a.N_px && oyl < a.TH && oxl < a.TW;
@@ -749,12 +808,27 @@ conv_tc_kernel(const __grid_constant__ G g) {
         if (kF32 || lane == 0) {
             // (fp32: all 32 lanes walk the loop; lane 0 issues the copies, then the warp splits the block that arrived)
             bool ok = true;
-            int sa = 0;
-            unsigned pa = 0;
+            Ring ra;
+            int pi = 0, cur_pi = -1;
+            unsigned n_sw = 0;   // geometry changes so far
             for (int unit = blockIdx.x; unit < n_tiles && ok; unit += gridDim.x) {
                 int local;
-                const int pi = find_problem<kMulti>(g, unit, local);
+                pi = find_problem<kMulti>(g, unit, local, pi);
                 const TcArgs& a = g.prob[pi];
+                if (kMulti && pi != cur_pi) {
+                    // another problem: if its rings are laid out differently, the old ones must have run empty; if it
+                    // depends on problems of this launch, they must be complete
+                    const bool regeo = cur_pi >= 0 && a.geo != g.prob[cur_pi].geo;
+                    if (lane == 0) {
+                        if (regeo) ok = mbar_wait(bar_switch, n_sw & 1u, g.wait_cycles);
+                        if (ok && a.dep_mask) ok = wait_deps(g, a.dep_mask);
+                    }
+                    if (regeo) {
+                        ++n_sw;
+                        ra.s = 0;
+                    }
+                    cur_pi = pi;
+                }
                 const int ks = local % a.KS;
                 int rest = local / a.KS / a.co_tiles;
                 const int tx = rest % a.tiles_x;
@@ -763,12 +837,14 @@ conv_tc_kernel(const __grid_constant__ G g) {
                 const int y0 = ty * a.TH, x0 = tx * a.TW;
                 const int cb_end = min(a.ncb, (ks + 1) * a.cb_per);
                 for (int cb = ks * a.cb_per; cb < cb_end; ++cb) {
+                    const int sa = ra.s;
+                    const unsigned pa = ra.parity();
                     if (lane == 0) {
-                        ok = mbar_wait(bar_emptyA + 8 * sa, pa ^ 1, g.wait_cycles);
+                        ok = ok && mbar_wait(bar_emptyA + 8 * sa, pa ^ 1, g.wait_cycles);
                         if (ok) {
                             mbar_expect_tx(bar_fullA + 8 * sa, a.a_tx_bytes * a.n_sub);
                             for (int sub = 0; sub < a.n_sub; ++sub)
-                                tma_load_4d(sA + sa * g.a_stage_bytes + sub * a.sub_bytes, &g.tmA[pi], cb * a.cb_ch, x0 * a.S + a.x_add[sub],
+                                tma_load_4d(sA + sa * a.a_stage + sub * a.sub_bytes, &g.tmA[pi], cb * a.cb_ch, x0 * a.S + a.x_add[sub],
                                             y0 * a.S + a.y_add[sub], n, bar_fullA + 8 * sa);
                         }
                     }
@@ -783,7 +859,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
                             ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
                         }
                         if (ok) {
-                            const unsigned src = sA + sa * g.a_stage_bytes, dst = src + (unsigned)a.lo_off;
+                            const unsigned src = sA + sa * a.a_stage, dst = src + (unsigned)a.lo_off;
                             const int n16 = (a.n_sub * a.sub_bytes) >> 4;
 #pragma unroll 4
                             for (int i = lane; i < n16; i += 32) {
@@ -803,10 +879,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
                         }
                     }
                     if (!ok) break;
-                    if (++sa == g.NA) {
-                        sa = 0;
-                        pa ^= 1;
-                    }
+                    ra.advance(a.NA);
                 }
             }
             if (!ok && lane == 0) atomicExch(g.status, 1);
@@ -816,28 +889,37 @@ conv_tc_kernel(const __grid_constant__ G g) {
         // ---------------- TMA producer of the weights: per tile and channel block, taps / G stages of G taps each
         if (lane == 0) {
             bool ok = true;
-            int sb = 0;
-            unsigned pb = 0;
+            Ring rb;
+            int pi = 0, cur_pi = -1;
+            unsigned n_sw = 0;
             for (int unit = blockIdx.x; unit < n_tiles && ok; unit += gridDim.x) {
                 int local;
-                const int pi = find_problem<kMulti>(g, unit, local);
+                pi = find_problem<kMulti>(g, unit, local, pi);
                 const TcArgs& a = g.prob[pi];
+                if (kMulti && pi != cur_pi) {
+                    if (cur_pi >= 0 && a.geo != g.prob[cur_pi].geo) {   // the old rings must have run empty
+                        ok = mbar_wait(bar_switch, n_sw & 1u, g.wait_cycles);
+                        if (!ok) break;
+                        ++n_sw;
+                        rb.s = 0;
+                    }
+                    cur_pi = pi;
+                }
+                const unsigned sB = sA + a.sB_off;
                 const int ks = local % a.KS, cot = (local / a.KS) % a.co_tiles;
                 const int co0 = cot * (a.pxm ? a.n_cols : kMTile);
                 const int cb_end = min(a.ncb, (ks + 1) * a.cb_per);
                 for (int cb = ks * a.cb_per; cb < cb_end && ok; ++cb) {
                     for (int t0 = 0; t0 < a.taps; t0 += a.G) {
-                        ok = mbar_wait(bar_emptyB + 8 * sb, pb ^ 1, g.wait_cycles);
+                        const int sb = rb.s;
+                        ok = mbar_wait(bar_emptyB + 8 * sb, rb.parity() ^ 1u, g.wait_cycles);
                         if (!ok) break;
                         // (failure-detection hook: the launch's very first weight copy is withheld, so the wait for it runs out)
                         if (!(g.inject == 1 && unit == (int)blockIdx.x && cb == ks * a.cb_per && t0 == 0)) {
                             mbar_expect_tx(bar_fullB + 8 * sb, a.b_tx_bytes * a.G);
-                            tma_load_3d(sB + sb * g.b_stage_bytes, &g.tmB[pi], cb * a.cb_ch, co0, t0, bar_fullB + 8 * sb);
+                            tma_load_3d(sB + sb * a.b_stage, &g.tmB[pi], cb * a.cb_ch, co0, t0, bar_fullB + 8 * sb);
                         }
-                        if (++sb == g.NB) {
-                            sb = 0;
-                            pb ^= 1;
-                        }
+                        rb.advance(a.NB);
                     }
                 }
             }
@@ -857,14 +939,15 @@ conv_tc_kernel(const __grid_constant__ G g) {
             bool ok = true;
             const unsigned long long d0 = make_sw128_desc(0);
             const unsigned desc_hi = (unsigned)(d0 >> 32), desc_lo0 = (unsigned)d0;
-            const unsigned astage16 = (unsigned)g.a_stage_bytes >> 4, bstage16 = (unsigned)g.b_stage_bytes >> 4;
             // per problem (recomputed when a tile belongs to another problem than the one before)
-            unsigned tap16[9], wtile16 = 0, idesc = 0, hi_cols = 0;
+            unsigned tap16[9], wtile16 = 0, idesc = 0, hi_cols = 0, astage16 = 0, bstage16 = 0, sB = 0;
+            int NA = 1, NB = 1;
             bool pxm = false, two = false, unrolled9 = false;
-            int cur_pi = -1;
+            int cur_pi = -1, pi = 0;
             const unsigned bar_rdyA = kF32 ? bar_loFull : bar_fullA;   // the barrier that says an activation stage may be read
-            int sa = 0, sb = 0, as = 0, n_done = 0;
-            unsigned pa = 0, pb = 0, pacc = 0;  // phase parities of the three rings
+            Ring ra, rb;
+            int as = 0, n_done = 0;
+            unsigned pacc = 0;                  // phase parity of the accumulator ring
             unsigned peek = 0;                  // what umma_block_peek saw of the stages now current
             auto mk = [desc_hi](unsigned lo) { return ((unsigned long long)desc_hi << 32) | lo; };
             // all instructions of one tap: the K slabs named by m4 (times two halves of positions with the positions as M)
@@ -890,10 +973,21 @@ conv_tc_kernel(const __grid_constant__ G g) {
             };
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++n_done) {
                 int local;
-                const int pi = find_problem<kMulti>(g, tile, local);
+                pi = find_problem<kMulti>(g, tile, local, pi);
                 const TcArgs& a = g.prob[pi];
                 if (pi != cur_pi) {
+                    if (kMulti && cur_pi >= 0 && a.geo != g.prob[cur_pi].geo) {
+                        // rings of another layout: the producers may write them once everything issued so far has read its operands
+                        umma_commit(bar_switch);
+                        ra.s = rb.s = 0;
+                        peek = 0;
+                    }
                     cur_pi = pi;
+                    astage16 = a.a_stage >> 4;
+                    bstage16 = a.b_stage >> 4;
+                    sB = sA + a.sB_off;
+                    NA = a.NA;
+                    NB = a.NB;
 #pragma unroll
                     for (int t = 0; t < 9; ++t) tap16[t] = (unsigned)(a.tap_sub[t] * a.sub_bytes + a.tap_shift[t] * kRowBytes) >> 4;
                     wtile16 = (unsigned)(a.w_rows * kRowBytes) >> 4;
@@ -918,13 +1012,17 @@ conv_tc_kernel(const __grid_constant__ G g) {
                     // 32-byte slabs of this block that hold channels (the rest of the 128 bytes is TMA zero fill)
                     const int nk4 = left >= a.cb_ch ? 4 : (left + a.slab_ch - 1) / a.slab_ch;
                     const unsigned nkmask = (1u << nk4) - 1u;
+                    const int sa = ra.s;
                     if (a.taps == 1) {
-                        if (!(peek & 1u)) ok = mbar_wait(bar_rdyA + 8 * sa, pa, g.wait_cycles);
-                        if (ok && !(peek & 2u)) ok = mbar_wait(bar_fullB + 8 * sb, pb, g.wait_cycles);
+                        const int sb = rb.s;
+                        if (!(peek & 1u)) ok = mbar_wait(bar_rdyA + 8 * sa, ra.parity(), g.wait_cycles);
+                        if (ok && !(peek & 2u)) ok = mbar_wait(bar_fullB + 8 * sb, rb.parity(), g.wait_cycles);
                         if (!ok) break;
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                        const int sa_n = sa + 1 == g.NA ? 0 : sa + 1, sb_n = sb + 1 == g.NB ? 0 : sb + 1;
-                        const unsigned pa_n = sa_n ? pa : pa ^ 1, pb_n = sb_n ? pb : pb ^ 1;
+                        ra.advance(NA);   // now at the next stages, which the instruction below looks at
+                        rb.advance(NB);
+                        const int sa_n = ra.s, sb_n = rb.s;
+                        const unsigned pa_n = ra.parity(), pb_n = rb.parity();
                         const unsigned wl0 = desc_lo0 + (sB >> 4) + (unsigned)sb * bstage16;
                         const unsigned xl0 = desc_lo0 + (sA >> 4) + (unsigned)sa * astage16;
                         if (!pxm) {
@@ -948,29 +1046,30 @@ conv_tc_kernel(const __grid_constant__ G g) {
                         acc = 1;
                         umma_commit(bar_emptyB + 8 * sb);
                         umma_commit(bar_emptyA + 8 * sa);
-                        sa = sa_n, pa = pa_n, sb = sb_n, pb = pb_n;
                         continue;
                     }
                     const unsigned long long bits_n = (iss && cb + 1 < cb_end) ? __ldg(iss + cb + 1) : ~0ull;
-                    if (!(peek & 1u)) ok = mbar_wait(bar_rdyA + 8 * sa, pa, g.wait_cycles);   // (peek stays 0 on the paths that do not look ahead)
+                    if (!(peek & 1u)) ok = mbar_wait(bar_rdyA + 8 * sa, ra.parity(), g.wait_cycles);   // (peek stays 0 on the paths that do not look ahead)
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const unsigned xl0 = desc_lo0 + (sA >> 4) + (unsigned)sa * astage16;
+                    ra.advance(NA);   // (sa stays this block's stage; ra is at the next one, which the look ahead reads)
                     if (unrolled9) {
-                        const int sa_n = sa + 1 == g.NA ? 0 : sa + 1;
-                        const unsigned pa_n = sa_n ? pa : pa ^ 1;
+                        const int sa_n = ra.s;
+                        const unsigned pa_n = ra.parity();
 #pragma unroll
                         for (int s3 = 0; s3 < 3; ++s3) {
-                            if (!(peek & 2u)) ok = ok && mbar_wait(bar_fullB + 8 * sb, pb, g.wait_cycles);
+                            const int sb = rb.s;
+                            if (!(peek & 2u)) ok = ok && mbar_wait(bar_fullB + 8 * sb, rb.parity(), g.wait_cycles);
                             if (ok) {
                                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                                 const unsigned wl0 = desc_lo0 + (sB >> 4) + (unsigned)sb * bstage16;
                                 const unsigned m_first = (unsigned)(bits >> (12 * s3)) & nkmask;
+                                rb.advance(NB);
                                 if (!pxm) {
                                     // the first tap of the stage goes out together with a look at the next stages
-                                    const int sb_n = sb + 1 == g.NB ? 0 : sb + 1;
                                     peek = umma_block_peek<kF32>(d_base, mk(wl0), mk(xl0 + tap16[s3 * 3]), idesc, acc, m_first,
-                                                           bar_rdyA + 8 * sa_n, pa_n, bar_fullB + 8 * sb_n, sb_n ? pb : pb ^ 1);
+                                                           bar_rdyA + 8 * sa_n, pa_n, bar_fullB + 8 * rb.s, rb.parity());
                                     if (m_first) acc = 1;
 #pragma unroll
                                     for (int i = 1; i < 3; ++i)
@@ -983,15 +1082,12 @@ conv_tc_kernel(const __grid_constant__ G g) {
                                                   (unsigned)(bits >> (12 * s3 + 4 * i)) & nkmask, acc);
                                 }
                                 umma_commit(bar_emptyB + 8 * sb);  // this weight stage may be refilled once the MMAs have read it
-                                if (++sb == g.NB) {
-                                    sb = 0;
-                                    pb ^= 1;
-                                }
                             }
                         }
                     } else {
                         for (int t0 = 0; t0 < a.taps && ok; t0 += a.G) {
-                            ok = mbar_wait(bar_fullB + 8 * sb, pb, g.wait_cycles);
+                            const int sb = rb.s;
+                            ok = mbar_wait(bar_fullB + 8 * sb, rb.parity(), g.wait_cycles);
                             if (!ok) break;
                             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                             const unsigned wl0 = desc_lo0 + (sB >> 4) + (unsigned)sb * bstage16;
@@ -1006,17 +1102,10 @@ conv_tc_kernel(const __grid_constant__ G g) {
                                 if (kF32 && v < a.taps_real) issue_tap(d_base, wl0 + i * wtile16, xl0 + off + ((unsigned)a.lo_off >> 4), m4, acc);
                             }
                             umma_commit(bar_emptyB + 8 * sb);
-                            if (++sb == g.NB) {
-                                sb = 0;
-                                pb ^= 1;
-                            }
+                            rb.advance(NB);
                         }
                     }
                     if (ok) umma_commit(bar_emptyA + 8 * sa);
-                    if (++sa == g.NA) {
-                        sa = 0;
-                        pa ^= 1;
-                    }
                     bits = bits_n;
                 }
                 if (ok) umma_commit(bar_accFull + 8 * as);
@@ -1102,13 +1191,14 @@ conv_tc_kernel(const __grid_constant__ G g) {
             }
             gt = -1;   // (done: the loop below does not run)
         }
+        int pi = 0;
         for (int tile = blockIdx.x; gt >= 0 && tile < n_tiles && ok; tile += gridDim.x, ++gt) {
             int local;
-            const int pi = find_problem<kMulti>(g, tile, local);
+            pi = find_problem<kMulti>(g, tile, local, pi);
             const TcArgs& a = g.prob[pi];
             T* __restrict__ yg = reinterpret_cast<T*>(a.y);
-            const uint2* pos_tab = pos_tab_all + pi * kMaxPx;
-            const unsigned s_tab = s_tab_all + (unsigned)pi * kMaxPx * 8;
+            const uint2* pos_tab = pos_tab_all + a.tab * kMaxPx;
+            const unsigned s_tab = s_tab_all + (unsigned)a.tab * kMaxPx * 8;
             int rest = local / a.KS;   // a unit is (tile proper, share of the channel blocks)
             const int cot = rest % a.co_tiles;
             rest /= a.co_tiles;
@@ -1208,7 +1298,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
                         const uint2 e = pos_tab[c0 + j];
                         const bool in_img = co_ok && (e.y >> 16) < ry && (e.y & 0xFFFFu) < rx;
                         float v = __uint_as_float(r[j]) + bv;
-                        if (rb && in_img && !post) v = to_f32<T>(from_f32<T>(v)) + to_f32<T>(rb[e.x + lane]);   // round, then add the residual
+                        if (rb && in_img && !post) v = to_f32<T>(from_f32<T>(v)) + to_f32<T>(__ldcg(rb + e.x + lane));   // round, then add the residual
                         if (a.act == RTOSS_ACT_RELU) v = fmaxf(v, 0.f);
                         if (a.act == RTOSS_ACT_SILU) {
                             if (kF32) {
@@ -1219,7 +1309,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
                                 v = v * fmaf(0.5f, th, 0.5f);
                             }
                         }
-                        if (rb && in_img && post) v = to_f32<T>(from_f32<T>(v)) + to_f32<T>(rb[e.x + lane]);   // behind the activation
+                        if (rb && in_img && post) v = to_f32<T>(from_f32<T>(v)) + to_f32<T>(__ldcg(rb + e.x + lane));   // behind the activation
                         if (co_ok && (e.y >> 16) < ry && (e.y & 0xFFFFu) < rx) yb[e.x + lane] = from_f32<T>(v);
                     }
                 }
@@ -1228,6 +1318,14 @@ conv_tc_kernel(const __grid_constant__ G g) {
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_accEmpty + 8 * as) : "memory");
+            if (kMulti && g.done && tile + (int)gridDim.x >= g.unit_end[pi]) {
+                // This was the CTA's last tile of the problem: the warp reports its share of the outputs written.  The
+                // lanes' stores are ordered before lane 0's fence by the __syncwarp above, the fence before the count.
+                if (lane == 0) {
+                    __threadfence();
+                    atomicAdd(g.done + pi, 1u);
+                }
+            }
         }
         if (!ok && lane == 0) atomicExch(g.status, 3);
     }
@@ -1241,6 +1339,14 @@ conv_tc_kernel(const __grid_constant__ G g) {
     if (warp == 1) {
         __syncwarp();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(g.tmem_cols) : "memory");
+    }
+    if (kMulti && g.done && threadIdx.x == 0) {
+        // The completion counters go back to zero for the next launch: by the last CTA to get here, when no CTA of this
+        // launch reads them any more.
+        __threadfence();
+        if (atomicAdd(g.done + kMaxProb, 1u) == gridDim.x - 1) {
+            for (int i = 0; i <= kMaxProb; ++i) g.done[i] = 0u;
+        }
     }
 }
 
@@ -1282,14 +1388,14 @@ struct TcPlan {
 // The plan picks TH, the column segment TW (images wider than a TMA box are cut into segments), the
 // ring depths, and how many taps share a weight stage.
 bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count, bool pxm, int w_rows, bool resid, TcPlan* out,
-             int n_prob = 1, bool f32 = false, int force_G = 0) {
+             int n_prob = 1, bool f32 = false, int force_G = 0, int n_tabs = 1) {
     const int halo = ksize == 3 ? (S == 1 ? 2 : 1) : 0;
     const int n_sub = (ksize == 3 && S == 2) ? 4 : 1;
     const int max_pitch = S == 1 ? 256 : 128;  // TMA box: at most 256 elements traversed per dimension
     const int fixed = 1024 /*alignment slack*/ + 512 /*barriers*/ + kEpiWarps * kPatchBytes /*epilogue patches*/ +
-                      n_prob * kMaxPx * 8 /*position tables*/ + (resid ? kEpiWarps * kResStage : 0) /*staging of the residual operand*/;
+                      n_tabs * kMaxPx * 8 /*position tables*/ + (resid ? kEpiWarps * kResStage : 0) /*staging of the residual operand*/;
     const int cap = 227 * 1024 - 64;
-    const bool grouped = n_prob > 1;   // one of several problems of a launch: the launch as a whole fills the SMs
+    const bool grouped = n_prob > 1;   // one of several problems that run side by side: together they fill the SMs
     double best = -1;
     for (int nseg = 1; nseg <= 16; ++nseg) {
         const int tw = (Wo + nseg - 1) / nseg;
@@ -1366,7 +1472,7 @@ struct ProbPlan {
 // Geometry, operand roles and TMA descriptors of one convolution.  The rings' depths and the split along K are the
 // launch's business (the caller's).  Returns a cudaError_t as int.
 int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y, const rtoss_conv_desc* d, int n_prob, int sms,
-                  TcArgs* out, ProbPlan* pp, CUtensorMap* tmA_out, CUtensorMap* tmB_out, int force_G = 0) {
+                  TcArgs* out, ProbPlan* pp, CUtensorMap* tmA_out, CUtensorMap* tmB_out, int force_G = 0, int n_tabs = 1) {
     const int taps = p->ksize == 3 ? 9 : 1;
     const int S = d->stride;
     const int Ho = (d->H - 1) / S + 1, Wo = (d->W - 1) / S + 1;
@@ -1378,7 +1484,7 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
     const bool f32 = p->dtype == RTOSS_F32;
     const int esize = f32 ? 4 : 2;
     if (!plan_tc(d->N, Ho, Wo, p->ksize, S, (p->Cout + kMTile - 1) / kMTile, sms, pxm, w_rows, d->residual_dev != nullptr, &plan, n_prob, f32,
-                 force_G))
+                 force_G, n_tabs))
         return (int)cudaErrorInvalidConfiguration;
 
     TcArgs& a = *out;
@@ -1571,10 +1677,16 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     TcArgs& a = g.prob[0];
     const TcPlan& plan = pp.plan;
     const bool f32 = p->dtype == RTOSS_F32;
-    g.a_stage_bytes = pp.a_stage_bytes;
-    g.b_stage_bytes = pp.b_stage_bytes;
-    g.NA = plan.NA;
-    g.NB = plan.NB;
+    a.NA = plan.NA;
+    a.NB = plan.NB;
+    a.a_stage = (unsigned)pp.a_stage_bytes;
+    a.b_stage = (unsigned)pp.b_stage_bytes;
+    a.sB_off = (unsigned)plan.NA * a.a_stage;
+    g.ring_bytes = (int)(a.sB_off + (unsigned)plan.NB * a.b_stage);
+    g.max_na = plan.NA;
+    g.max_nb = plan.NB;
+    g.n_tabs = 1;
+    g.done = nullptr;
     g.acc_stride = pp.acc_cols;
     launch_common(ctx, &g);
     // Split K where the layer has too few tiles for the SMs and several channel blocks: a tile's MMAs are one serial
@@ -1595,7 +1707,7 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
             while (want > 1) {
                 const int cb_per = (a.ncb + want - 1) / want, ks = (a.ncb + cb_per - 1) / cb_per;
                 const int n_chunks = (plan.N_px + 31) / 32, n_lc = (n_chunks + ks - 1) / ks;
-                if (ks > 1 && ks * n_lc <= 2 * n_lc_max && (size_t)ks * n_lc * 16384 <= (size_t)g.NA * g.a_stage_bytes + (size_t)g.NB * g.b_stage_bytes) {
+                if (ks > 1 && ks * n_lc <= 2 * n_lc_max && (size_t)ks * n_lc * 16384 <= (size_t)g.ring_bytes) {
                     a.cb_per = cb_per;
                     a.KS = ks;
                     break;
@@ -1638,91 +1750,172 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     return (int)le;
 }
 
-// Several independent convolutions in ONE launch.  All must qualify for the tensor path with the filters on M, share the
-// kernel size, the stride class and the data type (then the rings of a CTA fit them all), and be at most kMaxProb.
+// Several convolutions in ONE launch: independent ones side by side, dependent ones one behind the other.
+//
+// after[i] (null: none depends on another) has bit j set when convolution i must see convolution j (j < i) complete:
+// it reads what j writes, or overwrites what j reads or writes.  The kernel then keeps the CTAs that reach a tile of
+// i waiting until every CTA has reported its tiles of j done (a counter per problem in device memory; the waits are
+// bounded like all others).  That is only sound when all CTAs of the launch are on the device together: the grid is at
+// most one CTA per SM, and nothing else may hold SMs forever while such a launch runs.
+//
+// All convolutions must qualify for the tensor path with the filters on M and share the data type; at most kMaxProb.
+// They are sorted into levels (a convolution's level is one more than the highest level it waits for); the
+// convolutions of a level with the same kernel size (and stride class, for 3x3) share one ring layout, planned as the
+// grouped launches always were; a CTA that passes from one layout to another lets its rings run empty in between.
 // Returns 0 after a launch, -1 when the set cannot share a launch (nothing was launched: the caller runs the calls
-// one by one), or a cudaError_t.
-int rtoss_launch_conv_tc_group(const rtoss_ctx* ctx, int n, const rtoss_packed* const* ps, const void* const* xs, void* const* ys,
-                               const rtoss_conv_desc* const* ds, void* stream) {
+// one by one, in order), or a cudaError_t.
+int rtoss_launch_conv_tc_chain(const rtoss_ctx* ctx, int n, const rtoss_packed* const* ps, const void* const* xs, void* const* ys,
+                               const rtoss_conv_desc* const* ds, const uint32_t* after, void* stream) {
     if (n < 2 || n > kMaxProb || ctx->inject_next) return -1;
     const int sms = ctx->sm_count > 0 ? ctx->sm_count : 148;
+    bool resid = false, chained = false;
+    int level[kMaxProb], cls[kMaxProb];
     for (int i = 0; i < n; ++i) {
-        if (use_pxm(ps[i]) || ps[i]->ksize != ps[0]->ksize || ps[i]->dtype != ps[0]->dtype) return -1;
-        if (ps[i]->ksize == 3 && ds[i]->stride != ds[0]->stride) return -1;   // (3x3: stride 2 stages four sub-tiles per block)
+        if (use_pxm(ps[i]) || ps[i]->dtype != ps[0]->dtype) return -1;
         if (!rtoss_tc_eligible(ps[i], ds[i], xs[i], ys[i])) return -1;
+        resid = resid || ds[i]->residual_dev != nullptr;
+        level[i] = 0;
+        if (after && after[i]) {
+            if (i == 0 || (after[i] >> i)) return (int)cudaErrorInvalidValue;   // only earlier convolutions may be named
+            chained = true;
+            for (int j = 0; j < i; ++j)
+                if ((after[i] >> j) & 1u) level[i] = level[j] + 1 > level[i] ? level[j] + 1 : level[i];
+        }
+        cls[i] = ps[i]->ksize == 3 ? 3 + ds[i]->stride : 1;   // 1x1 (any stride), 3x3 stride 1, 3x3 stride 2
     }
+    if (chained && !ctx->chain_done) return -1;
     static thread_local TcLaunchN g;
+    static thread_local TcArgs args[kMaxProb];
+    static thread_local CUtensorMap mapA[kMaxProb], mapB[kMaxProb];
     ProbPlan pp[kMaxProb];
-    bool resid = false;
-    for (int i = 0; i < n; ++i) resid = resid || ds[i]->residual_dev != nullptr;
-    g.n_prob = n;
-    int a_max = 0, acc_max = 0, b_bytes = 0, units = 0;
     long n_tiles[kMaxProb];
-    // every problem is planned on its own first; where they disagree on the taps per weight stage, all are planned again
-    // with the smallest (a stage per tap fits whatever fits three)
-    int force_G = 0;
-    for (int pass = 0; pass < 2; ++pass) {
-        bool agree = true;
-        int g_min = 9;
-        a_max = acc_max = 0;
-        for (int i = 0; i < n; ++i) {
-            // (planned with the launch's fixed shared memory: all position tables, the residual staging if any needs it)
-            rtoss_conv_desc dd = *ds[i];
-            static const int dummy = 0;
-            if (resid && !dd.residual_dev) dd.residual_dev = &dummy;   // only the plan's memory budget looks at it here
-            TcArgs tmp;
-            int e = build_problem(ctx, ps[i], xs[i], ys[i], &dd, n, sms, &tmp, &pp[i], &g.tmA[i], &g.tmB[i], force_G);
-            if (e == (int)cudaErrorInvalidConfiguration) return -1;
-            if (e) return e;
-            tmp.resid = ds[i]->residual_dev;
-            tmp.resid_post = (ds[i]->residual_dev && ds[i]->residual_after_act) ? 1 : 0;
-            g.prob[i] = tmp;
-            if (i == 0) b_bytes = pp[i].b_stage_bytes;
-            if (tmp.n_sub != g.prob[0].n_sub) return -1;
-            if (pp[i].b_stage_bytes != b_bytes || tmp.G != g.prob[0].G) agree = false;
-            if (tmp.G < g_min) g_min = tmp.G;
-            if (pp[i].a_stage_bytes > a_max) a_max = pp[i].a_stage_bytes;
-            if (pp[i].acc_cols > acc_max) acc_max = pp[i].acc_cols;
-            n_tiles[i] = (long)tmp.N * tmp.tiles_y * tmp.tiles_x * tmp.co_tiles;
-        }
-        if (agree) break;
-        if (pass == 1) return -1;
-        force_G = g_min;
-    }
-    // insertion sort of the problems by falling tile count (stable), applied to every per-problem array
-    for (int i = 1; i < n; ++i)
-        for (int j = i; j > 0 && n_tiles[j] > n_tiles[j - 1]; --j) {
-            std::swap(n_tiles[j], n_tiles[j - 1]);
-            std::swap(g.prob[j], g.prob[j - 1]);
-            std::swap(pp[j], pp[j - 1]);
-            std::swap(g.tmA[j], g.tmA[j - 1]);
-            std::swap(g.tmB[j], g.tmB[j - 1]);
-        }
-    for (int i = 0; i < n; ++i) {
-        if (units + n_tiles[i] > 0x3FFFFFFF) return -1;
-        units += (int)n_tiles[i];
-        g.unit_end[i] = units;
-    }
-    // the rings every problem fits into
-    const int fixed = 1024 + 512 + kEpiWarps * kPatchBytes + n * kMaxPx * 8 + (resid ? kEpiWarps * kResStage : 0);
+    int geo_of[kMaxProb];
+    struct Geo {
+        int a, b, na, nb;
+    } geos[kMaxProb];
+    int n_geo = 0;
+    const int fixed = 1024 + 512 + kEpiWarps * kPatchBytes + kMaxTabs * kMaxPx * 8 + (resid ? kEpiWarps * kResStage : 0);
     const int cap = 227 * 1024 - 64;
-    int na = (cap - fixed - 2 * b_bytes) / a_max;
-    if (na > kMaxA) na = kMaxA;
-    if (na > 2 && ps[0]->ksize == 3) na = 2;
-    if (na < 1) return -1;
-    int nb = (cap - fixed - na * a_max) / b_bytes;
-    if (nb > kMaxB) nb = kMaxB;
-    if (nb < 2) return -1;
-    g.a_stage_bytes = a_max;
-    g.b_stage_bytes = b_bytes;
-    g.NA = na;
-    g.NB = nb;
+    bool seen[kMaxProb] = {};
+    int acc_max = 0;
+    for (int i0 = 0; i0 < n; ++i0) {
+        if (seen[i0]) continue;
+        // the set of this convolution: same level, same class
+        int set[kMaxProb], m = 0;
+        for (int j = i0; j < n; ++j)
+            if (!seen[j] && level[j] == level[i0] && cls[j] == cls[i0]) set[m++] = j, seen[j] = true;
+        // every problem is planned on its own first; where they disagree on the taps per weight stage, all are planned
+        // again with the smallest (a stage per tap fits whatever fits three)
+        int force_G = 0, a_max = 0, b_bytes = 0;
+        for (int pass = 0; pass < 2; ++pass) {
+            bool agree = true;
+            int g_min = 9;
+            a_max = 0;
+            for (int q = 0; q < m; ++q) {
+                const int i = set[q];
+                // (planned with the launch's fixed shared memory: all position tables, the residual staging if any needs it)
+                rtoss_conv_desc dd = *ds[i];
+                static const int dummy = 0;
+                if (resid && !dd.residual_dev) dd.residual_dev = &dummy;   // only the plan's memory budget looks at it here
+                int e = build_problem(ctx, ps[i], xs[i], ys[i], &dd, m, sms, &args[i], &pp[i], &mapA[i], &mapB[i], force_G, kMaxTabs);
+                if (e == (int)cudaErrorInvalidConfiguration) return -1;
+                if (e) return e;
+                args[i].resid = ds[i]->residual_dev;
+                args[i].resid_post = (ds[i]->residual_dev && ds[i]->residual_after_act) ? 1 : 0;
+                if (q == 0) b_bytes = pp[i].b_stage_bytes;
+                if (pp[i].b_stage_bytes != b_bytes || args[i].G != args[set[0]].G) agree = false;
+                if (args[i].G < g_min) g_min = args[i].G;
+                if (pp[i].a_stage_bytes > a_max) a_max = pp[i].a_stage_bytes;
+                if (pp[i].acc_cols > acc_max) acc_max = pp[i].acc_cols;
+                n_tiles[i] = (long)args[i].N * args[i].tiles_y * args[i].tiles_x * args[i].co_tiles;
+            }
+            if (agree) break;
+            if (pass == 1) return -1;
+            force_G = g_min;
+        }
+        // the rings every problem of the set fits into
+        int na = (cap - fixed - 2 * b_bytes) / a_max;
+        if (na > kMaxA) na = kMaxA;
+        if (na > 2 && ps[i0]->ksize == 3) na = 2;
+        if (na < 1) return -1;
+        int nb = (cap - fixed - na * a_max) / b_bytes;
+        if (nb > kMaxB) nb = kMaxB;
+        if (nb < 2) return -1;
+        int gi = 0;
+        while (gi < n_geo && !(geos[gi].a == a_max && geos[gi].b == b_bytes && geos[gi].na == na && geos[gi].nb == nb)) ++gi;
+        if (gi == n_geo) geos[n_geo++] = Geo{a_max, b_bytes, na, nb};
+        for (int q = 0; q < m; ++q) geo_of[set[q]] = gi;
+    }
+    // the launch's order: by level, inside a level by ring layout, then by falling tile count (stable)
+    int order[kMaxProb];
+    for (int i = 0; i < n; ++i) order[i] = i;
+    for (int i = 1; i < n; ++i)
+        for (int j = i; j > 0; --j) {
+            const int u = order[j], v = order[j - 1];
+            const bool before = level[u] != level[v] ? level[u] < level[v] : geo_of[u] != geo_of[v] ? geo_of[u] < geo_of[v] : n_tiles[u] > n_tiles[v];
+            if (!before) break;
+            std::swap(order[j], order[j - 1]);
+        }
+    int where[kMaxProb];   // position of convolution i in the launch
+    for (int k = 0; k < n; ++k) where[order[k]] = k;
+    g.n_prob = n;
+    g.n_tabs = 0;
+    g.ring_bytes = 0;
+    g.max_na = g.max_nb = 1;
+    long units = 0;
+    for (int k = 0; k < n; ++k) {
+        const int i = order[k];
+        TcArgs& a = g.prob[k];
+        a = args[i];
+        g.tmA[k] = mapA[i];
+        g.tmB[k] = mapB[i];
+        const Geo& ge = geos[geo_of[i]];
+        a.NA = ge.na;
+        a.NB = ge.nb;
+        a.a_stage = (unsigned)ge.a;
+        a.b_stage = (unsigned)ge.b;
+        a.sB_off = (unsigned)ge.na * (unsigned)ge.a;
+        a.geo = geo_of[i];
+        const int ring = ge.na * ge.a + ge.nb * ge.b;
+        if (ring > g.ring_bytes) g.ring_bytes = ring;
+        if (ge.na > g.max_na) g.max_na = ge.na;
+        if (ge.nb > g.max_nb) g.max_nb = ge.nb;
+        // position table: shared with an earlier problem of the same tile geometry and output pitch
+        a.tab = -1;
+        for (int q = 0; q < k && a.tab < 0; ++q) {
+            const TcArgs& b = g.prob[q];
+            if (b.Wq == a.Wq && b.TH == a.TH && b.TW == a.TW && b.N_px == a.N_px && b.Wo == a.Wo && b.y_c_stride == a.y_c_stride) a.tab = b.tab;
+        }
+        if (a.tab < 0) {
+            if (g.n_tabs == kMaxTabs) return -1;
+            a.tab = g.n_tabs++;
+        }
+        a.dep_mask = 0;
+        if (after)
+            for (int j = 0; j < i; ++j)
+                if ((after[i] >> j) & 1u) a.dep_mask |= 1u << where[j];
+        units += n_tiles[i];
+        if (units > 0x3FFFFFFF) return -1;
+        g.unit_end[k] = (int)units;
+    }
+    const int grid_n = (int)(units < sms ? units : sms);
+    for (int k = 0; k < n; ++k) {
+        const long mine = n_tiles[order[k]];
+        g.prob[k].done_target = (unsigned)((mine < grid_n ? mine : grid_n) * kEpiWarps);
+    }
+    g.done = nullptr;
+    if (chained) {
+        // a block of counters of the context, taken in turn (launches that share a block must follow one another in a stream)
+        g.done = ctx->chain_done + (size_t)(ctx->chain_next % RTOSS_CHAIN_SLOTS) * RTOSS_CHAIN_SLOT_WORDS;
+        ctx->chain_next = (ctx->chain_next + 1) % RTOSS_CHAIN_SLOTS;
+    }
     g.acc_stride = acc_max;
     launch_common(ctx, &g);
     if (g.tmem_cols > 512) return -1;
-    const size_t smem_need = (size_t)fixed + (size_t)na * a_max + (size_t)nb * b_bytes;
+    const size_t smem_need = (size_t)fixed + (size_t)g.ring_bytes;
+    if (smem_need > (size_t)cap) return -1;
     const size_t smem = smem_need > 116 * 1024 ? smem_need : 116 * 1024;
-    dim3 grid((unsigned)(units < sms ? units : sms));
+    dim3 grid((unsigned)grid_n);
     int e = ensure_smem_attr(ctx);
     if (e) return e;
     const bool bf = ps[0]->dtype == RTOSS_BF16, f32 = ps[0]->dtype == RTOSS_F32;
@@ -1731,3 +1924,15 @@ int rtoss_launch_conv_tc_group(const rtoss_ctx* ctx, int n, const rtoss_packed* 
                           : rtoss_dev::launch_pdl(conv_tc_kernel<__half, TcLaunchN>, grid, kTcThreads, smem, (cudaStream_t)stream, 1, g);
     return (int)le;
 }
+
+// Several independent convolutions of one class (kernel size, stride class, data type) in one launch.
+int rtoss_launch_conv_tc_group(const rtoss_ctx* ctx, int n, const rtoss_packed* const* ps, const void* const* xs, void* const* ys,
+                               const rtoss_conv_desc* const* ds, void* stream) {
+    for (int i = 1; i < n; ++i) {
+        if (ps[i]->ksize != ps[0]->ksize) return -1;
+        if (ps[i]->ksize == 3 && ds[i]->stride != ds[0]->stride) return -1;   // (3x3: stride 2 stages four sub-tiles per block)
+    }
+    return rtoss_launch_conv_tc_chain(ctx, n, ps, xs, ys, ds, nullptr, stream);
+}
+
+int rtoss_tc_max_problems() { return kMaxProb; }

@@ -131,6 +131,13 @@ rtoss_status rtoss_create(int device, rtoss_ctx** out) {
     cudaSetDevice(device);
     cudaError_t se = cudaMalloc((void**)&c->dev_status, sizeof(int));
     if (se == cudaSuccess) se = cudaMemset(c->dev_status, 0, sizeof(int));
+    const size_t chain_bytes = sizeof(unsigned) * RTOSS_CHAIN_SLOTS * RTOSS_CHAIN_SLOT_WORDS;
+    if (se == cudaSuccess) se = cudaMalloc((void**)&c->chain_done, chain_bytes);
+    if (se == cudaSuccess) se = cudaMemset(c->chain_done, 0, chain_bytes);
+    if (se != cudaSuccess) {
+        if (c->dev_status) cudaFree(c->dev_status);
+        if (c->chain_done) cudaFree(c->chain_done);
+    }
     cudaSetDevice(prev);
     if (se != cudaSuccess) {
         cudaGetLastError();
@@ -159,6 +166,7 @@ void rtoss_destroy(rtoss_ctx* ctx) {
     if (ctx->ws_x) cudaFree(ctx->ws_x);
     if (ctx->ws_y) cudaFree(ctx->ws_y);
     if (ctx->dev_status) cudaFree(ctx->dev_status);
+    if (ctx->chain_done) cudaFree(ctx->chain_done);
     cudaSetDevice(prev);
     delete ctx;
 }
@@ -465,17 +473,18 @@ rtoss_status rtoss_conv_group(rtoss_ctx* ctx, const rtoss_conv_item* items, int 
     }
     rtoss_device_guard on_device(ctx->device);
     // Items that can share a launch are collected class by class (kernel size, data type, stride for 3x3; tensor path,
-    // filters on M), at most ten to a launch; whatever is left over, or declined by the launcher, runs as single calls.
+    // filters on M), at most twenty to a launch; whatever is left over, or declined by the launcher, runs as single calls.
     std::vector<char> done((size_t)n, 0);
     int count = 0;
     for (int i = 0; i < n; ++i) {
         if (done[(size_t)i]) continue;
-        const rtoss_packed* ps[10];
-        const void* xs[10];
-        void* ys[10];
-        const rtoss_conv_desc* ds[10];
-        int idx[10], m = 0;
-        for (int j = i; j < n && m < 10; ++j) {
+        const rtoss_packed* ps[32];
+        const void* xs[32];
+        void* ys[32];
+        const rtoss_conv_desc* ds[32];
+        int idx[32], m = 0;
+        const int m_max = rtoss_tc_max_problems();
+        for (int j = i; j < n && m < m_max; ++j) {
             if (done[(size_t)j]) continue;
             const rtoss_conv_item& a = items[j];
             const rtoss_conv_item& b = items[i];
@@ -505,6 +514,121 @@ rtoss_status rtoss_conv_group(rtoss_ctx* ctx, const rtoss_conv_item* items, int 
     return RTOSS_OK;
 }
 
+namespace {
+
+// Bytes a convolution call touches: [lo, hi) of its input, its output (the whole pixel pitch where it writes a
+// channel slice) and its residual operand.
+struct Span {
+    uintptr_t lo, hi;
+};
+inline bool overlap(const Span& a, const Span& b) { return a.lo < b.hi && b.lo < a.hi && a.lo != a.hi && b.lo != b.hi; }
+void spans_of(const rtoss_conv_item& it, Span* x, Span* y, Span* r) {
+    const rtoss_packed* p = it.packed;
+    const rtoss_conv_desc& d = it.desc;
+    const size_t es = rtoss_dtype_size(d.io_dtype);
+    const int S = d.stride > 0 ? d.stride : 1;
+    const size_t Ho = (size_t)((d.H - 1) / S + 1), Wo = (size_t)((d.W - 1) / S + 1);
+    const size_t pitch = d.y_channel_stride ? (size_t)d.y_channel_stride : (size_t)p->Cout;
+    x->lo = reinterpret_cast<uintptr_t>(it.x_dev);
+    x->hi = x->lo + (size_t)d.N * d.H * d.W * p->Cin * es;
+    // (a call that writes a channel slice is given the buffer's base: the span is the whole buffer)
+    y->lo = reinterpret_cast<uintptr_t>(it.y_dev);
+    y->hi = y->lo + (size_t)d.N * Ho * Wo * pitch * es;
+    r->lo = reinterpret_cast<uintptr_t>(d.residual_dev);
+    r->hi = d.residual_dev ? r->lo + (size_t)d.N * Ho * Wo * pitch * es : r->lo;
+}
+
+}  // namespace
+
+rtoss_status rtoss_chain_deps(const rtoss_conv_item* items, int n, uint32_t* after) {
+    if (!items || !after || n < 1 || n > 32) return RTOSS_ERR_INVALID_ARG;
+    uint64_t spans[32 * 6];
+    for (int i = 0; i < n; ++i) {
+        if (!items[i].packed) return RTOSS_ERR_INVALID_ARG;
+        Span x, y, r;
+        spans_of(items[i], &x, &y, &r);
+        uint64_t* q = spans + 6 * i;
+        q[0] = x.lo, q[1] = x.hi, q[2] = y.lo, q[3] = y.hi, q[4] = r.lo, q[5] = r.hi;
+    }
+    return rtoss_chain_deps_spans(spans, n, after);
+}
+
+rtoss_status rtoss_chain_deps_spans(const uint64_t* spans, int n, uint32_t* after) {
+    if (!spans || !after || n < 1 || n > 32) return RTOSS_ERR_INVALID_ARG;
+    Span x[32], y[32], r[32];
+    for (int i = 0; i < n; ++i) {
+        const uint64_t* q = spans + 6 * i;
+        if (q[0] > q[1] || q[2] > q[3] || q[4] > q[5]) return RTOSS_ERR_INVALID_ARG;
+        x[i] = Span{(uintptr_t)q[0], (uintptr_t)q[1]};
+        y[i] = Span{(uintptr_t)q[2], (uintptr_t)q[3]};
+        r[i] = Span{(uintptr_t)q[4], (uintptr_t)q[5]};
+    }
+    for (int i = 0; i < n; ++i) {
+        after[i] = 0;
+        for (int j = 0; j < i; ++j) {
+            const bool reads_j = overlap(x[i], y[j]) || overlap(r[i], y[j]);                          // i reads what j writes
+            const bool clobbers_j = overlap(y[i], x[j]) || overlap(y[i], r[j]) || overlap(y[i], y[j]);  // i overwrites what j reads or writes
+            if (reads_j || clobbers_j) after[i] |= 1u << j;
+        }
+    }
+    return RTOSS_OK;
+}
+
+rtoss_status rtoss_conv_chain(rtoss_ctx* ctx, const rtoss_conv_item* items, int n, const uint32_t* after, int* launches,
+                              void* cuda_stream) {
+    if (!ctx) return RTOSS_ERR_INVALID_ARG;
+    if (launches) *launches = 0;
+    if (!items || n < 1 || n > 32) {
+        set_err(ctx, "conv chain", "null argument, no items or more than 32");
+        return RTOSS_ERR_INVALID_ARG;
+    }
+    for (int i = 0; i < n; ++i) {
+        if (!items[i].packed) {
+            set_err(ctx, "conv chain", "item without a packed handle");
+            return RTOSS_ERR_INVALID_ARG;
+        }
+        rtoss_status st = check_conv(ctx, items[i].packed, items[i].x_dev, items[i].y_dev, &items[i].desc, items[i].packed->ksize, true);
+        if (st != RTOSS_OK) return st;
+        if (after && (i == 0 ? after[0] != 0 : (after[i] >> i) != 0)) {
+            set_err(ctx, "conv chain", "an item may only be ordered behind earlier items");
+            return RTOSS_ERR_INVALID_ARG;
+        }
+    }
+    uint32_t derived[32];
+    if (!after) {
+        rtoss_chain_deps(items, n, derived);
+        after = derived;
+    }
+    rtoss_device_guard on_device(ctx->device);
+    bool one_launch = n >= 2 && n <= rtoss_tc_max_problems();
+    for (int i = 0; i < n && one_launch; ++i)
+        one_launch = items[i].desc.path != RTOSS_PATH_FMA && rtoss_tc_groupable(items[i].packed, &items[i].desc, items[i].x_dev, items[i].y_dev);
+    if (one_launch) {
+        const rtoss_packed* ps[32];
+        const void* xs[32];
+        void* ys[32];
+        const rtoss_conv_desc* ds[32];
+        for (int i = 0; i < n; ++i) ps[i] = items[i].packed, xs[i] = items[i].x_dev, ys[i] = items[i].y_dev, ds[i] = &items[i].desc;
+        const int e = rtoss_launch_conv_tc_chain(ctx, n, ps, xs, ys, ds, after, cuda_stream);
+        if (e == 0) {
+            if (launches) *launches = 1;
+            return RTOSS_OK;
+        }
+        if (e > 0) return cuda_fail(ctx, "conv chain launch", e);
+    }
+    // not one launch: the calls go out in the given order (the stream keeps them apart)
+    int count = 0;
+    for (int i = 0; i < n; ++i) {
+        rtoss_status st = RTOSS_OK;
+        const int e = dispatch_conv(ctx, items[i].packed, items[i].x_dev, items[i].y_dev, &items[i].desc, cuda_stream, &st);
+        if (st != RTOSS_OK) return st;
+        if (e) return cuda_fail(ctx, "conv launch", e);
+        ++count;
+    }
+    if (launches) *launches = count;
+    return RTOSS_OK;
+}
+
 rtoss_status rtoss_set_wait_limit(rtoss_ctx* ctx, long long sm_cycles) {
     if (!ctx || sm_cycles < 1000) return RTOSS_ERR_INVALID_ARG;
     ctx->wait_cycles = sm_cycles;
@@ -525,6 +649,8 @@ rtoss_status rtoss_device_status(rtoss_ctx* ctx, int* code) {
     if (e != cudaSuccess) return cuda_fail(ctx, "device status", (int)e);
     if (*code != 0) {
         cudaMemset(ctx->dev_status, 0, sizeof(int));
+        // a launch that gave up may have left its completion counters half counted
+        cudaMemset(ctx->chain_done, 0, sizeof(unsigned) * RTOSS_CHAIN_SLOTS * RTOSS_CHAIN_SLOT_WORDS);
         set_err(ctx, "device status", "a bounded wait in a tensor-path kernel ran out");
         return RTOSS_ERR_TIMEOUT;
     }

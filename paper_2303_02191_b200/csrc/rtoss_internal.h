@@ -17,6 +17,12 @@ struct rtoss_tmap_entry {
 
 constexpr int kHostChunks = 8;  // the host-buffer path cuts a batch into at most this many chunks
 
+// Launches that carry dependent convolutions count completed problems in device memory: a block of
+// RTOSS_CHAIN_SLOT_WORDS words per launch (one per problem and one exit counter, zero between launches), taken in
+// turn from RTOSS_CHAIN_SLOTS blocks of the context.
+constexpr int RTOSS_CHAIN_SLOTS = 64;
+constexpr int RTOSS_CHAIN_SLOT_WORDS = 32;
+
 struct rtoss_ctx {
     int device;
     int sm_count;
@@ -36,6 +42,8 @@ struct rtoss_ctx {
     mutable int inject_next;   // failure-detection test hook: the next tensor-path launch withholds its first weight copy
     mutable rtoss_tmap_entry tmap_cache[32];  // activation descriptors of the tensor path, round robin
     mutable int tmap_next;
+    unsigned* chain_done;      // device: RTOSS_CHAIN_SLOTS x RTOSS_CHAIN_SLOT_WORDS completion counters, all zero at rest
+    mutable int chain_next;    // the block the next launch with dependent convolutions takes
 };
 
 struct rtoss_packed {
@@ -130,5 +138,9 @@ bool rtoss_tc_groupable(const rtoss_packed* p, const rtoss_conv_desc* d, const v
 // several independent convolutions in one launch: 0 = launched, -1 = the set cannot share a launch (nothing launched)
 int rtoss_launch_conv_tc_group(const rtoss_ctx* ctx, int n, const rtoss_packed* const* ps, const void* const* xs,
                                void* const* ys, const rtoss_conv_desc* const* ds, void* stream);
+// the same with dependencies: bit j of after[i] = convolution i waits (inside the launch) for convolution j < i
+int rtoss_launch_conv_tc_chain(const rtoss_ctx* ctx, int n, const rtoss_packed* const* ps, const void* const* xs,
+                               void* const* ys, const rtoss_conv_desc* const* ds, const uint32_t* after, void* stream);
+int rtoss_tc_max_problems();   // most convolutions one launch carries
 
 #endif
