@@ -44,8 +44,8 @@ def workload_layers(name):
     if name == "retinanet_b4":
         return 4, "bf16", [(L, 4, "centre8") for L in synth.retinanet_r50fpn_stack()]
     if name == "retinanet_tower":
-        # the launch that dominates retinanet_b4: the first layer of both towers on the five pyramid levels
-        return 4, "bf16", [(L, 4, "centre8") for L in synth.retinanet_r50fpn_stack() if "_tower0." in L["name"]]
+        # the launch that dominates retinanet_b4: the first two layers of both towers on the five pyramid levels
+        return 4, "bf16", [(L, 4, "centre8") for L in synth.retinanet_r50fpn_stack() if "_tower0." in L["name"] or "_tower1." in L["name"]]
     raise SystemExit("unknown workload " + name)
 
 
@@ -283,12 +283,12 @@ def run_network(args):
     side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
         for _ in range(max(args.warmup, 3)):
-            net.run(grouped=args.group)
+            net.run(grouped=args.group, chained=args.chain)
     torch.cuda.current_stream().wait_stream(side)
     torch.cuda.synchronize()
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
-        net.run(grouped=args.group)
+        net.run(grouped=args.group, chained=args.chain)
     graph.replay()
     torch.cuda.synchronize()
     if ctx.rtoss_device_status() != 0:
@@ -392,7 +392,12 @@ def measure_workload(ctx, rt, dev, name, steps, warmup, args, world, rank, full,
             ev[1].record()
 
     # launch units: convolutions that are independent in the network share one grouped call
-    units = synth.independent_sets([st["L"] for st in L_state]) if args.group else [[i] for i in range(len(L_state))]
+    # (and, unless --no-chain, successive tower layers share a launch whose members wait for one another: rtoss_conv_chain)
+    if args.group and args.chain:
+        units, afters = synth.chained_units([st["L"] for st in L_state])
+    else:
+        units = synth.independent_sets([st["L"] for st in L_state]) if args.group else [[i] for i in range(len(L_state))]
+        afters = [None] * len(units)
     unit_launches = [1] * len(units)
 
     def run_unit(u, ev=None):
@@ -409,7 +414,7 @@ def measure_workload(ctx, rt, dev, name, steps, warmup, args, world, rank, full,
                                        rt.ACT_NAMES[L["act"]], st["wt"]["b"], path=st["path"]))
         if ev:
             ev[0].record()
-        n = ctx.rtoss_conv_group(items)
+        n = ctx.rtoss_conv_chain(items, afters[u]) if afters[u] else ctx.rtoss_conv_group(items)
         if ev:
             ev[1].record()
         return n
@@ -694,8 +699,9 @@ def run_gpu(args):
             "config": {"workload": args.workload, "batch": N, "layout": res["layout"], "layers": len(res["layers"]),
                        "l2": "flushed between steps (256 MB write)", "multi_gpu": "replicas only",
                        "launch": "one CUDA graph per step" if res["graph"] else "eager",
-                       "grouping": ("independent convolutions share a launch: %d launches for %d convolutions"
-                                    % (sum(res["unit_launches"]), len(res["layers"]))) if args.group else "one launch per convolution"},
+                       "grouping": ("independent convolutions%s share a launch: %d launches for %d convolutions"
+                                    % (" and successive tower layers" if args.chain else "", sum(res["unit_launches"]), len(res["layers"])))
+                                   if args.group else "one launch per convolution"},
             "paths": {"tensor_path_layers": int(sum(res["on_tc"])), "fma_path_layers": int(len(res["on_tc"]) - sum(res["on_tc"]))},
             "nnz_gflops_per_s": float(rf["flops"].sum()) / (ms_per_step * 1e-3) / 1e9 * world,
             "conv_ms": [float(v) for v in res["conv_ms"]] if len(res["conv_ms"]) <= 8 else None,
@@ -765,6 +771,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="retinanet_b4")
+    ap.add_argument("--no-chain", dest="chain", action="store_false",
+                    help="dependent convolutions do not share launches (rtoss_conv_chain is not used)")
     ap.add_argument("--no-others", dest="others", action="store_false",
                     help="skip the sub-records of the other configurations (layer32, layer128, yolov5s_b1, yolov5s_b16)")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")

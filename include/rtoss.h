@@ -347,14 +347,17 @@ rtoss_status rtoss_conv_group(rtoss_ctx* ctx, const rtoss_conv_item* items, int 
  * derives exactly that from the address ranges of the items' inputs, outputs and residual operands
  * (rtoss_chain_deps).  The result is that of the single calls issued in the given order.
  *
- * When all items qualify for a shared launch (tensor path, more than 64 filters or a 3x3 kernel, one data type, at
- * most 20 items) they go out as ONE kernel: its CTAs walk the items' tiles in order and, before the first tile of an
+ * Consecutive items that qualify for a shared launch (tensor path, more than 64 filters or a 3x3 kernel, one data
+ * type; at most 20) go out as ONE kernel: its CTAs walk the items' tiles in order and, before the first tile of an
  * item, wait until all tiles of the items it depends on are written (a counter per item in device memory; the wait is
  * bounded like every device-side wait, see rtoss_set_wait_limit, and reports through rtoss_device_status).  Items
  * that do not depend on one another run side by side as in rtoss_conv_group.  Such a launch relies on all its CTAs
  * (at most one per SM) being on the device together: while it runs, no other work may occupy SMs without end, and two
- * such launches must not run concurrently on different streams.  Otherwise the items run as single launches in the
- * given order.  *launches (nullable) receives the number of kernel launches made.
+ * such launches must not run concurrently on different streams.  An item that does not qualify, or that has nothing
+ * to run beside it and so few tiles and so many input channels that a launch of its own spreads it over more SMs
+ * (split along the channels), runs as a launch of its own between the shared ones (the stream orders them); an item
+ * whose desc.path is RTOSS_PATH_TENSOR rather than RTOSS_PATH_AUTO stays in the shared launch whenever it qualifies.  *launches (nullable) receives the number of kernel
+ * launches made.
  * Errors: RTOSS_ERR_INVALID_ARG (null items, n outside 1..32, a bit of after[i] at or above i) and those of the single
  * calls; nothing is launched when an argument check fails. */
 rtoss_status rtoss_conv_chain(rtoss_ctx* ctx, const rtoss_conv_item* items, int n, const uint32_t* after, int* launches,

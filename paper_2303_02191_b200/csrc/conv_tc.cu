@@ -126,6 +126,9 @@ struct TcArgs {
     unsigned a_stage, b_stage, sB_off;
     int geo;
     int tab;              // which of the launch's position tables
+    // over_res: this problem's rings reach into the launch's residual staging area (only problems without a residual
+    // operand may): a CTA that comes to it from a problem with one waits for that problem's epilogues first.
+    int over_res;
     // Dependent problems of one launch: bit j of dep_mask = problem j (earlier in the launch's order) must be complete
     // -- all its outputs written -- before this one reads an activation or writes an output; done_target = arrivals
     // on this problem's counter that make it complete (epilogue warps x CTAs that hold units of it).
@@ -145,6 +148,7 @@ struct TcLaunchT {
     int ring_bytes;           // the ring area: the most any problem's activation + weight stages take
     int max_na, max_nb;       // most activation / weight stages any problem uses (barriers to set up)
     int n_tabs;               // position tables
+    int res_off;              // where in the ring area the staging of residual operands lies (its top end), when a problem has one
     unsigned* done;           // dependent problems: kMaxProb completion counters + one exit counter, all zero between launches; else null
     int AS, acc_stride;                        // accumulator stages in TMEM and columns per stage
     int tmem_cols;
@@ -738,7 +742,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
     unsigned char* epi_patch = smem_dyn + (s_tmem_ptr + 16 - smem_u32(smem_dyn));  // [kEpiWarps][kPatchBytes], 16-byte aligned
     uint2* pos_tab_all = reinterpret_cast<uint2*>(epi_patch + kEpiWarps * kPatchBytes);  // [n_tabs][kMaxPx]
     const unsigned s_tab_all = s_tmem_ptr + 16 + kEpiWarps * kPatchBytes;                // the same, as a shared address
-    const unsigned s_res = s_tab_all + (unsigned)g.n_tabs * kMaxPx * 8;   // [kEpiWarps][kResStage], present when a call has a residual operand
+    const unsigned s_res = sA + (unsigned)g.res_off;   // [kEpiWarps][kResStage], present when a call has a residual operand
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = g.unit_end[g.n_prob - 1];  // units of work over all problems: (tile, share of the channel blocks)
@@ -949,6 +953,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
             int as = 0, n_done = 0;
             unsigned pacc = 0;                  // phase parity of the accumulator ring
             unsigned peek = 0;                  // what umma_block_peek saw of the stages now current
+            int since_res = 1 << 20;            // tiles issued since this CTA's last tile with a residual operand
             auto mk = [desc_hi](unsigned lo) { return ((unsigned long long)desc_hi << 32) | lo; };
             // all instructions of one tap: the K slabs named by m4 (times two halves of positions with the positions as M)
             auto issue_tap = [&](unsigned d_base, unsigned wl, unsigned xl, unsigned m4, unsigned& acc) {
@@ -977,6 +982,21 @@ conv_tc_kernel(const __grid_constant__ G g) {
                 const TcArgs& a = g.prob[pi];
                 if (pi != cur_pi) {
                     if (kMulti && cur_pi >= 0 && a.geo != g.prob[cur_pi].geo) {
+                        if (a.over_res) {
+                            // The new rings cover the staging area of residual operands.  An epilogue that may still use it
+                            // belongs to one of this CTA's last AS tiles (the accumulator stage of an older one has been
+                            // waited for since), and only if that tile had a residual operand: `since_res` tiles ago or earlier.
+                            int as_b = as;
+                            unsigned pacc_b = pacc;
+                            for (int i = 0; i < g.AS && i < n_done && ok; ++i) {
+                                if (--as_b < 0) {
+                                    as_b = g.AS - 1;
+                                    pacc_b ^= 1;
+                                }
+                                if (i >= since_res) ok = mbar_wait(bar_accEmpty + 8 * as_b, pacc_b, g.wait_cycles);
+                            }
+                            if (!ok) break;
+                        }
                         // rings of another layout: the producers may write them once everything issued so far has read its operands
                         umma_commit(bar_switch);
                         ra.s = rb.s = 0;
@@ -1109,6 +1129,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
                     bits = bits_n;
                 }
                 if (ok) umma_commit(bar_accFull + 8 * as);
+                since_res = a.resid ? 0 : since_res + 1;
                 if (++as == g.AS) {
                     as = 0;
                     pacc ^= 1;
@@ -1606,6 +1627,34 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
     return 0;
 }
 
+// Split K where the layer has too few tiles for the SMs and several channel blocks: a tile's MMAs are one serial chain
+// (an instruction costs the same however few positions it covers), so the blocks go to several CTAs.  The exchange
+// costs a few thousand cycles (two cluster barriers, 128 KB through distributed shared memory): chains of 72
+// instructions (3x3: two channel blocks) resp. 32 (1x1: eight blocks) and more are cut, a share keeps at least one
+// block (1x1: two); cutting shorter 1x1 chains was measured and lost.  The CTAs of a tile form one cluster (at most
+// 8), one CTA per share.  *ks = 1 leaves the layer uncut.
+void pick_split(int ksize, bool pxm, int R, long tiles, int ncb, int n_px, int rings, int sms, int* ks_out, int* cb_per_out) {
+    *ks_out = 1;
+    *cb_per_out = ncb;
+    const int min_cb = ksize == 3 ? 1 : 2;
+    const int min_ncb = ksize == 3 ? 2 : 8;
+    const int n_lc_max = 8;   // a tile has at most 8 chunks of 32 columns: the owner's buffers take KS * ceil(chunks / KS) * 16 KB
+    if (pxm || R != 1 || tiles * 2 > sms || ncb < min_ncb) return;
+    int want = (int)(sms / tiles);
+    if (want > ncb / min_cb) want = ncb / min_cb;
+    if (want > 8) want = 8;
+    while (want > 1) {
+        const int cb_per = (ncb + want - 1) / want, ks = (ncb + cb_per - 1) / cb_per;
+        const int n_chunks = (n_px + 31) / 32, n_lc = (n_chunks + ks - 1) / ks;
+        if (ks > 1 && ks * n_lc <= 2 * n_lc_max && (size_t)ks * n_lc * 16384 <= (size_t)rings) {
+            *cb_per_out = cb_per;
+            *ks_out = ks;
+            return;
+        }
+        --want;
+    }
+}
+
 // Both instantiations may use up to the whole shared memory of an SM; the attribute belongs to the (function, device)
 // pair, so there is one flag per device.
 int ensure_smem_attr(const rtoss_ctx* ctx) {
@@ -1666,6 +1715,24 @@ bool rtoss_tc_groupable(const rtoss_packed* p, const rtoss_conv_desc* d, const v
     return !use_pxm(p) && rtoss_tc_eligible(p, d, x, y);
 }
 
+// Would a launch of its own cut this call along K (few tiles, many channel blocks)?  Such a call is faster alone than
+// as a member of a shared launch, which never cuts.
+bool rtoss_tc_prefers_split(const rtoss_ctx* ctx, const rtoss_packed* p, const rtoss_conv_desc* d) {
+    const int sms = ctx->sm_count > 0 ? ctx->sm_count : 148;
+    const int Ho = (d->H - 1) / d->stride + 1, Wo = (d->W - 1) / d->stride + 1;
+    const bool pxm = use_pxm(p), f32 = p->dtype == RTOSS_F32;
+    const int w_rows = pxm ? round_up(p->Cout, 16) : kMTile, co_tiles = (p->Cout + kMTile - 1) / kMTile;
+    TcPlan plan;
+    if (!plan_tc(d->N, Ho, Wo, p->ksize, d->stride, co_tiles, sms, pxm, w_rows, d->residual_dev != nullptr, &plan, 1, f32)) return false;
+    const int a_stage = plan.n_sub * plan.sub_rows * kRowBytes * (f32 ? 2 : 1), b_stage = plan.G * w_rows * kRowBytes;
+    const int cb_ch = kRowBytes / (f32 ? 4 : 2);
+    const long tiles = (long)d->N * ((Ho + plan.TH - 1) / plan.TH) * plan.tiles_x * co_tiles;
+    int ks = 1, cb_per = 0;
+    pick_split(p->ksize, pxm, rtoss_wtc_layout_of(p->Cout, p->ksize).copies, tiles, (p->Cin + cb_ch - 1) / cb_ch, plan.N_px,
+               plan.NA * a_stage + plan.NB * b_stage, sms, &ks, &cb_per);
+    return ks > 1;
+}
+
 int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y, const rtoss_conv_desc* d,
                          void* stream) {
     const int sms = ctx->sm_count > 0 ? ctx->sm_count : 148;
@@ -1682,40 +1749,16 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     a.a_stage = (unsigned)pp.a_stage_bytes;
     a.b_stage = (unsigned)pp.b_stage_bytes;
     a.sB_off = (unsigned)plan.NA * a.a_stage;
-    g.ring_bytes = (int)(a.sB_off + (unsigned)plan.NB * a.b_stage);
+    const int rings = (int)(a.sB_off + (unsigned)plan.NB * a.b_stage);
+    g.res_off = rings;   // the staging of a residual operand lies behind the rings
+    g.ring_bytes = rings + (d->residual_dev ? kEpiWarps * kResStage : 0);
     g.max_na = plan.NA;
     g.max_nb = plan.NB;
     g.n_tabs = 1;
     g.done = nullptr;
     g.acc_stride = pp.acc_cols;
     launch_common(ctx, &g);
-    // Split K where the layer has too few tiles for the SMs and several channel blocks: a tile's MMAs are one serial
-    // chain (an instruction costs the same however few positions it covers), so the blocks go to several CTAs.
-    {
-        const long tiles = (long)d->N * a.tiles_y * a.tiles_x * a.co_tiles;
-        // The exchange costs a few thousand cycles (two cluster barriers, 128 KB through distributed shared memory):
-        // chains of 72 instructions (3x3: two channel blocks) resp. 32 (1x1: eight blocks) and more are cut, a share
-        // keeps at least one block (1x1: two); cutting shorter 1x1 chains was measured and lost.  The CTAs of a tile
-        // form one cluster (at most 8), one CTA per share.
-        const int min_cb = p->ksize == 3 ? 1 : 2;
-        const int min_ncb = p->ksize == 3 ? 2 : 8;
-        const int n_lc_max = 8;   // a tile has at most 8 chunks of 32 columns: the owner's buffers take KS * ceil(chunks / KS) * 16 KB
-        if (!a.pxm && a.R == 1 && tiles * 2 <= sms && a.ncb >= min_ncb) {
-            int want = (int)(sms / tiles);
-            if (want > a.ncb / min_cb) want = a.ncb / min_cb;
-            if (want > 8) want = 8;
-            while (want > 1) {
-                const int cb_per = (a.ncb + want - 1) / want, ks = (a.ncb + cb_per - 1) / cb_per;
-                const int n_chunks = (plan.N_px + 31) / 32, n_lc = (n_chunks + ks - 1) / ks;
-                if (ks > 1 && ks * n_lc <= 2 * n_lc_max && (size_t)ks * n_lc * 16384 <= (size_t)g.ring_bytes) {
-                    a.cb_per = cb_per;
-                    a.KS = ks;
-                    break;
-                }
-                --want;
-            }
-        }
-    }
+    pick_split(p->ksize, a.pxm != 0, a.R, (long)d->N * a.tiles_y * a.tiles_x * a.co_tiles, a.ncb, plan.N_px, rings, sms, &a.KS, &a.cb_per);
     // at least half an SM's shared memory, so that a second CTA (which would wait for TMEM) never shares the SM
     const size_t smem = (size_t)(plan.smem > 116 * 1024 ? plan.smem : 116 * 1024);
     size_t n_units = (size_t)d->N * a.tiles_y * a.tiles_x * a.co_tiles * a.KS;
@@ -1792,60 +1835,85 @@ int rtoss_launch_conv_tc_chain(const rtoss_ctx* ctx, int n, const rtoss_packed* 
     int geo_of[kMaxProb];
     struct Geo {
         int a, b, na, nb;
+        bool under;   // planned below the staging area of residual operands
     } geos[kMaxProb];
-    int n_geo = 0;
-    const int fixed = 1024 + 512 + kEpiWarps * kPatchBytes + kMaxTabs * kMaxPx * 8 + (resid ? kEpiWarps * kResStage : 0);
+    int n_geo = 0, acc_max = 0, n_tabs_planned = 0;
     const int cap = 227 * 1024 - 64;
-    bool seen[kMaxProb] = {};
-    int acc_max = 0;
-    for (int i0 = 0; i0 < n; ++i0) {
-        if (seen[i0]) continue;
-        // the set of this convolution: same level, same class
-        int set[kMaxProb], m = 0;
-        for (int j = i0; j < n; ++j)
-            if (!seen[j] && level[j] == level[i0] && cls[j] == cls[i0]) set[m++] = j, seen[j] = true;
-        // every problem is planned on its own first; where they disagree on the taps per weight stage, all are planned
-        // again with the smallest (a stage per tap fits whatever fits three)
-        int force_G = 0, a_max = 0, b_bytes = 0;
-        for (int pass = 0; pass < 2; ++pass) {
-            bool agree = true;
-            int g_min = 9;
-            a_max = 0;
-            for (int q = 0; q < m; ++q) {
-                const int i = set[q];
-                // (planned with the launch's fixed shared memory: all position tables, the residual staging if any needs it)
-                rtoss_conv_desc dd = *ds[i];
-                static const int dummy = 0;
-                if (resid && !dd.residual_dev) dd.residual_dev = &dummy;   // only the plan's memory budget looks at it here
-                int e = build_problem(ctx, ps[i], xs[i], ys[i], &dd, m, sms, &args[i], &pp[i], &mapA[i], &mapB[i], force_G, kMaxTabs);
-                if (e == (int)cudaErrorInvalidConfiguration) return -1;
-                if (e) return e;
-                args[i].resid = ds[i]->residual_dev;
-                args[i].resid_post = (ds[i]->residual_dev && ds[i]->residual_after_act) ? 1 : 0;
-                if (q == 0) b_bytes = pp[i].b_stage_bytes;
-                if (pp[i].b_stage_bytes != b_bytes || args[i].G != args[set[0]].G) agree = false;
-                if (args[i].G < g_min) g_min = args[i].G;
-                if (pp[i].a_stage_bytes > a_max) a_max = pp[i].a_stage_bytes;
-                if (pp[i].acc_cols > acc_max) acc_max = pp[i].acc_cols;
-                n_tiles[i] = (long)args[i].N * args[i].tiles_y * args[i].tiles_x * args[i].co_tiles;
+    const int res_bytes = resid ? kEpiWarps * kResStage : 0;
+    // Shared memory outside the rings: alignment slack, barriers, epilogue patches, the position tables.  How many
+    // tables the launch needs is known once every problem is planned: planned with four first, with kMaxTabs if that
+    // was too few.
+    for (int tabs_try = 4; tabs_try <= kMaxTabs; tabs_try += kMaxTabs - 4) {
+        const int fixed = 1024 + 512 + kEpiWarps * kPatchBytes + tabs_try * kMaxPx * 8;
+        bool seen[kMaxProb] = {};
+        n_geo = acc_max = 0;
+        for (int i0 = 0; i0 < n; ++i0) {
+            if (seen[i0]) continue;
+            // the set of this convolution: same level, same class
+            int set[kMaxProb], m = 0;
+            bool set_res = false;
+            for (int j = i0; j < n; ++j)
+                if (!seen[j] && level[j] == level[i0] && cls[j] == cls[i0]) set[m++] = j, seen[j] = true, set_res = set_res || ds[j]->residual_dev;
+            // The staging area of residual operands is the top end of the ring area.  A set of 3x3 convolutions none of
+            // which has a residual operand may lay its rings over it (the kernel then lets the epilogues that use the
+            // area finish first); every other set stays below it.
+            const bool under = resid && (set_res || ps[i0]->ksize != 3);
+            // every problem is planned on its own first; where they disagree on the taps per weight stage, all are
+            // planned again with the smallest (a stage per tap fits whatever fits three)
+            int force_G = 0, a_max = 0, b_bytes = 0;
+            for (int pass = 0; pass < 2; ++pass) {
+                bool agree = true;
+                int g_min = 9;
+                a_max = 0;
+                for (int q = 0; q < m; ++q) {
+                    const int i = set[q];
+                    rtoss_conv_desc dd = *ds[i];
+                    static const int dummy = 0;
+                    dd.residual_dev = under ? &dummy : nullptr;   // (only the plan's memory budget looks at it here)
+                    int e = build_problem(ctx, ps[i], xs[i], ys[i], &dd, m, sms, &args[i], &pp[i], &mapA[i], &mapB[i], force_G, tabs_try);
+                    if (e == (int)cudaErrorInvalidConfiguration) return -1;
+                    if (e) return e;
+                    args[i].resid = ds[i]->residual_dev;
+                    args[i].resid_post = (ds[i]->residual_dev && ds[i]->residual_after_act) ? 1 : 0;
+                    if (q == 0) b_bytes = pp[i].b_stage_bytes;
+                    if (pp[i].b_stage_bytes != b_bytes || args[i].G != args[set[0]].G) agree = false;
+                    if (args[i].G < g_min) g_min = args[i].G;
+                    if (pp[i].a_stage_bytes > a_max) a_max = pp[i].a_stage_bytes;
+                    if (pp[i].acc_cols > acc_max) acc_max = pp[i].acc_cols;
+                    n_tiles[i] = (long)args[i].N * args[i].tiles_y * args[i].tiles_x * args[i].co_tiles;
+                }
+                if (agree) break;
+                if (pass == 1) return -1;
+                force_G = g_min;
             }
-            if (agree) break;
-            if (pass == 1) return -1;
-            force_G = g_min;
+            // the rings every problem of the set fits into
+            const int room = cap - fixed - (under ? res_bytes : 0);
+            int na = (room - 2 * b_bytes) / a_max;
+            if (na > kMaxA) na = kMaxA;
+            if (na > 2 && ps[i0]->ksize == 3) na = 2;
+            if (na < 1) return -1;
+            int nb = (room - na * a_max) / b_bytes;
+            if (nb > kMaxB) nb = kMaxB;
+            if (nb < 2) return -1;
+            int gi = 0;
+            while (gi < n_geo && !(geos[gi].a == a_max && geos[gi].b == b_bytes && geos[gi].na == na && geos[gi].nb == nb && geos[gi].under == under)) ++gi;
+            if (gi == n_geo) geos[n_geo++] = Geo{a_max, b_bytes, na, nb, under};
+            for (int q = 0; q < m; ++q) geo_of[set[q]] = gi;
         }
-        // the rings every problem of the set fits into
-        int na = (cap - fixed - 2 * b_bytes) / a_max;
-        if (na > kMaxA) na = kMaxA;
-        if (na > 2 && ps[i0]->ksize == 3) na = 2;
-        if (na < 1) return -1;
-        int nb = (cap - fixed - na * a_max) / b_bytes;
-        if (nb > kMaxB) nb = kMaxB;
-        if (nb < 2) return -1;
-        int gi = 0;
-        while (gi < n_geo && !(geos[gi].a == a_max && geos[gi].b == b_bytes && geos[gi].na == na && geos[gi].nb == nb)) ++gi;
-        if (gi == n_geo) geos[n_geo++] = Geo{a_max, b_bytes, na, nb};
-        for (int q = 0; q < m; ++q) geo_of[set[q]] = gi;
+        // distinct position tables
+        int n_distinct = 0;
+        for (int i = 0; i < n; ++i) {
+            bool fresh = true;
+            for (int j = 0; j < i && fresh; ++j)
+                fresh = !(args[j].Wq == args[i].Wq && args[j].TH == args[i].TH && args[j].TW == args[i].TW && args[j].N_px == args[i].N_px &&
+                          args[j].Wo == args[i].Wo && args[j].y_c_stride == args[i].y_c_stride);
+            n_distinct += fresh ? 1 : 0;
+        }
+        n_tabs_planned = tabs_try;
+        if (n_distinct <= tabs_try) break;
+        if (tabs_try == kMaxTabs) return -1;
     }
+    const int fixed = 1024 + 512 + kEpiWarps * kPatchBytes + n_tabs_planned * kMaxPx * 8;
     // the launch's order: by level, inside a level by ring layout, then by falling tile count (stable)
     int order[kMaxProb];
     for (int i = 0; i < n; ++i) order[i] = i;
@@ -1860,7 +1928,7 @@ int rtoss_launch_conv_tc_chain(const rtoss_ctx* ctx, int n, const rtoss_packed* 
     for (int k = 0; k < n; ++k) where[order[k]] = k;
     g.n_prob = n;
     g.n_tabs = 0;
-    g.ring_bytes = 0;
+    g.ring_bytes = res_bytes;
     g.max_na = g.max_nb = 1;
     long units = 0;
     for (int k = 0; k < n; ++k) {
@@ -1876,7 +1944,7 @@ int rtoss_launch_conv_tc_chain(const rtoss_ctx* ctx, int n, const rtoss_packed* 
         a.b_stage = (unsigned)ge.b;
         a.sB_off = (unsigned)ge.na * (unsigned)ge.a;
         a.geo = geo_of[i];
-        const int ring = ge.na * ge.a + ge.nb * ge.b;
+        const int ring = ge.na * ge.a + ge.nb * ge.b + (ge.under ? res_bytes : 0);
         if (ring > g.ring_bytes) g.ring_bytes = ring;
         if (ge.na > g.max_na) g.max_na = ge.na;
         if (ge.nb > g.max_nb) g.max_nb = ge.nb;
@@ -1887,7 +1955,7 @@ int rtoss_launch_conv_tc_chain(const rtoss_ctx* ctx, int n, const rtoss_packed* 
             if (b.Wq == a.Wq && b.TH == a.TH && b.TW == a.TW && b.N_px == a.N_px && b.Wo == a.Wo && b.y_c_stride == a.y_c_stride) a.tab = b.tab;
         }
         if (a.tab < 0) {
-            if (g.n_tabs == kMaxTabs) return -1;
+            if (g.n_tabs == n_tabs_planned) return -1;
             a.tab = g.n_tabs++;
         }
         a.dep_mask = 0;
@@ -1899,9 +1967,12 @@ int rtoss_launch_conv_tc_chain(const rtoss_ctx* ctx, int n, const rtoss_packed* 
         g.unit_end[k] = (int)units;
     }
     const int grid_n = (int)(units < sms ? units : sms);
+    g.res_off = g.ring_bytes - res_bytes;
     for (int k = 0; k < n; ++k) {
         const long mine = n_tiles[order[k]];
-        g.prob[k].done_target = (unsigned)((mine < grid_n ? mine : grid_n) * kEpiWarps);
+        TcArgs& a = g.prob[k];
+        a.done_target = (unsigned)((mine < grid_n ? mine : grid_n) * kEpiWarps);
+        a.over_res = (resid && (int)(a.sB_off + (unsigned)a.NB * a.b_stage) > g.res_off) ? 1 : 0;
     }
     g.done = nullptr;
     if (chained) {

@@ -600,30 +600,57 @@ rtoss_status rtoss_conv_chain(rtoss_ctx* ctx, const rtoss_conv_item* items, int 
         after = derived;
     }
     rtoss_device_guard on_device(ctx->device);
-    bool one_launch = n >= 2 && n <= rtoss_tc_max_problems();
-    for (int i = 0; i < n && one_launch; ++i)
-        one_launch = items[i].desc.path != RTOSS_PATH_FMA && rtoss_tc_groupable(items[i].packed, &items[i].desc, items[i].x_dev, items[i].y_dev);
-    if (one_launch) {
-        const rtoss_packed* ps[32];
-        const void* xs[32];
-        void* ys[32];
-        const rtoss_conv_desc* ds[32];
-        for (int i = 0; i < n; ++i) ps[i] = items[i].packed, xs[i] = items[i].x_dev, ys[i] = items[i].y_dev, ds[i] = &items[i].desc;
-        const int e = rtoss_launch_conv_tc_chain(ctx, n, ps, xs, ys, ds, after, cuda_stream);
-        if (e == 0) {
-            if (launches) *launches = 1;
-            return RTOSS_OK;
-        }
-        if (e > 0) return cuda_fail(ctx, "conv chain launch", e);
+    // Maximal runs of consecutive items that can share a launch go out as one kernel each; an item that cannot (FMA
+    // path, positions on M) or that is better off alone (few tiles, many channel blocks and nothing to run beside it:
+    // a launch of its own cuts it along K over several CTAs, a shared launch never does) goes out on its own between them.  The stream orders the launches, so inside a run
+    // only the dependencies on items of the same run have to be carried into the kernel.
+    const int m_max = rtoss_tc_max_problems();
+    // (an item's level: one more than the highest level it waits for; items of one level run side by side)
+    int level[32], at_level[33] = {};
+    bool member[32];
+    for (int q = 0; q < n; ++q) {
+        level[q] = 0;
+        for (int j = 0; j < q; ++j)
+            if ((after[q] >> j) & 1u) level[q] = level[j] + 1 > level[q] ? level[j] + 1 : level[q];
+        ++at_level[level[q]];
     }
-    // not one launch: the calls go out in the given order (the stream keeps them apart)
-    int count = 0;
-    for (int i = 0; i < n; ++i) {
-        rtoss_status st = RTOSS_OK;
-        const int e = dispatch_conv(ctx, items[i].packed, items[i].x_dev, items[i].y_dev, &items[i].desc, cuda_stream, &st);
-        if (st != RTOSS_OK) return st;
-        if (e) return cuda_fail(ctx, "conv launch", e);
-        ++count;
+    for (int q = 0; q < n; ++q) {
+        const rtoss_conv_item& it = items[q];
+        member[q] = it.desc.path != RTOSS_PATH_FMA && rtoss_tc_groupable(it.packed, &it.desc, it.x_dev, it.y_dev) &&
+                    !(at_level[level[q]] == 1 && it.desc.path == RTOSS_PATH_AUTO && rtoss_tc_prefers_split(ctx, it.packed, &it.desc));
+    }
+    int count = 0, i = 0;
+    while (i < n) {
+        int m = 0;
+        while (i + m < n && m < m_max && member[i + m] && items[i + m].packed->dtype == items[i].packed->dtype) ++m;
+        if (m >= 2) {
+            const rtoss_packed* ps[32];
+            const void* xs[32];
+            void* ys[32];
+            const rtoss_conv_desc* ds[32];
+            uint32_t aft[32];
+            for (int q = 0; q < m; ++q) {
+                const rtoss_conv_item& it = items[i + q];
+                ps[q] = it.packed, xs[q] = it.x_dev, ys[q] = it.y_dev, ds[q] = &it.desc;
+                aft[q] = (after[i + q] >> i) & ((1u << q) - 1u);
+            }
+            const int e = rtoss_launch_conv_tc_chain(ctx, m, ps, xs, ys, ds, aft, cuda_stream);
+            if (e > 0) return cuda_fail(ctx, "conv chain launch", e);
+            if (e == 0) {
+                ++count;
+                i += m;
+                continue;
+            }
+        }
+        // a single item, or a run the launcher declined: one call per item, in order
+        const int single = m >= 2 ? m : 1;
+        for (int q = 0; q < single; ++q, ++i) {
+            rtoss_status st = RTOSS_OK;
+            const int e = dispatch_conv(ctx, items[i].packed, items[i].x_dev, items[i].y_dev, &items[i].desc, cuda_stream, &st);
+            if (st != RTOSS_OK) return st;
+            if (e) return cuda_fail(ctx, "conv launch", e);
+            ++count;
+        }
     }
     if (launches) *launches = count;
     return RTOSS_OK;

@@ -123,7 +123,7 @@ class GpuNet:
         if fuse_residual:
             self.ops = fuse_adds(self.ops, self.output_names)
         self.unfused = set()   # layers whose fused call the library declined: convolution and add run separately
-        self.rounds, self.probed = None, False
+        self.rounds, self.probed, self.steps = None, False, None
         tdt = {"bf16": torch.bfloat16, "f16": torch.float16}[dtype]
         self.t = {n: torch.zeros((N, H, W, C), dtype=tdt, device="cuda") for n, (C, H, W) in self.bufs.items()}
         self.zero = {}   # all-zero operands of the ReLU glue op, one per shape
@@ -157,7 +157,7 @@ class GpuNet:
     def _write(self, op):
         return op[{"conv": 3, "convres": 5, "add": 3, "up": 2, "relu": 2}[op[0]]]
 
-    def run(self, grouped=True):
+    def run(self, grouped=True, chained=False):
         """One pass.  grouped: operations are issued round by round (schedule.levels) and the convolutions of a round go
         out through rtoss_conv_group; else one call per operation in program order."""
         self.launches = 0      # kernel launches of this pass
@@ -169,6 +169,17 @@ class GpuNet:
         if self.rounds is None:
             # as late as possible: tower layer i of every pyramid level then shares a round (and a launch)
             self.rounds = schedule.levels(self.ops, self._reads, self._write, late=True)
+        is_conv_op = lambda op: op[0] == "conv" or (op[0] == "convres" and op[1] not in self.unfused)
+        if chained:
+            # convolutions of consecutive rounds go out together (rtoss_conv_chain: dependent convolutions in one launch)
+            if self.steps is None:
+                self.steps = schedule.chains(self.ops, self.rounds, self._reads, self._write, is_conv_op)
+            for step in self.steps:
+                if step[0] == "chain":
+                    self.launches += self.ctx.rtoss_conv_chain([self._item(self.ops[i]) for i in step[1]], step[2])
+                else:
+                    self._run_op(self.ops[step[1]])
+            return
         for rnd in self.rounds:
             convs = [self.ops[i] for i in rnd if self.ops[i][0] == "conv" or (self.ops[i][0] == "convres" and self.ops[i][1] not in self.unfused)]
             rest = [self.ops[i] for i in rnd if not (self.ops[i][0] == "conv" or (self.ops[i][0] == "convres" and self.ops[i][1] not in self.unfused))]
@@ -212,7 +223,7 @@ class GpuNet:
                     if err.status != rt.ERR_UNSUPPORTED:
                         raise
                     self.unfused.add(i)
-                    self.rounds = None
+                    self.rounds = self.steps = None
             fn(*args[:2], t[tmp], *args[3:], rt.ACT_NONE, self.bias[L["wid"]])
             rt.rtoss_add_act(t[tmp], t[other], t[dst], rt.ACT_NAMES[act])
             self.launches += 1

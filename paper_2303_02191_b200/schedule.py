@@ -40,3 +40,58 @@ def levels(ops, reads, write, late=True):
     for i, lv in enumerate(level):
         rounds[lv].append(i)
     return rounds
+
+
+def chains(ops, rounds, reads, write, is_conv, max_items=20, min_width=2):
+    """Issue order of a program whose dependent convolutions may share launches (rtoss_conv_chain).
+
+    Walks the rounds of `levels` in order and collects the convolutions (is_conv(op)) of consecutive rounds into
+    segments of at most max_items; an operation of another kind ends the segment before it is issued (it may read what
+    the segment writes), and so do a round that would not fit and a round of fewer than min_width convolutions (which
+    is issued on its own).  Returns a list of steps:
+      ('chain', [op indices in issue order], [after masks])  -- bit j of after[i]: item i reads what item j (earlier
+                                                                 in the same segment) writes
+      ('op', op index)                                        -- issued on its own
+    Every buffer region is written once per pass, so reads-after-writes are the only dependencies inside a segment."""
+    steps, seg = [], []
+
+    def flush():
+        if len(seg) == 1:
+            steps.append(("op", seg[0]))
+        elif seg:
+            pos = {i: q for q, i in enumerate(seg)}
+            writer = {}
+            for i in seg:
+                writer.setdefault(write(ops[i]), []).append(i)
+            after = []
+            for i in seg:
+                m = 0
+                for r in reads(ops[i]):
+                    for j in writer.get(r, ()):
+                        if pos[j] < pos[i]:
+                            m |= 1 << pos[j]
+                after.append(m)
+            steps.append(("chain", list(seg), after))
+        del seg[:]
+
+    for rnd in rounds:
+        convs = [i for i in rnd if is_conv(ops[i])]
+        rest = [i for i in rnd if not is_conv(ops[i])]
+        if len(convs) < min_width:
+            # a round of one convolution gains nothing inside a shared launch (the wait inside the kernel costs about a
+            # microsecond more than the boundary between two launches): it ends the segment and goes out alone
+            flush()
+            steps.extend(("op", i) for i in convs + rest)
+            continue
+        if len(seg) + len(convs) > max_items:
+            flush()
+        while len(convs) > max_items:     # a round wider than a launch
+            seg.extend(convs[:max_items])
+            convs = convs[max_items:]
+            flush()
+        seg.extend(convs)
+        if rest:
+            flush()
+            steps.extend(("op", i) for i in rest)
+    flush()
+    return steps

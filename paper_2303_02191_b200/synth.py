@@ -201,6 +201,45 @@ def independent_sets(layers):
     return units
 
 
+def chained_units(layers):
+    """independent_sets with successive tower layers merged: -> (units, afters).  In the RetinaNet-shaped network
+    tower layer i of a level reads tower layer i - 1 of the same tower and level and nothing else, so layers 0 + 1 and
+    2 + 3 of both towers on all levels (twenty convolutions each) can share a launch whose members wait for one another
+    (rtoss_conv_chain).  afters[u] is None for a unit of independent convolutions, else one bit mask per member: bit j
+    set when the member has to wait for member j of the same unit."""
+    import re
+    units = independent_sets(layers)
+    key = []
+    for u in units:
+        m = re.match(r"(cls|box)_tower(\d)\.p\d$", layers[u[0]]["name"])
+        key.append(int(m.group(2)) if m else None)
+    out_units, afters, skip = [], [], set()
+    for ui, u in enumerate(units):
+        if ui in skip:
+            continue
+        nxt = None
+        if key[ui] is not None and key[ui] % 2 == 0:
+            for vi in range(ui + 1, len(units)):
+                if key[vi] == key[ui] + 1:
+                    nxt = vi
+                    break
+        if nxt is None:
+            out_units.append(list(u))
+            afters.append(None)
+            continue
+        skip.add(nxt)
+        merged = list(u) + list(units[nxt])
+        name_at = {layers[i]["name"]: q for q, i in enumerate(merged)}
+        after = []
+        for i in merged:
+            m = re.match(r"(cls|box)_tower(\d)(\.p\d)$", layers[i]["name"])
+            prev = "%s_tower%d%s" % (m.group(1), int(m.group(2)) - 1, m.group(3))
+            after.append(1 << name_at[prev] if prev in name_at else 0)
+        out_units.append(merged)
+        afters.append(after)
+    return out_units, afters
+
+
 def layer_nnz_flops(layer, N, k):
     """2 * (kept multiply-adds) of one call at batch N with k kept taps."""
     Ho, Wo = out_hw(layer["H"], layer["W"], layer["stride"])

@@ -129,7 +129,7 @@ class GpuNet:
         if fuse_residual:
             self.ops = fuse_shortcuts(self.ops)
         self.unfused = set()   # layers whose fused call the library declined: convolution and add run separately
-        self.rounds, self.probed = None, False
+        self.rounds, self.probed, self.steps = None, False, None
         tdt = {"bf16": torch.bfloat16, "f16": torch.float16}[dtype]
         self.t = {n: torch.zeros((N, H, W, C), dtype=tdt, device="cuda") for n, (C, H, W) in self.bufs.items()}
         masks = rt.rtoss_pattern_preset(k, rt.PRESET_CENTRE8 if k == 4 else rt.PRESET_CONN4)
@@ -156,7 +156,7 @@ class GpuNet:
     def _write(self, op):
         return op[{"conv": 3, "convres": 5, "add": 3, "pool5": 2, "up": 2, "copy": 2}[op[0]]]
 
-    def run(self, grouped=True):
+    def run(self, grouped=True, chained=False):
         """One pass.  grouped: operations are issued round by round (schedule.levels: a buffer is ready when every slice
         of it has been written) and the convolutions of a round go out through rtoss_conv_group; else one call per
         operation in program order."""
@@ -169,6 +169,17 @@ class GpuNet:
         if self.rounds is None:
             # as soon as possible: the two 1x1 branches that open a C3 block then share a round (and a launch)
             self.rounds = schedule.levels(self.ops, self._reads, self._write, late=False)
+        is_conv_op = lambda op: op[0] == "conv" or (op[0] == "convres" and op[1] not in self.unfused)
+        if chained:
+            # convolutions of consecutive rounds go out together (rtoss_conv_chain: dependent convolutions in one launch)
+            if self.steps is None:
+                self.steps = schedule.chains(self.ops, self.rounds, self._reads, self._write, is_conv_op)
+            for step in self.steps:
+                if step[0] == "chain":
+                    self.launches += self.ctx.rtoss_conv_chain([self._item(self.ops[i]) for i in step[1]], step[2])
+                else:
+                    self._run_op(self.ops[step[1]])
+            return
         for rnd in self.rounds:
             is_conv = lambda op: op[0] == "conv" or (op[0] == "convres" and op[1] not in self.unfused)
             convs = [self.ops[i] for i in rnd if is_conv(self.ops[i])]
@@ -214,7 +225,7 @@ class GpuNet:
                     if err.status != rt.ERR_UNSUPPORTED:
                         raise
                     self.unfused.add(i)
-                    self.rounds = None
+                    self.rounds = self.steps = None
             fn(self.packed[i], t[src], t[tmp], N, L["H"], L["W"], L["stride"], rt.NHWC, rt.ACT_SILU, self.bias[i])
             rt.rtoss_add_act(t[other], t[tmp], t[dst], rt.ACT_NONE)
             self.launches += 1

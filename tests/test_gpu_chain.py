@@ -24,8 +24,8 @@ def _table(k):
 class Net:
     """A small program of convolutions over named NHWC buffers.  spec: (name, ks, Cout, stride, act, src, residual or None)."""
 
-    def __init__(self, seed, N, C0, H, W, spec, dt="bf16", k=4):
-        self.c, self.N, self.dt, self.k, self.spec = gu.ctx(), N, dt, k, spec
+    def __init__(self, seed, N, C0, H, W, spec, dt="bf16", k=4, path=0):
+        self.c, self.N, self.dt, self.k, self.spec, self.path = gu.ctx(), N, dt, k, spec, path
         self.masks = _table(k)
         self.shape = {"in": (C0, H, W)}
         self.layers = {}
@@ -55,7 +55,7 @@ class Net:
             L = self.layers[name]
             _, Hi, Wi = self.shape[src]
             out.append(self.c.conv_item(L["packed"], self.t[src], self.t[name], self.N, Hi, Wi, stride, rt.NHWC, ACT[act], L["bias"],
-                                        residual=self.t[res] if res else None))
+                                        residual=self.t[res] if res else None, path=self.path))
         return out
 
     def read(self):
@@ -93,7 +93,9 @@ STAGE = [
 
 
 def test_a_stage_of_bottleneck_blocks_is_one_launch():
-    net = Net(81, 2, 96, 40, 56, STAGE)
+    # (RTOSS_PATH_TENSOR keeps the small 3x3 layers in the shared launch; left to itself the library would give each a
+    # launch of its own, cut along the channels: the second run below)
+    net = Net(81, 2, 96, 40, 56, STAGE, path=rt.PATH_TENSOR)
     c = net.c
     items = net.items()
     after = rt.rtoss_chain_deps(items)
@@ -126,6 +128,13 @@ def test_a_stage_of_bottleneck_blocks_is_one_launch():
         again = net.read()
         for name in net.shape:
             assert np.array_equal(again[name].view(np.uint32), got[name].view(np.uint32)), (how, name)
+    # left to choose, the library takes the small 3x3 layers out of the shared launches
+    auto = Net(81, 2, 96, 40, 56, STAGE)
+    auto.poison()
+    assert 1 < c.rtoss_conv_chain(auto.items()) < len(STAGE)
+    torch.cuda.synchronize()
+    auto.check_each_layer(auto.read())
+    auto.close()
     # one call per convolution, in order: the same network (other tile plans, so other summation order)
     net.poison()
     for it in items:
@@ -181,7 +190,7 @@ def test_fp32_chain_and_buffer_reuse():
         ("p", 3, 96, 1, "silu", "in", None),
         ("q", 1, 96, 1, "none", "p", None),
     ]
-    net = Net(83, 1, 96, 18, 22, spec, dt="f32")
+    net = Net(83, 1, 96, 18, 22, spec, dt="f32", path=rt.PATH_TENSOR)
     c = net.c
     Lr = net.layers["q"]
     items = net.items()
@@ -191,7 +200,8 @@ def test_fp32_chain_and_buffer_reuse():
     packed = c.rtoss_pack(wd, 3, net.masks, net.k, c.rtoss_select_patterns(wd, 3, net.masks, net.k), rt.DTYPE_NAMES["f32"])
     wdense = gu.oracle_weights(w, 3, net.masks, net.k, "f32")[1]
     b = synth.bias(83, 7, 96)
-    items.append(c.conv_item(packed, net.t["q"], net.t["in"], 1, 18, 22, 1, rt.NHWC, ACT["relu"], torch.from_numpy(b).cuda()))
+    items.append(c.conv_item(packed, net.t["q"], net.t["in"], 1, 18, 22, 1, rt.NHWC, ACT["relu"], torch.from_numpy(b).cuda(),
+                             path=rt.PATH_TENSOR))
     assert rt.rtoss_chain_deps(items) == [0, 0b01, 0b11]
     net.poison()
     assert c.rtoss_conv_chain(items) == 1
@@ -207,7 +217,7 @@ def test_fp32_chain_and_buffer_reuse():
 
 
 def test_items_the_shared_launch_does_not_take_run_in_order():
-    """A narrow 1x1 layer (positions on M) in the middle: the chain goes out as single launches, same results."""
+    """A narrow 1x1 layer (positions on M) in front: it goes out on its own, the rest as one launch, same results."""
     spec = [
         ("u", 1, 48, 1, "relu", "in", None),      # 48 filters: not a member of shared launches
         ("v", 3, 128, 1, "relu", "u", None),
@@ -215,7 +225,7 @@ def test_items_the_shared_launch_does_not_take_run_in_order():
     ]
     net = Net(84, 2, 64, 20, 20, spec)
     net.poison()
-    assert net.c.rtoss_conv_chain(net.items()) == 3
+    assert net.c.rtoss_conv_chain(net.items()) == 2      # u on its own, then v and w together
     torch.cuda.synchronize()
     net.check_each_layer(net.read())
     with pytest.raises(rt.RtossError):
