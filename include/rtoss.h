@@ -353,9 +353,10 @@ rtoss_status rtoss_conv_group(rtoss_ctx* ctx, const rtoss_conv_item* items, int 
  * bounded like every device-side wait, see rtoss_set_wait_limit, and reports through rtoss_device_status).  Items
  * that do not depend on one another run side by side as in rtoss_conv_group.  Such a launch relies on all its CTAs
  * (at most one per SM) being on the device together: while it runs, no other work may occupy SMs without end, and two
- * such launches must not run concurrently on different streams.  An item that does not qualify, or that has nothing
- * to run beside it and so few tiles and so many input channels that a launch of its own spreads it over more SMs
- * (split along the channels), runs as a launch of its own between the shared ones (the stream orders them); an item
+ * such launches must not run concurrently on different streams.  An item that does not qualify, or that has so few
+ * tiles and so many input channels that a launch of its own spreads it over more SMs (split along the channels)
+ * while the items that could run beside it do not fill the SMs either, runs as a launch of its own between the shared
+ * ones (the stream orders them); an item
  * whose desc.path is RTOSS_PATH_TENSOR rather than RTOSS_PATH_AUTO stays in the shared launch whenever it qualifies.  *launches (nullable) receives the number of kernel
  * launches made.
  * Errors: RTOSS_ERR_INVALID_ARG (null items, n outside 1..32, a bit of after[i] at or above i) and those of the single

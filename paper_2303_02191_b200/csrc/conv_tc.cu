@@ -1716,17 +1716,20 @@ bool rtoss_tc_groupable(const rtoss_packed* p, const rtoss_conv_desc* d, const v
 }
 
 // Would a launch of its own cut this call along K (few tiles, many channel blocks)?  Such a call is faster alone than
-// as a member of a shared launch, which never cuts.
-bool rtoss_tc_prefers_split(const rtoss_ctx* ctx, const rtoss_packed* p, const rtoss_conv_desc* d) {
+// as a member of a shared launch, which never cuts -- unless the other members keep the SMs busy meanwhile.
+// *tiles_out (nullable): the call's tiles of 128 filters.
+bool rtoss_tc_prefers_split(const rtoss_ctx* ctx, const rtoss_packed* p, const rtoss_conv_desc* d, long* tiles_out) {
     const int sms = ctx->sm_count > 0 ? ctx->sm_count : 148;
     const int Ho = (d->H - 1) / d->stride + 1, Wo = (d->W - 1) / d->stride + 1;
     const bool pxm = use_pxm(p), f32 = p->dtype == RTOSS_F32;
     const int w_rows = pxm ? round_up(p->Cout, 16) : kMTile, co_tiles = (p->Cout + kMTile - 1) / kMTile;
     TcPlan plan;
+    if (tiles_out) *tiles_out = 0;
     if (!plan_tc(d->N, Ho, Wo, p->ksize, d->stride, co_tiles, sms, pxm, w_rows, d->residual_dev != nullptr, &plan, 1, f32)) return false;
     const int a_stage = plan.n_sub * plan.sub_rows * kRowBytes * (f32 ? 2 : 1), b_stage = plan.G * w_rows * kRowBytes;
     const int cb_ch = kRowBytes / (f32 ? 4 : 2);
     const long tiles = (long)d->N * ((Ho + plan.TH - 1) / plan.TH) * plan.tiles_x * co_tiles;
+    if (tiles_out) *tiles_out = tiles;
     int ks = 1, cb_per = 0;
     pick_split(p->ksize, pxm, rtoss_wtc_layout_of(p->Cout, p->ksize).copies, tiles, (p->Cin + cb_ch - 1) / cb_ch, plan.N_px,
                plan.NA * a_stage + plan.NB * b_stage, sms, &ks, &cb_per);

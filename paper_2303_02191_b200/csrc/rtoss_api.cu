@@ -606,19 +606,26 @@ rtoss_status rtoss_conv_chain(rtoss_ctx* ctx, const rtoss_conv_item* items, int 
     // only the dependencies on items of the same run have to be carried into the kernel.
     const int m_max = rtoss_tc_max_problems();
     // (an item's level: one more than the highest level it waits for; items of one level run side by side)
-    int level[32], at_level[33] = {};
+    int level[32];
     bool member[32];
     for (int q = 0; q < n; ++q) {
         level[q] = 0;
         for (int j = 0; j < q; ++j)
             if ((after[q] >> j) & 1u) level[q] = level[j] + 1 > level[q] ? level[j] + 1 : level[q];
-        ++at_level[level[q]];
     }
+    long tiles[32], level_tiles[33] = {};
+    bool alone[32];
     for (int q = 0; q < n; ++q) {
         const rtoss_conv_item& it = items[q];
-        member[q] = it.desc.path != RTOSS_PATH_FMA && rtoss_tc_groupable(it.packed, &it.desc, it.x_dev, it.y_dev) &&
-                    !(at_level[level[q]] == 1 && it.desc.path == RTOSS_PATH_AUTO && rtoss_tc_prefers_split(ctx, it.packed, &it.desc));
+        member[q] = it.desc.path != RTOSS_PATH_FMA && rtoss_tc_groupable(it.packed, &it.desc, it.x_dev, it.y_dev);
+        tiles[q] = 0;
+        alone[q] = member[q] && rtoss_tc_prefers_split(ctx, it.packed, &it.desc, &tiles[q]) && it.desc.path == RTOSS_PATH_AUTO;
+        if (member[q]) level_tiles[level[q]] += tiles[q];
     }
+    // (better alone, unless the others of its level keep every SM busy for several tiles: its own few, long tiles then
+    // hide among theirs)
+    for (int q = 0; q < n; ++q)
+        if (alone[q] && level_tiles[level[q]] - tiles[q] < 4L * ctx->sm_count) member[q] = false;
     int count = 0, i = 0;
     while (i < n) {
         int m = 0;

@@ -143,6 +143,6 @@ int rtoss_launch_conv_tc_chain(const rtoss_ctx* ctx, int n, const rtoss_packed* 
                                void* const* ys, const rtoss_conv_desc* const* ds, const uint32_t* after, void* stream);
 int rtoss_tc_max_problems();   // most convolutions one launch carries
 // a launch of its own would cut this call along K (few tiles, many channel blocks); a shared launch never does
-bool rtoss_tc_prefers_split(const rtoss_ctx* ctx, const rtoss_packed* p, const rtoss_conv_desc* d);
+bool rtoss_tc_prefers_split(const rtoss_ctx* ctx, const rtoss_packed* p, const rtoss_conv_desc* d, long* tiles_out);
 
 #endif

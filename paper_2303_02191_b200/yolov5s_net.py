@@ -176,7 +176,9 @@ class GpuNet:
                 self.steps = schedule.chains(self.ops, self.rounds, self._reads, self._write, is_conv_op)
             for step in self.steps:
                 if step[0] == "chain":
-                    self.launches += self.ctx.rtoss_conv_chain([self._item(self.ops[i]) for i in step[1]], step[2])
+                    items = [self._item(self.ops[i]) for i in step[1]]
+                    # (a segment without a dependency in it is a set of independent convolutions, as in the grouped run)
+                    self.launches += self.ctx.rtoss_conv_chain(items, step[2]) if any(step[2]) else self.ctx.rtoss_conv_group(items)
                 else:
                     self._run_op(self.ops[step[1]])
             return

@@ -167,9 +167,9 @@ def test_tower_layers_follow_their_own_level_only():
     bias = [torch.from_numpy(p["b"]).cuda() for p in packs]
     items = []
     for i, (h, w) in enumerate(levels):
-        items.append(c.conv_item(packs[0]["packed"], t_in[i], t_mid[i], N, h, w, 1, rt.NHWC, ACT["relu"], bias[0]))
+        items.append(c.conv_item(packs[0]["packed"], t_in[i], t_mid[i], N, h, w, 1, rt.NHWC, ACT["relu"], bias[0], path=rt.PATH_TENSOR))
     for i, (h, w) in enumerate(levels):
-        items.append(c.conv_item(packs[1]["packed"], t_mid[i], t_out[i], N, h, w, 1, rt.NHWC, ACT["relu"], bias[1]))
+        items.append(c.conv_item(packs[1]["packed"], t_mid[i], t_out[i], N, h, w, 1, rt.NHWC, ACT["relu"], bias[1], path=rt.PATH_TENSOR))
     assert rt.rtoss_chain_deps(items) == [0, 0, 0, 0b001, 0b010, 0b100]
     assert c.rtoss_conv_chain(items) == 1
     torch.cuda.synchronize()
