@@ -431,6 +431,27 @@ typedef struct {
 rtoss_status rtoss_fma_plan3x3(const rtoss_conv_desc* desc, int Cin, int Cout, int k, rtoss_dtype packed_dtype,
                                rtoss_fma_plan* out);
 
+/* The tensor path's tiling of a call, host arithmetic only (nothing is launched, no device is touched): what the
+ * launcher of a single call would choose for a layer of this shape on a device of sm_count SMs (0: 148).  desc gives N,
+ * H, W, stride, layout and whether there is a residual operand (any non-null residual_dev; it is not dereferenced).
+ * eligible = 0 when the tensor path does not take the shape (then the rest is zero).  Lets the CPU tests check the
+ * planner's invariants -- shared memory within an SM's, at most 256 positions and 256 box elements per dimension,
+ * stage sizes multiples of the swizzle atom -- and shows how a layer is cut.  Not part of the paper's method.
+ * RTOSS_ERR_INVALID_ARG for a null pointer or a size below 1. */
+typedef struct {
+    int eligible;
+    int rows_per_tile, cols_per_tile, pitch, positions;      /* output rows and columns of a tile, position pitch, the MMA's N */
+    int staged_rows, sub_tiles;                              /* input rows staged per tile; 4 parity sub-tiles for 3x3 stride 2 */
+    int act_stages, weight_stages, taps_per_weight_stage;    /* ring depths; taps fetched by one bulk copy */
+    int row_bytes, act_stage_bytes, weight_stage_bytes;      /* 128, or 64 for 16-bit layers of at most 32 input channels */
+    int shared_bytes;
+    int positions_on_m;                                      /* narrow 1x1 layers */
+    int split_k;                                             /* CTAs of a cluster sharing a tile's channel blocks (1: none) */
+    int tiles;
+} rtoss_tensor_plan;
+rtoss_status rtoss_tensor_plan_of(const rtoss_conv_desc* desc, int ksize, int Cin, int Cout, rtoss_dtype dtype, int sm_count,
+                                  rtoss_tensor_plan* out);
+
 /* ---- glue between the convolutions of a whole network ---------------------- */
 /* Not part of the paper's method (Table 3 and Fig. 6 time whole models, whose graphs need these between the
  * pruned convolutions).  Element-wise, bandwidth-bound; x and y in the given layout and dtype; y may be a

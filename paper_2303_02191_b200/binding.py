@@ -31,7 +31,7 @@ SYMBOLS = [
     "rtoss_pattern_rank", "rtoss_pattern_table_derive",
     "rtoss_batch_create", "rtoss_batch_select_pack", "rtoss_batch_destroy",
     "rtoss_select_patterns_shared", "rtoss_conv_group", "rtoss_set_wait_limit", "rtoss_inject_lost_copy",
-    "rtoss_fma_plan3x3", "rtoss_conv_chain", "rtoss_chain_deps", "rtoss_chain_deps_spans",
+    "rtoss_fma_plan3x3", "rtoss_conv_chain", "rtoss_chain_deps", "rtoss_chain_deps_spans", "rtoss_tensor_plan_of",
 ]
 
 
@@ -71,6 +71,13 @@ class FmaPlan(ctypes.Structure):
         "grid_x", "grid_y", "staged_rows", "staged_cols", "staging", "vector_bytes", "vectors_per_plane", "shared_bytes")]
 
 
+class TensorPlan(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in (
+        "eligible", "rows_per_tile", "cols_per_tile", "pitch", "positions", "staged_rows", "sub_tiles", "act_stages",
+        "weight_stages", "taps_per_weight_stage", "row_bytes", "act_stage_bytes", "weight_stage_bytes", "shared_bytes",
+        "positions_on_m", "split_k", "tiles")]
+
+
 class ConvItem(ctypes.Structure):
     _fields_ = [("packed", ctypes.c_void_p), ("x_dev", ctypes.c_void_p), ("y_dev", ctypes.c_void_p), ("desc", ConvDesc)]
 
@@ -108,6 +115,7 @@ def _load():
     lib.rtoss_conv_group.argtypes = [vp, ctypes.POINTER(ConvItem), ci, ctypes.POINTER(ci), vp]
     lib.rtoss_conv_chain.argtypes = [vp, ctypes.POINTER(ConvItem), ci, ctypes.POINTER(ctypes.c_uint32), ctypes.POINTER(ci), vp]
     lib.rtoss_chain_deps.argtypes = [ctypes.POINTER(ConvItem), ci, ctypes.POINTER(ctypes.c_uint32)]
+    lib.rtoss_tensor_plan_of.argtypes = [ctypes.POINTER(ConvDesc), ci, ci, ci, ci, ci, ctypes.POINTER(TensorPlan)]
     lib.rtoss_chain_deps_spans.argtypes = [ctypes.POINTER(ctypes.c_uint64), ci, ctypes.POINTER(ctypes.c_uint32)]
     lib.rtoss_set_wait_limit.argtypes = [vp, ctypes.c_longlong]
     lib.rtoss_inject_lost_copy.argtypes = [vp]
@@ -215,6 +223,18 @@ def rtoss_fma_plan3x3(N, H, W, stride, layout, io_dtype, Cin, Cout, k, packed_dt
     out = FmaPlan()
     st = lib.rtoss_fma_plan3x3(ctypes.byref(d), int(Cin), int(Cout), int(k), int(io_dtype if packed_dtype is None else packed_dtype),
                                ctypes.byref(out))
+    if st != OK:
+        raise RtossError(st, status_string(st))
+    return out
+
+
+def rtoss_tensor_plan_of(N, H, W, stride, ksize, Cin, Cout, dtype, sm_count=0, layout=NHWC, residual=False):
+    """The tiling the tensor path would use for a call (host only) -> TensorPlan; raises on an argument error."""
+    d = ConvDesc(int(N), int(H), int(W), int(stride), int(layout), int(dtype), 0, None, 0, 0, 0, None, 0)
+    if residual:
+        d.residual_dev = 1   # (only asked whether there is one)
+    out = TensorPlan()
+    st = lib.rtoss_tensor_plan_of(ctypes.byref(d), int(ksize), int(Cin), int(Cout), int(dtype), int(sm_count), ctypes.byref(out))
     if st != OK:
         raise RtossError(st, status_string(st))
     return out

@@ -117,6 +117,12 @@ struct TcArgs {
     // the partial sums are exchanged through distributed shared memory and every CTA finishes a part of the tile.
     int KS, cb_per;
     int cb_ch, slab_ch;   // channels per staged block (128 bytes) and per instruction (32 bytes): 64 / 16 for 16-bit data, 32 / 8 for fp32
+    // Bytes of a staged row (one padded pixel resp. one filter, one channel block): 128 with the 128-byte swizzle, or 64
+    // with the 64-byte swizzle for 16-bit layers of at most 32 input channels (half of a 128-byte row would be zero fill,
+    // and it is the traffic from L2 to shared memory that bounds such layers).  desc_hi: the matching upper word of the
+    // shared-memory matrix descriptors.
+    int row_bytes;
+    unsigned desc_hi;
     int taps_real;        // 9 or 1; `taps` counts weight tiles per channel block: twice that for fp32 (heads, then remainders)
     int lo_off;           // fp32: byte offset of the remainders inside an activation stage
     // The operand rings this problem runs with: NA activation stages of a_stage bytes from the start of the ring area, NB
@@ -228,13 +234,14 @@ __device__ __forceinline__ void tma_load_3d(unsigned dst, const CUtensorMap* map
 // is 1024-byte aligned: the swizzle is a function of the absolute shared-memory address, the same
 // function TMA applied when it wrote the tile, so a start in the middle of an 8-row group (a tap
 // shift) or 32 bytes into a row (a K step) needs no correction (base-offset field 0).
-__device__ __forceinline__ unsigned long long make_sw128_desc(unsigned addr) {
+// With rows of 64 bytes and the 64-byte swizzle the same holds for groups of 8 rows 512 bytes apart.
+__host__ __device__ __forceinline__ unsigned long long make_sw_desc(unsigned addr, int row_bytes) {
     unsigned long long d = 0;
     d |= (unsigned long long)((addr & 0x3FFFFu) >> 4);        // start address
     d |= (unsigned long long)1 << 16;                          // leading byte offset (unused for swizzled K-major)
-    d |= (unsigned long long)(1024 >> 4) << 32;                // stride byte offset: 8 rows * 128 bytes
+    d |= (unsigned long long)((8 * row_bytes) >> 4) << 32;     // stride byte offset: 8 rows
     d |= (unsigned long long)1 << 46;                          // descriptor version of this architecture
-    d |= (unsigned long long)2 << 61;                          // 128-byte swizzle
+    d |= (unsigned long long)(row_bytes == 64 ? 4 : 2) << 61;  // 64-byte resp. 128-byte swizzle
     return d;
 }
 
@@ -941,10 +948,9 @@ conv_tc_kernel(const __grid_constant__ G g) {
             // a 3x3 layer are unrolled), and K steps (+2 = 32 bytes = 16 channels) or the second half of the
             // positions (+1024 = 128 rows) are additions.
             bool ok = true;
-            const unsigned long long d0 = make_sw128_desc(0);
-            const unsigned desc_hi = (unsigned)(d0 >> 32), desc_lo0 = (unsigned)d0;
+            const unsigned desc_lo0 = (unsigned)make_sw_desc(0, 128);   // (the lower word does not depend on the row size)
             // per problem (recomputed when a tile belongs to another problem than the one before)
-            unsigned tap16[9], wtile16 = 0, idesc = 0, hi_cols = 0, astage16 = 0, bstage16 = 0, sB = 0;
+            unsigned tap16[9], wtile16 = 0, idesc = 0, hi_cols = 0, astage16 = 0, bstage16 = 0, sB = 0, desc_hi = 0, half16 = 0;
             int NA = 1, NB = 1;
             bool pxm = false, two = false, unrolled9 = false;
             int cur_pi = -1, pi = 0;
@@ -954,7 +960,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
             unsigned pacc = 0;                  // phase parity of the accumulator ring
             unsigned peek = 0;                  // what umma_block_peek saw of the stages now current
             int since_res = 1 << 20;            // tiles issued since this CTA's last tile with a residual operand
-            auto mk = [desc_hi](unsigned lo) { return ((unsigned long long)desc_hi << 32) | lo; };
+            auto mk = [&desc_hi](unsigned lo) { return ((unsigned long long)desc_hi << 32) | lo; };
             // all instructions of one tap: the K slabs named by m4 (times two halves of positions with the positions as M)
             auto issue_tap = [&](unsigned d_base, unsigned wl, unsigned xl, unsigned m4, unsigned& acc) {
                 if (pxm) {
@@ -962,7 +968,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
                     for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
                         if (m4 & (1u << k4)) {
                             umma_f16<kF32>(d_base, mk(xl + 2 * k4), mk(wl + 2 * k4), idesc, acc);
-                            if (two) umma_f16<kF32>(d_base + hi_cols, mk(xl + 1024 + 2 * k4), mk(wl + 2 * k4), idesc, acc);
+                            if (two) umma_f16<kF32>(d_base + hi_cols, mk(xl + half16 + 2 * k4), mk(wl + 2 * k4), idesc, acc);
                             acc = 1;
                         }
                     }
@@ -1009,8 +1015,10 @@ conv_tc_kernel(const __grid_constant__ G g) {
                     NA = a.NA;
                     NB = a.NB;
 #pragma unroll
-                    for (int t = 0; t < 9; ++t) tap16[t] = (unsigned)(a.tap_sub[t] * a.sub_bytes + a.tap_shift[t] * kRowBytes) >> 4;
-                    wtile16 = (unsigned)(a.w_rows * kRowBytes) >> 4;
+                    for (int t = 0; t < 9; ++t) tap16[t] = (unsigned)(a.tap_sub[t] * a.sub_bytes + a.tap_shift[t] * a.row_bytes) >> 4;
+                    wtile16 = (unsigned)(a.w_rows * a.row_bytes) >> 4;
+                    desc_hi = a.desc_hi;
+                    half16 = (unsigned)(128 * a.row_bytes) >> 4;   // the second 128 positions of a tile
                     idesc = a.idesc;
                     hi_cols = (unsigned)a.n_cols;
                     pxm = a.pxm != 0;
@@ -1029,8 +1037,8 @@ conv_tc_kernel(const __grid_constant__ G g) {
                 unsigned acc = 0;  // the first instruction of a tile overwrites the accumulator
                 int left = a.Cin - ks * a.cb_per * a.cb_ch;
                 for (int cb = ks * a.cb_per; cb < cb_end && ok; ++cb, left -= a.cb_ch) {
-                    // 32-byte slabs of this block that hold channels (the rest of the 128 bytes is TMA zero fill)
-                    const int nk4 = left >= a.cb_ch ? 4 : (left + a.slab_ch - 1) / a.slab_ch;
+                    // 32-byte slabs of this block that hold channels (the rest of the row is TMA zero fill)
+                    const int nk4 = (min(left, a.cb_ch) + a.slab_ch - 1) / a.slab_ch;
                     const unsigned nkmask = (1u << nk4) - 1u;
                     const int sa = ra.s;
                     if (a.taps == 1) {
@@ -1057,7 +1065,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
 #pragma unroll
                                 for (int k4 = 0; k4 < kKBlock / 16; ++k4) {
                                     if (k4 < nk4) {
-                                        umma_f16<kF32>(d_base + hi_cols, mk(xl0 + 1024 + 2 * k4), mk(wl0 + 2 * k4), idesc, acc2);
+                                        umma_f16<kF32>(d_base + hi_cols, mk(xl0 + half16 + 2 * k4), mk(wl0 + 2 * k4), idesc, acc2);
                                         acc2 = 1;
                                     }
                                 }
@@ -1116,7 +1124,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
                                 // resp. 1) the remainders of tap v - 9.  Heads meet the activations' heads and remainders,
                                 // remainders the heads only.
                                 const int v = t0 + i, t = v >= a.taps_real ? v - a.taps_real : v;
-                                const unsigned off = (unsigned)(a.tap_sub[t] * a.sub_bytes + a.tap_shift[t] * kRowBytes) >> 4;
+                                const unsigned off = (unsigned)(a.tap_sub[t] * a.sub_bytes + a.tap_shift[t] * a.row_bytes) >> 4;
                                 const unsigned m4 = (unsigned)(bits >> (4 * t)) & nkmask;
                                 issue_tap(d_base, wl0 + i * wtile16, xl0 + off, m4, acc);
                                 if (kF32 && v < a.taps_real) issue_tap(d_base, wl0 + i * wtile16, xl0 + off + ((unsigned)a.lo_off >> 4), m4, acc);
@@ -1394,6 +1402,15 @@ inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 // price is one instruction per 128 positions instead of per 256: taken where few instructions are needed anyway.
 bool use_pxm(const rtoss_packed* p) { return p->Cout <= kPxmMaxCout && p->ksize == 1 && p->dtype != RTOSS_F32; }
 
+// Bytes of a staged row: 16-bit layers of at most 32 input channels stage 64-byte rows (64-byte swizzle) instead of
+// 128-byte rows half of which would be zero fill.
+int row_bytes_of(const rtoss_packed* p) { return (p->dtype != RTOSS_F32 && p->Cin <= 32) ? 64 : kRowBytes; }
+// channel blocks (staged rows' worth of channels) of a layer
+int ncb_of(const rtoss_packed* p) {
+    const int cb_ch = row_bytes_of(p) / (p->dtype == RTOSS_F32 ? 4 : 2);
+    return (p->Cin + cb_ch - 1) / cb_ch;
+}
+
 struct TcPlan {
     int TH, TW, Wq, N_px, NA, NB, G, n_sub, sub_rows, rows_staged, tiles_x, smem;
 };
@@ -1409,7 +1426,7 @@ struct TcPlan {
 // The plan picks TH, the column segment TW (images wider than a TMA box are cut into segments), the
 // ring depths, and how many taps share a weight stage.
 bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count, bool pxm, int w_rows, bool resid, TcPlan* out,
-             int n_prob = 1, bool f32 = false, int force_G = 0, int n_tabs = 1) {
+             int n_prob = 1, bool f32 = false, int force_G = 0, int n_tabs = 1, int row_bytes = kRowBytes, int ncb = 2) {
     const int halo = ksize == 3 ? (S == 1 ? 2 : 1) : 0;
     const int n_sub = (ksize == 3 && S == 2) ? 4 : 1;
     const int max_pitch = S == 1 ? 256 : 128;  // TMA box: at most 256 elements traversed per dimension
@@ -1432,14 +1449,18 @@ bool plan_tc(int N, int Ho, int Wo, int ksize, int S, int co_tiles, int sm_count
             const int halves = n_px > 128 ? 2 : 1;
             if (pxm && max_shift + 128 * halves > need_rows) need_rows = max_shift + 128 * halves;
             const int sub_rows = round_up(need_rows, 8);
-            const int a_bytes = n_sub * sub_rows * kRowBytes * (f32 ? 2 : 1);   // (fp32: heads and remainders)
+            const int a_bytes = n_sub * sub_rows * row_bytes * (f32 ? 2 : 1);   // (fp32: heads and remainders)
             for (int G = (ksize == 3 ? 3 : 1); G >= 1; G -= 2) {
                 if (force_G && G != force_G) continue;   // (the problems of one launch share the weight ring: one G for all)
-                const int b_bytes = G * w_rows * kRowBytes;
+                const int b_bytes = G * w_rows * row_bytes;
                 int na = (cap - fixed - 2 * b_bytes) / a_bytes;
                 if (na < 1) continue;
                 if (na > kMaxA) na = kMaxA;
-                if (na > 2 && ksize == 3) na = 2;  // a channel block feeds nine taps: two stages cover the load
+                // A channel block feeds nine taps: with several blocks per tile two stages cover the load.  A layer of
+                // one block per tile (at most 64 channels; 32 with 64-byte rows) has the next TILE's block as its next
+                // stage, and its instructions (18 or 36 of at most 128 cycles) are over before a fetch from L2 returns:
+                // it keeps as many stages as fit.
+                if (na > 2 && ksize == 3 && ncb > 1) na = 2;
                 int nb = (cap - fixed - na * a_bytes) / b_bytes;
                 if (nb > kMaxB) nb = kMaxB;
                 if (nb < 2) continue;
@@ -1504,8 +1525,9 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
     const int w_rows = pxm ? round_up(p->Cout, 16) : kMTile;
     const bool f32 = p->dtype == RTOSS_F32;
     const int esize = f32 ? 4 : 2;
+    const int row_bytes = row_bytes_of(p);
     if (!plan_tc(d->N, Ho, Wo, p->ksize, S, (p->Cout + kMTile - 1) / kMTile, sms, pxm, w_rows, d->residual_dev != nullptr, &plan, n_prob, f32,
-                 force_G, n_tabs))
+                 force_G, n_tabs, row_bytes, (p->Cin + row_bytes / esize - 1) / (row_bytes / esize)))
         return (int)cudaErrorInvalidConfiguration;
 
     TcArgs& a = *out;
@@ -1526,11 +1548,13 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
     a.TW = plan.TW;
     a.taps = taps * (f32 ? 2 : 1);   // weight tiles per channel block: fp32 has the heads, then the remainders
     a.taps_real = taps;
-    a.cb_ch = kRowBytes / esize;
+    a.row_bytes = row_bytes;
+    a.desc_hi = (unsigned)(make_sw_desc(0, row_bytes) >> 32);
+    a.cb_ch = row_bytes / esize;
     a.slab_ch = 32 / esize;
     a.tiles_x = plan.tiles_x;
     a.n_sub = plan.n_sub;
-    a.sub_bytes = plan.sub_rows * kRowBytes;
+    a.sub_bytes = plan.sub_rows * row_bytes;
     if (p->ksize == 3 && S == 1) {
         a.x_add[0] = a.y_add[0] = -1;
         for (int t = 0; t < 9; ++t) a.tap_shift[t] = (t / 3) * plan.Wq + (t % 3);
@@ -1550,18 +1574,18 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
     a.ncb = (p->Cin + a.cb_ch - 1) / a.cb_ch;
     a.tiles_y = (Ho + plan.TH - 1) / plan.TH;
     a.co_tiles = (p->Cout + N_T - 1) / N_T;
-    a.lo_off = f32 ? plan.n_sub * plan.sub_rows * kRowBytes : 0;
-    pp->a_stage_bytes = plan.n_sub * plan.sub_rows * kRowBytes * (f32 ? 2 : 1);
+    a.lo_off = f32 ? plan.n_sub * plan.sub_rows * row_bytes : 0;
+    pp->a_stage_bytes = plan.n_sub * plan.sub_rows * row_bytes * (f32 ? 2 : 1);
     a.w_rows = w_rows;
     // narrow 3x3 layers keep the filters on M and repeat them down the 128 rows of the tile
     const rtoss_wtc_layout lay = rtoss_wtc_layout_of(p->Cout, p->ksize);  // how rtoss_pack laid the weights out
     a.rep_rows = lay.copies > 1 ? lay.rep_rows : 128;
     a.R = lay.copies;
-    pp->b_stage_bytes = plan.G * w_rows * kRowBytes;
+    pp->b_stage_bytes = plan.G * w_rows * row_bytes;
     a.G = plan.G;
     pp->acc_cols = round_up(plan.N_px, 32);  // the epilogue reads 32 columns at a time
-    a.a_tx_bytes = (unsigned)(kKBlock * 2 * plan.Wq * plan.rows_staged);  // per sub-tile
-    a.b_tx_bytes = (unsigned)(kKBlock * 2 * w_rows);
+    a.a_tx_bytes = (unsigned)(row_bytes * plan.Wq * plan.rows_staged);  // per sub-tile
+    a.b_tx_bytes = (unsigned)(row_bytes * w_rows);
     a.act = (int)d->act;
     a.y_c_off = d->y_channel_offset;
     a.y_c_stride = d->y_channel_stride ? d->y_channel_stride : p->Cout;
@@ -1584,7 +1608,7 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
     if (!enc) return (int)cudaErrorNotSupported;
     const CUtensorMapDataType dt = f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : a.is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
     // activations: descriptor cached per (pointer, shape, box)
-    const int key[6] = {d->N, d->H, d->W, p->Cin, plan.rows_staged * 8 + S, plan.Wq * 4 + (int)p->dtype};
+    const int key[6] = {d->N, d->H, d->W, p->Cin, plan.rows_staged * 8 + S, plan.Wq * 4 + (int)p->dtype};   // (row size: a function of Cin and dtype)
     rtoss_tmap_entry* ea = nullptr;
     for (rtoss_tmap_entry& e : ctx->tmap_cache)
         if (e.valid && e.base == x && memcmp(e.dims, key, sizeof(key)) == 0) ea = &e;
@@ -1598,7 +1622,7 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
         cuuint32_t es[4] = {1, (cuuint32_t)S, (cuuint32_t)S, 1};
         ea->valid = 0;
         CUresult r = enc(reinterpret_cast<CUtensorMap*>(ea->map), dt, 4, const_cast<void*>(x), dims, strides, box, es,
-                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return (int)cudaErrorInvalidValue;
         ea->base = x;
@@ -1614,7 +1638,7 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
         cuuint32_t es[3] = {1, 1, 1};
         eb->valid = 0;
         CUresult r = enc(reinterpret_cast<CUtensorMap*>(eb->map), dt, 3, p->wtc, dims, strides, box, es,
-                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return (int)cudaErrorInvalidValue;
         eb->base = p->wtc;
@@ -1707,7 +1731,7 @@ bool rtoss_tc_eligible(const rtoss_packed* p, const rtoss_conv_desc* d, const vo
     TcPlan plan;
     const bool pxm = use_pxm(p);
     return plan_tc(d->N, Ho, Wo, p->ksize, d->stride, (p->Cout + kMTile - 1) / kMTile, 148, pxm, pxm ? round_up(p->Cout, 16) : kMTile,
-                   d->residual_dev != nullptr, &plan, 1, p->dtype == RTOSS_F32);
+                   d->residual_dev != nullptr, &plan, 1, p->dtype == RTOSS_F32, 0, 1, row_bytes_of(p), ncb_of(p));
 }
 
 // May this call be one of several in a launch?  (Tensor path with the filters on M.)
@@ -1725,15 +1749,54 @@ bool rtoss_tc_prefers_split(const rtoss_ctx* ctx, const rtoss_packed* p, const r
     const int w_rows = pxm ? round_up(p->Cout, 16) : kMTile, co_tiles = (p->Cout + kMTile - 1) / kMTile;
     TcPlan plan;
     if (tiles_out) *tiles_out = 0;
-    if (!plan_tc(d->N, Ho, Wo, p->ksize, d->stride, co_tiles, sms, pxm, w_rows, d->residual_dev != nullptr, &plan, 1, f32)) return false;
-    const int a_stage = plan.n_sub * plan.sub_rows * kRowBytes * (f32 ? 2 : 1), b_stage = plan.G * w_rows * kRowBytes;
-    const int cb_ch = kRowBytes / (f32 ? 4 : 2);
+    const int row_bytes = row_bytes_of(p);
+    if (!plan_tc(d->N, Ho, Wo, p->ksize, d->stride, co_tiles, sms, pxm, w_rows, d->residual_dev != nullptr, &plan, 1, f32, 0, 1, row_bytes, ncb_of(p))) return false;
+    const int a_stage = plan.n_sub * plan.sub_rows * row_bytes * (f32 ? 2 : 1), b_stage = plan.G * w_rows * row_bytes;
+    const int cb_ch = row_bytes / (f32 ? 4 : 2);
     const long tiles = (long)d->N * ((Ho + plan.TH - 1) / plan.TH) * plan.tiles_x * co_tiles;
     if (tiles_out) *tiles_out = tiles;
     int ks = 1, cb_per = 0;
     pick_split(p->ksize, pxm, rtoss_wtc_layout_of(p->Cout, p->ksize).copies, tiles, (p->Cin + cb_ch - 1) / cb_ch, plan.N_px,
                plan.NA * a_stage + plan.NB * b_stage, sms, &ks, &cb_per);
     return ks > 1;
+}
+
+extern "C" rtoss_status rtoss_tensor_plan_of(const rtoss_conv_desc* d, int ksize, int Cin, int Cout, rtoss_dtype dtype, int sm_count,
+                                            rtoss_tensor_plan* out) {
+    if (!d || !out || (ksize != 1 && ksize != 3) || Cin < 1 || Cout < 1 || (int)dtype < 0 || (int)dtype > 2 || d->N < 1 || d->H < 1 ||
+        d->W < 1 || (d->stride != 1 && d->stride != 2))
+        return RTOSS_ERR_INVALID_ARG;
+    memset(out, 0, sizeof(*out));
+    rtoss_packed fake;
+    memset(&fake, 0, sizeof(fake));
+    fake.Cin = Cin, fake.Cout = Cout, fake.ksize = ksize, fake.dtype = dtype;
+    const rtoss_packed* p = &fake;
+    if (!rtoss_tc_weights_eligible(p) || d->layout != RTOSS_NHWC) return RTOSS_OK;   // (eligible stays 0)
+    const int sms = sm_count > 0 ? sm_count : 148;
+    const int Ho = (d->H - 1) / d->stride + 1, Wo = (d->W - 1) / d->stride + 1;
+    const bool pxm = use_pxm(p), f32 = dtype == RTOSS_F32;
+    const int w_rows = pxm ? round_up(Cout, 16) : kMTile, co_tiles = (Cout + kMTile - 1) / kMTile;
+    const int row_bytes = row_bytes_of(p);
+    TcPlan plan;
+    const int ncb = (Cin + row_bytes / (f32 ? 4 : 2) - 1) / (row_bytes / (f32 ? 4 : 2));
+    if (!plan_tc(d->N, Ho, Wo, ksize, d->stride, co_tiles, sms, pxm, w_rows, d->residual_dev != nullptr, &plan, 1, f32, 0, 1, row_bytes, ncb))
+        return RTOSS_OK;
+    out->eligible = 1;
+    out->rows_per_tile = plan.TH, out->cols_per_tile = plan.TW, out->pitch = plan.Wq, out->positions = plan.N_px;
+    out->act_stages = plan.NA, out->weight_stages = plan.NB, out->taps_per_weight_stage = plan.G;
+    out->row_bytes = row_bytes;
+    out->act_stage_bytes = plan.n_sub * plan.sub_rows * row_bytes * (f32 ? 2 : 1);
+    out->weight_stage_bytes = plan.G * w_rows * row_bytes;
+    out->staged_rows = plan.rows_staged, out->sub_tiles = plan.n_sub;
+    out->shared_bytes = plan.smem;
+    out->positions_on_m = pxm ? 1 : 0;
+    const long tiles = (long)d->N * ((Ho + plan.TH - 1) / plan.TH) * plan.tiles_x * (pxm ? 1 : co_tiles);
+    out->tiles = (int)(tiles > 0x7FFFFFFF ? 0x7FFFFFFF : tiles);
+    int ks = 1, cb_per = 0;
+    pick_split(ksize, pxm, rtoss_wtc_layout_of(Cout, ksize).copies, tiles, ncb, plan.N_px,
+               plan.NA * out->act_stage_bytes + plan.NB * out->weight_stage_bytes, sms, &ks, &cb_per);
+    out->split_k = ks;
+    return RTOSS_OK;
 }
 
 int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, void* y, const rtoss_conv_desc* d,
@@ -1893,7 +1956,9 @@ int rtoss_launch_conv_tc_chain(const rtoss_ctx* ctx, int n, const rtoss_packed* 
             const int room = cap - fixed - (under ? res_bytes : 0);
             int na = (room - 2 * b_bytes) / a_max;
             if (na > kMaxA) na = kMaxA;
-            if (na > 2 && ps[i0]->ksize == 3) na = 2;
+            bool one_block = true;   // (see plan_tc: layers of one channel block per tile keep more activation stages)
+            for (int q = 0; q < m; ++q) one_block = one_block && ncb_of(ps[set[q]]) == 1;
+            if (na > 2 && ps[i0]->ksize == 3 && !one_block) na = 2;
             if (na < 1) return -1;
             int nb = (room - na * a_max) / b_bytes;
             if (nb > kMaxB) nb = kMaxB;

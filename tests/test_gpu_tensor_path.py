@@ -153,6 +153,9 @@ NARROW = [
     (3, 1, 1, 48, 40, 33, 21, 2, "f16", "silu", True),       # ragged filter count (40 of 48 columns), ragged channels
     (3, 2, 3, 16, 64, 31, 45, 3, "bf16", "silu", True),      # stride 2, odd sizes
     (1, 2, 2, 256, 48, 40, 40, 4, "bf16", "relu", False),    # deep K, strided 1x1
+    (1, 1, 2, 32, 32, 40, 40, 4, "bf16", "silu", True),      # 32 channels: 64-byte rows, positions on M, many tiles
+    (3, 2, 2, 32, 64, 64, 64, 4, "bf16", "silu", True),      # 32 channels, stride 2: four 64-byte-row sub-tiles per block
+    (3, 1, 1, 24, 32, 20, 260, 3, "f16", "relu", True),      # 24 of 32 channels, column segments
 ]
 
 
