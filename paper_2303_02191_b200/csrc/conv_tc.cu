@@ -103,6 +103,9 @@ struct TcArgs {
     int Wq, TH, TW, taps;        // position pitch, output rows and columns per tile, 9 or 1
     int N_px, ncb;               // positions per tile (the MMA's N, multiple of 16), channel blocks
     int tiles_y, tiles_x, co_tiles;
+    // A unit's index is taken apart into (share of the channel blocks, filter tile, column segment, row band, image) by
+    // every role for every tile: the four divisors as multiply-and-shift pairs (see tile_of), set by the host.
+    unsigned div_ks[2], div_co[2], div_tx[2], div_ty[2];
     int n_sub, sub_bytes;        // staged sub-tiles per channel block (4 input phases for 3x3 stride 2) and their size
     int x_add[4], y_add[4];      // TMA start coordinate of sub-tile s: x = x0*S + x_add[s], y = y0*S + y_add[s]
     int tap_sub[9], tap_shift[9];  // which sub-tile tap t reads, and from which start row
@@ -112,6 +115,7 @@ struct TcArgs {
     unsigned idesc;
     int w_rows;           // filter rows per staged weight tile (128; fewer with positions as the M operand)
     int rep_rows, R;      // filters as M, narrow layer: the tile holds R copies of rep_rows filter rows (else 128, 1)
+    int rep_shift;        // log2(rep_rows)
     int pxm, MH, n_cols;  // positions as the M operand: M halves of 128 positions per tile, filters per tile (the MMA's N)
     // Split K: a tile's channel blocks are shared out to the KS CTAs of a thread-block cluster, cb_per blocks each;
     // the partial sums are exchanged through distributed shared memory and every CTA finishes a part of the tile.
@@ -690,6 +694,38 @@ __device__ __forceinline__ int find_problem(const G& g, int unit, int& local, in
     return pi;
 }
 
+// n / d for n < 2^31 by a multiplication: md = {ceil(2^(31 + l) / d), l - 1} with l = ceil(log2 d), or {0, 0} for d = 1
+// (exact: the multiplier's error, below 2^l / d <= 2 parts in 2^(31 + l), cannot carry a quotient of n < 2^31 over).
+__host__ __device__ __forceinline__ void magic_of(int d, unsigned (&md)[2]) {
+    md[0] = md[1] = 0;
+    if (d <= 1) return;
+    int l = 0;
+    while ((1ll << l) < d) ++l;
+    md[0] = (unsigned)((((unsigned long long)1 << (31 + l)) + (unsigned)d - 1) / (unsigned)d);
+    md[1] = (unsigned)(l - 1);
+}
+__device__ __forceinline__ int fdiv(int n, const unsigned (&md)[2]) {
+    return md[0] ? (int)(__umulhi((unsigned)n, md[0]) >> md[1]) : n;
+}
+// A unit of problem a taken apart.
+struct TileIdx {
+    int ks, cot, tx, ty, n;
+};
+__device__ __forceinline__ TileIdx tile_of(const TcArgs& a, int local) {
+    TileIdx t;
+    int rest = fdiv(local, a.div_ks);
+    t.ks = local - rest * a.KS;
+    int q = fdiv(rest, a.div_co);
+    t.cot = rest - q * a.co_tiles;
+    rest = q;
+    q = fdiv(rest, a.div_tx);
+    t.tx = rest - q * a.tiles_x;
+    rest = q;
+    t.n = fdiv(rest, a.div_ty);
+    t.ty = rest - t.n * a.tiles_y;
+    return t;
+}
+
 // A ring of stages with one "full" and one "empty" mbarrier per stage: position s and, per stage, the parity of the
 // phase its next use belongs to (bit i of par = stage i).  The parities are kept per stage because the problems of a
 // launch may run with different ring depths: the stages then do not all have the same number of uses behind them.
@@ -840,12 +876,9 @@ conv_tc_kernel(const __grid_constant__ G g) {
                     }
                     cur_pi = pi;
                 }
-                const int ks = local % a.KS;
-                int rest = local / a.KS / a.co_tiles;
-                const int tx = rest % a.tiles_x;
-                rest /= a.tiles_x;
-                const int ty = rest % a.tiles_y, n = rest / a.tiles_y;
-                const int y0 = ty * a.TH, x0 = tx * a.TW;
+                const TileIdx ti = tile_of(a, local);
+                const int ks = ti.ks, n = ti.n;
+                const int y0 = ti.ty * a.TH, x0 = ti.tx * a.TW;
                 const int cb_end = min(a.ncb, (ks + 1) * a.cb_per);
                 for (int cb = ks * a.cb_per; cb < cb_end; ++cb) {
                     const int sa = ra.s;
@@ -917,7 +950,8 @@ conv_tc_kernel(const __grid_constant__ G g) {
                     cur_pi = pi;
                 }
                 const unsigned sB = sA + a.sB_off;
-                const int ks = local % a.KS, cot = (local / a.KS) % a.co_tiles;
+                const TileIdx ti = tile_of(a, local);
+                const int ks = ti.ks, cot = ti.cot;
                 const int co0 = cot * (a.pxm ? a.n_cols : kMTile);
                 const int cb_end = min(a.ncb, (ks + 1) * a.cb_per);
                 for (int cb = ks * a.cb_per; cb < cb_end && ok; ++cb) {
@@ -1025,10 +1059,11 @@ conv_tc_kernel(const __grid_constant__ G g) {
                     two = a.MH == 2;
                     unrolled9 = !kF32 && a.taps == 9 && a.G == 3;
                 }
-                const int ks = local % a.KS, cb_end = min(a.ncb, (ks + 1) * a.cb_per);
+                const TileIdx ti = tile_of(a, local);
+                const int ks = ti.ks, cb_end = min(a.ncb, (ks + 1) * a.cb_per);
                 // which (tap, slab) pairs of this filter tile hold kept weights: one word per channel block, the next
                 // block's word asked for while this block's instructions go out
-                const unsigned long long* iss = a.issue ? a.issue + (size_t)((local / a.KS) % a.co_tiles) * a.ncb : nullptr;
+                const unsigned long long* iss = a.issue ? a.issue + (size_t)ti.cot * a.ncb : nullptr;
                 unsigned long long bits = iss ? __ldg(iss + ks * a.cb_per) : ~0ull;
                 ok = mbar_wait(bar_accEmpty + 8 * as, pacc ^ 1, g.wait_cycles);  // epilogue has drained this stage
                 if (!ok) break;
@@ -1175,14 +1210,13 @@ conv_tc_kernel(const __grid_constant__ G g) {
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
             const int n_chunks = a.n_cols >> 4, items = a.MH * n_chunks;
             const bool vec_ok = (a.y_c_stride % 8 == 0) && (a.y_c_off % 8 == 0);
-            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++gt) {
-                int rest = tile;
-                const int tx = rest % a.tiles_x;
-                rest /= a.tiles_x;
-                const int ty = rest % a.tiles_y, n = rest / a.tiles_y;
-                const int y0 = ty * a.TH, x0 = tx * a.TW;
-                const int as = gt % g.AS;
-                ok = mbar_wait(bar_accFull + 8 * as, (gt / g.AS) & 1, g.wait_cycles);
+            int as = 0;
+            unsigned pfull = 0;   // accumulator stage of this tile and the parity of its "full" phase
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++gt, pfull ^= (as + 1 == g.AS), as = as + 1 == g.AS ? 0 : as + 1) {
+                const TileIdx ti = tile_of(a, tile);
+                const int n = ti.n;
+                const int y0 = ti.ty * a.TH, x0 = ti.tx * a.TW;
+                ok = mbar_wait(bar_accFull + 8 * as, pfull, g.wait_cycles);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const unsigned d_base = tmem_base + (unsigned)(as * g.acc_stride) + ((unsigned)(quarter * 32) << 16);
@@ -1220,27 +1254,23 @@ conv_tc_kernel(const __grid_constant__ G g) {
             }
             gt = -1;   // (done: the loop below does not run)
         }
-        int pi = 0;
-        for (int tile = blockIdx.x; gt >= 0 && tile < n_tiles && ok; tile += gridDim.x, ++gt) {
+        int pi = 0, as = 0;
+        unsigned pfull = 0;   // accumulator stage of this tile and the parity of its "full" phase
+        for (int tile = blockIdx.x; gt >= 0 && tile < n_tiles && ok; tile += gridDim.x, ++gt, pfull ^= (as + 1 == g.AS), as = as + 1 == g.AS ? 0 : as + 1) {
             int local;
             pi = find_problem<kMulti>(g, tile, local, pi);
             const TcArgs& a = g.prob[pi];
             T* __restrict__ yg = reinterpret_cast<T*>(a.y);
             const uint2* pos_tab = pos_tab_all + a.tab * kMaxPx;
             const unsigned s_tab = s_tab_all + (unsigned)a.tab * kMaxPx * 8;
-            int rest = local / a.KS;   // a unit is (tile proper, share of the channel blocks)
-            const int cot = rest % a.co_tiles;
-            rest /= a.co_tiles;
-            const int tx = rest % a.tiles_x;
-            rest /= a.tiles_x;
-            const int ty = rest % a.tiles_y, n = rest / a.tiles_y;
-            const int y0 = ty * a.TH, x0 = tx * a.TW, co0 = cot * kMTile;
-            const int as = gt % g.AS;
+            const TileIdx ti = tile_of(a, local);   // a unit is (tile proper, share of the channel blocks)
+            const int n = ti.n;
+            const int y0 = ti.ty * a.TH, x0 = ti.tx * a.TW, co0 = ti.cot * kMTile;
             // Everything that does not need the accumulator comes before the wait for it: the bias is a global load
             // (a cold one costs more than a thousand cycles) and would otherwise sit on the path of every tile.
             // TMEM lane = filter.  A narrow layer's filters are repeated down the lanes (R copies): every lane quarter
             // then holds outputs, and the copies share the tile's columns between them.
-            const int row0 = (quarter * 32) % a.rep_rows, copy = (quarter * 32) / a.rep_rows;
+            const int copy = (quarter * 32) >> a.rep_shift, row0 = quarter * 32 - (copy << a.rep_shift);   // (rep_rows is 32, 64 or 128)
             const int co = co0 + row0 + lane;
             const bool co_ok = co < a.Cout;
             const float bv = (a.bias && co_ok) ? __ldg(a.bias + co) : 0.f;
@@ -1253,7 +1283,7 @@ conv_tc_kernel(const __grid_constant__ G g) {
             const T* rb = a.resid ? reinterpret_cast<const T*>(a.resid) + (yb - yg) : nullptr;   // laid out like y
             const bool post = a.resid_post != 0;
             const float bs = (!kF32 && a.act == RTOSS_ACT_SILU && (!rb || post)) ? 0.5f * bv : bv;   // (a residual in front of the activation, or fp32 data: plain bias)
-            ok = mbar_wait(bar_accFull + 8 * as, (gt / g.AS) & 1, g.wait_cycles);
+            ok = mbar_wait(bar_accFull + 8 * as, pfull, g.wait_cycles);
             if (!ok && a.KS == 1) break;   // (split K: the cluster barriers below must still be passed)
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const unsigned d_base = tmem_base + (unsigned)(as * g.acc_stride) + ((unsigned)(quarter * 32) << 16);
@@ -1581,6 +1611,7 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
     const rtoss_wtc_layout lay = rtoss_wtc_layout_of(p->Cout, p->ksize);  // how rtoss_pack laid the weights out
     a.rep_rows = lay.copies > 1 ? lay.rep_rows : 128;
     a.R = lay.copies;
+    a.rep_shift = a.rep_rows == 32 ? 5 : a.rep_rows == 64 ? 6 : 7;
     pp->b_stage_bytes = plan.G * w_rows * row_bytes;
     a.G = plan.G;
     pp->acc_cols = round_up(plan.N_px, 32);  // the epilogue reads 32 columns at a time
@@ -1603,6 +1634,10 @@ int build_problem(const rtoss_ctx* ctx, const rtoss_packed* p, const void* x, vo
     }
     a.KS = 1;
     a.cb_per = a.ncb;
+    magic_of(a.KS, a.div_ks);
+    magic_of(pxm ? 1 : a.co_tiles, a.div_co);   // (positions on M: one filter tile covers the layer)
+    magic_of(a.tiles_x, a.div_tx);
+    magic_of(a.tiles_y, a.div_ty);
 
     PFN_cuTensorMapEncodeTiled_v12000 enc = encode_fn();
     if (!enc) return (int)cudaErrorNotSupported;
@@ -1825,6 +1860,7 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
     g.acc_stride = pp.acc_cols;
     launch_common(ctx, &g);
     pick_split(p->ksize, a.pxm != 0, a.R, (long)d->N * a.tiles_y * a.tiles_x * a.co_tiles, a.ncb, plan.N_px, rings, sms, &a.KS, &a.cb_per);
+    magic_of(a.KS, a.div_ks);
     // at least half an SM's shared memory, so that a second CTA (which would wait for TMEM) never shares the SM
     const size_t smem = (size_t)(plan.smem > 116 * 1024 ? plan.smem : 116 * 1024);
     size_t n_units = (size_t)d->N * a.tiles_y * a.tiles_x * a.co_tiles * a.KS;
@@ -1848,6 +1884,7 @@ int rtoss_launch_conv_tc(const rtoss_ctx* ctx, const rtoss_packed* p, const void
         if (le == cudaSuccess) return 0;
         cudaGetLastError();
         a.KS = 1;
+        magic_of(a.KS, a.div_ks);
         a.cb_per = a.ncb;
         n_units = (size_t)d->N * a.tiles_y * a.tiles_x * a.co_tiles;
         g.unit_end[0] = (int)n_units;
