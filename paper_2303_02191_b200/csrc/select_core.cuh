@@ -52,20 +52,24 @@ __device__ __forceinline__ void pack_one(const float (&w)[9], unsigned m, int64_
                                          V* __restrict__ wtc, int ksize, int Cin, int rows, int rep_rows, int copies) {
     V* out = val + i * k;
     if (k * (int)sizeof(V) == 8) {
-        // the k kept values of a kernel are 8 aligned bytes (four 16-bit or two 32-bit values): gathered in registers
-        // (the j-th set bit of the mask picks the j-th slot) and written with one store
-        V slot[8 / sizeof(V)];
-        unsigned rest = m;
+        // the k kept values of a kernel are 8 aligned bytes (four 16-bit or two 32-bit values): pushed into a 64-bit word
+        // from the top, tap by tap in ascending order, so that after k pushes the first kept value sits in the lowest
+        // bits (a valid mask has exactly k bits); written with one store
+        unsigned long long word = 0;
 #pragma unroll
-        for (int j = 0; j < (int)(8 / sizeof(V)); ++j) {
-            const int t = __ffs(rest) - 1;   // (a valid mask has exactly k bits)
-            rest &= rest - 1;
-            float wt = 0.f;
-#pragma unroll
-            for (int u = 0; u < 9; ++u) wt = (u == t) ? w[u] : wt;
-            slot[j] = narrow_to<V>(wt);
+        for (int t = 0; t < 9; ++t) {
+            if (m & (1u << t)) {
+                const V v = narrow_to<V>(w[t]);
+                unsigned long long bits;
+                if constexpr (sizeof(V) == 4) {
+                    bits = (unsigned long long)__float_as_uint(v);
+                } else {
+                    bits = (unsigned long long)*reinterpret_cast<const unsigned short*>(&v);
+                }
+                word = (word >> (8 * sizeof(V))) | (bits << (64 - 8 * sizeof(V)));
+            }
         }
-        *reinterpret_cast<uint2*>(out) = *reinterpret_cast<const uint2*>(slot);
+        *reinterpret_cast<unsigned long long*>(out) = word;
     } else {
         int j = 0;
 #pragma unroll
